@@ -1,0 +1,241 @@
+"""Pins for the oracle's encoder half: outlier extraction, per-channel Lloyd, the cosine gate
+and auto-select (Algorithm 1), LibFit.
+
+The Lloyd pins are closed forms (uniform source), textbook Lloyd-Max distortions (Gaussian
+source, tests/golden/lloyd_max_gaussian.txt), exact recovery of discrete sources, and the
+paper's printed XFP3 bulk cosines.  LibFit has only sanity properties (parity unpinned).
+"""
+import os
+
+import numpy as np
+import pytest
+
+from conftest import read_golden
+from oracle import xfp_oracle as xo
+from paper_2605_14844_b200 import synth
+
+
+def _f16(a):
+    return np.asarray(a, np.uint16).view(np.float16).astype(np.float64)
+
+
+# ---------------------------------------------------------------- outlier extraction
+
+def test_outlier_mask_equals_brute_force_predicate():
+    W = synth.config1_weights(seed=21, rows=64, cols=512)
+    mask, mu, sg = xo.outlier_mask(W, k=4.0, cap=0.02)
+    Wd = W.astype(np.float64)
+    assert abs(mu - Wd.mean()) < 1e-15 and abs(sg - Wd.std()) < 1e-14   # population std
+    assert np.array_equal(mask.astype(bool), np.abs(Wd - mu) > 4.0 * sg)
+    assert 0 < mask.mean() <= 0.02
+
+
+def test_outlier_cap_keeps_largest_with_index_tiebreak():
+    rng = np.random.default_rng(5)
+    W = rng.standard_normal((32, 256)).astype(np.float32)
+    W[3, 10] = W[1, 7] = 9.0           # an exact tie in |w - mu| is impossible to guarantee after the mean
+    mask, mu, sg = xo.outlier_mask(W, k=1.0, cap=0.02)     # k=1 would take ~32 %; the cap bites
+    keep = int(np.floor(0.02 * W.size))
+    assert mask.sum() == keep
+    key = np.abs(W.astype(np.float64) - mu).reshape(-1)
+    order = np.lexsort((np.arange(key.size), -key))        # by key descending, then flat index ascending
+    assert np.array_equal(np.flatnonzero(mask.reshape(-1)), np.sort(order[:keep]))
+
+
+def test_outlier_top_rate_is_exact():
+    W = synth.gaussian_weights(48, 512, seed=9)
+    for rate in (0.0, 0.003, 0.02):
+        mask, mu, _ = xo.outlier_mask(W, rate=rate)
+        keep = int(np.floor(rate * W.size))
+        assert mask.sum() == keep
+        if keep:
+            key = np.abs(W.astype(np.float64) - mu)
+            assert key[mask.astype(bool)].min() >= key[~mask.astype(bool)].max()
+
+
+def test_robust_sigma_sees_the_bulk():
+    W = synth.config1_weights(seed=2, rows=256, cols=1024)
+    _, _, sg_matrix = xo.outlier_mask(W)
+    mask, _, sg_robust = xo.outlier_mask(W, k=6.0, sigma_mode="robust")
+    assert abs(sg_robust - 0.02) < 0.0005 < sg_matrix - 0.02          # the planted tail inflates the plain sigma
+    assert abs(mask.mean() - 0.003) < 2e-4                            # k=6 on the bulk sigma takes the planted set
+
+
+def test_residual_reconstructs_outliers_to_half_an_ulp():
+    W = synth.config1_weights(seed=4, rows=64, cols=512)
+    mask, mu, _ = xo.outlier_mask(W, k=4.0)
+    m = xo.quantize_v2(W, 4, mask, mu)
+    assert m.nnz == mask.sum()
+    rec = _f16(xo.dequant(m))
+    pos = mask.astype(bool)
+    w = W.astype(np.float64)[pos]
+    # two fp16 roundings (the residual, then the sum): within one fp16 ulp of the original
+    ulp = np.spacing(np.abs(w).astype(np.float16)).astype(np.float64)
+    assert np.all(np.abs(rec[pos] - w) <= ulp)
+    # CSR is well formed: ascending columns in every row, positions = the mask
+    for i in range(m.rows):
+        c = m.ocol[m.rowptr[i]:m.rowptr[i + 1]]
+        assert np.all(np.diff(c) > 0) and np.array_equal(c, np.flatnonzero(mask[i]))
+
+
+# ---------------------------------------------------------------- Lloyd
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_lloyd_uniform_source_closed_form(bits):
+    # uniform on [-1, 1]: the optimal quantiser is the uniform one, D = (2/2^N)^2 / 12, and
+    # cos = sqrt(1 - D/var) with var = 1/3  =>  sqrt(1 - 2^-2N)
+    K = 1 << 16
+    v = (np.arange(K) + 0.5) / K * 2.0 - 1.0
+    cb, idx, _, trace = xo.lloyd_row(v, bits, iters=50, want_trace=True)
+    rec = _f16(cb)[idx]
+    cos = rec @ v / np.linalg.norm(rec) / np.linalg.norm(v)
+    assert abs(cos - np.sqrt(1 - 2.0 ** (-2 * bits))) < 2e-4
+    step = 2.0 / (1 << bits)
+    assert np.allclose(_f16(cb), -1 + step * (np.arange(1 << bits) + 0.5), atol=2e-3)
+    assert abs(trace[-1] - step * step / 12) < 1e-5
+
+
+def test_lloyd_gaussian_source_reaches_lloyd_max(golden_dir):
+    rng = np.random.default_rng(17)
+    v = rng.standard_normal(400000)
+    for n, levels, dist in read_golden(os.path.join(golden_dir, "lloyd_max_gaussian.txt")):
+        n, dist = int(n), float(dist)
+        cb, idx, _, trace = xo.lloyd_row(v, n, iters=400, want_trace=True)
+        assert abs(trace[-1] / v.var() - dist) < 0.03 * dist + 2e-4, (n, trace[-1])
+
+
+def test_lloyd_distortion_never_increases_and_entries_are_cell_means():
+    rng = np.random.default_rng(23)
+    v = rng.standard_normal(4096) * 0.02
+    cb, idx, done, trace = xo.lloyd_row(v, 4, iters=20, want_trace=True)
+    assert np.all(np.diff(trace) <= 1e-18)
+    c = _f16(cb)
+    assert np.all(np.diff(c) >= 0)
+    # every stored index is the nearest stored entry (ties to the lower index)
+    d = np.abs(v[:, None] - c[None, :])
+    assert np.array_equal(idx, d.argmin(axis=1))
+    # run to convergence: each entry equals the mean of the values assigned to it (up to the fp16
+    # rounding of the entries, which also moves a few values across cell borders)
+    cb, idx, done, _ = xo.lloyd_row(v, 3, iters=500, want_trace=True)
+    assert done < 500
+    c = _f16(cb)
+    for j in range(8):
+        sel = v[idx == j]
+        assert sel.size and abs(sel.mean() - c[j]) <= 2e-5        # values have sigma 0.02
+
+
+def test_lloyd_discrete_source_is_exact():
+    rng = np.random.default_rng(29)
+    levels = np.array([-0.75, -0.25, 0.125, 0.5])                     # fp16-exact values
+    v = levels[rng.integers(0, 4, 4096)]
+    for bits in (2, 3):
+        cb, idx, _ = xo.lloyd_row(v, bits, iters=20)
+        assert np.array_equal(_f16(cb)[idx], v)
+
+
+def test_lloyd_first_round_uses_cdf_quantile_init():
+    # with zero rounds the codebook is the initialisation: entry j = sorted[floor((j+0.5) K / 2^N)]
+    rng = np.random.default_rng(31)
+    v = rng.standard_normal(1000)
+    cb, _, done = xo.lloyd_row(v, 3, iters=0)
+    s = np.sort(v)
+    want = s[np.floor((np.arange(8) + 0.5) * 1000 / 8).astype(int)].astype(np.float16)
+    assert done == 0 and np.array_equal(cb.view(np.float16), want)
+
+
+def test_gaussian_rows_reproduce_paper_xfp3_bulk_cosine(golden_dir):
+    """On near-Gaussian layers the paper prints XFP3 bulk cosines of 0.980-0.983; per-channel Lloyd
+    with quantile initialisation on Gaussian rows must land in the same band (5 to 20 rounds)."""
+    printed = [float(r[2]) for r in read_golden(os.path.join(golden_dir, "paper_bulk_cosine.txt"))]
+    W = synth.gaussian_weights(256, 4096, seed=33)
+    none = np.zeros(W.shape, np.uint8)
+    for iters, want in ((5, 0.9808), (20, 0.9825)):
+        m = xo.quantize_v2(W, 3, none, 0.0, iters=iters)
+        med = xo.median(xo.row_cosine(W, xo.dequant(m)))
+        assert abs(med - want) < 0.001
+        assert min(printed) - 0.001 <= med <= max(printed) + 0.001
+
+
+@pytest.mark.parametrize("bits,want", [(2, 0.9393), (4, 0.9946), (5, 0.9980)])
+def test_gaussian_rows_cosine_at_twenty_rounds(bits, want):
+    # sqrt(1 - D) for the textbook distortions is the ceiling; 20 rounds from the quantile start sit just under
+    W = synth.gaussian_weights(128, 4096, seed=35)
+    m = xo.quantize_v2(W, bits, np.zeros(W.shape, np.uint8), 0.0, iters=20)
+    med = xo.median(xo.row_cosine(W, xo.dequant(m)))
+    ceiling = {2: np.sqrt(1 - 0.1175), 4: np.sqrt(1 - 0.009497), 5: np.sqrt(1 - 0.002499)}[bits]
+    assert abs(med - want) < 0.001 and med <= ceiling + 5e-4
+
+
+# ---------------------------------------------------------------- cosine gate and auto-select
+
+def test_row_cosine_and_median():
+    rng = np.random.default_rng(37)
+    W = rng.standard_normal((5, 64)).astype(np.float32)
+    R = (W * np.float32(1.5)).astype(np.float16)
+    R[1] = -R[1]
+    W[4] = 0
+    cosv = xo.row_cosine(W, R.view(np.uint16))
+    Rd = R.astype(np.float64)
+    for i in range(4):
+        want = W[i].astype(np.float64) @ Rd[i] / np.linalg.norm(W[i].astype(np.float64)) / np.linalg.norm(Rd[i])
+        assert abs(cosv[i] - want) < 1e-12
+    assert cosv[1] < -0.99 and cosv[4] == 1.0
+    assert xo.median(np.array([3.0, 1.0, 2.0])) == 2.0 and xo.median(np.array([4.0, 1.0, 2.0, 3.0])) == 2.5
+
+
+def test_auto_select_on_gaussian_rows_brackets_the_paper():
+    W = synth.gaussian_weights(64, 4096, seed=41)
+    picks = {}
+    for tau in (0.93, 0.95, 0.96, 0.98, 0.99):
+        m = xo.auto_select(W, "attention", candidates=(2, 3, 4), tau_strict=tau, k=4.0)
+        picks[tau] = m.bits
+        assert not m.info["fallback"] and m.info["median_cos"] >= tau
+        # the next smaller candidate (if any) failed the floor
+        for n, med in m.info["tried"][:-1]:
+            assert med < tau
+    assert picks == {0.93: 2, 0.95: 3, 0.96: 3, 0.98: 3, 0.99: 4}
+    # the lazy floor applies to routed experts only; the strict one to everything else
+    lazy = xo.auto_select(W, "moe_routed", candidates=(2, 4), tau_strict=0.96, tau_lazy=0.93, mode=xo.MODE_V2)
+    strict = xo.auto_select(W, "shared_expert", candidates=(2, 4), tau_strict=0.96, tau_lazy=0.93, mode=xo.MODE_V2)
+    assert (lazy.bits, strict.bits) == (2, 4) and lazy.info["tau"] == 0.93 and strict.info["tau"] == 0.96
+
+
+def test_auto_select_falls_back_to_largest_candidate():
+    W = synth.gaussian_weights(32, 1024, seed=43)
+    m = xo.auto_select(W, candidates=(2, 3), tau_strict=0.999)
+    assert m.bits == 3 and m.info["fallback"] and m.info["median_cos"] < 0.999
+
+
+def test_outlier_extraction_raises_cosine_on_heavy_tailed_layer():
+    # the effect Table 4 reports for attention layers: bulk-only reconstruction is worse than bulk + outliers
+    W = synth.attention_weights(seed=45, rows=128, cols=2048)
+    mask, mu, _ = xo.outlier_mask(W, k=4.0)
+    none = np.zeros_like(mask)
+    with_out = xo.median(xo.row_cosine(W, xo.dequant(xo.quantize_v2(W, 3, mask, mu))))
+    without = xo.median(xo.row_cosine(W, xo.dequant(xo.quantize_v2(W, 3, none, mu))))
+    assert with_out > without + 0.005
+
+
+# ---------------------------------------------------------------- LibFit (sanity only; parity unpinned)
+
+def test_libfit_sanity():
+    W = synth.gaussian_weights(96, 1024, seed=47)
+    mask, mu, _ = xo.outlier_mask(W, rate=0.001)
+    v2 = xo.quantize_v2(W, 4, mask, mu)
+    va = xo.quantize_v2a(W, 4, mask, mu, lib_size=32)
+    assert va.codebook.shape == (32, 16) and va.gid.max() < 32 and va.idx.max() < 16
+    lib = _f16(va.codebook)
+    assert np.all(np.diff(lib, axis=1) >= 0) and np.abs(lib).max() <= 1.0 + 1e-3
+    assert np.all(_f16(va.gscale) >= 0)
+    Wd = W.astype(np.float64)
+    sse2 = ((_f16(xo.dequant(v2)) - Wd) ** 2).sum()
+    ssea = ((_f16(xo.dequant(va)) - Wd) ** 2).sum()
+    cos2 = xo.median(xo.row_cosine(W, xo.dequant(v2)))
+    cosa = xo.median(xo.row_cosine(W, xo.dequant(va)))
+    assert cosa > 0.985 and abs(cosa - cos2) < 0.006
+    # a constant group decodes exactly
+    Wc = W.copy()
+    Wc[5, 128:256] = np.float32(0.03125)
+    vc = xo.quantize_v2a(Wc, 2, np.zeros(W.shape, np.uint8), 0.0, lib_size=8)
+    assert vc.gscale[5, 1] == 0 and np.all(_f16(xo.dequant(vc))[5, 128:256] == 0.03125)
+    assert sse2 > 0 and ssea > 0
