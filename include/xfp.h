@@ -1,0 +1,126 @@
+/*
+ * xfp.h -- C ABI of the B200 (sm_100a) XFP decode library.
+ *
+ * XFP stores a weight matrix W [rows = output channels][cols = input features K] as
+ *     W  ~=  S + Codebook[Q]                                   (paper Eq. 1, "Decomposition")
+ * Q: dense N-bit indices (N in 2..6, "Sub-Byte Packing"); S: sparse fp16 outlier residual.
+ * Two codebook storage modes ("The XFP Format"):
+ *   V2  : one fp16 codebook of 2^N entries per output channel:  D_ik = codebook_i[q_ik]
+ *   V2a : a per-layer library of L codebooks; every group of 128 consecutive k of one channel
+ *         carries a library id, an fp16 scale and an fp16 mid-point
+ *         ("V2a: Shared Codebook Library"):  D_ik = mid_ig + scale_ig * lib[id_ig][q_ik],  g = k / 128
+ * The hot path is the fused decode kernel y = (D + S) x of "Fused Decode Kernel": depack, codebook
+ * gather, outlier add and multiply-accumulate in one launch, fp32 accumulation.
+ *
+ * Conventions
+ *  - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller and
+ *    16-byte aligned.  fp16 values travel as uint16_t bit patterns.
+ *  - The library allocates no memory, creates no streams and never synchronises; work is queued
+ *    on `stream` (a cudaStream_t passed as void*, NULL = the legacy default stream).
+ *  - The return value (xfp_status) is the only error channel.  Problems the host can see (NULL or
+ *    misaligned pointers, unsupported shapes, small buffers, mode mismatch) are rejected before any
+ *    launch.  Problems in the data are found by xfp_pack on the device and reported through
+ *    err_word; GEMV and dequant trust a packed blob (xfp_pack clamps bad values so that a blob
+ *    packed from bad data is still safe to read).
+ *  - `packed` is opaque, position independent (may be copied with cudaMemcpy) and fully
+ *    determined by the descriptor; keep the descriptor with it.
+ */
+#ifndef XFP_H
+#define XFP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    XFP_OK = 0,
+    XFP_ERR_NULL = 1,             /* a required pointer is NULL                         */
+    XFP_ERR_ALIGN = 2,            /* a pointer is not 16-byte aligned                   */
+    XFP_ERR_SHAPE = 3,            /* rows/cols/bits/group/lib/batch outside the domain  */
+    XFP_ERR_UNSUPPORTED = 4,      /* valid in the format, not built (e.g. cols > 65536) */
+    XFP_ERR_BUFFER_TOO_SMALL = 5, /* packed_bytes / workspace_bytes too small           */
+    XFP_ERR_BAD_DATA = 6,         /* reserved for callers that decode err_word          */
+    XFP_ERR_CUDA = 7              /* a CUDA runtime call failed (launch, copy)          */
+} xfp_status;
+
+/* bits of *err_word written by xfp_pack (0 = the data were clean) */
+#define XFP_BAD_INDEX 1u    /* an index >= 2^bits                                  */
+#define XFP_BAD_GROUP_ID 2u /* a V2a group id >= lib_size                          */
+#define XFP_BAD_ROWPTR 4u   /* rowptr not monotone, rowptr[0] != 0 or rowptr[rows] != nnz */
+#define XFP_BAD_COLUMN 8u   /* an outlier column >= cols                           */
+#define XFP_BAD_ORDER 16u   /* outlier columns of a row not strictly ascending     */
+
+typedef struct {
+    int32_t mode;       /* 0 = V2 (per-channel codebook), 1 = V2a (library + per-group id)          */
+    int32_t rows, cols; /* output channels; input features K, a multiple of group_size, <= 65536    */
+    int32_t bits;       /* N in {2,3,4,5,6}, both modes (the paper's own V2a kernel: {2,4} only)    */
+    int32_t group_size; /* 128                                                                      */
+    int32_t lib_size;   /* V2a: L in 1..256 (paper default 32); V2: 0                               */
+    int32_t col_bits;   /* width of the CSR column indices handed to xfp_pack: 16 or 32             */
+    int64_t nnz;        /* number of outliers, 0 <= nnz < 2^31                                      */
+} xfp_desc;
+
+/* Size of the packed blob and of the GEMV workspace for this descriptor (host call, no GPU work).
+ * The workspace holds split-K partial sums and counters; it must be zero-filled once before its
+ * first use and is left zero-filled in its counter part by every call.  One workspace serves any
+ * batch and either GEMV entry point for this shape, but not two calls that overlap in time. */
+int xfp_packed_size(const xfp_desc* desc, size_t* packed_bytes, size_t* workspace_bytes);
+
+/* Re-tile the unpacked tensors (the last stage of the encoder, "Sub-Byte Packing") into the
+ * device layout read by the decode kernels, validating value ranges on the device.
+ *   idx        [rows][cols] one index per byte
+ *   codebook   V2: [rows][2^bits] fp16;  V2a: [lib_size][2^bits] fp16
+ *   group_id   V2a: [rows][cols/group_size] u8;  V2: NULL
+ *   group_scale, group_mid   V2a: [rows][cols/group_size] fp16;  V2: NULL
+ *   out_rowptr [rows+1] int32, monotone, out_rowptr[rows] == nnz   (may be NULL when nnz == 0)
+ *   out_col    [nnz] uint16 or int32 (desc->col_bits), strictly ascending inside a row
+ *   out_val    [nnz] fp16
+ *   packed     receives packed_bytes (>= xfp_packed_size) bytes
+ *   err_word   optional int32 on the device: OR of XFP_BAD_* bits; the caller zeroes it before the
+ *              call and reads it after its own synchronisation */
+int xfp_pack(const xfp_desc* desc, const uint8_t* idx, const uint16_t* codebook, const uint8_t* group_id,
+             const uint16_t* group_scale, const uint16_t* group_mid, const int32_t* out_rowptr,
+             const void* out_col, const uint16_t* out_val, void* packed, size_t packed_bytes,
+             int32_t* err_word, void* stream);
+
+/* Fused decode GEMV for a V2 blob ("Fused Decode Kernel"):  y[b][i] = sum_k (D_ik + S_ik) x[b][k].
+ *   x  [batch][cols] fp16, batch in 1..16
+ *   y  [batch][rows] fp32, or fp16 (round to nearest even of the fp32 sum) when y_is_fp16 != 0
+ * Products are exact in fp32 and accumulated in fp32; the summation order is fixed, so repeated
+ * calls give identical bits.  workspace/workspace_bytes as returned by xfp_packed_size. */
+int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
+                int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same for a V2a blob ("V2a: Shared Codebook Library"). */
+int xfp_gemv_v2a(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
+                 int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Materialise W^ = fp16(D16 + S) as fp16 [rows][cols] ("Reconstruct" in Algorithm 1; Eq. 1).
+ * D16 is the fp16 value the index decodes to: the codebook entry (V2), or
+ * fp16(fp32(scale * lib + mid)) (V2a, one fp32 rounding then one fp16 rounding).  The sum with an
+ * outlier is rounded once.  Bit-exact and unique. */
+int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* stream);
+
+/* n independent GEMVs of one shape in one launch (the active experts of a routed-MoE layer,
+ * "MoE-native" dispatch): packed[j], x[j] ([cols] fp16, batch 1), y[j] ([rows]) are DEVICE arrays of
+ * n device pointers.  All blobs share `desc` (same mode, shape, bits, lib_size; nnz is the largest
+ * of the group and sizes nothing at run time).  The workspace must hold n * workspace_bytes. */
+int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
+                     void* const* y, int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Convenience for callers whose activations live in host memory: copies x_host (pinned for
+ * asynchrony) to x_dev, runs the GEMV for desc->mode, copies y_dev to y_host, all on `stream`.
+ * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller. */
+int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_host, uint16_t* x_dev,
+                  int32_t batch, void* y_host, void* y_dev, int32_t y_is_fp16, void* workspace,
+                  size_t workspace_bytes, void* stream);
+
+const char* xfp_status_str(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XFP_H */

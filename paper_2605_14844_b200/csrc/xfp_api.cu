@@ -1,0 +1,147 @@
+// extern "C" boundary of libxfp: host-side validation, layout computation, kernel selection.
+#include "../../include/xfp.h"
+#include "xfp_internal.h"
+
+using namespace xfp;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_desc(const xfp_desc* d) {
+    if (!d) return XFP_ERR_NULL;
+    if (d->mode != 0 && d->mode != 1) return XFP_ERR_SHAPE;
+    if (d->rows <= 0 || d->cols <= 0) return XFP_ERR_SHAPE;
+    if (d->bits < 2 || d->bits > 6) return XFP_ERR_SHAPE;
+    if (d->group_size != 128) return d->group_size > 0 ? XFP_ERR_UNSUPPORTED : XFP_ERR_SHAPE;
+    if (d->cols % d->group_size) return XFP_ERR_SHAPE;
+    if (d->cols > 65536) return XFP_ERR_UNSUPPORTED;
+    if (d->mode == 1 && (d->lib_size < 1 || d->lib_size > 256)) return XFP_ERR_SHAPE;
+    if (d->mode == 0 && d->lib_size != 0) return XFP_ERR_SHAPE;
+    if (d->col_bits != 16 && d->col_bits != 32) return XFP_ERR_SHAPE;
+    if (d->nnz < 0 || d->nnz >= (int64_t(1) << 31)) return XFP_ERR_SHAPE;
+    if (d->nnz > (int64_t)d->rows * d->cols) return XFP_ERR_SHAPE;
+    if ((int64_t)d->rows > (int64_t(1) << 24)) return XFP_ERR_UNSUPPORTED;
+    return XFP_OK;
+}
+
+Layout layout_of(const xfp_desc* d) { return make_layout(d->mode, d->rows, d->cols, d->bits, d->lib_size, d->nnz); }
+
+int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* stream) {
+    int st = check_desc(desc);
+    if (st) return st;
+    if (desc->mode != want_mode) return XFP_ERR_SHAPE;
+    if (c.batch < 1 || c.batch > 16) return XFP_ERR_SHAPE;
+    if (c.n == 1 && !c.packed_list) {
+        if (!c.packed || !c.x || !c.y) return XFP_ERR_NULL;
+        if (!aligned16(c.packed) || !aligned16(c.x) || !aligned16(c.y)) return XFP_ERR_ALIGN;
+    } else {
+        if (!c.packed_list || !c.x_list || !c.y_list) return XFP_ERR_NULL;
+    }
+    const Layout l = layout_of(desc);
+    const size_t need = generic_workspace_bytes(l);
+    if (!c.workspace) return XFP_ERR_NULL;
+    if (!aligned16(c.workspace)) return XFP_ERR_ALIGN;
+    if (c.workspace_bytes < need) return XFP_ERR_BUFFER_TOO_SMALL;
+    GemvCall cc = c;
+    cc.workspace_bytes = need;
+    return launch_gemv_generic(l, cc, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int xfp_packed_size(const xfp_desc* desc, size_t* packed_bytes, size_t* workspace_bytes) {
+    int st = check_desc(desc);
+    if (st) return st;
+    const Layout l = layout_of(desc);
+    if (packed_bytes) *packed_bytes = l.total;
+    if (workspace_bytes) *workspace_bytes = generic_workspace_bytes(l);
+    return XFP_OK;
+}
+
+int xfp_pack(const xfp_desc* desc, const uint8_t* idx, const uint16_t* codebook, const uint8_t* group_id,
+             const uint16_t* group_scale, const uint16_t* group_mid, const int32_t* out_rowptr, const void* out_col,
+             const uint16_t* out_val, void* packed, size_t packed_bytes, int32_t* err_word, void* stream) {
+    int st = check_desc(desc);
+    if (st) return st;
+    if (!idx || !codebook || !packed) return XFP_ERR_NULL;
+    if (desc->mode == 1 && (!group_id || !group_scale || !group_mid)) return XFP_ERR_NULL;
+    if (desc->nnz > 0 && (!out_rowptr || !out_col || !out_val)) return XFP_ERR_NULL;
+    if (!aligned16(idx) || !aligned16(codebook) || !aligned16(packed)) return XFP_ERR_ALIGN;
+    if (err_word && (reinterpret_cast<uintptr_t>(err_word) & 3u)) return XFP_ERR_ALIGN;
+    const Layout l = layout_of(desc);
+    if (packed_bytes < l.total) return XFP_ERR_BUFFER_TOO_SMALL;
+    PackInputs in{idx, codebook, group_id, group_scale, group_mid, out_rowptr, out_col, desc->col_bits, out_val};
+    return launch_pack(l, in, packed, err_word, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+}
+
+int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
+                int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream) {
+    GemvCall c{packed, x, y, nullptr, nullptr, nullptr, 1, batch, y_is_fp16, workspace, workspace_bytes};
+    return gemv_common(desc, 0, c, stream);
+}
+
+int xfp_gemv_v2a(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
+                 int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream) {
+    GemvCall c{packed, x, y, nullptr, nullptr, nullptr, 1, batch, y_is_fp16, workspace, workspace_bytes};
+    return gemv_common(desc, 1, c, stream);
+}
+
+int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
+                     void* const* y, int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!desc) return XFP_ERR_NULL;
+    if (n < 1 || n > 65535) return XFP_ERR_SHAPE;
+    if (!packed || !x || !y) return XFP_ERR_NULL;
+    int st = check_desc(desc);
+    if (st) return st;
+    const Layout l = layout_of(desc);
+    const size_t need = generic_workspace_bytes(l);
+    if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
+    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16, workspace, need};
+    return gemv_common(desc, desc->mode, c, stream);
+}
+
+int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* stream) {
+    int st = check_desc(desc);
+    if (st) return st;
+    if (!packed || !W) return XFP_ERR_NULL;
+    if (!aligned16(packed) || !aligned16(W)) return XFP_ERR_ALIGN;
+    return launch_dequant(layout_of(desc), packed, W, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+}
+
+int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_host, uint16_t* x_dev, int32_t batch,
+                  void* y_host, void* y_dev, int32_t y_is_fp16, void* workspace, size_t workspace_bytes,
+                  void* stream) {
+    int st = check_desc(desc);
+    if (st) return st;
+    if (!x_host || !x_dev || !y_host || !y_dev) return XFP_ERR_NULL;
+    if (batch < 1 || batch > 16) return XFP_ERR_SHAPE;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)batch * desc->cols * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return XFP_ERR_CUDA;
+    st = desc->mode ? xfp_gemv_v2a(desc, packed, x_dev, batch, y_dev, y_is_fp16, workspace, workspace_bytes, stream)
+                    : xfp_gemv_v2(desc, packed, x_dev, batch, y_dev, y_is_fp16, workspace, workspace_bytes, stream);
+    if (st) return st;
+    if (cudaMemcpyAsync(y_host, y_dev, (size_t)batch * desc->rows * (y_is_fp16 ? 2 : 4), cudaMemcpyDeviceToHost, s) !=
+        cudaSuccess)
+        return XFP_ERR_CUDA;
+    return XFP_OK;
+}
+
+const char* xfp_status_str(int status) {
+    switch (status) {
+        case XFP_OK: return "ok";
+        case XFP_ERR_NULL: return "null pointer";
+        case XFP_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case XFP_ERR_SHAPE: return "shape or parameter outside the domain";
+        case XFP_ERR_UNSUPPORTED: return "not supported by this build";
+        case XFP_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case XFP_ERR_BAD_DATA: return "bad data";
+        case XFP_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

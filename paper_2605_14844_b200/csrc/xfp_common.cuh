@@ -1,0 +1,69 @@
+// Shared device helpers of the XFP kernels: bit-field extraction from a lane's index stream,
+// cache-hinted loads, fp16 bit casts.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "xfp_layout.h"
+
+namespace xfp {
+
+// Index j (compile-time after unrolling) of a lane's 128*N-bit stream held in w[4*N].
+template <int N>
+__device__ __forceinline__ uint32_t field(const uint32_t* w, int j) {
+    const int bit = j * N;
+    const int wi = bit >> 5;
+    const int off = bit & 31;
+    uint32_t v;
+    if (off + N > 32)
+        v = __funnelshift_r(w[wi], w[wi + 1], off);
+    else
+        v = w[wi] >> off;
+    return v & ((1u << N) - 1u);
+}
+
+// Streaming 16-byte load of packed indices: read-only path, no L1 allocation (touched once).
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float h2f(uint16_t b) { return __half2float(__ushort_as_half(b)); }
+__device__ __forceinline__ uint16_t f2h(float f) { return __half_as_ushort(__float2half_rn(f)); }
+
+// Pointers of one packed blob.
+struct Blob {
+    const uint4* idx;
+    const uint16_t* cb;
+    const uint8_t* gid;
+    const uint32_t* gsm;  // half2 bits: scale | mid << 16
+    const int* rowptr;
+    const uint32_t* oent;
+};
+
+struct Offsets {
+    size_t idx, cb, gid, gsm, rowptr, oent;
+};
+
+__host__ __device__ inline Blob blob_at(const void* packed, const Offsets& o) {
+    const char* b = (const char*)packed;
+    Blob r;
+    r.idx = (const uint4*)(b + o.idx);
+    r.cb = (const uint16_t*)(b + o.cb);
+    r.gid = (const uint8_t*)(b + o.gid);
+    r.gsm = (const uint32_t*)(b + o.gsm);
+    r.rowptr = (const int*)(b + o.rowptr);
+    r.oent = (const uint32_t*)(b + o.oent);
+    return r;
+}
+
+inline Offsets offsets_of(const Layout& l) {
+    return Offsets{l.off_idx, l.off_cb, l.off_gid, l.off_gsm, l.off_rowptr, l.off_oent};
+}
+
+}  // namespace xfp

@@ -1,0 +1,45 @@
+// Launchers shared between the translation units of libxfp.  Every launcher queues work on
+// `stream` and returns the cudaError_t of the launch.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "xfp_common.cuh"
+
+namespace xfp {
+
+struct PackInputs {
+    const uint8_t* idx;
+    const uint16_t* codebook;
+    const uint8_t* gid;
+    const uint16_t* gscale;
+    const uint16_t* gmid;
+    const int32_t* rowptr;
+    const void* ocol;
+    int col_bits;
+    const uint16_t* oval;
+};
+
+cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int* err_word, cudaStream_t s);
+cudaError_t launch_dequant(const Layout& l, const void* packed, uint16_t* W, cudaStream_t s);
+
+// One GEMV problem set: either a single blob (packed/x/y) or n blobs through device pointer lists.
+struct GemvCall {
+    const void* packed;
+    const uint16_t* x;
+    void* y;
+    const void* const* packed_list;
+    const uint16_t* const* x_list;
+    void* const* y_list;
+    int n;          // number of problems (1 for the single form)
+    int batch;      // rows of x (1..16)
+    int y_is_fp16;
+    void* workspace;
+    size_t workspace_bytes;  // per problem
+};
+
+// Split-K factor the generic kernel uses for this shape and batch tile (host-side policy).
+int generic_ksplit(const Layout& l, int batch_tile);
+size_t generic_workspace_bytes(const Layout& l);
+cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t s);
+
+}  // namespace xfp

@@ -1,0 +1,250 @@
+// xfp_pack: unpacked tensors -> device layout (with range validation and clamping);
+// xfp_dequant: device layout -> fp16 matrix W^ = fp16(D16 + S), bit-exact.
+#include "xfp_internal.h"
+
+namespace xfp {
+
+// ------------------------------------------------------------------------------------ pack
+
+// One thread per (row-block, super-chunk, lane): 128 byte-indices of one channel -> N uint4.
+template <int N>
+__global__ void __launch_bounds__(128) pack_idx_kernel(const uint8_t* __restrict__ idx, uint4* __restrict__ out,
+                                                       int rows, int cols, int RB, int SC, int* err_word) {
+    constexpr uint32_t E = 1u << N;
+    const int lane = threadIdx.x & 31;
+    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (unit >= (long long)RB * SC) return;
+    const int rb = (int)(unit / SC), sc = (int)(unit % SC);
+    const int row = rb * kRowsPerBlock + lane;
+    uint32_t w[4 * N + 1];
+#pragma unroll
+    for (int i = 0; i < 4 * N + 1; ++i) w[i] = 0u;
+    bool bad = false;
+    if (row < rows) {
+        const uint4* src = (const uint4*)(idx + (size_t)row * cols + (size_t)sc * kSuper);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint4 t = __ldg(src + i);
+            const uint32_t tw[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+            for (int b = 0; b < 16; ++b) {
+                uint32_t q = (tw[b >> 2] >> ((b & 3) * 8)) & 0xffu;
+                bad |= (q >= E);
+                q &= E - 1u;
+                const int j = i * 16 + b;
+                const int bit = j * N, wi = bit >> 5, off = bit & 31;
+                w[wi] |= q << off;
+                if (off + N > 32) w[wi + 1] |= q >> (32 - off);
+            }
+        }
+    }
+    if (bad && err_word) atomicOr(err_word, 1);
+    uint4* dst = out + ((size_t)unit * N) * 32 + lane;
+#pragma unroll
+    for (int v = 0; v < N; ++v) dst[(size_t)v * 32] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+}
+
+__global__ void pack_codebook_kernel(const uint16_t* __restrict__ cb, uint16_t* __restrict__ out, long long n_src,
+                                     long long n_dst) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n_dst) out[t] = t < n_src ? cb[t] : (uint16_t)0;
+}
+
+__global__ void pack_group_kernel(const uint8_t* __restrict__ gid, const uint16_t* __restrict__ gscale,
+                                  const uint16_t* __restrict__ gmid, uint8_t* __restrict__ out_gid,
+                                  uint32_t* __restrict__ out_gsm, int rows, int RB, int SC, int L, int* err_word) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (long long)RB * SC * 32) return;
+    const int lane = (int)(t & 31);
+    const long long unit = t >> 5;
+    const int rb = (int)(unit / SC), sc = (int)(unit % SC);
+    const int row = rb * kRowsPerBlock + lane;
+    uint32_t id = 0, sm = 0;
+    if (row < rows) {
+        id = gid[(size_t)row * SC + sc];
+        if ((int)id >= L) {
+            if (err_word) atomicOr(err_word, 2);
+            id = (uint32_t)(L - 1);
+        }
+        sm = (uint32_t)gscale[(size_t)row * SC + sc] | ((uint32_t)gmid[(size_t)row * SC + sc] << 16);
+    }
+    out_gid[t] = (uint8_t)id;
+    out_gsm[t] = sm;
+}
+
+__device__ __forceinline__ int clampi(long long v, long long lo, long long hi) {
+    return (int)(v < lo ? lo : (v > hi ? hi : v));
+}
+
+// rowptr -> clamped copy (padding rows empty); checks monotonicity and the end points;
+// each thread also checks that its row's columns ascend strictly.
+__global__ void pack_rowptr_kernel(const int32_t* __restrict__ rowptr, const void* __restrict__ ocol, int col_bits,
+                                   int* __restrict__ out, int rows, int rows_pad, long long nnz, int* err_word) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t > rows_pad) return;
+    if (rowptr == nullptr) {  // nnz == 0
+        out[t] = 0;
+        return;
+    }
+    int bad = 0;
+    long long v = t <= rows ? (long long)rowptr[t] : nnz;
+    if (t == 0 && v != 0) bad |= 4;
+    if (t == rows && v != nnz) bad |= 4;
+    if (v < 0 || v > nnz) bad |= 4;
+    if (t < rows) {
+        long long nx = rowptr[t + 1];
+        if (nx < v) bad |= 4;
+        const int p0 = clampi(v, 0, nnz), p1 = clampi(nx, 0, nnz);
+        long long prev = -1;
+        for (int p = p0; p < p1; ++p) {
+            const long long c = col_bits == 16 ? (long long)((const uint16_t*)ocol)[p] : (long long)((const int32_t*)ocol)[p];
+            if (c <= prev) bad |= 16;
+            prev = c;
+        }
+    }
+    out[t] = clampi(v, 0, nnz);
+    if (bad && err_word) atomicOr(err_word, bad);
+}
+
+__global__ void pack_entries_kernel(const void* __restrict__ ocol, int col_bits, const uint16_t* __restrict__ oval,
+                                    uint32_t* __restrict__ out, long long nnz, int cols, int* err_word) {
+    const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= nnz) return;
+    long long c = col_bits == 16 ? (long long)((const uint16_t*)ocol)[p] : (long long)((const int32_t*)ocol)[p];
+    uint32_t v = oval[p];
+    if (c < 0 || c >= cols) {  // neutralise: column 0, value +0
+        if (err_word) atomicOr(err_word, 8);
+        c = 0;
+        v = 0;
+    }
+    out[p] = (uint32_t)c | (v << 16);
+}
+
+template <int N>
+static void launch_pack_idx(const Layout& l, const uint8_t* idx, uint4* out, int* err, cudaStream_t s) {
+    const long long units = (long long)l.RB * l.SC;
+    const unsigned grid = (unsigned)((units + 3) / 4);
+    pack_idx_kernel<N><<<grid, 128, 0, s>>>(idx, out, l.rows, l.cols, l.RB, l.SC, err);
+}
+
+cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int* err_word, cudaStream_t s) {
+    char* base = (char*)packed;
+    uint4* oidx = (uint4*)(base + l.off_idx);
+    switch (l.bits) {
+        case 2: launch_pack_idx<2>(l, in.idx, oidx, err_word, s); break;
+        case 3: launch_pack_idx<3>(l, in.idx, oidx, err_word, s); break;
+        case 4: launch_pack_idx<4>(l, in.idx, oidx, err_word, s); break;
+        case 5: launch_pack_idx<5>(l, in.idx, oidx, err_word, s); break;
+        default: launch_pack_idx<6>(l, in.idx, oidx, err_word, s); break;
+    }
+    const long long n_src = (long long)(l.mode ? l.L : l.rows) * l.E;
+    const long long n_dst = (long long)(l.mode ? l.L : l.rows_pad) * l.E;
+    pack_codebook_kernel<<<(unsigned)((n_dst + 255) / 256), 256, 0, s>>>(in.codebook, (uint16_t*)(base + l.off_cb), n_src,
+                                                                        n_dst);
+    if (l.mode) {
+        const long long n = (long long)l.RB * l.SC * 32;
+        pack_group_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(in.gid, in.gscale, in.gmid,
+                                                                     (uint8_t*)(base + l.off_gid),
+                                                                     (uint32_t*)(base + l.off_gsm), l.rows, l.RB, l.SC,
+                                                                     l.L, err_word);
+    }
+    pack_rowptr_kernel<<<(unsigned)((l.rows_pad + 1 + 255) / 256), 256, 0, s>>>(
+        l.nnz ? in.rowptr : nullptr, in.ocol, in.col_bits, (int*)(base + l.off_rowptr), l.rows, l.rows_pad, l.nnz,
+        err_word);
+    if (l.nnz)
+        pack_entries_kernel<<<(unsigned)((l.nnz + 255) / 256), 256, 0, s>>>(in.ocol, in.col_bits, in.oval,
+                                                                           (uint32_t*)(base + l.off_oent), l.nnz,
+                                                                           l.cols, err_word);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------ dequant
+
+constexpr int kTileStride = 130;  // halves per tile row: 65 words, so 32 lanes hit 32 banks
+
+// One warp per (row-block, super-chunk): each lane decodes the 128 values of its channel into a
+// shared tile, then the warp writes the tile row by row (256 contiguous bytes per row).
+template <int N, int MODE>
+__global__ void __launch_bounds__(128) dequant_kernel(Blob b, uint16_t* __restrict__ W, int rows, int cols, int RB,
+                                                      int SC) {
+    constexpr int E = 1 << N;
+    __shared__ uint16_t tile[4][32 * kTileStride];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long unit = (long long)blockIdx.x * 4 + warp;
+    if (unit >= (long long)RB * SC) return;
+    const int rb = (int)(unit / SC), sc = (int)(unit % SC);
+    const int row = rb * kRowsPerBlock + lane;
+    uint32_t w[4 * N + 1];
+    const uint4* src = b.idx + ((size_t)unit * N) * 32 + lane;
+#pragma unroll
+    for (int v = 0; v < N; ++v) {
+        const uint4 t = ld_stream(src + (size_t)v * 32);
+        w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
+    }
+    w[4 * N] = 0u;
+    uint16_t* trow = &tile[warp][lane * kTileStride];
+    if (MODE == 0) {
+        const uint16_t* cb = b.cb + (size_t)row * E;  // padding rows exist in the blob
+#pragma unroll
+        for (int j = 0; j < kSuper; ++j) trow[j] = __ldg(cb + field<N>(w, j));
+    } else {
+        const uint32_t id = b.gid[(size_t)unit * 32 + lane];
+        const uint32_t sm = b.gsm[(size_t)unit * 32 + lane];
+        const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
+        const uint16_t* lib = b.cb + (size_t)id * E;
+#pragma unroll
+        for (int j = 0; j < kSuper; ++j) {
+            // scale*lib is exact in fp32; one fp32 rounding for the sum, one fp16 rounding after it
+            const float d = __fmaf_rn(scale, h2f(__ldg(lib + field<N>(w, j))), mid);
+            trow[j] = f2h(d);
+        }
+    }
+    __syncwarp();
+    for (int r = 0; r < 32; ++r) {
+        const int orow = rb * kRowsPerBlock + r;
+        if (orow >= rows) break;
+        const uint32_t* srow = (const uint32_t*)&tile[warp][r * kTileStride];
+        uint32_t* drow = (uint32_t*)(W + (size_t)orow * cols + (size_t)sc * kSuper);
+        drow[lane] = srow[lane];
+        drow[lane + 32] = srow[lane + 32];
+    }
+}
+
+// W^ += S at the outlier positions: one correctly rounded fp16 addition per outlier.
+__global__ void dequant_outlier_kernel(Blob b, uint16_t* __restrict__ W, int rows, int cols) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const int p0 = b.rowptr[row], p1 = b.rowptr[row + 1];
+    for (int p = p0 + lane; p < p1; p += 32) {
+        const uint32_t e = b.oent[p];
+        uint16_t* dst = W + (size_t)row * cols + (e & 0xffffu);
+        const __half s = __hadd(__ushort_as_half(*dst), __ushort_as_half((uint16_t)(e >> 16)));
+        *dst = __half_as_ushort(s);
+    }
+}
+
+template <int N>
+static void launch_dequant_n(const Layout& l, const Blob& b, uint16_t* W, cudaStream_t s) {
+    const long long units = (long long)l.RB * l.SC;
+    const unsigned grid = (unsigned)((units + 3) / 4);
+    if (l.mode == 0)
+        dequant_kernel<N, 0><<<grid, 128, 0, s>>>(b, W, l.rows, l.cols, l.RB, l.SC);
+    else
+        dequant_kernel<N, 1><<<grid, 128, 0, s>>>(b, W, l.rows, l.cols, l.RB, l.SC);
+}
+
+cudaError_t launch_dequant(const Layout& l, const void* packed, uint16_t* W, cudaStream_t s) {
+    const Blob b = blob_at(packed, offsets_of(l));
+    switch (l.bits) {
+        case 2: launch_dequant_n<2>(l, b, W, s); break;
+        case 3: launch_dequant_n<3>(l, b, W, s); break;
+        case 4: launch_dequant_n<4>(l, b, W, s); break;
+        case 5: launch_dequant_n<5>(l, b, W, s); break;
+        default: launch_dequant_n<6>(l, b, W, s); break;
+    }
+    if (l.nnz) dequant_outlier_kernel<<<(unsigned)((l.rows + 7) / 8), 256, 0, s>>>(b, W, l.rows, l.cols);
+    return cudaGetLastError();
+}
+
+}  // namespace xfp

@@ -1,0 +1,88 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares, and
+rejects bad arguments on the host before touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2605_14844_b200 as xfp
+from paper_2605_14844_b200 import binding, build as xbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    xbuild.build()
+    return xfp.load_library()
+
+
+def test_exports_match_header(lib):
+    text = open(os.path.join(ROOT, "include", "xfp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(xfp_[a-z0-9_]+)\s*\(", text))
+    assert declared and declared == set(binding.EXPORTS) | {n for n in declared if hasattr(lib, n)}
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def _desc(**kw):
+    d = dict(mode=0, rows=64, cols=256, bits=4, group_size=128, lib_size=0, col_bits=32, nnz=0)
+    d.update(kw)
+    return xfp.XfpDesc(*[d[n] for n, _ in xfp.XfpDesc._fields_])
+
+
+def test_packed_size_accounting(lib):
+    pb, wb = xfp.xfp_packed_size(_desc(rows=4096, cols=4096, nnz=50000))
+    idx_bytes = 4096 * 4096 // 2
+    # indices at exactly N bits per weight, codebooks, row pointers, 4 bytes per outlier
+    assert idx_bytes + 4096 * 16 * 2 + 4097 * 4 + 50000 * 4 <= pb <= idx_bytes + 4096 * 16 * 2 + 4097 * 4 + 50000 * 4 + 5 * 256
+    for bits in (2, 3, 4, 5, 6):
+        pb, _ = xfp.xfp_packed_size(_desc(rows=32, cols=128, bits=bits))
+        assert pb >= 32 * 128 * bits // 8
+    pa, _ = xfp.xfp_packed_size(_desc(mode=1, lib_size=32, rows=3072, cols=4096, bits=3, nnz=0))
+    assert pa >= 3072 * 4096 * 3 // 8 + 3072 * 32 * 5 + 32 * 8 * 2
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(bits=1), 3), (dict(bits=7), 3), (dict(cols=200), 3), (dict(rows=0), 3), (dict(mode=2), 3),
+    (dict(group_size=64), 4), (dict(cols=131072), 4), (dict(mode=1, lib_size=0), 3), (dict(mode=1, lib_size=300), 3),
+    (dict(mode=0, lib_size=32), 3), (dict(col_bits=8), 3), (dict(nnz=-1), 3),
+])
+def test_bad_descriptors_are_rejected(lib, kw, status):
+    pb, wb = C.c_size_t(), C.c_size_t()
+    d = _desc(**kw)
+    assert lib.xfp_packed_size(C.byref(d), C.byref(pb), C.byref(wb)) == status
+
+
+def test_null_alignment_and_size_checks_need_no_gpu(lib):
+    d = _desc(nnz=5)
+    a = C.c_void_p(0x1000)      # never dereferenced: every call below must fail on the host
+    odd = C.c_void_p(0x1008)
+    n = None
+    assert lib.xfp_pack(C.byref(d), n, a, n, n, n, a, a, a, a, 1 << 30, n, n) == 1
+    assert lib.xfp_pack(C.byref(d), a, a, n, n, n, n, a, a, a, 1 << 30, n, n) == 1        # nnz > 0 needs CSR
+    assert lib.xfp_pack(C.byref(d), odd, a, n, n, n, a, a, a, a, 1 << 30, n, n) == 2
+    assert lib.xfp_pack(C.byref(d), a, a, n, n, n, a, a, a, a, 16, n, n) == 5
+    da = _desc(mode=1, lib_size=32)
+    assert lib.xfp_pack(C.byref(da), a, a, n, a, a, n, n, n, a, 1 << 30, n, n) == 1       # V2a needs group ids
+    assert lib.xfp_gemv_v2(C.byref(d), n, a, 1, a, 0, a, 1 << 30, n) == 1
+    assert lib.xfp_gemv_v2(C.byref(d), a, a, 0, a, 0, a, 1 << 30, n) == 3
+    assert lib.xfp_gemv_v2(C.byref(d), a, a, 17, a, 0, a, 1 << 30, n) == 3
+    assert lib.xfp_gemv_v2(C.byref(d), a, odd, 1, a, 0, a, 1 << 30, n) == 2
+    assert lib.xfp_gemv_v2(C.byref(d), a, a, 1, a, 0, a, 8, n) == 5
+    assert lib.xfp_gemv_v2a(C.byref(d), a, a, 1, a, 0, a, 1 << 30, n) == 3                # V2 blob, V2a entry
+    assert lib.xfp_gemv_v2(C.byref(da), a, a, 1, a, 0, a, 1 << 30, n) == 3
+    assert lib.xfp_dequant(C.byref(d), a, n, n) == 1
+    assert lib.xfp_dequant(C.byref(d), a, odd, n) == 2
+    assert lib.xfp_gemv_grouped(C.byref(d), 0, a, a, a, 0, a, 1 << 30, n) == 3
+    assert lib.xfp_gemv_grouped(C.byref(d), 4, a, a, a, 0, a, 64, n) == 5
+    assert xfp.xfp_status_str(0) == "ok" and "aligned" in xfp.xfp_status_str(2)
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "_HERE", str(tmp_path))
+    with pytest.raises(xfp.XfpError):
+        binding.load_library()

@@ -1,0 +1,232 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI.
+
+xfp_dequant must match the oracle bit for bit.  The fused GEMV must satisfy
+    max_i |y_i - y_ref_i| <= 1e-3 * sum_k |W_ik x_k|
+(the tolerance the benchmark spec states; fp32 accumulation of exact products sits far inside it).
+"""
+import numpy as np
+import pytest
+import torch
+
+from conftest import from_oracle, to_oracle
+from oracle import xfp_oracle as xo
+import paper_2605_14844_b200 as xfp
+from paper_2605_14844_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-3
+
+
+def _x_dev(x16):
+    return torch.from_numpy(x16.view(np.int16)).cuda().view(torch.float16)
+
+
+def _check_gemv(q, pm, x16, y_fp16=False, rows=None):
+    """Run the GEMV and compare against the oracle (all rows, or the sampled `rows`)."""
+    xd = _x_dev(x16)
+    y = pm.gemv(xd, y_fp16=y_fp16)
+    torch.cuda.synchronize()
+    got = y.float().cpu().numpy().astype(np.float64)
+    m = to_oracle(q)
+    if rows is None:
+        ref, absum = xo.gemv(m, x16)
+        sel = slice(None)
+    else:
+        ref = np.zeros((x16.shape[0], q.rows)); absum = np.zeros_like(ref)
+        for r in rows:
+            yr, ar = xo.gemv(m, x16, int(r), int(r) + 1)
+            ref[:, r] = yr[:, r]; absum[:, r] = ar[:, r]
+        sel = np.asarray(rows)
+    err = np.abs(got[:, sel] - ref[:, sel])
+    bound = TOL * absum[:, sel]
+    assert np.all(np.isfinite(got[:, sel]))
+    assert np.all(err <= bound + 1e-30), float((err / (bound + 1e-30)).max())
+    return float((err / (bound + 1e-300)).max()), y
+
+
+def _check_dequant(q, pm):
+    W = pm.dequant()
+    torch.cuda.synchronize()
+    got = W.view(torch.int16).cpu().numpy().view(np.uint16)
+    want = xo.dequant(to_oracle(q))
+    assert np.array_equal(got, want)
+    assert int(pm.err_word.item()) == 0
+
+
+CASES = [(mode, bits) for mode in (0, 1) for bits in (2, 3, 4, 5, 6)]
+
+
+@pytest.mark.parametrize("mode,bits", CASES)
+def test_dequant_bit_exact_small(mode, bits):
+    # 70 rows: three row-blocks with a ragged tail; 384 columns: three super-chunks
+    q = synth.random_quantized(mode, 70, 384, bits, 0.02, seed=500 + 10 * mode + bits)
+    _check_dequant(q, xfp.pack_tensors(q))
+
+
+@pytest.mark.parametrize("mode,bits", CASES)
+@pytest.mark.parametrize("batch", [1, 3, 16])
+def test_gemv_within_bound_small(mode, bits, batch):
+    q = synth.random_quantized(mode, 70, 640, bits, 0.02, seed=600 + 10 * mode + bits)
+    pm = xfp.pack_tensors(q, col_bits=16 if bits % 2 else 32)
+    x16 = synth.activations(batch, q.cols, seed=77 + batch)
+    _check_gemv(q, pm, x16)
+    _check_gemv(q, pm, x16, y_fp16=True)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("rows,cols", [(1, 128), (33, 128), (256, 1536), (96, 12288), (2048, 4096)])
+def test_gemv_shapes_and_split_k(mode, rows, cols):
+    q = synth.random_quantized(mode, rows, cols, 4, 0.01, seed=rows + cols + mode)
+    pm = xfp.pack_tensors(q)
+    for batch in (1, 2):
+        _check_gemv(q, pm, synth.activations(batch, cols, seed=5))
+    _check_dequant(q, pm)
+
+
+@pytest.mark.parametrize("placement,rate", [("uniform", 0.0), ("clustered", 0.02), ("one_row", 0.01)])
+def test_outlier_structures(placement, rate):
+    for mode in (0, 1):
+        q = synth.random_quantized(mode, 128, 1024, 4, rate, seed=31 + mode, placement=placement)
+        pm = xfp.pack_tensors(q, col_bits=16)
+        _check_gemv(q, pm, synth.activations(2, q.cols, seed=6))
+        _check_dequant(q, pm)
+
+
+def test_adversarial_activations():
+    q = synth.random_quantized(0, 64, 1024, 4, 0.01, seed=91)
+    qa = synth.random_quantized(1, 64, 1024, 3, 0.01, seed=92)
+    K = q.cols
+    f16 = lambda a: np.ascontiguousarray(np.asarray(a, np.float32).astype(np.float16)).view(np.uint16).reshape(1, K)
+    hot = np.zeros(K); hot[517] = 3.0
+    alt = np.where(np.arange(K) % 2 == 0, 1.0, -1.0)
+    tiny = np.full(K, 6e-8)            # fp16 subnormals
+    big = np.full(K, 60000.0)          # near the fp16 maximum
+    for x in (np.ones(K), alt, hot, tiny, big, np.zeros(K)):
+        for qq in (q, qa):
+            _check_gemv(qq, xfp.pack_tensors(qq), f16(x))
+
+
+def test_gemv_is_deterministic_and_leaves_workspace_clean():
+    q = synth.random_quantized(0, 256, 4096, 4, 0.01, seed=93)
+    pm = xfp.pack_tensors(q)
+    xd = _x_dev(synth.activations(1, q.cols, seed=8))
+    y1 = pm.gemv(xd).clone()
+    y2 = pm.gemv(xd).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+    tickets = pm.workspace[: ((q.rows + 31) // 32) * 4].view(torch.int32)
+    assert int(tickets.abs().sum().item()) == 0
+
+
+def test_encoder_output_round_trip():
+    """Weights -> oracle encoder (outliers, Lloyd, auto-select) -> xfp_pack -> GPU; both modes."""
+    W = synth.config1_weights(seed=1, rows=192, cols=1024)
+    m = xo.auto_select(W, "attention", candidates=(3, 4), tau_strict=0.96, k=6.0, sigma_mode="robust")
+    q = from_oracle(m)
+    pm = xfp.pack_tensors(q)
+    _check_dequant(q, pm)
+    _check_gemv(q, pm, synth.activations(1, q.cols, seed=2))
+    mask, mu, _ = xo.outlier_mask(W, rate=0.001)
+    ma = xo.quantize_v2a(W, 3, mask, mu, lib_size=32)
+    qa = from_oracle(ma)
+    pa = xfp.pack_tensors(qa)
+    _check_dequant(qa, pa)
+    _check_gemv(qa, pa, synth.activations(1, qa.cols, seed=3))
+
+
+def test_pack_reports_bad_data_and_stays_safe():
+    q = synth.random_quantized(1, 64, 256, 3, 0.02, seed=95)
+    bad = synth.QuantTensors(**{**q.__dict__})
+    bad.idx = q.idx.copy(); bad.idx[3, 7] = 9                # >= 2^3
+    bad.gid = q.gid.copy(); bad.gid[5, 1] = 200              # >= L
+    bad.ocol = q.ocol.copy()
+    if q.rowptr[1] - q.rowptr[0] >= 2:
+        bad.ocol[q.rowptr[0] + 1] = bad.ocol[q.rowptr[0]]    # not strictly ascending
+    bad.ocol[-1] = 70000                                      # >= cols
+    pm = xfp.pack_tensors(bad)
+    torch.cuda.synchronize()
+    err = int(pm.err_word.item())
+    assert err & 1 and err & 2 and err & 8
+    y = pm.gemv(_x_dev(synth.activations(1, q.cols, seed=4)))   # must run without faulting
+    torch.cuda.synchronize()
+    assert torch.isfinite(y).all()
+
+
+def test_grouped_matches_single_calls():
+    n, rows, cols = 8, 160, 1536
+    qs = [synth.random_quantized(1, rows, cols, 3, 0.001, seed=700 + j) for j in range(n)]
+    for q in qs[1:]:
+        q.codebook = qs[0].codebook               # one library per layer, shared by its experts
+    pms = [xfp.pack_tensors(q, col_bits=16) for q in qs]
+    xs = [_x_dev(synth.activations(1, cols, seed=800 + j)) for j in range(n)]
+    ys = torch.zeros((n, rows), dtype=torch.float32, device="cuda")
+    desc = pms[0].desc
+    desc.nnz = max(p.desc.nnz for p in pms)
+    _, wb = xfp.xfp_packed_size(desc)
+    ws = torch.zeros(n * wb, dtype=torch.uint8, device="cuda")
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    xfp.xfp_gemv_grouped(desc, n, ptr([p.packed for p in pms]), ptr(xs), ptr([ys[j] for j in range(n)]), False, ws)
+    torch.cuda.synchronize()
+    for j in range(n):
+        single = pms[j].gemv(xs[j])
+        assert torch.equal(single[0], ys[j])
+        ref, absum = xo.gemv(to_oracle(qs[j]), xs[j].view(torch.int16).cpu().numpy().view(np.uint16))
+        assert np.all(np.abs(ys[j].cpu().numpy() - ref[0]) <= TOL * absum[0])
+
+
+def test_gemv_host_entry():
+    q = synth.random_quantized(0, 96, 512, 5, 0.01, seed=97)
+    pm = xfp.pack_tensors(q)
+    x16 = synth.activations(2, q.cols, seed=9)
+    xh = torch.from_numpy(x16.view(np.int16)).pin_memory()
+    yh = torch.zeros((2, q.rows), dtype=torch.float32).pin_memory()
+    xd = torch.empty_like(xh, device="cuda")
+    yd = torch.empty((2, q.rows), dtype=torch.float32, device="cuda")
+    xfp.xfp_gemv_host(pm.desc, pm.packed, xh, xd, 2, yh, yd, False, pm.workspace)
+    torch.cuda.synchronize()
+    ref, absum = xo.gemv(to_oracle(q), x16)
+    assert np.all(np.abs(yh.numpy() - ref) <= TOL * absum)
+
+
+# ---------------------------------------------------------------- full-size configurations
+
+def _sample_rows(rows, n, seed):
+    rng = np.random.default_rng(seed)
+    return np.unique(np.concatenate([[0, 31, 32, rows - 1], rng.integers(0, rows, n)]))
+
+
+def test_config1_full_size_encoder_to_gpu():
+    """4096 x 4096, V2 N=4, 0.3 % planted outliers, robust 6-sigma extraction: the whole chain."""
+    W = synth.config1_weights(seed=1)
+    mask, mu, _ = xo.outlier_mask(W, k=6.0, sigma_mode="robust")
+    m = xo.quantize_v2(W, 4, mask, mu)
+    q = from_oracle(m)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    _check_dequant(q, pm)
+    x16 = synth.activations(1, 4096, seed=2)
+    worst, y = _check_gemv(q, pm, x16)
+    y16 = pm.gemv(_x_dev(x16), y_fp16=True)
+    torch.cuda.synchronize()
+    assert torch.equal(y16, y.half())
+    assert worst < 0.05           # fp32 accumulation sits far inside the 1e-3 bound
+
+
+@pytest.mark.parametrize("mode,rows,cols,bits,rate", [
+    (0, 4096, 4096, 5, 0.01),      # attention block member at 5 bits
+    (1, 3072, 4096, 3, 0.001),     # MoE gate_up expert
+    (1, 4096, 1536, 3, 0.001),     # MoE down expert
+    (0, 8192, 8192, 4, 0.003),     # sweep shape
+    (0, 12288, 4096, 6, 0.02),     # decoder MLP up, widest codebook, highest outlier rate
+    (1, 4096, 12288, 2, 0.005),    # decoder MLP down, K = 12288
+])
+def test_full_size_sampled_rows(mode, rows, cols, bits, rate):
+    q = synth.random_quantized(mode, rows, cols, bits, rate, seed=rows + bits)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    sample = _sample_rows(rows, 200, seed=bits)
+    _check_gemv(q, pm, synth.activations(1, cols, seed=3), rows=sample)
+    # dequant: the sampled rows, bit for bit
+    W = pm.dequant()
+    torch.cuda.synchronize()
+    got = W[torch.from_numpy(sample).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, xo.dequant(to_oracle(q))[sample])
