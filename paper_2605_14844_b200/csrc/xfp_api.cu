@@ -39,13 +39,16 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
         if (!c.packed_list || !c.x_list || !c.y_list) return XFP_ERR_NULL;
     }
     const Layout l = layout_of(desc);
-    const size_t need = generic_workspace_bytes(l);
+    const size_t need = workspace_bytes_for(l);
     if (!c.workspace) return XFP_ERR_NULL;
     if (!aligned16(c.workspace)) return XFP_ERR_ALIGN;
     if (c.workspace_bytes < need) return XFP_ERR_BUFFER_TOO_SMALL;
     GemvCall cc = c;
     cc.workspace_bytes = need;
-    return launch_gemv_generic(l, cc, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+    const cudaError_t e = pair_supported(l, c.batch, c.n) && !c.packed_list
+                              ? launch_gemv_pair(l, cc, (cudaStream_t)stream)
+                              : launch_gemv_generic(l, cc, (cudaStream_t)stream);
+    return e == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 
 }  // namespace
@@ -57,7 +60,7 @@ int xfp_packed_size(const xfp_desc* desc, size_t* packed_bytes, size_t* workspac
     if (st) return st;
     const Layout l = layout_of(desc);
     if (packed_bytes) *packed_bytes = l.total;
-    if (workspace_bytes) *workspace_bytes = generic_workspace_bytes(l);
+    if (workspace_bytes) *workspace_bytes = workspace_bytes_for(l);
     return XFP_OK;
 }
 
@@ -97,7 +100,7 @@ int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed,
     int st = check_desc(desc);
     if (st) return st;
     const Layout l = layout_of(desc);
-    const size_t need = generic_workspace_bytes(l);
+    const size_t need = workspace_bytes_for(l);
     if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
     GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16, workspace, need};
     return gemv_common(desc, desc->mode, c, stream);
@@ -129,6 +132,9 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
         return XFP_ERR_CUDA;
     return XFP_OK;
 }
+
+void xfp_debug_set_ksplit(int ks) { pair_set_ksplit_override(ks); }
+void xfp_debug_set_prefetch(int d) { pair_set_prefetch(d); }
 
 const char* xfp_status_str(int status) {
     switch (status) {

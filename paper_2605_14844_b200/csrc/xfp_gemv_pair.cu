@@ -1,0 +1,501 @@
+// Fast fused decode GEMV for V2 blobs at batch <= 2:  y = (D + S) x.
+//
+// Mapping.  A CTA owns a block of 32*RPL output channels (RPL = rows per lane: 2 for N <= 4,
+// 1 for N = 5) and all of K, or a slice of K for the blocks of the last scheduling round.  Each
+// lane of a dense warp owns RPL channels (lane, lane+32 of the block) and the warps of the CTA
+// share K in super-chunks of 128 weights.  The channels' codebooks are expanded once per CTA into
+// PAIR tables in shared memory: entry t = (cb[t & (E-1)], cb[t >> N]) as a half2, so one 32-bit
+// shared-memory load decodes two weights ("codebook gather from shared memory", step 2 of the
+// fused kernel).  The tables are laid out so that lane l only ever touches bank l: byte address
+//     t * (128 * RPL) + channel_half * 128 + lane * 4
+// hence any index pattern is bank-conflict free.
+//
+// Multiply-accumulate (step 4).  The looked-up half2 of a lane's channels are exactly the A
+// fragment of mma.sync.m16n8k16 (f16 x f16 -> f32): fragment rows g and g+8 of lane (g, t) are that
+// lane's two channels (the second is zero when RPL = 1), and its k slots are four consecutive k.
+// The B fragment carries x on the "diagonal" lanes only (column n = t gets the k slots of
+// lane-group t), so D[g][t] accumulates the dot product of lane (g,t)'s own channel: every lane
+// keeps its own rows although the fragment nominally shares a row between four lanes.  Products
+// of two fp16 numbers are exact in fp32 and the accumulation is fp32.  Columns 4..7 carry a second
+// batch row.  (The scalar route, one mixed-precision FMA per weight, needs the halves unpacked
+// first and measured ~8 issue slots per pair against ~3 here; that is why the dot product runs on
+// the tensor pipe even at batch 1.)
+//
+// Outliers (step 3) are summed by one extra warp per CTA, concurrently with the dense warps: the
+// block's CSR entries are contiguous, so the warp reads them coalesced, gathers x from the staged
+// copy in shared memory, writes the products to shared memory, and each lane then adds up the
+// segments of its own rows in CSR order (deterministic).
+//
+// Schedule.  Blocks that fill whole rounds of CTA slots run over all of K; the blocks of the last,
+// partial round are cut along K so that they occupy the idle slots, and their partial sums are
+// combined by the last CTA of a block in fixed order (no waiting, no atomics on data).
+//
+// Launch overlap.  Weights do not depend on earlier kernels, so every CTA first issues its index,
+// codebook and row-pointer loads and fills its pair tables, and only then executes
+// griddepcontrol.wait (programmatic dependent launch) before it touches x, y or the workspace.
+// Back-to-back calls on one stream therefore overlap the next call's weight streaming with the
+// current call's tail.
+#include "xfp_internal.h"
+
+namespace xfp {
+
+constexpr int kOutBatch = 512;  // outlier entries fetched and staged per round
+
+struct PairArgs {
+    Offsets off;
+    const void* packed;
+    const uint16_t* x;
+    void* y;
+    float* partial;  // [KS][NB][rows_ws]
+    int* tickets;    // [blocks]
+    int rows, cols, RB, SC, rows_ws;
+    int nb, y_is_fp16;
+    // schedule: work items [0, n_full) are whole blocks; the remaining blocks are cut into kst
+    // K-slices of sc_per_split super-chunks each
+    int n_full, kst, sc_per_split;
+    int pf_dist;  // L2 prefetch distance in warp iterations (0 = off)
+};
+
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Byte offset of the table entry of pair p (compile time) of a 128-weight stream w[4N]:
+// t * 128 * RPL merged with `base` (= channel_half * 128 + lane * 4, below the t field).
+template <int N, int RPL>
+__device__ __forceinline__ uint32_t pair_addr(const uint32_t* w, int p, uint32_t base) {
+    constexpr int SH = RPL == 2 ? 8 : 7;  // log2 of the entry stride
+    if (N == 4 && RPL == 2) {
+        // pair p is byte (p & 3) of word p >> 2: one PRMT builds [base.b0, byte, 0, 0]
+        return __byte_perm(w[p >> 2], base, 0x5504u | ((uint32_t)(p & 3) << 4));
+    } else {
+        constexpr uint32_t mask = ((1u << (2 * N)) - 1u) << SH;
+        const int bit = p * 2 * N, wi = bit >> 5, off = bit & 31;
+        uint32_t v;
+        if (off + 2 * N > 32)
+            v = __funnelshift_r(w[wi], w[wi + 1], off) << SH;
+        else if (off >= SH)
+            v = w[wi] >> (off - SH);
+        else
+            v = w[wi] << (SH - off);
+        return (v & mask) | base;
+    }
+}
+
+template <int N, int NB, int RPL, int W>
+__global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
+    constexpr int E = 1 << N;
+    constexpr int T = E * E;                   // pair-table entries per channel
+    constexpr int ROWS = 32 * RPL;             // channels per CTA
+    constexpr int kStride = 128 * RPL;         // bytes between consecutive entries
+    constexpr int kTabBytes = T * kStride;
+    constexpr int kDense = W * 32;
+    extern __shared__ __align__(16) unsigned char smem[];
+    // [tables | x fp16 [NB][K] | red[W][NB][ROWS] | osum[NB][ROWS] | rps[ROWS + 4] | sprod[NB][kOutBatch]]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.launch_dependents;");
+    int blk, ks, KS, spp;
+    if ((int)blockIdx.x < a.n_full) {
+        blk = blockIdx.x; ks = 0; KS = 1; spp = a.SC;
+    } else {
+        const int t = blockIdx.x - a.n_full;
+        blk = a.n_full + t / a.kst; ks = t % a.kst; KS = a.kst; spp = a.sc_per_split;
+    }
+    const Blob b = blob_at(a.packed, a.off);
+    const int sc0 = ks * spp;
+    const int nsc = max(0, min(a.SC, sc0 + spp) - sc0);
+    const int K = a.SC * kSuper;
+
+    unsigned char* tab = smem;
+    uint16_t* xs = (uint16_t*)(smem + kTabBytes);               // [NB][K]
+    float* red = (float*)(xs + (size_t)NB * K);                 // [W][NB][ROWS]
+    float* osum = red + W * NB * ROWS;                          // [NB][ROWS]
+    int* rps = (int*)(osum + NB * ROWS);                        // [ROWS + 1] row pointers of the block
+    float* sprod = (float*)(rps + ROWS + 4);                    // [NB][kOutBatch]
+
+    // the 32-row blocks of this CTA (the second is clamped when RB is odd; its results are dropped)
+    const int blk0 = RPL * blk;
+    const int blk1 = min(RPL * blk + (RPL - 1), a.RB - 1);
+
+    if (warp == W) {
+        // ------------------------------------------------ outlier warp: CSR entries of this CTA's rows
+        const int row0 = blk * ROWS;
+        {
+            const int last = a.RB * kRowsPerBlock;               // rowptr has rows_pad + 1 entries
+#pragma unroll
+            for (int h = 0; h < RPL; ++h) rps[32 * h + lane] = __ldg(b.rowptr + min(row0 + 32 * h + lane, last));
+            if (lane == 0) rps[ROWS] = __ldg(b.rowptr + min(row0 + ROWS, last));
+        }
+        __syncwarp();
+        // this CTA's share of the block's entries (an even cut when K is split)
+        const int e_lo = rps[0], e_hi = rps[ROWS];
+        const int e0 = e_lo + (int)(((long long)(e_hi - e_lo) * ks) / KS);
+        const int e1 = e_lo + (int)(((long long)(e_hi - e_lo) * (ks + 1)) / KS);
+        // Entries are fetched kOutBatch = 512 at a time (16 per lane, all loads of a batch in flight
+        // together); the next batch travels while the current one is processed, and the first batch
+        // travels while the dense warps fill the tables.
+        uint32_t ea[16], eb[16];
+        auto fetch = [&](uint32_t (&d)[16], int c) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) d[j] = (c + j * 32 + lane < e1) ? __ldg(b.oent + c + j * 32 + lane) : 0u;
+        };
+        float acc[NB][RPL];
+#pragma unroll
+        for (int bb = 0; bb < NB; ++bb)
+#pragma unroll
+            for (int h = 0; h < RPL; ++h) acc[bb][h] = 0.f;
+        auto consume = [&](const uint32_t (&d)[16], int c) {
+            const int n = min(kOutBatch, e1 - c);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float v = h2f((uint16_t)(d[j] >> 16));     // entries past e1 are zero
+                const uint32_t col = d[j] & 0xffffu;
+#pragma unroll
+                for (int bb = 0; bb < NB; ++bb) sprod[bb * kOutBatch + j * 32 + lane] = v * h2f(xs[(size_t)bb * K + col]);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int h = 0; h < RPL; ++h) {
+                const int r = lane + 32 * h;
+                const int s0 = max(rps[r], c), s1 = min(rps[r + 1], c + n);
+                for (int p = s0; p < s1; ++p) {
+#pragma unroll
+                    for (int bb = 0; bb < NB; ++bb) acc[bb][h] += sprod[bb * kOutBatch + (p - c)];
+                }
+            }
+            __syncwarp();
+        };
+        if (e0 < e1) fetch(ea, e0);
+        asm volatile("bar.sync 1, %0;" ::"n"(kDense + 32) : "memory");   // x staged by the dense warps
+        for (int c = e0; c < e1; c += 2 * kOutBatch) {
+            if (c + kOutBatch < e1) fetch(eb, c + kOutBatch);
+            consume(ea, c);
+            if (c + kOutBatch < e1) {
+                if (c + 2 * kOutBatch < e1) fetch(ea, c + 2 * kOutBatch);
+                consume(eb, c + kOutBatch);
+            }
+        }
+#pragma unroll
+        for (int bb = 0; bb < NB; ++bb)
+#pragma unroll
+            for (int h = 0; h < RPL; ++h) osum[bb * ROWS + 32 * h + lane] = acc[bb][h];
+        __syncthreads();  // partial sums ready
+    } else {
+        // ------------------------------------------------ dense warps
+        // (0) start streaming this warp's first super-chunk before anything else
+        uint32_t w0[4 * N + 1], w1[RPL == 2 ? 4 * N + 1 : 1];
+        w0[4 * N] = 0u;
+        if (RPL == 2) w1[4 * N] = 0u;
+        const uint4* i0 = b.idx + ((size_t)(blk0 * a.SC + sc0) * N) * 32 + lane;
+        const uint4* i1 = b.idx + ((size_t)(blk1 * a.SC + sc0) * N) * 32 + lane;
+        auto prefetch_sc = [&](int sidx) {   // the RPL * N * 512 bytes of a super-chunk are RPL * 4N lines
+            if (lane < RPL * 4 * N) {
+                const int half = lane / (4 * N), line = lane % (4 * N);
+                const char* p = (const char*)((half ? i1 : i0) - lane + (size_t)sidx * N * 32) + line * 128;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+            }
+        };
+        if (warp < nsc) {
+#pragma unroll
+            for (int v = 0; v < N; ++v) {
+                const uint4 t0 = ld_stream(i0 + ((size_t)warp * N + v) * 32);
+                w0[4 * v] = t0.x; w0[4 * v + 1] = t0.y; w0[4 * v + 2] = t0.z; w0[4 * v + 3] = t0.w;
+                if (RPL == 2) {
+                    const uint4 t1 = ld_stream(i1 + ((size_t)warp * N + v) * 32);
+                    w1[4 * v] = t1.x; w1[4 * v + 1] = t1.y; w1[4 * v + 2] = t1.z; w1[4 * v + 3] = t1.w;
+                }
+            }
+        }
+        if (a.pf_dist > 0)
+            for (int r = 1; r <= a.pf_dist; ++r)
+                if (warp + r * W < nsc) prefetch_sc(warp + r * W);
+
+        // (1) pair tables: warp w fills entries t in [w*T/W, (w+1)*T/W) of every channel half
+        {
+            constexpr int TW = T / W;  // entries per warp
+#pragma unroll
+            for (int half = 0; half < RPL; ++half) {
+                const int row = (half ? blk1 : blk0) * kRowsPerBlock + lane;
+                const uint16_t* cb = b.cb + (size_t)row * E;
+                unsigned char* dst = tab + half * 128 + lane * 4;
+                if (TW >= E) {
+                    // all low indices, TW/E high indices per warp
+                    uint32_t c[E / 2];
+#pragma unroll
+                    for (int i = 0; i < E / 8; ++i) {
+                        const uint4 t = __ldg((const uint4*)cb + i);
+                        c[4 * i] = t.x; c[4 * i + 1] = t.y; c[4 * i + 2] = t.z; c[4 * i + 3] = t.w;
+                    }
+#pragma unroll
+                    for (int hh = 0; hh < TW / E; ++hh) {
+                        const int hi = warp * (TW / E) + hh;
+                        const uint32_t hv = __ldg(cb + hi);
+#pragma unroll
+                        for (int lo = 0; lo < E; ++lo) {
+                            const uint32_t lv = (lo & 1) ? (c[lo >> 1] >> 16) : (c[lo >> 1] & 0xffffu);
+                            *(uint32_t*)(dst + (size_t)(hi * E + lo) * kStride) = lv | (hv << 16);
+                        }
+                    }
+                } else {
+                    // small tables (N = 2): TW < E entries per warp
+#pragma unroll
+                    for (int i = 0; i < TW; ++i) {
+                        const int t = warp * TW + i;
+                        const uint32_t lv = __ldg(cb + (t & (E - 1))), hv = __ldg(cb + (t >> N));
+                        *(uint32_t*)(dst + (size_t)t * kStride) = lv | (hv << 16);
+                    }
+                }
+            }
+        }
+        // (2) x (fp16 bits, all of K: the outlier warp gathers from it); x may come from the previous kernel
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        {
+            const int nvec = K / 8;  // uint4 per batch row
+            for (int t = threadIdx.x; t < NB * nvec; t += kDense) {
+                const int bb = t / nvec, kk = (t - bb * nvec) * 8;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
+                *(uint4*)(xs + (size_t)bb * K + kk) = v;
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kDense + 32) : "memory");  // tables and x visible
+
+        // (3) main loop
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t base0 = (uint32_t)lane * 4u, base1 = base0 | 128u;
+        const int g = lane >> 2, t4 = lane & 3;
+        // B fragment: lane (g', t') feeds column n = g' with the k slots of group t'.  Column t' of
+        // batch row 0 is fed by g' == t'; column 4 + t' of batch row 1 by g' == t' + 4.
+        const bool diag0 = (g == t4);
+        const bool diag1 = (NB > 1) && (g == t4 + 4);
+        const bool diag = diag0 || diag1;
+        const unsigned char* xrow =
+            (const unsigned char*)xs + (diag1 ? (size_t)K * 2 : 0) + (size_t)sc0 * (kSuper * 2);
+
+        auto lookup = [&](uint32_t (&f)[4], const uint32_t* u0, const uint32_t* u1, int m) {
+            f[0] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u0, 2 * m, base0));
+            f[2] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u0, 2 * m + 1, base0));
+            if (RPL == 2) {
+                f[1] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u1, 2 * m, base1));
+                f[3] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u1, 2 * m + 1, base1));
+            } else {
+                f[1] = 0u; f[3] = 0u;
+            }
+        };
+        // One super-chunk.  Look-ups run one mma ahead of the tensor pipe; as soon as the last pair of
+        // a 16-byte vector has been looked up, the vector's registers are reloaded with the same
+        // vector of this warp's next super-chunk (the index stream needs 4 * N * RPL registers).
+        auto compute_sc = [&](uint32_t* u0, uint32_t* u1, int sidx, bool has_next, int snext) {
+            const unsigned char* xp = xrow + (size_t)sidx * (kSuper * 2);
+            uint32_t fa[4], fb[4];
+            uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = make_uint4(0u, 0u, 0u, 0u);
+            if (diag) xa = *(const uint4*)xp;
+            lookup(fa, u0, u1, 0);
+            auto reload = [&](int gi) {   // gi: group whose look-ups were just issued (compile time)
+#pragma unroll
+                for (int v = 0; v < N; ++v) {
+                    const int plast = (128 * (v + 1) + 2 * N - 1) / (2 * N) - 1;   // last pair touching vector v
+                    if (plast / 2 == gi && has_next) {
+                        const uint4 t0 = ld_stream(i0 + ((size_t)snext * N + v) * 32);
+                        u0[4 * v] = t0.x; u0[4 * v + 1] = t0.y; u0[4 * v + 2] = t0.z; u0[4 * v + 3] = t0.w;
+                        if (RPL == 2) {
+                            const uint4 t1 = ld_stream(i1 + ((size_t)snext * N + v) * 32);
+                            u1[4 * v] = t1.x; u1[4 * v + 1] = t1.y; u1[4 * v + 2] = t1.z; u1[4 * v + 3] = t1.w;
+                        }
+                    }
+                }
+            };
+#pragma unroll
+            for (int m = 0; m < kSuper / 4; m += 4) {   // one mma per 4 consecutive k
+                if (diag) xb = *(const uint4*)(xp + (m + 2) * 8);
+                lookup(fb, u0, u1, m + 1);
+                reload(m + 1);
+                mma16816(c0, fa[0], fa[1], fa[2], fa[3], xa.x, xa.y);
+                lookup(fa, u0, u1, m + 2);
+                reload(m + 2);
+                mma16816(c1, fb[0], fb[1], fb[2], fb[3], xa.z, xa.w);
+                if (m + 4 < kSuper / 4) { if (diag) xa = *(const uint4*)(xp + (m + 4) * 8); }
+                lookup(fb, u0, u1, m + 3);
+                reload(m + 3);
+                mma16816(c0, fa[0], fa[1], fa[2], fa[3], xb.x, xb.y);
+                if (m + 4 < kSuper / 4) {
+                    lookup(fa, u0, u1, m + 4);
+                    reload(m + 4);
+                }
+                mma16816(c1, fb[0], fb[1], fb[2], fb[3], xb.z, xb.w);
+            }
+        };
+#pragma unroll 1
+        for (int s = warp; s < nsc; s += W) {
+            if (a.pf_dist > 0 && s + (a.pf_dist + 1) * W < nsc) prefetch_sc(s + (a.pf_dist + 1) * W);
+            compute_sc(w0, w1, s, s + W < nsc, s + W);
+        }
+
+        // (4) scatter the fragment to channel order: lane (g, t) holds D[g][2t], D[g][2t+1], D[g+8][..]
+        //     column n < 4: batch 0 of lane 4g + n; column n >= 4: batch 1 of lane 4g + n - 4
+        {
+            const float v0 = c0[0] + c1[0], v1 = c0[1] + c1[1], v2 = c0[2] + c1[2], v3 = c0[3] + c1[3];
+            const int bb = t4 >> 1;                  // batch row held by this lane's columns
+            const int l0 = 4 * g + 2 * (t4 & 1);     // channel lane of column 2t
+            if (bb < NB) {
+                float* r = red + ((size_t)warp * NB + bb) * ROWS;
+                r[l0] = v0; r[l0 + 1] = v1;
+                if (RPL == 2) { r[32 + l0] = v2; r[32 + l0 + 1] = v3; }
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---------------------------------------------------- fixed-order reduction, store / split-K finish
+    const int t = threadIdx.x;
+    const int bb = t / ROWS, r = t % ROWS;
+    const bool active = t < NB * ROWS;
+    // channel r of the block: rows of blk0 for r < 32, of blk1 for r >= 32
+    const bool dup = (r >= 32) && (RPL * blk + 1 >= a.RB);
+    const int row = blk * ROWS + r;
+    float total = 0.f;
+    if (active) {
+        total = osum[bb * ROWS + r];
+#pragma unroll
+        for (int w = 0; w < W; ++w) total += red[((size_t)w * NB + bb) * ROWS + r];
+    }
+    if (KS > 1) {
+        __shared__ int s_last;
+        if (active) a.partial[((size_t)ks * NB + bb) * a.rows_ws + row] = total;
+        __threadfence();
+        __syncthreads();
+        if (t == 0) s_last = (atomicAdd(a.tickets + blk, 1) == KS - 1);
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        if (active) {
+            total = 0.f;
+            for (int k2 = 0; k2 < KS; ++k2) total += __ldcg(a.partial + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+        }
+        if (t == 0) a.tickets[blk] = 0;
+    }
+    if (active && !dup && bb < a.nb && row < a.rows) {
+        if (a.y_is_fp16)
+            ((uint16_t*)a.y)[(size_t)bb * a.rows + row] = f2h(total);
+        else
+            ((float*)a.y)[(size_t)bb * a.rows + row] = total;
+    }
+}
+
+// ------------------------------------------------------------------------------------ host side
+
+static int g_pair_ks_override = 0;  // 0 = policy below
+static int g_pair_pf_dist = 0;  // L2 prefetch measured slower than none on B200
+
+void pair_set_ksplit_override(int ks) { g_pair_ks_override = ks; }
+void pair_set_prefetch(int d) { g_pair_pf_dist = d; }
+
+struct PairConfig { int rpl, warps, slots; };
+
+static PairConfig pair_config(int bits) {
+    // N <= 4: two rows per lane, 8 dense warps, two CTAs per SM.  N = 5: the pair table of a row is
+    // 4 KB, so one row per lane (128 KB of tables), 16 dense warps, one CTA per SM.
+    if (bits == 5) return PairConfig{1, 16, 148};
+    return PairConfig{2, 8, 296};
+}
+
+struct PairSchedule { int blocks, n_full, kst, sc_per_split, grid; };
+
+static PairSchedule pair_schedule(const Layout& l) {
+    const PairConfig cfg = pair_config(l.bits);
+    PairSchedule sc{};
+    sc.blocks = (l.RB + cfg.rpl - 1) / cfg.rpl;
+    int rem = sc.blocks % cfg.slots;
+    int kst = 1;
+    if (g_pair_ks_override > 0) {
+        rem = sc.blocks; kst = g_pair_ks_override;
+    } else if (rem > 0) {
+        // cut the blocks of the last, partial round along K so that they fill the idle slots; every cut
+        // costs another fill of the pair tables and a trip through global memory, so keep slices >= 1024
+        kst = (cfg.slots + rem / 2) / rem;
+        const int kmax = l.SC / 8 > 1 ? l.SC / 8 : 1;
+        if (kst > kmax) kst = kmax;
+        if (kst < 1) kst = 1;
+    }
+    if (kst > l.SC) kst = l.SC;
+    if (kst <= 1) { rem = 0; kst = 1; }
+    sc.n_full = sc.blocks - rem;
+    sc.sc_per_split = (l.SC + kst - 1) / kst;
+    sc.kst = (l.SC + sc.sc_per_split - 1) / sc.sc_per_split;
+    sc.grid = sc.n_full + rem * sc.kst;
+    return sc;
+}
+
+static size_t pair_smem_bytes(const Layout& l, int nb) {
+    const PairConfig cfg = pair_config(l.bits);
+    const int rows = 32 * cfg.rpl;
+    const size_t T = (size_t)l.E * l.E;
+    return T * 128 * cfg.rpl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4 + (size_t)nb * rows * 4 +
+           (size_t)(rows + 4) * 4 + (size_t)nb * kOutBatch * 4;
+}
+
+bool pair_supported(const Layout& l, int batch, int n_problems) {
+    if (l.mode != 0 || l.bits < 2 || l.bits > 5 || batch > 2 || n_problems != 1) return false;
+    return pair_smem_bytes(l, batch) <= (pair_config(l.bits).rpl == 2 ? 110u : 220u) * 1024u;
+}
+
+size_t pair_workspace_bytes(const Layout& l) {
+    const int ksmax = 64 < l.SC ? 64 : l.SC;
+    return align256((size_t)l.RB * 4) + align256((size_t)ksmax * 2 * (size_t)(l.RB + 1) * 32 * 4);
+}
+
+template <int N, int NB, int RPL, int W>
+static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_pair_kernel<N, NB, RPL, W>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3((W + 1) * 32, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_pair_kernel<N, NB, RPL, W>, a);
+}
+
+cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s) {
+    const PairConfig cfg = pair_config(l.bits);
+    const PairSchedule sch = pair_schedule(l);
+    PairArgs a{};
+    a.off = offsets_of(l);
+    a.packed = c.packed; a.x = c.x; a.y = c.y;
+    a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC;
+    a.rows_ws = sch.blocks * 32 * cfg.rpl;
+    a.n_full = sch.n_full; a.kst = sch.kst; a.sc_per_split = sch.sc_per_split;
+    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
+    a.pf_dist = g_pair_pf_dist;
+    a.tickets = (int*)c.workspace;
+    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
+    const size_t smem = pair_smem_bytes(l, c.batch);
+    dim3 grid((unsigned)sch.grid, 1, 1);
+    switch (l.bits * 10 + c.batch) {
+        case 21: return launch_pair<2, 1, 2, 8>(a, grid, smem, s);
+        case 22: return launch_pair<2, 2, 2, 8>(a, grid, smem, s);
+        case 31: return launch_pair<3, 1, 2, 8>(a, grid, smem, s);
+        case 32: return launch_pair<3, 2, 2, 8>(a, grid, smem, s);
+        case 41: return launch_pair<4, 1, 2, 8>(a, grid, smem, s);
+        case 42: return launch_pair<4, 2, 2, 8>(a, grid, smem, s);
+        case 51: return launch_pair<5, 1, 1, 16>(a, grid, smem, s);
+        case 52: return launch_pair<5, 2, 1, 16>(a, grid, smem, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace xfp

@@ -42,4 +42,16 @@ int generic_ksplit(const Layout& l, int batch_tile);
 size_t generic_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t s);
 
+// Fast V2 path (pair tables + mma.sync fragments); see xfp_gemv_pair.cu.
+bool pair_supported(const Layout& l, int batch, int n_problems);
+size_t pair_workspace_bytes(const Layout& l);
+cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s);
+void pair_set_ksplit_override(int ks);
+void pair_set_prefetch(int d);
+
+inline size_t workspace_bytes_for(const Layout& l) {
+    const size_t g = generic_workspace_bytes(l), p = pair_workspace_bytes(l);
+    return g > p ? g : p;
+}
+
 }  // namespace xfp
