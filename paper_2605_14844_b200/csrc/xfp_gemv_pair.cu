@@ -21,10 +21,13 @@
 // first and measured ~8 issue slots per pair against ~3 here; that is why the dot product runs on
 // the tensor pipe even at batch 1.)
 //
-// Outliers (step 3) are summed by one extra warp per CTA, concurrently with the dense warps: the
-// block's CSR entries are contiguous, so the warp reads them coalesced, gathers x from the staged
-// copy in shared memory, writes the products to shared memory, and each lane then adds up the
-// segments of its own rows in CSR order (deterministic).
+// Outliers (step 3) ride in the same pass: xfp_pack stores every 32-row block's outliers as a
+// transposed slab (slot j of channel l at slab + j*32 + l), so a warp reads one slot of all 32
+// channels with one coalesced load and every lane adds val * x[col] (x gathered from the staged
+// copy in shared memory) to an accumulator of its own channel.  Slots are dealt round-robin to the
+// dense warps and consumed between super-chunks, their loads issued one iteration ahead.  Rows
+// longer than the slab (pathological skew) finish from the CSR arrays.  The order of additions is
+// fixed by the schedule, so results are reproducible.
 //
 // Schedule.  Blocks that fill whole rounds of CTA slots run over all of K; the blocks of the last,
 // partial round are cut along K so that they occupy the idle slots, and their partial sums are
@@ -39,7 +42,7 @@
 
 namespace xfp {
 
-constexpr int kOutBatch = 512;  // outlier entries fetched and staged per round
+constexpr int kSlotsPerRound = 4;  // outlier slots a warp keeps in flight per channel half
 
 struct PairArgs {
     Offsets off;
@@ -87,7 +90,7 @@ __device__ __forceinline__ uint32_t pair_addr(const uint32_t* w, int p, uint32_t
 }
 
 template <int N, int NB, int RPL, int W>
-__global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
+__global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
     constexpr int E = 1 << N;
     constexpr int T = E * E;                   // pair-table entries per channel
     constexpr int ROWS = 32 * RPL;             // channels per CTA
@@ -95,7 +98,7 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
     constexpr int kTabBytes = T * kStride;
     constexpr int kDense = W * 32;
     extern __shared__ __align__(16) unsigned char smem[];
-    // [tables | x fp16 [NB][K] | red[W][NB][ROWS] | osum[NB][ROWS] | rps[ROWS + 4] | sprod[NB][kOutBatch]]
+    // [tables | x fp16 [NB][K] | red[W][NB][ROWS]]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
     int blk, ks, KS, spp;
@@ -113,78 +116,12 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
     unsigned char* tab = smem;
     uint16_t* xs = (uint16_t*)(smem + kTabBytes);               // [NB][K]
     float* red = (float*)(xs + (size_t)NB * K);                 // [W][NB][ROWS]
-    float* osum = red + W * NB * ROWS;                          // [NB][ROWS]
-    int* rps = (int*)(osum + NB * ROWS);                        // [ROWS + 1] row pointers of the block
-    float* sprod = (float*)(rps + ROWS + 4);                    // [NB][kOutBatch]
 
     // the 32-row blocks of this CTA (the second is clamped when RB is odd; its results are dropped)
     const int blk0 = RPL * blk;
     const int blk1 = min(RPL * blk + (RPL - 1), a.RB - 1);
 
-    if (warp == W) {
-        // ------------------------------------------------ outlier warp: CSR entries of this CTA's rows
-        const int row0 = blk * ROWS;
-        {
-            const int last = a.RB * kRowsPerBlock;               // rowptr has rows_pad + 1 entries
-#pragma unroll
-            for (int h = 0; h < RPL; ++h) rps[32 * h + lane] = __ldg(b.rowptr + min(row0 + 32 * h + lane, last));
-            if (lane == 0) rps[ROWS] = __ldg(b.rowptr + min(row0 + ROWS, last));
-        }
-        __syncwarp();
-        // this CTA's share of the block's entries (an even cut when K is split)
-        const int e_lo = rps[0], e_hi = rps[ROWS];
-        const int e0 = e_lo + (int)(((long long)(e_hi - e_lo) * ks) / KS);
-        const int e1 = e_lo + (int)(((long long)(e_hi - e_lo) * (ks + 1)) / KS);
-        // Entries are fetched kOutBatch = 512 at a time (16 per lane, all loads of a batch in flight
-        // together); the next batch travels while the current one is processed, and the first batch
-        // travels while the dense warps fill the tables.
-        uint32_t ea[16], eb[16];
-        auto fetch = [&](uint32_t (&d)[16], int c) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) d[j] = (c + j * 32 + lane < e1) ? __ldg(b.oent + c + j * 32 + lane) : 0u;
-        };
-        float acc[NB][RPL];
-#pragma unroll
-        for (int bb = 0; bb < NB; ++bb)
-#pragma unroll
-            for (int h = 0; h < RPL; ++h) acc[bb][h] = 0.f;
-        auto consume = [&](const uint32_t (&d)[16], int c) {
-            const int n = min(kOutBatch, e1 - c);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float v = h2f((uint16_t)(d[j] >> 16));     // entries past e1 are zero
-                const uint32_t col = d[j] & 0xffffu;
-#pragma unroll
-                for (int bb = 0; bb < NB; ++bb) sprod[bb * kOutBatch + j * 32 + lane] = v * h2f(xs[(size_t)bb * K + col]);
-            }
-            __syncwarp();
-#pragma unroll
-            for (int h = 0; h < RPL; ++h) {
-                const int r = lane + 32 * h;
-                const int s0 = max(rps[r], c), s1 = min(rps[r + 1], c + n);
-                for (int p = s0; p < s1; ++p) {
-#pragma unroll
-                    for (int bb = 0; bb < NB; ++bb) acc[bb][h] += sprod[bb * kOutBatch + (p - c)];
-                }
-            }
-            __syncwarp();
-        };
-        if (e0 < e1) fetch(ea, e0);
-        asm volatile("bar.sync 1, %0;" ::"n"(kDense + 32) : "memory");   // x staged by the dense warps
-        for (int c = e0; c < e1; c += 2 * kOutBatch) {
-            if (c + kOutBatch < e1) fetch(eb, c + kOutBatch);
-            consume(ea, c);
-            if (c + kOutBatch < e1) {
-                if (c + 2 * kOutBatch < e1) fetch(ea, c + 2 * kOutBatch);
-                consume(eb, c + kOutBatch);
-            }
-        }
-#pragma unroll
-        for (int bb = 0; bb < NB; ++bb)
-#pragma unroll
-            for (int h = 0; h < RPL; ++h) osum[bb * ROWS + 32 * h + lane] = acc[bb][h];
-        __syncthreads();  // partial sums ready
-    } else {
+    {
         // ------------------------------------------------ dense warps
         // (0) start streaming this warp's first super-chunk before anything else
         uint32_t w0[4 * N + 1], w1[RPL == 2 ? 4 * N + 1 : 1];
@@ -213,6 +150,56 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
         if (a.pf_dist > 0)
             for (int r = 1; r <= a.pf_dist; ++r)
                 if (warp + r * W < nsc) prefetch_sc(warp + r * W);
+        // outlier slabs of this CTA's row-blocks: slots gw, gw + stride, ... belong to this warp
+        const int gw = ks * W + warp, ostride = KS * W;
+        const uint32_t* slab[RPL];
+        int width[RPL];
+        uint32_t oe[RPL][kSlotsPerRound];
+        float oacc[NB][RPL];
+        int oround = 0, nrounds = 0;
+#pragma unroll
+        for (int h = 0; h < RPL; ++h) {
+            const int bh = h ? blk1 : blk0;
+            const int q0 = __ldg(b.ellptr + bh), q1 = __ldg(b.ellptr + bh + 1);
+            slab[h] = b.ell + q0 + lane;
+            width[h] = (q1 - q0) >> 5;
+            const int mine = width[h] > gw ? (width[h] - gw + ostride - 1) / ostride : 0;   // slots of this warp
+            nrounds = max(nrounds, (mine + kSlotsPerRound - 1) / kSlotsPerRound);
+#pragma unroll
+            for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = 0.f;
+        }
+        auto fetch_slots = [&](int round) {
+#pragma unroll
+            for (int h = 0; h < RPL; ++h)
+#pragma unroll
+                for (int q = 0; q < kSlotsPerRound; ++q) {
+                    const int j = gw + (round * kSlotsPerRound + q) * ostride;
+                    oe[h][q] = j < width[h] ? __ldg(slab[h] + (size_t)j * 32) : 0u;
+                }
+        };
+        auto consume_slots = [&]() {
+#pragma unroll
+            for (int h = 0; h < RPL; ++h)
+#pragma unroll
+                for (int q = 0; q < kSlotsPerRound; ++q) {
+                    const float v = h2f((uint16_t)(oe[h][q] >> 16));
+                    const uint32_t col = oe[h][q] & 0xffffu;
+#pragma unroll
+                    for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = fmaf(v, h2f(xs[(size_t)bb * K + col]), oacc[bb][h]);
+                }
+        };
+        if (nrounds > 0) fetch_slots(0);
+        // rows longer than their slab (warp 0 of the first K slice finishes them from the CSR arrays)
+        int sp0[RPL], sp1[RPL];
+#pragma unroll
+        for (int h = 0; h < RPL; ++h) {
+            sp0[h] = sp1[h] = 0;
+            if (warp == 0 && ks == 0) {
+                const int row = (h ? blk1 : blk0) * kRowsPerBlock + lane;
+                sp0[h] = __ldg(b.rowptr + row) + width[h];
+                sp1[h] = __ldg(b.rowptr + row + 1);
+            }
+        }
 
         // (1) pair tables: warp w fills entries t in [w*T/W, (w+1)*T/W) of every channel half
         {
@@ -262,7 +249,7 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
                 *(uint4*)(xs + (size_t)bb * K + kk) = v;
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kDense + 32) : "memory");  // tables and x visible
+        __syncthreads();  // tables and x visible
 
         // (3) main loop
         float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -332,8 +319,24 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
 #pragma unroll 1
         for (int s = warp; s < nsc; s += W) {
             if (a.pf_dist > 0 && s + (a.pf_dist + 1) * W < nsc) prefetch_sc(s + (a.pf_dist + 1) * W);
+            if (oround < nrounds) {
+                consume_slots();
+                if (++oround < nrounds) fetch_slots(oround);
+            }
             compute_sc(w0, w1, s, s + W < nsc, s + W);
         }
+        while (oround < nrounds) {   // more outlier rounds than super-chunks
+            consume_slots();
+            if (++oround < nrounds) fetch_slots(oround);
+        }
+#pragma unroll
+        for (int h = 0; h < RPL; ++h)
+            for (int p = sp0[h]; p < sp1[h]; ++p) {   // spill of an over-long row (rare)
+                const uint32_t e = __ldg(b.oent + p);
+#pragma unroll
+                for (int bb = 0; bb < NB; ++bb)
+                    oacc[bb][h] = fmaf(h2f((uint16_t)(e >> 16)), h2f(xs[(size_t)bb * K + (e & 0xffffu)]), oacc[bb][h]);
+            }
 
         // (4) scatter the fragment to channel order: lane (g, t) holds D[g][2t], D[g][2t+1], D[g+8][..]
         //     column n < 4: batch 0 of lane 4g + n; column n >= 4: batch 1 of lane 4g + n - 4
@@ -346,6 +349,11 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
                 r[l0] = v0; r[l0 + 1] = v1;
                 if (RPL == 2) { r[32 + l0] = v2; r[32 + l0 + 1] = v3; }
             }
+            __syncwarp();
+#pragma unroll
+            for (int bb2 = 0; bb2 < NB; ++bb2)
+#pragma unroll
+                for (int h = 0; h < RPL; ++h) red[((size_t)warp * NB + bb2) * ROWS + 32 * h + lane] += oacc[bb2][h];
         }
         __syncthreads();
     }
@@ -359,7 +367,6 @@ __global__ void __launch_bounds__((W + 1) * 32, RPL == 2 ? 2 : 1) gemv_pair_kern
     const int row = blk * ROWS + r;
     float total = 0.f;
     if (active) {
-        total = osum[bb * ROWS + r];
 #pragma unroll
         for (int w = 0; w < W; ++w) total += red[((size_t)w * NB + bb) * ROWS + r];
     }
@@ -434,8 +441,7 @@ static size_t pair_smem_bytes(const Layout& l, int nb) {
     const PairConfig cfg = pair_config(l.bits);
     const int rows = 32 * cfg.rpl;
     const size_t T = (size_t)l.E * l.E;
-    return T * 128 * cfg.rpl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4 + (size_t)nb * rows * 4 +
-           (size_t)(rows + 4) * 4 + (size_t)nb * kOutBatch * 4;
+    return T * 128 * cfg.rpl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4;
 }
 
 bool pair_supported(const Layout& l, int batch, int n_problems) {
@@ -459,7 +465,7 @@ static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaSt
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3((W + 1) * 32, 1, 1);
+    cfg.blockDim = dim3(W * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];

@@ -13,6 +13,11 @@
 //   gsm     V2a: half2 [RB][SC][32]    (scale, mid) of the same group
 //   rowptr  int32 [rows_pad + 1]       clamped to [0, nnz]
 //   oent    u32 [nnz]                  column | fp16 value << 16, CSR order
+//   ellptr  int32 [RB + 1]             start of each row-block's transposed outlier slab, in entries
+//   ell     u32 [ell_cap]              slab of row-block b: slot j of channel b*32+l at ellptr[b] + j*32 + l,
+//                                      width W_b = min(longest row of the block, 2*ceil(nnz_b/32) + 8) slots,
+//                                      unused slots hold column 0 / value +0.  Rows longer than W_b keep their
+//                                      remaining entries in the CSR arrays only (the "spill").
 #pragma once
 #include <cstddef>
 #include <cstdint>
@@ -26,7 +31,8 @@ struct Layout {
     int mode, rows, cols, bits, L, E;
     int RB, SC, rows_pad;
     long long nnz;
-    size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_oent, total;
+    size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_oent, off_ellptr, off_ell, total;
+    long long ell_cap;  // entries reserved for the transposed slabs (an upper bound from nnz and RB)
 };
 
 inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
@@ -45,6 +51,9 @@ inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, 
     l.off_gsm = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * 32 * 4 : 0));
     l.off_rowptr = o; o = align256(o + (size_t)(l.rows_pad + 1) * 4);
     l.off_oent = o;   o = align256(o + (size_t)nnz * 4);
+    l.ell_cap = nnz ? 2 * nnz + 320LL * l.RB : 0;
+    l.off_ellptr = o; o = align256(o + (size_t)(l.RB + 1) * 4);
+    l.off_ell = o;    o = align256(o + (size_t)l.ell_cap * 4);
     l.total = o;
     return l;
 }
