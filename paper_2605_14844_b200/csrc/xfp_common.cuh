@@ -44,12 +44,11 @@ struct Blob {
     const uint32_t* gsm;  // half2 bits: scale | mid << 16
     const int* rowptr;
     const uint32_t* oent;
-    const int* ellptr;
     const uint32_t* ell;
 };
 
 struct Offsets {
-    size_t idx, cb, gid, gsm, rowptr, oent, ellptr, ell;
+    size_t idx, cb, gid, gsm, rowptr, oent, ell;
 };
 
 __host__ __device__ inline Blob blob_at(const void* packed, const Offsets& o) {
@@ -61,13 +60,12 @@ __host__ __device__ inline Blob blob_at(const void* packed, const Offsets& o) {
     r.gsm = (const uint32_t*)(b + o.gsm);
     r.rowptr = (const int*)(b + o.rowptr);
     r.oent = (const uint32_t*)(b + o.oent);
-    r.ellptr = (const int*)(b + o.ellptr);
     r.ell = (const uint32_t*)(b + o.ell);
     return r;
 }
 
 inline Offsets offsets_of(const Layout& l) {
-    return Offsets{l.off_idx, l.off_cb, l.off_gid, l.off_gsm, l.off_rowptr, l.off_oent, l.off_ellptr, l.off_ell};
+    return Offsets{l.off_idx, l.off_cb, l.off_gid, l.off_gsm, l.off_rowptr, l.off_oent, l.off_ell};
 }
 
 }  // namespace xfp

@@ -38,6 +38,8 @@
 // griddepcontrol.wait (programmatic dependent launch) before it touches x, y or the workspace.
 // Back-to-back calls on one stream therefore overlap the next call's weight streaming with the
 // current call's tail.
+#include <cooperative_groups.h>
+
 #include "xfp_internal.h"
 
 namespace xfp {
@@ -51,13 +53,24 @@ struct PairArgs {
     void* y;
     float* partial;  // [KS][NB][rows_ws]
     int* tickets;    // [blocks]
-    int rows, cols, RB, SC, rows_ws;
+    int rows, cols, RB, SC, rows_ws, ell_slots;
     int nb, y_is_fp16;
     // schedule: work items [0, n_full) are whole blocks; the remaining blocks are cut into kst
     // K-slices of sc_per_split super-chunks each
     int n_full, kst, sc_per_split;
     int pf_dist;  // L2 prefetch distance in warp iterations (0 = off)
+    int cluster;  // 1: the kst CTAs of a block form a thread-block cluster and reduce through DSMEM
+    int dbg;      // timing probes only: 1 = return after the dependency wait, 2 = skip the main loop, 3 = no PDL
+    unsigned long long* trace;  // timing probes only: per CTA 8 globaltimer stamps
 };
+
+__device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
+    if (a.trace && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        a.trace[(size_t)blockIdx.x * 8 + slot] = t;
+    }
+}
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -90,7 +103,7 @@ __device__ __forceinline__ uint32_t pair_addr(const uint32_t* w, int p, uint32_t
 }
 
 template <int N, int NB, int RPL, int W>
-__global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
+__global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
     constexpr int E = 1 << N;
     constexpr int T = E * E;                   // pair-table entries per channel
     constexpr int ROWS = 32 * RPL;             // channels per CTA
@@ -101,6 +114,11 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
     // [tables | x fp16 [NB][K] | red[W][NB][ROWS]]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
+    stamp(a, 0);
+    if (a.dbg == 1) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     int blk, ks, KS, spp;
     if ((int)blockIdx.x < a.n_full) {
         blk = blockIdx.x; ks = 0; KS = 1; spp = a.SC;
@@ -147,24 +165,37 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
                 }
             }
         }
+        // one row per lane leaves registers for a second super-chunk in flight (short K loops are
+        // otherwise a chain of DRAM round trips)
+        constexpr bool kTwoDeep = (RPL == 1);
+        uint32_t z0[kTwoDeep ? 4 * N + 1 : 1];
+        if (kTwoDeep) {
+            z0[4 * N] = 0u;
+            if (warp + W < nsc) {
+#pragma unroll
+                for (int v = 0; v < N; ++v) {
+                    const uint4 t0 = ld_stream(i0 + ((size_t)(warp + W) * N + v) * 32);
+                    z0[4 * v] = t0.x; z0[4 * v + 1] = t0.y; z0[4 * v + 2] = t0.z; z0[4 * v + 3] = t0.w;
+                }
+            }
+        }
         if (a.pf_dist > 0)
             for (int r = 1; r <= a.pf_dist; ++r)
                 if (warp + r * W < nsc) prefetch_sc(warp + r * W);
-        // outlier slabs of this CTA's row-blocks: slots gw, gw + stride, ... belong to this warp
+        // outlier slabs of this CTA's row-blocks: slots gw, gw + stride, ... belong to this warp.  The first
+        // round is fetched before the rows' lengths are known (any slot below the capacity is readable).
         const int gw = ks * W + warp, ostride = KS * W;
         const uint32_t* slab[RPL];
         int width[RPL];
+        uint32_t olen[RPL];
         uint32_t oe[RPL][kSlotsPerRound];
         float oacc[NB][RPL];
         int oround = 0, nrounds = 0;
 #pragma unroll
         for (int h = 0; h < RPL; ++h) {
-            const int bh = h ? blk1 : blk0;
-            const int q0 = __ldg(b.ellptr + bh), q1 = __ldg(b.ellptr + bh + 1);
-            slab[h] = b.ell + q0 + lane;
-            width[h] = (q1 - q0) >> 5;
-            const int mine = width[h] > gw ? (width[h] - gw + ostride - 1) / ostride : 0;   // slots of this warp
-            nrounds = max(nrounds, (mine + kSlotsPerRound - 1) / kSlotsPerRound);
+            slab[h] = b.ell + (size_t)(h ? blk1 : blk0) * (a.ell_slots + 1) * 32 + lane;
+            width[h] = a.ell_slots;
+            olen[h] = a.ell_slots ? __ldg(slab[h]) : 0u;
 #pragma unroll
             for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = 0.f;
         }
@@ -174,7 +205,7 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
 #pragma unroll
                 for (int q = 0; q < kSlotsPerRound; ++q) {
                     const int j = gw + (round * kSlotsPerRound + q) * ostride;
-                    oe[h][q] = j < width[h] ? __ldg(slab[h] + (size_t)j * 32) : 0u;
+                    oe[h][q] = j < width[h] ? __ldg(slab[h] + (size_t)(1 + j) * 32) : 0u;
                 }
         };
         auto consume_slots = [&]() {
@@ -188,47 +219,43 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
                     for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = fmaf(v, h2f(xs[(size_t)bb * K + col]), oacc[bb][h]);
                 }
         };
-        if (nrounds > 0) fetch_slots(0);
-        // rows longer than their slab (warp 0 of the first K slice finishes them from the CSR arrays)
-        int sp0[RPL], sp1[RPL];
-#pragma unroll
-        for (int h = 0; h < RPL; ++h) {
-            sp0[h] = sp1[h] = 0;
-            if (warp == 0 && ks == 0) {
-                const int row = (h ? blk1 : blk0) * kRowsPerBlock + lane;
-                sp0[h] = __ldg(b.rowptr + row) + width[h];
-                sp1[h] = __ldg(b.rowptr + row + 1);
-            }
-        }
-
-        // (1) pair tables: warp w fills entries t in [w*T/W, (w+1)*T/W) of every channel half
-        {
-            constexpr int TW = T / W;  // entries per warp
+        if (a.ell_slots) fetch_slots(0);
+        // codebooks of this lane's channels (for the table fill below)
+        constexpr int TW = T / W;  // table entries per warp
+        uint32_t cbw[RPL][TW >= E ? E / 2 : 1];
+        uint32_t cbh[RPL][TW >= E ? TW / E : 1];
+        if (TW >= E) {
 #pragma unroll
             for (int half = 0; half < RPL; ++half) {
-                const int row = (half ? blk1 : blk0) * kRowsPerBlock + lane;
-                const uint16_t* cb = b.cb + (size_t)row * E;
+                const uint16_t* cb = b.cb + (size_t)((half ? blk1 : blk0) * kRowsPerBlock + lane) * E;
+#pragma unroll
+                for (int i = 0; i < E / 8; ++i) {
+                    const uint4 t = __ldg((const uint4*)cb + i);
+                    cbw[half][4 * i] = t.x; cbw[half][4 * i + 1] = t.y; cbw[half][4 * i + 2] = t.z; cbw[half][4 * i + 3] = t.w;
+                }
+#pragma unroll
+                for (int hh = 0; hh < TW / E; ++hh) cbh[half][hh] = __ldg(cb + warp * (TW / E) + hh);
+            }
+        }
+        // (1) pair tables: warp w fills entries t in [w*T/W, (w+1)*T/W) of every channel half
+        {
+#pragma unroll
+            for (int half = 0; half < RPL; ++half) {
                 unsigned char* dst = tab + half * 128 + lane * 4;
                 if (TW >= E) {
-                    // all low indices, TW/E high indices per warp
-                    uint32_t c[E / 2];
-#pragma unroll
-                    for (int i = 0; i < E / 8; ++i) {
-                        const uint4 t = __ldg((const uint4*)cb + i);
-                        c[4 * i] = t.x; c[4 * i + 1] = t.y; c[4 * i + 2] = t.z; c[4 * i + 3] = t.w;
-                    }
 #pragma unroll
                     for (int hh = 0; hh < TW / E; ++hh) {
                         const int hi = warp * (TW / E) + hh;
-                        const uint32_t hv = __ldg(cb + hi);
+                        const uint32_t hv = cbh[half][hh];
 #pragma unroll
                         for (int lo = 0; lo < E; ++lo) {
-                            const uint32_t lv = (lo & 1) ? (c[lo >> 1] >> 16) : (c[lo >> 1] & 0xffffu);
+                            const uint32_t lv = (lo & 1) ? (cbw[half][lo >> 1] >> 16) : (cbw[half][lo >> 1] & 0xffffu);
                             *(uint32_t*)(dst + (size_t)(hi * E + lo) * kStride) = lv | (hv << 16);
                         }
                     }
                 } else {
                     // small tables (N = 2): TW < E entries per warp
+                    const uint16_t* cb = b.cb + (size_t)((half ? blk1 : blk0) * kRowsPerBlock + lane) * E;
 #pragma unroll
                     for (int i = 0; i < TW; ++i) {
                         const int t = warp * TW + i;
@@ -238,18 +265,48 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
                 }
             }
         }
-        // (2) x (fp16 bits, all of K: the outlier warp gathers from it); x may come from the previous kernel
+        // x may come from the previous kernel: everything above overlaps that kernel's tail
+        stamp(a, 1);
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        {
-            const int nvec = K / 8;  // uint4 per batch row
-            for (int t = threadIdx.x; t < NB * nvec; t += kDense) {
-                const int bb = t / nvec, kk = (t - bb * nvec) * 8;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
-                *(uint4*)(xs + (size_t)bb * K + kk) = v;
+        stamp(a, 2);
+        constexpr int XV = 4;                       // uint4 of x per thread per pass
+        const int nvec = NB * (K / 8);
+        uint4 xv[XV];
+#pragma unroll
+        for (int i = 0; i < XV; ++i) {
+            const int t = threadIdx.x + i * kDense;
+            xv[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (t < nvec) {
+                const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
+                if (bb < a.nb) xv[i] = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
             }
         }
+
+        stamp(a, 3);
+        // (2) x (fp16 bits, all of K: outlier columns are gathered from it) -> shared memory
+#pragma unroll
+        for (int i = 0; i < XV; ++i) {
+            const int t = threadIdx.x + i * kDense;
+            if (t < nvec) *(uint4*)(xs + (size_t)t * 8) = xv[i];
+        }
+        for (int t = threadIdx.x + XV * kDense; t < nvec; t += kDense) {   // K beyond XV passes
+            const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
+            *(uint4*)(xs + (size_t)t * 8) = v;
+        }
+        // the rows' slot counts are here by now: this warp's number of outlier rounds
+#pragma unroll
+        for (int h = 0; h < RPL; ++h) {
+            int wmax = (int)olen[h];
+#pragma unroll
+            for (int o = 16; o; o >>= 1) wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
+            width[h] = min(wmax, a.ell_slots);
+            const int mine = width[h] > gw ? (width[h] - gw + ostride - 1) / ostride : 0;
+            nrounds = max(nrounds, (mine + kSlotsPerRound - 1) / kSlotsPerRound);
+        }
         __syncthreads();  // tables and x visible
+        stamp(a, 4);
 
         // (3) main loop
         float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -316,28 +373,55 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
                 mma16816(c1, fb[0], fb[1], fb[2], fb[3], xb.z, xb.w);
             }
         };
+        if (kTwoDeep) {
 #pragma unroll 1
-        for (int s = warp; s < nsc; s += W) {
-            if (a.pf_dist > 0 && s + (a.pf_dist + 1) * W < nsc) prefetch_sc(s + (a.pf_dist + 1) * W);
-            if (oround < nrounds) {
-                consume_slots();
-                if (++oround < nrounds) fetch_slots(oround);
+            for (int s = warp; s < (a.dbg == 2 ? 0 : nsc); s += 2 * W) {
+                if (oround < nrounds) {
+                    consume_slots();
+                    if (++oround < nrounds) fetch_slots(oround);
+                }
+                compute_sc(w0, w1, s, s + 2 * W < nsc, s + 2 * W);
+                if (s + W < nsc) {
+                    if (oround < nrounds) {
+                        consume_slots();
+                        if (++oround < nrounds) fetch_slots(oround);
+                    }
+                    compute_sc(z0, w1, s + W, s + 3 * W < nsc, s + 3 * W);
+                }
             }
-            compute_sc(w0, w1, s, s + W < nsc, s + W);
+        } else {
+#pragma unroll 1
+            for (int s = warp; s < (a.dbg == 2 ? 0 : nsc); s += W) {
+                if (a.pf_dist > 0 && s + (a.pf_dist + 1) * W < nsc) prefetch_sc(s + (a.pf_dist + 1) * W);
+                if (oround < nrounds) {
+                    consume_slots();
+                    if (++oround < nrounds) fetch_slots(oround);
+                }
+                compute_sc(w0, w1, s, s + W < nsc, s + W);
+            }
         }
         while (oround < nrounds) {   // more outlier rounds than super-chunks
             consume_slots();
             if (++oround < nrounds) fetch_slots(oround);
         }
+        // Rows that fill their slab may continue in the CSR arrays (pathological skew only): warp 0 of
+        // the first K slice finishes them, one lane per row.
+        if (warp == 0 && ks == 0 && a.ell_slots) {
 #pragma unroll
-        for (int h = 0; h < RPL; ++h)
-            for (int p = sp0[h]; p < sp1[h]; ++p) {   // spill of an over-long row (rare)
-                const uint32_t e = __ldg(b.oent + p);
+            for (int h = 0; h < RPL; ++h) {
+                if ((int)olen[h] >= a.ell_slots) {
+                    const int row = (h ? blk1 : blk0) * kRowsPerBlock + lane;
+                    const int p1 = __ldg(b.rowptr + row + 1);
+                    for (int p = __ldg(b.rowptr + row) + a.ell_slots; p < p1; ++p) {
+                        const uint32_t e = __ldg(b.oent + p);
 #pragma unroll
-                for (int bb = 0; bb < NB; ++bb)
-                    oacc[bb][h] = fmaf(h2f((uint16_t)(e >> 16)), h2f(xs[(size_t)bb * K + (e & 0xffffu)]), oacc[bb][h]);
+                        for (int bb = 0; bb < NB; ++bb)
+                            oacc[bb][h] = fmaf(h2f((uint16_t)(e >> 16)), h2f(xs[(size_t)bb * K + (e & 0xffffu)]), oacc[bb][h]);
+                    }
+                }
             }
-
+        }
+        stamp(a, 5);
         // (4) scatter the fragment to channel order: lane (g, t) holds D[g][2t], D[g][2t+1], D[g+8][..]
         //     column n < 4: batch 0 of lane 4g + n; column n >= 4: batch 1 of lane 4g + n - 4
         {
@@ -370,7 +454,19 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
 #pragma unroll
         for (int w = 0; w < W; ++w) total += red[((size_t)w * NB + bb) * ROWS + r];
     }
-    if (KS > 1) {
+    if (KS > 1 && a.cluster) {
+        // K slices of one block are the CTAs of one cluster: rank 0 adds the partial sums of its peers
+        // straight out of their shared memory, in rank order.
+        namespace cg = cooperative_groups;
+        cg::cluster_group cl = cg::this_cluster();
+        if (active) red[t] = total;          // slot t of red is read by thread t only
+        cl.sync();
+        if (ks == 0 && active) {
+            for (int k2 = 1; k2 < KS; ++k2) total += *cl.map_shared_rank(red + t, k2);
+        }
+        cl.sync();                            // peers keep their shared memory alive until rank 0 has read it
+        if (ks != 0) return;
+    } else if (KS > 1) {
         __shared__ int s_last;
         if (active) a.partial[((size_t)ks * NB + bb) * a.rows_ws + row] = total;
         __threadfence();
@@ -391,11 +487,17 @@ __global__ void __launch_bounds__(W * 32, RPL == 2 ? 2 : 1) gemv_pair_kernel(con
         else
             ((float*)a.y)[(size_t)bb * a.rows + row] = total;
     }
+    stamp(a, 6);
 }
 
 // ------------------------------------------------------------------------------------ host side
 
 static int g_pair_ks_override = 0;  // 0 = policy below
+static unsigned long long* g_pair_trace = nullptr;
+static size_t g_pair_trace_calls = 0, g_pair_trace_idx = 0;
+void pair_set_trace(void* p, size_t calls) { g_pair_trace = (unsigned long long*)p; g_pair_trace_calls = calls; g_pair_trace_idx = 0; }
+static int g_pair_dbg = 0;
+void pair_set_debug(int m) { g_pair_dbg = m; }
 static int g_pair_pf_dist = 0;  // L2 prefetch measured slower than none on B200
 
 void pair_set_ksplit_override(int ks) { g_pair_ks_override = ks; }
@@ -403,42 +505,53 @@ void pair_set_prefetch(int d) { g_pair_pf_dist = d; }
 
 struct PairConfig { int rpl, warps, slots; };
 
-static PairConfig pair_config(int bits) {
+static int g_pair_small = 1;   // probe switch: one row per lane for matrices with few row blocks
+void pair_set_small(int v) { g_pair_small = v; }
+
+static PairConfig pair_config(const Layout& l) {
     // N <= 4: two rows per lane, 8 dense warps, two CTAs per SM.  N = 5: the pair table of a row is
-    // 4 KB, so one row per lane (128 KB of tables), 16 dense warps, one CTA per SM.
-    if (bits == 5) return PairConfig{1, 16, 148};
+    // 4 KB, so one row per lane (128 KB of tables), 16 dense warps, one CTA per SM.  Matrices with
+    // fewer 64-row blocks than SMs also take one row per lane: twice the CTAs, no split along K.
+    if (l.bits == 5) return PairConfig{1, 16, 148};
+    if (g_pair_small == 1 && l.RB <= 148 && l.bits >= 3) return PairConfig{1, 16, 148};
+    if (g_pair_small == 2 && l.RB <= 148 && l.bits >= 3 && l.bits <= 4) return PairConfig{1, 8, 148};
     return PairConfig{2, 8, 296};
 }
 
-struct PairSchedule { int blocks, n_full, kst, sc_per_split, grid; };
+struct PairSchedule { int blocks, n_full, kst, sc_per_split, grid, cluster; };
 
 static PairSchedule pair_schedule(const Layout& l) {
-    const PairConfig cfg = pair_config(l.bits);
+    const PairConfig cfg = pair_config(l);
     PairSchedule sc{};
     sc.blocks = (l.RB + cfg.rpl - 1) / cfg.rpl;
     int rem = sc.blocks % cfg.slots;
     int kst = 1;
+    const int kmax = l.SC / 4 > 1 ? l.SC / 4 : 1;   // keep K slices of at least 512 weights
     if (g_pair_ks_override > 0) {
         rem = sc.blocks; kst = g_pair_ks_override;
+    } else if (sc.blocks < cfg.slots) {
+        // fewer blocks than CTA slots: cut every block into 2, 4 or 8 K slices that form a cluster
+        kst = 1;
+        while (kst < 8 && sc.blocks * kst * 2 <= cfg.slots && kst * 2 <= kmax) kst *= 2;
+        sc.cluster = kst > 1;
     } else if (rem > 0) {
-        // cut the blocks of the last, partial round along K so that they fill the idle slots; every cut
-        // costs another fill of the pair tables and a trip through global memory, so keep slices >= 1024
-        kst = (cfg.slots + rem / 2) / rem;
-        const int kmax = l.SC / 8 > 1 ? l.SC / 8 : 1;
+        // blocks of the last, partial round: cut along K so that the pieces fit the slots of one round
+        kst = cfg.slots / rem;
         if (kst > kmax) kst = kmax;
-        if (kst < 1) kst = 1;
+        if (kst > 64) kst = 64;
     }
     if (kst > l.SC) kst = l.SC;
-    if (kst <= 1) { rem = 0; kst = 1; }
+    if (kst <= 1) { rem = 0; kst = 1; sc.cluster = 0; }
     sc.n_full = sc.blocks - rem;
     sc.sc_per_split = (l.SC + kst - 1) / kst;
     sc.kst = (l.SC + sc.sc_per_split - 1) / sc.sc_per_split;
+    if (sc.cluster && (sc.kst & (sc.kst - 1))) sc.cluster = 0;   // cluster sizes are powers of two
     sc.grid = sc.n_full + rem * sc.kst;
     return sc;
 }
 
 static size_t pair_smem_bytes(const Layout& l, int nb) {
-    const PairConfig cfg = pair_config(l.bits);
+    const PairConfig cfg = pair_config(l);
     const int rows = 32 * cfg.rpl;
     const size_t T = (size_t)l.E * l.E;
     return T * 128 * cfg.rpl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4;
@@ -446,7 +559,7 @@ static size_t pair_smem_bytes(const Layout& l, int nb) {
 
 bool pair_supported(const Layout& l, int batch, int n_problems) {
     if (l.mode != 0 || l.bits < 2 || l.bits > 5 || batch > 2 || n_problems != 1) return false;
-    return pair_smem_bytes(l, batch) <= (pair_config(l.bits).rpl == 2 ? 110u : 220u) * 1024u;
+    return pair_smem_bytes(l, batch) <= (pair_config(l).rpl == 2 ? 110u : 220u) * 1024u;
 }
 
 size_t pair_workspace_bytes(const Layout& l) {
@@ -456,6 +569,7 @@ size_t pair_workspace_bytes(const Layout& l) {
 
 template <int N, int NB, int RPL, int W>
 static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+    const int cluster = a.cluster ? a.kst : 1;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gemv_pair_kernel<N, NB, RPL, W>,
@@ -468,29 +582,61 @@ static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaSt
     cfg.blockDim = dim3(W * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = cluster > 1 ? 2 : 1;
+    if (a.dbg == 3) {   // probe: plain stream order
+        attr[0] = attr[1];
+        cfg.numAttrs = cluster > 1 ? 1 : 0;
+    }
     return cudaLaunchKernelEx(&cfg, gemv_pair_kernel<N, NB, RPL, W>, a);
 }
 
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s) {
-    const PairConfig cfg = pair_config(l.bits);
+    const PairConfig cfg = pair_config(l);
     const PairSchedule sch = pair_schedule(l);
     PairArgs a{};
     a.off = offsets_of(l);
     a.packed = c.packed; a.x = c.x; a.y = c.y;
-    a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC;
+    a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
     a.rows_ws = sch.blocks * 32 * cfg.rpl;
     a.n_full = sch.n_full; a.kst = sch.kst; a.sc_per_split = sch.sc_per_split;
     a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
     a.pf_dist = g_pair_pf_dist;
+    a.cluster = sch.cluster && g_pair_ks_override == 0;
+    a.dbg = g_pair_dbg;
+    a.trace = nullptr;
+    if (g_pair_trace && g_pair_trace_idx < g_pair_trace_calls) a.trace = g_pair_trace + (g_pair_trace_idx++) * 1024 * 8;
     a.tickets = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
     const size_t smem = pair_smem_bytes(l, c.batch);
     dim3 grid((unsigned)sch.grid, 1, 1);
+    if (cfg.rpl == 1 && cfg.warps == 8) {
+        switch (l.bits * 10 + c.batch) {
+            case 31: return launch_pair<3, 1, 1, 8>(a, grid, smem, s);
+            case 32: return launch_pair<3, 2, 1, 8>(a, grid, smem, s);
+            case 41: return launch_pair<4, 1, 1, 8>(a, grid, smem, s);
+            case 42: return launch_pair<4, 2, 1, 8>(a, grid, smem, s);
+        }
+        return cudaErrorInvalidValue;
+    }
+    if (cfg.rpl == 1) {
+        switch (l.bits * 10 + c.batch) {
+            case 31: return launch_pair<3, 1, 1, 16>(a, grid, smem, s);
+            case 32: return launch_pair<3, 2, 1, 16>(a, grid, smem, s);
+            case 41: return launch_pair<4, 1, 1, 16>(a, grid, smem, s);
+            case 42: return launch_pair<4, 2, 1, 16>(a, grid, smem, s);
+            case 51: return launch_pair<5, 1, 1, 16>(a, grid, smem, s);
+            case 52: return launch_pair<5, 2, 1, 16>(a, grid, smem, s);
+        }
+        return cudaErrorInvalidValue;
+    }
     switch (l.bits * 10 + c.batch) {
         case 21: return launch_pair<2, 1, 2, 8>(a, grid, smem, s);
         case 22: return launch_pair<2, 2, 2, 8>(a, grid, smem, s);
@@ -498,8 +644,6 @@ cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s)
         case 32: return launch_pair<3, 2, 2, 8>(a, grid, smem, s);
         case 41: return launch_pair<4, 1, 2, 8>(a, grid, smem, s);
         case 42: return launch_pair<4, 2, 2, 8>(a, grid, smem, s);
-        case 51: return launch_pair<5, 1, 1, 16>(a, grid, smem, s);
-        case 52: return launch_pair<5, 2, 1, 16>(a, grid, smem, s);
     }
     return cudaErrorInvalidValue;
 }

@@ -48,6 +48,9 @@ size_t pair_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s);
 void pair_set_ksplit_override(int ks);
 void pair_set_prefetch(int d);
+void pair_set_debug(int m);
+void pair_set_small(int v);
+void pair_set_trace(void* p, size_t calls);
 
 inline size_t workspace_bytes_for(const Layout& l) {
     const size_t g = generic_workspace_bytes(l), p = pair_workspace_bytes(l);

@@ -13,11 +13,12 @@
 //   gsm     V2a: half2 [RB][SC][32]    (scale, mid) of the same group
 //   rowptr  int32 [rows_pad + 1]       clamped to [0, nnz]
 //   oent    u32 [nnz]                  column | fp16 value << 16, CSR order
-//   ellptr  int32 [RB + 1]             start of each row-block's transposed outlier slab, in entries
-//   ell     u32 [ell_cap]              slab of row-block b: slot j of channel b*32+l at ellptr[b] + j*32 + l,
-//                                      width W_b = min(longest row of the block, 2*ceil(nnz_b/32) + 8) slots,
-//                                      unused slots hold column 0 / value +0.  Rows longer than W_b keep their
-//                                      remaining entries in the CSR arrays only (the "spill").
+//   ell     u32 [RB][C + 1][32]        transposed outlier slab of every row-block, C = ell_slots(nnz, rows) slots:
+//                                      word [b][0][l]   = number of slots channel b*32+l uses (min(row length, C)),
+//                                      word [b][1+j][l] = j-th outlier of that channel, or column 0 / value +0.
+//                                      C comes from the descriptor alone (mean row length + 4 sigma + 8), so a slab's
+//                                      address needs no pointer load.  Rows longer than C keep their remaining
+//                                      entries in the CSR arrays only (the "spill").
 #pragma once
 #include <cstddef>
 #include <cstdint>
@@ -31,11 +32,22 @@ struct Layout {
     int mode, rows, cols, bits, L, E;
     int RB, SC, rows_pad;
     long long nnz;
-    size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_oent, off_ellptr, off_ell, total;
-    long long ell_cap;  // entries reserved for the transposed slabs (an upper bound from nnz and RB)
+    size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_oent, off_ell, total;
+    int ell_slots;  // C: slots per channel in the transposed outlier slabs (0 when nnz == 0)
 };
 
 inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+// Slots per channel of the transposed outlier slabs: mean row length m plus four binomial standard
+// deviations plus 8; rows beyond it spill to the CSR arrays.
+inline int ell_slots(long long nnz, int rows) {
+    if (nnz <= 0) return 0;
+    const long long m = (nnz + rows - 1) / rows;
+    long long r = 1;
+    while (r * r < m) ++r;  // ceil(sqrt(m))
+    const long long c = m + 4 * r + 8;
+    return (int)(c > 65535 ? 65535 : c);
+}
 
 inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, long long nnz) {
     Layout l{};
@@ -51,9 +63,8 @@ inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, 
     l.off_gsm = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * 32 * 4 : 0));
     l.off_rowptr = o; o = align256(o + (size_t)(l.rows_pad + 1) * 4);
     l.off_oent = o;   o = align256(o + (size_t)nnz * 4);
-    l.ell_cap = nnz ? 2 * nnz + 320LL * l.RB : 0;
-    l.off_ellptr = o; o = align256(o + (size_t)(l.RB + 1) * 4);
-    l.off_ell = o;    o = align256(o + (size_t)l.ell_cap * 4);
+    l.ell_slots = ell_slots(nnz, rows);
+    l.off_ell = o;    o = align256(o + (l.ell_slots ? (size_t)l.RB * (l.ell_slots + 1) * 32 * 4 : 0));
     l.total = o;
     return l;
 }

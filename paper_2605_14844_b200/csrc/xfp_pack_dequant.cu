@@ -120,59 +120,18 @@ __global__ void pack_entries_kernel(const void* __restrict__ ocol, int col_bits,
     out[p] = (uint32_t)c | (v << 16);
 }
 
-// Width (in slots) of every row-block's transposed outlier slab, from the packed (clamped) row pointers.
-__global__ void ell_width_kernel(const int* __restrict__ rp, int* __restrict__ width, int RB) {
-    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (b >= RB) return;
-    const int p0 = rp[b * 32 + lane], p1 = rp[b * 32 + lane + 1];
-    int len = p1 > p0 ? p1 - p0 : 0;
-#pragma unroll
-    for (int o = 16; o; o >>= 1) len = max(len, __shfl_xor_sync(0xffffffffu, len, o));
-    const int first = rp[b * 32], last = rp[b * 32 + 32];
-    const int nnz_b = last > first ? last - first : 0;
-    const int cap = 2 * ((nnz_b + 31) / 32) + 8;
-    if (lane == 0) width[b] = min(len, cap);
-}
-
-// ellptr[b] = 32 * sum of the widths before b (one CTA, chunked scan: RB is at most a few hundred thousand).
-__global__ void ell_scan_kernel(const int* __restrict__ width, int* __restrict__ ellptr, int RB, long long ell_cap) {
-    const int cap32 = (int)((ell_cap < 0x7fffffe0LL ? ell_cap : 0x7fffffe0LL) & ~31LL);  // slabs never pass the reserved area
-    __shared__ int s_part[1024];
-    __shared__ int s_carry;
-    if (threadIdx.x == 0) s_carry = 0;
-    __syncthreads();
-    for (int base = 0; base < RB; base += 1024) {
-        const int i = base + threadIdx.x;
-        const int v = i < RB ? width[i] * 32 : 0;
-        s_part[threadIdx.x] = v;
-        __syncthreads();
-        for (int o = 1; o < 1024; o <<= 1) {
-            const int t = threadIdx.x >= o ? s_part[threadIdx.x - o] : 0;
-            __syncthreads();
-            s_part[threadIdx.x] += t;
-            __syncthreads();
-        }
-        if (i < RB) ellptr[i] = min(s_carry + s_part[threadIdx.x] - v, cap32);
-        __syncthreads();
-        if (threadIdx.x == 1023) s_carry += s_part[1023];
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) ellptr[RB] = min(s_carry, cap32);
-}
-
-// Slab of row-block b: slot j of channel b*32+lane <- j-th outlier of that row, or the neutral entry.
+// Transposed outlier slab of row-block b (one warp per block): word [0][lane] = slots used by channel
+// b*32+lane, word [1+j][lane] = its j-th outlier or the neutral entry (column 0, value +0).
 __global__ void ell_fill_kernel(const int* __restrict__ rp, const uint32_t* __restrict__ oent,
-                                const int* __restrict__ ellptr, uint32_t* __restrict__ ell, int RB, long long ell_cap) {
+                                uint32_t* __restrict__ ell, int RB, int C) {
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (b >= RB) return;
-    const int e0 = ellptr[b], w = (ellptr[b + 1] - e0) >> 5;
     const int p0 = rp[b * 32 + lane], p1 = rp[b * 32 + lane + 1];
-    for (int j = 0; j < w; ++j) {
-        const long long dst = (long long)e0 + (long long)j * 32 + lane;
-        if (dst < ell_cap) ell[dst] = (p0 + j < p1) ? oent[p0 + j] : 0u;
-    }
+    const int len = p1 > p0 ? min(p1 - p0, C) : 0;
+    uint32_t* slab = ell + (size_t)b * (C + 1) * 32 + lane;
+    slab[0] = (uint32_t)len;
+    for (int j = 0; j < C; ++j) slab[(size_t)(1 + j) * 32] = j < len ? oent[p0 + j] : 0u;
 }
 
 template <int N>
@@ -206,20 +165,13 @@ cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int
     pack_rowptr_kernel<<<(unsigned)((l.rows_pad + 1 + 255) / 256), 256, 0, s>>>(
         l.nnz ? in.rowptr : nullptr, in.ocol, in.col_bits, (int*)(base + l.off_rowptr), l.rows, l.rows_pad, l.nnz,
         err_word);
-    int* ellptr = (int*)(base + l.off_ellptr);
     if (l.nnz) {
         pack_entries_kernel<<<(unsigned)((l.nnz + 255) / 256), 256, 0, s>>>(in.ocol, in.col_bits, in.oval,
                                                                            (uint32_t*)(base + l.off_oent), l.nnz,
                                                                            l.cols, err_word);
-        // transposed slabs: widths are staged in the slab area itself (it is at least RB ints large)
-        int* width = (int*)(base + l.off_ell);
-        const int* rp = (const int*)(base + l.off_rowptr);
-        ell_width_kernel<<<(unsigned)((l.RB + 7) / 8), 256, 0, s>>>(rp, width, l.RB);
-        ell_scan_kernel<<<1, 1024, 0, s>>>(width, ellptr, l.RB, l.ell_cap);
-        ell_fill_kernel<<<(unsigned)((l.RB + 7) / 8), 256, 0, s>>>(rp, (const uint32_t*)(base + l.off_oent), ellptr,
-                                                                   (uint32_t*)(base + l.off_ell), l.RB, l.ell_cap);
-    } else {
-        cudaMemsetAsync(ellptr, 0, (size_t)(l.RB + 1) * 4, s);
+        ell_fill_kernel<<<(unsigned)((l.RB + 7) / 8), 256, 0, s>>>((const int*)(base + l.off_rowptr),
+                                                                   (const uint32_t*)(base + l.off_oent),
+                                                                   (uint32_t*)(base + l.off_ell), l.RB, l.ell_slots);
     }
     return cudaGetLastError();
 }
