@@ -34,9 +34,9 @@ import numpy as np
 ROWS = COLS = 4096
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/ (None until a capture exists for the current kernel)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the two GEMV kernels of this workload, from
+# the ncu captures summarised in profiles/gemv_pair_attention_4096x4096.md (bits -> bytes)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {4: 9634560, 5: 11866624}
 
 
 def block_spec(layer: int):
@@ -215,25 +215,35 @@ def run_xfp(args, rank: int, world: int):
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=stream):
             step()
-        for _ in range(max(args.warmup, 3)):
-            graph.replay()
-        stream.synchronize()
-
         def barrier():
             if dist is not None:
                 dist.barrier()
             torch.cuda.synchronize()
 
+        # the clock sampler needs a moment to come up: warm up until it has delivered a sample (at
+        # least the requested warm-up steps, at most ~2 s), so that the timed region is covered
         sampler = ClockSampler(local)
-        barrier()
         sampler.start()
+        t_w = time.perf_counter()
+        n_warm = 0
+        while n_warm < max(args.warmup, 3) or (len(sampler.rows) < 2 and time.perf_counter() - t_w < 2.0):
+            graph.replay()
+            n_warm += 1
+            if n_warm % 64 == 0:
+                stream.synchronize()
+        stream.synchronize()
+        n_before = len(sampler.rows)
+        barrier()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
         ev[0].record(stream)
         for i in range(args.steps):
             graph.replay()
             ev[i + 1].record(stream)
         barrier()
+        time.sleep(0.12)   # one more sampling period, so a short timed region still sees a sample taken under load
         clocks = sampler.stop()
+        clocks["samples_before_timed_region"] = n_before
+        clocks["warmup_steps_run"] = n_warm
         total_ms = ev[0].elapsed_time(ev[-1])
         per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
 
@@ -272,7 +282,7 @@ def run_xfp(args, rank: int, world: int):
     per_gpu = step_bytes / (ms_per_step * 1e-3) / 1e9
     out = {
         "metric": "fused XFP GEMV effective GB/s at batch 1", "value": value, "unit": "GB/s", "n_gpus": world,
-        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "us_per_call": ms_per_step * 1e3 / n_calls,
         "ms_per_step_median": statistics.median(per_step),
@@ -282,7 +292,7 @@ def run_xfp(args, rank: int, world: int):
                    "126 MB of other weights passed" % (step_bytes / 1e6), "launch": "one CUDA graph per step"},
         "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
                      "peak_kind": peak_kind, "frac_of_nominal_8000": per_gpu / NOMINAL_HBM_GBS,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "bytes_per_launch": step_bytes / n_calls,
+                     "traffic": sum(NCU_TRAFFIC_BYTES_PER_LAUNCH[n[2]] for n in names) / n_calls, "bytes_per_launch": step_bytes / n_calls,
                      "kernel": "gemv (all calls of a step)"},
         "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": n_calls * COLS * 2,
                 "d2h_bytes_per_step": n_calls * ROWS * 2, "us_per_call": e2e_ms / args.steps * 1e3 / n_calls},
@@ -305,7 +315,7 @@ def algorithmic_bytes_from(pm, q) -> int:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="xfp", choices=["xfp", "reference"])
     ap.add_argument("--layers", type=int, default=8)

@@ -34,10 +34,17 @@ def _desc(**kw):
 
 
 def test_packed_size_accounting(lib):
+    import math
     pb, wb = xfp.xfp_packed_size(_desc(rows=4096, cols=4096, nnz=50000))
     idx_bytes = 4096 * 4096 // 2
-    # indices at exactly N bits per weight, codebooks, row pointers, 4 bytes per outlier
-    assert idx_bytes + 4096 * 16 * 2 + 4097 * 4 + 50000 * 4 <= pb <= idx_bytes + 4096 * 16 * 2 + 4097 * 4 + 50000 * 4 + 5 * 256
+    # indices at exactly N bits per weight, codebooks, row pointers, 4 bytes per outlier (CSR), plus the
+    # transposed outlier slabs: per 32-row block (C + 1) slots of 32 words, C = mean + 4 sqrt(mean) + 8
+    m = math.ceil(50000 / 4096)
+    slab = (4096 // 32) * (m + 4 * math.ceil(math.sqrt(m)) + 8 + 1) * 32 * 4
+    base = idx_bytes + 4096 * 16 * 2 + 4097 * 4 + 50000 * 4 + slab
+    assert base <= pb <= base + 6 * 256
+    p0, _ = xfp.xfp_packed_size(_desc(rows=4096, cols=4096, nnz=0))
+    assert p0 <= idx_bytes + 4096 * 16 * 2 + 4097 * 4 + 6 * 256
     for bits in (2, 3, 4, 5, 6):
         pb, _ = xfp.xfp_packed_size(_desc(rows=32, cols=128, bits=bits))
         assert pb >= 32 * 128 * bits // 8
