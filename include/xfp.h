@@ -118,6 +118,28 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
                   int32_t batch, void* y_host, void* y_dev, int32_t y_is_fp16, void* workspace,
                   size_t workspace_bytes, void* stream);
 
+/* xfp_gemv_v2 for callers that cannot allocate device memory.  The paper has no counterpart: this is a
+ * packaging variant of the same GEMV, not another operation.
+ * Who needs it: code that is handed a fixed set of buffers and may not ask the driver for more -- for
+ * instance a plug-in inside a host application that reserved the whole GPU at start-up, or a component
+ * on a latency-critical path where cudaMalloc (which synchronises the device) is forbidden.  Such a
+ * caller cannot supply the split-K workspace xfp_gemv_v2 asks for, so the library keeps one in a
+ * built-in device array of 8 MiB (present on every GPU that loads the library, until the process exits).
+ *   desc, packed, x, batch, y, y_is_fp16, stream: as for xfp_gemv_v2; the caller still owns inputs and outputs.
+ * Limits and behaviour:
+ *   - shapes whose workspace (see xfp_packed_size) exceeds 8 MiB return XFP_ERR_BUFFER_TOO_SMALL;
+ *     roughly: (rows / 32) * min(64, cols / 128) <= 32k, e.g. anything up to 8192 x 8192.
+ *   - the first call on each device looks up the array's device address (once per device, with that
+ *     device current); make that first call before starting any stream capture.
+ *   - no cudaMalloc, cudaFree or other allocating call is made; the only extra work is a small
+ *     cudaMemsetAsync on `stream` that zeroes the workspace counters, because the array keeps the
+ *     previous call's contents.
+ *   - all calls share the one array: two calls that may run at the same time on the GPU (different
+ *     streams, or different host threads without ordering) race on it and give wrong results.  Order
+ *     them on one stream, or use xfp_gemv_v2 with separate workspaces. */
+int xfp_gemv_v2_noalloc(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
+                        int32_t y_is_fp16, void* stream);
+
 const char* xfp_status_str(int status);
 
 #ifdef __cplusplus

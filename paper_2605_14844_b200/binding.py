@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 EXPORTS = ("xfp_packed_size", "xfp_pack", "xfp_gemv_v2", "xfp_gemv_v2a", "xfp_gemv_grouped", "xfp_gemv_host",
-           "xfp_dequant", "xfp_status_str")
+           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc")
 
 
 class XfpError(RuntimeError):
@@ -54,6 +54,7 @@ def load_library() -> C.CDLL:
     lib.xfp_gemv_grouped.argtypes = [dp, i32, vp, vp, vp, i32, vp, sz, vp]
     lib.xfp_gemv_host.argtypes = [dp, vp, vp, vp, i32, vp, vp, i32, vp, sz, vp]
     lib.xfp_dequant.argtypes = [dp, vp, vp, vp]
+    lib.xfp_gemv_v2_noalloc.argtypes = [dp, vp, vp, i32, vp, i32, vp]
     lib.xfp_status_str.argtypes = [C.c_int]
     lib.xfp_status_str.restype = C.c_char_p
     for name in EXPORTS:
@@ -125,6 +126,13 @@ def xfp_gemv_host(desc, packed, x_host: torch.Tensor, x_dev, batch, y_host: torc
                                         _ptr(y_host), _ptr(y_dev), int(bool(y_is_fp16)), _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), _stream(stream)),
            "xfp_gemv_host")
+
+
+def xfp_gemv_v2_noalloc(desc, packed, x, batch, y, y_is_fp16, stream=None) -> None:
+    """V2 GEMV that uses the library's built-in 8 MiB scratch instead of a caller workspace: for callers
+    that are not allowed to allocate device memory.  Calls must not overlap on the GPU (shared scratch)."""
+    _check(load_library().xfp_gemv_v2_noalloc(C.byref(desc), _ptr(packed), _ptr(x), int(batch), _ptr(y),
+                                              int(bool(y_is_fp16)), _stream(stream)), "xfp_gemv_v2_noalloc")
 
 
 def xfp_dequant(desc, packed, W: torch.Tensor, stream=None) -> None:
