@@ -48,7 +48,7 @@ struct Blob {
 };
 
 struct Offsets {
-    size_t idx, cb, gid, gsm, rowptr, oent, ell;
+    size_t idx, cb, gid, gsm, rowptr, hdr, oent, ell;
 };
 
 __host__ __device__ inline Blob blob_at(const void* packed, const Offsets& o) {
@@ -65,7 +65,7 @@ __host__ __device__ inline Blob blob_at(const void* packed, const Offsets& o) {
 }
 
 inline Offsets offsets_of(const Layout& l) {
-    return Offsets{l.off_idx, l.off_cb, l.off_gid, l.off_gsm, l.off_rowptr, l.off_oent, l.off_ell};
+    return Offsets{l.off_idx, l.off_cb, l.off_gid, l.off_gsm, l.off_rowptr, l.off_hdr, l.off_oent, l.off_ell};
 }
 
 }  // namespace xfp

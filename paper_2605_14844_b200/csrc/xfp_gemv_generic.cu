@@ -5,8 +5,12 @@
 //
 //   steps of "Fused Decode Kernel": (1) depack  -> field<N>()
 //                                   (2) codebook gather from shared memory -> tab[]
-//                                   (3) sparse outlier add -> CSR rows of the row-block
+//                                   (3) sparse outlier add -> the row-block's transposed slab, one slot of
+//                                       all 32 channels per coalesced load, each lane adding to its own row
 //                                   (4) multiply-accumulate, fp32
+// Index vectors and V2a group metadata of the next super-chunk are fetched while the current one is
+// decoded.  Weights are loaded before griddepcontrol.wait (programmatic dependent launch); x, y and
+// the workspace are touched after it.
 #include "xfp_internal.h"
 
 namespace xfp {
@@ -26,7 +30,7 @@ struct GenericArgs {
     float* partial;  // [problem][KS][BT][rows_pad]
     int* tickets;    // [problem][RB]
     int rows, cols, RB, SC, rows_pad;
-    int KS, sc_per_split, nb, y_is_fp16, L, rep;
+    int KS, sc_per_split, nb, y_is_fp16, L, rep, ell_slots;
 };
 
 template <int N, int MODE, int BT>
@@ -35,6 +39,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rb = blockIdx.x, ks = blockIdx.y, prob = blockIdx.z;
+    asm volatile("griddepcontrol.launch_dependents;");
     const void* packed = a.packed_list ? a.packed_list[prob] : a.packed;
     const uint16_t* x = a.x_list ? a.x_list[prob] : a.x;
     void* y = a.y_list ? a.y_list[prob] : a.y;
@@ -49,7 +54,48 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
     float* xs = tab + tab_floats;                   // [BT][kseg]
     float* xg = xs + BT * kseg;                     // [BT][sc_per_split]   (V2a group sums of x)
     float* red = xg + BT * a.sc_per_split;          // [warps][BT][32]
-    float* osum = red + kGenericWarps * BT * 32;    // [BT][32]
+
+    // ---- start streaming: first super-chunk of this warp, its group metadata, first outlier slots
+    uint32_t cur[4 * N + 1], nxt[4 * N + 1];
+    cur[4 * N] = nxt[4 * N] = 0u;
+    const uint4* ibase = b.idx + ((size_t)(rb * a.SC + sc0) * N) * 32 + lane;
+    uint32_t gid_c = 0, gsm_c = 0, gid_n = 0, gsm_n = 0;
+    if (warp < nsc) {
+#pragma unroll
+        for (int v = 0; v < N; ++v) {
+            const uint4 t = ld_stream(ibase + ((size_t)warp * N + v) * 32);
+            cur[4 * v] = t.x; cur[4 * v + 1] = t.y; cur[4 * v + 2] = t.z; cur[4 * v + 3] = t.w;
+        }
+        if (MODE == 1) {
+            const size_t unit = (size_t)(rb * a.SC + sc0 + warp) * 32 + lane;
+            gid_c = b.gid[unit];
+            gsm_c = b.gsm[unit];
+        }
+    }
+    // outlier slab of this row-block: slots gw, gw + stride, ... belong to this warp (first round fetched
+    // before the rows' lengths are known: every slot below the capacity is readable)
+    constexpr int kSlots = 4;
+    const int gw = ks * kGenericWarps + warp, ostride = a.KS * kGenericWarps;
+    // launches over several blobs read the slab geometry from each blob (their outlier counts differ)
+    int ell_slots = a.ell_slots;
+    const uint32_t* ell = b.ell;
+    if (a.packed_list) {
+        const int* hdr = (const int*)((const char*)packed + a.off.hdr);
+        ell_slots = __ldg(hdr);
+        ell = (const uint32_t*)((const char*)packed + *(const long long*)(hdr + 2));
+    }
+    const uint32_t* slab = ell + (size_t)rb * (ell_slots + 1) * 32 + lane;
+    const uint32_t olen = ell_slots ? __ldg(slab) : 0u;
+    uint32_t oe[kSlots];
+    int width = ell_slots, oround = 0, nrounds = 0;
+    auto fetch_slots = [&](int round) {
+#pragma unroll
+        for (int q = 0; q < kSlots; ++q) {
+            const int j = gw + (round * kSlots + q) * ostride;
+            oe[q] = j < width ? __ldg(slab + (size_t)(1 + j) * 32) : 0u;
+        }
+    };
+    if (ell_slots) fetch_slots(0);
 
     // ---- stage the codebook (per-lane bank) or the library
     if (MODE == 0) {
@@ -60,14 +106,14 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
     } else {
         for (int t = threadIdx.x; t < tab_floats; t += kGenericThreads) tab[t] = h2f(b.cb[a.rep == 32 ? (t >> 5) : t]);
     }
-    // ---- stage this split's slice of x as fp32
+    // ---- x may come from the previous kernel: stage this split's slice as fp32
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int t = threadIdx.x; t < BT * kseg; t += kGenericThreads) {
         const int bb = t / kseg, kk = t - bb * kseg;
         float v = 0.f;
         if (bb < a.nb && kk < nsc * kSuper) v = h2f(x[(size_t)bb * a.cols + (size_t)sc0 * kSuper + kk]);
         xs[t] = v;
     }
-    for (int t = threadIdx.x; t < BT * 32; t += kGenericThreads) osum[t] = 0.f;
     __syncthreads();
     if (MODE == 1) {
         for (int u = warp; u < BT * nsc; u += kGenericWarps) {
@@ -78,51 +124,35 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
             for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
             if (lane == 0) xg[bb * a.sc_per_split + s] = t;
         }
+        __syncthreads();  // xg visible to every warp
     }
 
-    // ---- outliers of this row-block (first split only): a warp per row, lanes stride the row
-    if (ks == 0) {
-        for (int r = warp; r < 32; r += kGenericWarps) {
-            const int row = rb * kRowsPerBlock + r;
-            const int p0 = b.rowptr[row], p1 = b.rowptr[row + 1];
-            if (p1 <= p0) continue;
-            float oa[BT];
-#pragma unroll
-            for (int bb = 0; bb < BT; ++bb) oa[bb] = 0.f;
-            for (int p = p0 + lane; p < p1; p += 32) {
-                const uint32_t e = __ldg(b.oent + p);
-                const float v = h2f((uint16_t)(e >> 16));
-                const uint32_t col = e & 0xffffu;
-#pragma unroll
-                for (int bb = 0; bb < BT; ++bb)
-                    if (bb < a.nb) oa[bb] = fmaf(v, h2f(__ldg(x + (size_t)bb * a.cols + col)), oa[bb]);
-            }
-#pragma unroll
-            for (int bb = 0; bb < BT; ++bb) {
-                float t = oa[bb];
-#pragma unroll
-                for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-                if (lane == 0) osum[bb * 32 + r] = t;
-            }
-        }
-    }
-    if (MODE == 1) __syncthreads();  // xg visible to every warp
-
-    // ---- dense part
     float acc[BT];
 #pragma unroll
     for (int bb = 0; bb < BT; ++bb) acc[bb] = 0.f;
 
-    uint32_t cur[4 * N + 1], nxt[4 * N + 1];
-    cur[4 * N] = nxt[4 * N] = 0u;
-    const uint4* ibase = b.idx + ((size_t)(rb * a.SC + sc0) * N) * 32 + lane;
-    if (warp < nsc) {
+    // ---- outliers: every lane adds the slots of its own channel (x gathered from global memory:
+    //      the staged copy only covers this split's slice of K)
+    {
+        int wmax = (int)olen;
 #pragma unroll
-        for (int v = 0; v < N; ++v) {
-            const uint4 t = ld_stream(ibase + ((size_t)warp * N + v) * 32);
-            cur[4 * v] = t.x; cur[4 * v + 1] = t.y; cur[4 * v + 2] = t.z; cur[4 * v + 3] = t.w;
-        }
+        for (int o = 16; o; o >>= 1) wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
+        width = min(wmax, ell_slots);
+        const int mine = width > gw ? (width - gw + ostride - 1) / ostride : 0;
+        nrounds = (mine + kSlots - 1) / kSlots;
     }
+    auto consume_slots = [&]() {
+#pragma unroll
+        for (int q = 0; q < kSlots; ++q) {
+            const float v = h2f((uint16_t)(oe[q] >> 16));
+            const uint32_t col = oe[q] & 0xffffu;
+#pragma unroll
+            for (int bb = 0; bb < BT; ++bb)
+                if (bb < a.nb) acc[bb] = fmaf(v, h2f(__ldg(x + (size_t)bb * a.cols + col)), acc[bb]);
+        }
+    };
+
+    // ---- dense part
 #pragma unroll 1
     for (int s = warp; s < nsc; s += kGenericWarps) {
         const int sn = s + kGenericWarps;
@@ -132,6 +162,15 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
                 const uint4 t = ld_stream(ibase + ((size_t)sn * N + v) * 32);
                 nxt[4 * v] = t.x; nxt[4 * v + 1] = t.y; nxt[4 * v + 2] = t.z; nxt[4 * v + 3] = t.w;
             }
+            if (MODE == 1) {
+                const size_t unit_n = (size_t)(rb * a.SC + sc0 + sn) * 32 + lane;
+                gid_n = b.gid[unit_n];
+                gsm_n = b.gsm[unit_n];
+            }
+        }
+        if (oround < nrounds) {
+            consume_slots();
+            if (++oround < nrounds) fetch_slots(oround);
         }
         const float* xrow = xs + s * kSuper;
         if (MODE == 0) {
@@ -153,9 +192,8 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
                 }
             }
         } else {
-            const size_t unit = (size_t)(rb * a.SC + sc0 + s) * 32 + lane;
-            const uint32_t id = b.gid[unit];
-            const uint32_t sm = b.gsm[unit];
+            const uint32_t id = gid_c;
+            const uint32_t sm = gsm_c;
             const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
             const float* t = tab + (size_t)id * E * a.rep + (a.rep == 32 ? lane : 0);
             float gs[BT];
@@ -185,6 +223,24 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
         }
 #pragma unroll
         for (int i = 0; i < 4 * N; ++i) cur[i] = nxt[i];
+        gid_c = gid_n;
+        gsm_c = gsm_n;
+    }
+    while (oround < nrounds) {   // more outlier rounds than super-chunks
+        consume_slots();
+        if (++oround < nrounds) fetch_slots(oround);
+    }
+    // rows that fill their slab may continue in the CSR arrays (pathological skew): warp 0 of the first split
+    if (warp == 0 && ks == 0 && ell_slots && (int)olen >= ell_slots) {
+        const int row = rb * kRowsPerBlock + lane;
+        const int p1 = __ldg(b.rowptr + row + 1);
+        for (int p = __ldg(b.rowptr + row) + ell_slots; p < p1; ++p) {
+            const uint32_t e = __ldg(b.oent + p);
+#pragma unroll
+            for (int bb = 0; bb < BT; ++bb)
+                if (bb < a.nb)
+                    acc[bb] = fmaf(h2f((uint16_t)(e >> 16)), h2f(__ldg(x + (size_t)bb * a.cols + (e & 0xffffu))), acc[bb]);
+        }
     }
 
     // ---- fixed-order reduction over the CTA's warps, then over the K splits
@@ -196,7 +252,6 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
     const int row = rb * kRowsPerBlock + l;
     float total = 0.f;
     if (t < BT * 32) {
-        total = osum[bb * 32 + l];
 #pragma unroll
         for (int w = 0; w < kGenericWarps; ++w) total += red[(w * BT + bb) * 32 + l];
     }
@@ -262,8 +317,17 @@ static cudaError_t launch_one(const GenericArgs& a, dim3 grid, size_t smem, cuda
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    gemv_generic_kernel<N, MODE, BT><<<grid, kGenericThreads, smem, s>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kGenericThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_generic_kernel<N, MODE, BT>, a);
 }
 
 template <int N, int MODE>
@@ -303,7 +367,7 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
         const int ks = generic_ksplit(l, bt);
         a.sc_per_split = (l.SC + ks - 1) / ks;
         a.KS = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
-        a.nb = nb; a.y_is_fp16 = c.y_is_fp16; a.L = l.L;
+        a.nb = nb; a.y_is_fp16 = c.y_is_fp16; a.L = l.L; a.ell_slots = l.ell_slots;
         // V2a: a per-bank copy of the library when it fits, else a single copy (bank conflicts)
         a.rep = (l.mode && (size_t)l.L * l.E * 32 * 4 <= 128 * 1024) ? 32 : 1;
         // grouped calls stride the workspace by the per-problem size the caller was told
@@ -312,7 +376,7 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
         (void)per_problem;
         const size_t tab = l.mode ? (size_t)l.L * l.E * a.rep : (size_t)l.E * 32;
         const size_t smem = 4 * (tab + (size_t)bt * a.sc_per_split * kSuper + (size_t)bt * a.sc_per_split +
-                                 (size_t)kGenericWarps * bt * 32 + (size_t)bt * 32);
+                                 (size_t)kGenericWarps * bt * 32);
         dim3 grid((unsigned)l.RB, (unsigned)a.KS, (unsigned)c.n);
         cudaError_t e = l.mode ? launch_n<1>(l.bits, bt, a, grid, smem, s) : launch_n<0>(l.bits, bt, a, grid, smem, s);
         if (e != cudaSuccess) return e;

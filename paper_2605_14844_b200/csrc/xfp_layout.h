@@ -12,6 +12,9 @@
 //   gid     V2a: u8  [RB][SC][32]      library id of (channel rb*32+l, group sc)
 //   gsm     V2a: half2 [RB][SC][32]    (scale, mid) of the same group
 //   rowptr  int32 [rows_pad + 1]       clamped to [0, nnz]
+//   hdr     256 bytes                  {int32 ell_slots, int32 0, int64 off_ell}: the two values of this layout that
+//                                      depend on nnz, for launches over several blobs of one shape whose outlier
+//                                      counts differ (everything before hdr is independent of nnz)
 //   oent    u32 [nnz]                  column | fp16 value << 16, CSR order
 //   ell     u32 [RB][C + 1][32]        transposed outlier slab of every row-block, C = ell_slots(nnz, rows) slots:
 //                                      word [b][0][l]   = number of slots channel b*32+l uses (min(row length, C)),
@@ -32,7 +35,7 @@ struct Layout {
     int mode, rows, cols, bits, L, E;
     int RB, SC, rows_pad;
     long long nnz;
-    size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_oent, off_ell, total;
+    size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_hdr, off_oent, off_ell, total;
     int ell_slots;  // C: slots per channel in the transposed outlier slabs (0 when nnz == 0)
 };
 
@@ -62,6 +65,7 @@ inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, 
     l.off_gid = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * 32 : 0));
     l.off_gsm = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * 32 * 4 : 0));
     l.off_rowptr = o; o = align256(o + (size_t)(l.rows_pad + 1) * 4);
+    l.off_hdr = o;    o = align256(o + 256);
     l.off_oent = o;   o = align256(o + (size_t)nnz * 4);
     l.ell_slots = ell_slots(nnz, rows);
     l.off_ell = o;    o = align256(o + (l.ell_slots ? (size_t)l.RB * (l.ell_slots + 1) * 32 * 4 : 0));

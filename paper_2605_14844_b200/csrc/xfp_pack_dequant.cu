@@ -134,6 +134,14 @@ __global__ void ell_fill_kernel(const int* __restrict__ rp, const uint32_t* __re
     for (int j = 0; j < C; ++j) slab[(size_t)(1 + j) * 32] = j < len ? oent[p0 + j] : 0u;
 }
 
+__global__ void pack_header_kernel(int* hdr, int ell_slots, long long off_ell) {
+    if (threadIdx.x == 0) {
+        hdr[0] = ell_slots;
+        hdr[1] = 0;
+        *(long long*)(hdr + 2) = off_ell;
+    }
+}
+
 template <int N>
 static void launch_pack_idx(const Layout& l, const uint8_t* idx, uint4* out, int* err, cudaStream_t s) {
     const long long units = (long long)l.RB * l.SC;
@@ -165,6 +173,7 @@ cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int
     pack_rowptr_kernel<<<(unsigned)((l.rows_pad + 1 + 255) / 256), 256, 0, s>>>(
         l.nnz ? in.rowptr : nullptr, in.ocol, in.col_bits, (int*)(base + l.off_rowptr), l.rows, l.rows_pad, l.nnz,
         err_word);
+    pack_header_kernel<<<1, 32, 0, s>>>((int*)(base + l.off_hdr), l.ell_slots, (long long)l.off_ell);
     if (l.nnz) {
         pack_entries_kernel<<<(unsigned)((l.nnz + 255) / 256), 256, 0, s>>>(in.ocol, in.col_bits, in.oval,
                                                                            (uint32_t*)(base + l.off_oent), l.nnz,

@@ -161,8 +161,10 @@ def test_grouped_matches_single_calls():
     pms = [xfp.pack_tensors(q, col_bits=16) for q in qs]
     xs = [_x_dev(synth.activations(1, cols, seed=800 + j)) for j in range(n)]
     ys = torch.zeros((n, rows), dtype=torch.float32, device="cuda")
-    desc = pms[0].desc
-    desc.nnz = max(p.desc.nnz for p in pms)
+    d0 = pms[0].desc
+    # one descriptor for the group: same shape and mode; nnz = the largest count of the group
+    desc = xfp.XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                       max(p.desc.nnz for p in pms))
     _, wb = xfp.xfp_packed_size(desc)
     ws = torch.zeros(n * wb, dtype=torch.uint8, device="cuda")
     ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
