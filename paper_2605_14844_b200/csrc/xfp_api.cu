@@ -45,9 +45,13 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     if (c.workspace_bytes < need) return XFP_ERR_BUFFER_TOO_SMALL;
     GemvCall cc = c;
     cc.workspace_bytes = need;
-    const cudaError_t e = pair_supported(l, c.batch, c.n) && !c.packed_list
-                              ? launch_gemv_pair(l, cc, (cudaStream_t)stream)
-                              : launch_gemv_generic(l, cc, (cudaStream_t)stream);
+    cudaError_t e;
+    if (pair_supported(l, c.batch, c.n) && !c.packed_list)
+        e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
+    else if (v2a_supported(l, c.batch))
+        e = launch_gemv_v2a(l, cc, (cudaStream_t)stream);
+    else
+        e = launch_gemv_generic(l, cc, (cudaStream_t)stream);
     return e == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 

@@ -1,0 +1,445 @@
+// Fast fused decode GEMV for V2a blobs (shared codebook library) at batch <= 2:
+//     y_i = sum_g [ scale_ig * sum_{k in g} lib[id_ig][q_ik] x_k  +  mid_ig * sum_{k in g} x_k ]  +  (S x)_i
+// ("V2a: Shared Codebook Library").  One launch serves one blob or the n blobs of a routed-MoE layer
+// (blockIdx.y = blob).
+//
+// Mapping.  As in the V2 kernel a CTA owns 64 output channels, each lane of a warp two of them
+// (lane, lane+32), and the warps share K in super-chunks of 128 weights -- which are exactly the
+// format's 128-weight groups, so a lane meets one (id, scale, mid) triple per channel and
+// super-chunk.
+//
+// Look-up.  Every lane may need a different library entry, so a pair table per entry does not fit
+// (L * 4^N * 32 banks).  Instead the library itself is replicated once per bank: word
+// (id * 2^N + q) * 32 + lane holds lib[id][q] (fp16 in the low half).  Lane l only touches bank l, so
+// look-ups are conflict free for any mix of ids; one look-up decodes one weight and a PRMT joins two
+// of them into the half2 the tensor pipe wants.
+//
+// Multiply-accumulate.  The half2 of a lane's two channels form the A fragment of
+// mma.sync.m16n8k16 and x sits on the diagonal lanes of the B fragment (see xfp_gemv_pair.cu).  The
+// fragment accumulates sum lib*x of ONE group; after the group's 32 mma the sums are moved to the
+// lanes that own the channels (two shuffles per channel) and folded into an fp32 accumulator with the
+// group's scale and mid-point: acc += scale * G + mid * X_g, X_g = sum of x over the group, computed
+// once per CTA.  Products of fp16 numbers are exact in fp32; nothing is rounded to fp16 on the way.
+//
+// Outliers, schedule, launch overlap: as in the V2 kernel (transposed slabs consumed by the lanes that
+// own the rows; whole-K blocks first, the last partial round cut along K with a fixed-order finish
+// through the workspace; weights before griddepcontrol.wait, x/y/workspace after it).
+#include "xfp_internal.h"
+
+namespace xfp {
+
+constexpr int kAWarps = 8;
+constexpr int kAThreads = kAWarps * 32;
+constexpr int kARows = 64;
+constexpr int kASlots = 4;
+
+struct V2aArgs {
+    Offsets off;
+    const void* packed;
+    const uint16_t* x;
+    void* y;
+    const void* const* packed_list;
+    const uint16_t* const* x_list;
+    void* const* y_list;
+    float* partial;  // [blob][KS][NB][rows_ws]
+    int* tickets;    // [blob][blocks]
+    int rows, cols, RB, SC, rows_ws, ell_slots, L;
+    int nb, y_is_fp16;
+    int blocks, n_full, kst, sc_per_split;
+};
+
+__device__ __forceinline__ void mma16816a(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Byte offset (q << 7) of index j (compile time) of a 128-weight stream, merged with `base`
+// (= id * 2^N * 128 + lane * 4; the q field occupies bits 7 .. 7+N, which base leaves clear).
+template <int N>
+__device__ __forceinline__ uint32_t entry_addr(const uint32_t* w, int j, uint32_t base) {
+    constexpr uint32_t mask = ((1u << N) - 1u) << 7;
+    const int bit = j * N, wi = bit >> 5, off = bit & 31;
+    uint32_t v;
+    if (off + N > 32)
+        v = __funnelshift_r(w[wi], w[wi + 1], off) << 7;
+    else if (off >= 7)
+        v = w[wi] >> (off - 7);
+    else
+        v = w[wi] << (7 - off);
+    return (v & mask) | base;
+}
+
+template <int N, int NB>
+__global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a) {
+    constexpr int E = 1 << N;
+    extern __shared__ __align__(16) unsigned char smem[];
+    // [library L*E*128 bytes | x fp16 [NB][K] | xg fp32 [NB][SC] | red fp32 [W][NB][64]]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.launch_dependents;");
+    const int prob = blockIdx.y;
+    int blk, ks, KS, spp;
+    if ((int)blockIdx.x < a.n_full) {
+        blk = blockIdx.x; ks = 0; KS = 1; spp = a.SC;
+    } else {
+        const int t = blockIdx.x - a.n_full;
+        blk = a.n_full + t / a.kst; ks = t % a.kst; KS = a.kst; spp = a.sc_per_split;
+    }
+    const void* packed = a.packed_list ? a.packed_list[prob] : a.packed;
+    const uint16_t* x = a.x_list ? a.x_list[prob] : a.x;
+    void* y = a.y_list ? a.y_list[prob] : a.y;
+    const Blob b = blob_at(packed, a.off);
+    const int sc0 = ks * spp;
+    const int nsc = max(0, min(a.SC, sc0 + spp) - sc0);
+    const int K = a.SC * kSuper;
+    const int tab_bytes = a.L * E * 128;
+
+    unsigned char* tab = smem;
+    uint16_t* xs = (uint16_t*)(smem + tab_bytes);             // [NB][K]
+    float* xg = (float*)(xs + (size_t)NB * K);                // [NB][SC]
+    float* red = xg + NB * a.SC;                              // [W][NB][64]
+
+    const int blk0 = 2 * blk;
+    const int blk1 = min(2 * blk + 1, a.RB - 1);              // clamped when RB is odd; its results are dropped
+
+    // ---- (0) start streaming: first super-chunk of this warp (indices and group metadata of both channels)
+    uint32_t w0[4 * N + 1], w1[4 * N + 1];
+    w0[4 * N] = w1[4 * N] = 0u;
+    const uint4* i0 = b.idx + ((size_t)(blk0 * a.SC + sc0) * N) * 32 + lane;
+    const uint4* i1 = b.idx + ((size_t)(blk1 * a.SC + sc0) * N) * 32 + lane;
+    const size_t m0 = (size_t)(blk0 * a.SC + sc0) * 32 + lane, m1 = (size_t)(blk1 * a.SC + sc0) * 32 + lane;
+    uint32_t id0 = 0, id1 = 0, sm0 = 0, sm1 = 0;              // current group: library ids and (scale, mid)
+    uint32_t nid0 = 0, nid1 = 0, nsm0 = 0, nsm1 = 0;          // next group
+    if (warp < nsc) {
+#pragma unroll
+        for (int v = 0; v < N; ++v) {
+            const uint4 t0 = ld_stream(i0 + ((size_t)warp * N + v) * 32);
+            const uint4 t1 = ld_stream(i1 + ((size_t)warp * N + v) * 32);
+            w0[4 * v] = t0.x; w0[4 * v + 1] = t0.y; w0[4 * v + 2] = t0.z; w0[4 * v + 3] = t0.w;
+            w1[4 * v] = t1.x; w1[4 * v + 1] = t1.y; w1[4 * v + 2] = t1.z; w1[4 * v + 3] = t1.w;
+        }
+        id0 = b.gid[m0 + (size_t)warp * 32]; id1 = b.gid[m1 + (size_t)warp * 32];
+        sm0 = b.gsm[m0 + (size_t)warp * 32]; sm1 = b.gsm[m1 + (size_t)warp * 32];
+    }
+    // outlier slabs of this CTA's two row-blocks: slots gw, gw + stride, ... belong to this warp.  Launches
+    // over several blobs read the slab geometry from each blob (their outlier counts differ).
+    int ell_slots = a.ell_slots;
+    const uint32_t* ell = b.ell;
+    if (a.packed_list) {
+        const int* hdr = (const int*)((const char*)packed + a.off.hdr);
+        ell_slots = __ldg(hdr);
+        ell = (const uint32_t*)((const char*)packed + *(const long long*)(hdr + 2));
+    }
+    const int gw = ks * kAWarps + warp, ostride = KS * kAWarps;
+    const uint32_t* slab[2];
+    uint32_t olen[2];
+    uint32_t oe[2][kASlots];
+    int width[2];
+    float acc[NB][2];
+    int oround = 0, nrounds = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        slab[h] = ell + (size_t)(h ? blk1 : blk0) * (ell_slots + 1) * 32 + lane;
+        width[h] = ell_slots;
+        olen[h] = ell_slots ? __ldg(slab[h]) : 0u;
+#pragma unroll
+        for (int bb = 0; bb < NB; ++bb) acc[bb][h] = 0.f;
+    }
+    auto fetch_slots = [&](int round) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int q = 0; q < kASlots; ++q) {
+                const int j = gw + (round * kASlots + q) * ostride;
+                oe[h][q] = j < width[h] ? __ldg(slab[h] + (size_t)(1 + j) * 32) : 0u;
+            }
+    };
+    auto consume_slots = [&]() {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int q = 0; q < kASlots; ++q) {
+                const float v = h2f((uint16_t)(oe[h][q] >> 16));
+                const uint32_t col = oe[h][q] & 0xffffu;
+#pragma unroll
+                for (int bb = 0; bb < NB; ++bb) acc[bb][h] = fmaf(v, h2f(xs[(size_t)bb * K + col]), acc[bb][h]);
+            }
+    };
+    if (ell_slots) fetch_slots(0);
+
+    // ---- (1) library, one copy per bank: word (e * 32 + lane) = lib[e] for every lane
+    for (int e = warp; e < a.L * E; e += kAWarps)
+        *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+
+    // ---- (2) x: wait for the previous kernel, stage fp16 x (all of K) and the group sums X_g
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    {
+        const int nvec = NB * (K / 8);
+        for (int t = threadIdx.x; t < nvec; t += kAThreads) {
+            const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (bb < a.nb) v = __ldg((const uint4*)(x + (size_t)bb * a.cols + kk));
+            *(uint4*)(xs + (size_t)t * 8) = v;
+        }
+    }
+    __syncthreads();
+    for (int u = warp; u < NB * a.SC; u += kAWarps) {   // X_g: 128 values per group, 4 per lane, fixed butterfly
+        const uint2 hv = *(const uint2*)(xs + (size_t)u * kSuper + lane * 4);
+        const float2 p0 = __half22float2(*(const __half2*)&hv.x), p1 = __half22float2(*(const __half2*)&hv.y);
+        float t = (p0.x + p0.y) + (p1.x + p1.y);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0) xg[u] = t;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {   // the rows' slot counts have arrived: this warp's number of outlier rounds
+        int wmax = (int)olen[h];
+#pragma unroll
+        for (int o = 16; o; o >>= 1) wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
+        width[h] = min(wmax, ell_slots);
+        const int mine = width[h] > gw ? (width[h] - gw + ostride - 1) / ostride : 0;
+        nrounds = max(nrounds, (mine + kASlots - 1) / kASlots);
+    }
+
+    // ---- (3) main loop over this warp's groups
+    const int g = lane >> 2, t4 = lane & 3;
+    const bool diag0 = (g == t4);
+    const bool diag1 = (NB > 1) && (g == t4 + 4);
+    const bool diag = diag0 || diag1;
+    const unsigned char* xrow = (const unsigned char*)xs + (diag1 ? (size_t)K * 2 : 0) + (size_t)sc0 * (kSuper * 2);
+    // where this lane's own sums land: D[g][t] sits in lane (g, t >> 1), register t & 1 (batch row 0), and in
+    // lane (g, 2 + (t >> 1)) for batch row 1
+    const int src0 = (lane & ~3) | (t4 >> 1);
+    const bool odd = t4 & 1;
+
+    auto lookup = [&](uint32_t (&f)[4], int m, uint32_t base0, uint32_t base1) {
+        const uint32_t l00 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 0, base0));
+        const uint32_t l01 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 1, base0));
+        const uint32_t l02 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 2, base0));
+        const uint32_t l03 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 3, base0));
+        const uint32_t l10 = *(const uint32_t*)(tab + entry_addr<N>(w1, 4 * m + 0, base1));
+        const uint32_t l11 = *(const uint32_t*)(tab + entry_addr<N>(w1, 4 * m + 1, base1));
+        const uint32_t l12 = *(const uint32_t*)(tab + entry_addr<N>(w1, 4 * m + 2, base1));
+        const uint32_t l13 = *(const uint32_t*)(tab + entry_addr<N>(w1, 4 * m + 3, base1));
+        f[0] = __byte_perm(l00, l01, 0x5410);   // (k, k+1) of channel 0
+        f[1] = __byte_perm(l10, l11, 0x5410);   // (k, k+1) of channel 1
+        f[2] = __byte_perm(l02, l03, 0x5410);   // (k+2, k+3) of channel 0
+        f[3] = __byte_perm(l12, l13, 0x5410);   // (k+2, k+3) of channel 1
+    };
+
+#pragma unroll 1
+    for (int s = warp; s < nsc; s += kAWarps) {
+        const int sn = s + kAWarps;
+        const bool has_next = sn < nsc;
+        if (has_next) {   // metadata of the next group travels during this one
+            nid0 = b.gid[m0 + (size_t)sn * 32]; nid1 = b.gid[m1 + (size_t)sn * 32];
+            nsm0 = b.gsm[m0 + (size_t)sn * 32]; nsm1 = b.gsm[m1 + (size_t)sn * 32];
+        }
+        if (oround < nrounds) {
+            consume_slots();
+            if (++oround < nrounds) fetch_slots(oround);
+        }
+        const uint32_t base0 = id0 * (uint32_t)(E * 128) + (uint32_t)lane * 4u;
+        const uint32_t base1 = id1 * (uint32_t)(E * 128) + (uint32_t)lane * 4u;
+        const unsigned char* xp = xrow + (size_t)s * (kSuper * 2);
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t fa[4], fb[4];
+        uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = make_uint4(0u, 0u, 0u, 0u);
+        if (diag) xa = *(const uint4*)xp;
+        lookup(fa, 0, base0, base1);
+        auto reload = [&](int gi) {   // index vectors are reloaded for the next group once fully consumed
+#pragma unroll
+            for (int v = 0; v < N; ++v) {
+                const int jlast = (128 * (v + 1) + N - 1) / N - 1;   // last index touching vector v
+                if (jlast / 4 == gi && has_next) {
+                    const uint4 t0 = ld_stream(i0 + ((size_t)sn * N + v) * 32);
+                    const uint4 t1 = ld_stream(i1 + ((size_t)sn * N + v) * 32);
+                    w0[4 * v] = t0.x; w0[4 * v + 1] = t0.y; w0[4 * v + 2] = t0.z; w0[4 * v + 3] = t0.w;
+                    w1[4 * v] = t1.x; w1[4 * v + 1] = t1.y; w1[4 * v + 2] = t1.z; w1[4 * v + 3] = t1.w;
+                }
+            }
+        };
+#pragma unroll
+        for (int m = 0; m < kSuper / 4; m += 4) {   // one mma per 4 consecutive k, look-ups one mma ahead
+            if (diag) xb = *(const uint4*)(xp + (m + 2) * 8);
+            lookup(fb, m + 1, base0, base1);
+            reload(m + 1);
+            mma16816a(c0, fa[0], fa[1], fa[2], fa[3], xa.x, xa.y);
+            lookup(fa, m + 2, base0, base1);
+            reload(m + 2);
+            mma16816a(c1, fb[0], fb[1], fb[2], fb[3], xa.z, xa.w);
+            if (m + 4 < kSuper / 4) { if (diag) xa = *(const uint4*)(xp + (m + 4) * 8); }
+            lookup(fb, m + 3, base0, base1);
+            reload(m + 3);
+            mma16816a(c0, fa[0], fa[1], fa[2], fa[3], xb.x, xb.y);
+            if (m + 4 < kSuper / 4) {
+                lookup(fa, m + 4, base0, base1);
+                reload(m + 4);
+            }
+            mma16816a(c1, fb[0], fb[1], fb[2], fb[3], xb.z, xb.w);
+        }
+        // group sums to their owners, then  acc += scale * G + mid * X_g
+        const float d0 = c0[0] + c1[0], d1 = c0[1] + c1[1], d2 = c0[2] + c1[2], d3 = c0[3] + c1[3];
+#pragma unroll
+        for (int bb = 0; bb < NB; ++bb) {
+            const int src = src0 + 2 * bb;
+            const float e0 = __shfl_sync(0xffffffffu, d0, src), e1 = __shfl_sync(0xffffffffu, d1, src);
+            const float e2 = __shfl_sync(0xffffffffu, d2, src), e3 = __shfl_sync(0xffffffffu, d3, src);
+            const float G0 = odd ? e1 : e0, G1 = odd ? e3 : e2;
+            const float X = xg[bb * a.SC + sc0 + s];
+            acc[bb][0] = fmaf(h2f((uint16_t)(sm0 & 0xffffu)), G0, fmaf(h2f((uint16_t)(sm0 >> 16)), X, acc[bb][0]));
+            acc[bb][1] = fmaf(h2f((uint16_t)(sm1 & 0xffffu)), G1, fmaf(h2f((uint16_t)(sm1 >> 16)), X, acc[bb][1]));
+        }
+        id0 = nid0; id1 = nid1; sm0 = nsm0; sm1 = nsm1;
+    }
+    while (oround < nrounds) {   // more outlier rounds than groups
+        consume_slots();
+        if (++oround < nrounds) fetch_slots(oround);
+    }
+    if (warp == 0 && ks == 0 && ell_slots) {   // rows that overflow their slab finish from the CSR arrays
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if ((int)olen[h] >= ell_slots) {
+                const int row = (h ? blk1 : blk0) * kRowsPerBlock + lane;
+                const int p1 = __ldg(b.rowptr + row + 1);
+                for (int p = __ldg(b.rowptr + row) + ell_slots; p < p1; ++p) {
+                    const uint32_t e = __ldg(b.oent + p);
+#pragma unroll
+                    for (int bb = 0; bb < NB; ++bb)
+                        acc[bb][h] = fmaf(h2f((uint16_t)(e >> 16)), h2f(xs[(size_t)bb * K + (e & 0xffffu)]), acc[bb][h]);
+                }
+            }
+        }
+    }
+
+    // ---- (4) fixed-order reduction over the warps, store or split-K finish
+#pragma unroll
+    for (int bb = 0; bb < NB; ++bb) {
+        red[((size_t)warp * NB + bb) * kARows + lane] = acc[bb][0];
+        red[((size_t)warp * NB + bb) * kARows + 32 + lane] = acc[bb][1];
+    }
+    __syncthreads();
+    const int t = threadIdx.x;
+    const int bb = t / kARows, r = t % kARows;
+    const bool active = t < NB * kARows;
+    const bool dup = (r >= 32) && (2 * blk + 1 >= a.RB);
+    const int row = blk * kARows + r;
+    float total = 0.f;
+    if (active) {
+#pragma unroll
+        for (int w = 0; w < kAWarps; ++w) total += red[((size_t)w * NB + bb) * kARows + r];
+    }
+    if (KS > 1) {
+        __shared__ int s_last;
+        float* part = a.partial + (size_t)prob * 64 * NB * a.rows_ws;
+        int* ticket = a.tickets + (size_t)prob * a.blocks + blk;
+        if (active) part[((size_t)ks * NB + bb) * a.rows_ws + row] = total;
+        __threadfence();
+        __syncthreads();
+        if (t == 0) s_last = (atomicAdd(ticket, 1) == KS - 1);
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        if (active) {
+            total = 0.f;
+            for (int k2 = 0; k2 < KS; ++k2) total += __ldcg(part + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+        }
+        if (t == 0) *ticket = 0;
+    }
+    if (active && !dup && bb < a.nb && row < a.rows) {
+        if (a.y_is_fp16)
+            ((uint16_t*)y)[(size_t)bb * a.rows + row] = f2h(total);
+        else
+            ((float*)y)[(size_t)bb * a.rows + row] = total;
+    }
+}
+
+// ------------------------------------------------------------------------------------ host side
+
+constexpr int kASlotsPerWave = 296;   // 148 SMs x 2 resident CTAs
+
+static size_t v2a_smem_bytes(const Layout& l, int nb) {
+    return (size_t)l.L * l.E * 128 + (size_t)nb * l.cols * 2 + (size_t)nb * l.SC * 4 + (size_t)kAWarps * nb * kARows * 4;
+}
+
+bool v2a_supported(const Layout& l, int batch) {
+    if (l.mode != 1 || l.bits < 2 || l.bits > 5 || batch > 2) return false;
+    return v2a_smem_bytes(l, batch) <= 110u * 1024u;   // two CTAs per SM
+}
+
+size_t v2a_workspace_bytes(const Layout& l) {
+    const int blocks = (l.RB + 1) / 2;
+    return align256((size_t)blocks * 4) + align256((size_t)64 * 2 * (size_t)blocks * kARows * 4);
+}
+
+template <int N, int NB>
+static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             112 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kAThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_v2a_kernel<N, NB>, a);
+}
+
+cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) {
+    V2aArgs a{};
+    a.off = offsets_of(l);
+    a.packed = c.packed; a.x = c.x; a.y = c.y;
+    a.packed_list = c.packed_list; a.x_list = c.x_list; a.y_list = c.y_list;
+    a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots; a.L = l.L;
+    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
+    a.blocks = (l.RB + 1) / 2;
+    a.rows_ws = a.blocks * kARows;
+    // schedule: whole-K blocks fill whole rounds of CTA slots (all blobs of the launch count); the blocks of
+    // the last partial round are cut along K into slices of at least 512 weights
+    const long long total = (long long)a.blocks * c.n;
+    int kst = 1;
+    int rem = 0;
+    const long long tail = total % kASlotsPerWave;
+    if (tail > 0 && c.n == 1) {
+        rem = (int)tail;
+        kst = kASlotsPerWave / rem;
+        const int kmax = l.SC / 4 > 1 ? l.SC / 4 : 1;
+        if (kst > kmax) kst = kmax;
+        if (kst > 64) kst = 64;
+        if (kst > l.SC) kst = l.SC;
+        if (kst <= 1) { kst = 1; rem = 0; }
+    }
+    a.n_full = a.blocks - rem;
+    a.sc_per_split = (l.SC + kst - 1) / kst;
+    a.kst = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
+    if (a.kst <= 1) { a.kst = 1; a.n_full = a.blocks; rem = 0; }
+    a.tickets = (int*)c.workspace;
+    a.partial = (float*)((char*)c.workspace + align256((size_t)a.blocks * 4 * c.n));
+    const size_t smem = v2a_smem_bytes(l, c.batch);
+    dim3 grid((unsigned)(a.n_full + rem * a.kst), (unsigned)c.n, 1);
+    switch (l.bits * 10 + c.batch) {
+        case 21: return launch_v2a<2, 1>(a, grid, smem, s);
+        case 22: return launch_v2a<2, 2>(a, grid, smem, s);
+        case 31: return launch_v2a<3, 1>(a, grid, smem, s);
+        case 32: return launch_v2a<3, 2>(a, grid, smem, s);
+        case 41: return launch_v2a<4, 1>(a, grid, smem, s);
+        case 42: return launch_v2a<4, 2>(a, grid, smem, s);
+        case 51: return launch_v2a<5, 1>(a, grid, smem, s);
+        case 52: return launch_v2a<5, 2>(a, grid, smem, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace xfp

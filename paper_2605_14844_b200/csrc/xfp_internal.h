@@ -52,9 +52,15 @@ void pair_set_debug(int m);
 void pair_set_small(int v);
 void pair_set_trace(void* p, size_t calls);
 
+// Fast V2a path (per-bank library + mma.sync fragments, one or several blobs); see xfp_gemv_v2a.cu.
+bool v2a_supported(const Layout& l, int batch);
+size_t v2a_workspace_bytes(const Layout& l);
+cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
+
 inline size_t workspace_bytes_for(const Layout& l) {
-    const size_t g = generic_workspace_bytes(l), p = pair_workspace_bytes(l);
-    return g > p ? g : p;
+    size_t w = generic_workspace_bytes(l);
+    const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);
+    return w > p ? w : p;
 }
 
 }  // namespace xfp

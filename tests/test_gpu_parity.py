@@ -172,9 +172,12 @@ def test_grouped_matches_single_calls():
     torch.cuda.synchronize()
     for j in range(n):
         single = pms[j].gemv(xs[j])
-        assert torch.equal(single[0], ys[j])
         ref, absum = xo.gemv(to_oracle(qs[j]), xs[j].view(torch.int16).cpu().numpy().view(np.uint16))
+        # the single call may split K differently from the group launch: both obey the bound, and they
+        # agree with each other far inside it
         assert np.all(np.abs(ys[j].cpu().numpy() - ref[0]) <= TOL * absum[0])
+        assert np.all(np.abs(single[0].cpu().numpy() - ref[0]) <= TOL * absum[0])
+        assert np.all(np.abs(single[0].cpu().numpy() - ys[j].cpu().numpy()) <= 0.05 * TOL * absum[0])
 
 
 def test_gemv_host_entry():
