@@ -9,6 +9,12 @@
         graph of P calls, median of 20 replays) and print microseconds per call and effective GB/s over
         the algorithmic bytes.
 
+    python -m paper_2605_14844_b200.probe moe [EXPERTS] [TOKENS] [BITS]
+        routed-MoE decode layer: EXPERTS (default 128) V2a experts with a gate_up projection 3072 x 4096
+        and a down projection 4096 x 1536 (one library per projection, 0.1 % outliers), top-8 routing per
+        token; every token-layer is two xfp_gemv_grouped launches (8 gate_up, 8 down).  Prints
+        microseconds per token-layer and effective GB/s.
+
 MODE 0 = V2, 1 = V2a; PLACEMENT uniform | clustered | one_row.  Inputs come from synth.random_quantized.
 """
 from __future__ import annotations
@@ -84,7 +90,69 @@ def time_shape(mode, rows, cols, bits, rate, batch=1, placement="uniform", reps=
     return out
 
 
+def moe(experts=128, tokens=64, bits=3, distinct=8, reps=10):
+    from . import XfpDesc, xfp_gemv_grouped, xfp_packed_size
+    shapes = {"gate_up": (3072, 4096), "down": (4096, 1536)}
+    packed, descs, nbytes = {}, {}, {}
+    for name, (rows, cols) in shapes.items():
+        base = [synth.random_quantized(1, rows, cols, bits, 0.001, seed=100 + j) for j in range(distinct)]
+        for q in base[1:]:
+            q.codebook = base[0].codebook            # one library per projection, shared by the layer's experts
+        packed[name] = [pack_tensors(base[e % distinct], col_bits=16) for e in range(experts)]
+        d0 = packed[name][0].desc
+        descs[name] = XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                              max(p.desc.nnz for p in packed[name]))
+        nbytes[name] = algorithmic_bytes(base[0])
+    route = synth.moe_routing(tokens, experts, 8, seed=7)
+    dev = "cuda"
+    x_up = [_x(1, 4096) for _ in range(tokens)]
+    h = [torch.zeros((8, 1536), dtype=torch.float16, device=dev) for _ in range(tokens)]     # down inputs
+    y_up = [torch.empty((8, 3072), dtype=torch.float16, device=dev) for _ in range(tokens)]
+    y_dn = [torch.empty((8, 4096), dtype=torch.float16, device=dev) for _ in range(tokens)]
+    for t in h:
+        t.copy_(_x(8, 1536))
+    ptrs = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device=dev)
+    args = []
+    for t in range(tokens):
+        ex = route[t]
+        args.append((ptrs([packed["gate_up"][e].packed for e in ex]), ptrs([x_up[t]] * 8), ptrs([y_up[t][j] for j in range(8)]),
+                     ptrs([packed["down"][e].packed for e in ex]), ptrs([h[t][j] for j in range(8)]),
+                     ptrs([y_dn[t][j] for j in range(8)])))
+    ws = {n: torch.zeros(8 * xfp_packed_size(descs[n])[1], dtype=torch.uint8, device=dev) for n in shapes}
+
+    def layer(a):
+        xfp_gemv_grouped(descs["gate_up"], 8, a[0], a[1], a[2], True, ws["gate_up"])
+        xfp_gemv_grouped(descs["down"], 8, a[3], a[4], a[5], True, ws["down"])
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        layer(args[0])
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for a in args:
+                layer(a)
+        for _ in range(3):
+            g.replay()
+        s.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(s)
+            g.replay()
+            e1.record(s)
+            s.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3 / tokens)
+    per_layer = 8 * (nbytes["gate_up"] + nbytes["down"])
+    t = float(np.median(ts))
+    print(json.dumps(dict(workload="moe_v2a", experts=experts, tokens=tokens, bits=bits, MB_per_token_layer=round(per_layer / 1e6, 2),
+                          us_per_token_layer=round(t, 2), GBs=round(per_layer / t / 1e3, 1))), flush=True)
+
+
 def main(argv):
+    if len(argv) > 1 and argv[1] == "moe":
+        moe(*(int(v) for v in argv[2:5]))
+        return 0
     if len(argv) < 7 or argv[1] not in ("launch", "time"):
         print(__doc__)
         return 2
