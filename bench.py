@@ -171,6 +171,21 @@ def run_reference(args, rank: int):
     }))
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (the timed region of a multi-GPU run is
+    as long as its slowest rank); identity when torch.distributed is not initialised."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized():
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_value(step_bytes: int, world: int, ms_per_step: float) -> float:
+    """Whole-job GB/s of `world` replicas that each move step_bytes per step (weak scaling)."""
+    return world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+
 def run_xfp(args, rank: int, world: int):
     import torch
     import paper_2605_14844_b200 as xfp
@@ -266,18 +281,15 @@ def run_xfp(args, rank: int, world: int):
         barrier()
         e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = t.tolist()
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     ms_per_step = total_ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
-    e2e_val = world * step_bytes / (e2e_ms / args.steps * 1e-3) / 1e9
+    value = aggregate_value(step_bytes, world, ms_per_step)
+    e2e_val = aggregate_value(step_bytes, world, e2e_ms / args.steps)
     peak, peak_kind = measured_peak()
     per_gpu = step_bytes / (ms_per_step * 1e-3) / 1e9
     out = {
