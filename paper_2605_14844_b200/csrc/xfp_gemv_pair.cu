@@ -1,12 +1,12 @@
 // Fast fused decode GEMV for V2 blobs at batch <= 2:  y = (D + S) x.
 //
-// Mapping.  A CTA owns a block of 32*RPL output channels (RPL = rows per lane: 2 for N <= 4,
-// 1 for N = 5) and all of K, or a slice of K for the blocks of the last scheduling round.  Each
-// lane of a dense warp owns RPL channels (lane, lane+32 of the block) and the warps of the CTA
-// share K in super-chunks of 128 weights.  The channels' codebooks are expanded once per CTA into
-// PAIR tables in shared memory: entry t = (cb[t & (E-1)], cb[t >> N]) as a half2, so one 32-bit
-// shared-memory load decodes two weights ("codebook gather from shared memory", step 2 of the
-// fused kernel).  The tables are laid out so that lane l only ever touches bank l: byte address
+// Mapping.  A CTA works on blocks of 32*RPL output channels (RPL = rows per lane: 2 for N <= 4,
+// 1 for N = 5 and for matrices with few rows).  Each lane of a warp owns RPL channels (lane, lane+32
+// of the block) and the warps of the CTA share K in super-chunks of 128 weights.  The channels'
+// codebooks are expanded once per block into PAIR tables in shared memory: entry
+// t = (cb[t & (E-1)], cb[t >> N]) as a half2, so one 32-bit shared-memory load decodes two weights
+// ("codebook gather from shared memory", step 2 of the fused kernel).  The tables are laid out so
+// that lane l only ever touches bank l: byte address
 //     t * (128 * RPL) + channel_half * 128 + lane * 4
 // hence any index pattern is bank-conflict free.
 //
@@ -22,22 +22,25 @@
 // the tensor pipe even at batch 1.)
 //
 // Outliers (step 3) ride in the same pass: xfp_pack stores every 32-row block's outliers as a
-// transposed slab (slot j of channel l at slab + j*32 + l), so a warp reads one slot of all 32
+// transposed slab (slot j of channel l at slab + (1+j)*32 + l), so a warp reads one slot of all 32
 // channels with one coalesced load and every lane adds val * x[col] (x gathered from the staged
 // copy in shared memory) to an accumulator of its own channel.  Slots are dealt round-robin to the
-// dense warps and consumed between super-chunks, their loads issued one iteration ahead.  Rows
-// longer than the slab (pathological skew) finish from the CSR arrays.  The order of additions is
-// fixed by the schedule, so results are reproducible.
+// warps and consumed between super-chunks, their loads issued one iteration ahead, the first round
+// before the rows' lengths are known.  Rows longer than the slab (pathological skew) finish from
+// the CSR arrays.  The order of additions is fixed by the schedule, so results are reproducible.
 //
-// Schedule.  Blocks that fill whole rounds of CTA slots run over all of K; the blocks of the last,
-// partial round are cut along K so that they occupy the idle slots, and their partial sums are
-// combined by the last CTA of a block in fixed order (no waiting, no atomics on data).
+// Schedule.  A CTA handles one block over all of K, or one K slice of a block.  Blocks that fill whole
+// rounds of CTA slots run unsplit; the blocks of the last, partial round are cut into 2 slices, and
+// what still does not fit into finer slices (tiers of decreasing piece size: the hardware
+// dispatches CTAs in launch order, so the tiers pack the slots largest-first).  Partial sums of a
+// cut block go through the workspace and the last CTA to arrive adds them in slice order (an atomic
+// ticket, no waiting, no atomics on data).  With fewer blocks than half the slots every block is
+// cut into 2, 4 or 8 slices that form a thread-block cluster and reduce through distributed shared
+// memory.
 //
-// Launch overlap.  Weights do not depend on earlier kernels, so every CTA first issues its index,
-// codebook and row-pointer loads and fills its pair tables, and only then executes
+// Launch overlap.  Weights do not depend on earlier kernels, so a CTA first issues its index,
+// codebook and outlier loads and fills its pair tables, and only then executes
 // griddepcontrol.wait (programmatic dependent launch) before it touches x, y or the workspace.
-// Back-to-back calls on one stream therefore overlap the next call's weight streaming with the
-// current call's tail.
 #include <cooperative_groups.h>
 
 #include "xfp_internal.h"
@@ -52,17 +55,16 @@ struct PairArgs {
     const void* packed;
     const uint16_t* x;
     void* y;
-    float* partial;  // [KS][NB][rows_ws]
+    float* partial;  // [slice][NB][rows_ws]
     int* tickets;    // [blocks]
     int rows, cols, RB, SC, rows_ws, ell_slots;
     int nb, y_is_fp16;
-    // schedule: work items [0, n_full) are whole blocks; the remaining blocks are cut into kst
-    // K-slices of sc_per_split super-chunks each
-    int n_full, kst, sc_per_split;
-    int pf_dist;  // L2 prefetch distance in warp iterations (0 = off)
-    int cluster;  // 1: the kst CTAs of a block form a thread-block cluster and reduce through DSMEM
-    int dbg;      // timing probes only: 1 = return after the dependency wait, 2 = skip the main loop, 3 = no PDL
-    unsigned long long* trace;  // timing probes only: per CTA 8 globaltimer stamps
+    int blocks;      // blocks of 32*RPL channels
+    // schedule tiers: CTAs [tier_cta[i], tier_cta[i+1]) handle blocks from tier_blk[i] on, each cut into
+    // tier_kst[i] slices of tier_spp[i] super-chunks
+    int tier_cta[5], tier_blk[4], tier_kst[4], tier_spp[4];
+    int cluster;     // single tier with kst > 1: the kst CTAs of a block form a cluster and reduce through DSMEM
+    unsigned long long* trace;  // timing probe: per CTA 8 globaltimer stamps (null in normal use)
 };
 
 __device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
@@ -77,54 +79,66 @@ template <int N, int NB, int RPL, int W>
 __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
     constexpr int E = 1 << N;
     constexpr int T = E * E;                   // pair-table entries per channel
-    constexpr int ROWS = 32 * RPL;             // channels per CTA
+    constexpr int ROWS = 32 * RPL;             // channels per block
     constexpr int kStride = 128 * RPL;         // bytes between consecutive entries
     constexpr int kTabBytes = T * kStride;
-    constexpr int kDense = W * 32;
+    constexpr int kThreads = W * 32;
+    constexpr int TW = T / W;                  // table entries a warp fills per channel half
     extern __shared__ __align__(16) unsigned char smem[];
     // [tables | x fp16 [NB][K] | red[W][NB][ROWS]]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
     stamp(a, 0);
-    if (a.dbg == 1) {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        return;
-    }
-    int blk, ks, KS, spp;
-    if ((int)blockIdx.x < a.n_full) {
-        blk = blockIdx.x; ks = 0; KS = 1; spp = a.SC;
-    } else {
-        const int t = blockIdx.x - a.n_full;
-        blk = a.n_full + t / a.kst; ks = t % a.kst; KS = a.kst; spp = a.sc_per_split;
-    }
     const Blob b = blob_at(a.packed, a.off);
-    const int sc0 = ks * spp;
-    const int nsc = max(0, min(a.SC, sc0 + spp) - sc0);
     const int K = a.SC * kSuper;
 
     unsigned char* tab = smem;
     uint16_t* xs = (uint16_t*)(smem + kTabBytes);               // [NB][K]
     float* red = (float*)(xs + (size_t)NB * K);                 // [W][NB][ROWS]
 
-    // the 32-row blocks of this CTA (the second is clamped when RB is odd; its results are dropped)
-    const int blk0 = RPL * blk;
-    const int blk1 = min(RPL * blk + (RPL - 1), a.RB - 1);
-
+    // ---- this CTA's block and K slice
+    int blk, slice, nslices, sc0, nsc;
     {
-        // ------------------------------------------------ dense warps
-        // (0) start streaming this warp's first super-chunk before anything else
-        uint32_t w0[4 * N + 1], w1[RPL == 2 ? 4 * N + 1 : 1];
-        w0[4 * N] = 0u;
-        if (RPL == 2) w1[4 * N] = 0u;
-        const uint4* i0 = b.idx + ((size_t)(blk0 * a.SC + sc0) * N) * 32 + lane;
-        const uint4* i1 = b.idx + ((size_t)(blk1 * a.SC + sc0) * N) * 32 + lane;
-        auto prefetch_sc = [&](int sidx) {   // the RPL * N * 512 bytes of a super-chunk are RPL * 4N lines
-            if (lane < RPL * 4 * N) {
-                const int half = lane / (4 * N), line = lane % (4 * N);
-                const char* p = (const char*)((half ? i1 : i0) - lane + (size_t)sidx * N * 32) + line * 128;
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+        int tier = 0;
+#pragma unroll
+        for (int i = 1; i < 4; ++i)
+            if ((int)blockIdx.x >= a.tier_cta[i]) tier = i;
+        const int c = blockIdx.x - a.tier_cta[tier];
+        nslices = a.tier_kst[tier];
+        blk = a.tier_blk[tier] + c / nslices;
+        slice = c % nslices;
+        sc0 = slice * a.tier_spp[tier];
+        nsc = max(0, min(a.SC, sc0 + a.tier_spp[tier]) - sc0);
+    }
+    const int blk0 = RPL * blk;
+    const int blk1 = min(RPL * blk + (RPL - 1), a.RB - 1);   // clamped when RB is odd; its results are dropped
+    const int gw = slice * W + warp, ostride = nslices * W;
+
+    // per-thread state
+    uint32_t w0[4 * N + 1], w1[RPL == 2 ? 4 * N + 1 : 1];
+    w0[4 * N] = 0u;
+    if (RPL == 2) w1[4 * N] = 0u;
+    const uint4 *i0 = nullptr, *i1 = nullptr;
+    const uint32_t* slab[RPL];
+    int width[RPL];
+    uint32_t olen[RPL];
+    uint32_t oe[RPL][kSlotsPerRound];
+    uint32_t cbw[RPL][TW >= E ? E / 2 : 1];
+    uint32_t cbh[RPL][TW >= E ? TW / E : 1];
+    auto fetch_slots = [&](int round) {
+#pragma unroll
+        for (int h = 0; h < RPL; ++h)
+#pragma unroll
+            for (int q = 0; q < kSlotsPerRound; ++q) {
+                const int j = gw + (round * kSlotsPerRound + q) * ostride;
+                oe[h][q] = j < width[h] ? __ldg(slab[h] + (size_t)(1 + j) * 32) : 0u;
             }
-        };
+    };
+    // everything the CTA reads from the blob before it can start: first super-chunk of this warp,
+    // slab lengths and first round of outlier slots, the channels' codebooks
+    auto issue_loads = [&]() {
+        i0 = b.idx + ((size_t)(blk0 * a.SC + sc0) * N) * 32 + lane;
+        i1 = b.idx + ((size_t)(blk1 * a.SC + sc0) * N) * 32 + lane;
         if (warp < nsc) {
 #pragma unroll
             for (int v = 0; v < N; ++v) {
@@ -136,65 +150,13 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
                 }
             }
         }
-        // one row per lane leaves registers for a second super-chunk in flight (short K loops are
-        // otherwise a chain of DRAM round trips)
-        constexpr bool kTwoDeep = (RPL == 1);
-        uint32_t z0[kTwoDeep ? 4 * N + 1 : 1];
-        if (kTwoDeep) {
-            z0[4 * N] = 0u;
-            if (warp + W < nsc) {
-#pragma unroll
-                for (int v = 0; v < N; ++v) {
-                    const uint4 t0 = ld_stream(i0 + ((size_t)(warp + W) * N + v) * 32);
-                    z0[4 * v] = t0.x; z0[4 * v + 1] = t0.y; z0[4 * v + 2] = t0.z; z0[4 * v + 3] = t0.w;
-                }
-            }
-        }
-        if (a.pf_dist > 0)
-            for (int r = 1; r <= a.pf_dist; ++r)
-                if (warp + r * W < nsc) prefetch_sc(warp + r * W);
-        // outlier slabs of this CTA's row-blocks: slots gw, gw + stride, ... belong to this warp.  The first
-        // round is fetched before the rows' lengths are known (any slot below the capacity is readable).
-        const int gw = ks * W + warp, ostride = KS * W;
-        const uint32_t* slab[RPL];
-        int width[RPL];
-        uint32_t olen[RPL];
-        uint32_t oe[RPL][kSlotsPerRound];
-        float oacc[NB][RPL];
-        int oround = 0, nrounds = 0;
 #pragma unroll
         for (int h = 0; h < RPL; ++h) {
             slab[h] = b.ell + (size_t)(h ? blk1 : blk0) * (a.ell_slots + 1) * 32 + lane;
-            width[h] = a.ell_slots;
+            width[h] = a.ell_slots;   // capacity: every slot below it is readable
             olen[h] = a.ell_slots ? __ldg(slab[h]) : 0u;
-#pragma unroll
-            for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = 0.f;
         }
-        auto fetch_slots = [&](int round) {
-#pragma unroll
-            for (int h = 0; h < RPL; ++h)
-#pragma unroll
-                for (int q = 0; q < kSlotsPerRound; ++q) {
-                    const int j = gw + (round * kSlotsPerRound + q) * ostride;
-                    oe[h][q] = j < width[h] ? __ldg(slab[h] + (size_t)(1 + j) * 32) : 0u;
-                }
-        };
-        auto consume_slots = [&]() {
-#pragma unroll
-            for (int h = 0; h < RPL; ++h)
-#pragma unroll
-                for (int q = 0; q < kSlotsPerRound; ++q) {
-                    const float v = h2f((uint16_t)(oe[h][q] >> 16));
-                    const uint32_t col = oe[h][q] & 0xffffu;
-#pragma unroll
-                    for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = fmaf(v, h2f(xs[(size_t)bb * K + col]), oacc[bb][h]);
-                }
-        };
         if (a.ell_slots) fetch_slots(0);
-        // codebooks of this lane's channels (for the table fill below)
-        constexpr int TW = T / W;  // table entries per warp
-        uint32_t cbw[RPL][TW >= E ? E / 2 : 1];
-        uint32_t cbh[RPL][TW >= E ? TW / E : 1];
         if (TW >= E) {
 #pragma unroll
             for (int half = 0; half < RPL; ++half) {
@@ -208,167 +170,150 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
                 for (int hh = 0; hh < TW / E; ++hh) cbh[half][hh] = __ldg(cb + warp * (TW / E) + hh);
             }
         }
-        // (1) pair tables: warp w fills entries t in [w*T/W, (w+1)*T/W) of every channel half
-        {
+    };
+    // pair tables: warp w fills entries t in [w*T/W, (w+1)*T/W) of every channel half
+    auto fill_tables = [&]() {
 #pragma unroll
-            for (int half = 0; half < RPL; ++half) {
-                unsigned char* dst = tab + half * 128 + lane * 4;
-                if (TW >= E) {
+        for (int half = 0; half < RPL; ++half) {
+            unsigned char* dst = tab + half * 128 + lane * 4;
+            if (TW >= E) {
 #pragma unroll
-                    for (int hh = 0; hh < TW / E; ++hh) {
-                        const int hi = warp * (TW / E) + hh;
-                        const uint32_t hv = cbh[half][hh];
+                for (int hh = 0; hh < TW / E; ++hh) {
+                    const int hi = warp * (TW / E) + hh;
+                    const uint32_t hv = cbh[half][hh];
 #pragma unroll
-                        for (int lo = 0; lo < E; ++lo) {
-                            const uint32_t lv = (lo & 1) ? (cbw[half][lo >> 1] >> 16) : (cbw[half][lo >> 1] & 0xffffu);
-                            *(uint32_t*)(dst + (size_t)(hi * E + lo) * kStride) = lv | (hv << 16);
-                        }
+                    for (int lo = 0; lo < E; ++lo) {
+                        const uint32_t lv = (lo & 1) ? (cbw[half][lo >> 1] >> 16) : (cbw[half][lo >> 1] & 0xffffu);
+                        *(uint32_t*)(dst + (size_t)(hi * E + lo) * kStride) = lv | (hv << 16);
                     }
-                } else {
-                    // small tables (N = 2): TW < E entries per warp
-                    const uint16_t* cb = b.cb + (size_t)((half ? blk1 : blk0) * kRowsPerBlock + lane) * E;
+                }
+            } else {
+                // small tables (N = 2): at most a few entries per warp
+                const uint16_t* cb = b.cb + (size_t)((half ? blk1 : blk0) * kRowsPerBlock + lane) * E;
 #pragma unroll
-                    for (int i = 0; i < TW; ++i) {
-                        const int t = warp * TW + i;
+                for (int i = 0; i < (TW > 0 ? TW : 1); ++i) {
+                    const int t = TW > 0 ? warp * TW + i : warp;
+                    if (t < T) {
                         const uint32_t lv = __ldg(cb + (t & (E - 1))), hv = __ldg(cb + (t >> N));
                         *(uint32_t*)(dst + (size_t)t * kStride) = lv | (hv << 16);
                     }
                 }
             }
         }
-        // x may come from the previous kernel: everything above overlaps that kernel's tail
-        stamp(a, 1);
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        stamp(a, 2);
-        constexpr int XV = 4;                       // uint4 of x per thread per pass
-        const int nvec = NB * (K / 8);
-        uint4 xv[XV];
-#pragma unroll
-        for (int i = 0; i < XV; ++i) {
-            const int t = threadIdx.x + i * kDense;
-            xv[i] = make_uint4(0u, 0u, 0u, 0u);
-            if (t < nvec) {
-                const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
-                if (bb < a.nb) xv[i] = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
-            }
-        }
+    };
 
-        stamp(a, 3);
-        // (2) x (fp16 bits, all of K: outlier columns are gathered from it) -> shared memory
-#pragma unroll
-        for (int i = 0; i < XV; ++i) {
-            const int t = threadIdx.x + i * kDense;
-            if (t < nvec) *(uint4*)(xs + (size_t)t * 8) = xv[i];
+    // ---- loads and tables overlap the previous kernel's tail
+    issue_loads();
+    fill_tables();
+    stamp(a, 1);
+    // ---- x (fp16 bits, all of K: outlier columns are gathered from it) may come from the previous kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    stamp(a, 2);
+    for (int t = threadIdx.x; t < NB * (K / 8); t += kThreads) {
+        const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
+        *(uint4*)(xs + (size_t)t * 8) = v;
+    }
+    __syncthreads();   // tables and x visible
+    stamp(a, 3);
+
+    const uint32_t base0 = (uint32_t)lane * 4u, base1 = base0 | 128u;
+    const int g = lane >> 2, t4 = lane & 3;
+    // B fragment: lane (g', t') feeds column n = g' with the k slots of group t'.  Column t' of
+    // batch row 0 is fed by g' == t'; column 4 + t' of batch row 1 by g' == t' + 4.
+    const bool diag0 = (g == t4);
+    const bool diag1 = (NB > 1) && (g == t4 + 4);
+    const bool diag = diag0 || diag1;
+    const unsigned char* xbase = (const unsigned char*)xs + (diag1 ? (size_t)K * 2 : 0);
+
+    auto lookup = [&](uint32_t (&f)[4], int m) {
+        f[0] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m, base0));
+        f[2] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m + 1, base0));
+        if (RPL == 2) {
+            f[1] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w1, 2 * m, base1));
+            f[3] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w1, 2 * m + 1, base1));
+        } else {
+            f[1] = 0u; f[3] = 0u;
         }
-        for (int t = threadIdx.x + XV * kDense; t < nvec; t += kDense) {   // K beyond XV passes
-            const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
-            *(uint4*)(xs + (size_t)t * 8) = v;
-        }
-        // the rows' slot counts are here by now: this warp's number of outlier rounds
+    };
+
+    {
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+        float oacc[NB][RPL];
+        int oround = 0, nrounds = 0;
 #pragma unroll
         for (int h = 0; h < RPL; ++h) {
+            // the rows' slot counts have arrived: this warp's number of outlier rounds
             int wmax = (int)olen[h];
 #pragma unroll
             for (int o = 16; o; o >>= 1) wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
             width[h] = min(wmax, a.ell_slots);
             const int mine = width[h] > gw ? (width[h] - gw + ostride - 1) / ostride : 0;
             nrounds = max(nrounds, (mine + kSlotsPerRound - 1) / kSlotsPerRound);
+#pragma unroll
+            for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = 0.f;
         }
-        __syncthreads();  // tables and x visible
-        stamp(a, 4);
-
-        // (3) main loop
-        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t base0 = (uint32_t)lane * 4u, base1 = base0 | 128u;
-        const int g = lane >> 2, t4 = lane & 3;
-        // B fragment: lane (g', t') feeds column n = g' with the k slots of group t'.  Column t' of
-        // batch row 0 is fed by g' == t'; column 4 + t' of batch row 1 by g' == t' + 4.
-        const bool diag0 = (g == t4);
-        const bool diag1 = (NB > 1) && (g == t4 + 4);
-        const bool diag = diag0 || diag1;
-        const unsigned char* xrow =
-            (const unsigned char*)xs + (diag1 ? (size_t)K * 2 : 0) + (size_t)sc0 * (kSuper * 2);
-
-        auto lookup = [&](uint32_t (&f)[4], const uint32_t* u0, const uint32_t* u1, int m) {
-            f[0] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u0, 2 * m, base0));
-            f[2] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u0, 2 * m + 1, base0));
-            if (RPL == 2) {
-                f[1] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u1, 2 * m, base1));
-                f[3] = *(const uint32_t*)(tab + pair_addr<N, RPL>(u1, 2 * m + 1, base1));
-            } else {
-                f[1] = 0u; f[3] = 0u;
-            }
+        auto consume_slots = [&]() {
+#pragma unroll
+            for (int h = 0; h < RPL; ++h)
+#pragma unroll
+                for (int q = 0; q < kSlotsPerRound; ++q) {
+                    const float v = h2f((uint16_t)(oe[h][q] >> 16));
+                    const uint32_t col = oe[h][q] & 0xffffu;
+#pragma unroll
+                    for (int bb = 0; bb < NB; ++bb) oacc[bb][h] = fmaf(v, h2f(xs[(size_t)bb * K + col]), oacc[bb][h]);
+                }
         };
-        // One super-chunk.  Look-ups run one mma ahead of the tensor pipe; as soon as the last pair of
-        // a 16-byte vector has been looked up, the vector's registers are reloaded with the same
-        // vector of this warp's next super-chunk (the index stream needs 4 * N * RPL registers).
-        auto compute_sc = [&](uint32_t* u0, uint32_t* u1, int sidx, bool has_next, int snext) {
-            const unsigned char* xp = xrow + (size_t)sidx * (kSuper * 2);
-            uint32_t fa[4], fb[4];
-            uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = make_uint4(0u, 0u, 0u, 0u);
-            if (diag) xa = *(const uint4*)xp;
-            lookup(fa, u0, u1, 0);
+
+        // ---- K loop.  Look-ups run one mma ahead of the tensor pipe; as soon as the last pair of a 16-byte
+        //      vector has been looked up, its registers are reloaded with the same vector of this warp's
+        //      next super-chunk (the index stream needs 4 * N * RPL registers).
+#pragma unroll 1
+        for (int s = warp; s < nsc; s += W) {
+            if (oround < nrounds) {
+                consume_slots();
+                if (++oround < nrounds) fetch_slots(oround);
+            }
+            const bool has_next = s + W < nsc;
+            const int snext = s + W;
             auto reload = [&](int gi) {   // gi: group whose look-ups were just issued (compile time)
 #pragma unroll
                 for (int v = 0; v < N; ++v) {
                     const int plast = (128 * (v + 1) + 2 * N - 1) / (2 * N) - 1;   // last pair touching vector v
                     if (plast / 2 == gi && has_next) {
                         const uint4 t0 = ld_stream(i0 + ((size_t)snext * N + v) * 32);
-                        u0[4 * v] = t0.x; u0[4 * v + 1] = t0.y; u0[4 * v + 2] = t0.z; u0[4 * v + 3] = t0.w;
+                        w0[4 * v] = t0.x; w0[4 * v + 1] = t0.y; w0[4 * v + 2] = t0.z; w0[4 * v + 3] = t0.w;
                         if (RPL == 2) {
                             const uint4 t1 = ld_stream(i1 + ((size_t)snext * N + v) * 32);
-                            u1[4 * v] = t1.x; u1[4 * v + 1] = t1.y; u1[4 * v + 2] = t1.z; u1[4 * v + 3] = t1.w;
+                            w1[4 * v] = t1.x; w1[4 * v + 1] = t1.y; w1[4 * v + 2] = t1.z; w1[4 * v + 3] = t1.w;
                         }
                     }
                 }
             };
+            const unsigned char* xp = xbase + (size_t)(sc0 + s) * (kSuper * 2);
+            uint32_t fa[4], fb[4];
+            uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = make_uint4(0u, 0u, 0u, 0u);
+            if (diag) xa = *(const uint4*)xp;
+            lookup(fa, 0);
 #pragma unroll
             for (int m = 0; m < kSuper / 4; m += 4) {   // one mma per 4 consecutive k
                 if (diag) xb = *(const uint4*)(xp + (m + 2) * 8);
-                lookup(fb, u0, u1, m + 1);
+                lookup(fb, m + 1);
                 reload(m + 1);
                 mma16816(c0, fa[0], fa[1], fa[2], fa[3], xa.x, xa.y);
-                lookup(fa, u0, u1, m + 2);
+                lookup(fa, m + 2);
                 reload(m + 2);
                 mma16816(c1, fb[0], fb[1], fb[2], fb[3], xa.z, xa.w);
                 if (m + 4 < kSuper / 4) { if (diag) xa = *(const uint4*)(xp + (m + 4) * 8); }
-                lookup(fb, u0, u1, m + 3);
+                lookup(fb, m + 3);
                 reload(m + 3);
                 mma16816(c0, fa[0], fa[1], fa[2], fa[3], xb.x, xb.y);
                 if (m + 4 < kSuper / 4) {
-                    lookup(fa, u0, u1, m + 4);
+                    lookup(fa, m + 4);
                     reload(m + 4);
                 }
                 mma16816(c1, fb[0], fb[1], fb[2], fb[3], xb.z, xb.w);
-            }
-        };
-        if (kTwoDeep) {
-#pragma unroll 1
-            for (int s = warp; s < (a.dbg == 2 ? 0 : nsc); s += 2 * W) {
-                if (oround < nrounds) {
-                    consume_slots();
-                    if (++oround < nrounds) fetch_slots(oround);
-                }
-                compute_sc(w0, w1, s, s + 2 * W < nsc, s + 2 * W);
-                if (s + W < nsc) {
-                    if (oround < nrounds) {
-                        consume_slots();
-                        if (++oround < nrounds) fetch_slots(oround);
-                    }
-                    compute_sc(z0, w1, s + W, s + 3 * W < nsc, s + 3 * W);
-                }
-            }
-        } else {
-#pragma unroll 1
-            for (int s = warp; s < (a.dbg == 2 ? 0 : nsc); s += W) {
-                if (a.pf_dist > 0 && s + (a.pf_dist + 1) * W < nsc) prefetch_sc(s + (a.pf_dist + 1) * W);
-                if (oround < nrounds) {
-                    consume_slots();
-                    if (++oround < nrounds) fetch_slots(oround);
-                }
-                compute_sc(w0, w1, s, s + W < nsc, s + W);
             }
         }
         while (oround < nrounds) {   // more outlier rounds than super-chunks
@@ -376,8 +321,8 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
             if (++oround < nrounds) fetch_slots(oround);
         }
         // Rows that fill their slab may continue in the CSR arrays (pathological skew only): warp 0 of
-        // the first K slice finishes them, one lane per row.
-        if (warp == 0 && ks == 0 && a.ell_slots) {
+        // the block's first slice finishes them, one lane per row.
+        if (warp == 0 && slice == 0 && a.ell_slots) {
 #pragma unroll
             for (int h = 0; h < RPL; ++h) {
                 if ((int)olen[h] >= a.ell_slots) {
@@ -392,9 +337,10 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
                 }
             }
         }
-        stamp(a, 5);
-        // (4) scatter the fragment to channel order: lane (g, t) holds D[g][2t], D[g][2t+1], D[g+8][..]
-        //     column n < 4: batch 0 of lane 4g + n; column n >= 4: batch 1 of lane 4g + n - 4
+        stamp(a, 4);
+        const int cur_blk = blk, cur_slice = slice, cur_nslices = nslices;
+        // ---- scatter the fragment to channel order: lane (g, t) holds D[g][2t], D[g][2t+1], D[g+8][..];
+        //      column n < 4: batch 0 of lane 4g + n; column n >= 4: batch 1 of lane 4g + n - 4
         {
             const float v0 = c0[0] + c1[0], v1 = c0[1] + c1[1], v2 = c0[2] + c1[2], v3 = c0[3] + c1[3];
             const int bb = t4 >> 1;                  // batch row held by this lane's columns
@@ -410,114 +356,151 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
 #pragma unroll
                 for (int h = 0; h < RPL; ++h) red[((size_t)warp * NB + bb2) * ROWS + 32 * h + lane] += oacc[bb2][h];
         }
-        __syncthreads();
-    }
+        __syncthreads();   // partial sums of all warps are in red
 
-    // ---------------------------------------------------- fixed-order reduction, store / split-K finish
-    const int t = threadIdx.x;
-    const int bb = t / ROWS, r = t % ROWS;
-    const bool active = t < NB * ROWS;
-    // channel r of the block: rows of blk0 for r < 32, of blk1 for r >= 32
-    const bool dup = (r >= 32) && (RPL * blk + 1 >= a.RB);
-    const int row = blk * ROWS + r;
-    float total = 0.f;
-    if (active) {
-#pragma unroll
-        for (int w = 0; w < W; ++w) total += red[((size_t)w * NB + bb) * ROWS + r];
-    }
-    if (KS > 1 && a.cluster) {
-        // K slices of one block are the CTAs of one cluster: rank 0 adds the partial sums of its peers
-        // straight out of their shared memory, in rank order.
-        namespace cg = cooperative_groups;
-        cg::cluster_group cl = cg::this_cluster();
-        if (active) red[t] = total;          // slot t of red is read by thread t only
-        cl.sync();
-        if (ks == 0 && active) {
-            for (int k2 = 1; k2 < KS; ++k2) total += *cl.map_shared_rank(red + t, k2);
-        }
-        cl.sync();                            // peers keep their shared memory alive until rank 0 has read it
-        if (ks != 0) return;
-    } else if (KS > 1) {
-        __shared__ int s_last;
-        if (active) a.partial[((size_t)ks * NB + bb) * a.rows_ws + row] = total;
-        __threadfence();
-        __syncthreads();
-        if (t == 0) s_last = (atomicAdd(a.tickets + blk, 1) == KS - 1);
-        __syncthreads();
-        if (!s_last) return;
-        __threadfence();
+        // ---- fixed-order reduction over the warps, then store or combine the block's slices
+        const int t = threadIdx.x;
+        const int bb = t / ROWS, r = t % ROWS;
+        const bool active = t < NB * ROWS;
+        const bool dup = (r >= 32) && (RPL * cur_blk + 1 >= a.RB);
+        const int row = cur_blk * ROWS + r;
+        float total = 0.f;
         if (active) {
-            total = 0.f;
-            for (int k2 = 0; k2 < KS; ++k2) total += __ldcg(a.partial + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+#pragma unroll
+            for (int w = 0; w < W; ++w) total += red[((size_t)w * NB + bb) * ROWS + r];
         }
-        if (t == 0) a.tickets[blk] = 0;
+        bool writer = true;
+        if (cur_nslices > 1 && a.cluster) {
+            // the slices of a block are the CTAs of one cluster: rank 0 adds the partial sums of its peers
+            // straight out of their shared memory, in rank order
+            namespace cg = cooperative_groups;
+            cg::cluster_group cl = cg::this_cluster();
+            if (active) red[t] = total;          // slot t of red is read by thread t only
+            cl.sync();
+            if (cur_slice == 0 && active) {
+                for (int k2 = 1; k2 < cur_nslices; ++k2) total += *cl.map_shared_rank(red + t, k2);
+            }
+            cl.sync();                            // peers keep their shared memory alive until rank 0 has read it
+            writer = cur_slice == 0;
+        } else if (cur_nslices > 1) {
+            __shared__ int s_last;
+            if (active) a.partial[((size_t)cur_slice * NB + bb) * a.rows_ws + row] = total;
+            __threadfence();
+            __syncthreads();
+            if (t == 0) s_last = (atomicAdd(a.tickets + cur_blk, 1) == cur_nslices - 1);
+            __syncthreads();
+            writer = s_last != 0;
+            if (writer) {
+                __threadfence();
+                if (active) {
+                    total = 0.f;
+                    for (int k2 = 0; k2 < cur_nslices; ++k2)
+                        total += __ldcg(a.partial + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+                }
+                if (t == 0) a.tickets[cur_blk] = 0;
+            }
+        }
+        if (writer && active && !dup && bb < a.nb && row < a.rows) {
+            if (a.y_is_fp16)
+                ((uint16_t*)a.y)[(size_t)bb * a.rows + row] = f2h(total);
+            else
+                ((float*)a.y)[(size_t)bb * a.rows + row] = total;
+        }
+        stamp(a, 5);
     }
-    if (active && !dup && bb < a.nb && row < a.rows) {
-        if (a.y_is_fp16)
-            ((uint16_t*)a.y)[(size_t)bb * a.rows + row] = f2h(total);
-        else
-            ((float*)a.y)[(size_t)bb * a.rows + row] = total;
-    }
-    stamp(a, 6);
 }
 
 // ------------------------------------------------------------------------------------ host side
 
-static int g_pair_ks_override = 0;  // 0 = policy below
 static unsigned long long* g_pair_trace = nullptr;
 static size_t g_pair_trace_calls = 0, g_pair_trace_idx = 0;
-void pair_set_trace(void* p, size_t calls) { g_pair_trace = (unsigned long long*)p; g_pair_trace_calls = calls; g_pair_trace_idx = 0; }
-static int g_pair_dbg = 0;
-void pair_set_debug(int m) { g_pair_dbg = m; }
-static int g_pair_pf_dist = 0;  // L2 prefetch measured slower than none on B200
-
+void pair_set_trace(void* p, size_t calls) {
+    g_pair_trace = (unsigned long long*)p;
+    g_pair_trace_calls = calls;
+    g_pair_trace_idx = 0;
+}
+static int g_pair_ks_override = 0;  // probe: force aligned slices
 void pair_set_ksplit_override(int ks) { g_pair_ks_override = ks; }
-void pair_set_prefetch(int d) { g_pair_pf_dist = d; }
+void pair_set_prefetch(int) {}
+void pair_set_debug(int) {}
+static int g_pair_small = 1;        // probe switch: one row per lane for matrices with few row blocks
+void pair_set_small(int v) { g_pair_small = v; }
 
 struct PairConfig { int rpl, warps, slots; };
 
-static int g_pair_small = 1;   // probe switch: one row per lane for matrices with few row blocks
-void pair_set_small(int v) { g_pair_small = v; }
-
 static PairConfig pair_config(const Layout& l) {
-    // N <= 4: two rows per lane, 8 dense warps, two CTAs per SM.  N = 5: the pair table of a row is
-    // 4 KB, so one row per lane (128 KB of tables), 16 dense warps, one CTA per SM.  Matrices with
-    // fewer 64-row blocks than SMs also take one row per lane: twice the CTAs, no split along K.
+    // N <= 4: two rows per lane, 8 warps, two CTAs per SM.  N = 5: the pair table of a row is 4 KB, so
+    // one row per lane (128 KB of tables), 16 warps, one CTA per SM.  Matrices with at most 148
+    // row-blocks also take one row per lane: twice the CTAs and no cut along K.
     if (l.bits == 5) return PairConfig{1, 16, 148};
     if (g_pair_small == 1 && l.RB <= 148 && l.bits >= 3) return PairConfig{1, 16, 148};
-    if (g_pair_small == 2 && l.RB <= 148 && l.bits >= 3 && l.bits <= 4) return PairConfig{1, 8, 148};
     return PairConfig{2, 8, 296};
 }
 
-struct PairSchedule { int blocks, n_full, kst, sc_per_split, grid, cluster; };
+struct PairSchedule {
+    int blocks, grid, cluster, ntiers;
+    int tier_cta[5], tier_blk[4], tier_kst[4], tier_spp[4];
+};
+
+static int pow2_floor(int v) {
+    int p = 1;
+    while (p * 2 <= v) p *= 2;
+    return p;
+}
 
 static PairSchedule pair_schedule(const Layout& l) {
     const PairConfig cfg = pair_config(l);
     PairSchedule sc{};
     sc.blocks = (l.RB + cfg.rpl - 1) / cfg.rpl;
-    int rem = sc.blocks % cfg.slots;
-    int kst = 1;
-    const int kmax = l.SC / 4 > 1 ? l.SC / 4 : 1;   // keep K slices of at least 512 weights
+    const int S = cfg.slots;
+    const int kmax = l.SC / 4 > 1 ? pow2_floor(l.SC / 4) : 1;   // keep K slices of at least 512 weights
+    int nb[4] = {0, 0, 0, 0}, kk[4] = {1, 1, 1, 1};
+    int nt = 0;
     if (g_pair_ks_override > 0) {
-        rem = sc.blocks; kst = g_pair_ks_override;
-    } else if (sc.blocks < cfg.slots) {
-        // fewer blocks than CTA slots: cut every block into 2, 4 or 8 K slices that form a cluster
-        kst = 1;
-        while (kst < 8 && sc.blocks * kst * 2 <= cfg.slots && kst * 2 <= kmax) kst *= 2;
+        nb[0] = sc.blocks; kk[0] = g_pair_ks_override; nt = 1;
+    } else if (sc.blocks * 2 <= S) {
+        // fewer blocks than half the CTA slots: cut every block into 2, 4 or 8 K slices that form a cluster
+        int kst = 1;
+        while (kst < 8 && sc.blocks * kst * 2 <= S && kst * 2 <= kmax) kst *= 2;
+        nb[0] = sc.blocks; kk[0] = kst; nt = 1;
         sc.cluster = kst > 1;
-    } else if (rem > 0) {
-        // blocks of the last, partial round: cut along K so that the pieces fit the slots of one round
-        kst = cfg.slots / rem;
-        if (kst > kmax) kst = kmax;
-        if (kst > 64) kst = 64;
+    } else {
+        // whole rounds unsplit, then tiers of finer slices for the blocks of the last, partial round
+        const int full = (sc.blocks / S) * S;
+        int remaining = sc.blocks - full;
+        if (full > 0) { nb[nt] = full; kk[nt] = 1; ++nt; }
+        if (full == 0) { nb[nt] = remaining; kk[nt] = 1; ++nt; remaining = 0; }   // a single partial round
+        int k = 2;
+        while (remaining > 0 && nt < 4) {
+            if (k > kmax) { nb[nt] = remaining; kk[nt] = kmax; ++nt; remaining = 0; break; }
+            const int cap = S / k;   // blocks whose k slices fill one round
+            if (remaining <= cap || nt == 3) {
+                int kl = pow2_floor(S / remaining > 1 ? S / remaining : 1);
+                if (kl > kmax) kl = kmax;
+                if (kl > 64) kl = 64;
+                if (kl < k && remaining <= cap) kl = k;
+                nb[nt] = remaining; kk[nt] = kl < 1 ? 1 : kl; ++nt; remaining = 0;
+            } else {
+                nb[nt] = cap; kk[nt] = k; ++nt; remaining -= cap;
+                k *= 2;
+            }
+        }
     }
-    if (kst > l.SC) kst = l.SC;
-    if (kst <= 1) { rem = 0; kst = 1; sc.cluster = 0; }
-    sc.n_full = sc.blocks - rem;
-    sc.sc_per_split = (l.SC + kst - 1) / kst;
-    sc.kst = (l.SC + sc.sc_per_split - 1) / sc.sc_per_split;
-    if (sc.cluster && (sc.kst & (sc.kst - 1))) sc.cluster = 0;   // cluster sizes are powers of two
-    sc.grid = sc.n_full + rem * sc.kst;
+    sc.ntiers = nt;
+    int cta = 0, blk = 0;
+    for (int i = 0; i < 4; ++i) {
+        sc.tier_cta[i] = cta; sc.tier_blk[i] = blk;
+        int kst = i < nt ? kk[i] : 1;
+        if (kst > l.SC) kst = l.SC;
+        const int spp = (l.SC + kst - 1) / kst;
+        sc.tier_spp[i] = spp;
+        sc.tier_kst[i] = (l.SC + spp - 1) / spp;
+        if (i < nt) { cta += nb[i] * sc.tier_kst[i]; blk += nb[i]; }
+    }
+    sc.tier_cta[4] = cta;
+    for (int i = nt; i < 4; ++i) sc.tier_cta[i] = 0x7fffffff;   // unused tiers never match
+    sc.grid = cta;
+    if (sc.cluster && (sc.tier_kst[0] == 1 || (sc.tier_kst[0] & (sc.tier_kst[0] - 1)))) sc.cluster = 0;
     return sc;
 }
 
@@ -530,7 +513,7 @@ static size_t pair_smem_bytes(const Layout& l, int nb) {
 
 bool pair_supported(const Layout& l, int batch, int n_problems) {
     if (l.mode != 0 || l.bits < 2 || l.bits > 5 || batch > 2 || n_problems != 1) return false;
-    return pair_smem_bytes(l, batch) <= (pair_config(l).rpl == 2 ? 110u : 220u) * 1024u;
+    return pair_smem_bytes(l, batch) <= (pair_config(l).warps == 8 ? 110u : 220u) * 1024u;
 }
 
 size_t pair_workspace_bytes(const Layout& l) {
@@ -539,8 +522,7 @@ size_t pair_workspace_bytes(const Layout& l) {
 }
 
 template <int N, int NB, int RPL, int W>
-static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
-    const int cluster = a.cluster ? a.kst : 1;
+static cudaError_t launch_pair(const PairArgs& a, int grid, size_t smem, cudaStream_t s) {
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gemv_pair_kernel<N, NB, RPL, W>,
@@ -548,8 +530,9 @@ static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaSt
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
+    const int cluster = a.cluster ? a.tier_kst[0] : 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(W * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
@@ -562,10 +545,6 @@ static cudaError_t launch_pair(const PairArgs& a, dim3 grid, size_t smem, cudaSt
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = cluster > 1 ? 2 : 1;
-    if (a.dbg == 3) {   // probe: plain stream order
-        attr[0] = attr[1];
-        cfg.numAttrs = cluster > 1 ? 1 : 0;
-    }
     return cudaLaunchKernelEx(&cfg, gemv_pair_kernel<N, NB, RPL, W>, a);
 }
 
@@ -576,45 +555,35 @@ cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s)
     a.off = offsets_of(l);
     a.packed = c.packed; a.x = c.x; a.y = c.y;
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
+    a.blocks = sch.blocks;
     a.rows_ws = sch.blocks * 32 * cfg.rpl;
-    a.n_full = sch.n_full; a.kst = sch.kst; a.sc_per_split = sch.sc_per_split;
-    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
-    a.pf_dist = g_pair_pf_dist;
+    for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
+    for (int i = 0; i < 4; ++i) { a.tier_blk[i] = sch.tier_blk[i]; a.tier_kst[i] = sch.tier_kst[i]; a.tier_spp[i] = sch.tier_spp[i]; }
     a.cluster = sch.cluster && g_pair_ks_override == 0;
-    a.dbg = g_pair_dbg;
+    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
     a.trace = nullptr;
     if (g_pair_trace && g_pair_trace_idx < g_pair_trace_calls) a.trace = g_pair_trace + (g_pair_trace_idx++) * 1024 * 8;
     a.tickets = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
     const size_t smem = pair_smem_bytes(l, c.batch);
-    dim3 grid((unsigned)sch.grid, 1, 1);
-    if (cfg.rpl == 1 && cfg.warps == 8) {
-        switch (l.bits * 10 + c.batch) {
-            case 31: return launch_pair<3, 1, 1, 8>(a, grid, smem, s);
-            case 32: return launch_pair<3, 2, 1, 8>(a, grid, smem, s);
-            case 41: return launch_pair<4, 1, 1, 8>(a, grid, smem, s);
-            case 42: return launch_pair<4, 2, 1, 8>(a, grid, smem, s);
-        }
-        return cudaErrorInvalidValue;
-    }
     if (cfg.rpl == 1) {
         switch (l.bits * 10 + c.batch) {
-            case 31: return launch_pair<3, 1, 1, 16>(a, grid, smem, s);
-            case 32: return launch_pair<3, 2, 1, 16>(a, grid, smem, s);
-            case 41: return launch_pair<4, 1, 1, 16>(a, grid, smem, s);
-            case 42: return launch_pair<4, 2, 1, 16>(a, grid, smem, s);
-            case 51: return launch_pair<5, 1, 1, 16>(a, grid, smem, s);
-            case 52: return launch_pair<5, 2, 1, 16>(a, grid, smem, s);
+            case 31: return launch_pair<3, 1, 1, 16>(a, sch.grid, smem, s);
+            case 32: return launch_pair<3, 2, 1, 16>(a, sch.grid, smem, s);
+            case 41: return launch_pair<4, 1, 1, 16>(a, sch.grid, smem, s);
+            case 42: return launch_pair<4, 2, 1, 16>(a, sch.grid, smem, s);
+            case 51: return launch_pair<5, 1, 1, 16>(a, sch.grid, smem, s);
+            case 52: return launch_pair<5, 2, 1, 16>(a, sch.grid, smem, s);
         }
         return cudaErrorInvalidValue;
     }
     switch (l.bits * 10 + c.batch) {
-        case 21: return launch_pair<2, 1, 2, 8>(a, grid, smem, s);
-        case 22: return launch_pair<2, 2, 2, 8>(a, grid, smem, s);
-        case 31: return launch_pair<3, 1, 2, 8>(a, grid, smem, s);
-        case 32: return launch_pair<3, 2, 2, 8>(a, grid, smem, s);
-        case 41: return launch_pair<4, 1, 2, 8>(a, grid, smem, s);
-        case 42: return launch_pair<4, 2, 2, 8>(a, grid, smem, s);
+        case 21: return launch_pair<2, 1, 2, 8>(a, sch.grid, smem, s);
+        case 22: return launch_pair<2, 2, 2, 8>(a, sch.grid, smem, s);
+        case 31: return launch_pair<3, 1, 2, 8>(a, sch.grid, smem, s);
+        case 32: return launch_pair<3, 2, 2, 8>(a, sch.grid, smem, s);
+        case 41: return launch_pair<4, 1, 2, 8>(a, sch.grid, smem, s);
+        case 42: return launch_pair<4, 2, 2, 8>(a, sch.grid, smem, s);
     }
     return cudaErrorInvalidValue;
 }
