@@ -52,6 +52,10 @@ void pair_set_debug(int m);
 void pair_set_small(int v);
 void pair_set_trace(void* p, size_t calls);
 
+// Several V2 problems (batch 1) in one launch; see xfp_gemv_pair.cu.
+bool multi_supported(int n, const Layout* ls, const GemvCall* cs);
+cudaError_t launch_gemv_multi(int n, const Layout* ls, const GemvCall* cs, cudaStream_t s);
+
 // Fast V2a path (per-bank library + mma.sync fragments, one or several blobs); see xfp_gemv_v2a.cu.
 bool v2a_supported(const Layout& l, int batch);
 size_t v2a_workspace_bytes(const Layout& l);
