@@ -46,7 +46,9 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     GemvCall cc = c;
     cc.workspace_bytes = need;
     cudaError_t e;
-    if (pair_supported(l, c.batch, c.n) && !c.packed_list)
+    if (c.n == 1 && !c.packed_list && ring_supported(1, &l, &cc))
+        e = launch_gemv_ring(1, &l, &cc, (cudaStream_t)stream);
+    else if (pair_supported(l, c.batch, c.n) && !c.packed_list)
         e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && batch_supported(l, c.batch))
         e = launch_gemv_batch(l, cc, (cudaStream_t)stream);
@@ -129,6 +131,8 @@ int xfp_gemv_multi(int32_t n, const xfp_desc* const* descs, const void* const* p
         cs[j] = GemvCall{packed[j], x[j], y[j], nullptr, nullptr, nullptr, 1, 1, y_is_fp16, workspace[j],
                          workspace_bytes_for(ls[j])};
     }
+    if (n > 1 && ring_supported(n, ls, cs))
+        return launch_gemv_ring(n, ls, cs, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
     if (multi_supported(n, ls, cs))
         return launch_gemv_multi(n, ls, cs, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
     for (int j = 0; j < n; ++j) {   // shapes the shared launch does not cover: one call each, same results
@@ -168,6 +172,7 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
 void xfp_debug_set_ksplit(int ks) { pair_set_ksplit_override(ks); }
 void xfp_debug_set_prefetch(int d) { pair_set_prefetch(d); }
 void xfp_debug_set_mode(int m) { pair_set_debug(m); }
+void xfp_debug_ring(int what, long long v) { ring_set(what, v); }
 void xfp_debug_set_small(int v) { pair_set_small(v); }
 void xfp_debug_set_trace(void* p, size_t calls) { pair_set_trace(p, calls); }
 
