@@ -219,22 +219,9 @@ def run_xfp(args, rank: int, world: int):
     xd = [torch.from_numpy(x.view(np.int16)).to(dev).view(torch.float16) for x in x16]
     yd = [torch.empty((1, ROWS), dtype=torch.float16, device=dev) for _ in range(n_calls)]
 
-    # q, k and v of a block do not depend on one another: one xfp_gemv_multi launch; o is its own call
-    multi = {}
-    if args.qkv == "multi":
-        for j in range(0, n_calls, 4):
-            multi[j] = xfp.MultiCall(pms[j:j + 3], xd[j:j + 3], yd[j:j + 3], True)
-    n_launches = n_calls - 2 * len(multi)
-
     def step():
-        j = 0
-        while j < n_calls:
-            if j in multi:
-                multi[j].launch(stream)
-                j += 3
-            else:
-                pms[j].gemv(xd[j], y=yd[j], y_fp16=True)
-                j += 1
+        for pm, x, y in zip(pms, xd, yd):
+            pm.gemv(x, y=y, y_fp16=True)
 
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
@@ -314,15 +301,14 @@ def run_xfp(args, rank: int, world: int):
         "config": {"workload": "attention_block_v2", "layers": args.layers, "calls_per_step": n_calls, "rows": ROWS,
                    "cols": COLS, "bits": [n[2] for n in names[:4]], "mode": "V2", "batch": 1, "outlier_rate": 0.009,
                    "bytes_per_step": step_bytes, "l2": "weights of a step (%.0f MB) exceed L2; none re-read before "
-                   "126 MB of other weights passed" % (step_bytes / 1e6), "launch": "one CUDA graph per step; " + ("q/k/v of a block in one xfp_gemv_multi launch, o in its own"
-                                                            if multi else "one launch per projection")},
+                   "126 MB of other weights passed" % (step_bytes / 1e6), "launch": "one CUDA graph per step"},
         "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
                      "peak_kind": peak_kind, "frac_of_nominal_8000": per_gpu / NOMINAL_HBM_GBS,
                      "traffic": sum(NCU_TRAFFIC_BYTES_PER_LAUNCH[n[2]] for n in names) / n_calls, "bytes_per_launch": step_bytes / n_calls,
                      "kernel": "gemv (all calls of a step)"},
         "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": n_calls * COLS * 2,
                 "d2h_bytes_per_step": n_calls * ROWS * 2, "us_per_call": e2e_ms / args.steps * 1e3 / n_calls},
-        "gpu_launches": args.steps * n_launches,
+        "gpu_launches": args.steps * n_calls,
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
@@ -347,8 +333,6 @@ def main():
     ap.add_argument("--layers", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--qkv", default="single", choices=["multi", "single"],
-                    help="q/k/v of a block in one launch (xfp_gemv_multi) or one launch per projection")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -111,17 +111,6 @@ int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* str
 int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
                      void* const* y, int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
 
-/* n <= 8 independent batch-1 GEMVs in one launch, each with its own descriptor (bit widths and shapes may
- * differ; V2 or V2a) -- e.g. the q, k and v projections of an attention block, which read the same x
- * ("Fused Decode Kernel"; the paper notes that kernel-launch overhead dominates single-stream decode).
- * descs, packed, x, y, workspace, workspace_bytes are HOST arrays of n entries; packed[j], x[j] ([cols_j]
- * fp16), y[j] ([rows_j]) and workspace[j] are device pointers as for xfp_gemv_v2.  Small V2 matrices
- * (rows <= 4736, 3..5 bits) share one kernel and one schedule; any other mix runs as n ordinary calls
- * on the stream with identical results. */
-int xfp_gemv_multi(int32_t n, const xfp_desc* const* descs, const void* const* packed, const uint16_t* const* x,
-                   void* const* y, int32_t y_is_fp16, void* const* workspace, const size_t* workspace_bytes,
-                   void* stream);
-
 /* Convenience for callers whose activations live in host memory: copies x_host (pinned for
  * asynchrony) to x_dev, runs the GEMV for desc->mode, copies y_dev to y_host, all on `stream`.
  * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller. */

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 EXPORTS = ("xfp_packed_size", "xfp_pack", "xfp_gemv_v2", "xfp_gemv_v2a", "xfp_gemv_grouped", "xfp_gemv_host",
-           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_multi")
+           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc")
 
 
 class XfpError(RuntimeError):
@@ -55,7 +55,6 @@ def load_library() -> C.CDLL:
     lib.xfp_gemv_host.argtypes = [dp, vp, vp, vp, i32, vp, vp, i32, vp, sz, vp]
     lib.xfp_dequant.argtypes = [dp, vp, vp, vp]
     lib.xfp_gemv_v2_noalloc.argtypes = [dp, vp, vp, i32, vp, i32, vp]
-    lib.xfp_gemv_multi.argtypes = [i32, vp, vp, vp, vp, i32, vp, vp, vp]
     lib.xfp_status_str.argtypes = [C.c_int]
     lib.xfp_status_str.restype = C.c_char_p
     for name in EXPORTS:
@@ -127,31 +126,6 @@ def xfp_gemv_host(desc, packed, x_host: torch.Tensor, x_dev, batch, y_host: torc
                                         _ptr(y_host), _ptr(y_dev), int(bool(y_is_fp16)), _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), _stream(stream)),
            "xfp_gemv_host")
-
-
-class MultiCall:
-    """Marshalled argument arrays of one xfp_gemv_multi call (build once, launch many times)."""
-
-    def __init__(self, mats: Sequence["PackedMatrix"], xs: Sequence[torch.Tensor], ys: Sequence[torch.Tensor],
-                 y_is_fp16: bool):
-        n = len(mats)
-        self.n, self.y_is_fp16 = n, int(bool(y_is_fp16))
-        self.keep = (list(mats), list(xs), list(ys))
-        self.descs = (C.POINTER(XfpDesc) * n)(*[C.pointer(m.desc) for m in mats])
-        self.packed = (C.c_void_p * n)(*[m.packed.data_ptr() for m in mats])
-        self.x = (C.c_void_p * n)(*[t.data_ptr() for t in xs])
-        self.y = (C.c_void_p * n)(*[t.data_ptr() for t in ys])
-        self.ws = (C.c_void_p * n)(*[m.workspace.data_ptr() for m in mats])
-        self.wsb = (C.c_size_t * n)(*[m.workspace.numel() * m.workspace.element_size() for m in mats])
-
-    def launch(self, stream=None) -> None:
-        _check(load_library().xfp_gemv_multi(self.n, self.descs, self.packed, self.x, self.y, self.y_is_fp16,
-                                             self.ws, self.wsb, _stream(stream)), "xfp_gemv_multi")
-
-
-def xfp_gemv_multi(mats, xs, ys, y_is_fp16, stream=None) -> None:
-    """Several independent batch-1 GEMVs (their own descriptors) in one launch."""
-    MultiCall(mats, xs, ys, y_is_fp16).launch(stream)
 
 
 def xfp_gemv_v2_noalloc(desc, packed, x, batch, y, y_is_fp16, stream=None) -> None:

@@ -46,9 +46,7 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     GemvCall cc = c;
     cc.workspace_bytes = need;
     cudaError_t e;
-    if (c.n == 1 && !c.packed_list && ring_supported(1, &l, &cc))
-        e = launch_gemv_ring(1, &l, &cc, (cudaStream_t)stream);
-    else if (pair_supported(l, c.batch, c.n) && !c.packed_list)
+    if (pair_supported(l, c.batch, c.n) && !c.packed_list)
         e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && batch_supported(l, c.batch))
         e = launch_gemv_batch(l, cc, (cudaStream_t)stream);
@@ -114,34 +112,6 @@ int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed,
     return gemv_common(desc, desc->mode, c, stream);
 }
 
-int xfp_gemv_multi(int32_t n, const xfp_desc* const* descs, const void* const* packed, const uint16_t* const* x,
-                   void* const* y, int32_t y_is_fp16, void* const* workspace, const size_t* workspace_bytes,
-                   void* stream) {
-    if (n < 1 || n > 8) return XFP_ERR_SHAPE;
-    if (!descs || !packed || !x || !y || !workspace || !workspace_bytes) return XFP_ERR_NULL;
-    Layout ls[8];
-    GemvCall cs[8];
-    for (int j = 0; j < n; ++j) {
-        const int st = check_desc(descs[j]);
-        if (st) return st;
-        if (!packed[j] || !x[j] || !y[j] || !workspace[j]) return XFP_ERR_NULL;
-        if (!aligned16(packed[j]) || !aligned16(x[j]) || !aligned16(y[j]) || !aligned16(workspace[j])) return XFP_ERR_ALIGN;
-        ls[j] = layout_of(descs[j]);
-        if (workspace_bytes[j] < workspace_bytes_for(ls[j])) return XFP_ERR_BUFFER_TOO_SMALL;
-        cs[j] = GemvCall{packed[j], x[j], y[j], nullptr, nullptr, nullptr, 1, 1, y_is_fp16, workspace[j],
-                         workspace_bytes_for(ls[j])};
-    }
-    if (n > 1 && ring_supported(n, ls, cs))
-        return launch_gemv_ring(n, ls, cs, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
-    if (multi_supported(n, ls, cs))
-        return launch_gemv_multi(n, ls, cs, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
-    for (int j = 0; j < n; ++j) {   // shapes the shared launch does not cover: one call each, same results
-        const int st = gemv_common(descs[j], descs[j]->mode, cs[j], stream);
-        if (st) return st;
-    }
-    return XFP_OK;
-}
-
 int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* stream) {
     int st = check_desc(desc);
     if (st) return st;
@@ -172,7 +142,6 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
 void xfp_debug_set_ksplit(int ks) { pair_set_ksplit_override(ks); }
 void xfp_debug_set_prefetch(int d) { pair_set_prefetch(d); }
 void xfp_debug_set_mode(int m) { pair_set_debug(m); }
-void xfp_debug_ring(int what, long long v) { ring_set(what, v); }
 void xfp_debug_set_small(int v) { pair_set_small(v); }
 void xfp_debug_set_trace(void* p, size_t calls) { pair_set_trace(p, calls); }
 

@@ -75,10 +75,8 @@ __device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
     }
 }
 
-// The work of one CTA: K slice `slice` of `nslices` (spp super-chunks each) of block `blk`.
 template <int N, int NB, int RPL, int W>
-__device__ __forceinline__ void pair_body(const PairArgs& a, const int blk, const int slice, const int nslices,
-                                          const int spp) {
+__global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
     constexpr int E = 1 << N;
     constexpr int T = E * E;                   // pair-table entries per channel
     constexpr int ROWS = 32 * RPL;             // channels per block
@@ -98,8 +96,20 @@ __device__ __forceinline__ void pair_body(const PairArgs& a, const int blk, cons
     uint16_t* xs = (uint16_t*)(smem + kTabBytes);               // [NB][K]
     float* red = (float*)(xs + (size_t)NB * K);                 // [W][NB][ROWS]
 
-    const int sc0 = slice * spp;
-    const int nsc = max(0, min(a.SC, sc0 + spp) - sc0);
+    // ---- this CTA's block and K slice
+    int blk, slice, nslices, sc0, nsc;
+    {
+        int tier = 0;
+#pragma unroll
+        for (int i = 1; i < 4; ++i)
+            if ((int)blockIdx.x >= a.tier_cta[i]) tier = i;
+        const int c = blockIdx.x - a.tier_cta[tier];
+        nslices = a.tier_kst[tier];
+        blk = a.tier_blk[tier] + c / nslices;
+        slice = c % nslices;
+        sc0 = slice * a.tier_spp[tier];
+        nsc = max(0, min(a.SC, sc0 + a.tier_spp[tier]) - sc0);
+    }
     const int blk0 = RPL * blk;
     const int blk1 = min(RPL * blk + (RPL - 1), a.RB - 1);   // clamped when RB is odd; its results are dropped
     const int gw = slice * W + warp, ostride = nslices * W;
@@ -400,60 +410,6 @@ __device__ __forceinline__ void pair_body(const PairArgs& a, const int blk, cons
     }
 }
 
-template <int N, int NB, int RPL, int W>
-__global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
-    int tier = 0;
-#pragma unroll
-    for (int i = 1; i < 4; ++i)
-        if ((int)blockIdx.x >= a.tier_cta[i]) tier = i;
-    const int c = blockIdx.x - a.tier_cta[tier];
-    const int nslices = a.tier_kst[tier];
-    pair_body<N, NB, RPL, W>(a, a.tier_blk[tier] + c / nslices, c % nslices, nslices, a.tier_spp[tier]);
-}
-
-// Several independent V2 GEMVs (batch 1) in one launch -- e.g. the q, k and v projections of an attention
-// block, which read the same x.  The problems may differ in bit width and shape; their blocks form one
-// pool that is scheduled like a single matrix (whole rounds unsplit, tiers of finer K slices for the
-// rest), so small matrices share the launch, dependency wait and tail instead of paying them each.
-constexpr int kMultiMax = 8;
-
-struct MultiArgs {
-    PairArgs p[kMultiMax];
-    int bits[kMultiMax];
-    int blk_begin[kMultiMax + 1];   // pooled block index of each problem's first block
-    int n;
-    int tier_cta[5], tier_blk[4], tier_kst[4];
-};
-
-__global__ void __launch_bounds__(512, 1) gemv_multi_kernel(const __grid_constant__ MultiArgs m) {
-    int tier = 0;
-#pragma unroll
-    for (int i = 1; i < 4; ++i)
-        if ((int)blockIdx.x >= m.tier_cta[i]) tier = i;
-    const int c = blockIdx.x - m.tier_cta[tier];
-    const int nslices = m.tier_kst[tier];
-    const int pooled = m.tier_blk[tier] + c / nslices, slice = c % nslices;
-    int j = 0;
-#pragma unroll
-    for (int i = 1; i < kMultiMax; ++i)
-        if (i < m.n && pooled >= m.blk_begin[i]) j = i;
-    const PairArgs& a = m.p[j];
-    const int blk = pooled - m.blk_begin[j];
-    // slices of this problem: equal cuts of its own K, at least one super-chunk each
-    const int ns = min(nslices, a.SC);
-    const int spp = (a.SC + ns - 1) / ns;
-    const int ns_eff = (a.SC + spp - 1) / spp;
-    if (slice >= ns_eff) {   // this problem's K is too short for the tier's cut: nothing to do here
-        asm volatile("griddepcontrol.launch_dependents;");
-        return;
-    }
-    switch (m.bits[j]) {
-        case 3: pair_body<3, 1, 1, 16>(a, blk, slice, ns_eff, spp); break;
-        case 4: pair_body<4, 1, 1, 16>(a, blk, slice, ns_eff, spp); break;
-        default: pair_body<5, 1, 1, 16>(a, blk, slice, ns_eff, spp); break;
-    }
-}
-
 // ------------------------------------------------------------------------------------ host side
 
 static unsigned long long* g_pair_trace = nullptr;
@@ -492,53 +448,44 @@ static int pow2_floor(int v) {
     return p;
 }
 
-// Tiers for `blocks` equal blocks on S CTA slots (kmax: finest allowed cut).  Returns the number of tiers;
-// nb[i] blocks are cut into kk[i] slices.
-static int compute_tiers(int blocks, int S, int kmax, bool allow_cluster, int nb[4], int kk[4], int* cluster) {
-    int nt = 0;
-    *cluster = 0;
-    for (int i = 0; i < 4; ++i) { nb[i] = 0; kk[i] = 1; }
-    if (g_pair_ks_override > 0) {
-        nb[0] = blocks; kk[0] = g_pair_ks_override; return 1;
-    }
-    if (blocks * 2 <= S) {
-        // fewer blocks than half the CTA slots: cut every block into 2, 4 or 8 K slices (a cluster when allowed)
-        int kst = 1;
-        while (kst < 8 && blocks * kst * 2 <= S && kst * 2 <= kmax) kst *= 2;
-        nb[0] = blocks; kk[0] = kst;
-        *cluster = allow_cluster && kst > 1;
-        return 1;
-    }
-    // whole rounds unsplit, then tiers of finer slices for the blocks of the last, partial round
-    const int full = (blocks / S) * S;
-    int remaining = blocks - full;
-    if (full > 0) { nb[nt] = full; kk[nt] = 1; ++nt; }
-    if (full == 0) { nb[nt] = remaining; kk[nt] = 1; ++nt; remaining = 0; }   // a single partial round
-    int k = 2;
-    while (remaining > 0 && nt < 4) {
-        if (k > kmax) { nb[nt] = remaining; kk[nt] = kmax; ++nt; remaining = 0; break; }
-        const int cap = S / k;   // blocks whose k slices fill one round
-        if (remaining <= cap || nt == 3) {
-            int kl = pow2_floor(S / remaining > 1 ? S / remaining : 1);
-            if (kl > kmax) kl = kmax;
-            if (kl > 64) kl = 64;
-            if (kl < k && remaining <= cap) kl = k;
-            nb[nt] = remaining; kk[nt] = kl < 1 ? 1 : kl; ++nt; remaining = 0;
-        } else {
-            nb[nt] = cap; kk[nt] = k; ++nt; remaining -= cap;
-            k *= 2;
-        }
-    }
-    return nt;
-}
-
 static PairSchedule pair_schedule(const Layout& l) {
     const PairConfig cfg = pair_config(l);
     PairSchedule sc{};
     sc.blocks = (l.RB + cfg.rpl - 1) / cfg.rpl;
+    const int S = cfg.slots;
     const int kmax = l.SC / 4 > 1 ? pow2_floor(l.SC / 4) : 1;   // keep K slices of at least 512 weights
-    int nb[4], kk[4];
-    const int nt = compute_tiers(sc.blocks, cfg.slots, kmax, true, nb, kk, &sc.cluster);
+    int nb[4] = {0, 0, 0, 0}, kk[4] = {1, 1, 1, 1};
+    int nt = 0;
+    if (g_pair_ks_override > 0) {
+        nb[0] = sc.blocks; kk[0] = g_pair_ks_override; nt = 1;
+    } else if (sc.blocks * 2 <= S) {
+        // fewer blocks than half the CTA slots: cut every block into 2, 4 or 8 K slices that form a cluster
+        int kst = 1;
+        while (kst < 8 && sc.blocks * kst * 2 <= S && kst * 2 <= kmax) kst *= 2;
+        nb[0] = sc.blocks; kk[0] = kst; nt = 1;
+        sc.cluster = kst > 1;
+    } else {
+        // whole rounds unsplit, then tiers of finer slices for the blocks of the last, partial round
+        const int full = (sc.blocks / S) * S;
+        int remaining = sc.blocks - full;
+        if (full > 0) { nb[nt] = full; kk[nt] = 1; ++nt; }
+        if (full == 0) { nb[nt] = remaining; kk[nt] = 1; ++nt; remaining = 0; }   // a single partial round
+        int k = 2;
+        while (remaining > 0 && nt < 4) {
+            if (k > kmax) { nb[nt] = remaining; kk[nt] = kmax; ++nt; remaining = 0; break; }
+            const int cap = S / k;   // blocks whose k slices fill one round
+            if (remaining <= cap || nt == 3) {
+                int kl = pow2_floor(S / remaining > 1 ? S / remaining : 1);
+                if (kl > kmax) kl = kmax;
+                if (kl > 64) kl = 64;
+                if (kl < k && remaining <= cap) kl = k;
+                nb[nt] = remaining; kk[nt] = kl < 1 ? 1 : kl; ++nt; remaining = 0;
+            } else {
+                nb[nt] = cap; kk[nt] = k; ++nt; remaining -= cap;
+                k *= 2;
+            }
+        }
+    }
     sc.ntiers = nt;
     int cta = 0, blk = 0;
     for (int i = 0; i < 4; ++i) {
@@ -601,87 +548,23 @@ static cudaError_t launch_pair(const PairArgs& a, int grid, size_t smem, cudaStr
     return cudaLaunchKernelEx(&cfg, gemv_pair_kernel<N, NB, RPL, W>, a);
 }
 
-static void fill_pair_args(PairArgs& a, const Layout& l, const GemvCall& c, const PairConfig& cfg, int blocks) {
-    a.off = offsets_of(l);
-    a.packed = c.packed; a.x = c.x; a.y = c.y;
-    a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
-    a.blocks = blocks;
-    a.rows_ws = blocks * 32 * cfg.rpl;
-    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
-    a.trace = nullptr;
-    a.tickets = (int*)c.workspace;
-    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
-}
-
-// Can these problems share one launch?  All V2, batch 1, 3..5 bits, and the one-row-per-lane / 16-warp
-// configuration (what a single call of such a matrix would use as well).
-bool multi_supported(int n, const Layout* ls, const GemvCall* cs) {
-    if (n < 2 || n > kMultiMax) return false;
-    for (int j = 0; j < n; ++j) {
-        if (!pair_supported(ls[j], cs[j].batch, 1) || cs[j].batch != 1) return false;
-        const PairConfig cfg = pair_config(ls[j]);
-        if (cfg.rpl != 1 || cfg.warps != 16 || ls[j].bits < 3) return false;
-        if (cs[j].y_is_fp16 != cs[0].y_is_fp16) return false;
-    }
-    return true;
-}
-
-cudaError_t launch_gemv_multi(int n, const Layout* ls, const GemvCall* cs, cudaStream_t s) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    MultiArgs m{};
-    m.n = n;
-    size_t smem = 0;
-    int total = 0, sc_min = 1 << 30;
-    for (int j = 0; j < n; ++j) {
-        const PairConfig cfg = pair_config(ls[j]);
-        fill_pair_args(m.p[j], ls[j], cs[j], cfg, ls[j].RB);
-        m.p[j].cluster = 0;
-        m.bits[j] = ls[j].bits;
-        m.blk_begin[j] = total;
-        total += ls[j].RB;
-        const size_t sm = pair_smem_bytes(ls[j], 1);
-        if (sm > smem) smem = sm;
-        if (ls[j].SC < sc_min) sc_min = ls[j].SC;
-    }
-    m.blk_begin[n] = total;
-    const int kmax = sc_min / 4 > 1 ? pow2_floor(sc_min / 4) : 1;
-    int nb[4], kk[4], cluster = 0;
-    const int nt = compute_tiers(total, 148, kmax, false, nb, kk, &cluster);
-    int cta = 0, blk = 0;
-    for (int i = 0; i < 4; ++i) {
-        m.tier_cta[i] = i < nt ? cta : 0x7fffffff;
-        m.tier_blk[i] = blk;
-        m.tier_kst[i] = i < nt ? kk[i] : 1;
-        if (i < nt) { cta += nb[i] * kk[i]; blk += nb[i]; }
-    }
-    m.tier_cta[4] = cta;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)cta, 1, 1);
-    cfg.blockDim = dim3(512, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_multi_kernel, m);
-}
-
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s) {
     const PairConfig cfg = pair_config(l);
     const PairSchedule sch = pair_schedule(l);
     PairArgs a{};
-    fill_pair_args(a, l, c, cfg, sch.blocks);
+    a.off = offsets_of(l);
+    a.packed = c.packed; a.x = c.x; a.y = c.y;
+    a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
+    a.blocks = sch.blocks;
+    a.rows_ws = sch.blocks * 32 * cfg.rpl;
     for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
     for (int i = 0; i < 4; ++i) { a.tier_blk[i] = sch.tier_blk[i]; a.tier_kst[i] = sch.tier_kst[i]; a.tier_spp[i] = sch.tier_spp[i]; }
     a.cluster = sch.cluster && g_pair_ks_override == 0;
+    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
+    a.trace = nullptr;
     if (g_pair_trace && g_pair_trace_idx < g_pair_trace_calls) a.trace = g_pair_trace + (g_pair_trace_idx++) * 1024 * 8;
+    a.tickets = (int*)c.workspace;
+    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
     const size_t smem = pair_smem_bytes(l, c.batch);
     if (cfg.rpl == 1) {
         switch (l.bits * 10 + c.batch) {

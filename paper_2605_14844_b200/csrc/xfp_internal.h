@@ -52,10 +52,6 @@ void pair_set_debug(int m);
 void pair_set_small(int v);
 void pair_set_trace(void* p, size_t calls);
 
-// Several V2 problems (batch 1) in one launch; see xfp_gemv_pair.cu.
-bool multi_supported(int n, const Layout* ls, const GemvCall* cs);
-cudaError_t launch_gemv_multi(int n, const Layout* ls, const GemvCall* cs, cudaStream_t s);
-
 // Fast V2a path (per-bank library + mma.sync fragments, one or several blobs); see xfp_gemv_v2a.cu.
 bool v2a_supported(const Layout& l, int batch);
 size_t v2a_workspace_bytes(const Layout& l);
@@ -65,21 +61,10 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
 bool batch_supported(const Layout& l, int batch);
 cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s);
 
-// Persistent V2 path at batch 1, one or several problems per launch; see xfp_gemv_ring.cu.
-bool ring_supported(int n, const Layout* ls, const GemvCall* cs);
-size_t ring_workspace_bytes(const Layout& l);
-cudaError_t launch_gemv_ring(int n, const Layout* ls, const GemvCall* cs, cudaStream_t s);
-void ring_set(int what, long long v);
-
-// Workspace of one problem: the largest need of the kernels that may serve it, then 256 bytes whose first
-// word is a status flag (nonzero once a kernel gave up on an internal wait; never cleared by the library).
-inline size_t status_offset(const Layout& l) {
+inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);
-    if (p > w) w = p;
-    if (!l.mode && ring_workspace_bytes(l) > w) w = ring_workspace_bytes(l);
-    return align256(w);
+    return w > p ? w : p;
 }
-inline size_t workspace_bytes_for(const Layout& l) { return status_offset(l) + 256; }
 
 }  // namespace xfp

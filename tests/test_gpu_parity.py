@@ -180,37 +180,6 @@ def test_grouped_matches_single_calls():
         assert np.all(np.abs(single[0].cpu().numpy() - ys[j].cpu().numpy()) <= 0.05 * TOL * absum[0])
 
 
-@pytest.mark.parametrize("shapes", [
-    # q/k/v-like: same K, mixed bit widths and row counts (ragged last row-block), one shared launch
-    [(0, 200, 1536, 4), (0, 96, 1536, 5), (0, 70, 1536, 3)],
-    # different K per problem: the pooled cut is finer than the short problem's K allows
-    [(0, 64, 4096, 4), (0, 64, 256, 5), (0, 33, 128, 4), (0, 1, 640, 3)],
-    # more than one round of row-blocks in the pool
-    [(0, 3072, 512, 4), (0, 2048, 512, 5)],
-    # a mix the shared launch does not cover (V2a member, 2-bit member): falls back to separate calls
-    [(0, 128, 1024, 4), (1, 128, 1024, 3), (0, 96, 1024, 2)],
-])
-def test_multi_launch_within_bound(shapes):
-    qs = [synth.random_quantized(mode, rows, cols, bits, 0.01, seed=900 + 7 * j + rows)
-          for j, (mode, rows, cols, bits) in enumerate(shapes)]
-    pms = [xfp.pack_tensors(q, col_bits=16) for q in qs]
-    x16s = [synth.activations(1, q.cols, seed=40 + j) for j, q in enumerate(qs)]
-    xs = [_x_dev(x) for x in x16s]
-    for y_fp16 in (False, True):
-        ys = [torch.full((q.rows,), float("nan"), dtype=torch.float16 if y_fp16 else torch.float32, device="cuda")
-              for q in qs]
-        call = xfp.MultiCall(pms, xs, ys, y_fp16)
-        call.launch()
-        call.launch()                      # tickets must be back at zero after the first launch
-        torch.cuda.synchronize()
-        for q, pm, x16, y in zip(qs, pms, x16s, ys):
-            ref, absum = xo.gemv(to_oracle(q), x16)
-            got = y.float().cpu().numpy().astype(np.float64)
-            assert np.all(np.abs(got - ref[0]) <= TOL * absum[0] + 1e-30)
-            nblk = (q.rows + 31) // 32
-            assert int(pm.workspace[: nblk * 4].view(torch.int32).abs().sum().item()) == 0
-
-
 def test_gemv_host_entry():
     q = synth.random_quantized(0, 96, 512, 5, 0.01, seed=97)
     pm = xfp.pack_tensors(q)
