@@ -142,6 +142,7 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
 void xfp_debug_set_ksplit(int ks) { pair_set_ksplit_override(ks); }
 void xfp_debug_set_prefetch(int d) { pair_set_prefetch(d); }
 void xfp_debug_set_mode(int m) { pair_set_debug(m); }
+void xfp_debug_v2a_pair(int v) { v2a_set_pair(v); }
 void xfp_debug_set_small(int v) { pair_set_small(v); }
 void xfp_debug_set_trace(void* p, size_t calls) { pair_set_trace(p, calls); }
 

@@ -8,11 +8,18 @@
 // format's 128-weight groups, so a lane meets one (id, scale, mid) triple per channel and
 // super-chunk.
 //
-// Look-up.  Every lane may need a different library entry, so a pair table per entry does not fit
-// (L * 4^N * 32 banks).  Instead the library itself is replicated once per bank: word
-// (id * 2^N + q) * 32 + lane holds lib[id][q] (fp16 in the low half).  Lane l only touches bank l, so
-// look-ups are conflict free for any mix of ids; one look-up decodes one weight and a PRMT joins two
-// of them into the half2 the tensor pipe wants.
+// Look-up.  Every lane may need a different library codebook, so the tables cannot be private to a
+// channel as in the V2 kernel.  Two layouts, chosen by the bit width:
+//   * N <= 3 (the routed-MoE mode): PAIR tables of the whole library, replicated 16 times: word
+//     (id * 4^N + pair) * 16 + (lane & 15) holds the half2 (lib[id][pair & (E-1)], lib[id][pair >> N]).
+//     One look-up decodes two weights.  Lanes l and l+16 share a copy; their words fall into the
+//     same bank only when their pair indices have the same parity (the bank is
+//     16 * (pair & 1) + (lane & 15)), so a look-up costs 1.5 shared-memory wavefronts on average,
+//     0.75 per weight.  128 KB at N = 3, L = 32: one CTA of 12 or 16 warps per SM.
+//   * N >= 4: the pair tables would not fit, so the library itself is replicated once per bank: word
+//     (id * 2^N + q) * 32 + lane holds lib[id][q] (fp16 in the low half).  Lane l only touches bank l;
+//     one look-up decodes one weight and a PRMT joins two of them into the half2 the tensor pipe
+//     wants.  Two CTAs of 8 warps per SM.
 //
 // Multiply-accumulate.  The half2 of a lane's two channels form the A fragment of
 // mma.sync.m16n8k16 and x sits on the diagonal lanes of the B fragment (see xfp_gemv_pair.cu).  The
@@ -28,8 +35,6 @@
 
 namespace xfp {
 
-constexpr int kAWarps = 8;
-constexpr int kAThreads = kAWarps * 32;
 constexpr int kARows = 64;
 constexpr int kASlots = 4;
 
@@ -46,6 +51,7 @@ struct V2aArgs {
     int rows, cols, RB, SC, rows_ws, ell_slots, L;
     int nb, y_is_fp16;
     int blocks, n_full, kst, sc_per_split;
+    int items_x, n;   // work items per blob (whole blocks + K slices), blobs
 };
 
 __device__ __forceinline__ void mma16816a(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -72,19 +78,54 @@ __device__ __forceinline__ uint32_t entry_addr(const uint32_t* w, int j, uint32_
     return (v & mask) | base;
 }
 
-template <int N, int NB>
-__global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a) {
+// Byte offset (pair << 6) of pair p (compile time) of a 128-weight stream, merged with `base`
+// (= id * 4^N * 64 + (lane & 15) * 4; the pair field occupies bits 6 .. 6+2N, which base leaves clear).
+template <int N>
+__device__ __forceinline__ uint32_t pair_entry_addr(const uint32_t* w, int p, uint32_t base) {
+    constexpr uint32_t mask = ((1u << (2 * N)) - 1u) << 6;
+    const int bit = p * 2 * N, wi = bit >> 5, off = bit & 31;
+    uint32_t v;
+    if (off + 2 * N > 32)
+        v = __funnelshift_r(w[wi], w[wi + 1], off) << 6;
+    else if (off >= 6)
+        v = w[wi] >> (off - 6);
+    else
+        v = w[wi] << (6 - off);
+    return (v & mask) | base;
+}
+
+template <int N, int NB, int W, bool PAIR>
+__global__ void __launch_bounds__(W * 32, PAIR ? 1 : 2) gemv_v2a_kernel(const V2aArgs a) {
     constexpr int E = 1 << N;
+    constexpr int kAWarps = W;
+    constexpr int kAThreads = W * 32;
     extern __shared__ __align__(16) unsigned char smem[];
-    // [library L*E*128 bytes | x fp16 [NB][K] | xg fp32 [NB][SC] | red fp32 [W][NB][64]]
+    // [library tables | x fp16 [NB][K] | xg fp32 [NB][SC] | red fp32 [W][NB][64] | library copy]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
-    const int prob = blockIdx.y;
+    const int K = a.SC * kSuper;
+    const int tab_bytes = PAIR ? a.L * E * E * 64 : a.L * E * 128;
+    unsigned char* tab = smem;
+    uint16_t* xs = (uint16_t*)(smem + tab_bytes);             // [NB][K]
+    float* xg = (float*)(xs + (size_t)NB * K);                // [NB][SC]
+    float* red = xg + NB * a.SC;                              // [W][NB][64]
+    __shared__ int s_last;
+
+    // the library the tables were built from, on the next 16-byte boundary (NB * SC floats of xg precede red)
+    uint4* libcopy = (uint4*)(((uintptr_t)(red + (size_t)kAWarps * NB * kARows) + 15) & ~(uintptr_t)15);
+    bool have_tables = false;
+    bool waited = false;
+    const uint16_t* x_staged = nullptr;
+
+    // ---- work items: (blob, whole block or K slice of a block), dealt round-robin to the CTAs of the launch
+#pragma unroll 1
+    for (int item = blockIdx.x; item < a.items_x * a.n; item += gridDim.x) {
+    const int prob = item / a.items_x, bx = item - prob * a.items_x;
     int blk, ks, KS, spp;
-    if ((int)blockIdx.x < a.n_full) {
-        blk = blockIdx.x; ks = 0; KS = 1; spp = a.SC;
+    if (bx < a.n_full) {
+        blk = bx; ks = 0; KS = 1; spp = a.SC;
     } else {
-        const int t = blockIdx.x - a.n_full;
+        const int t = bx - a.n_full;
         blk = a.n_full + t / a.kst; ks = t % a.kst; KS = a.kst; spp = a.sc_per_split;
     }
     const void* packed = a.packed_list ? a.packed_list[prob] : a.packed;
@@ -93,13 +134,6 @@ __global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a)
     const Blob b = blob_at(packed, a.off);
     const int sc0 = ks * spp;
     const int nsc = max(0, min(a.SC, sc0 + spp) - sc0);
-    const int K = a.SC * kSuper;
-    const int tab_bytes = a.L * E * 128;
-
-    unsigned char* tab = smem;
-    uint16_t* xs = (uint16_t*)(smem + tab_bytes);             // [NB][K]
-    float* xg = (float*)(xs + (size_t)NB * K);                // [NB][SC]
-    float* red = xg + NB * a.SC;                              // [W][NB][64]
 
     const int blk0 = 2 * blk;
     const int blk1 = min(2 * blk + 1, a.RB - 1);              // clamped when RB is odd; its results are dropped
@@ -169,31 +203,66 @@ __global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a)
     };
     if (ell_slots) fetch_slots(0);
 
-    // ---- (1) library, one copy per bank: word (e * 32 + lane) = lib[e] for every lane
-    for (int e = warp; e < a.L * E; e += kAWarps)
-        *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
-
-    // ---- (2) x: wait for the previous kernel, stage fp16 x (all of K) and the group sums X_g
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // ---- (1) library tables (after the item's first loads are on their way).  The blobs of a launch normally share one library (one per layer), so the tables are
+    //      built once per CTA; a blob whose library differs from the one they were built from rebuilds them.
     {
-        const int nvec = NB * (K / 8);
-        for (int t = threadIdx.x; t < nvec; t += kAThreads) {
-            const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (bb < a.nb) v = __ldg((const uint4*)(x + (size_t)bb * a.cols + kk));
-            *(uint4*)(xs + (size_t)t * 8) = v;
+        const uint4* cb4 = (const uint4*)b.cb;
+        const int nvec = a.L * E / 8;   // the library in 16-byte vectors (L * E is a multiple of 8)
+        int differs = !have_tables;
+        if (have_tables)
+            for (int i = threadIdx.x; i < nvec; i += kAThreads) {
+                const uint4 u = __ldg(cb4 + i), v = libcopy[i];
+                differs |= (u.x != v.x) | (u.y != v.y) | (u.z != v.z) | (u.w != v.w);
+            }
+        if (__syncthreads_or(differs)) {
+            for (int i = threadIdx.x; i < nvec; i += kAThreads) libcopy[i] = __ldg(cb4 + i);
+            if (PAIR) {
+                // pair tables, 16 copies: words (id * E*E + pair) * 16 .. + 15 hold the same half2
+                for (int e = threadIdx.x; e < a.L * E * E; e += kAThreads) {
+                    const int id = e / (E * E), pr = e % (E * E);
+                    const uint32_t v = (uint32_t)__ldg(b.cb + id * E + (pr & (E - 1))) |
+                                       ((uint32_t)__ldg(b.cb + id * E + (pr >> N)) << 16);
+                    const uint4 v4 = make_uint4(v, v, v, v);
+                    uint4* dst = (uint4*)(tab + (size_t)e * 64);
+                    dst[0] = v4; dst[1] = v4; dst[2] = v4; dst[3] = v4;
+                }
+            } else {
+                // one copy per bank: word (e * 32 + lane) = lib[e] for every lane
+                for (int e = warp; e < a.L * E; e += kAWarps)
+                    *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+            }
+            have_tables = true;
         }
     }
-    __syncthreads();
-    for (int u = warp; u < NB * a.SC; u += kAWarps) {   // X_g: 128 values per group, 4 per lane, fixed butterfly
-        const uint2 hv = *(const uint2*)(xs + (size_t)u * kSuper + lane * 4);
-        const float2 p0 = __half22float2(*(const __half2*)&hv.x), p1 = __half22float2(*(const __half2*)&hv.y);
-        float t = (p0.x + p0.y) + (p1.x + p1.y);
-#pragma unroll
-        for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (lane == 0) xg[u] = t;
+
+    // ---- (2) x: wait for the previous kernel, stage fp16 x (all of K) and the group sums X_g -- once per
+    //      distinct x of the launch (the experts of a routed layer share it)
+    if (!waited) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited = true;
     }
-    __syncthreads();
+    if (x != x_staged) {
+        {
+            const int nvec = NB * (K / 8);
+            for (int t = threadIdx.x; t < nvec; t += kAThreads) {
+                const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (bb < a.nb) v = __ldg((const uint4*)(x + (size_t)bb * a.cols + kk));
+                *(uint4*)(xs + (size_t)t * 8) = v;
+            }
+        }
+        __syncthreads();
+        for (int u = warp; u < NB * a.SC; u += kAWarps) {   // X_g: 128 values per group, 4 per lane, fixed butterfly
+            const uint2 hv = *(const uint2*)(xs + (size_t)u * kSuper + lane * 4);
+            const float2 p0 = __half22float2(*(const __half2*)&hv.x), p1 = __half22float2(*(const __half2*)&hv.y);
+            float t = (p0.x + p0.y) + (p1.x + p1.y);
+#pragma unroll
+            for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            if (lane == 0) xg[u] = t;
+        }
+        x_staged = x;
+    }
+    __syncthreads();   // tables, x and X_g visible
 #pragma unroll
     for (int h = 0; h < 2; ++h) {   // the rows' slot counts have arrived: this warp's number of outlier rounds
         int wmax = (int)olen[h];
@@ -216,6 +285,13 @@ __global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a)
     const bool odd = t4 & 1;
 
     auto lookup = [&](uint32_t (&f)[4], int m, uint32_t base0, uint32_t base1) {
+        if (PAIR) {
+            f[0] = *(const uint32_t*)(tab + pair_entry_addr<N>(w0, 2 * m, base0));       // (k, k+1) of channel 0
+            f[1] = *(const uint32_t*)(tab + pair_entry_addr<N>(w1, 2 * m, base1));       // (k, k+1) of channel 1
+            f[2] = *(const uint32_t*)(tab + pair_entry_addr<N>(w0, 2 * m + 1, base0));   // (k+2, k+3) of channel 0
+            f[3] = *(const uint32_t*)(tab + pair_entry_addr<N>(w1, 2 * m + 1, base1));   // (k+2, k+3) of channel 1
+            return;
+        }
         const uint32_t l00 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 0, base0));
         const uint32_t l01 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 1, base0));
         const uint32_t l02 = *(const uint32_t*)(tab + entry_addr<N>(w0, 4 * m + 2, base0));
@@ -242,8 +318,10 @@ __global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a)
             consume_slots();
             if (++oround < nrounds) fetch_slots(oround);
         }
-        const uint32_t base0 = id0 * (uint32_t)(E * 128) + (uint32_t)lane * 4u;
-        const uint32_t base1 = id1 * (uint32_t)(E * 128) + (uint32_t)lane * 4u;
+        const uint32_t base0 = PAIR ? id0 * (uint32_t)(E * E * 64) + (uint32_t)(lane & 15) * 4u
+                                    : id0 * (uint32_t)(E * 128) + (uint32_t)lane * 4u;
+        const uint32_t base1 = PAIR ? id1 * (uint32_t)(E * E * 64) + (uint32_t)(lane & 15) * 4u
+                                    : id1 * (uint32_t)(E * 128) + (uint32_t)lane * 4u;
         const unsigned char* xp = xrow + (size_t)s * (kSuper * 2);
         float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
         uint32_t fa[4], fb[4];
@@ -332,8 +410,8 @@ __global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a)
 #pragma unroll
         for (int w = 0; w < kAWarps; ++w) total += red[((size_t)w * NB + bb) * kARows + r];
     }
+    bool writer = true;
     if (KS > 1) {
-        __shared__ int s_last;
         float* part = a.partial + (size_t)prob * 64 * NB * a.rows_ws;
         int* ticket = a.tickets + (size_t)prob * a.blocks + blk;
         if (active) part[((size_t)ks * NB + bb) * a.rows_ws + row] = total;
@@ -341,33 +419,56 @@ __global__ void __launch_bounds__(kAThreads, 2) gemv_v2a_kernel(const V2aArgs a)
         __syncthreads();
         if (t == 0) s_last = (atomicAdd(ticket, 1) == KS - 1);
         __syncthreads();
-        if (!s_last) return;
-        __threadfence();
-        if (active) {
-            total = 0.f;
-            for (int k2 = 0; k2 < KS; ++k2) total += __ldcg(part + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+        writer = s_last != 0;
+        if (writer) {
+            __threadfence();
+            if (active) {
+                total = 0.f;
+                for (int k2 = 0; k2 < KS; ++k2) total += __ldcg(part + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+            }
+            if (t == 0) *ticket = 0;
         }
-        if (t == 0) *ticket = 0;
     }
-    if (active && !dup && bb < a.nb && row < a.rows) {
+    if (writer && active && !dup && bb < a.nb && row < a.rows) {
         if (a.y_is_fp16)
             ((uint16_t*)y)[(size_t)bb * a.rows + row] = f2h(total);
         else
             ((float*)y)[(size_t)bb * a.rows + row] = total;
     }
+    if (!PAIR) break;   // the per-bank library is launched with one CTA per item
+    __syncthreads();   // red, x and the ticket flag are reused by the CTA's next item
+    }
 }
 
 // ------------------------------------------------------------------------------------ host side
 
-constexpr int kASlotsPerWave = 296;   // 148 SMs x 2 resident CTAs
+// Launch configuration of a layout: pair tables (one CTA per SM, 12 or 16 warps) when they fit, else the
+// per-bank library (two CTAs of 8 warps per SM).
+struct V2aConfig { bool pair; int warps, slots; size_t smem; };
 
-static size_t v2a_smem_bytes(const Layout& l, int nb) {
-    return (size_t)l.L * l.E * 128 + (size_t)nb * l.cols * 2 + (size_t)nb * l.SC * 4 + (size_t)kAWarps * nb * kARows * 4;
+static size_t v2a_smem_bytes(const Layout& l, int nb, bool pair, int warps) {
+    const size_t tab = pair ? (size_t)l.L * l.E * l.E * 64 : (size_t)l.L * l.E * 128;
+    return tab + (size_t)nb * l.cols * 2 + (size_t)nb * l.SC * 4 + (size_t)warps * nb * kARows * 4 +
+           (size_t)l.L * l.E * 2 + 16;   // + the copy of the library the tables were built from, 16-byte aligned
+}
+
+static int g_v2a_pair = 1;   // probe switch: 0 keeps every layout on the per-bank library
+void v2a_set_pair(int v) { g_v2a_pair = v; }
+
+static V2aConfig v2a_config(const Layout& l, int nb) {
+    if (g_v2a_pair && l.bits <= 3) {
+        // K is shared by the warps in super-chunks: 12 warps when that divides the count and 16 does not
+        const int warps = (l.SC % 16 != 0 && l.SC % 12 == 0) ? 12 : 16;
+        const size_t sm = v2a_smem_bytes(l, nb, true, warps);
+        if (sm <= 224u * 1024u) return V2aConfig{true, warps, 148, sm};
+    }
+    return V2aConfig{false, 8, 296, v2a_smem_bytes(l, nb, false, 8)};
 }
 
 bool v2a_supported(const Layout& l, int batch) {
     if (l.mode != 1 || l.bits < 2 || l.bits > 5 || batch > 2) return false;
-    return v2a_smem_bytes(l, batch) <= 110u * 1024u;   // two CTAs per SM
+    const V2aConfig cfg = v2a_config(l, batch);
+    return cfg.pair || cfg.smem <= 110u * 1024u;   // per-bank library: two CTAs per SM
 }
 
 size_t v2a_workspace_bytes(const Layout& l) {
@@ -375,18 +476,18 @@ size_t v2a_workspace_bytes(const Layout& l) {
     return align256((size_t)blocks * 4) + align256((size_t)64 * 2 * (size_t)blocks * kARows * 4);
 }
 
-template <int N, int NB>
+template <int N, int NB, int W, bool PAIR>
 static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             112 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB, W, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             PAIR ? 226 * 1024 : 112 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(kAThreads, 1, 1);
+    cfg.blockDim = dim3(W * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -394,10 +495,19 @@ static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_v2a_kernel<N, NB>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_v2a_kernel<N, NB, W, PAIR>, a);
+}
+
+template <int N, int NB>
+static cudaError_t launch_v2a_cfg(const V2aConfig& cfg, const V2aArgs& a, dim3 grid, cudaStream_t s) {
+    if (N <= 3 && cfg.pair)
+        return cfg.warps == 12 ? launch_v2a<(N <= 3 ? N : 3), NB, 12, true>(a, grid, cfg.smem, s)
+                               : launch_v2a<(N <= 3 ? N : 3), NB, 16, true>(a, grid, cfg.smem, s);
+    return launch_v2a<N, NB, 8, false>(a, grid, cfg.smem, s);
 }
 
 cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) {
+    const V2aConfig cfg = v2a_config(l, c.batch);
     V2aArgs a{};
     a.off = offsets_of(l);
     a.packed = c.packed; a.x = c.x; a.y = c.y;
@@ -411,10 +521,10 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     const long long total = (long long)a.blocks * c.n;
     int kst = 1;
     int rem = 0;
-    const long long tail = total % kASlotsPerWave;
+    const long long tail = total % cfg.slots;
     if (tail > 0 && c.n == 1) {
         rem = (int)tail;
-        kst = kASlotsPerWave / rem;
+        kst = cfg.slots / rem;
         const int kmax = l.SC / 4 > 1 ? l.SC / 4 : 1;
         if (kst > kmax) kst = kmax;
         if (kst > 64) kst = 64;
@@ -427,17 +537,20 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     if (a.kst <= 1) { a.kst = 1; a.n_full = a.blocks; rem = 0; }
     a.tickets = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + align256((size_t)a.blocks * 4 * c.n));
-    const size_t smem = v2a_smem_bytes(l, c.batch);
-    dim3 grid((unsigned)(a.n_full + rem * a.kst), (unsigned)c.n, 1);
+    a.items_x = a.n_full + rem * a.kst;
+    a.n = c.n;
+    const long long items = (long long)a.items_x * c.n;
+    // pair tables are expensive to build: resident CTAs walk the items; the per-bank library launches one CTA per item
+    dim3 grid((unsigned)(cfg.pair ? (items < cfg.slots ? items : cfg.slots) : items), 1, 1);
     switch (l.bits * 10 + c.batch) {
-        case 21: return launch_v2a<2, 1>(a, grid, smem, s);
-        case 22: return launch_v2a<2, 2>(a, grid, smem, s);
-        case 31: return launch_v2a<3, 1>(a, grid, smem, s);
-        case 32: return launch_v2a<3, 2>(a, grid, smem, s);
-        case 41: return launch_v2a<4, 1>(a, grid, smem, s);
-        case 42: return launch_v2a<4, 2>(a, grid, smem, s);
-        case 51: return launch_v2a<5, 1>(a, grid, smem, s);
-        case 52: return launch_v2a<5, 2>(a, grid, smem, s);
+        case 21: return launch_v2a_cfg<2, 1>(cfg, a, grid, s);
+        case 22: return launch_v2a_cfg<2, 2>(cfg, a, grid, s);
+        case 31: return launch_v2a_cfg<3, 1>(cfg, a, grid, s);
+        case 32: return launch_v2a_cfg<3, 2>(cfg, a, grid, s);
+        case 41: return launch_v2a_cfg<4, 1>(cfg, a, grid, s);
+        case 42: return launch_v2a_cfg<4, 2>(cfg, a, grid, s);
+        case 51: return launch_v2a_cfg<5, 1>(cfg, a, grid, s);
+        case 52: return launch_v2a_cfg<5, 2>(cfg, a, grid, s);
     }
     return cudaErrorInvalidValue;
 }

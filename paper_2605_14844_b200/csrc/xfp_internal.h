@@ -56,6 +56,7 @@ void pair_set_trace(void* p, size_t calls);
 bool v2a_supported(const Layout& l, int batch);
 size_t v2a_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
+void v2a_set_pair(int v);
 
 // Batched V2 path (3..16 rows of x); see xfp_gemv_batch.cu.
 bool batch_supported(const Layout& l, int batch);

@@ -180,6 +180,33 @@ def test_grouped_matches_single_calls():
         assert np.all(np.abs(single[0].cpu().numpy() - ys[j].cpu().numpy()) <= 0.05 * TOL * absum[0])
 
 
+@pytest.mark.parametrize("bits", [2, 3])
+def test_grouped_v2a_many_items_and_mixed_libraries(bits):
+    """More work items than resident CTAs (every CTA walks several blocks of several blobs), and blobs
+    whose libraries differ: the tables must follow the blob."""
+    n, rows, cols = 6, 2112, 384            # 33 blocks of 64 channels per blob, 198 items in all
+    qs = [synth.random_quantized(1, rows, cols, bits, 0.002, seed=1300 + j) for j in range(n)]
+    qs[1].codebook = qs[0].codebook          # blobs 0, 1 share a library, 2 and 3 share another, 4 and 5 their own
+    qs[3].codebook = qs[2].codebook
+    pms = [xfp.pack_tensors(q, col_bits=16) for q in qs]
+    x16s = [synth.activations(1, cols, seed=1400 + (j // 3)) for j in range(n)]   # two distinct x
+    xs = [_x_dev(x) for x in x16s]
+    xs = [xs[0], xs[0], xs[0], xs[3], xs[3], xs[3]]
+    ys = torch.full((n, rows), float("nan"), dtype=torch.float32, device="cuda")
+    d0 = pms[0].desc
+    desc = xfp.XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                       max(p.desc.nnz for p in pms))
+    _, wb = xfp.xfp_packed_size(desc)
+    ws = torch.zeros(n * wb, dtype=torch.uint8, device="cuda")
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    for _ in range(2):
+        xfp.xfp_gemv_grouped(desc, n, ptr([p.packed for p in pms]), ptr(xs), ptr([ys[j] for j in range(n)]), False, ws)
+    torch.cuda.synchronize()
+    for j in range(n):
+        ref, absum = xo.gemv(to_oracle(qs[j]), x16s[0 if j < 3 else 3])
+        assert np.all(np.abs(ys[j].cpu().numpy() - ref[0]) <= TOL * absum[0])
+
+
 def test_gemv_host_entry():
     q = synth.random_quantized(0, 96, 512, 5, 0.01, seed=97)
     pm = xfp.pack_tensors(q)
