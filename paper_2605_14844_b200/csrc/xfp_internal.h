@@ -62,6 +62,10 @@ void v2a_set_pair(int v);
 bool batch_supported(const Layout& l, int batch);
 cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s);
 
+// Batched V2a path (3..16 rows of x); see xfp_gemv_batch_v2a.cu.
+bool batch_v2a_supported(const Layout& l, int batch);
+cudaError_t launch_gemv_batch_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
+
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);

@@ -15,6 +15,16 @@
         token; every token-layer is two xfp_gemv_grouped launches (8 gate_up, 8 down).  Prints
         microseconds per token-layer and effective GB/s.
 
+    python -m paper_2605_14844_b200.probe sweep [quick]
+        batch and shape sweep: 8192 x 8192 and 28672 x 8192, 4-bit codebooks, V2 and V2a, x batch 1, 2, 4, 8, 16,
+        outlier rate 0 / 0.3 % / 2 %, uniform and column-clustered placement (`quick`: batch 1 and 16 only).
+
+    python -m paper_2605_14844_b200.probe stack [LAYERS]
+        mixed-bit decoder stack: LAYERS (default 48) layers of q/k/v/o 4096 x 4096 plus an MLP of
+        12288 x 4096 and 4096 x 12288, per-layer bit width from {2,3,4,5,6} and outlier rate from
+        {0, 0.5, 1, 2} % (seeded), V2 and V2a on the same draws; one token through the stack is one CUDA graph.  Prints
+        milliseconds per token and effective GB/s.
+
 MODE 0 = V2, 1 = V2a; PLACEMENT uniform | clustered | one_row.  Inputs come from synth.random_quantized.
 """
 from __future__ import annotations
@@ -149,9 +159,76 @@ def moe(experts=128, tokens=64, bits=3, distinct=8, reps=10):
                           us_per_token_layer=round(t, 2), GBs=round(per_layer / t / 1e3, 1))), flush=True)
 
 
+def sweep(quick=False):
+    batches = (1, 16) if quick else (1, 2, 4, 8, 16)
+    for mode in (0, 1):
+        for rows, cols in ((8192, 8192), (28672, 8192)):
+            for rate, placement in ((0.0, "uniform"), (0.003, "uniform"), (0.003, "clustered"), (0.02, "uniform"),
+                                    (0.02, "clustered")):
+                for batch in batches:
+                    if quick and (rate, placement) not in ((0.003, "uniform"), (0.02, "clustered")):
+                        continue
+                    time_shape(mode, rows, cols, 4, rate, batch, placement, reps=10)
+                    torch.cuda.empty_cache()
+
+
+def stack(layers=48, reps=5):
+    """One token through `layers` decoder layers (6 linears each), every matrix its own packed blob."""
+    shapes = [(4096, 4096)] * 4 + [(12288, 4096), (4096, 12288)]
+    for mode in (0, 1):
+        pms, xs, ys, total = [], {}, [], 0
+        rng_l = np.random.default_rng(4)   # same bit widths and outlier rates for both modes
+        cache = {}
+        for layer in range(layers):
+            bits = int(rng_l.integers(2, 7))
+            rate = (0.0, 0.005, 0.01, 0.02)[int(rng_l.integers(0, 4))]
+            for j, (rows, cols) in enumerate(shapes):
+                # layers that drew the same (bits, rate) reuse the host tensors; every layer packs its own blobs
+                key = (bits, rate, j)
+                if key not in cache:
+                    cache[key] = synth.random_quantized(mode, rows, cols, bits, rate, seed=5000 + 97 * len(cache) + j)
+                q = cache[key]
+                pms.append(pack_tensors(q, col_bits=16))
+                total += algorithmic_bytes(q)
+                xs.setdefault(cols, _x(1, cols))
+                ys.append(torch.empty((1, rows), dtype=torch.float16, device="cuda"))
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            def token():
+                for pm, y in zip(pms, ys):
+                    pm.gemv(xs[pm.desc.cols], y=y, y_fp16=True)
+            token()
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                token()
+            for _ in range(2):
+                g.replay()
+            s.synchronize()
+            ts = []
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s)
+                g.replay()
+                e1.record(s)
+                s.synchronize()
+                ts.append(e0.elapsed_time(e1))
+        t = float(np.median(ts))
+        print(json.dumps(dict(workload="decoder_stack", mode=mode, layers=layers, calls=len(pms), GB_per_token=round(total / 1e9, 3),
+                              ms_per_token=round(t, 4), GBs=round(total / t / 1e6, 1))), flush=True)
+        del pms, ys
+        torch.cuda.empty_cache()
+
+
 def main(argv):
     if len(argv) > 1 and argv[1] == "moe":
         moe(*(int(v) for v in argv[2:5]))
+        return 0
+    if len(argv) > 1 and argv[1] == "sweep":
+        sweep(len(argv) > 2 and argv[2] == "quick")
+        return 0
+    if len(argv) > 1 and argv[1] == "stack":
+        stack(*(int(v) for v in argv[2:3]))
         return 0
     if len(argv) < 7 or argv[1] not in ("launch", "time"):
         print(__doc__)

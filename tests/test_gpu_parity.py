@@ -84,6 +84,19 @@ def test_gemv_shapes_and_split_k(mode, rows, cols):
     _check_dequant(q, pm)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("rows,cols,bits", [(33, 128, 4), (256, 1536, 3), (2048, 4096, 4), (640, 2048, 5)])
+def test_batched_shapes_and_split_k(mode, rows, cols, bits):
+    """Batches 5 and 12 (a partial tile; a full tile plus a partial one) on shapes whose blocks are cut along K."""
+    q = synth.random_quantized(mode, rows, cols, bits, 0.01, seed=3 * rows + cols + mode)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    for batch in (5, 12):
+        _check_gemv(q, pm, synth.activations(batch, cols, seed=50 + batch))
+        _check_gemv(q, pm, synth.activations(batch, cols, seed=60 + batch), y_fp16=True)
+    tickets = pm.workspace[: ((q.rows + 31) // 32) * 4].view(torch.int32)
+    assert int(tickets.abs().sum().item()) == 0
+
+
 @pytest.mark.parametrize("placement,rate", [("uniform", 0.0), ("clustered", 0.02), ("one_row", 0.01)])
 def test_outlier_structures(placement, rate):
     for mode in (0, 1):
