@@ -78,7 +78,8 @@ __device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
 template <int N, int NB, int RPL, int W>
 __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
     constexpr int E = 1 << N;
-    constexpr int T = E * E;                   // pair-table entries per channel
+    constexpr bool kSingle = N > 5;            // N = 6: a pair table (4096 entries) does not fit, one entry per index
+    constexpr int T = kSingle ? E : E * E;     // table entries per channel
     constexpr int ROWS = 32 * RPL;             // channels per block
     constexpr int kStride = 128 * RPL;         // bytes between consecutive entries
     constexpr int kTabBytes = T * kStride;
@@ -194,7 +195,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
                 for (int i = 0; i < (TW > 0 ? TW : 1); ++i) {
                     const int t = TW > 0 ? warp * TW + i : warp;
                     if (t < T) {
-                        const uint32_t lv = __ldg(cb + (t & (E - 1))), hv = __ldg(cb + (t >> N));
+                        const uint32_t lv = __ldg(cb + (t & (E - 1))), hv = kSingle ? 0u : (uint32_t)__ldg(cb + (t >> N));
                         *(uint32_t*)(dst + (size_t)t * kStride) = lv | (hv << 16);
                     }
                 }
@@ -228,6 +229,26 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
     const unsigned char* xbase = (const unsigned char*)xs + (diag1 ? (size_t)K * 2 : 0);
 
     auto lookup = [&](uint32_t (&f)[4], int m) {
+        if (kSingle) {
+            // one entry per index; a PRMT joins two of them into the half2 of the fragment
+            const uint32_t a0 = *(const uint32_t*)(tab + single_addr<N, RPL>(w0, 4 * m + 0, base0));
+            const uint32_t a1 = *(const uint32_t*)(tab + single_addr<N, RPL>(w0, 4 * m + 1, base0));
+            const uint32_t a2 = *(const uint32_t*)(tab + single_addr<N, RPL>(w0, 4 * m + 2, base0));
+            const uint32_t a3 = *(const uint32_t*)(tab + single_addr<N, RPL>(w0, 4 * m + 3, base0));
+            f[0] = __byte_perm(a0, a1, 0x5410);
+            f[2] = __byte_perm(a2, a3, 0x5410);
+            if (RPL == 2) {
+                const uint32_t b0 = *(const uint32_t*)(tab + single_addr<N, RPL>(w1, 4 * m + 0, base1));
+                const uint32_t b1 = *(const uint32_t*)(tab + single_addr<N, RPL>(w1, 4 * m + 1, base1));
+                const uint32_t b2 = *(const uint32_t*)(tab + single_addr<N, RPL>(w1, 4 * m + 2, base1));
+                const uint32_t b3 = *(const uint32_t*)(tab + single_addr<N, RPL>(w1, 4 * m + 3, base1));
+                f[1] = __byte_perm(b0, b1, 0x5410);
+                f[3] = __byte_perm(b2, b3, 0x5410);
+            } else {
+                f[1] = 0u; f[3] = 0u;
+            }
+            return;
+        }
         f[0] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m, base0));
         f[2] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m + 1, base0));
         if (RPL == 2) {
@@ -507,12 +528,12 @@ static PairSchedule pair_schedule(const Layout& l) {
 static size_t pair_smem_bytes(const Layout& l, int nb) {
     const PairConfig cfg = pair_config(l);
     const int rows = 32 * cfg.rpl;
-    const size_t T = (size_t)l.E * l.E;
+    const size_t T = l.bits > 5 ? (size_t)l.E : (size_t)l.E * l.E;   // N = 6: one entry per index
     return T * 128 * cfg.rpl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4;
 }
 
 bool pair_supported(const Layout& l, int batch, int n_problems) {
-    if (l.mode != 0 || l.bits < 2 || l.bits > 5 || batch > 2 || n_problems != 1) return false;
+    if (l.mode != 0 || l.bits < 2 || l.bits > 6 || batch > 2 || n_problems != 1) return false;
     return pair_smem_bytes(l, batch) <= (pair_config(l).warps == 8 ? 110u : 220u) * 1024u;
 }
 
@@ -574,6 +595,8 @@ cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s)
             case 42: return launch_pair<4, 2, 1, 16>(a, sch.grid, smem, s);
             case 51: return launch_pair<5, 1, 1, 16>(a, sch.grid, smem, s);
             case 52: return launch_pair<5, 2, 1, 16>(a, sch.grid, smem, s);
+            case 61: return launch_pair<6, 1, 1, 16>(a, sch.grid, smem, s);
+            case 62: return launch_pair<6, 2, 1, 16>(a, sch.grid, smem, s);
         }
         return cudaErrorInvalidValue;
     }
@@ -584,6 +607,8 @@ cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s)
         case 32: return launch_pair<3, 2, 2, 8>(a, sch.grid, smem, s);
         case 41: return launch_pair<4, 1, 2, 8>(a, sch.grid, smem, s);
         case 42: return launch_pair<4, 2, 2, 8>(a, sch.grid, smem, s);
+        case 61: return launch_pair<6, 1, 2, 8>(a, sch.grid, smem, s);
+        case 62: return launch_pair<6, 2, 2, 8>(a, sch.grid, smem, s);
     }
     return cudaErrorInvalidValue;
 }

@@ -95,7 +95,7 @@ __device__ __forceinline__ uint32_t pair_entry_addr(const uint32_t* w, int p, ui
 }
 
 template <int N, int NB, int W, bool PAIR>
-__global__ void __launch_bounds__(W * 32, PAIR ? 1 : 2) gemv_v2a_kernel(const V2aArgs a) {
+__global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const V2aArgs a) {
     constexpr int E = 1 << N;
     constexpr int kAWarps = W;
     constexpr int kAThreads = W * 32;
@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(W * 32, PAIR ? 1 : 2) gemv_v2a_kernel(const V2
 // ------------------------------------------------------------------------------------ host side
 
 // Launch configuration of a layout: pair tables (one CTA per SM, 12 or 16 warps) when they fit, else the
-// per-bank library (two CTAs of 8 warps per SM).
+// per-bank library (two CTAs of 8 warps per SM, or one of 16 warps when the library is too large for two).
 struct V2aConfig { bool pair; int warps, slots; size_t smem; };
 
 static size_t v2a_smem_bytes(const Layout& l, int nb, bool pair, int warps) {
@@ -462,13 +462,15 @@ static V2aConfig v2a_config(const Layout& l, int nb) {
         const size_t sm = v2a_smem_bytes(l, nb, true, warps);
         if (sm <= 224u * 1024u) return V2aConfig{true, warps, 148, sm};
     }
-    return V2aConfig{false, 8, 296, v2a_smem_bytes(l, nb, false, 8)};
+    const size_t sm8 = v2a_smem_bytes(l, nb, false, 8);
+    if (sm8 <= 110u * 1024u) return V2aConfig{false, 8, 296, sm8};
+    return V2aConfig{false, 16, 148, v2a_smem_bytes(l, nb, false, 16)};   // large library (N = 5): one CTA per SM
 }
 
 bool v2a_supported(const Layout& l, int batch) {
     if (l.mode != 1 || l.bits < 2 || l.bits > 5 || batch > 2) return false;
     const V2aConfig cfg = v2a_config(l, batch);
-    return cfg.pair || cfg.smem <= 110u * 1024u;   // per-bank library: two CTAs per SM
+    return cfg.smem <= (cfg.warps == 8 ? 110u : 224u) * 1024u;
 }
 
 size_t v2a_workspace_bytes(const Layout& l) {
@@ -481,7 +483,7 @@ static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStre
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB, W, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             PAIR ? 226 * 1024 : 112 * 1024);
+                                             W == 8 ? 112 * 1024 : 226 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -503,6 +505,7 @@ static cudaError_t launch_v2a_cfg(const V2aConfig& cfg, const V2aArgs& a, dim3 g
     if (N <= 3 && cfg.pair)
         return cfg.warps == 12 ? launch_v2a<(N <= 3 ? N : 3), NB, 12, true>(a, grid, cfg.smem, s)
                                : launch_v2a<(N <= 3 ? N : 3), NB, 16, true>(a, grid, cfg.smem, s);
+    if (cfg.warps == 16) return launch_v2a<N, NB, 16, false>(a, grid, cfg.smem, s);
     return launch_v2a<N, NB, 8, false>(a, grid, cfg.smem, s);
 }
 

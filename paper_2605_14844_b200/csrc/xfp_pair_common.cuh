@@ -34,5 +34,21 @@ __device__ __forceinline__ uint32_t pair_addr(const uint32_t* w, int p, uint32_t
     }
 }
 
+// Byte offset of the table entry of index j (compile time) for tables that hold one entry per index
+// (N = 6): q * 128 * RPL merged with `base`.
+template <int N, int RPL>
+__device__ __forceinline__ uint32_t single_addr(const uint32_t* w, int j, uint32_t base) {
+    constexpr int SH = RPL == 2 ? 8 : 7;
+    constexpr uint32_t mask = ((1u << N) - 1u) << SH;
+    const int bit = j * N, wi = bit >> 5, off = bit & 31;
+    uint32_t v;
+    if (off + N > 32)
+        v = __funnelshift_r(w[wi], w[wi + 1], off) << SH;
+    else if (off >= SH)
+        v = w[wi] >> (off - SH);
+    else
+        v = w[wi] << (SH - off);
+    return (v & mask) | base;
+}
 
 }  // namespace xfp
