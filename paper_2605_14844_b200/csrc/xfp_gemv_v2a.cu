@@ -31,6 +31,9 @@
 // Outliers, schedule, launch overlap: as in the V2 kernel (transposed slabs consumed by the lanes that
 // own the rows; whole-K blocks first, the last partial round cut along K with a fixed-order finish
 // through the workspace; weights before griddepcontrol.wait, x/y/workspace after it).
+#include <algorithm>
+#include <utility>
+
 #include "xfp_internal.h"
 
 namespace xfp {
@@ -51,6 +54,7 @@ struct V2aArgs {
     int rows, cols, RB, SC, rows_ws, ell_slots, L;
     int nb, y_is_fp16;
     int blocks, n_full, kst, sc_per_split;
+    int n_a, kst_b, sc_per_split_b;   // of the cut blocks the first n_a use kst slices, the rest kst_b (finer) slices
     int items_x, n;   // work items per blob (whole blocks + K slices), blobs
 };
 
@@ -124,9 +128,12 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
     int blk, ks, KS, spp;
     if (bx < a.n_full) {
         blk = bx; ks = 0; KS = 1; spp = a.SC;
-    } else {
+    } else if (bx - a.n_full < a.n_a * a.kst) {
         const int t = bx - a.n_full;
         blk = a.n_full + t / a.kst; ks = t % a.kst; KS = a.kst; spp = a.sc_per_split;
+    } else {
+        const int t = bx - a.n_full - a.n_a * a.kst;
+        blk = a.n_full + a.n_a + t / a.kst_b; ks = t % a.kst_b; KS = a.kst_b; spp = a.sc_per_split_b;
     }
     const void* packed = a.packed_list ? a.packed_list[prob] : a.packed;
     const uint16_t* x = a.x_list ? a.x_list[prob] : a.x;
@@ -522,25 +529,42 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     // schedule: whole-K blocks fill whole rounds of CTA slots (all blobs of the launch count); the blocks of
     // the last partial round are cut along K into slices of at least 512 weights
     const long long total = (long long)a.blocks * c.n;
-    int kst = 1;
+    const int kmax = std::min(64, std::max(1, l.SC / 4));
+    auto slices = [&](int want) {   // (slices, super-chunks per slice) for a cut into about `want` pieces
+        int k = std::max(1, std::min(want, std::min(kmax, l.SC)));
+        const int spp = (l.SC + k - 1) / k;
+        k = (l.SC + spp - 1) / spp;
+        return std::make_pair(k, spp);
+    };
     int rem = 0;
-    const long long tail = total % cfg.slots;
+    a.kst = 1; a.sc_per_split = l.SC; a.n_a = 0; a.kst_b = 1; a.sc_per_split_b = l.SC;
+    const int tail = (int)(total % cfg.slots);
     if (tail > 0 && c.n == 1) {
-        rem = (int)tail;
-        kst = cfg.slots / rem;
-        const int kmax = l.SC / 4 > 1 ? l.SC / 4 : 1;
-        if (kst > kmax) kst = kmax;
-        if (kst > 64) kst = 64;
-        if (kst > l.SC) kst = l.SC;
-        if (kst <= 1) { kst = 1; rem = 0; }
+        rem = tail;
+        auto ka = slices(cfg.slots / rem);
+        if (ka.first > 1) {
+            // the whole tail fits one round when cut into ka pieces per block
+            a.kst = ka.first; a.sc_per_split = ka.second; a.n_a = rem;
+        } else if (kmax >= 2 && total > cfg.slots) {
+            // whole rounds came before and more than half a round is left: halves for as many blocks as fill one round, finer slices for the rest
+            auto k2 = slices(2);
+            a.kst = k2.first; a.sc_per_split = k2.second;
+            a.n_a = std::min(rem, cfg.slots / a.kst);
+            const int rest = rem - a.n_a;
+            if (rest > 0) {
+                auto kb = slices(std::max(2, cfg.slots / rest));
+                a.kst_b = kb.first; a.sc_per_split_b = kb.second;
+            }
+            if (a.kst <= 1) { a.n_a = 0; rem = 0; }
+        } else {
+            rem = 0;
+        }
     }
     a.n_full = a.blocks - rem;
-    a.sc_per_split = (l.SC + kst - 1) / kst;
-    a.kst = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
-    if (a.kst <= 1) { a.kst = 1; a.n_full = a.blocks; rem = 0; }
+    const int n_b = rem - a.n_a;
     a.tickets = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + align256((size_t)a.blocks * 4 * c.n));
-    a.items_x = a.n_full + rem * a.kst;
+    a.items_x = a.n_full + a.n_a * a.kst + n_b * a.kst_b;
     a.n = c.n;
     const long long items = (long long)a.items_x * c.n;
     // pair tables are expensive to build: resident CTAs walk the items; the per-bank library launches one CTA per item
