@@ -81,7 +81,13 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
     constexpr bool kSingle = N > 5;            // N = 6: a pair table (4096 entries) does not fit, one entry per index
     constexpr int T = kSingle ? E : E * E;     // table entries per channel
     constexpr int ROWS = 32 * RPL;             // channels per block
-    constexpr int kStride = 128 * RPL;         // bytes between consecutive entries
+    // bytes between consecutive entries: 128 per channel half; N = 4 keeps 256 also with one channel per lane,
+    // so that an index byte is the table offset's second byte and one PRMT builds the address
+    constexpr int SL = (RPL == 2 || N == 4) ? 2 : 1;
+    constexpr int kStride = 128 * SL;
+    // one channel per lane at batch 1: the fragment's second row slot carries the channel's NEXT four weights
+    // and columns 4..7 of the B fragment their x, so one mma covers 8 consecutive k
+    constexpr bool kDual = (RPL == 1 && NB == 1 && !kSingle);
     constexpr int kTabBytes = T * kStride;
     constexpr int kThreads = W * 32;
     constexpr int TW = T / W;                  // table entries a warp fills per channel half
@@ -249,11 +255,11 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
             }
             return;
         }
-        f[0] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m, base0));
-        f[2] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m + 1, base0));
+        f[0] = *(const uint32_t*)(tab + pair_addr<N, SL>(w0, 2 * m, base0));
+        f[2] = *(const uint32_t*)(tab + pair_addr<N, SL>(w0, 2 * m + 1, base0));
         if (RPL == 2) {
-            f[1] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w1, 2 * m, base1));
-            f[3] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w1, 2 * m + 1, base1));
+            f[1] = *(const uint32_t*)(tab + pair_addr<N, SL>(w1, 2 * m, base1));
+            f[3] = *(const uint32_t*)(tab + pair_addr<N, SL>(w1, 2 * m + 1, base1));
         } else {
             f[1] = 0u; f[3] = 0u;
         }
@@ -314,6 +320,46 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
             };
             const unsigned char* xp = xbase + (size_t)(sc0 + s) * (kSuper * 2);
             uint32_t fa[4], fb[4];
+            if (kDual) {
+                // 16 mma of 8 consecutive k: pairs 4j, 4j+1 in the fragment's g rows, pairs 4j+2, 4j+3 in its g+8
+                // rows; lanes g == t feed columns 0..3 with x[8j .. 8j+3], lanes g == t+4 columns 4..7 with
+                // x[8j+4 .. 8j+7].  D[g][n] and D[g+8][4+n] are the two halves of channel lane 4g+n.
+                const bool dq = diag0 || (g == t4 + 4);
+                const unsigned char* xq = xp + ((g == t4 + 4) ? 8 : 0);
+                auto lookup2 = [&](uint32_t (&f)[4], int j) {
+                    f[0] = *(const uint32_t*)(tab + pair_addr<N, SL>(w0, 4 * j, base0));
+                    f[2] = *(const uint32_t*)(tab + pair_addr<N, SL>(w0, 4 * j + 1, base0));
+                    f[1] = *(const uint32_t*)(tab + pair_addr<N, SL>(w0, 4 * j + 2, base0));
+                    f[3] = *(const uint32_t*)(tab + pair_addr<N, SL>(w0, 4 * j + 3, base0));
+                };
+                auto reload2 = [&](int gi) {   // gi: mma whose look-ups were just issued (compile time)
+#pragma unroll
+                    for (int v = 0; v < N; ++v) {
+                        const int plast = (128 * (v + 1) + 2 * N - 1) / (2 * N) - 1;   // last pair touching vector v
+                        if (plast / 4 == gi && has_next) {
+                            const uint4 t0 = ld_stream(i0 + ((size_t)snext * N + v) * 32);
+                            w0[4 * v] = t0.x; w0[4 * v + 1] = t0.y; w0[4 * v + 2] = t0.z; w0[4 * v + 3] = t0.w;
+                        }
+                    }
+                };
+                uint2 xa = make_uint2(0u, 0u), xb = make_uint2(0u, 0u);
+                if (dq) xa = *(const uint2*)xq;
+                lookup2(fa, 0);
+#pragma unroll
+                for (int j = 0; j < kSuper / 8; j += 2) {
+                    if (dq) xb = *(const uint2*)(xq + (j + 1) * 16);
+                    lookup2(fb, j + 1);
+                    reload2(j + 1);
+                    mma16816(c0, fa[0], fa[1], fa[2], fa[3], xa.x, xa.y);
+                    if (j + 2 < kSuper / 8) {
+                        if (dq) xa = *(const uint2*)(xq + (j + 2) * 16);
+                        lookup2(fa, j + 2);
+                        reload2(j + 2);
+                    }
+                    mma16816(c1, fb[0], fb[1], fb[2], fb[3], xb.x, xb.y);
+                }
+                continue;
+            }
             uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = make_uint4(0u, 0u, 0u, 0u);
             if (diag) xa = *(const uint4*)xp;
             lookup(fa, 0);
@@ -372,6 +418,13 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
                 if (RPL == 2) { r[32 + l0] = v2; r[32 + l0 + 1] = v3; }
             }
             __syncwarp();
+            if (kDual) {   // the second halves sit in rows g+8, columns 4..7: lanes t >= 2 add them
+                if (t4 >= 2) {
+                    float* r = red + (size_t)warp * ROWS;
+                    r[l0] += v2; r[l0 + 1] += v3;
+                }
+                __syncwarp();
+            }
 #pragma unroll
             for (int bb2 = 0; bb2 < NB; ++bb2)
 #pragma unroll
@@ -529,7 +582,8 @@ static size_t pair_smem_bytes(const Layout& l, int nb) {
     const PairConfig cfg = pair_config(l);
     const int rows = 32 * cfg.rpl;
     const size_t T = l.bits > 5 ? (size_t)l.E : (size_t)l.E * l.E;   // N = 6: one entry per index
-    return T * 128 * cfg.rpl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4;
+    const int sl = (cfg.rpl == 2 || l.bits == 4) ? 2 : 1;              // entry stride in units of 128 bytes
+    return T * 128 * sl + (size_t)nb * l.cols * 2 + (size_t)cfg.warps * nb * rows * 4;
 }
 
 bool pair_supported(const Layout& l, int batch, int n_problems) {
