@@ -48,7 +48,7 @@ __device__ __forceinline__ uint32_t lib_entry_addr(const uint32_t* w, int j, uin
     const int bit = j * N, wi = bit >> 5, off = bit & 31;
     uint32_t v;
     if (off + N > 32)
-        v = __funnelshift_r(w[wi], w[wi + 1], off) << 7;
+        v = __funnelshift_r(w[wi], w[wi + 1], off - 7);   // field straight to bit 7 (off > 7 whenever it straddles)
     else if (off >= 7)
         v = w[wi] >> (off - 7);
     else

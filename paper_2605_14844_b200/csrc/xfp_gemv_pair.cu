@@ -507,7 +507,7 @@ static PairConfig pair_config(const Layout& l) {
     // one row per lane (128 KB of tables), 16 warps, one CTA per SM.  Matrices with at most 148
     // row-blocks also take one row per lane: twice the CTAs and no cut along K.
     if (l.bits == 5) return PairConfig{1, 16, 148};
-    if (g_pair_small == 1 && l.RB <= 148 && l.bits >= 3) return PairConfig{1, 16, 148};
+    if (g_pair_small >= 1 && l.RB <= 148 * g_pair_small && l.bits >= 3) return PairConfig{1, 16, 148};
     return PairConfig{2, 8, 296};
 }
 

@@ -74,7 +74,7 @@ __device__ __forceinline__ uint32_t entry_addr(const uint32_t* w, int j, uint32_
     const int bit = j * N, wi = bit >> 5, off = bit & 31;
     uint32_t v;
     if (off + N > 32)
-        v = __funnelshift_r(w[wi], w[wi + 1], off) << 7;
+        v = __funnelshift_r(w[wi], w[wi + 1], off - 7);   // field straight to bit 7 (off > 7 whenever it straddles)
     else if (off >= 7)
         v = w[wi] >> (off - 7);
     else
@@ -90,7 +90,7 @@ __device__ __forceinline__ uint32_t pair_entry_addr(const uint32_t* w, int p, ui
     const int bit = p * 2 * N, wi = bit >> 5, off = bit & 31;
     uint32_t v;
     if (off + 2 * N > 32)
-        v = __funnelshift_r(w[wi], w[wi + 1], off) << 6;
+        v = __funnelshift_r(w[wi], w[wi + 1], off - 6);   // field straight to bit 6
     else if (off >= 6)
         v = w[wi] >> (off - 6);
     else

@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t pair_addr(const uint32_t* w, int p, uint32_t
         const int bit = p * 2 * N, wi = bit >> 5, off = bit & 31;
         uint32_t v;
         if (off + 2 * N > 32)
-            v = __funnelshift_r(w[wi], w[wi + 1], off) << SH;
+            v = __funnelshift_r(w[wi], w[wi + 1], off - SH);   // field straight to bit SH (off > SH whenever it straddles)
         else if (off >= SH)
             v = w[wi] >> (off - SH);
         else
@@ -43,7 +43,7 @@ __device__ __forceinline__ uint32_t single_addr(const uint32_t* w, int j, uint32
     const int bit = j * N, wi = bit >> 5, off = bit & 31;
     uint32_t v;
     if (off + N > 32)
-        v = __funnelshift_r(w[wi], w[wi + 1], off) << SH;
+        v = __funnelshift_r(w[wi], w[wi + 1], off - SH);   // field straight to bit SH (off > SH whenever it straddles)
     else if (off >= SH)
         v = w[wi] >> (off - SH);
     else
