@@ -272,11 +272,19 @@ def run_xfp(args, rank: int, world: int):
 
         for _ in range(3):
             step_host()
+        stream.synchronize()
+        # the step's host copies and launches are captured once and replayed: every replay copies the 32
+        # x vectors from pinned host memory, runs the 32 fused GEMVs and copies the 32 results back
+        graph_host = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_host, stream=stream):
+            step_host()
+        for _ in range(3):
+            graph_host.replay()
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(args.steps):
-            step_host()
+            graph_host.replay()
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1)
@@ -307,7 +315,9 @@ def run_xfp(args, rank: int, world: int):
                      "traffic": sum(NCU_TRAFFIC_BYTES_PER_LAUNCH[n[2]] for n in names) / n_calls, "bytes_per_launch": step_bytes / n_calls,
                      "kernel": "gemv (all calls of a step)"},
         "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": n_calls * COLS * 2,
-                "d2h_bytes_per_step": n_calls * ROWS * 2, "us_per_call": e2e_ms / args.steps * 1e3 / n_calls},
+                "d2h_bytes_per_step": n_calls * ROWS * 2, "us_per_call": e2e_ms / args.steps * 1e3 / n_calls,
+                "how": "xfp_gemv_host per projection (pinned x in, fused GEMV, pinned y out), the step captured once "
+                       "as a CUDA graph and replayed"},
         "gpu_launches": args.steps * n_calls,
         "clocks": clocks,
     }

@@ -111,9 +111,12 @@ int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* str
 int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
                      void* const* y, int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
 
-/* Convenience for callers whose activations live in host memory: copies x_host (pinned for
- * asynchrony) to x_dev, runs the GEMV for desc->mode, copies y_dev to y_host, all on `stream`.
- * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller. */
+/* Convenience for callers whose activations live in host memory: brings x_host to x_dev, runs the GEMV for
+ * desc->mode and delivers y in y_host, all on `stream` (the host sees y once the stream reached this point).
+ * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller.  Pinned,
+ * device-mapped host buffers (cudaHostAlloc / cudaHostRegister under unified addressing) are used in
+ * place: a small kernel reads x_host and the GEMV stores into y_host directly (y_dev is then not
+ * touched); other host memory goes through cudaMemcpyAsync in both directions. */
 int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_host, uint16_t* x_dev,
                   int32_t batch, void* y_host, void* y_dev, int32_t y_is_fp16, void* workspace,
                   size_t workspace_bytes, void* stream);

@@ -59,6 +59,45 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     return e == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 
+// Device alias of a pinned, mapped host pointer; null for anything else (pageable memory, device memory).
+const void* mapped_alias(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();   // pageable memory may report an error on older runtimes: not ours to keep
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
+// x from mapped host memory to its device staging buffer.  The host loads are issued before the dependency
+// wait (x_host is not written by earlier kernels of the stream; the staging buffer may still be read by one).
+__global__ void __launch_bounds__(256) host_in_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n) {
+    asm volatile("griddepcontrol.launch_dependents;");
+    const int i = blockIdx.x * 1024 + threadIdx.x;
+    uint4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (i + j * 256 < n) v[j] = src[i + j * 256];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (i + j * 256 < n) dst[i + j * 256] = v[j];
+}
+
+cudaError_t launch_host_in(const void* src, void* dst, size_t bytes, cudaStream_t s) {
+    const int n = (int)(bytes / 16);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((n + 1023) / 1024), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, host_in_kernel, (const uint4*)src, (uint4*)dst, n);
+}
+
 }  // namespace
 
 extern "C" {
@@ -130,14 +169,22 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
     if (!x_host || !x_dev || !y_host || !y_dev) return XFP_ERR_NULL;
     if (batch < 1 || batch > 16) return XFP_ERR_SHAPE;
     cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(x_dev, x_host, (size_t)batch * desc->cols * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    const size_t xbytes = (size_t)batch * desc->cols * 2, ybytes = (size_t)batch * desc->rows * (y_is_fp16 ? 2 : 4);
+    // Pinned, device-mapped host buffers are used in place: a small kernel fetches x over the bus (its loads
+    // overlap the tail of the previous kernel) and the GEMV stores y straight into host memory.  Two DMA
+    // copies of a few KB cost more than the GEMV itself.  Pageable or unmapped buffers take the copies.
+    const void* xmap = mapped_alias(x_host);
+    void* ymap = (void*)mapped_alias(y_host);
+    if (xmap && aligned16(xmap) && aligned16(x_dev) && xbytes % 16 == 0) {
+        if (launch_host_in(xmap, x_dev, xbytes, s) != cudaSuccess) return XFP_ERR_CUDA;
+    } else if (cudaMemcpyAsync(x_dev, x_host, xbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
         return XFP_ERR_CUDA;
-    st = desc->mode ? xfp_gemv_v2a(desc, packed, x_dev, batch, y_dev, y_is_fp16, workspace, workspace_bytes, stream)
-                    : xfp_gemv_v2(desc, packed, x_dev, batch, y_dev, y_is_fp16, workspace, workspace_bytes, stream);
+    }
+    void* y = (ymap && aligned16(ymap)) ? ymap : y_dev;
+    st = desc->mode ? xfp_gemv_v2a(desc, packed, x_dev, batch, y, y_is_fp16, workspace, workspace_bytes, stream)
+                    : xfp_gemv_v2(desc, packed, x_dev, batch, y, y_is_fp16, workspace, workspace_bytes, stream);
     if (st) return st;
-    if (cudaMemcpyAsync(y_host, y_dev, (size_t)batch * desc->rows * (y_is_fp16 ? 2 : 4), cudaMemcpyDeviceToHost, s) !=
-        cudaSuccess)
-        return XFP_ERR_CUDA;
+    if (y == y_dev && cudaMemcpyAsync(y_host, y_dev, ybytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return XFP_ERR_CUDA;
     return XFP_OK;
 }
 

@@ -220,15 +220,21 @@ def test_grouped_v2a_many_items_and_mixed_libraries(bits):
         assert np.all(np.abs(ys[j].cpu().numpy() - ref[0]) <= TOL * absum[0])
 
 
-def test_gemv_host_entry():
-    q = synth.random_quantized(0, 96, 512, 5, 0.01, seed=97)
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("mode,batch", [(0, 2), (1, 1), (0, 5)])
+def test_gemv_host_entry(pinned, mode, batch):
+    """Host buffers: pinned (used in place by the device) and pageable (copied)."""
+    q = synth.random_quantized(mode, 96, 512, 5 if mode == 0 else 3, 0.01, seed=97)
     pm = xfp.pack_tensors(q)
-    x16 = synth.activations(2, q.cols, seed=9)
-    xh = torch.from_numpy(x16.view(np.int16)).pin_memory()
-    yh = torch.zeros((2, q.rows), dtype=torch.float32).pin_memory()
-    xd = torch.empty_like(xh, device="cuda")
-    yd = torch.empty((2, q.rows), dtype=torch.float32, device="cuda")
-    xfp.xfp_gemv_host(pm.desc, pm.packed, xh, xd, 2, yh, yd, False, pm.workspace)
+    x16 = synth.activations(batch, q.cols, seed=9)
+    xh = torch.from_numpy(x16.view(np.int16).copy())
+    yh = torch.full((batch, q.rows), float("nan"), dtype=torch.float32)
+    if pinned:
+        xh, yh = xh.pin_memory(), yh.pin_memory()
+    xd = torch.empty((batch, q.cols), dtype=torch.int16, device="cuda")
+    yd = torch.empty((batch, q.rows), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        xfp.xfp_gemv_host(pm.desc, pm.packed, xh, xd, batch, yh, yd, False, pm.workspace)
     torch.cuda.synchronize()
     ref, absum = xo.gemv(to_oracle(q), x16)
     assert np.all(np.abs(yh.numpy() - ref) <= TOL * absum)
