@@ -13,6 +13,9 @@ LIB = os.path.join(HERE, "libxfp.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
+# XFP_TRACE=1 compiles the per-CTA phase stamps of the pair kernel in (a timing probe; use with --force)
+if os.environ.get("XFP_TRACE") == "1":
+    FLAGS.append("-DXFP_TRACE=1")
 
 
 def _sources():

@@ -67,12 +67,17 @@ struct PairArgs {
     unsigned long long* trace;  // timing probe: per CTA 8 globaltimer stamps (null in normal use)
 };
 
+// Phase stamps for the timing probe; compiled in only with -DXFP_TRACE=1 (they cost issue slots).
 __device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
+#ifdef XFP_TRACE
     if (a.trace && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         a.trace[(size_t)blockIdx.x * 8 + slot] = t;
     }
+#else
+    (void)a; (void)slot;
+#endif
 }
 
 template <int N, int NB, int RPL, int W>
