@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the two GEMV kernels of this workload, from
 # the ncu captures summarised in profiles/gemv_pair_attention_4096x4096.md (bits -> bytes)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {4: 9625088, 5: 11854848}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {4: 9623296, 5: 11855616}
 
 
 def block_spec(layer: int):
