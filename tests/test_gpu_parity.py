@@ -97,6 +97,16 @@ def test_batched_shapes_and_split_k(mode, rows, cols, bits):
     assert int(tickets.abs().sum().item()) == 0
 
 
+@pytest.mark.parametrize("mode,bits", [(0, 4), (0, 5), (1, 3), (1, 4)])
+def test_longest_rows(mode, bits):
+    """K = 65536, the largest the descriptor admits (u16 outlier columns): x alone is 128 KB per batch row."""
+    q = synth.random_quantized(mode, 40, 65536, bits, 0.005, seed=77 + bits + mode)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    for batch in (1, 2, 3):
+        _check_gemv(q, pm, synth.activations(batch, q.cols, seed=70 + batch))
+    _check_dequant(q, pm)
+
+
 @pytest.mark.parametrize("placement,rate", [("uniform", 0.0), ("clustered", 0.02), ("one_row", 0.01)])
 def test_outlier_structures(placement, rate):
     for mode in (0, 1):
