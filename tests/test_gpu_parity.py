@@ -291,3 +291,19 @@ def test_full_size_sampled_rows(mode, rows, cols, bits, rate):
     torch.cuda.synchronize()
     got = W[torch.from_numpy(sample).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
     assert np.array_equal(got, xo.dequant(to_oracle(q))[sample])
+
+
+@pytest.mark.parametrize("mode,batch,rate,placement", [(0, 1, 0.02, "clustered"), (0, 16, 0.003, "uniform"),
+                                                        (1, 2, 0.003, "uniform"), (1, 8, 0.02, "clustered")])
+def test_sweep_shape_28672x8192_sampled_rows(mode, batch, rate, placement):
+    """The large shape of the batch sweep in the launch configurations the timing runs use: 4-bit, V2 and V2a,
+    whole rounds of CTAs plus the tiers of K slices; sampled rows against the oracle for every batch row."""
+    rows, cols = 28672, 8192
+    q = synth.random_quantized(mode, rows, cols, 4, rate, seed=4242 + mode, placement=placement)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    sample = _sample_rows(rows, 96, seed=batch)
+    sample = np.unique(np.concatenate([sample, [18943, 18944, 28640, 28671]]))   # around the cut blocks and the end
+    _check_gemv(q, pm, synth.activations(batch, cols, seed=30 + batch), rows=sample)
+    tickets = pm.workspace[: ((rows + 31) // 32) * 4].view(torch.int32)
+    assert int(tickets.abs().sum().item()) == 0
+
