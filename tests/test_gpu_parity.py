@@ -203,6 +203,31 @@ def test_grouped_matches_single_calls():
         assert np.all(np.abs(single[0].cpu().numpy() - ys[j].cpu().numpy()) <= 0.05 * TOL * absum[0])
 
 
+@pytest.mark.parametrize("mode,bits", [(0, 4), (0, 6), (1, 5), (1, 6)])
+def test_grouped_other_modes(mode, bits):
+    """Grouped launches outside the routed-MoE mode: V2 blobs (every blob its own codebooks) and wide V2a."""
+    n, rows, cols = 5, 224, 640
+    qs = [synth.random_quantized(mode, rows, cols, bits, 0.004 * (j + 1), seed=1500 + 11 * j + bits) for j in range(n)]
+    if mode == 1:
+        for q in qs[1:]:
+            q.codebook = qs[0].codebook
+    pms = [xfp.pack_tensors(q, col_bits=32) for q in qs]
+    x16s = [synth.activations(1, cols, seed=1600 + j) for j in range(n)]
+    xs = [_x_dev(x) for x in x16s]
+    ys = torch.full((n, rows), float("nan"), dtype=torch.float16, device="cuda")
+    d0 = pms[0].desc
+    desc = xfp.XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                       max(p.desc.nnz for p in pms))
+    _, wb = xfp.xfp_packed_size(desc)
+    ws = torch.zeros(n * wb, dtype=torch.uint8, device="cuda")
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    xfp.xfp_gemv_grouped(desc, n, ptr([p.packed for p in pms]), ptr(xs), ptr([ys[j] for j in range(n)]), True, ws)
+    torch.cuda.synchronize()
+    for j in range(n):
+        ref, absum = xo.gemv(to_oracle(qs[j]), x16s[j])
+        assert np.all(np.abs(ys[j].float().cpu().numpy().astype(np.float64) - ref[0]) <= TOL * absum[0])
+
+
 @pytest.mark.parametrize("bits", [2, 3])
 def test_grouped_v2a_many_items_and_mixed_libraries(bits):
     """More work items than resident CTAs (every CTA walks several blocks of several blobs), and blobs
