@@ -1,0 +1,152 @@
+"""Python binding of the encoder's C ABI (include/xfp_quant.h): argument marshalling only.
+
+Every function hands device pointers of torch tensors to libxfp.so; the statistics, the selection of the
+extracted weights, Lloyd, LibFit, the residual and the cosine gate all run in the library's kernels.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Optional, Sequence
+
+import torch
+
+from .binding import XfpDesc, XfpError, _check, _ptr, _stream, load_library
+
+QUANT_EXPORTS = ("xfp_quant_workspace_size", "xfp_quant_stats", "xfp_quant_outliers", "xfp_quant_lloyd",
+                 "xfp_quant_libfit_library", "xfp_quant_libfit_assign", "xfp_quant_residual", "xfp_quant_cosine",
+                 "xfp_quant_median", "xfp_quantize")
+
+
+class XfpQuantParams(C.Structure):
+    """Mirror of xfp_quant_params."""
+    _fields_ = [("sigma_mode", C.c_int32), ("outlier_mode", C.c_int32), ("k_sigma", C.c_double),
+                ("cap_frac", C.c_double), ("rate", C.c_double), ("lloyd_iters", C.c_int32), ("reserved", C.c_int32)]
+
+
+class XfpQuantResult(C.Structure):
+    """Mirror of xfp_quant_result."""
+    _fields_ = [("bits", C.c_int32), ("fallback", C.c_int32), ("tried", C.c_int32), ("reserved", C.c_int32),
+                ("nnz", C.c_int64), ("mu", C.c_double), ("sigma", C.c_double), ("median_cos", C.c_double)]
+
+
+_DECLARED = False
+
+
+def _lib():
+    global _DECLARED
+    lib = load_library()
+    if not _DECLARED:
+        vp, sz, i32, i64, f64 = C.c_void_p, C.c_size_t, C.c_int32, C.c_int64, C.c_double
+        dp = C.POINTER(XfpDesc)
+        lib.xfp_quant_workspace_size.argtypes = [i32, i32, C.POINTER(sz)]
+        lib.xfp_quant_stats.argtypes = [vp, i64, i32, vp, vp, sz, vp]
+        lib.xfp_quant_outliers.argtypes = [vp, i64, vp, i32, f64, f64, vp, vp, vp, sz, vp]
+        lib.xfp_quant_lloyd.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp]
+        lib.xfp_quant_libfit_library.argtypes = [vp, i32, i32, i32, i32, vp, vp, sz, vp]
+        lib.xfp_quant_libfit_assign.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        lib.xfp_quant_residual.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
+        lib.xfp_quant_cosine.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.xfp_quant_median.argtypes = [vp, i64, vp, vp, sz, vp]
+        lib.xfp_quantize.argtypes = [i32, vp, i32, i32, C.POINTER(XfpQuantParams), C.POINTER(i32), i32, f64, i32,
+                                     vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, C.POINTER(XfpQuantResult),
+                                     vp, sz, vp]
+        for name in QUANT_EXPORTS:
+            getattr(lib, name).restype = C.c_int
+        _DECLARED = True
+    return lib
+
+
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
+def xfp_quant_workspace_size(rows: int, cols: int) -> int:
+    b = C.c_size_t()
+    _check(_lib().xfp_quant_workspace_size(int(rows), int(cols), C.byref(b)), "xfp_quant_workspace_size")
+    return b.value
+
+
+def xfp_quant_stats(W, sigma_mode: int, mu_sigma, workspace, stream=None) -> None:
+    _check(_lib().xfp_quant_stats(_ptr(W), W.numel(), int(sigma_mode), _ptr(mu_sigma), _ptr(workspace),
+                                  _nbytes(workspace), _stream(stream)), "xfp_quant_stats")
+
+
+def xfp_quant_outliers(W, mu_sigma, outlier_mode: int, k_or_rate: float, cap_frac: float, mask, count, workspace,
+                       stream=None) -> None:
+    _check(_lib().xfp_quant_outliers(_ptr(W), W.numel(), _ptr(mu_sigma), int(outlier_mode), float(k_or_rate),
+                                     float(cap_frac), _ptr(mask), _ptr(count), _ptr(workspace), _nbytes(workspace),
+                                     _stream(stream)), "xfp_quant_outliers")
+
+
+def xfp_quant_lloyd(W, mask, mu_sigma, bits: int, iters: int, codebook, idx, stream=None) -> None:
+    rows, cols = W.shape
+    _check(_lib().xfp_quant_lloyd(_ptr(W), _ptr(mask), _ptr(mu_sigma), rows, cols, int(bits), int(iters),
+                                  _ptr(codebook), _ptr(idx), _stream(stream)), "xfp_quant_lloyd")
+
+
+def xfp_quant_libfit_library(codebook, rows: int, bits: int, L: int, iters: int, lib, workspace, stream=None) -> None:
+    _check(_lib().xfp_quant_libfit_library(_ptr(codebook), int(rows), int(bits), int(L), int(iters), _ptr(lib),
+                                           _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "xfp_quant_libfit_library")
+
+
+def xfp_quant_libfit_assign(W, mask, mu_sigma, bits: int, L: int, lib, idx, gid, gscale, gmid, stream=None) -> None:
+    rows, cols = W.shape
+    _check(_lib().xfp_quant_libfit_assign(_ptr(W), _ptr(mask), _ptr(mu_sigma), rows, cols, int(bits), int(L),
+                                          _ptr(lib), _ptr(idx), _ptr(gid), _ptr(gscale), _ptr(gmid),
+                                          _stream(stream)), "xfp_quant_libfit_assign")
+
+
+def xfp_quant_residual(desc: XfpDesc, W, mask, idx, codebook, gid, gscale, gmid, out_rowptr, out_col, out_val,
+                       workspace, stream=None) -> None:
+    cap = 0 if out_col is None else out_col.numel()
+    _check(_lib().xfp_quant_residual(C.byref(desc), _ptr(W), _ptr(mask), _ptr(idx), _ptr(codebook), _ptr(gid),
+                                     _ptr(gscale), _ptr(gmid), _ptr(out_rowptr), _ptr(out_col), _ptr(out_val),
+                                     int(cap), _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "xfp_quant_residual")
+
+
+def xfp_quant_cosine(desc: XfpDesc, W, mask, idx, codebook, gid, gscale, gmid, cos, stream=None) -> None:
+    _check(_lib().xfp_quant_cosine(C.byref(desc), _ptr(W), _ptr(mask), _ptr(idx), _ptr(codebook), _ptr(gid),
+                                   _ptr(gscale), _ptr(gmid), _ptr(cos), _stream(stream)), "xfp_quant_cosine")
+
+
+def xfp_quant_median(v, median, workspace, stream=None) -> None:
+    _check(_lib().xfp_quant_median(_ptr(v), v.numel(), _ptr(median), _ptr(workspace), _nbytes(workspace),
+                                   _stream(stream)), "xfp_quant_median")
+
+
+class QuantBuffers:
+    """Device buffers xfp_quantize writes, sized for a rows x cols matrix (allocation only)."""
+
+    def __init__(self, rows: int, cols: int, mode: int, max_bits: int, lib_size: int, capacity: int, device="cuda"):
+        G = cols // 128
+        e = torch.empty
+        self.rows, self.cols, self.mode, self.lib_size = rows, cols, mode, lib_size
+        self.mask = e((rows, cols), dtype=torch.uint8, device=device)
+        self.idx = e((rows, cols), dtype=torch.uint8, device=device)
+        self.codebook = e((rows, 1 << max_bits), dtype=torch.int16, device=device)
+        self.lib = e((max(lib_size, 1), 1 << max_bits), dtype=torch.int16, device=device) if mode else None
+        self.gid = e((rows, G), dtype=torch.uint8, device=device) if mode else None
+        self.gscale = e((rows, G), dtype=torch.int16, device=device) if mode else None
+        self.gmid = e((rows, G), dtype=torch.int16, device=device) if mode else None
+        self.rowptr = e(rows + 1, dtype=torch.int32, device=device)
+        self.ocol = e(max(capacity, 4), dtype=torch.int32, device=device)
+        self.oval = e(max(capacity, 8), dtype=torch.int16, device=device)
+        self.capacity = capacity
+        self.cos = e(rows, dtype=torch.float64, device=device)
+        self.workspace = e(xfp_quant_workspace_size(rows, cols) + 256, dtype=torch.uint8, device=device)
+
+
+def xfp_quantize(mode: int, W: torch.Tensor, params: XfpQuantParams, candidates: Sequence[int], tau: float,
+                 buf: QuantBuffers, stream=None) -> XfpQuantResult:
+    """Algorithm 1 on the GPU; fills `buf` and returns the host-side result record."""
+    rows, cols = W.shape
+    cand = (C.c_int32 * len(candidates))(*[int(c) for c in candidates])
+    res = XfpQuantResult()
+    _check(_lib().xfp_quantize(int(mode), _ptr(W), rows, cols, C.byref(params), cand, len(candidates), float(tau),
+                               int(buf.lib_size if mode else 0), _ptr(buf.mask), _ptr(buf.idx), _ptr(buf.codebook),
+                               _ptr(buf.lib), _ptr(buf.gid), _ptr(buf.gscale), _ptr(buf.gmid), _ptr(buf.rowptr),
+                               _ptr(buf.ocol), _ptr(buf.oval), int(buf.capacity), _ptr(buf.cos), C.byref(res),
+                               _ptr(buf.workspace), _nbytes(buf.workspace), _stream(stream)), "xfp_quantize")
+    return res

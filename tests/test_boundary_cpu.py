@@ -18,13 +18,70 @@ def lib():
     return xfp.load_library()
 
 
-def test_exports_match_header(lib):
-    text = open(os.path.join(ROOT, "include", "xfp.h")).read()
+def _declared(header):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    declared = set(re.findall(r"\b(xfp_[a-z0-9_]+)\s*\(", text))
+    return set(re.findall(r"\b(xfp_[a-z0-9_]+)\s*\(", text))
+
+
+def test_exports_match_header(lib):
+    declared = _declared("xfp.h")
     assert declared and declared == set(binding.EXPORTS) | {n for n in declared if hasattr(lib, n)}
     for name in declared:
         assert hasattr(lib, name), name
+
+
+def test_encoder_exports_match_header(lib):
+    from paper_2605_14844_b200 import quant_binding
+    assert sorted(f for f in os.listdir(os.path.join(ROOT, "include")) if f.endswith(".h")) == ["xfp.h", "xfp_quant.h"]
+    declared = _declared("xfp_quant.h")
+    assert declared == set(quant_binding.QUANT_EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_encoder_rejects_bad_arguments_on_the_host(lib):
+    from paper_2605_14844_b200 import quant_binding as qb
+    qb._lib()
+    a, odd, n = C.c_void_p(0x1000), C.c_void_p(0x1008), None
+    sz = C.c_size_t()
+    assert lib.xfp_quant_workspace_size(64, 256, C.byref(sz)) == 0 and sz.value > 0
+    assert lib.xfp_quant_workspace_size(64, 200, C.byref(sz)) == 3
+    assert lib.xfp_quant_workspace_size(0, 256, C.byref(sz)) == 3
+    big = 1 << 30
+    assert lib.xfp_quant_stats(n, 100, 0, a, a, big, n) == 1
+    assert lib.xfp_quant_stats(odd, 100, 0, a, a, big, n) == 2
+    assert lib.xfp_quant_stats(a, 0, 0, a, a, big, n) == 3
+    assert lib.xfp_quant_stats(a, 100, 2, a, a, big, n) == 3
+    assert lib.xfp_quant_stats(a, 100, 0, a, a, 8, n) == 5
+    assert lib.xfp_quant_outliers(a, 100, a, 0, 4.0, 0.02, n, a, a, big, n) == 1
+    assert lib.xfp_quant_outliers(a, 100, a, 3, 4.0, 0.02, a, a, a, big, n) == 3
+    assert lib.xfp_quant_outliers(a, 100, a, 1, 1.5, 0.0, a, a, a, big, n) == 3          # rate > 1
+    assert lib.xfp_quant_outliers(a, 1 << 30, a, 0, 4.0, 0.02, a, a, a, 4096, n) == 5
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 256, 7, 20, a, a, n) == 3
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 200, 4, 20, a, a, n) == 3
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 16384, 4, 20, a, a, n) == 4                   # channel too long for shared memory
+    assert lib.xfp_quant_lloyd(a, odd, a, 64, 256, 4, 20, a, a, n) == 2
+    assert lib.xfp_quant_libfit_library(a, 64, 4, 0, 20, a, a, big, n) == 3
+    assert lib.xfp_quant_libfit_library(a, 64, 4, 32, 20, a, a, 64, n) == 5
+    assert lib.xfp_quant_libfit_assign(a, n, a, 64, 256, 4, 32, a, a, n, a, a, n) == 1
+    d = _desc(mode=1, lib_size=32)
+    assert lib.xfp_quant_residual(C.byref(d), a, a, a, a, n, n, n, a, a, a, 10, a, big, n) == 1   # V2a needs group data
+    d0 = _desc()
+    assert lib.xfp_quant_residual(C.byref(d0), a, a, a, a, n, n, n, a, n, n, 10, a, big, n) == 1
+    assert lib.xfp_quant_residual(C.byref(d0), a, a, a, a, n, n, n, a, a, a, 10, a, 64, n) == 5
+    assert lib.xfp_quant_cosine(C.byref(d0), a, n, a, a, n, n, n, n, n) == 1
+    assert lib.xfp_quant_median(a, 0, a, a, big, n) == 3
+    p = qb.XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 20, 0)
+    r = qb.XfpQuantResult()
+    cand = (C.c_int32 * 2)(4, 3)                                                          # not ascending
+    assert lib.xfp_quantize(0, a, 64, 256, C.byref(p), cand, 2, 0.96, 0, a, a, a, n, n, n, n, a, a, a, 100, a,
+                            C.byref(r), a, big, n) == 3
+    cand = (C.c_int32 * 1)(4)
+    assert lib.xfp_quantize(1, a, 64, 256, C.byref(p), cand, 1, 0.93, 32, a, a, a, n, n, n, n, a, a, a, 100, a,
+                            C.byref(r), a, big, n) == 1                                   # V2a needs its outputs
+    assert lib.xfp_quantize(0, a, 64, 256, C.byref(p), cand, 1, 0.96, 0, a, a, a, n, n, n, n, a, a, a, 100, a,
+                            C.byref(r), a, 128, n) == 5
 
 
 def _desc(**kw):
