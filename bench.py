@@ -13,6 +13,11 @@ values and columns, row pointers, x, y), microseconds per call, the HBM roofline
 kernel, the same measured end to end from host buffers, and the CPU oracle timed beside it.
 
 `--impl reference` times the CPU oracle alone on the same workload (bounded sample per step).
+
+`--encoder` is a separate, optional measurement (not the headline line): Algorithm 1 on one 4096 x 4096
+attention projection (float weights with heavy outlier columns -> extraction, per-channel Lloyd over the
+candidates {4, 5}, residual, cosine gate) through xfp_quantize on the GPU, with the oracle's encoder timed
+beside it on the host cores.
 """
 from __future__ import annotations
 
@@ -334,6 +339,42 @@ def algorithmic_bytes_from(pm, q) -> int:
     return (d.rows * d.cols * d.bits // 8 + d.rows * E * 2 + d.nnz * 4 + (d.rows + 1) * 4 + d.cols * 2 + d.rows * 2)
 
 
+def run_encoder(args):
+    """One JSON line: the GPU encoder on a dense-attention projection, the oracle's encoder beside it."""
+    import torch
+    from paper_2605_14844_b200 import quant_binding as qb
+    from paper_2605_14844_b200 import synth
+    W = synth.attention_weights(10, ROWS, COLS)
+    Wd = torch.from_numpy(W).cuda()
+    cands, tau = (4, 5), 0.96
+    buf = qb.QuantBuffers(ROWS, COLS, 0, max(cands), 0, int(0.02 * W.size))
+    params = qb.XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 20, 0)
+    walls = []
+    for it in range(args.warmup + 5):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        res = qb.xfp_quantize(0, Wd, params, cands, tau, buf)
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            walls.append(time.perf_counter() - t0)
+    gpu_s = statistics.median(walls)
+    line = {"metric": "XFP encoder (Algorithm 1, V2) weights per second", "value": W.size / gpu_s / 1e6,
+            "unit": "Mweights/s", "ms_per_matrix": gpu_s * 1e3, "n_gpus": 1, "higher_is_better": True,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "one 4096x4096 attention projection, heavy outlier columns, candidates {4,5}, "
+                                   "tau 0.96, 20 Lloyd rounds", "bits_chosen": int(res.bits), "nnz": int(res.nnz),
+                       "median_cos": res.median_cos}}
+    if not args.no_cpu_baseline:
+        from oracle import xfp_oracle as xo
+        t0 = time.perf_counter()
+        ref = xo.auto_select(W, "attention", cands, tau_strict=tau, iters=20)
+        cpu_s = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": W.size / cpu_s / 1e6, "unit": "Mweights/s", "cores": xo.threads(),
+                                "kind": "oracle", "sample": "the same matrix, whole", "seconds": cpu_s,
+                                "same_bits": int(ref.bits) == int(res.bits), "same_nnz": ref.nnz == int(res.nnz)}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -343,10 +384,14 @@ def main():
     ap.add_argument("--layers", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--encoder", action="store_true", help="time the GPU encoder instead of the decode path")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
-    if args.impl == "reference":
+    if args.encoder:
+        if rank == 0:
+            run_encoder(args)
+    elif args.impl == "reference":
         run_reference(args, rank)
     else:
         run_xfp(args, rank, world)

@@ -416,9 +416,17 @@ __global__ void __launch_bounds__(kLloydThreads) lloyd_kernel(const float* __res
     if (tid == 0) {
         double run = 0.0;
         pre[0] = 0.0;
-        for (int t = 0; t < K; ++t) {
-            run = __dadd_rn(run, s[t]);
-            pre[t + 1] = run;
+        for (int t = 0; t < K; t += 16) {   // K is a multiple of 128; loads of a batch are issued together
+            double v[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[e] = s[t + e];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                run = __dadd_rn(run, v[e]);
+                v[e] = run;
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) pre[t + 1 + e] = v[e];
         }
     }
     if (tid < E) {
@@ -635,20 +643,31 @@ __global__ void libfit_assign_rows(const double* __restrict__ u, const double* _
     asg[i] = best;
 }
 
-// centroid l, entry j <- mean of its members, summed in channel order; one thread per (l, j)
-__global__ void libfit_update(const double* __restrict__ u, const int* __restrict__ asg, int rows, int E, int L,
-                              double* cen, int* changed, const int* done) {
+// centroid l <- mean of its members, every entry summed in channel order.  One block per centroid: the
+// members of each tile of 256 channels are compacted in order, then thread j adds them to entry j.
+__global__ void __launch_bounds__(256) libfit_update(const double* __restrict__ u, const int* __restrict__ asg,
+                                                      int rows, int E, int L, double* cen, int* changed,
+                                                      const int* done) {
+    __shared__ int sh[8];
+    __shared__ int total;
+    __shared__ int member[256];
     if (*done) return;
     const int l = blockIdx.x, j = threadIdx.x;
-    if (j >= E) return;
     double acc = 0.0;
     long long cnt = 0;
-    for (int i = 0; i < rows; ++i)
-        if (asg[i] == l) {
-            acc = __dadd_rn(acc, u[(int64_t)i * E + j]);
-            ++cnt;
-        }
-    if (cnt > 0) {
+    for (int i0 = 0; i0 < rows; i0 += 256) {
+        const int i = i0 + threadIdx.x;
+        const int f = i < rows && asg[i] == l;
+        const int off = block_excl_scan(f, sh, &total);
+        if (f) member[off] = i;
+        __syncthreads();
+        const int n = total;
+        if (j < E)
+            for (int m = 0; m < n; ++m) acc = __dadd_rn(acc, u[(int64_t)member[m] * E + j]);
+        cnt += n;
+        __syncthreads();
+    }
+    if (j < E && cnt > 0) {
         const double m = __ddiv_rn(acc, (double)cnt);
         if (m != cen[l * E + j]) { cen[l * E + j] = m; *changed = 1; }
     }
@@ -678,87 +697,107 @@ __global__ void libfit_store(const double* __restrict__ cen, int E, uint16_t* li
 
 // ------------------------------------------------------------------ LibFit: per-group assignment
 
-// One block per (channel, group of 128): thread l < L scores library entry l serially over the 128
-// values; then the 128 threads index the values against the winner.
+// A block of 128 threads takes `gpb` consecutive groups of 128 weights (4 when L <= 32).  Thread (s, l)
+// scores library entry l on group s serially over the 128 values; one thread per group picks the winner;
+// then the 128 threads index each group against its winner.
 __global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restrict__ W,
                                                             const uint8_t* __restrict__ mask,
-                                                            const double* __restrict__ ms, int K, int bits, int L,
-                                                            const uint16_t* __restrict__ lib, uint8_t* idx,
-                                                            uint8_t* gid, uint16_t* gscale, uint16_t* gmid) {
+                                                            const double* __restrict__ ms, int64_t groups, int bits,
+                                                            int L, int gpb, const uint16_t* __restrict__ lib,
+                                                            uint8_t* idx, uint8_t* gid, uint16_t* gscale,
+                                                            uint16_t* gmid) {
     constexpr int GS = 128;
-    __shared__ double gv[GS];
-    __shared__ double red_lo[4], red_hi[4];
+    __shared__ double gv[4][GS];
+    __shared__ double red_lo[4][4], red_hi[4][4];
     __shared__ double sse[256];
-    __shared__ double dec[64];
-    __shared__ int s_best;
+    __shared__ double dec[4][64];
+    __shared__ uint16_t s_mid[4], s_sc[4];
+    __shared__ int s_best[4], s_const[4];
     const int E = 1 << bits;
-    const int G = K / GS;
-    const int row = blockIdx.x / G, g = blockIdx.x % G;
     const int tid = threadIdx.x;
+    const int lw = GS / gpb;                   // threads per group while scoring
     const double mu = ms[0];
-    const int64_t t0 = (int64_t)row * K + (int64_t)g * GS;
-    const double v = bulk_value(W, mask, t0 + tid, mu);
-    gv[tid] = v;
-    double lo = v, hi = v;
-    for (int d = 16; d > 0; d >>= 1) {
-        lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, d));
-        hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, d));
-    }
-    if ((tid & 31) == 0) { red_lo[tid >> 5] = lo; red_hi[tid >> 5] = hi; }
-    __syncthreads();
-    lo = fmin(fmin(red_lo[0], red_lo[1]), fmin(red_lo[2], red_lo[3]));
-    hi = fmax(fmax(red_hi[0], red_hi[1]), fmax(red_hi[2], red_hi[3]));
-    const int64_t go = (int64_t)row * G + g;
-    if (hi == lo) {   // a constant group: scale 0, entry 0, indices 0
-        if (tid == 0) {
-            gmid[go] = d2h(__dmul_rn(0.5, __dadd_rn(hi, lo)));
-            gscale[go] = 0;
-            gid[go] = 0;
+    const int64_t g0 = (int64_t)blockIdx.x * gpb;
+    for (int s = 0; s < gpb; ++s) {
+        const int64_t grp = g0 + s;
+        if (grp >= groups) break;
+        const double v = bulk_value(W, mask, grp * GS + tid, mu);
+        gv[s][tid] = v;
+        double lo = v, hi = v;
+        for (int d = 16; d > 0; d >>= 1) {
+            lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+            hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, d));
         }
-        idx[t0 + tid] = 0;
-        return;
-    }
-    const uint16_t mid16 = d2h(__dmul_rn(0.5, __dadd_rn(hi, lo)));
-    const uint16_t sc16 = d2h(__dmul_rn(0.5, __dsub_rn(hi, lo)));
-    for (int l = tid; l < L; l += GS) {
-        double d16[64];
-        for (int j = 0; j < E; ++j) d16[j] = h2d(v2a_value16(sc16, lib[l * E + j], mid16));
-        double acc = 0.0;
-        for (int t = 0; t < GS; ++t) {
-            const double x = gv[t];
-            double bd = fabs(__dsub_rn(x, d16[0]));
-            int bj = 0;
-            for (int j = 1; j < E; ++j) {
-                const double d = fabs(__dsub_rn(x, d16[j]));
-                if (d < bd) { bd = d; bj = j; }
-            }
-            const double d = __dsub_rn(x, d16[bj]);
-            acc = __dadd_rn(acc, __dmul_rn(d, d));
-        }
-        sse[l] = acc;
+        if ((tid & 31) == 0) { red_lo[s][tid >> 5] = lo; red_hi[s][tid >> 5] = hi; }
     }
     __syncthreads();
-    if (tid == 0) {
-        int best = 0;
-        double b = INFINITY;
-        for (int l = 0; l < L; ++l)
-            if (sse[l] < b) { b = sse[l]; best = l; }
-        s_best = best;
-        gid[go] = (uint8_t)best;
-        gscale[go] = sc16;
-        gmid[go] = mid16;
+    if (tid < gpb && g0 + tid < groups) {
+        const double lo = fmin(fmin(red_lo[tid][0], red_lo[tid][1]), fmin(red_lo[tid][2], red_lo[tid][3]));
+        const double hi = fmax(fmax(red_hi[tid][0], red_hi[tid][1]), fmax(red_hi[tid][2], red_hi[tid][3]));
+        s_mid[tid] = d2h(__dmul_rn(0.5, __dadd_rn(hi, lo)));
+        s_sc[tid] = d2h(__dmul_rn(0.5, __dsub_rn(hi, lo)));
+        s_const[tid] = hi == lo;
     }
-    __syncthreads();
-    if (tid < E) dec[tid] = h2d(v2a_value16(sc16, lib[s_best * E + tid], mid16));
     __syncthreads();
     {
-        double bd = fabs(__dsub_rn(v, dec[0]));
-        int bj = 0;
-        for (int j = 1; j < E; ++j) {
-            const double d = fabs(__dsub_rn(v, dec[j]));
-            if (d < bd) { bd = d; bj = j; }
+        const int s = tid / lw;
+        const int64_t grp = g0 + s;
+        if (grp < groups && !s_const[s]) {
+            const uint16_t mid16 = s_mid[s], sc16 = s_sc[s];
+            for (int l = tid % lw; l < L; l += lw) {
+                double d16[64];
+                for (int j = 0; j < E; ++j) d16[j] = h2d(v2a_value16(sc16, lib[l * E + j], mid16));
+                double acc = 0.0;
+                for (int t = 0; t < GS; ++t) {
+                    const double x = gv[s][t];
+                    double bd = fabs(__dsub_rn(x, d16[0]));
+                    int bj = 0;
+                    for (int j = 1; j < E; ++j) {
+                        const double d = fabs(__dsub_rn(x, d16[j]));
+                        if (d < bd) { bd = d; bj = j; }
+                    }
+                    const double d = __dsub_rn(x, d16[bj]);
+                    acc = __dadd_rn(acc, __dmul_rn(d, d));
+                }
+                sse[gpb == 1 ? l : s * lw + l] = acc;
+            }
         }
-        idx[t0 + tid] = (uint8_t)bj;
+    }
+    __syncthreads();
+    if (tid < gpb && g0 + tid < groups) {
+        const int64_t grp = g0 + tid;
+        int best = 0;
+        if (!s_const[tid]) {
+            double b = INFINITY;
+            for (int l = 0; l < L; ++l) {
+                const double e = sse[gpb == 1 ? l : tid * lw + l];
+                if (e < b) { b = e; best = l; }
+            }
+        }
+        s_best[tid] = best;
+        gid[grp] = (uint8_t)best;
+        gscale[grp] = s_const[tid] ? (uint16_t)0 : s_sc[tid];   // a constant group: scale 0, entry 0, indices 0
+        gmid[grp] = s_mid[tid];
+    }
+    __syncthreads();
+    for (int e = tid; e < gpb * E; e += GS) {
+        const int s = e / E, j = e % E;
+        if (g0 + s < groups) dec[s][j] = h2d(v2a_value16(s_sc[s], lib[s_best[s] * E + j], s_mid[s]));
+    }
+    __syncthreads();
+    for (int s = 0; s < gpb; ++s) {
+        const int64_t grp = g0 + s;
+        if (grp >= groups) break;
+        int bj = 0;
+        if (!s_const[s]) {
+            const double v = gv[s][tid];
+            double bd = fabs(__dsub_rn(v, dec[s][0]));
+            for (int j = 1; j < E; ++j) {
+                const double d = fabs(__dsub_rn(v, dec[s][j]));
+                if (d < bd) { bd = d; bj = j; }
+            }
+        }
+        idx[grp * GS + tid] = (uint8_t)bj;
     }
 }
 
@@ -936,7 +975,7 @@ int xfp_quant_libfit_library(const uint16_t* codebook, int32_t rows, int32_t bit
     libfit_flags_init<<<1, 1, 0, s>>>(w.flags, w.flags + 1);
     for (int it = 0; it < iters; ++it) {
         libfit_assign_rows<<<rb, 256, 0, s>>>(w.u, w.cen, rows, E, L, w.asg, w.flags + 1);
-        libfit_update<<<L, 64, 0, s>>>(w.u, w.asg, rows, E, L, w.cen, w.flags, w.flags + 1);
+        libfit_update<<<L, 256, 0, s>>>(w.u, w.asg, rows, E, L, w.cen, w.flags, w.flags + 1);
         libfit_round_end<<<1, 1, 0, s>>>(w.flags, w.flags + 1);
     }
     libfit_store<<<L, 32, 0, s>>>(w.cen, E, lib);
@@ -955,8 +994,9 @@ int xfp_quant_libfit_assign(const float* W, const uint8_t* mask, const double* m
     if (bits < 2 || bits > 6 || L < 1 || L > 256) return XFP_ERR_SHAPE;
     const int64_t groups = (int64_t)rows * (cols / 128);
     if (groups > 0x7fffffff) return XFP_ERR_UNSUPPORTED;
-    libfit_group_kernel<<<(unsigned)groups, 128, 0, (cudaStream_t)stream>>>(W, mask, mu_sigma, cols, bits, L, lib, idx,
-                                                                            gid, gscale, gmid);
+    const int gpb = L <= 32 ? 4 : (L <= 64 ? 2 : 1);
+    libfit_group_kernel<<<(unsigned)((groups + gpb - 1) / gpb), 128, 0, (cudaStream_t)stream>>>(
+        W, mask, mu_sigma, groups, bits, L, gpb, lib, idx, gid, gscale, gmid);
     return cudaGetLastError() == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 

@@ -25,6 +25,11 @@
         {0, 0.5, 1, 2} % (seeded), V2 and V2a on the same draws; one token through the stack is one CUDA graph.  Prints
         milliseconds per token and effective GB/s.
 
+    python -m paper_2605_14844_b200.probe quant MODE ROWS COLS BITS [REPS]
+        the encoder on one synthetic float matrix (Gaussian bulk with heavy outlier columns for V2, 0.1 % uniform
+        outliers for V2a): device time of every stage (statistics, extraction, Lloyd, LibFit, residual,
+        cosine, median) and wall time of the whole xfp_quantize call with BITS as its only candidate.
+
 MODE 0 = V2, 1 = V2a; PLACEMENT uniform | clustered | one_row.  Inputs come from synth.random_quantized.
 """
 from __future__ import annotations
@@ -220,7 +225,72 @@ def stack(layers=48, reps=5):
         torch.cuda.empty_cache()
 
 
+def quant(mode, rows, cols, bits, reps=3):
+    """Device time per encoder stage, and the whole Algorithm 1 call, on one rows x cols float matrix."""
+    from . import XfpDesc
+    from . import quant_binding as qb
+    if mode == 0:
+        W = synth.attention_weights(10, rows, cols)
+    else:
+        W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, 30), 0.001, 31)
+    Wd = torch.from_numpy(W).cuda()
+    L = 32
+    cap = int(0.02 * W.size)
+    buf = qb.QuantBuffers(rows, cols, mode, bits, L, cap)
+    ms = torch.zeros(2, dtype=torch.float64, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.int64, device="cuda")
+    med = torch.zeros(2, dtype=torch.float64, device="cuda")
+    desc = XfpDesc(mode, rows, cols, bits, 128, L if mode else 0, 32, 0)
+    table = buf.lib if mode else buf.codebook
+    stages = [
+        ("stats", lambda: qb.xfp_quant_stats(Wd, 0, ms, buf.workspace)),
+        ("outliers", lambda: qb.xfp_quant_outliers(Wd, ms, 0, 4.0, 0.02, buf.mask, cnt, buf.workspace)),
+        ("lloyd", lambda: qb.xfp_quant_lloyd(Wd, buf.mask, ms, bits, 20, buf.codebook, buf.idx)),
+    ]
+    if mode:
+        stages += [
+            ("libfit_library", lambda: qb.xfp_quant_libfit_library(buf.codebook, rows, bits, L, 20, buf.lib, buf.workspace)),
+            ("libfit_assign", lambda: qb.xfp_quant_libfit_assign(Wd, buf.mask, ms, bits, L, buf.lib, buf.idx, buf.gid,
+                                                                 buf.gscale, buf.gmid)),
+        ]
+    stages += [
+        ("residual", lambda: qb.xfp_quant_residual(desc, Wd, buf.mask, buf.idx, table, buf.gid, buf.gscale, buf.gmid,
+                                                   buf.rowptr, buf.ocol, buf.oval, buf.workspace)),
+        ("cosine", lambda: qb.xfp_quant_cosine(desc, Wd, buf.mask, buf.idx, table, buf.gid, buf.gscale, buf.gmid, buf.cos)),
+        ("median", lambda: qb.xfp_quant_median(buf.cos, med, buf.workspace)),
+    ]
+    out = {}
+    for name, fn in stages:
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        out[name + "_ms"] = round(float(np.median(ts)), 4)
+    import time
+    params = qb.XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 20, 0)
+    walls = []
+    for _ in range(reps):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        res = qb.xfp_quantize(mode, Wd, params, (bits,), 0.0, buf)
+        torch.cuda.synchronize()
+        walls.append((time.perf_counter() - t0) * 1e3)
+    print(json.dumps(dict(workload="encoder", mode=mode, rows=rows, cols=cols, bits=bits, nnz=int(res.nnz),
+                          median_cos=round(res.median_cos, 6), stages=out, stage_sum_ms=round(sum(out.values()), 3),
+                          quantize_wall_ms=round(float(np.median(walls)), 3),
+                          Mweights_per_s=round(rows * cols / np.median(walls) / 1e3, 1))), flush=True)
+
+
 def main(argv):
+    if len(argv) > 1 and argv[1] == "quant":
+        quant(*(int(v) for v in argv[2:7]))
+        return 0
     if len(argv) > 1 and argv[1] == "moe":
         moe(*(int(v) for v in argv[2:5]))
         return 0

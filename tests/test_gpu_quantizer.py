@@ -298,3 +298,53 @@ def test_quantize_reports_a_small_outlier_buffer():
     buf = qb.QuantBuffers(rows, cols, 0, 4, 0, 16)
     with pytest.raises(xfp.XfpError):
         qb.xfp_quantize(0, _dev(W), _params(), (4,), 0.9, buf)
+
+
+# ------------------------------------------------------------------ the paper's layer sizes
+
+@pytest.mark.parametrize("mode,rows,cols,bits", [(0, 4096, 4096, 4), (1, 3072, 4096, 3)])
+def test_full_size_layers_are_bit_exact(mode, rows, cols, bits):
+    """A dense-attention projection (V2, heavy outlier columns) and a routed expert's gate_up projection (V2a)
+    at the sizes the decode benchmarks use, every output of every stage compared in full."""
+    L = 32
+    if mode == 0:
+        W = synth.attention_weights(10, rows, cols)
+    else:
+        W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, 30), 0.001, 31)
+    mask, mu, sg = xo.outlier_mask(W)
+    ref = xo.quantize_v2(W, bits, mask, mu, 20) if mode == 0 else xo.quantize_v2a(W, bits, mask, mu, L, 20)
+    Wd, msd, ws = _dev(W), _ms(mu, sg), _ws(rows, cols)
+    maskd = torch.empty((rows, cols), dtype=torch.uint8, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.int64, device="cuda")
+    qb.xfp_quant_outliers(Wd, msd, 0, 4.0, 0.02, maskd, cnt, ws)
+    assert np.array_equal(maskd.cpu().numpy(), mask)
+    E = 1 << bits
+    cb = torch.empty((rows, E), dtype=torch.int16, device="cuda")
+    idx = torch.empty((rows, cols), dtype=torch.uint8, device="cuda")
+    qb.xfp_quant_lloyd(Wd, maskd, msd, bits, 20, cb, idx)
+    gid = gs = gm = None
+    table = cb
+    if mode:
+        G = cols // 128
+        lib = torch.empty((L, E), dtype=torch.int16, device="cuda")
+        gid = torch.empty((rows, G), dtype=torch.uint8, device="cuda")
+        gs = torch.empty((rows, G), dtype=torch.int16, device="cuda")
+        gm = torch.empty((rows, G), dtype=torch.int16, device="cuda")
+        qb.xfp_quant_libfit_library(cb, rows, bits, L, 20, lib, ws)
+        qb.xfp_quant_libfit_assign(Wd, maskd, msd, bits, L, lib, idx, gid, gs, gm)
+        table = lib
+        assert np.array_equal(gid.cpu().numpy(), ref.gid)
+        assert np.array_equal(_u16(gs), ref.gscale) and np.array_equal(_u16(gm), ref.gmid)
+    assert np.array_equal(_u16(table), ref.codebook)
+    assert np.array_equal(idx.cpu().numpy(), ref.idx)
+    nnz = ref.nnz
+    rowptr = torch.empty(rows + 1, dtype=torch.int32, device="cuda")
+    ocol = torch.empty(nnz, dtype=torch.int32, device="cuda")
+    oval = torch.empty(nnz + 8, dtype=torch.int16, device="cuda")[:nnz]
+    desc = xfp.XfpDesc(mode, rows, cols, bits, 128, L if mode else 0, 32, 0)
+    qb.xfp_quant_residual(desc, Wd, maskd, idx, table, gid, gs, gm, rowptr, ocol, oval, ws)
+    assert np.array_equal(rowptr.cpu().numpy(), ref.rowptr)
+    assert np.array_equal(ocol.cpu().numpy(), ref.ocol) and np.array_equal(_u16(oval), ref.oval)
+    cos = torch.empty(rows, dtype=torch.float64, device="cuda")
+    qb.xfp_quant_cosine(desc, Wd, maskd, idx, table, gid, gs, gm, cos)
+    assert np.max(np.abs(cos.cpu().numpy() - xo.row_cosine(W, xo.dequant(ref)))) <= 1e-12
