@@ -225,6 +225,43 @@ __global__ void median_finish(const SelState* st, int64_t n, double scale, doubl
     *out = scale == 1.0 ? m : __dmul_rn(scale, m);
 }
 
+// The same descent for a short array of doubles (the per-channel cosines), one block, one launch.
+__global__ void __launch_bounds__(1024) median_small_kernel(const double* __restrict__ v, int n, double* out) {
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ long long s_k;
+    __shared__ double val[2];
+    const SrcDouble src{v};
+    for (int slot = 0; slot < 2; ++slot) {
+        if (threadIdx.x == 0) { s_prefix = 0; s_k = slot == 0 ? (n - 1) / 2 : n / 2; }
+        for (int shift = 56; shift >= 0; shift -= 8) {
+            if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+            __syncthreads();
+            const unsigned long long prefix = s_prefix;
+            for (int t = threadIdx.x; t < n; t += 1024) {
+                const unsigned long long key = src.key(t, 0.0);
+                if (shift == 56 || ((key ^ prefix) >> (shift + 8)) == 0) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                long long k = s_k;
+                int d;
+                for (d = 0; d < 255; ++d) {
+                    const long long c = hist[d];
+                    if (k < c) break;
+                    k -= c;
+                }
+                s_k = k;
+                s_prefix = prefix | ((unsigned long long)d << shift);
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) val[slot] = unflip(s_prefix);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = (n & 1) ? val[1] : __dmul_rn(0.5, __dadd_rn(val[0], val[1]));
+}
+
 template <class Src>
 static cudaError_t run_select(Src src, int64_t n, SelState* st, cudaStream_t s) {
     int blocks = (int)((n + 256 * 16 - 1) / (256 * 16));
@@ -374,68 +411,141 @@ __global__ void __launch_bounds__(256) tie_apply(Src src, int64_t n, const SelSt
 
 // ------------------------------------------------------------------ Lloyd, one channel per block
 
-constexpr int kLloydThreads = 512;
+constexpr int kLloydThreads = 256;
+
+#ifdef XFP_TRACE
+// phase boundaries of block 0 (clock64), read back by xfp_debug_lloyd_phases: a timing probe
+__device__ long long g_lloyd_phase[8];
+#define LLOYD_STAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_lloyd_phase[i] = clock64(); } while (0)
+#else
+#define LLOYD_STAMP(i) do { } while (0)
+#endif
 
 __device__ __forceinline__ double bulk_value(const float* __restrict__ W, const uint8_t* __restrict__ mask,
                                              int64_t t, double mu) {
     return (mask != nullptr && mask[t]) ? mu : (double)W[t];
 }
 
-__global__ void __launch_bounds__(kLloydThreads) lloyd_kernel(const float* __restrict__ W,
+// The channel's bulk values in ascending order without storing them as doubles: the weights that were not
+// extracted, sorted as floats, with the m copies of mu (one per extracted position) inserted at p0.
+struct SortedBulk {
+    const float* r;
+    int p0, m;
+    double mu;
+    __device__ __forceinline__ double at(int t) const {   // one load, then a select: no branch
+        const int u = t < p0 ? t : (t - m > 0 ? t - m : 0);
+        const double v = (double)r[u];
+        return (t >= p0 && t < p0 + m) ? mu : v;
+    }
+};
+
+__global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __restrict__ W,
                                                                const uint8_t* __restrict__ mask,
                                                                const double* __restrict__ ms, int K, int Kp2,
                                                                int bits, int iters, uint16_t* __restrict__ cb16,
                                                                uint8_t* __restrict__ idx) {
     extern __shared__ double sm[];
-    double* s = sm;            // [Kp2] the channel's bulk values, ascending (padding = +inf)
-    double* pre = sm + Kp2;    // [K + 1] serial prefix sums of s
+    double* pre = sm;                      // [K + 1] serial prefix sums of the sorted bulk values
+    float* r = (float*)(sm + K + 1);       // [Kp2] kept weights, ascending (extracted slots and padding = +inf)
     __shared__ double c[64];
     __shared__ double e16[64];
     __shared__ int cut[65];
+    __shared__ int s_m, s_p0;
     const int tid = threadIdx.x;
     const int E = 1 << bits;
     const int64_t row0 = (int64_t)blockIdx.x * K;
     const double mu = ms[0];
 
-    for (int k = tid; k < Kp2; k += kLloydThreads) s[k] = k < K ? bulk_value(W, mask, row0 + k, mu) : INFINITY;
+    LLOYD_STAMP(0);
+    if (tid == 0) s_m = 0;
     __syncthreads();
-    // bitonic sort, ascending
+    int extracted = 0;
+    for (int kb = tid; kb < Kp2; kb += 8 * kLloydThreads) {   // eight loads in flight per thread
+        float v[8];
+        uint8_t x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int k = kb + e * kLloydThreads;
+            v[e] = k < K ? W[row0 + k] : INFINITY;
+            x[e] = (k < K && mask != nullptr) ? mask[row0 + k] : (uint8_t)0;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int k = kb + e * kLloydThreads;
+            if (k < Kp2) r[k] = x[e] ? INFINITY : v[e];
+            extracted += x[e] != 0;
+        }
+    }
+    if (extracted) atomicAdd(&s_m, extracted);
+    __syncthreads();
+    LLOYD_STAMP(1);
+    // bitonic sort, ascending; a thread's eight pairs of a stage are loaded before any is written back
+    const int half = Kp2 >> 1;
     for (int size = 2; size <= Kp2; size <<= 1) {
         for (int j = size >> 1; j > 0; j >>= 1) {
-            for (int p = tid; p < (Kp2 >> 1); p += kLloydThreads) {
-                const int i = ((p & ~(j - 1)) << 1) | (p & (j - 1));
-                const int q = i + j;
-                const bool asc = (i & size) == 0;
-                const double a = s[i], b = s[q];
-                if ((a > b) == asc) { s[i] = b; s[q] = a; }
+            for (int pb = tid; pb < half; pb += 8 * kLloydThreads) {
+                int ia[8];
+                float a[8], b[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int p = pb + e * kLloydThreads;
+                    ia[e] = p < half ? (((p & ~(j - 1)) << 1) | (p & (j - 1))) : -1;
+                    if (ia[e] >= 0) { a[e] = r[ia[e]]; b[e] = r[ia[e] + j]; }
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (ia[e] >= 0 && (a[e] > b[e]) == ((ia[e] & size) == 0)) { r[ia[e]] = b[e]; r[ia[e] + j] = a[e]; }
             }
             __syncthreads();
         }
     }
-    // serial prefix sums: cell sums below are differences of these, as in a one-pass CPU evaluation
+    LLOYD_STAMP(2);
+    if (tid == 0) {   // where mu sits among the kept weights
+        int lo = 0, hi = K - s_m;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((double)r[mid] <= mu) lo = mid + 1; else hi = mid;
+        }
+        s_p0 = lo;
+    }
+    __syncthreads();
+    SortedBulk s{r, s_p0, s_m, mu};
+    // serial prefix sums: cell sums below are differences of these, as in a one-pass CPU evaluation.
+    // All threads first lay the sorted values out as doubles in pre[1..K]; one thread then scans in place,
+    // fetching the next eight values before it starts the current chain of eight dependent adds.
+    for (int t = tid; t < K; t += kLloydThreads) pre[t + 1] = s.at(t);
+    __syncthreads();
     if (tid == 0) {
         double run = 0.0;
+        double f[8], g[8];
         pre[0] = 0.0;
-        for (int t = 0; t < K; t += 16) {   // K is a multiple of 128; loads of a batch are issued together
-            double v[16];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) v[e] = s[t + e];
+        for (int e = 0; e < 8; ++e) f[e] = pre[1 + e];
+        for (int t = 0; t < K; t += 8) {   // K is a multiple of 128
+            if (t + 8 < K) {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                run = __dadd_rn(run, v[e]);
-                v[e] = run;
+                for (int e = 0; e < 8; ++e) g[e] = pre[t + 9 + e];
             }
 #pragma unroll
-            for (int e = 0; e < 16; ++e) pre[t + 1 + e] = v[e];
+            for (int e = 0; e < 8; ++e) {
+                run = __dadd_rn(run, f[e]);
+                f[e] = run;
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) pre[t + 1 + e] = f[e];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = g[e];
         }
     }
-    if (tid < E) {
-        long long q = (long long)floor(__ddiv_rn(__dmul_rn(__dadd_rn((double)tid, 0.5), (double)K), (double)E));
+    if (tid >= 32 && tid < 32 + E) {   // a warp other than the one that runs the prefix
+        const int j = tid - 32;
+        long long q = (long long)floor(__ddiv_rn(__dmul_rn(__dadd_rn((double)j, 0.5), (double)K), (double)E));
         if (q >= K) q = K - 1;
-        c[tid] = s[q];
+        c[j] = s.at((int)q);
     }
-    if (tid == 0) { cut[0] = 0; cut[E] = K; }
+    if (tid == 32) { cut[0] = 0; cut[E] = K; }
     __syncthreads();
+    LLOYD_STAMP(3);
 
     for (int it = 0; it < iters; ++it) {
         // cell j = (b_{j-1}, b_j], b_j the midpoint of entries j and j+1: cut[j+1] = #{t : s[t] <= b_j}
@@ -444,7 +554,7 @@ __global__ void __launch_bounds__(kLloydThreads) lloyd_kernel(const float* __res
             int lo = 0, hi = K;
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
-                if (s[mid] <= b) lo = mid + 1; else hi = mid;
+                if (s.at(mid) <= b) lo = mid + 1; else hi = mid;
             }
             cut[tid + 1] = lo;
         }
@@ -459,6 +569,7 @@ __global__ void __launch_bounds__(kLloydThreads) lloyd_kernel(const float* __res
         }
         if (!__syncthreads_or(changed)) break;
     }
+    LLOYD_STAMP(4);
     if (tid < E) {
         const uint16_t h = d2h(c[tid]);
         cb16[(int64_t)blockIdx.x * E + tid] = h;
@@ -476,6 +587,7 @@ __global__ void __launch_bounds__(kLloydThreads) lloyd_kernel(const float* __res
         }
         idx[row0 + k] = (uint8_t)best;
     }
+    LLOYD_STAMP(5);
 }
 
 // ------------------------------------------------------------------ decoded value of a stored index
@@ -851,7 +963,7 @@ static int lloyd_smem(int cols, int* kp2_out) {
     int kp2 = 1;
     while (kp2 < cols) kp2 <<= 1;
     *kp2_out = kp2;
-    return (int)(sizeof(double) * ((size_t)kp2 + (size_t)cols + 1));
+    return (int)(sizeof(double) * ((size_t)cols + 1) + sizeof(float) * (size_t)kp2);
 }
 
 static Unpacked unpacked_of(const xfp_desc* d, const uint8_t* idx, const uint16_t* cb, const uint8_t* gid,
@@ -951,7 +1063,8 @@ int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma,
     int kp2;
     const int smem = lloyd_smem(cols, &kp2);
     if (smem > 227 * 1024 - 2048) return XFP_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(lloyd_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess)
         return XFP_ERR_CUDA;
     lloyd_kernel<<<rows, kLloydThreads, smem, (cudaStream_t)stream>>>(W, mask, mu_sigma, cols, kp2, bits, iters,
                                                                       codebook, idx);
@@ -1047,6 +1160,10 @@ int xfp_quant_median(const double* v, int64_t n, double* median, void* workspace
     if (!aligned16(v) || !aligned16(workspace)) return XFP_ERR_ALIGN;
     if (n < 1) return XFP_ERR_SHAPE;
     if (workspace_bytes < carve(nullptr, 1, 128).bytes) return XFP_ERR_BUFFER_TOO_SMALL;
+    if (n <= (1 << 16)) {
+        median_small_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(v, (int)n, median);
+        return cudaGetLastError() == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+    }
     Workspace w = carve(workspace, 1, 128);
     SrcDouble src{v};
     return run_median(src, n, 1.0, false, median, w.sel, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
@@ -1124,5 +1241,12 @@ int xfp_quantize(int32_t mode, const float* W, int32_t rows, int32_t cols, const
     return xfp_quant_residual(&d, W, mask, idx, mode ? lib : codebook, gid, gscale, gmid, out_rowptr, out_col, out_val,
                               capacity, workspace, need, stream);
 }
+
+#ifdef XFP_TRACE
+/* timing probe: clock64 at the six phase boundaries of block 0 of the last xfp_quant_lloyd launch (host array) */
+int xfp_debug_lloyd_phases(long long* out) {
+    return cudaMemcpyFromSymbol(out, g_lloyd_phase, sizeof(long long) * 8) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+}
+#endif
 
 }  // extern "C"

@@ -60,7 +60,7 @@ def test_encoder_rejects_bad_arguments_on_the_host(lib):
     assert lib.xfp_quant_outliers(a, 1 << 30, a, 0, 4.0, 0.02, a, a, a, 4096, n) == 5
     assert lib.xfp_quant_lloyd(a, n, a, 64, 256, 7, 20, a, a, n) == 3
     assert lib.xfp_quant_lloyd(a, n, a, 64, 200, 4, 20, a, a, n) == 3
-    assert lib.xfp_quant_lloyd(a, n, a, 64, 16384, 4, 20, a, a, n) == 4                   # channel too long for shared memory
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 32768, 4, 20, a, a, n) == 4                   # channel too long for shared memory
     assert lib.xfp_quant_lloyd(a, odd, a, 64, 256, 4, 20, a, a, n) == 2
     assert lib.xfp_quant_libfit_library(a, 64, 4, 0, 20, a, a, big, n) == 3
     assert lib.xfp_quant_libfit_library(a, 64, 4, 32, 20, a, a, 64, n) == 5

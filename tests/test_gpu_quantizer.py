@@ -229,7 +229,7 @@ def test_residual_and_cosine(mode, bits):
 
 def test_median_handles_signs_and_duplicates():
     rng = np.random.default_rng(2)
-    for n in (1, 2, 5, 1000, 4097):
+    for n in (1, 2, 5, 1000, 4097, 65536, 65537, 200000):   # one-block kernel up to 65536, device-wide above
         v = np.round(rng.standard_normal(n), 1)          # many duplicates, both signs, zeros
         med = torch.zeros(2, dtype=torch.float64, device="cuda")
         qb.xfp_quant_median(_dev(v), med, _ws(1, 128))
