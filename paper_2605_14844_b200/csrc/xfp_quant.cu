@@ -547,16 +547,31 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
     __syncthreads();
     LLOYD_STAMP(3);
 
+    // P lanes share one boundary search (P = 256 / 2^N, at most a warp): each round probes P positions of
+    // the remaining range at once, so 4096 values take three rounds at N = 4 instead of twelve steps.
+    const int P = (kLloydThreads >> bits) > 32 ? 32 : (kLloydThreads >> bits);
+    const int jb = tid / P, sub = tid % P;
+    const unsigned gmask = (P == 32 ? 0xffffffffu : ((1u << P) - 1u)) << ((tid & 31) & ~(P - 1));
     for (int it = 0; it < iters; ++it) {
         // cell j = (b_{j-1}, b_j], b_j the midpoint of entries j and j+1: cut[j+1] = #{t : s[t] <= b_j}
-        if (tid < E - 1) {
-            const double b = __dmul_rn(0.5, __dadd_rn(c[tid], c[tid + 1]));
-            int lo = 0, hi = K;
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (s.at(mid) <= b) lo = mid + 1; else hi = mid;
+        {
+            const bool mine = jb < E - 1;
+            const double b = mine ? __dmul_rn(0.5, __dadd_rn(c[jb], c[jb + 1])) : 0.0;
+            int lo = 0, hi = mine ? K : 0;   // every t < lo has s[t] <= b, every t >= hi has s[t] > b
+            while (__any_sync(0xffffffffu, lo < hi)) {
+                const int step = (hi - lo + P - 1) / P;
+                const int pos = lo + (sub + 1) * step - 1;
+                const bool below = lo < hi && pos < hi && s.at(pos) <= b;
+                const int cnt = __popc(__ballot_sync(0xffffffffu, below) & gmask);   // the probes are ordered
+                if (lo < hi) {
+                    const int nlo = lo + cnt * step;
+                    const int nhi = cnt < P ? lo + (cnt + 1) * step - 1 : hi;
+                    lo = nlo < hi ? nlo : hi;
+                    hi = nhi < hi ? nhi : hi;
+                    if (hi < lo) hi = lo;
+                }
             }
-            cut[tid + 1] = lo;
+            if (mine && sub == 0) cut[jb + 1] = lo;
         }
         __syncthreads();
         int changed = 0;
@@ -576,16 +591,31 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
         e16[tid] = h2d(h);
     }
     __syncthreads();
-    // every weight goes to the nearest STORED entry (ties: lower index)
-    for (int k = tid; k < K; k += kLloydThreads) {
-        const double v = bulk_value(W, mask, row0 + k, mu);
-        int best = 0;
-        double bd = fabs(__dsub_rn(v, e16[0]));
-        for (int j = 1; j < E; ++j) {
-            const double d = fabs(__dsub_rn(v, e16[j]));
-            if (d < bd) { bd = d; best = j; }
+    // every weight goes to the nearest STORED entry (ties: lower index); four weights per thread at a time,
+    // so that four chains of compares are in flight
+    for (int kb = tid; kb < K; kb += 4 * kLloydThreads) {
+        double v[4], bd[4];
+        int best[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int k = kb + e * kLloydThreads;
+            v[e] = k < K ? bulk_value(W, mask, row0 + k, mu) : 0.0;
+            bd[e] = fabs(__dsub_rn(v[e], e16[0]));
+            best[e] = 0;
         }
-        idx[row0 + k] = (uint8_t)best;
+        for (int j = 1; j < E; ++j) {
+            const double ej = e16[j];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const double d = fabs(__dsub_rn(v[e], ej));
+                if (d < bd[e]) { bd[e] = d; best[e] = j; }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int k = kb + e * kLloydThreads;
+            if (k < K) idx[row0 + k] = (uint8_t)best[e];
+        }
     }
     LLOYD_STAMP(5);
 }
