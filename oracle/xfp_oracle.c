@@ -16,8 +16,9 @@
  *   - per-channel Lloyd with CDF-quantile initialisation ("Learned Codebook via Lloyd Iteration")
  *   - per-channel cosine                              (Algorithm 1, cos_sim line)
  *   - LibFit for V2a                                  ("V2a: Shared Codebook Library / Library learning")
- *     LibFit: parity unpinned beyond sanity properties -- the paper gives one sentence and no
- *     reconstruction figure for it.
+ *     LibFit: the paper gives one sentence and no reconstruction figure for it, so the READING is this
+ *     file's own (parity with the paper unpinned); what the functions compute is pinned: the group
+ *     assignment against exhaustive search, the library against the fixed-point properties of k-means.
  *
  * Arithmetic is fp64 except the one V2a step the format fixes to fp32 (see xo_v2a_value16).
  * Build: gcc -O2 -fopenmp -ffp-contract=off -shared -fPIC.

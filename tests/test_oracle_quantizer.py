@@ -3,7 +3,9 @@ and auto-select (Algorithm 1), LibFit.
 
 The Lloyd pins are closed forms (uniform source), textbook Lloyd-Max distortions (Gaussian
 source, tests/golden/lloyd_max_gaussian.txt), exact recovery of discrete sources, and the
-paper's printed XFP3 bulk cosines.  LibFit has only sanity properties (parity unpinned).
+paper's printed XFP3 bulk cosines.  LibFit: the group assignment is checked against exhaustive search and
+the library against k-means fixed-point invariants; the paper prints no V2a figure, so the reading of LibFit
+itself stays unpinned against the paper.
 """
 import os
 
@@ -216,7 +218,7 @@ def test_outlier_extraction_raises_cosine_on_heavy_tailed_layer():
     assert with_out > without + 0.005
 
 
-# ---------------------------------------------------------------- LibFit (sanity only; parity unpinned)
+# ---------------------------------------------------------------- LibFit (no figure in the paper to pin the reading)
 
 def test_libfit_sanity():
     W = synth.gaussian_weights(96, 1024, seed=47)
@@ -239,3 +241,71 @@ def test_libfit_sanity():
     vc = xo.quantize_v2a(Wc, 2, np.zeros(W.shape, np.uint8), 0.0, lib_size=8)
     assert vc.gscale[5, 1] == 0 and np.all(_f16(xo.dequant(vc))[5, 128:256] == 0.03125)
     assert sse2 > 0 and ssea > 0
+
+
+def _decoded(scale16, lib16, mid16):
+    """fp16(fp32(scale*lib + mid)) with numpy's own conversions: the fp16 x fp16 product is exact in fp32."""
+    s = np.asarray(scale16, np.uint16).view(np.float16).astype(np.float32)
+    l = np.asarray(lib16, np.uint16).view(np.float16).astype(np.float32)
+    m = np.asarray(mid16, np.uint16).view(np.float16).astype(np.float32)
+    return (s * l + m).astype(np.float16).astype(np.float64)
+
+
+@pytest.mark.parametrize("bits,L", [(2, 8), (3, 32), (4, 16)])
+def test_libfit_assignment_is_the_brute_force_optimum(bits, L):
+    """Second half of LibFit against exhaustive search: for every group the stored (mid, scale) are the
+    fp16 roundings of the range's middle and half-width, no other library entry gives a smaller squared
+    error under nearest-value decoding, and every index points at a nearest decoded value."""
+    rows, cols = 12, 512
+    W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, seed=81), 0.01, 82)
+    mask, mu, _ = xo.outlier_mask(W)
+    m = xo.quantize_v2a(W, bits, mask, mu, lib_size=L)
+    bulk = np.where(mask != 0, mu, W.astype(np.float64))
+    for i in range(rows):
+        for g in range(cols // 128):
+            v = bulk[i, g * 128:(g + 1) * 128]
+            lo, hi = v.min(), v.max()
+            assert m.gmid[i, g] == np.float16(0.5 * (hi + lo)).view(np.uint16)
+            assert m.gscale[i, g] == np.float16(0.5 * (hi - lo)).view(np.uint16)
+            sse = np.empty(L)
+            for l in range(L):
+                dec = _decoded(m.gscale[i, g], m.codebook[l], m.gmid[i, g])
+                sse[l] = (np.abs(v[:, None] - dec[None, :]).min(axis=1) ** 2).sum()
+            chosen = int(m.gid[i, g])
+            assert sse[chosen] <= sse.min() * (1 + 1e-12)
+            assert chosen == int(np.flatnonzero(sse <= sse.min() * (1 + 1e-12))[0])      # ties: the lower entry
+            dec = _decoded(m.gscale[i, g], m.codebook[chosen], m.gmid[i, g])
+            dist = np.abs(v[:, None] - dec[None, :])
+            q = m.idx[i, g * 128:(g + 1) * 128].astype(int)
+            assert np.array_equal(dist[np.arange(128), q], dist.min(axis=1))
+            assert np.array_equal(q, dist.argmin(axis=1))                                # ties: the lower index
+
+
+def test_libfit_library_invariants():
+    """First half of LibFit (k-means over normalised codebooks) by what any correct run must satisfy: every
+    normalised codebook spans [-1, 1] exactly at its ends, so every centroid does; entries ascend; after
+    enough rounds each centroid is the mean of the codebooks nearest to it (a k-means fixed point); and the
+    library beats its own starting point."""
+    rows, bits, L = 160, 3, 8
+    W = synth.gaussian_weights(rows, 1024, seed=83)
+    W *= np.linspace(0.5, 2.0, rows, dtype=np.float32)[:, None]          # channels of different scale
+    v2 = xo.quantize_v2(W, bits, np.zeros(W.shape, np.uint8), 0.0, 20)
+    E = 1 << bits
+    lib16 = np.empty((L, E), dtype=np.uint16)
+    xo._lib.xo_libfit_library(v2.codebook.reshape(-1), rows, bits, L, 200, lib16.reshape(-1))
+    lib = _f16(lib16)
+    assert np.all(lib[:, 0] == -1.0) and np.all(lib[:, -1] == 1.0)
+    assert np.all(np.diff(lib, axis=1) >= 0)
+    c = _f16(v2.codebook)
+    mid, half = 0.5 * (c.max(1) + c.min(1)), 0.5 * (c.max(1) - c.min(1))
+    u = (c - mid[:, None]) / half[:, None]
+    d = ((u[:, None, :] - lib[None, :, :]) ** 2).sum(-1)
+    near = d.argmin(1)
+    for l in range(L):
+        members = u[near == l]
+        if len(members):
+            assert np.max(np.abs(members.mean(0) - lib[l])) <= 2e-3       # fp16 rounding of entries in [-1, 1]
+    one = np.empty((L, E), dtype=np.uint16)
+    xo._lib.xo_libfit_library(v2.codebook.reshape(-1), rows, bits, L, 0, one.reshape(-1))   # the seeding alone
+    d0 = ((u[:, None, :] - _f16(one)[None, :, :]) ** 2).sum(-1).min(1).sum()
+    assert d.min(1).sum() < d0
