@@ -111,6 +111,24 @@ int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* str
 int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
                      void* const* y, int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
 
+/* xfp_gemv_grouped with the element-wise step that follows it in a routed expert's feed-forward block fused
+ * into the store, so that one token-layer is two launches ("MoE-native" dispatch; the paper blames the
+ * launch count of the unfused expert path for its power plateau).  V2a blobs the fast kernel supports
+ * (bits 2..5), batch 1; anything else returns XFP_ERR_UNSUPPORTED.
+ *   XFP_EPI_NONE     y[j][rows] as xfp_gemv_grouped.
+ *   XFP_EPI_SWIGLU   the blob is a gate_up projection whose channels were ordered, before quantisation, in
+ *                    blocks of 64: 32 gate channels followed by the 32 matching up channels.  y[j] receives
+ *                    rows/2 values h = SiLU(gate) * up, SiLU(g) = g / (1 + exp(-g)), evaluated in fp32 on
+ *                    the fp32 sums.  rows must be a multiple of 64.
+ *   XFP_EPI_COMBINE  y[0][rows] = sum_j weights[j] * (W_j x[j]) added in blob order in fp32 (the routing
+ *                    weights of the token, `weights` [n] floats on the device); y[1..] are not used. */
+#define XFP_EPI_NONE 0
+#define XFP_EPI_SWIGLU 1
+#define XFP_EPI_COMBINE 2
+int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
+                              void* const* y, int32_t y_is_fp16, int32_t epilogue, const float* weights,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 /* Convenience for callers whose activations live in host memory: brings x_host to x_dev, runs the GEMV for
  * desc->mode and delivers y in y_host, all on `stream` (the host sees y once the stream reached this point).
  * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller.  Pinned,

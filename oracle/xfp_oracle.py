@@ -186,6 +186,16 @@ def set_threads(n: int) -> None:
     _lib.xo_set_threads(int(n))
 
 
+# ---------------------------------------------------------------- a routed expert's feed-forward block
+
+def silu_mul(gate: np.ndarray, up: np.ndarray) -> np.ndarray:
+    """h = SiLU(gate) * up with SiLU(g) = g / (1 + exp(-g)), in fp64: the element-wise step between the
+    gate_up and the down projection of a gated feed-forward block (the routed experts of the paper's MoE
+    models; the fused decode path applies it in the store of the gate_up GEMV)."""
+    g = np.asarray(gate, dtype=np.float64)
+    return g / (1.0 + np.exp(-g)) * np.asarray(up, dtype=np.float64)
+
+
 # ---------------------------------------------------------------- encoder
 
 def stats(W: np.ndarray):

@@ -16,7 +16,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 EXPORTS = ("xfp_packed_size", "xfp_pack", "xfp_gemv_v2", "xfp_gemv_v2a", "xfp_gemv_grouped", "xfp_gemv_host",
-           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc")
+           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_grouped_epilogue")
+
+XFP_EPI_NONE, XFP_EPI_SWIGLU, XFP_EPI_COMBINE = 0, 1, 2
 
 
 class XfpError(RuntimeError):
@@ -52,6 +54,7 @@ def load_library() -> C.CDLL:
     lib.xfp_gemv_v2.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_v2a.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_grouped.argtypes = [dp, i32, vp, vp, vp, i32, vp, sz, vp]
+    lib.xfp_gemv_grouped_epilogue.argtypes = [dp, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
     lib.xfp_gemv_host.argtypes = [dp, vp, vp, vp, i32, vp, vp, i32, vp, sz, vp]
     lib.xfp_dequant.argtypes = [dp, vp, vp, vp]
     lib.xfp_gemv_v2_noalloc.argtypes = [dp, vp, vp, i32, vp, i32, vp]
@@ -118,6 +121,17 @@ def xfp_gemv_grouped(desc, n: int, packed_ptrs: torch.Tensor, x_ptrs: torch.Tens
                                            int(bool(y_is_fp16)), _ptr(workspace),
                                            workspace.numel() * workspace.element_size(), _stream(stream)),
            "xfp_gemv_grouped")
+
+
+def xfp_gemv_grouped_epilogue(desc, n: int, packed_ptrs: torch.Tensor, x_ptrs: torch.Tensor, y_ptrs: torch.Tensor,
+                              y_is_fp16, epilogue: int, weights: Optional[torch.Tensor], workspace: torch.Tensor,
+                              stream=None) -> None:
+    """xfp_gemv_grouped with a fused store: XFP_EPI_SWIGLU (y[j] gets rows/2 values SiLU(gate)*up) or
+    XFP_EPI_COMBINE (y[0] = sum_j weights[j] * W_j x[j]; weights: float32 device tensor of n values)."""
+    _check(load_library().xfp_gemv_grouped_epilogue(C.byref(desc), int(n), _ptr(packed_ptrs), _ptr(x_ptrs),
+                                                    _ptr(y_ptrs), int(bool(y_is_fp16)), int(epilogue), _ptr(weights),
+                                                    _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                    _stream(stream)), "xfp_gemv_grouped_epilogue")
 
 
 def xfp_gemv_host(desc, packed, x_host: torch.Tensor, x_dev, batch, y_host: torch.Tensor, y_dev, y_is_fp16,

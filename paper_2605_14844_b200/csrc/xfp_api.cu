@@ -46,6 +46,12 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     GemvCall cc = c;
     cc.workspace_bytes = need;
     cudaError_t e;
+    if (c.epilogue != 0) {
+        // fused epilogues exist in the V2a kernel only (batch 1)
+        if (!v2a_supported(l, c.batch) || c.batch != 1) return XFP_ERR_UNSUPPORTED;
+        e = launch_gemv_v2a(l, cc, (cudaStream_t)stream);
+        return e == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+    }
     if (pair_supported(l, c.batch, c.n) && !c.packed_list)
         e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && batch_supported(l, c.batch))
@@ -150,6 +156,26 @@ int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed,
     const size_t need = workspace_bytes_for(l);
     if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
     GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16, workspace, need};
+    return gemv_common(desc, desc->mode, c, stream);
+}
+
+int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
+                              void* const* y, int32_t y_is_fp16, int32_t epilogue, const float* weights,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+    if (!desc) return XFP_ERR_NULL;
+    if (n < 1 || n > 65535) return XFP_ERR_SHAPE;
+    if (!packed || !x || !y) return XFP_ERR_NULL;
+    if (epilogue != XFP_EPI_NONE && epilogue != XFP_EPI_SWIGLU && epilogue != XFP_EPI_COMBINE) return XFP_ERR_SHAPE;
+    if (epilogue == XFP_EPI_COMBINE && !weights) return XFP_ERR_NULL;
+    int st = check_desc(desc);
+    if (st) return st;
+    if (epilogue == XFP_EPI_SWIGLU && desc->rows % 64 != 0) return XFP_ERR_SHAPE;
+    const Layout l = layout_of(desc);
+    const size_t need = workspace_bytes_for(l);
+    if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
+    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16, workspace, need};
+    c.epilogue = epilogue;
+    c.epi_weights = weights;
     return gemv_common(desc, desc->mode, c, stream);
 }
 

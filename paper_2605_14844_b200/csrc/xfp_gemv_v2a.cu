@@ -56,6 +56,9 @@ struct V2aArgs {
     int blocks, n_full, kst, sc_per_split;
     int n_a, kst_b, sc_per_split_b;   // of the cut blocks the first n_a use kst slices, the rest kst_b (finer) slices
     int items_x, n;   // work items per blob (whole blocks + K slices), blobs
+    int epi;                 // 0 plain store; 1 SiLU(gate) * up inside every 64-channel block; 2 weighted sum over the blobs
+    const float* epi_w;      // epi 2: [n] weights
+    int comb_G, comb_ng;     // epi 2: runs per block of channels, blobs per run
 };
 
 __device__ __forceinline__ void mma16816a(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -122,9 +125,26 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
     const uint16_t* x_staged = nullptr;
 
     // ---- work items: (blob, whole block or K slice of a block), dealt round-robin to the CTAs of the launch
+    // The weighted sum over the blobs (epi 2) deals RUNS instead: a CTA takes comb_ng consecutive blobs of
+    // one block of channels and adds their weighted results in registers; only the comb_G runs of a block
+    // meet in the scratch (none when one run covers all blobs).
+    const int per = a.epi == 2 ? a.comb_ng : 1;
+    const int nrun = a.epi == 2 ? a.blocks * a.comb_G : a.items_x * a.n;
+    float csum = 0.f;   // epi 2: this thread's channel, weighted sum over the blobs of the run
 #pragma unroll 1
-    for (int item = blockIdx.x; item < a.items_x * a.n; item += gridDim.x) {
-    const int prob = item / a.items_x, bx = item - prob * a.items_x;
+    for (int run = blockIdx.x; run < nrun; run += gridDim.x) {
+#pragma unroll 1
+    for (int jj = 0; jj < per; ++jj) {
+    int prob, bx;
+    if (a.epi == 2) {
+        bx = run / a.comb_G;
+        prob = (run - bx * a.comb_G) * a.comb_ng + jj;
+        if (prob >= a.n) break;
+        if (jj == 0) csum = 0.f;
+    } else {
+        prob = run / a.items_x;
+        bx = run - prob * a.items_x;
+    }
     int blk, ks, KS, spp;
     if (bx < a.n_full) {
         blk = bx; ks = 0; KS = 1; spp = a.SC;
@@ -135,6 +155,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
         const int t = bx - a.n_full - a.n_a * a.kst;
         blk = a.n_full + a.n_a + t / a.kst_b; ks = t % a.kst_b; KS = a.kst_b; spp = a.sc_per_split_b;
     }
+    const float epi_wj = a.epi == 2 ? __ldg(a.epi_w + prob) : 0.f;   // fetched now, used in the store
     const void* packed = a.packed_list ? a.packed_list[prob] : a.packed;
     const uint16_t* x = a.x_list ? a.x_list[prob] : a.x;
     void* y = a.y_list ? a.y_list[prob] : a.y;
@@ -436,14 +457,65 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
             if (t == 0) *ticket = 0;
         }
     }
-    if (writer && active && !dup && bb < a.nb && row < a.rows) {
-        if (a.y_is_fp16)
-            ((uint16_t*)y)[(size_t)bb * a.rows + row] = f2h(total);
-        else
-            ((float*)y)[(size_t)bb * a.rows + row] = total;
+    if (a.epi == 0) {
+        if (writer && active && !dup && bb < a.nb && row < a.rows) {
+            if (a.y_is_fp16)
+                ((uint16_t*)y)[(size_t)bb * a.rows + row] = f2h(total);
+            else
+                ((float*)y)[(size_t)bb * a.rows + row] = total;
+        }
+    } else if (a.epi == 1) {
+        // gated activation of a routed expert: channels 0..31 of the block are gates, 32..63 the matching
+        // up channels; the block stores 32 values h = SiLU(gate) * up  (batch 1, rows a multiple of 64)
+        if (writer) {
+            __syncthreads();   // every thread has read its column of red
+            if (t < kARows) red[t] = total;
+            __syncthreads();
+            if (t < 32) {
+                const float g = red[t], u = red[t + 32];
+                const float h = g / (1.f + expf(-g)) * u;
+                const size_t o = (size_t)blk * 32 + t;
+                if (a.y_is_fp16) ((uint16_t*)y)[o] = f2h(h);
+                else ((float*)y)[o] = h;
+            }
+        }
+    } else {
+        // weighted sum over the blobs of the launch (the routed experts' down projections)
+        if (t < kARows) csum = fmaf(epi_wj, total, csum);
+        const bool run_done = jj == per - 1 || prob == a.n - 1;
+        if (run_done && a.comb_G == 1) {
+            if (t < kARows && !dup && row < a.rows) {
+                void* y0 = a.y_list ? a.y_list[0] : a.y;
+                if (a.y_is_fp16) ((uint16_t*)y0)[row] = f2h(csum);
+                else ((float*)y0)[row] = csum;
+            }
+        } else if (run_done) {
+            // the runs of this block leave their sums in the scratch, the last one to arrive adds them in run order
+            float* comb = a.partial;            // [run of the block][rows_ws]; the K-split scratch is idle in these launches
+            int* ticket = a.tickets + blk;      // one counter per block of channels
+            const int g = run - bx * a.comb_G;
+            if (t < kARows) comb[(size_t)g * a.rows_ws + row] = csum;
+            __threadfence();
+            __syncthreads();
+            if (t == 0) s_last = (atomicAdd(ticket, 1) == a.comb_G - 1);
+            __syncthreads();
+            if (s_last) {
+                __threadfence();
+                if (t < kARows && !dup && row < a.rows) {
+                    float sum = 0.f;
+                    for (int g2 = 0; g2 < a.comb_G; ++g2) sum += __ldcg(comb + (size_t)g2 * a.rows_ws + row);
+                    void* y0 = a.y_list ? a.y_list[0] : a.y;
+                    if (a.y_is_fp16) ((uint16_t*)y0)[row] = f2h(sum);
+                    else ((float*)y0)[row] = sum;
+                }
+                if (t == 0) *ticket = 0;
+            }
+        }
     }
     if (!PAIR) break;   // the per-bank library is launched with one CTA per item
     __syncthreads();   // red, x and the ticket flag are reused by the CTA's next item
+    }
+    if (!PAIR) break;
     }
 }
 
@@ -539,7 +611,7 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     int rem = 0;
     a.kst = 1; a.sc_per_split = l.SC; a.n_a = 0; a.kst_b = 1; a.sc_per_split_b = l.SC;
     const int tail = (int)(total % cfg.slots);
-    if (tail > 0 && c.n == 1) {
+    if (tail > 0 && c.n == 1 && c.epilogue != 2) {   // the weighted sum uses the K-split scratch for itself
         rem = tail;
         auto ka = slices(cfg.slots / rem);
         if (ka.first > 1) {
@@ -566,7 +638,16 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     a.partial = (float*)((char*)c.workspace + align256((size_t)a.blocks * 4 * c.n));
     a.items_x = a.n_full + a.n_a * a.kst + n_b * a.kst_b;
     a.n = c.n;
-    const long long items = (long long)a.items_x * c.n;
+    a.epi = c.epilogue; a.epi_w = c.epi_weights;
+    long long items = (long long)a.items_x * c.n;
+    a.comb_G = 1; a.comb_ng = 1;
+    if (c.epilogue == 2) {
+        // pair tables: as few runs per block as still fill the resident CTAs; per-bank library: one blob per CTA
+        int G = cfg.pair ? std::max(1, std::min(c.n, cfg.slots / std::max(1, a.blocks))) : c.n;
+        a.comb_ng = (c.n + G - 1) / G;
+        a.comb_G = (c.n + a.comb_ng - 1) / a.comb_ng;
+        items = (long long)a.blocks * a.comb_G;
+    }
     // pair tables are expensive to build: resident CTAs walk the items; the per-bank library launches one CTA per item
     dim3 grid((unsigned)(cfg.pair ? (items < cfg.slots ? items : cfg.slots) : items), 1, 1);
     switch (l.bits * 10 + c.batch) {

@@ -35,6 +35,8 @@ struct GemvCall {
     int y_is_fp16;
     void* workspace;
     size_t workspace_bytes;  // per problem
+    int epilogue = 0;                      // XFP_EPI_* (grouped V2a launches only)
+    const float* epi_weights = nullptr;    // XFP_EPI_COMBINE: [n] routing weights on the device
 };
 
 // Split-K factor the generic kernel uses for this shape and batch tile (host-side policy).

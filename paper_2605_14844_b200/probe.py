@@ -9,11 +9,14 @@
         graph of P calls, median of 20 replays) and print microseconds per call and effective GB/s over
         the algorithmic bytes.
 
-    python -m paper_2605_14844_b200.probe moe [EXPERTS] [TOKENS] [BITS]
+    python -m paper_2605_14844_b200.probe moe [EXPERTS] [TOKENS] [BITS] [FUSED]
         routed-MoE decode layer: EXPERTS (default 128) V2a experts with a gate_up projection 3072 x 4096
         and a down projection 4096 x 1536 (one library per projection, 0.1 % outliers), top-8 routing per
-        token; every token-layer is two xfp_gemv_grouped launches (8 gate_up, 8 down).  Prints
-        microseconds per token-layer and effective GB/s.
+        token; every token-layer is two xfp_gemv_grouped launches (8 gate_up, 8 down).  FUSED = 1 uses
+        xfp_gemv_grouped_epilogue instead: SiLU(gate)*up in the store of the first launch, the routing-weighted
+        sum over the experts in the store of the second (the complete expert block); FUSED = 2 computes the
+        same block with the plain grouped launches and the two element-wise steps as separate kernels.
+        Prints microseconds per token-layer and effective GB/s.
 
     python -m paper_2605_14844_b200.probe sweep [quick]
         batch and shape sweep: 8192 x 8192 and 28672 x 8192, 4-bit codebooks, V2 and V2a, x batch 1, 2, 4, 8, 16,
@@ -105,8 +108,8 @@ def time_shape(mode, rows, cols, bits, rate, batch=1, placement="uniform", reps=
     return out
 
 
-def moe(experts=128, tokens=64, bits=3, distinct=8, reps=10):
-    from . import XfpDesc, xfp_gemv_grouped, xfp_packed_size
+def moe(experts=128, tokens=64, bits=3, fused=0, distinct=8, reps=10):
+    from . import XFP_EPI_COMBINE, XFP_EPI_SWIGLU, XfpDesc, xfp_gemv_grouped, xfp_gemv_grouped_epilogue, xfp_packed_size
     shapes = {"gate_up": (3072, 4096), "down": (4096, 1536)}
     packed, descs, nbytes = {}, {}, {}
     for name, (rows, cols) in shapes.items():
@@ -124,6 +127,8 @@ def moe(experts=128, tokens=64, bits=3, distinct=8, reps=10):
     h = [torch.zeros((8, 1536), dtype=torch.float16, device=dev) for _ in range(tokens)]     # down inputs
     y_up = [torch.empty((8, 3072), dtype=torch.float16, device=dev) for _ in range(tokens)]
     y_dn = [torch.empty((8, 4096), dtype=torch.float16, device=dev) for _ in range(tokens)]
+    y_out = [torch.empty(4096, dtype=torch.float16, device=dev) for _ in range(tokens)]
+    gate_w16 = torch.full((8,), 0.125, dtype=torch.float16, device=dev)
     for t in h:
         t.copy_(_x(8, 1536))
     ptrs = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device=dev)
@@ -132,12 +137,32 @@ def moe(experts=128, tokens=64, bits=3, distinct=8, reps=10):
         ex = route[t]
         args.append((ptrs([packed["gate_up"][e].packed for e in ex]), ptrs([x_up[t]] * 8), ptrs([y_up[t][j] for j in range(8)]),
                      ptrs([packed["down"][e].packed for e in ex]), ptrs([h[t][j] for j in range(8)]),
-                     ptrs([y_dn[t][j] for j in range(8)])))
+                     ptrs([y_dn[t][j] for j in range(8)]), y_up[t], h[t], y_dn[t], y_out[t]))
     ws = {n: torch.zeros(8 * xfp_packed_size(descs[n])[1], dtype=torch.uint8, device=dev) for n in shapes}
 
+    gate_w = torch.full((8,), 0.125, dtype=torch.float32, device=dev)   # routing weights of the token
+
     def layer(a):
-        xfp_gemv_grouped(descs["gate_up"], 8, a[0], a[1], a[2], True, ws["gate_up"])
-        xfp_gemv_grouped(descs["down"], 8, a[3], a[4], a[5], True, ws["down"])
+        if fused in (3, 4):   # measurement aids: only the first (3) or only the second (4) fused store
+            if fused == 3:
+                xfp_gemv_grouped_epilogue(descs["gate_up"], 8, a[0], a[1], a[4], True, XFP_EPI_SWIGLU, None, ws["gate_up"])
+                xfp_gemv_grouped(descs["down"], 8, a[3], a[4], a[5], True, ws["down"])
+            else:
+                xfp_gemv_grouped(descs["gate_up"], 8, a[0], a[1], a[2], True, ws["gate_up"])
+                xfp_gemv_grouped_epilogue(descs["down"], 8, a[3], a[4], a[5], True, XFP_EPI_COMBINE, gate_w, ws["down"])
+        elif fused == 1:
+            # the whole expert block in two launches: gate_up with SiLU(gate)*up in its store (writes the
+            # down projections' inputs), down with the routing-weighted sum over the experts in its store
+            xfp_gemv_grouped_epilogue(descs["gate_up"], 8, a[0], a[1], a[4], True, XFP_EPI_SWIGLU, None, ws["gate_up"])
+            xfp_gemv_grouped_epilogue(descs["down"], 8, a[3], a[4], a[5], True, XFP_EPI_COMBINE, gate_w, ws["down"])
+        else:
+            xfp_gemv_grouped(descs["gate_up"], 8, a[0], a[1], a[2], True, ws["gate_up"])
+            if fused == 2:   # the same block with the two element-wise steps as separate (torch) kernels
+                yu, hh = a[6], a[7]
+                torch.mul(torch.nn.functional.silu(yu[:, :1536]), yu[:, 1536:], out=hh)
+            xfp_gemv_grouped(descs["down"], 8, a[3], a[4], a[5], True, ws["down"])
+            if fused == 2:
+                torch.sum(a[8] * gate_w16[:, None], dim=0, out=a[9])
 
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
@@ -160,7 +185,8 @@ def moe(experts=128, tokens=64, bits=3, distinct=8, reps=10):
             ts.append(e0.elapsed_time(e1) * 1e3 / tokens)
     per_layer = 8 * (nbytes["gate_up"] + nbytes["down"])
     t = float(np.median(ts))
-    print(json.dumps(dict(workload="moe_v2a", experts=experts, tokens=tokens, bits=bits, MB_per_token_layer=round(per_layer / 1e6, 2),
+    print(json.dumps(dict(workload=("moe_v2a", "moe_v2a_fused_ffn", "moe_v2a_ffn_with_separate_elementwise_kernels",
+                                    "moe_v2a_fused_activation_only", "moe_v2a_fused_sum_only")[fused], experts=experts, tokens=tokens, bits=bits, MB_per_token_layer=round(per_layer / 1e6, 2),
                           us_per_token_layer=round(t, 2), GBs=round(per_layer / t / 1e3, 1))), flush=True)
 
 
@@ -292,7 +318,7 @@ def main(argv):
         quant(*(int(v) for v in argv[2:7]))
         return 0
     if len(argv) > 1 and argv[1] == "moe":
-        moe(*(int(v) for v in argv[2:5]))
+        moe(*(int(v) for v in argv[2:6]))
         return 0
     if len(argv) > 1 and argv[1] == "sweep":
         sweep(len(argv) > 2 and argv[2] == "quick")

@@ -142,6 +142,14 @@ def test_null_alignment_and_size_checks_need_no_gpu(lib):
     assert lib.xfp_dequant(C.byref(d), a, odd, n) == 2
     assert lib.xfp_gemv_grouped(C.byref(d), 0, a, a, a, 0, a, 1 << 30, n) == 3
     assert lib.xfp_gemv_grouped(C.byref(d), 4, a, a, a, 0, a, 64, n) == 5
+    da64 = _desc(mode=1, lib_size=32, rows=128)
+    assert lib.xfp_gemv_grouped_epilogue(C.byref(da64), 2, a, a, a, 0, 5, n, a, 1 << 30, n) == 3     # unknown epilogue
+    assert lib.xfp_gemv_grouped_epilogue(C.byref(da64), 2, a, a, a, 0, 2, n, a, 1 << 30, n) == 1     # weighted sum without weights
+    da96 = _desc(mode=1, lib_size=32, rows=96)
+    assert lib.xfp_gemv_grouped_epilogue(C.byref(da96), 2, a, a, a, 0, 1, n, a, 1 << 30, n) == 3     # rows = 64 * k for SiLU*up
+    assert lib.xfp_gemv_grouped_epilogue(C.byref(da64), 2, a, a, a, 0, 1, n, a, 64, n) == 5
+    d128 = _desc(rows=128)
+    assert lib.xfp_gemv_grouped_epilogue(C.byref(d128), 2, a, a, a, 0, 1, n, a, 1 << 30, n) == 4     # V2 blobs: not built
     assert xfp.xfp_status_str(0) == "ok" and "aligned" in xfp.xfp_status_str(2)
 
 

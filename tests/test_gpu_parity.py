@@ -332,3 +332,102 @@ def test_sweep_shape_28672x8192_sampled_rows(mode, batch, rate, placement):
     tickets = pm.workspace[: ((rows + 31) // 32) * 4].view(torch.int32)
     assert int(tickets.abs().sum().item()) == 0
 
+
+
+def _group_desc(pms):
+    d0 = pms[0].desc
+    return xfp.XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                       max(p.desc.nnz for p in pms))
+
+
+@pytest.mark.parametrize("bits,n,rows_gu,hidden", [(3, 8, 256, 512), (2, 3, 2304, 384), (4, 4, 256, 256), (5, 2, 768, 128),
+                                                 (3, 8, 3072, 4096)])
+@pytest.mark.parametrize("y_fp16", [True, False])
+def test_fused_expert_block(bits, n, rows_gu, hidden, y_fp16):
+    """A routed expert block in two launches: gate_up with SiLU(gate)*up in its store, down with the
+    routing-weighted sum over the experts in its store.
+
+    Stage 1 is compared with the oracle's fp64 h = SiLU(g)*u under the bound propagated through the
+    activation: |SiLU'| <= 1.1, so |dh| <= 1.1 |u| e_g + |SiLU(g)| e_u + one output rounding, with e = 1e-3 sum|W x|
+    of the gate and up channel.  Stage 2 takes the GPU's own h as its input on both sides and must obey
+    1e-3 * sum_j |w_j| sum_k |W_jik h_jk|."""
+    inter = rows_gu // 2
+    gus = [synth.random_quantized(1, rows_gu, hidden, bits, 0.002, seed=2100 + j) for j in range(n)]
+    dns = [synth.random_quantized(1, hidden, inter, bits, 0.002, seed=2200 + j) for j in range(n)]
+    for q in gus[1:]:
+        q.codebook = gus[0].codebook
+    for q in dns[1:]:
+        q.codebook = dns[0].codebook
+    pg = [xfp.pack_tensors(q, col_bits=16) for q in gus]
+    pd = [xfp.pack_tensors(q, col_bits=16) for q in dns]
+    x16 = synth.activations(1, hidden, seed=2300)
+    xd = _x_dev(x16)
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    dt = torch.float16 if y_fp16 else torch.float32
+    h = torch.full((n, inter), float("nan"), dtype=dt, device="cuda")
+    dg, dd = _group_desc(pg), _group_desc(pd)
+    wsg = torch.zeros(n * xfp.xfp_packed_size(dg)[1], dtype=torch.uint8, device="cuda")
+    wsd = torch.zeros(n * xfp.xfp_packed_size(dd)[1], dtype=torch.uint8, device="cuda")
+    for _ in range(2):      # twice: the counters must come back to zero
+        xfp.xfp_gemv_grouped_epilogue(dg, n, ptr([p.packed for p in pg]), ptr([xd] * n), ptr([h[j] for j in range(n)]),
+                                      y_fp16, xfp.XFP_EPI_SWIGLU, None, wsg)
+    torch.cuda.synchronize()
+    hg = h.float().cpu().numpy().astype(np.float64)
+    blocks = rows_gu // 64
+    gate_rows = (np.arange(blocks)[:, None] * 64 + np.arange(32)[None, :]).reshape(-1)
+    for j in range(n):
+        ref, absum = xo.gemv(to_oracle(gus[j]), x16)
+        g, u = ref[0][gate_rows], ref[0][gate_rows + 32]
+        eg, eu = TOL * absum[0][gate_rows], TOL * absum[0][gate_rows + 32]
+        want = xo.silu_mul(g, u)
+        sil = g / (1.0 + np.exp(-g))
+        bound = 1.1 * np.abs(u) * eg + np.abs(sil) * eu + 1.1 * eg * eu + 2.0 ** -10 * np.abs(want) + 1e-30
+        assert np.all(np.abs(hg[j] - want) <= bound), float((np.abs(hg[j] - want) / bound).max())
+
+    # stage 2 on the GPU's own h (as fp16, the down projection's input type)
+    h16 = h.to(torch.float16).contiguous()
+    wts = np.random.default_rng(2400).random(n).astype(np.float32)
+    wts /= wts.sum()
+    y = torch.full((n, hidden), float("nan"), dtype=dt, device="cuda")
+    for _ in range(2):
+        xfp.xfp_gemv_grouped_epilogue(dd, n, ptr([p.packed for p in pd]), ptr([h16[j] for j in range(n)]),
+                                      ptr([y[j] for j in range(n)]), y_fp16, xfp.XFP_EPI_COMBINE,
+                                      torch.from_numpy(wts).cuda(), wsd)
+    torch.cuda.synchronize()
+    h16_host = h16.view(torch.int16).cpu().numpy().view(np.uint16)
+    want = np.zeros(hidden)
+    bound = np.zeros(hidden)
+    for j in range(n):
+        ref, absum = xo.gemv(to_oracle(dns[j]), h16_host[j:j + 1])
+        want += float(wts[j]) * ref[0]
+        bound += abs(float(wts[j])) * absum[0]
+    got = y[0].float().cpu().numpy().astype(np.float64)
+    tol = TOL * bound + (2.0 ** -10 * np.abs(want) if y_fp16 else 0.0) + 1e-30
+    assert np.all(np.abs(got - want) <= tol), float((np.abs(got - want) / tol).max())
+    assert torch.isnan(y[1:].float()).all()          # only y[0] is written
+    # the unfused path gives the same sums
+    yu = torch.zeros((n, hidden), dtype=torch.float32, device="cuda")
+    xfp.xfp_gemv_grouped(dd, n, ptr([p.packed for p in pd]), ptr([h16[j] for j in range(n)]),
+                         ptr([yu[j] for j in range(n)]), False, wsd)
+    torch.cuda.synchronize()
+    plain = (yu.cpu().numpy().astype(np.float64) * wts[:, None].astype(np.float64)).sum(0)
+    assert np.all(np.abs(got - plain) <= 0.05 * TOL * bound + (2.0 ** -10 * np.abs(want) if y_fp16 else 0.0) + 1e-30)
+
+
+def test_fused_epilogues_are_refused_where_not_built():
+    q = synth.random_quantized(0, 128, 256, 4, 0.0, seed=2500)      # V2 blobs have no fused store
+    pm = xfp.pack_tensors(q)
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    x = _x_dev(synth.activations(1, 256, seed=1))
+    y = torch.zeros(128, dtype=torch.float32, device="cuda")
+    with pytest.raises(xfp.XfpError):
+        xfp.xfp_gemv_grouped_epilogue(pm.desc, 1, ptr([pm.packed]), ptr([x]), ptr([y]), False, xfp.XFP_EPI_SWIGLU, None,
+                                      pm.workspace)
+    qa = synth.random_quantized(1, 96, 256, 3, 0.0, seed=2501)      # rows not a multiple of 64
+    pa = xfp.pack_tensors(qa)
+    with pytest.raises(xfp.XfpError):
+        xfp.xfp_gemv_grouped_epilogue(pa.desc, 1, ptr([pa.packed]), ptr([x]), ptr([y]), False, xfp.XFP_EPI_SWIGLU, None,
+                                      pa.workspace)
+    with pytest.raises(xfp.XfpError):                                # the weighted sum needs its weights
+        xfp.xfp_gemv_grouped_epilogue(pa.desc, 1, ptr([pa.packed]), ptr([x]), ptr([y]), False, xfp.XFP_EPI_COMBINE, None,
+                                      pa.workspace)
