@@ -98,6 +98,19 @@ int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int
 int xfp_gemv_v2a(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
                  int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The fused GEMV of desc->mode with bf16 activations and/or outputs (bf16 is the paper's native activation
+ * type; its kernel "outputs bf16 natively").
+ *   x  [batch][cols] of x_type: XFP_T_F16, or XFP_T_BF16 -- converted to fp16 while the kernel stages it
+ *      (round to nearest even, clamped to +-65504; a bf16 value with 2^-14 <= |x| <= 65504 converts
+ *      exactly, smaller ones land on the fp16 subnormal grid, absolute error <= 2^-25)
+ *   y  [batch][rows] of y_type: XFP_T_F32, XFP_T_F16 or XFP_T_BF16 (one rounding of the fp32 sum)
+ * Everything else as xfp_gemv_v2 / xfp_gemv_v2a. */
+#define XFP_T_F32 0
+#define XFP_T_F16 1
+#define XFP_T_BF16 2
+int xfp_gemv_typed(const xfp_desc* desc, const void* packed, const void* x, int32_t x_type, int32_t batch, void* y,
+                   int32_t y_type, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Materialise W^ = fp16(D16 + S) as fp16 [rows][cols] ("Reconstruct" in Algorithm 1; Eq. 1).
  * D16 is the fp16 value the index decodes to: the codebook entry (V2), or
  * fp16(fp32(scale * lib + mid)) (V2a, one fp32 rounding then one fp16 rounding).  The sum with an

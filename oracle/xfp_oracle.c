@@ -189,12 +189,11 @@ void xo_dequant(const xo_matrix* m, uint16_t* W) {
 }
 
 /* y[b][i] = sum_k (D_ik + S_ik) x[b][k] in fp64, k ascending; absum[b][i] = sum_k |(D_ik+S_ik) x[b][k]|.
- * Rows [row0, row1) only (lets a caller sample rows of a large matrix). */
-void xo_gemv_rows(const xo_matrix* m, const uint16_t* x, int32_t batch, int64_t row0, int64_t row1,
-                  double* y, double* absum) {
+ * Rows [row0, row1) only (lets a caller sample rows of a large matrix).  x as doubles: any activation type
+ * (fp16, or the paper's native bf16) is exact in fp64. */
+void xo_gemv_rows_x64(const xo_matrix* m, const double* xd, int32_t batch, int64_t row0, int64_t row1,
+                      double* y, double* absum) {
     int64_t K = m->cols;
-    double* xd = (double*)malloc(sizeof(double) * (size_t)batch * (size_t)K);
-    for (int64_t t = 0; t < (int64_t)batch * K; ++t) xd[t] = xo_half_to_double(x[t]);
 #pragma omp parallel
     {
         double* w = (double*)malloc(sizeof(double) * (size_t)K);
@@ -217,6 +216,15 @@ void xo_gemv_rows(const xo_matrix* m, const uint16_t* x, int32_t batch, int64_t 
         }
         free(w);
     }
+}
+
+/* the same with x as fp16 bit patterns */
+void xo_gemv_rows(const xo_matrix* m, const uint16_t* x, int32_t batch, int64_t row0, int64_t row1,
+                  double* y, double* absum) {
+    int64_t K = m->cols;
+    double* xd = (double*)malloc(sizeof(double) * (size_t)batch * (size_t)K);
+    for (int64_t t = 0; t < (int64_t)batch * K; ++t) xd[t] = xo_half_to_double(x[t]);
+    xo_gemv_rows_x64(m, xd, batch, row0, row1, y, absum);
     free(xd);
 }
 

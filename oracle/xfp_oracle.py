@@ -47,6 +47,7 @@ _lib.xo_table1_pack_row.argtypes = [C.c_int, _u8p, C.c_int64, C.c_void_p]
 _lib.xo_table1_unpack_row.argtypes = [C.c_int, C.c_void_p, C.c_int64, _u8p]
 _lib.xo_dequant.argtypes = [C.POINTER(_CMatrix), _u16p]
 _lib.xo_gemv_rows.argtypes = [C.POINTER(_CMatrix), _u16p, C.c_int32, C.c_int64, C.c_int64, _f64p, _f64p]
+_lib.xo_gemv_rows_x64.argtypes = [C.POINTER(_CMatrix), _f64p, C.c_int32, C.c_int64, C.c_int64, _f64p, _f64p]
 _lib.xo_threads.restype = C.c_int
 _lib.xo_set_threads.argtypes = [C.c_int]
 _lib.xo_stats.argtypes = [_f32p, C.c_int64, C.POINTER(C.c_double), C.POINTER(C.c_double)]
@@ -175,6 +176,18 @@ def gemv(m: QuantizedMatrix, x16: np.ndarray, row0: int = 0, row1: Optional[int]
     a = np.zeros((batch, m.rows), dtype=np.float64)
     cm = m._c()
     _lib.xo_gemv_rows(C.byref(cm), x16.reshape(-1), batch, row0, row1, y.reshape(-1), a.reshape(-1))
+    return y, a
+
+
+def gemv_x64(m: QuantizedMatrix, x: np.ndarray, row0: int = 0, row1: Optional[int] = None):
+    """gemv for activations given as real numbers [batch, cols] (bf16 values are exact in fp64)."""
+    x = np.ascontiguousarray(x, dtype=np.float64).reshape(-1, m.cols)
+    batch = x.shape[0]
+    row1 = m.rows if row1 is None else row1
+    y = np.zeros((batch, m.rows), dtype=np.float64)
+    a = np.zeros((batch, m.rows), dtype=np.float64)
+    cm = m._c()
+    _lib.xo_gemv_rows_x64(C.byref(cm), x.reshape(-1), batch, row0, row1, y.reshape(-1), a.reshape(-1))
     return y, a
 
 

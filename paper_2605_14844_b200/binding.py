@@ -16,9 +16,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 EXPORTS = ("xfp_packed_size", "xfp_pack", "xfp_gemv_v2", "xfp_gemv_v2a", "xfp_gemv_grouped", "xfp_gemv_host",
-           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_grouped_epilogue")
+           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_grouped_epilogue", "xfp_gemv_typed")
 
 XFP_EPI_NONE, XFP_EPI_SWIGLU, XFP_EPI_COMBINE = 0, 1, 2
+XFP_T_F32, XFP_T_F16, XFP_T_BF16 = 0, 1, 2
 
 
 class XfpError(RuntimeError):
@@ -54,6 +55,7 @@ def load_library() -> C.CDLL:
     lib.xfp_gemv_v2.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_v2a.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_grouped.argtypes = [dp, i32, vp, vp, vp, i32, vp, sz, vp]
+    lib.xfp_gemv_typed.argtypes = [dp, vp, vp, i32, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_grouped_epilogue.argtypes = [dp, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
     lib.xfp_gemv_host.argtypes = [dp, vp, vp, vp, i32, vp, vp, i32, vp, sz, vp]
     lib.xfp_dequant.argtypes = [dp, vp, vp, vp]
@@ -112,6 +114,16 @@ def xfp_gemv_v2(desc, packed, x, batch, y, y_is_fp16, workspace, stream=None) ->
 
 def xfp_gemv_v2a(desc, packed, x, batch, y, y_is_fp16, workspace, stream=None) -> None:
     _gemv(load_library().xfp_gemv_v2a, desc, packed, x, batch, y, y_is_fp16, workspace, stream)
+
+
+_TORCH_TYPE = {torch.float32: XFP_T_F32, torch.float16: XFP_T_F16, torch.bfloat16: XFP_T_BF16}
+
+
+def xfp_gemv_typed(desc, packed, x: torch.Tensor, batch, y: torch.Tensor, workspace, stream=None) -> None:
+    """The fused GEMV of desc.mode with x in fp16 or bf16 and y in fp32, fp16 or bf16 (taken from the tensors' dtypes)."""
+    _check(load_library().xfp_gemv_typed(C.byref(desc), _ptr(packed), _ptr(x), _TORCH_TYPE[x.dtype], int(batch), _ptr(y),
+                                         _TORCH_TYPE[y.dtype], _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)), "xfp_gemv_typed")
 
 
 def xfp_gemv_grouped(desc, n: int, packed_ptrs: torch.Tensor, x_ptrs: torch.Tensor, y_ptrs: torch.Tensor,

@@ -135,14 +135,24 @@ int xfp_pack(const xfp_desc* desc, const uint8_t* idx, const uint16_t* codebook,
 
 int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
                 int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream) {
-    GemvCall c{packed, x, y, nullptr, nullptr, nullptr, 1, batch, y_is_fp16, workspace, workspace_bytes};
+    GemvCall c{packed, x, y, nullptr, nullptr, nullptr, 1, batch, y_is_fp16 ? 1 : 0, workspace, workspace_bytes};
     return gemv_common(desc, 0, c, stream);
 }
 
 int xfp_gemv_v2a(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
                  int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream) {
-    GemvCall c{packed, x, y, nullptr, nullptr, nullptr, 1, batch, y_is_fp16, workspace, workspace_bytes};
+    GemvCall c{packed, x, y, nullptr, nullptr, nullptr, 1, batch, y_is_fp16 ? 1 : 0, workspace, workspace_bytes};
     return gemv_common(desc, 1, c, stream);
+}
+
+int xfp_gemv_typed(const xfp_desc* desc, const void* packed, const void* x, int32_t x_type, int32_t batch, void* y,
+                   int32_t y_type, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!desc) return XFP_ERR_NULL;
+    if (x_type != XFP_T_F16 && x_type != XFP_T_BF16) return XFP_ERR_SHAPE;
+    if (y_type != XFP_T_F32 && y_type != XFP_T_F16 && y_type != XFP_T_BF16) return XFP_ERR_SHAPE;
+    GemvCall c{packed, (const uint16_t*)x, y, nullptr, nullptr, nullptr, 1, batch, y_type, workspace, workspace_bytes};
+    c.x_bf16 = x_type == XFP_T_BF16;
+    return gemv_common(desc, desc->mode, c, stream);
 }
 
 int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
@@ -155,7 +165,7 @@ int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed,
     const Layout l = layout_of(desc);
     const size_t need = workspace_bytes_for(l);
     if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
-    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16, workspace, need};
+    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16 ? 1 : 0, workspace, need};
     return gemv_common(desc, desc->mode, c, stream);
 }
 
@@ -173,7 +183,7 @@ int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const
     const Layout l = layout_of(desc);
     const size_t need = workspace_bytes_for(l);
     if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
-    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16, workspace, need};
+    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16 ? 1 : 0, workspace, need};
     c.epilogue = epilogue;
     c.epi_weights = weights;
     return gemv_common(desc, desc->mode, c, stream);

@@ -1,6 +1,7 @@
 // Shared device helpers of the XFP kernels: bit-field extraction from a lane's index stream,
 // cache-hinted loads, fp16 bit casts.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -35,6 +36,46 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 
 __device__ __forceinline__ float h2f(uint16_t b) { return __half2float(__ushort_as_half(b)); }
 __device__ __forceinline__ uint16_t f2h(float f) { return __half_as_ushort(__float2half_rn(f)); }
+
+// Activations may arrive as bf16 (the paper's native type): they are converted to fp16 while they are staged,
+// round to nearest even, clamped to the finite fp16 range.  A bf16 value with |x| in [2^-14, 65504] has 8
+// significant bits and converts exactly; smaller ones land on the fp16 subnormal grid (absolute error <= 2^-25).
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v) {
+    float lo = __uint_as_float(v << 16), hi = __uint_as_float(v & 0xffff0000u);
+    lo = fminf(fmaxf(lo, -65504.f), 65504.f);
+    hi = fminf(fmaxf(hi, -65504.f), 65504.f);
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *(const uint32_t*)&h;
+}
+__device__ __forceinline__ uint4 x8_as_f16(uint4 v, int x_bf16) {
+    if (x_bf16) {
+        v.x = bf16x2_to_f16x2(v.x); v.y = bf16x2_to_f16x2(v.y);
+        v.z = bf16x2_to_f16x2(v.z); v.w = bf16x2_to_f16x2(v.w);
+    }
+    return v;
+}
+__device__ __forceinline__ float x_as_float(uint16_t bits, int x_bf16) {
+    return x_bf16 ? fminf(fmaxf(__uint_as_float((uint32_t)bits << 16), -65504.f), 65504.f) : h2f(bits);
+}
+// Output element i of y: fp32 (kind 0), fp16 (1) or bf16 (2), one rounding of the fp32 sum.
+__device__ __forceinline__ void put_y(void* y, size_t i, float v, int kind) {
+    if (kind == 1) ((uint16_t*)y)[i] = f2h(v);
+    else if (kind == 2) ((uint16_t*)y)[i] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    else ((float*)y)[i] = v;
+}
+
+// TIO (typed IO) instantiations take bf16 x and store any y type; the plain ones keep the two-way store so that
+// the code of the fp16 path is what it was before typed IO existed.
+template <bool TIO>
+__device__ __forceinline__ void store_y(void* y, size_t i, float v, int kind) {
+    if (TIO) {
+        put_y(y, i, v, kind);
+    } else if (kind) {
+        ((uint16_t*)y)[i] = f2h(v);
+    } else {
+        ((float*)y)[i] = v;
+    }
+}
 
 // Pointers of one packed blob.
 struct Blob {

@@ -28,7 +28,7 @@ struct BatchArgs {
     float* partial;  // [KS][NB][rows_ws]
     int* tickets;    // [blocks]
     int rows, cols, RB, SC, rows_ws, ell_slots;
-    int nb, y_is_fp16;
+    int nb, y_is_fp16, x_bf16;
     int n_full, kst, sc_per_split;
 };
 
@@ -38,7 +38,7 @@ __device__ __forceinline__ uint32_t xoff(int bb, uint32_t k) {
     return (((k >> 3) * NB + (uint32_t)bb) << 4) + ((k & 7u) << 1);
 }
 
-template <int N, int NB, int RPL>
+template <int N, int NB, int RPL, bool TIO>
 __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArgs a) {
     constexpr int E = 1 << N;
     constexpr int T = E * E;
@@ -167,6 +167,7 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
         const int k8 = t / NB, bb = t - k8 * NB;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + (size_t)k8 * 8));
+        if (TIO) v = x8_as_f16(v, a.x_bf16);
         *(uint4*)(xs + (size_t)t * 16) = v;
     }
 #pragma unroll
@@ -320,10 +321,7 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
         const int row = blk * ROWS + r;
         const bool dup = (r >= 32) && (RPL * blk + 1 >= a.RB);
         if (!dup && bb < a.nb && row < a.rows) {
-            if (a.y_is_fp16)
-                ((uint16_t*)a.y)[(size_t)bb * a.rows + row] = f2h(red[t]);
-            else
-                ((float*)a.y)[(size_t)bb * a.rows + row] = red[t];
+            store_y<TIO>(a.y, (size_t)bb * a.rows + row, red[t], a.y_is_fp16);
         }
     }
 }
@@ -348,11 +346,11 @@ static int batch_tile(const Layout& l, int batch) {
 
 bool batch_supported(const Layout& l, int batch) { return batch > 2 && batch_tile(l, batch) != 0; }
 
-template <int N, int NB, int RPL>
-static cudaError_t launch_batch(const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+template <int N, int NB, int RPL, bool TIO>
+static cudaError_t launch_batch_io(const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_batch_kernel<N, NB, RPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_batch_kernel<N, NB, RPL, TIO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              224 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -367,7 +365,13 @@ static cudaError_t launch_batch(const BatchArgs& a, dim3 grid, size_t smem, cuda
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_batch_kernel<N, NB, RPL>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_batch_kernel<N, NB, RPL, TIO>, a);
+}
+
+template <int N, int NB, int RPL>
+static cudaError_t launch_batch(const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_batch_io<N, NB, RPL, true>(a, grid, smem, s);
+    return launch_batch_io<N, NB, RPL, false>(a, grid, smem, s);
 }
 
 cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s) {
@@ -388,7 +392,7 @@ cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s
             a.y = (void*)((char*)c.y + (size_t)(b0 + b1) * l.rows * (c.y_is_fp16 ? 2 : 4));
             a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
             a.rows_ws = blocks * 32 * rpl;
-            a.nb = n1; a.y_is_fp16 = c.y_is_fp16;
+            a.nb = n1; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16;
             // schedule: whole-K blocks in whole rounds of slots; the last partial round cut along K (<= 16 slices)
             int rem = blocks % slots, kst = 1;
             if (rem > 0) {

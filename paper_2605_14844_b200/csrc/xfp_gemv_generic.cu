@@ -30,7 +30,7 @@ struct GenericArgs {
     float* partial;  // [problem][KS][BT][rows_pad]
     int* tickets;    // [problem][RB]
     int rows, cols, RB, SC, rows_pad;
-    int KS, sc_per_split, nb, y_is_fp16, L, rep, ell_slots;
+    int KS, sc_per_split, nb, y_is_fp16, L, rep, ell_slots, x_bf16;
 };
 
 template <int N, int MODE, int BT>
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
     for (int t = threadIdx.x; t < BT * kseg; t += kGenericThreads) {
         const int bb = t / kseg, kk = t - bb * kseg;
         float v = 0.f;
-        if (bb < a.nb && kk < nsc * kSuper) v = h2f(x[(size_t)bb * a.cols + (size_t)sc0 * kSuper + kk]);
+        if (bb < a.nb && kk < nsc * kSuper) v = x_as_float(x[(size_t)bb * a.cols + (size_t)sc0 * kSuper + kk], a.x_bf16);
         xs[t] = v;
     }
     __syncthreads();
@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
             const uint32_t col = oe[q] & 0xffffu;
 #pragma unroll
             for (int bb = 0; bb < BT; ++bb)
-                if (bb < a.nb) acc[bb] = fmaf(v, h2f(__ldg(x + (size_t)bb * a.cols + col)), acc[bb]);
+                if (bb < a.nb) acc[bb] = fmaf(v, x_as_float(__ldg(x + (size_t)bb * a.cols + col), a.x_bf16), acc[bb]);
         }
     };
 
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
 #pragma unroll
             for (int bb = 0; bb < BT; ++bb)
                 if (bb < a.nb)
-                    acc[bb] = fmaf(h2f((uint16_t)(e >> 16)), h2f(__ldg(x + (size_t)bb * a.cols + (e & 0xffffu))), acc[bb]);
+                    acc[bb] = fmaf(h2f((uint16_t)(e >> 16)), x_as_float(__ldg(x + (size_t)bb * a.cols + (e & 0xffffu)), a.x_bf16), acc[bb]);
         }
     }
 
@@ -272,10 +272,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
         if (t == 0) a.tickets[(size_t)prob * a.RB + rb] = 0;
     }
     if (t < BT * 32 && bb < a.nb && row < a.rows) {
-        if (a.y_is_fp16)
-            ((uint16_t*)y)[(size_t)bb * a.rows + row] = f2h(total);
-        else
-            ((float*)y)[(size_t)bb * a.rows + row] = total;
+        put_y(y, (size_t)bb * a.rows + row, total, a.y_is_fp16);
     }
 }
 
@@ -367,7 +364,7 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
         const int ks = generic_ksplit(l, bt);
         a.sc_per_split = (l.SC + ks - 1) / ks;
         a.KS = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
-        a.nb = nb; a.y_is_fp16 = c.y_is_fp16; a.L = l.L; a.ell_slots = l.ell_slots;
+        a.nb = nb; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16; a.L = l.L; a.ell_slots = l.ell_slots;
         // V2a: a per-bank copy of the library when it fits, else a single copy (bank conflicts)
         a.rep = (l.mode && (size_t)l.L * l.E * 32 * 4 <= 128 * 1024) ? 32 : 1;
         // grouped calls stride the workspace by the per-problem size the caller was told

@@ -58,7 +58,7 @@ struct PairArgs {
     float* partial;  // [slice][NB][rows_ws]
     int* tickets;    // [blocks]
     int rows, cols, RB, SC, rows_ws, ell_slots;
-    int nb, y_is_fp16;
+    int nb, y_is_fp16, x_bf16;
     int blocks;      // blocks of 32*RPL channels
     // schedule tiers: CTAs [tier_cta[i], tier_cta[i+1]) handle blocks from tier_blk[i] on, each cut into
     // tier_kst[i] slices of tier_spp[i] super-chunks
@@ -80,7 +80,7 @@ __device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
 #endif
 }
 
-template <int N, int NB, int RPL, int W>
+template <int N, int NB, int RPL, int W, bool TIO>
 __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const PairArgs a) {
     constexpr int E = 1 << N;
     constexpr bool kSingle = N > 5;            // N = 6: a pair table (4096 entries) does not fit, one entry per index
@@ -225,6 +225,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
         const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
+        if (TIO) v = x8_as_f16(v, a.x_bf16);
         *(uint4*)(xs + (size_t)t * 8) = v;
     }
     __syncthreads();   // tables and x visible
@@ -480,10 +481,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
             }
         }
         if (writer && active && !dup && bb < a.nb && row < a.rows) {
-            if (a.y_is_fp16)
-                ((uint16_t*)a.y)[(size_t)bb * a.rows + row] = f2h(total);
-            else
-                ((float*)a.y)[(size_t)bb * a.rows + row] = total;
+            store_y<TIO>(a.y, (size_t)bb * a.rows + row, total, a.y_is_fp16);
         }
         stamp(a, 5);
     }
@@ -601,11 +599,11 @@ size_t pair_workspace_bytes(const Layout& l) {
     return align256((size_t)l.RB * 4) + align256((size_t)ksmax * 2 * (size_t)(l.RB + 1) * 32 * 4);
 }
 
-template <int N, int NB, int RPL, int W>
-static cudaError_t launch_pair(const PairArgs& a, int grid, size_t smem, cudaStream_t s) {
+template <int N, int NB, int RPL, int W, bool TIO>
+static cudaError_t launch_pair_io(const PairArgs& a, int grid, size_t smem, cudaStream_t s) {
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_pair_kernel<N, NB, RPL, W>,
+        cudaError_t e = cudaFuncSetAttribute(gemv_pair_kernel<N, NB, RPL, W, TIO>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -625,7 +623,14 @@ static cudaError_t launch_pair(const PairArgs& a, int grid, size_t smem, cudaStr
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = cluster > 1 ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, gemv_pair_kernel<N, NB, RPL, W>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_pair_kernel<N, NB, RPL, W, TIO>, a);
+}
+
+// bf16 activations or bf16 outputs take the typed-IO instantiation; everything else the plain one
+template <int N, int NB, int RPL, int W>
+static cudaError_t launch_pair(const PairArgs& a, int grid, size_t smem, cudaStream_t s) {
+    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_pair_io<N, NB, RPL, W, true>(a, grid, smem, s);
+    return launch_pair_io<N, NB, RPL, W, false>(a, grid, smem, s);
 }
 
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s) {
@@ -640,7 +645,7 @@ cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s)
     for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
     for (int i = 0; i < 4; ++i) { a.tier_blk[i] = sch.tier_blk[i]; a.tier_kst[i] = sch.tier_kst[i]; a.tier_spp[i] = sch.tier_spp[i]; }
     a.cluster = sch.cluster && g_pair_ks_override == 0;
-    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
+    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16;
     a.trace = nullptr;
     if (g_pair_trace && g_pair_trace_idx < g_pair_trace_calls) a.trace = g_pair_trace + (g_pair_trace_idx++) * 1024 * 8;
     a.tickets = (int*)c.workspace;

@@ -52,7 +52,7 @@ struct V2aArgs {
     float* partial;  // [blob][KS][NB][rows_ws]
     int* tickets;    // [blob][blocks]
     int rows, cols, RB, SC, rows_ws, ell_slots, L;
-    int nb, y_is_fp16;
+    int nb, y_is_fp16, x_bf16;
     int blocks, n_full, kst, sc_per_split;
     int n_a, kst_b, sc_per_split_b;   // of the cut blocks the first n_a use kst slices, the rest kst_b (finer) slices
     int items_x, n;   // work items per blob (whole blocks + K slices), blobs
@@ -101,8 +101,10 @@ __device__ __forceinline__ uint32_t pair_entry_addr(const uint32_t* w, int p, ui
     return (v & mask) | base;
 }
 
-template <int N, int NB, int W, bool PAIR>
+// FEAT instantiations carry typed IO (bf16 x, bf16 y) and the fused stores; the plain ones compile them out.
+template <int N, int NB, int W, bool PAIR, bool FEAT>
 __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const V2aArgs a) {
+    const int epi = FEAT ? a.epi : 0;
     constexpr int E = 1 << N;
     constexpr int kAWarps = W;
     constexpr int kAThreads = W * 32;
@@ -128,15 +130,15 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
     // The weighted sum over the blobs (epi 2) deals RUNS instead: a CTA takes comb_ng consecutive blobs of
     // one block of channels and adds their weighted results in registers; only the comb_G runs of a block
     // meet in the scratch (none when one run covers all blobs).
-    const int per = a.epi == 2 ? a.comb_ng : 1;
-    const int nrun = a.epi == 2 ? a.blocks * a.comb_G : a.items_x * a.n;
+    const int per = epi == 2 ? a.comb_ng : 1;
+    const int nrun = epi == 2 ? a.blocks * a.comb_G : a.items_x * a.n;
     float csum = 0.f;   // epi 2: this thread's channel, weighted sum over the blobs of the run
 #pragma unroll 1
     for (int run = blockIdx.x; run < nrun; run += gridDim.x) {
 #pragma unroll 1
     for (int jj = 0; jj < per; ++jj) {
     int prob, bx;
-    if (a.epi == 2) {
+    if (epi == 2) {
         bx = run / a.comb_G;
         prob = (run - bx * a.comb_G) * a.comb_ng + jj;
         if (prob >= a.n) break;
@@ -155,7 +157,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
         const int t = bx - a.n_full - a.n_a * a.kst;
         blk = a.n_full + a.n_a + t / a.kst_b; ks = t % a.kst_b; KS = a.kst_b; spp = a.sc_per_split_b;
     }
-    const float epi_wj = a.epi == 2 ? __ldg(a.epi_w + prob) : 0.f;   // fetched now, used in the store
+    const float epi_wj = epi == 2 ? __ldg(a.epi_w + prob) : 0.f;   // fetched now, used in the store
     const void* packed = a.packed_list ? a.packed_list[prob] : a.packed;
     const uint16_t* x = a.x_list ? a.x_list[prob] : a.x;
     void* y = a.y_list ? a.y_list[prob] : a.y;
@@ -276,6 +278,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
                 const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
                 if (bb < a.nb) v = __ldg((const uint4*)(x + (size_t)bb * a.cols + kk));
+                if (FEAT) v = x8_as_f16(v, a.x_bf16);
                 *(uint4*)(xs + (size_t)t * 8) = v;
             }
         }
@@ -457,14 +460,11 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
             if (t == 0) *ticket = 0;
         }
     }
-    if (a.epi == 0) {
+    if (epi == 0) {
         if (writer && active && !dup && bb < a.nb && row < a.rows) {
-            if (a.y_is_fp16)
-                ((uint16_t*)y)[(size_t)bb * a.rows + row] = f2h(total);
-            else
-                ((float*)y)[(size_t)bb * a.rows + row] = total;
+            store_y<FEAT>(y, (size_t)bb * a.rows + row, total, a.y_is_fp16);
         }
-    } else if (a.epi == 1) {
+    } else if (epi == 1) {
         // gated activation of a routed expert: channels 0..31 of the block are gates, 32..63 the matching
         // up channels; the block stores 32 values h = SiLU(gate) * up  (batch 1, rows a multiple of 64)
         if (writer) {
@@ -475,8 +475,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
                 const float g = red[t], u = red[t + 32];
                 const float h = g / (1.f + expf(-g)) * u;
                 const size_t o = (size_t)blk * 32 + t;
-                if (a.y_is_fp16) ((uint16_t*)y)[o] = f2h(h);
-                else ((float*)y)[o] = h;
+                put_y(y, o, h, a.y_is_fp16);
             }
         }
     } else {
@@ -486,8 +485,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
         if (run_done && a.comb_G == 1) {
             if (t < kARows && !dup && row < a.rows) {
                 void* y0 = a.y_list ? a.y_list[0] : a.y;
-                if (a.y_is_fp16) ((uint16_t*)y0)[row] = f2h(csum);
-                else ((float*)y0)[row] = csum;
+                put_y(y0, row, csum, a.y_is_fp16);
             }
         } else if (run_done) {
             // the runs of this block leave their sums in the scratch, the last one to arrive adds them in run order
@@ -505,8 +503,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
                     float sum = 0.f;
                     for (int g2 = 0; g2 < a.comb_G; ++g2) sum += __ldcg(comb + (size_t)g2 * a.rows_ws + row);
                     void* y0 = a.y_list ? a.y_list[0] : a.y;
-                    if (a.y_is_fp16) ((uint16_t*)y0)[row] = f2h(sum);
-                    else ((float*)y0)[row] = sum;
+                    put_y(y0, row, sum, a.y_is_fp16);
                 }
                 if (t == 0) *ticket = 0;
             }
@@ -557,11 +554,11 @@ size_t v2a_workspace_bytes(const Layout& l) {
     return align256((size_t)blocks * 4) + align256((size_t)64 * 2 * (size_t)blocks * kARows * 4);
 }
 
-template <int N, int NB, int W, bool PAIR>
-static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+template <int N, int NB, int W, bool PAIR, bool FEAT>
+static cudaError_t launch_v2a_feat(const V2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB, W, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB, W, PAIR, FEAT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              W == 8 ? 112 * 1024 : 226 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -576,7 +573,13 @@ static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_v2a_kernel<N, NB, W, PAIR>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_v2a_kernel<N, NB, W, PAIR, FEAT>, a);
+}
+
+template <int N, int NB, int W, bool PAIR>
+static cudaError_t launch_v2a(const V2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+    if (a.epi != 0 || a.x_bf16 || a.y_is_fp16 == 2) return launch_v2a_feat<N, NB, W, PAIR, true>(a, grid, smem, s);
+    return launch_v2a_feat<N, NB, W, PAIR, false>(a, grid, smem, s);
 }
 
 template <int N, int NB>
@@ -595,7 +598,7 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     a.packed = c.packed; a.x = c.x; a.y = c.y;
     a.packed_list = c.packed_list; a.x_list = c.x_list; a.y_list = c.y_list;
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots; a.L = l.L;
-    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16;
+    a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16;
     a.blocks = (l.RB + 1) / 2;
     a.rows_ws = a.blocks * kARows;
     // schedule: whole-K blocks fill whole rounds of CTA slots (all blobs of the launch count); the blocks of

@@ -32,11 +32,12 @@ struct GemvCall {
     void* const* y_list;
     int n;          // number of problems (1 for the single form)
     int batch;      // rows of x (1..16)
-    int y_is_fp16;
+    int y_is_fp16;  // type of y: 0 fp32, 1 fp16, 2 bf16
     void* workspace;
     size_t workspace_bytes;  // per problem
     int epilogue = 0;                      // XFP_EPI_* (grouped V2a launches only)
     const float* epi_weights = nullptr;    // XFP_EPI_COMBINE: [n] routing weights on the device
+    int x_bf16 = 0;                        // x holds bf16 instead of fp16
 };
 
 // Split-K factor the generic kernel uses for this shape and batch tile (host-side policy).

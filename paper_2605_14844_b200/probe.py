@@ -4,7 +4,7 @@
         pack one synthetic matrix and call the GEMV LAUNCHES times, evicting the matrix from L2 (a
         512 MB fill) before every call -- the target of `ncu -k regex:gemv` captures.
 
-    python -m paper_2605_14844_b200.probe time MODE ROWS COLS BITS RATE [BATCH] [PLACEMENT]
+    python -m paper_2605_14844_b200.probe time MODE ROWS COLS BITS RATE [BATCH] [PLACEMENT] [fp16|bf16]
         time back-to-back calls over enough distinct packed copies to exceed twice the L2 (one CUDA
         graph of P calls, median of 20 replays) and print microseconds per call and effective GB/s over
         the algorithmic bytes.
@@ -73,22 +73,33 @@ def launch(mode, rows, cols, bits, rate, n=3, placement="uniform"):
     print("ok", float(y.float().abs().sum()))
 
 
-def time_shape(mode, rows, cols, bits, rate, batch=1, placement="uniform", reps=20):
+def time_shape(mode, rows, cols, bits, rate, batch=1, placement="uniform", reps=20, dtype="fp16"):
+    from . import xfp_gemv_typed
     q = synth.random_quantized(mode, rows, cols, bits, rate, seed=1, placement=placement)
     nb = algorithmic_bytes(q, batch=batch)
     copies = max(2, int(300e6 // nb) + 1)
     pms = [pack_tensors(q, col_bits=16) for _ in range(copies)]
     x = _x(batch, cols)
-    ys = [torch.empty((batch, rows), dtype=torch.float16, device="cuda") for _ in range(copies)]
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float16
+    if dtype == "bf16":
+        x = x.to(torch.bfloat16)
+    ys = [torch.empty((batch, rows), dtype=tdt, device="cuda") for _ in range(copies)]
+
+    def call(pm, y):
+        if dtype == "bf16":    # bf16 activations and outputs through the typed entry point
+            xfp_gemv_typed(pm.desc, pm.packed, x, batch, y, pm.workspace)
+        else:
+            pm.gemv(x, y=y, y_fp16=True)
+
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
         for pm, y in zip(pms, ys):
-            pm.gemv(x, y=y, y_fp16=True)
+            call(pm, y)
         s.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=s):
             for pm, y in zip(pms, ys):
-                pm.gemv(x, y=y, y_fp16=True)
+                call(pm, y)
         for _ in range(3):
             g.replay()
         s.synchronize()
@@ -101,7 +112,7 @@ def time_shape(mode, rows, cols, bits, rate, batch=1, placement="uniform", reps=
             s.synchronize()
             ts.append(e0.elapsed_time(e1) * 1e3 / copies)
     t = float(np.median(ts))
-    out = dict(mode=mode, rows=rows, cols=cols, bits=bits, rate=rate, batch=batch, placement=placement,
+    out = dict(mode=mode, rows=rows, cols=cols, bits=bits, rate=rate, batch=batch, placement=placement, dtype=dtype,
                copies=copies, MB=round(nb / 1e6, 2), us_per_call=round(t, 3), us_best=round(float(np.min(ts)), 3),
                GBs=round(nb / t / 1e3, 1))
     print(json.dumps(out), flush=True)
@@ -335,7 +346,7 @@ def main(argv):
         launch(mode, rows, cols, bits, rate, int(argv[7]) if len(argv) > 7 else 3, argv[8] if len(argv) > 8 else "uniform")
     else:
         time_shape(mode, rows, cols, bits, rate, int(argv[7]) if len(argv) > 7 else 1,
-                   argv[8] if len(argv) > 8 else "uniform")
+                   argv[8] if len(argv) > 8 else "uniform", dtype=argv[9] if len(argv) > 9 else "fp16")
     return 0
 
 

@@ -431,3 +431,53 @@ def test_fused_epilogues_are_refused_where_not_built():
     with pytest.raises(xfp.XfpError):                                # the weighted sum needs its weights
         xfp.xfp_gemv_grouped_epilogue(pa.desc, 1, ptr([pa.packed]), ptr([x]), ptr([y]), False, xfp.XFP_EPI_COMBINE, None,
                                       pa.workspace)
+
+
+def _bf16_x(batch, cols, seed):
+    """N(0,1) activations rounded to bf16 (torch), with their exact values as doubles."""
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn((batch, cols), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    return x.cuda(), x.to(torch.float64).numpy()
+
+
+@pytest.mark.parametrize("mode,bits", CASES)
+@pytest.mark.parametrize("batch", [1, 2, 5, 16])
+def test_bf16_activations_and_outputs(mode, bits, batch):
+    """xfp_gemv_typed: bf16 x (converted to fp16 while staged) and y in fp32 / bf16 / fp16, every kernel the
+    dispatcher can pick.  Reference: the oracle on the exact bf16 values.  Tolerance: the GEMV bound, plus
+    2^-25 sum|W| for activations below 2^-14 (they land on the fp16 subnormal grid), plus the output rounding."""
+    rows, cols = 288, 1152
+    q = synth.random_quantized(mode, rows, cols, bits, 0.01, seed=2600 + 10 * mode + bits)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    xd, x64 = _bf16_x(batch, cols, 2700 + batch)
+    ref, absum = xo.gemv_x64(to_oracle(q), x64)
+    tiny = 2.0 ** -25 * np.abs(xo.dequant(to_oracle(q)).view(np.float16).astype(np.float64)).sum(1)[None, :]
+    for dt, ulp in ((torch.float32, 0.0), (torch.bfloat16, 2.0 ** -8), (torch.float16, 2.0 ** -11)):
+        y = torch.full((batch, rows), float("nan"), dtype=dt, device="cuda")
+        xfp.xfp_gemv_typed(pm.desc, pm.packed, xd, batch, y, pm.workspace)
+        torch.cuda.synchronize()
+        got = y.to(torch.float64).cpu().numpy()
+        tol = TOL * absum + tiny + ulp * np.abs(ref) + 1e-30
+        assert np.all(np.abs(got - ref) <= tol), (dt, float((np.abs(got - ref) / tol).max()))
+    # fp16 x through the typed entry is the plain entry
+    x16 = synth.activations(batch, cols, seed=2800)
+    y1 = torch.empty((batch, rows), dtype=torch.float32, device="cuda")
+    xfp.xfp_gemv_typed(pm.desc, pm.packed, _x_dev(x16), batch, y1, pm.workspace)
+    y2 = pm.gemv(_x_dev(x16))
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+
+
+def test_bf16_activations_outside_the_fp16_range_are_clamped():
+    q = synth.random_quantized(0, 64, 256, 4, 0.0, seed=2900)
+    pm = xfp.pack_tensors(q)
+    x = torch.zeros((1, 256), dtype=torch.bfloat16)
+    x[0, 3], x[0, 100], x[0, 200] = 1.0e6, -3.0e38, 2.0 ** -30
+    y = torch.empty((1, 64), dtype=torch.float32, device="cuda")
+    xfp.xfp_gemv_typed(pm.desc, pm.packed, x.cuda(), 1, y, pm.workspace)
+    torch.cuda.synchronize()
+    xc = x.to(torch.float64).numpy().clip(-65504.0, 65504.0)
+    xc[0, 200] = 0.0                                   # below half the smallest fp16 subnormal: rounds to zero
+    ref, absum = xo.gemv_x64(to_oracle(q), xc)
+    assert np.all(np.isfinite(y.cpu().numpy()))
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * absum + 1e-30)

@@ -287,3 +287,29 @@ def test_gemv_row_window():
     full, _ = xo.gemv(to_oracle(q), x16)
     part, _ = xo.gemv(to_oracle(q), x16, 7, 19)
     assert np.array_equal(part[:, 7:19], full[:, 7:19]) and not part[:, :7].any() and not part[:, 19:].any()
+
+
+def test_gemv_with_real_activations_matches_the_fp16_entry_and_a_dense_matvec():
+    """gemv_x64 (activations as doubles, for bf16 inputs) is the same sum as gemv on fp16-representable x,
+    and equals a dense numpy matvec on values fp16 cannot hold."""
+    from paper_2605_14844_b200 import synth
+    from conftest import to_oracle
+    for mode in (0, 1):
+        q = synth.random_quantized(mode, 48, 384, 4, 0.01, seed=61 + mode)
+        m = to_oracle(q)
+        x16 = synth.activations(2, 384, seed=62)
+        y16, a16 = xo.gemv(m, x16)
+        y64, a64 = xo.gemv_x64(m, x16.view(np.float16).astype(np.float64))
+        assert np.array_equal(y16, y64) and np.array_equal(a16, a64)
+        # bf16-like values outside the fp16 range: 8 significant bits, exponents down to 2^-30 and up to 2^20
+        rng = np.random.default_rng(63)
+        xr = np.round(rng.uniform(1, 2, (2, 384)) * 128) / 128 * 2.0 ** rng.integers(-30, 21, (2, 384))
+        y, a = xo.gemv_x64(m, xr)
+        if mode == 0:           # V2: D + S written out densely (the sum before any rounding), then a plain matvec
+            cb = q.codebook.view(np.float16).astype(np.float64)
+            Wd = np.take_along_axis(cb, q.idx.astype(np.int64), axis=1)
+            for i in range(q.rows):
+                for p_ in range(q.rowptr[i], q.rowptr[i + 1]):
+                    Wd[i, q.ocol[p_]] += float(q.oval[p_:p_ + 1].view(np.float16)[0])
+            assert np.allclose(y, (Wd @ xr.T).T, rtol=1e-12, atol=0)
+        assert np.all(a >= np.abs(y))
