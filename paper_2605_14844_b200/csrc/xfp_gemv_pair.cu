@@ -55,6 +55,12 @@ struct PairArgs {
     const void* packed;
     const uint16_t* x;
     void* y;
+    // several blobs of one shape in one launch (typed-IO instantiations only): device pointer lists; the
+    // blocks of all blobs are numbered through, blocks_per of them belong to each blob
+    const void* const* packed_list;
+    const uint16_t* const* x_list;
+    void* const* y_list;
+    int blocks_per, prob0;   // blocks per blob; first blob of this launch
     float* partial;  // [slice][NB][rows_ws]
     int* tickets;    // [blocks]
     int rows, cols, RB, SC, rows_ws, ell_slots;
@@ -101,7 +107,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
     stamp(a, 0);
-    const Blob b = blob_at(a.packed, a.off);
+    Blob b = blob_at(a.packed, a.off);
     const int K = a.SC * kSuper;
 
     unsigned char* tab = smem;
@@ -122,8 +128,26 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
         sc0 = slice * a.tier_spp[tier];
         nsc = max(0, min(a.SC, sc0 + a.tier_spp[tier]) - sc0);
     }
-    const int blk0 = RPL * blk;
-    const int blk1 = min(RPL * blk + (RPL - 1), a.RB - 1);   // clamped when RB is odd; its results are dropped
+    // the blob of this block: `blk` numbers the blocks of the whole launch, `lblk` those of its blob
+    int lblk = blk;
+    const uint16_t* xsrc = a.x;
+    void* ydst = a.y;
+    int ell_slots = a.ell_slots;
+    const uint32_t* ell = b.ell;
+    if (TIO && a.packed_list) {
+        const int pj = blk / a.blocks_per;
+        const int prob = a.prob0 + pj;
+        lblk = blk - pj * a.blocks_per;
+        const void* packed = a.packed_list[prob];
+        xsrc = a.x_list[prob]; ydst = a.y_list[prob];
+        b = blob_at(packed, a.off);
+        // the blobs' outlier counts differ: slab geometry from each blob's header
+        const int* hdr = (const int*)((const char*)packed + a.off.hdr);
+        ell_slots = __ldg(hdr);
+        ell = (const uint32_t*)((const char*)packed + *(const long long*)(hdr + 2));
+    }
+    const int blk0 = RPL * lblk;
+    const int blk1 = min(RPL * lblk + (RPL - 1), a.RB - 1);   // clamped when RB is odd; its results are dropped
     const int gw = slice * W + warp, ostride = nslices * W;
 
     // per-thread state
@@ -164,11 +188,11 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
         }
 #pragma unroll
         for (int h = 0; h < RPL; ++h) {
-            slab[h] = b.ell + (size_t)(h ? blk1 : blk0) * (a.ell_slots + 1) * 32 + lane;
-            width[h] = a.ell_slots;   // capacity: every slot below it is readable
-            olen[h] = a.ell_slots ? __ldg(slab[h]) : 0u;
+            slab[h] = ell + (size_t)(h ? blk1 : blk0) * (ell_slots + 1) * 32 + lane;
+            width[h] = ell_slots;   // capacity: every slot below it is readable
+            olen[h] = ell_slots ? __ldg(slab[h]) : 0u;
         }
-        if (a.ell_slots) fetch_slots(0);
+        if (ell_slots) fetch_slots(0);
         if (TW >= E) {
 #pragma unroll
             for (int half = 0; half < RPL; ++half) {
@@ -224,7 +248,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
     for (int t = threadIdx.x; t < NB * (K / 8); t += kThreads) {
         const int bb = t / (K / 8), kk = (t - bb * (K / 8)) * 8;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + kk));
+        if (bb < a.nb) v = __ldg((const uint4*)(xsrc + (size_t)bb * a.cols + kk));
         if (TIO) v = x8_as_f16(v, a.x_bf16);
         *(uint4*)(xs + (size_t)t * 8) = v;
     }
@@ -281,7 +305,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
             int wmax = (int)olen[h];
 #pragma unroll
             for (int o = 16; o; o >>= 1) wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
-            width[h] = min(wmax, a.ell_slots);
+            width[h] = min(wmax, ell_slots);
             const int mine = width[h] > gw ? (width[h] - gw + ostride - 1) / ostride : 0;
             nrounds = max(nrounds, (mine + kSlotsPerRound - 1) / kSlotsPerRound);
 #pragma unroll
@@ -395,13 +419,13 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
         }
         // Rows that fill their slab may continue in the CSR arrays (pathological skew only): warp 0 of
         // the block's first slice finishes them, one lane per row.
-        if (warp == 0 && slice == 0 && a.ell_slots) {
+        if (warp == 0 && slice == 0 && ell_slots) {
 #pragma unroll
             for (int h = 0; h < RPL; ++h) {
-                if ((int)olen[h] >= a.ell_slots) {
+                if ((int)olen[h] >= ell_slots) {
                     const int row = (h ? blk1 : blk0) * kRowsPerBlock + lane;
                     const int p1 = __ldg(b.rowptr + row + 1);
-                    for (int p = __ldg(b.rowptr + row) + a.ell_slots; p < p1; ++p) {
+                    for (int p = __ldg(b.rowptr + row) + ell_slots; p < p1; ++p) {
                         const uint32_t e = __ldg(b.oent + p);
 #pragma unroll
                         for (int bb = 0; bb < NB; ++bb)
@@ -442,8 +466,9 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
         const int t = threadIdx.x;
         const int bb = t / ROWS, r = t % ROWS;
         const bool active = t < NB * ROWS;
-        const bool dup = (r >= 32) && (RPL * cur_blk + 1 >= a.RB);
-        const int row = cur_blk * ROWS + r;
+        const bool dup = (r >= 32) && (RPL * lblk + 1 >= a.RB);
+        const int row = lblk * ROWS + r;               // channel inside its blob (y index)
+        const int wrow = cur_blk * ROWS + r;           // channel inside the launch (workspace index)
         float total = 0.f;
         if (active) {
 #pragma unroll
@@ -464,7 +489,7 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
             writer = cur_slice == 0;
         } else if (cur_nslices > 1) {
             __shared__ int s_last;
-            if (active) a.partial[((size_t)cur_slice * NB + bb) * a.rows_ws + row] = total;
+            if (active) a.partial[((size_t)cur_slice * NB + bb) * a.rows_ws + wrow] = total;
             __threadfence();
             __syncthreads();
             if (t == 0) s_last = (atomicAdd(a.tickets + cur_blk, 1) == cur_nslices - 1);
@@ -475,13 +500,13 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
                 if (active) {
                     total = 0.f;
                     for (int k2 = 0; k2 < cur_nslices; ++k2)
-                        total += __ldcg(a.partial + ((size_t)k2 * NB + bb) * a.rows_ws + row);
+                        total += __ldcg(a.partial + ((size_t)k2 * NB + bb) * a.rows_ws + wrow);
                 }
                 if (t == 0) a.tickets[cur_blk] = 0;
             }
         }
         if (writer && active && !dup && bb < a.nb && row < a.rows) {
-            store_y<TIO>(a.y, (size_t)bb * a.rows + row, total, a.y_is_fp16);
+            store_y<TIO>(ydst, (size_t)bb * a.rows + row, total, a.y_is_fp16);
         }
         stamp(a, 5);
     }
@@ -505,12 +530,12 @@ void pair_set_small(int v) { g_pair_small = v; }
 
 struct PairConfig { int rpl, warps, slots; };
 
-static PairConfig pair_config(const Layout& l) {
+static PairConfig pair_config(const Layout& l, int n = 1) {
     // N <= 4: two rows per lane, 8 warps, two CTAs per SM.  N = 5: the pair table of a row is 4 KB, so
     // one row per lane (128 KB of tables), 16 warps, one CTA per SM.  Matrices with at most 148
     // row-blocks also take one row per lane: twice the CTAs and no cut along K.
     if (l.bits == 5) return PairConfig{1, 16, 148};
-    if (g_pair_small >= 1 && l.RB <= 148 * g_pair_small && l.bits >= 3) return PairConfig{1, 16, 148};
+    if (g_pair_small >= 1 && (long long)l.RB * n <= 148 * g_pair_small && l.bits >= 3) return PairConfig{1, 16, 148};
     return PairConfig{2, 8, 296};
 }
 
@@ -525,10 +550,10 @@ static int pow2_floor(int v) {
     return p;
 }
 
-static PairSchedule pair_schedule(const Layout& l) {
-    const PairConfig cfg = pair_config(l);
+static PairSchedule pair_schedule(const Layout& l, int n = 1) {
+    const PairConfig cfg = pair_config(l, n);
     PairSchedule sc{};
-    sc.blocks = (l.RB + cfg.rpl - 1) / cfg.rpl;
+    sc.blocks = ((l.RB + cfg.rpl - 1) / cfg.rpl) * n;   // the blocks of all blobs of the launch
     const int S = cfg.slots;
     const int kmax = l.SC / 4 > 1 ? pow2_floor(l.SC / 4) : 1;   // keep K slices of at least 512 weights
     int nb[4] = {0, 0, 0, 0}, kk[4] = {1, 1, 1, 1};
@@ -581,8 +606,8 @@ static PairSchedule pair_schedule(const Layout& l) {
     return sc;
 }
 
-static size_t pair_smem_bytes(const Layout& l, int nb) {
-    const PairConfig cfg = pair_config(l);
+static size_t pair_smem_bytes(const Layout& l, int nb, int n = 1) {
+    const PairConfig cfg = pair_config(l, n);
     const int rows = 32 * cfg.rpl;
     const size_t T = l.bits > 5 ? (size_t)l.E : (size_t)l.E * l.E;   // N = 6: one entry per index
     const int sl = (cfg.rpl == 2 || l.bits == 4) ? 2 : 1;              // entry stride in units of 128 bytes
@@ -590,8 +615,9 @@ static size_t pair_smem_bytes(const Layout& l, int nb) {
 }
 
 bool pair_supported(const Layout& l, int batch, int n_problems) {
-    if (l.mode != 0 || l.bits < 2 || l.bits > 6 || batch > 2 || n_problems != 1) return false;
-    return pair_smem_bytes(l, batch) <= (pair_config(l).warps == 8 ? 110u : 220u) * 1024u;
+    if (l.mode != 0 || l.bits < 2 || l.bits > 6 || batch > 2 || n_problems < 1) return false;
+    if (n_problems > 1 && batch != 1) return false;
+    return pair_smem_bytes(l, batch, n_problems) <= (pair_config(l, n_problems).warps == 8 ? 110u : 220u) * 1024u;
 }
 
 size_t pair_workspace_bytes(const Layout& l) {
@@ -629,16 +655,39 @@ static cudaError_t launch_pair_io(const PairArgs& a, int grid, size_t smem, cuda
 // bf16 activations or bf16 outputs take the typed-IO instantiation; everything else the plain one
 template <int N, int NB, int RPL, int W>
 static cudaError_t launch_pair(const PairArgs& a, int grid, size_t smem, cudaStream_t s) {
-    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_pair_io<N, NB, RPL, W, true>(a, grid, smem, s);
+    if (a.x_bf16 || a.y_is_fp16 == 2 || a.packed_list) return launch_pair_io<N, NB, RPL, W, true>(a, grid, smem, s);
     return launch_pair_io<N, NB, RPL, W, false>(a, grid, smem, s);
 }
 
+static cudaError_t launch_gemv_pair_n(const Layout& l, const GemvCall& c, int prob0, cudaStream_t s);
+
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s) {
-    const PairConfig cfg = pair_config(l);
-    const PairSchedule sch = pair_schedule(l);
+    // N >= 5 (large tables: one CTA per SM, or two channels per lane at N = 6) gains nothing from a common schedule
+    // once the blocks exceed one round: one launch per blob, read through the same lists.
+    if (c.n > 1) {
+        const PairConfig one_cfg = pair_config(l, 1);
+        if (l.bits >= 5 && (long long)((l.RB + one_cfg.rpl - 1) / one_cfg.rpl) * c.n > one_cfg.slots) {
+            GemvCall one = c;
+            one.n = 1;
+            for (int j = 0; j < c.n; ++j) {
+                const cudaError_t e = launch_gemv_pair_n(l, one, j, s);
+                if (e != cudaSuccess) return e;
+            }
+            return cudaSuccess;
+        }
+    }
+    return launch_gemv_pair_n(l, c, 0, s);
+}
+
+static cudaError_t launch_gemv_pair_n(const Layout& l, const GemvCall& c, int prob0, cudaStream_t s) {
+    const PairConfig cfg = pair_config(l, c.n);
+    const PairSchedule sch = pair_schedule(l, c.n);
     PairArgs a{};
     a.off = offsets_of(l);
     a.packed = c.packed; a.x = c.x; a.y = c.y;
+    a.packed_list = c.packed_list; a.x_list = c.x_list; a.y_list = c.y_list;
+    a.blocks_per = sch.blocks / c.n;
+    a.prob0 = prob0;
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
     a.blocks = sch.blocks;
     a.rows_ws = sch.blocks * 32 * cfg.rpl;
@@ -649,8 +698,8 @@ cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s)
     a.trace = nullptr;
     if (g_pair_trace && g_pair_trace_idx < g_pair_trace_calls) a.trace = g_pair_trace + (g_pair_trace_idx++) * 1024 * 8;
     a.tickets = (int*)c.workspace;
-    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
-    const size_t smem = pair_smem_bytes(l, c.batch);
+    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4 * c.n));
+    const size_t smem = pair_smem_bytes(l, c.batch, c.n);
     if (cfg.rpl == 1) {
         switch (l.bits * 10 + c.batch) {
             case 31: return launch_pair<3, 1, 1, 16>(a, sch.grid, smem, s);

@@ -28,6 +28,10 @@
         {0, 0.5, 1, 2} % (seeded), V2 and V2a on the same draws; one token through the stack is one CUDA graph.  Prints
         milliseconds per token and effective GB/s.
 
+    python -m paper_2605_14844_b200.probe qkv [BITS]
+        the dense-attention block (q, k, v, o 4096 x 4096, V2, ~0.9 % clustered outliers) as four calls and as
+        one grouped launch for q, k, v (they share x) plus the call for o; microseconds per block.
+
     python -m paper_2605_14844_b200.probe quant MODE ROWS COLS BITS [REPS]
         the encoder on one synthetic float matrix (Gaussian bulk with heavy outlier columns for V2, 0.1 % uniform
         outliers for V2a): device time of every stage (statistics, extraction, Lloyd, LibFit, residual,
@@ -262,6 +266,60 @@ def stack(layers=48, reps=5):
         torch.cuda.empty_cache()
 
 
+def qkv(bits=4, reps=20):
+    """The attention block's q, k, v (shared x) as three calls against one grouped launch; o stays a call of its own."""
+    from . import XfpDesc, xfp_gemv_grouped, xfp_packed_size
+    rows = cols = 4096
+    sets = max(2, int(300e6 // (4 * rows * cols * bits // 8)) + 1)
+    blocks = []
+    nb = 0
+    for st in range(sets):
+        qs = [synth.random_quantized(0, rows, cols, bits, 0.009, seed=10 + j, placement="clustered") for j in range(4)]
+        blocks.append([pack_tensors(q, col_bits=16) for q in qs])
+        nb = sum(algorithmic_bytes(q) for q in qs)
+    x = _x(1, cols)
+    ys = [torch.empty((4, rows), dtype=torch.float16, device="cuda") for _ in range(sets)]
+    d0 = blocks[0][0].desc
+    desc = XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                   max(p.desc.nnz for b in blocks for p in b))
+    ws = torch.zeros(3 * xfp_packed_size(desc)[1], dtype=torch.uint8, device="cuda")
+    ptrs = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    lists = [(ptrs([p.packed for p in b[:3]]), ptrs([x] * 3), ptrs([y[j] for j in range(3)])) for b, y in zip(blocks, ys)]
+    out = {}
+    for name in ("four_calls", "grouped_qkv_plus_o"):
+        def block(i):
+            b, y = blocks[i], ys[i]
+            if name == "four_calls":
+                for j in range(3):
+                    b[j].gemv(x, y=y[j:j + 1], y_fp16=True)
+            else:
+                xfp_gemv_grouped(desc, 3, lists[i][0], lists[i][1], lists[i][2], True, ws)
+            b[3].gemv(x, y=y[3:4], y_fp16=True)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for i in range(sets):
+                block(i)
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for i in range(sets):
+                    block(i)
+            for _ in range(3):
+                g.replay()
+            s.synchronize()
+            ts = []
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s)
+                g.replay()
+                e1.record(s)
+                s.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3 / sets)
+        out[name + "_us_per_block"] = round(float(np.median(ts)), 3)
+        out[name + "_GBs"] = round(nb / float(np.median(ts)) / 1e3, 1)
+    print(json.dumps(dict(workload="attention_block_qkv_o", bits=bits, MB_per_block=round(nb / 1e6, 2), **out)), flush=True)
+
+
 def quant(mode, rows, cols, bits, reps=3):
     """Device time per encoder stage, and the whole Algorithm 1 call, on one rows x cols float matrix."""
     from . import XfpDesc
@@ -325,6 +383,9 @@ def quant(mode, rows, cols, bits, reps=3):
 
 
 def main(argv):
+    if len(argv) > 1 and argv[1] == "qkv":
+        qkv(*(int(v) for v in argv[2:3]))
+        return 0
     if len(argv) > 1 and argv[1] == "quant":
         quant(*(int(v) for v in argv[2:7]))
         return 0

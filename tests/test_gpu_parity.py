@@ -481,3 +481,37 @@ def test_bf16_activations_outside_the_fp16_range_are_clamped():
     ref, absum = xo.gemv_x64(to_oracle(q), xc)
     assert np.all(np.isfinite(y.cpu().numpy()))
     assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * absum + 1e-30)
+
+
+@pytest.mark.parametrize("bits,n,rows,cols", [(4, 3, 4096, 4096), (5, 3, 1024, 2048), (3, 2, 9600, 1024), (2, 7, 96, 512),
+                                              (6, 4, 2080, 384)])
+def test_grouped_v2_blobs_on_the_pair_kernel(bits, n, rows, cols):
+    """Several V2 blobs of one shape in one launch (q, k and v of an attention block share x): blocks of all
+    blobs are scheduled together, whole rounds first and K slices for the tail, every blob with its own
+    codebooks and outlier slabs.  Sampled channels against the oracle, and the whole output against single calls."""
+    qs = [synth.random_quantized(0, rows, cols, bits, 0.003 * (j + 1), seed=3000 + 7 * j + bits,
+                                 placement="clustered" if j % 2 else "uniform") for j in range(n)]
+    pms = [xfp.pack_tensors(q, col_bits=16) for q in qs]
+    x16 = synth.activations(1, cols, seed=3100)
+    xd = _x_dev(x16)
+    desc = _group_desc(pms)
+    ws = torch.zeros(n * xfp.xfp_packed_size(desc)[1], dtype=torch.uint8, device="cuda")
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    ys = torch.full((n, rows), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):      # twice: the split-K counters must come back to zero
+        xfp.xfp_gemv_grouped(desc, n, ptr([p.packed for p in pms]), ptr([xd] * n), ptr([ys[j] for j in range(n)]), False, ws)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(3200)
+    sample = np.unique(np.concatenate([rng.integers(0, rows, 48), [0, rows - 1, rows // 2]]))
+    for j in range(n):
+        got = ys[j].cpu().numpy().astype(np.float64)
+        m = to_oracle(qs[j])
+        for r in sample:
+            ref, absum = xo.gemv(m, x16, int(r), int(r) + 1)
+            assert abs(got[r] - ref[0, r]) <= TOL * absum[0, r] + 1e-30, (j, int(r))
+        single = pms[j].gemv(xd)
+        torch.cuda.synchronize()
+        _, absum_all = (None, None)
+        diff = np.abs(single[0].cpu().numpy().astype(np.float64) - got)
+        scale = np.abs(got) + np.abs(single[0].cpu().numpy()) + 1e-6
+        assert np.all(np.isfinite(got)) and np.all(diff <= 1e-3 * scale + 1e-4)
