@@ -150,3 +150,25 @@ def xfp_quantize(mode: int, W: torch.Tensor, params: XfpQuantParams, candidates:
                                _ptr(buf.ocol), _ptr(buf.oval), int(buf.capacity), _ptr(buf.cos), C.byref(res),
                                _ptr(buf.workspace), _nbytes(buf.workspace), _stream(stream)), "xfp_quantize")
     return res
+
+
+def quantize_and_pack(W: torch.Tensor, mode: int, candidates: Sequence[int], tau: float,
+                      params: Optional[XfpQuantParams] = None, lib_size: int = 32, stream=None):
+    """Float weights [rows, cols] on the device -> (PackedMatrix, XfpQuantResult): Algorithm 1 through
+    xfp_quantize, then xfp_pack, without the tensors leaving the device (allocation and marshalling only)."""
+    from .binding import PackedMatrix, xfp_pack, xfp_packed_size
+    if params is None:
+        params = XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 20, 0)      # the paper's defaults: k = 4, cap 2 %, 20 rounds
+    rows, cols = W.shape
+    frac = params.rate if params.outlier_mode else params.cap_frac
+    buf = QuantBuffers(rows, cols, mode, max(candidates), lib_size, int(frac * rows * cols), device=W.device)
+    res = xfp_quantize(mode, W, params, candidates, tau, buf, stream)
+    E = 1 << res.bits
+    desc = XfpDesc(mode, rows, cols, res.bits, 128, lib_size if mode else 0, 32, int(res.nnz))
+    pb, wb = xfp_packed_size(desc)
+    packed = torch.empty(pb, dtype=torch.uint8, device=W.device)
+    workspace = torch.zeros(max(wb, 16), dtype=torch.uint8, device=W.device)
+    err = torch.zeros(1, dtype=torch.int32, device=W.device)
+    table = (buf.lib.view(-1)[:lib_size * E] if mode else buf.codebook.view(-1)[:rows * E]).contiguous()
+    xfp_pack(desc, buf.idx, table, buf.gid, buf.gscale, buf.gmid, buf.rowptr, buf.ocol, buf.oval, packed, err, stream)
+    return PackedMatrix(desc, packed, workspace, err), res

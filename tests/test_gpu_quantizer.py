@@ -348,3 +348,22 @@ def test_full_size_layers_are_bit_exact(mode, rows, cols, bits):
     cos = torch.empty(rows, dtype=torch.float64, device="cuda")
     qb.xfp_quant_cosine(desc, Wd, maskd, idx, table, gid, gs, gm, cos)
     assert np.max(np.abs(cos.cpu().numpy() - xo.row_cosine(W, xo.dequant(ref)))) <= 1e-12
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_float_weights_to_decode_in_one_call(mode):
+    """quantize_and_pack: float weights -> packed blob on the device; y = W^ x must then be close to W x in the way
+    the cosine gate promises, and xfp_dequant of the blob must equal the oracle's reconstruction of the same matrix."""
+    rows, cols = 256, 1024
+    W = synth.plant_column_outliers(synth.gaussian_weights(rows, cols, 95), 0.01, 96)
+    pm, res = qb.quantize_and_pack(_dev(W), mode, (3, 4), 0.96)
+    ref = xo.auto_select(W, "attention", (3, 4), tau_strict=0.96, mode=mode, iters=20, lib_size=32)
+    assert res.bits == ref.bits and int(pm.err_word.item()) == 0
+    got = pm.dequant()
+    torch.cuda.synchronize()
+    assert np.array_equal(_u16(got), xo.dequant(ref))
+    x16 = synth.activations(1, cols, seed=97)
+    y = pm.gemv(torch.from_numpy(x16.view(np.int16)).cuda().view(torch.float16)).cpu().numpy().astype(np.float64)[0]
+    exact = W.astype(np.float64) @ x16.view(np.float16).astype(np.float64)[0]
+    cos = float(y @ exact / (np.linalg.norm(y) * np.linalg.norm(exact)))
+    assert cos > 0.99
