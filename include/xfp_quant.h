@@ -70,9 +70,12 @@ int xfp_quant_outliers(const float* W, int64_t n, const double* mu_sigma, int32_
  * `iters` rounds of nearest-entry cells (a tie goes to the lower entry) and cell means (an empty cell
  * keeps its entry), stopping early when nothing moves; the entries are rounded to fp16 and every
  * weight is re-assigned to its nearest STORED entry.  mask may be NULL (nothing extracted).
- *   codebook [rows][2^bits] fp16, idx [rows][cols] one index per byte.   cols <= 16384. */
+ *   codebook [rows][2^bits] fp16, idx [rows][cols] one index per byte.
+ * Channels of up to 16384 weights are sorted in shared memory and need no workspace (NULL is accepted); longer
+ * ones (up to the format's 65536) use the workspace of xfp_quant_workspace_size for their arrays. */
 int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma, int32_t rows, int32_t cols,
-                    int32_t bits, int32_t iters, uint16_t* codebook, uint8_t* idx, void* stream);
+                    int32_t bits, int32_t iters, uint16_t* codebook, uint8_t* idx, void* workspace,
+                    size_t workspace_bytes, void* stream);
 
 /* LibFit, first half: a second Lloyd pass over the per-channel codebooks.  Each codebook is normalised to
  * (c - m) / s, m and s the middle and half-width of its range; k-means with L centroids, started from L

@@ -439,23 +439,31 @@ struct SortedBulk {
     }
 };
 
+// LONG = false: one channel per CTA, its two arrays in shared memory (channels of up to 16384 weights).
+// LONG = true: the arrays live in a slice of global scratch owned by the CTA (L1/L2 resident; the CTA's own
+// writes are ordered by its barriers) and the resident CTAs walk the channels; any length the format allows.
+template <bool LONG>
 __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __restrict__ W,
                                                                const uint8_t* __restrict__ mask,
-                                                               const double* __restrict__ ms, int K, int Kp2,
+                                                               const double* __restrict__ ms, int rows, int K, int Kp2,
                                                                int bits, int iters, uint16_t* __restrict__ cb16,
-                                                               uint8_t* __restrict__ idx) {
+                                                               uint8_t* __restrict__ idx, double* scratch,
+                                                               size_t slice_doubles) {
     extern __shared__ double sm[];
-    double* pre = sm;                      // [K + 1] serial prefix sums of the sorted bulk values
-    float* r = (float*)(sm + K + 1);       // [Kp2] kept weights, ascending (extracted slots and padding = +inf)
+    double* base = LONG ? scratch + (size_t)blockIdx.x * slice_doubles : sm;
+    double* pre = base;                      // [K + 1] serial prefix sums of the sorted bulk values
+    float* r = (float*)(base + K + 1);       // [Kp2] kept weights, ascending (extracted slots and padding = +inf)
     __shared__ double c[64];
     __shared__ double e16[64];
     __shared__ int cut[65];
     __shared__ int s_m, s_p0;
     const int tid = threadIdx.x;
     const int E = 1 << bits;
-    const int64_t row0 = (int64_t)blockIdx.x * K;
     const double mu = ms[0];
 
+#pragma unroll 1
+    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    const int64_t row0 = (int64_t)row * K;
     LLOYD_STAMP(0);
     if (tid == 0) s_m = 0;
     __syncthreads();
@@ -587,7 +595,7 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
     LLOYD_STAMP(4);
     if (tid < E) {
         const uint16_t h = d2h(c[tid]);
-        cb16[(int64_t)blockIdx.x * E + tid] = h;
+        cb16[(int64_t)row * E + tid] = h;
         e16[tid] = h2d(h);
     }
     __syncthreads();
@@ -618,6 +626,9 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
         }
     }
     LLOYD_STAMP(5);
+    if (!LONG) break;  // one channel per CTA
+    __syncthreads();   // the arrays and the small tables are reused by the CTA's next channel
+    }
 }
 
 // ------------------------------------------------------------------ decoded value of a stored index
@@ -977,6 +988,13 @@ static Workspace carve(void* base, int64_t rows, int64_t cols) {
     w.order = (int*)take(sizeof(int) * (size_t)rows);
     w.asg = (int*)take(sizeof(int) * (size_t)rows);
     w.cen = (double*)take(sizeof(double) * 256 * 64);
+    if (cols > 16384) {   // channels too long for shared memory: the Lloyd kernel's arrays (it uses the scratch from its start)
+        size_t kp2 = 1;
+        while ((int64_t)kp2 < cols) kp2 <<= 1;
+        const size_t slice = (((size_t)cols + 1) + (kp2 + 1) / 2 + 1) & ~(size_t)1;
+        const size_t need = slice * sizeof(double) * (size_t)(rows < 296 ? rows : 296);
+        if (o < need) o = align256(need);
+    }
     w.bytes = o;
     return w;
 }
@@ -1083,8 +1101,13 @@ int xfp_quant_outliers(const float* W, int64_t n, const double* mu_sigma, int32_
     return cudaGetLastError() == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 
+// long channels: resident CTAs, each with a slice of scratch for its two arrays
+static const int kLloydLongCtas = 148 * 2;
+static size_t lloyd_slice_doubles(int cols, int kp2) { return (((size_t)cols + 1) + ((size_t)kp2 + 1) / 2 + 1) & ~(size_t)1; }
+
 int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma, int32_t rows, int32_t cols,
-                    int32_t bits, int32_t iters, uint16_t* codebook, uint8_t* idx, void* stream) {
+                    int32_t bits, int32_t iters, uint16_t* codebook, uint8_t* idx, void* workspace,
+                    size_t workspace_bytes, void* stream) {
     if (!W || !mu_sigma || !codebook || !idx) return XFP_ERR_NULL;
     if (!aligned16(W) || !aligned16(codebook) || !aligned16(idx) || (mask && !aligned16(mask))) return XFP_ERR_ALIGN;
     const int st = shape_status(rows, cols);
@@ -1092,12 +1115,21 @@ int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma,
     if (bits < 2 || bits > 6 || iters < 0) return XFP_ERR_SHAPE;
     int kp2;
     const int smem = lloyd_smem(cols, &kp2);
-    if (smem > 227 * 1024 - 2048) return XFP_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(lloyd_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess)
-        return XFP_ERR_CUDA;
-    lloyd_kernel<<<rows, kLloydThreads, smem, (cudaStream_t)stream>>>(W, mask, mu_sigma, cols, kp2, bits, iters,
-                                                                      codebook, idx);
+    if (smem <= 227 * 1024 - 2048) {
+        if (cudaFuncSetAttribute(lloyd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+            cudaFuncSetAttribute(lloyd_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess)
+            return XFP_ERR_CUDA;
+        lloyd_kernel<false><<<rows, kLloydThreads, smem, (cudaStream_t)stream>>>(W, mask, mu_sigma, rows, cols, kp2, bits,
+                                                                                 iters, codebook, idx, nullptr, 0);
+    } else {
+        if (!workspace) return XFP_ERR_NULL;
+        if (!aligned16(workspace)) return XFP_ERR_ALIGN;
+        const size_t slice = lloyd_slice_doubles(cols, kp2);
+        const int ctas = rows < kLloydLongCtas ? rows : kLloydLongCtas;
+        if (workspace_bytes < slice * sizeof(double) * (size_t)ctas) return XFP_ERR_BUFFER_TOO_SMALL;
+        lloyd_kernel<true><<<ctas, kLloydThreads, 0, (cudaStream_t)stream>>>(W, mask, mu_sigma, rows, cols, kp2, bits, iters,
+                                                                             codebook, idx, (double*)workspace, slice);
+    }
     return cudaGetLastError() == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 
@@ -1245,7 +1277,7 @@ int xfp_quantize(int32_t mode, const float* W, int32_t rows, int32_t cols, const
     result->fallback = 1; result->tried = 0; result->reserved = 0;
     for (int c = 0; c < n_candidates; ++c) {
         d.bits = candidates[c];
-        st = xfp_quant_lloyd(W, mask, ms, rows, cols, d.bits, p->lloyd_iters, codebook, idx, stream);
+        st = xfp_quant_lloyd(W, mask, ms, rows, cols, d.bits, p->lloyd_iters, codebook, idx, workspace, need, stream);
         if (st) return st;
         const uint16_t* table = codebook;
         if (mode == 1) {

@@ -340,7 +340,7 @@ def quant(mode, rows, cols, bits, reps=3):
     stages = [
         ("stats", lambda: qb.xfp_quant_stats(Wd, 0, ms, buf.workspace)),
         ("outliers", lambda: qb.xfp_quant_outliers(Wd, ms, 0, 4.0, 0.02, buf.mask, cnt, buf.workspace)),
-        ("lloyd", lambda: qb.xfp_quant_lloyd(Wd, buf.mask, ms, bits, 20, buf.codebook, buf.idx)),
+        ("lloyd", lambda: qb.xfp_quant_lloyd(Wd, buf.mask, ms, bits, 20, buf.codebook, buf.idx, buf.workspace)),
     ]
     if mode:
         stages += [

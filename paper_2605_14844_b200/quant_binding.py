@@ -41,7 +41,7 @@ def _lib():
         lib.xfp_quant_workspace_size.argtypes = [i32, i32, C.POINTER(sz)]
         lib.xfp_quant_stats.argtypes = [vp, i64, i32, vp, vp, sz, vp]
         lib.xfp_quant_outliers.argtypes = [vp, i64, vp, i32, f64, f64, vp, vp, vp, sz, vp]
-        lib.xfp_quant_lloyd.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp]
+        lib.xfp_quant_lloyd.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         lib.xfp_quant_libfit_library.argtypes = [vp, i32, i32, i32, i32, vp, vp, sz, vp]
         lib.xfp_quant_libfit_assign.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.xfp_quant_residual.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
@@ -78,10 +78,12 @@ def xfp_quant_outliers(W, mu_sigma, outlier_mode: int, k_or_rate: float, cap_fra
                                      _stream(stream)), "xfp_quant_outliers")
 
 
-def xfp_quant_lloyd(W, mask, mu_sigma, bits: int, iters: int, codebook, idx, stream=None) -> None:
+def xfp_quant_lloyd(W, mask, mu_sigma, bits: int, iters: int, codebook, idx, workspace=None, stream=None) -> None:
+    """workspace: needed only for channels longer than 16384 weights."""
     rows, cols = W.shape
     _check(_lib().xfp_quant_lloyd(_ptr(W), _ptr(mask), _ptr(mu_sigma), rows, cols, int(bits), int(iters),
-                                  _ptr(codebook), _ptr(idx), _stream(stream)), "xfp_quant_lloyd")
+                                  _ptr(codebook), _ptr(idx), _ptr(workspace),
+                                  0 if workspace is None else _nbytes(workspace), _stream(stream)), "xfp_quant_lloyd")
 
 
 def xfp_quant_libfit_library(codebook, rows: int, bits: int, L: int, iters: int, lib, workspace, stream=None) -> None:

@@ -58,10 +58,12 @@ def test_encoder_rejects_bad_arguments_on_the_host(lib):
     assert lib.xfp_quant_outliers(a, 100, a, 3, 4.0, 0.02, a, a, a, big, n) == 3
     assert lib.xfp_quant_outliers(a, 100, a, 1, 1.5, 0.0, a, a, a, big, n) == 3          # rate > 1
     assert lib.xfp_quant_outliers(a, 1 << 30, a, 0, 4.0, 0.02, a, a, a, 4096, n) == 5
-    assert lib.xfp_quant_lloyd(a, n, a, 64, 256, 7, 20, a, a, n) == 3
-    assert lib.xfp_quant_lloyd(a, n, a, 64, 200, 4, 20, a, a, n) == 3
-    assert lib.xfp_quant_lloyd(a, n, a, 64, 32768, 4, 20, a, a, n) == 4                   # channel too long for shared memory
-    assert lib.xfp_quant_lloyd(a, odd, a, 64, 256, 4, 20, a, a, n) == 2
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 256, 7, 20, a, a, n, 0, n) == 3
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 200, 4, 20, a, a, n, 0, n) == 3
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 32768, 4, 20, a, a, n, 0, n) == 1             # long channels need the workspace
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 32768, 4, 20, a, a, a, 4096, n) == 5
+    assert lib.xfp_quant_lloyd(a, n, a, 64, 131072, 4, 20, a, a, a, big, n) == 4          # beyond the format's 65536
+    assert lib.xfp_quant_lloyd(a, odd, a, 64, 256, 4, 20, a, a, n, 0, n) == 2
     assert lib.xfp_quant_libfit_library(a, 64, 4, 0, 20, a, a, big, n) == 3
     assert lib.xfp_quant_libfit_library(a, 64, 4, 32, 20, a, a, 64, n) == 5
     assert lib.xfp_quant_libfit_assign(a, n, a, 64, 256, 4, 32, a, a, n, a, a, n) == 1

@@ -367,3 +367,30 @@ def test_float_weights_to_decode_in_one_call(mode):
     exact = W.astype(np.float64) @ x16.view(np.float16).astype(np.float64)[0]
     cos = float(y @ exact / (np.linalg.norm(y) * np.linalg.norm(exact)))
     assert cos > 0.99
+
+
+@pytest.mark.parametrize("cols,bits,iters", [(28672, 4, 20), (16512, 3, 5), (65536, 5, 5)])
+def test_lloyd_on_channels_too_long_for_shared_memory(cols, bits, iters):
+    """Above 16384 weights per channel the sorted arrays live in global scratch; the results are the same bits."""
+    rows = 10
+    W = _weights(rows, cols, 120 + bits)
+    mask, mu, _ = xo.outlier_mask(W)
+    m = xo.quantize_v2(W, bits, mask, mu, iters)
+    cb = torch.zeros((rows, 1 << bits), dtype=torch.int16, device="cuda")
+    idx = torch.full((rows, cols), 255, dtype=torch.uint8, device="cuda")
+    qb.xfp_quant_lloyd(_dev(W), _dev(mask), _ms(mu, 0.0), bits, iters, cb, idx, _ws(rows, cols))
+    torch.cuda.synchronize()
+    assert np.array_equal(_u16(cb), m.codebook)
+    assert np.array_equal(idx.cpu().numpy(), m.idx)
+    with pytest.raises(xfp.XfpError):          # the workspace is not optional here
+        qb.xfp_quant_lloyd(_dev(W), _dev(mask), _ms(mu, 0.0), bits, iters, cb, idx, None)
+
+
+def test_auto_select_on_a_wide_matrix():
+    rows, cols = 320, 28672        # more channels than resident CTAs: every CTA walks several
+    W = synth.plant_column_outliers(synth.gaussian_weights(rows, cols, 130), 0.005, 131)
+    ref = xo.auto_select(W, "attention", (4,), tau_strict=0.9, iters=5)
+    pm, res = qb.quantize_and_pack(_dev(W), 0, (4,), 0.9, qb.XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 5, 0))
+    got = pm.dequant()
+    torch.cuda.synchronize()
+    assert int(res.nnz) == ref.nnz and np.array_equal(_u16(got), xo.dequant(ref))
