@@ -28,6 +28,10 @@
         {0, 0.5, 1, 2} % (seeded), V2 and V2a on the same draws; one token through the stack is one CUDA graph.  Prints
         milliseconds per token and effective GB/s.
 
+    python -m paper_2605_14844_b200.probe packdq MODE ROWS COLS BITS RATE
+        device time of xfp_pack (unpacked tensors -> blob) and xfp_dequant (blob -> fp16 matrix), cold L2, with
+        the bytes each must move and the resulting GB/s.
+
     python -m paper_2605_14844_b200.probe qkv [BITS]
         the dense-attention block (q, k, v, o 4096 x 4096, V2, ~0.9 % clustered outliers) as four calls and as
         one grouped launch for q, k, v (they share x) plus the call for o; microseconds per block.
@@ -266,6 +270,50 @@ def stack(layers=48, reps=5):
         torch.cuda.empty_cache()
 
 
+def packdq(mode, rows, cols, bits, rate, reps=10):
+    """Device time of xfp_pack and xfp_dequant on one matrix, with the bytes each has to move."""
+    from . import XfpDesc, xfp_dequant, xfp_pack, xfp_packed_size
+    from .binding import _dev
+    q = synth.random_quantized(mode, rows, cols, bits, rate, seed=1)
+    nnz = int(q.rowptr[-1])
+    desc = XfpDesc(q.mode, q.rows, q.cols, q.bits, q.group_size, q.lib_size if q.mode else 0, 16, nnz)
+    pb, _ = xfp_packed_size(desc)
+    dev = "cuda"
+    idx, cb = _dev(q.idx, torch.uint8, dev), _dev(q.codebook, torch.int16, dev)
+    gid = _dev(q.gid, torch.uint8, dev) if mode else None
+    gs = _dev(q.gscale, torch.int16, dev) if mode else None
+    gm = _dev(q.gmid, torch.int16, dev) if mode else None
+    rowptr = _dev(q.rowptr, torch.int32, dev)
+    ocol = _dev(q.ocol.astype(np.uint16), torch.int16, dev)
+    oval = _dev(q.oval, torch.int16, dev)
+    packed = torch.empty(pb, dtype=torch.uint8, device=dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    Wout = torch.empty((rows, cols), dtype=torch.float16, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(fn):
+        ts = []
+        for _ in range(reps + 2):
+            flush.fill_(1)     # inputs and outputs start outside L2
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts[2:]))
+
+    t_pack = timed(lambda: xfp_pack(desc, idx, cb, gid, gs, gm, rowptr, ocol, oval, packed, err))
+    t_dq = timed(lambda: xfp_dequant(desc, packed, Wout))
+    meta = algorithmic_bytes(q) - rows * cols * bits // 8
+    pack_bytes = rows * cols + rows * cols * bits // 8 + 2 * meta       # byte indices in, bit stream out, metadata in and out
+    dq_bytes = rows * cols * bits // 8 + meta + rows * cols * 2          # blob in, fp16 matrix out
+    print(json.dumps(dict(workload="pack_dequant", mode=mode, rows=rows, cols=cols, bits=bits, rate=rate, nnz=nnz,
+                          pack_us=round(t_pack, 1), pack_MB=round(pack_bytes / 1e6, 1), pack_GBs=round(pack_bytes / t_pack / 1e3, 1),
+                          dequant_us=round(t_dq, 1), dequant_MB=round(dq_bytes / 1e6, 1),
+                          dequant_GBs=round(dq_bytes / t_dq / 1e3, 1), err_word=int(err.item()))), flush=True)
+
+
 def qkv(bits=4, reps=20):
     """The attention block's q, k, v (shared x) as three calls against one grouped launch; o stays a call of its own."""
     from . import XfpDesc, xfp_gemv_grouped, xfp_packed_size
@@ -383,6 +431,9 @@ def quant(mode, rows, cols, bits, reps=3):
 
 
 def main(argv):
+    if len(argv) > 1 and argv[1] == "packdq":
+        packdq(int(argv[2]), int(argv[3]), int(argv[4]), int(argv[5]), float(argv[6]))
+        return 0
     if len(argv) > 1 and argv[1] == "qkv":
         qkv(*(int(v) for v in argv[2:3]))
         return 0
