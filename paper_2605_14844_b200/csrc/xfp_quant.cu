@@ -1075,8 +1075,9 @@ int xfp_quant_outliers(const float* W, int64_t n, const double* mu_sigma, int32_
         (outlier_mode == 1 && k_or_rate > 1.0))
         return XFP_ERR_SHAPE;
     const int64_t nblk = (n + kTieChunk - 1) / kTieChunk;
-    // the tie counters are the only part of the scratch that grows with n
-    if (workspace_bytes < carve(nullptr, 1, 128).bytes + (size_t)nblk * sizeof(int)) return XFP_ERR_BUFFER_TOO_SMALL;
+    // the tie counters are the only part of the scratch that grows with n; they start where the smallest layout puts them
+    const size_t tie_offset = (size_t)((char*)carve(nullptr, 1, 128).tie - (char*)nullptr);
+    if (workspace_bytes < tie_offset + (size_t)nblk * sizeof(int)) return XFP_ERR_BUFFER_TOO_SMALL;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(workspace, 1, 128);   // part, sel, flags, then the tie counters
     const int sweep = (int)(nblk < 148 * 8 ? (nblk < 1 ? 1 : nblk) : 148 * 8);

@@ -515,3 +515,49 @@ def test_grouped_v2_blobs_on_the_pair_kernel(bits, n, rows, cols):
         diff = np.abs(single[0].cpu().numpy().astype(np.float64) - got)
         scale = np.abs(got) + np.abs(single[0].cpu().numpy()) + 1e-6
         assert np.all(np.isfinite(got)) and np.all(diff <= 1e-3 * scale + 1e-4)
+
+
+def _random_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(count):
+        mode = int(rng.integers(0, 2))
+        bits = int(rng.integers(2, 7))
+        rows = int(rng.choice([1, 7, 31, 32, 33, 63, 64, 65, 95, 160, 257, 416, 700, 1000]))
+        cols = 128 * int(rng.choice([1, 2, 3, 5, 8, 11, 12, 13, 16, 24, 33]))
+        batch = int(rng.choice([1, 1, 1, 2, 3, 4, 7, 8, 9, 16]))
+        rate = float(rng.choice([0.0, 0.0005, 0.004, 0.02, 0.06]))
+        placement = str(rng.choice(["uniform", "clustered", "one_row"]))
+        ytype = str(rng.choice(["f32", "f16", "bf16"]))
+        xtype = str(rng.choice(["f16", "f16", "bf16"]))
+        cases.append((i, mode, bits, rows, cols, batch, rate, placement, xtype, ytype))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(72, 4242), ids=lambda c: "-".join(str(v) for v in c))
+def test_randomized_shapes_types_and_outlier_structure(case):
+    """A seeded sweep over everything the dispatcher keys on at once: mode, bit width, ragged channel counts
+    (1 ... 1000), K from one to 33 super-chunks, batch 1..16, outlier rate and placement (including all outliers in one
+    channel), activation and output types."""
+    i, mode, bits, rows, cols, batch, rate, placement, xtype, ytype = case
+    q = synth.random_quantized(mode, rows, cols, bits, rate, seed=5000 + i, placement=placement)
+    pm = xfp.pack_tensors(q, col_bits=16 if i % 2 else 32)
+    _check_dequant(q, pm)
+    m = to_oracle(q)
+    if xtype == "bf16":
+        xd, x64 = _bf16_x(batch, cols, 6000 + i)
+    else:
+        x16 = synth.activations(batch, cols, seed=6000 + i)
+        xd, x64 = _x_dev(x16), x16.view(np.float16).astype(np.float64)
+    ref, absum = xo.gemv_x64(m, x64)
+    dt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[ytype]
+    ulp = {"f32": 0.0, "f16": 2.0 ** -11, "bf16": 2.0 ** -8}[ytype]
+    y = torch.full((batch, rows), float("nan"), dtype=dt, device="cuda")
+    for _ in range(2):
+        xfp.xfp_gemv_typed(pm.desc, pm.packed, xd, batch, y, pm.workspace)
+    torch.cuda.synchronize()
+    got = y.to(torch.float64).cpu().numpy()
+    tiny = 2.0 ** -25 * np.abs(xo.dequant(m).view(np.float16).astype(np.float64)).sum(1)[None, :] if xtype == "bf16" else 0.0
+    tol = TOL * absum + tiny + ulp * np.abs(ref) + 1e-30
+    assert np.all(np.isfinite(got))
+    assert np.all(np.abs(got - ref) <= tol), float((np.abs(got - ref) / tol).max())

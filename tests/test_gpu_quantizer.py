@@ -394,3 +394,49 @@ def test_auto_select_on_a_wide_matrix():
     got = pm.dequant()
     torch.cuda.synchronize()
     assert int(res.nnz) == ref.nnz and np.array_equal(_u16(got), xo.dequant(ref))
+
+
+def _random_encoder_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(count):
+        out.append((i, int(rng.integers(0, 2)), int(rng.choice([1, 5, 33, 64, 130, 300])), 128 * int(rng.choice([1, 2, 3, 7, 12, 20])),
+                    tuple(sorted(set(int(b) for b in rng.integers(2, 7, size=int(rng.integers(1, 4)))))),
+                    float(rng.choice([0.5, 0.93, 0.96, 0.99, 0.9999])), int(rng.choice([0, 1, 5, 20])),
+                    int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.choice([1, 5, 32, 40]))))
+    return out
+
+
+@pytest.mark.parametrize("case", _random_encoder_cases(36, 777), ids=lambda c: "-".join(str(v) for v in c))
+def test_randomized_auto_select(case):
+    """A seeded sweep of Algorithm 1 end to end against the oracle: mode, ragged channel counts, channel lengths,
+    candidate lists, floors that pass early, late or never, 0..20 Lloyd rounds, both sigma modes, both extraction
+    modes, library sizes including ones larger than the channel count."""
+    i, mode, rows, cols, cands, tau, iters, sigma_mode, outlier_mode, L = case
+    W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, 8000 + i), 0.01, 8100 + i)
+    rate = 0.004 if outlier_mode else None
+    ref = xo.auto_select(W, "attention", cands, tau_strict=tau, mode=mode, k=3.0, cap=0.01,
+                         sigma_mode="robust" if sigma_mode else "matrix", rate=rate, iters=iters, lib_size=L)
+    params = qb.XfpQuantParams(sigma_mode, outlier_mode, 3.0, 0.01, 0.004, iters, 0)
+    buf = qb.QuantBuffers(rows, cols, mode, max(cands), L, int(0.02 * W.size) + 8)
+    res = qb.xfp_quantize(mode, _dev(W), params, cands, tau, buf)
+    torch.cuda.synchronize()
+    assert (res.bits, bool(res.fallback), res.tried) == (ref.bits, ref.info["fallback"], len(ref.info["tried"]))
+    E, nnz = 1 << res.bits, int(res.nnz)
+    assert nnz == ref.nnz and np.array_equal(buf.mask.cpu().numpy(), _oracle_mask(W, ref))
+    assert np.array_equal(buf.idx.cpu().numpy(), ref.idx)
+    table = buf.lib.view(-1)[:L * E].view(L, E) if mode else buf.codebook.view(-1)[:rows * E].view(rows, E)
+    assert np.array_equal(_u16(table), ref.codebook)
+    if mode:
+        assert np.array_equal(buf.gid.cpu().numpy(), ref.gid)
+        assert np.array_equal(_u16(buf.gscale), ref.gscale) and np.array_equal(_u16(buf.gmid), ref.gmid)
+    assert np.array_equal(buf.rowptr.cpu().numpy(), ref.rowptr)
+    assert np.array_equal(buf.ocol[:nnz].cpu().numpy(), ref.ocol) and np.array_equal(_u16(buf.oval[:nnz]), ref.oval)
+    assert abs(res.median_cos - ref.info["median_cos"]) <= 1e-12
+
+
+def _oracle_mask(W, ref):
+    m = np.zeros(W.shape, dtype=np.uint8)
+    for r in range(ref.rows):
+        m[r, ref.ocol[ref.rowptr[r]:ref.rowptr[r + 1]]] = 1
+    return m
