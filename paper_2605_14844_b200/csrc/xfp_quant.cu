@@ -33,6 +33,34 @@ __device__ __forceinline__ uint16_t v2a_value16(uint16_t scale, uint16_t lib, ui
     return __half_as_ushort(__float2half_rn(r));
 }
 
+// Index of the entry nearest to x among e[0..E), ties to the lower index: the answer of a linear scan that keeps an
+// entry only when it is strictly nearer.  When the entries ascend (codebooks and decoded library entries do) x is
+// bracketed by bisection and only its two neighbours are measured; the scan's answer is the nearer of the two
+// (the lower on an exact tie: fp64 rounding is monotone and distinct fp16 values are too far apart to round to
+// the same distance), moved down over duplicates of its value.
+__device__ __forceinline__ int nearest_entry(const double* e, int E, double x, bool ascending) {
+    if (!ascending) {
+        int best = 0;
+        double bd = fabs(__dsub_rn(x, e[0]));
+        for (int j = 1; j < E; ++j) {
+            const double d = fabs(__dsub_rn(x, e[j]));
+            if (d < bd) { bd = d; best = j; }
+        }
+        return best;
+    }
+    int lo = 0, hi = E;   // first index whose entry is >= x
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (e[mid] < x) lo = mid + 1; else hi = mid;
+    }
+    int best;
+    if (lo == 0) best = 0;
+    else if (lo == E) best = E - 1;
+    else best = fabs(__dsub_rn(x, e[lo - 1])) <= fabs(__dsub_rn(x, e[lo])) ? lo - 1 : lo;
+    while (best > 0 && e[best - 1] == e[best]) --best;
+    return best;
+}
+
 // Sum over the block in a fixed tree order; every thread gets the result.
 __device__ double block_sum(double v, double* sh) {
     sh[threadIdx.x] = v;
@@ -599,30 +627,20 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
         e16[tid] = h2d(h);
     }
     __syncthreads();
-    // every weight goes to the nearest STORED entry (ties: lower index); four weights per thread at a time,
-    // so that four chains of compares are in flight
+    // every weight goes to the nearest STORED entry (ties: lower index)
+    bool e_asc = true;
+    for (int j = 1; j < E; ++j) e_asc = e_asc && e16[j] >= e16[j - 1];
     for (int kb = tid; kb < K; kb += 4 * kLloydThreads) {
-        double v[4], bd[4];
-        int best[4];
+        double v[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int k = kb + e * kLloydThreads;
             v[e] = k < K ? bulk_value(W, mask, row0 + k, mu) : 0.0;
-            bd[e] = fabs(__dsub_rn(v[e], e16[0]));
-            best[e] = 0;
-        }
-        for (int j = 1; j < E; ++j) {
-            const double ej = e16[j];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const double d = fabs(__dsub_rn(v[e], ej));
-                if (d < bd[e]) { bd[e] = d; best[e] = j; }
-            }
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int k = kb + e * kLloydThreads;
-            if (k < K) idx[row0 + k] = (uint8_t)best[e];
+            if (k < K) idx[row0 + k] = (uint8_t)nearest_entry(e16, E, v[e], e_asc);
         }
     }
     LLOYD_STAMP(5);
@@ -899,18 +917,21 @@ __global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restri
             const uint16_t mid16 = s_mid[s], sc16 = s_sc[s];
             for (int l = tid % lw; l < L; l += lw) {
                 double d16[64];
-                for (int j = 0; j < E; ++j) d16[j] = h2d(v2a_value16(sc16, lib[l * E + j], mid16));
+                bool asc = true;
+                for (int j = 0; j < E; ++j) {
+                    d16[j] = h2d(v2a_value16(sc16, lib[l * E + j], mid16));
+                    if (j && d16[j] < d16[j - 1]) asc = false;
+                }
                 double acc = 0.0;
-                for (int t = 0; t < GS; ++t) {
-                    const double x = gv[s][t];
-                    double bd = fabs(__dsub_rn(x, d16[0]));
-                    int bj = 0;
-                    for (int j = 1; j < E; ++j) {
-                        const double d = fabs(__dsub_rn(x, d16[j]));
-                        if (d < bd) { bd = d; bj = j; }
+                for (int t = 0; t < GS; t += 4) {   // four searches in flight, the sum stays in value order
+                    double d[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const double x = gv[s][t + e];
+                        d[e] = __dsub_rn(x, d16[nearest_entry(d16, E, x, asc)]);
                     }
-                    const double d = __dsub_rn(x, d16[bj]);
-                    acc = __dadd_rn(acc, __dmul_rn(d, d));
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc = __dadd_rn(acc, __dmul_rn(d[e], d[e]));
                 }
                 sse[gpb == 1 ? l : s * lw + l] = acc;
             }
@@ -943,12 +964,9 @@ __global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restri
         if (grp >= groups) break;
         int bj = 0;
         if (!s_const[s]) {
-            const double v = gv[s][tid];
-            double bd = fabs(__dsub_rn(v, dec[s][0]));
-            for (int j = 1; j < E; ++j) {
-                const double d = fabs(__dsub_rn(v, dec[s][j]));
-                if (d < bd) { bd = d; bj = j; }
-            }
+            bool asc = true;
+            for (int j = 1; j < E; ++j) asc = asc && dec[s][j] >= dec[s][j - 1];
+            bj = nearest_entry(dec[s], E, gv[s][tid], asc);
         }
         idx[grp * GS + tid] = (uint8_t)bj;
     }
