@@ -348,12 +348,13 @@ bool batch_supported(const Layout& l, int batch) { return batch > 2 && batch_til
 
 template <int N, int NB, int RPL, bool TIO>
 static cudaError_t launch_batch_io(const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce attr_done;
+    const int dev = DeviceOnce::current();
+    if (!attr_done.is_set(dev)) {
         cudaError_t e = cudaFuncSetAttribute(gemv_batch_kernel<N, NB, RPL, TIO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              224 * 1024);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.set(dev);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;

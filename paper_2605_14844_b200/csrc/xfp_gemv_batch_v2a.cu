@@ -358,12 +358,13 @@ bool batch_v2a_supported(const Layout& l, int batch) { return batch > 2 && batch
 
 template <int N, int NB, bool TIO>
 static cudaError_t launch_batch_v2a_io(const BatchV2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce attr_done;
+    const int dev = DeviceOnce::current();
+    if (!attr_done.is_set(dev)) {
         cudaError_t e = cudaFuncSetAttribute(gemv_batch_v2a_kernel<N, NB, TIO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              224 * 1024);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.set(dev);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;

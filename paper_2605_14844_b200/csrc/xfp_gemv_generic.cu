@@ -307,12 +307,13 @@ size_t generic_workspace_bytes(const Layout& l) {
 
 template <int N, int MODE, int BT>
 static cudaError_t launch_one(const GenericArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce attr_done;
+    const int dev = DeviceOnce::current();
+    if (!attr_done.is_set(dev)) {
         cudaError_t e = cudaFuncSetAttribute(gemv_generic_kernel<N, MODE, BT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.set(dev);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;

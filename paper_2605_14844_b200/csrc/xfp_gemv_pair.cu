@@ -627,12 +627,13 @@ size_t pair_workspace_bytes(const Layout& l) {
 
 template <int N, int NB, int RPL, int W, bool TIO>
 static cudaError_t launch_pair_io(const PairArgs& a, int grid, size_t smem, cudaStream_t s) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce attr_done;
+    const int dev = DeviceOnce::current();
+    if (!attr_done.is_set(dev)) {
         cudaError_t e = cudaFuncSetAttribute(gemv_pair_kernel<N, NB, RPL, W, TIO>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.set(dev);
     }
     const int cluster = a.cluster ? a.tier_kst[0] : 1;
     cudaLaunchConfig_t cfg = {};

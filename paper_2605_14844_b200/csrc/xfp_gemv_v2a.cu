@@ -556,12 +556,13 @@ size_t v2a_workspace_bytes(const Layout& l) {
 
 template <int N, int NB, int W, bool PAIR, bool FEAT>
 static cudaError_t launch_v2a_feat(const V2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce attr_done;
+    const int dev = DeviceOnce::current();
+    if (!attr_done.is_set(dev)) {
         cudaError_t e = cudaFuncSetAttribute(gemv_v2a_kernel<N, NB, W, PAIR, FEAT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              W == 8 ? 112 * 1024 : 226 * 1024);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.set(dev);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;

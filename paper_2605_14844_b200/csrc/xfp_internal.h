@@ -7,6 +7,19 @@
 
 namespace xfp {
 
+// Function attributes (the opt-in shared-memory size) belong to a device: every kernel instantiation remembers
+// on which devices it has set them, so a process that drives several GPUs sets them on each.
+struct DeviceOnce {
+    unsigned long long mask[4] = {0, 0, 0, 0};   // devices 0..255
+    static int current() {
+        int d = 0;
+        cudaGetDevice(&d);
+        return d & 255;
+    }
+    bool is_set(int d) const { return (mask[d >> 6] >> (d & 63)) & 1ull; }
+    void set(int d) { mask[d >> 6] |= 1ull << (d & 63); }
+};
+
 struct PackInputs {
     const uint8_t* idx;
     const uint16_t* codebook;
