@@ -528,11 +528,16 @@ static size_t v2a_smem_bytes(const Layout& l, int nb, bool pair, int warps) {
            (size_t)l.L * l.E * 2 + 16;   // + the copy of the library the tables were built from, 16-byte aligned
 }
 
-static int g_v2a_pair = 1;   // probe switch: 0 keeps every layout on the per-bank library
+static int g_v2a_pair = 1;   // probe switch: 0 keeps every layout on the per-bank library, 2 forces pair tables where they fit
 void v2a_set_pair(int v) { g_v2a_pair = v; }
 
-static V2aConfig v2a_config(const Layout& l, int nb) {
-    if (g_v2a_pair && l.bits <= 3) {
+static V2aConfig v2a_config(const Layout& l, int nb, int n = 1) {
+    // Pair tables cost 128 KB of fills per resident CTA and run one CTA of 12 or 16 warps per SM: they pay off
+    // when every SM has a few hundred thousand weights to decode and K is long enough to keep those warps busy
+    // (measured: 28672 x 8192 53 vs 61 us, 8192 x 8192 18.6 vs 22.9, 12288 x 4096 18.7 vs 20.0 in their favour;
+    // 4096 x 4096 10.4 vs 9.1 and the routed experts' 4096 x 1536 down projections 20.6 vs 18.7 against them).
+    const bool big = (long long)l.rows * l.cols * n >= 40ll * 1000 * 1000 && l.SC >= 32;
+    if (g_v2a_pair && l.bits <= 3 && (big || g_v2a_pair == 2)) {
         // K is shared by the warps in super-chunks: 12 warps when that divides the count and 16 does not
         const int warps = (l.SC % 16 != 0 && l.SC % 12 == 0) ? 12 : 16;
         const size_t sm = v2a_smem_bytes(l, nb, true, warps);
@@ -593,7 +598,7 @@ static cudaError_t launch_v2a_cfg(const V2aConfig& cfg, const V2aArgs& a, dim3 g
 }
 
 cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) {
-    const V2aConfig cfg = v2a_config(l, c.batch);
+    const V2aConfig cfg = v2a_config(l, c.batch, c.n);
     V2aArgs a{};
     a.off = offsets_of(l);
     a.packed = c.packed; a.x = c.x; a.y = c.y;
