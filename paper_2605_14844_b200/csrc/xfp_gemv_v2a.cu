@@ -59,6 +59,7 @@ struct V2aArgs {
     int epi;                 // 0 plain store; 1 SiLU(gate) * up inside every 64-channel block; 2 weighted sum over the blobs
     const float* epi_w;      // epi 2: [n] weights
     int comb_G, comb_ng;     // epi 2: runs per block of channels, blobs per run
+    int persist;             // per-bank library: resident CTAs walk the items
 };
 
 __device__ __forceinline__ void mma16816a(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -509,10 +510,10 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
             }
         }
     }
-    if (!PAIR) break;   // the per-bank library is launched with one CTA per item
+    if (!PAIR && !a.persist) break;   // the per-bank library is launched with one CTA per item
     __syncthreads();   // red, x and the ticket flag are reused by the CTA's next item
     }
-    if (!PAIR) break;
+    if (!PAIR && !a.persist) break;
     }
 }
 
@@ -658,7 +659,10 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
         items = (long long)a.blocks * a.comb_G;
     }
     // pair tables are expensive to build: resident CTAs walk the items; the per-bank library launches one CTA per item
-    dim3 grid((unsigned)(cfg.pair ? (items < cfg.slots ? items : cfg.slots) : items), 1, 1);
+    // several blobs on the per-bank library with more items than CTA slots: resident CTAs walk the items, so the
+    // tables are not rebuilt for the later rounds (routed experts' down projections: 1 % per token-layer)
+    a.persist = (!cfg.pair && c.n > 1 && items > cfg.slots) ? 1 : 0;
+    dim3 grid((unsigned)((cfg.pair || a.persist) ? (items < cfg.slots ? items : cfg.slots) : items), 1, 1);
     switch (l.bits * 10 + c.batch) {
         case 21: return launch_v2a_cfg<2, 1>(cfg, a, grid, s);
         case 22: return launch_v2a_cfg<2, 2>(cfg, a, grid, s);
