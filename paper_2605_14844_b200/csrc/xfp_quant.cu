@@ -454,6 +454,28 @@ __device__ __forceinline__ double bulk_value(const float* __restrict__ W, const 
     return (mask != nullptr && mask[t]) ? mu : (double)W[t];
 }
 
+// Compare-exchange of the bitonic network: after it a <= b when `asc`, a >= b otherwise; equal keys stay put.
+__device__ __forceinline__ void cswap(float& a, float& b, bool asc) {
+    const bool sw = (a > b) == asc;
+    const float x = sw ? b : a, y = sw ? a : b;
+    a = x;
+    b = y;
+}
+// the stages with partner distance 4, 2, 1 on eight consecutive elements
+__device__ __forceinline__ void last3(float (&v)[8], bool asc) {
+    cswap(v[0], v[4], asc); cswap(v[1], v[5], asc); cswap(v[2], v[6], asc); cswap(v[3], v[7], asc);
+    cswap(v[0], v[2], asc); cswap(v[1], v[3], asc); cswap(v[4], v[6], asc); cswap(v[5], v[7], asc);
+    cswap(v[0], v[1], asc); cswap(v[2], v[3], asc); cswap(v[4], v[5], asc); cswap(v[6], v[7], asc);
+}
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+    const float4 a = *(const float4*)p, b = *(const float4*)(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
+    *(float4*)p = make_float4(v[0], v[1], v[2], v[3]);
+    *(float4*)(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+
 // The channel's bulk values in ascending order without storing them as doubles: the weights that were not
 // extracted, sorted as floats, with the m copies of mu (one per extracted position) inserted at p0.
 struct SortedBulk {
@@ -477,10 +499,10 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
                                                                int bits, int iters, uint16_t* __restrict__ cb16,
                                                                uint8_t* __restrict__ idx, double* scratch,
                                                                size_t slice_doubles) {
-    extern __shared__ double sm[];
+    extern __shared__ __align__(16) double sm[];
     double* base = LONG ? scratch + (size_t)blockIdx.x * slice_doubles : sm;
     double* pre = base;                      // [K + 1] serial prefix sums of the sorted bulk values
-    float* r = (float*)(base + K + 1);       // [Kp2] kept weights, ascending (extracted slots and padding = +inf)
+    float* r = (float*)(base + ((K + 2) & ~1));   // [Kp2] kept weights, ascending (extracted slots and padding = +inf); 16-byte aligned
     __shared__ double c[64];
     __shared__ double e16[64];
     __shared__ int cut[65];
@@ -515,10 +537,22 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
     if (extracted) atomicAdd(&s_m, extracted);
     __syncthreads();
     LLOYD_STAMP(1);
-    // bitonic sort, ascending; a thread's eight pairs of a stage are loaded before any is written back
-    const int half = Kp2 >> 1;
-    for (int size = 2; size <= Kp2; size <<= 1) {
-        for (int j = size >> 1; j > 0; j >>= 1) {
+    // bitonic sort, ascending.  The stages with partner distance 4, 2, 1 stay inside blocks of 8 consecutive
+    // elements and run in registers (one pass per step instead of three trips through the array); the wider
+    // stages go through the array, a thread's eight pairs loaded before any is written back.
+    const int half = Kp2 >> 1, nblk8 = Kp2 >> 3;
+    for (int b8 = tid; b8 < nblk8; b8 += kLloydThreads) {   // steps 2, 4 and 8 entirely in registers
+        float v[8];
+        load8(r + 8 * b8, v);
+        cswap(v[0], v[1], true); cswap(v[2], v[3], false); cswap(v[4], v[5], true); cswap(v[6], v[7], false);
+        cswap(v[0], v[2], true); cswap(v[1], v[3], true); cswap(v[4], v[6], false); cswap(v[5], v[7], false);
+        cswap(v[0], v[1], true); cswap(v[2], v[3], true); cswap(v[4], v[5], false); cswap(v[6], v[7], false);
+        last3(v, ((8 * b8) & 8) == 0);
+        store8(r + 8 * b8, v);
+    }
+    __syncthreads();
+    for (int size = 16; size <= Kp2; size <<= 1) {
+        for (int j = size >> 1; j >= 8; j >>= 1) {
             for (int pb = tid; pb < half; pb += 8 * kLloydThreads) {
                 int ia[8];
                 float a[8], b[8];
@@ -534,6 +568,13 @@ __global__ void __launch_bounds__(kLloydThreads, 4) lloyd_kernel(const float* __
             }
             __syncthreads();
         }
+        for (int b8 = tid; b8 < nblk8; b8 += kLloydThreads) {
+            float v[8];
+            load8(r + 8 * b8, v);
+            last3(v, ((8 * b8) & size) == 0);
+            store8(r + 8 * b8, v);
+        }
+        __syncthreads();
     }
     LLOYD_STAMP(2);
     if (tid == 0) {   // where mu sits among the kept weights
@@ -1009,7 +1050,7 @@ static Workspace carve(void* base, int64_t rows, int64_t cols) {
     if (cols > 16384) {   // channels too long for shared memory: the Lloyd kernel's arrays (it uses the scratch from its start)
         size_t kp2 = 1;
         while ((int64_t)kp2 < cols) kp2 <<= 1;
-        const size_t slice = (((size_t)cols + 1) + (kp2 + 1) / 2 + 1) & ~(size_t)1;
+        const size_t slice = (((size_t)cols + 2) & ~(size_t)1) + kp2 / 2;
         const size_t need = slice * sizeof(double) * (size_t)(rows < 296 ? rows : 296);
         if (o < need) o = align256(need);
     }
@@ -1029,7 +1070,7 @@ static int lloyd_smem(int cols, int* kp2_out) {
     int kp2 = 1;
     while (kp2 < cols) kp2 <<= 1;
     *kp2_out = kp2;
-    return (int)(sizeof(double) * ((size_t)cols + 1) + sizeof(float) * (size_t)kp2);
+    return (int)(sizeof(double) * (((size_t)cols + 2) & ~(size_t)1) + sizeof(float) * (size_t)kp2);
 }
 
 static Unpacked unpacked_of(const xfp_desc* d, const uint8_t* idx, const uint16_t* cb, const uint8_t* gid,
@@ -1122,7 +1163,7 @@ int xfp_quant_outliers(const float* W, int64_t n, const double* mu_sigma, int32_
 
 // long channels: resident CTAs, each with a slice of scratch for its two arrays
 static const int kLloydLongCtas = 148 * 2;
-static size_t lloyd_slice_doubles(int cols, int kp2) { return (((size_t)cols + 1) + ((size_t)kp2 + 1) / 2 + 1) & ~(size_t)1; }
+static size_t lloyd_slice_doubles(int cols, int kp2) { return (((size_t)cols + 2) & ~(size_t)1) + (size_t)kp2 / 2; }
 
 int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma, int32_t rows, int32_t cols,
                     int32_t bits, int32_t iters, uint16_t* codebook, uint8_t* idx, void* workspace,
