@@ -1,6 +1,7 @@
 // xfp_pack: unpacked tensors -> device layout (with range validation and clamping);
 // xfp_dequant: device layout -> fp16 matrix W^ = fp16(D16 + S), bit-exact.
 #include "xfp_internal.h"
+#include "xfp_pair_common.cuh"
 
 namespace xfp {
 
@@ -237,6 +238,77 @@ __global__ void __launch_bounds__(128) dequant_kernel(Blob b, uint16_t* __restri
     }
 }
 
+// The same for V2 blobs with the codebooks in shared memory.  The kernel above looks every weight up in global
+// memory, one 2-byte load per lane with 32 distinct sectors per request, and that is what it is bound by (ncu: 49 M
+// LSU wavefronts, the pipe 98 % busy, 183 us at 28672 x 8192).  Here a CTA of 8 warps takes one row-block and a
+// range of super-chunks and stages the block's codebooks once, one word per lane and entry so that every look-up is
+// conflict free: up to N = 3 as tables indexed by a PAIR of indices (one look-up yields the two fp16 values of a
+// 4-byte tile store), above as one entry per index.  (A V2a variant with the library replicated per bank measured
+// slower than the kernel above -- 64 KB of table fill per CTA, one CTA per SM -- and is not kept.)
+template <int N>
+__global__ void __launch_bounds__(256) dequant_lut_kernel(Blob b, uint16_t* __restrict__ W, int rows, int cols, int RB,
+                                                          int SC, int sc_per_cta) {
+    constexpr int E = 1 << N;
+    constexpr bool kPair = N <= 3;   // at N = 4 the 32 KB pair table costs a CTA per SM: slower than one entry per index
+    constexpr int T = kPair ? E * E : E;
+    constexpr int kWarps = 8;
+    constexpr int kStrideW = 65;   // words per tile row: 32 lanes hit 32 banks
+    extern __shared__ __align__(16) uint32_t dq_smem[];
+    uint32_t* tab = dq_smem;                                        // [T][32]
+    uint32_t* tiles = dq_smem + T * 32;                             // [kWarps][32 * kStrideW]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int rb = blockIdx.x % RB, part = blockIdx.x / RB;
+    const int sc_begin = part * sc_per_cta;
+    const int sc_end = min(SC, sc_begin + sc_per_cta);
+    {
+        // the lane's codebook goes through the first tile (one word per entry), the pair table is built from there
+        const uint16_t* cb = b.cb + (size_t)(rb * kRowsPerBlock + lane) * E;   // padding rows exist in the blob
+        uint32_t* one = kPair ? tiles : tab;
+        for (int e = warp; e < E; e += kWarps) one[e * 32 + lane] = __ldg(cb + e);
+        if (kPair) {
+            __syncthreads();
+            for (int t = warp; t < T; t += kWarps)
+                tab[t * 32 + lane] = one[(t & (E - 1)) * 32 + lane] | (one[(t >> N) * 32 + lane] << 16);
+        }
+    }
+    __syncthreads();
+    const uint32_t base = (uint32_t)lane * 4u;
+    uint32_t* tile = tiles + warp * 32 * kStrideW;
+    for (int sc = sc_begin + warp; sc < sc_end; sc += kWarps) {
+        const size_t unit = (size_t)rb * SC + sc;
+        uint32_t w[4 * N + 1];
+        const uint4* src = b.idx + (unit * N) * 32 + lane;
+#pragma unroll
+        for (int v = 0; v < N; ++v) {
+            const uint4 t = ld_stream(src + (size_t)v * 32);
+            w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
+        }
+        w[4 * N] = 0u;
+        uint32_t* trow = tile + lane * kStrideW;
+#pragma unroll
+        for (int p = 0; p < kSuper / 2; ++p) {
+            if (kPair) {
+                trow[p] = *(const uint32_t*)((const unsigned char*)tab + pair_addr<N, 1>(w, p, base));
+            } else {
+                const uint32_t lo = *(const uint32_t*)((const unsigned char*)tab + single_addr<N, 1>(w, 2 * p, base));
+                const uint32_t hi = *(const uint32_t*)((const unsigned char*)tab + single_addr<N, 1>(w, 2 * p + 1, base));
+                trow[p] = lo | (hi << 16);
+            }
+        }
+        __syncwarp();
+#pragma unroll 4
+        for (int r = 0; r < 32; ++r) {
+            const int orow = rb * kRowsPerBlock + r;
+            if (orow >= rows) break;
+            const uint32_t* srow = tile + r * kStrideW;
+            uint32_t* drow = (uint32_t*)(W + (size_t)orow * cols + (size_t)sc * kSuper);
+            drow[lane] = srow[lane];
+            drow[lane + 32] = srow[lane + 32];
+        }
+        __syncwarp();   // the tile is rewritten for the warp's next super-chunk
+    }
+}
+
 // W^ += S at the outlier positions: one correctly rounded fp16 addition per outlier.
 __global__ void dequant_outlier_kernel(Blob b, uint16_t* __restrict__ W, int rows, int cols) {
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -252,7 +324,28 @@ __global__ void dequant_outlier_kernel(Blob b, uint16_t* __restrict__ W, int row
 }
 
 template <int N>
+static bool launch_dequant_lut(const Layout& l, const Blob& b, uint16_t* W, cudaStream_t s) {
+    const size_t tab_bytes = (size_t)(N <= 3 ? l.E * l.E : l.E) * 128;
+    const size_t smem = tab_bytes + (size_t)8 * 32 * 65 * 4;
+    static DeviceOnce attr_done;
+    const int dev = DeviceOnce::current();
+    if (!attr_done.is_set(dev)) {
+        if (cudaFuncSetAttribute(dequant_lut_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) != cudaSuccess)
+            return false;
+        attr_done.set(dev);
+    }
+    // a CTA per row-block; row-blocks too few to fill the GPU are cut along K (at least 8 super-chunks per CTA)
+    int parts = 1;
+    while (l.RB * parts < 2 * 148 && l.SC / (parts * 2) >= 8) parts *= 2;
+    const int sc_per_cta = (l.SC + parts - 1) / parts;
+    parts = (l.SC + sc_per_cta - 1) / sc_per_cta;
+    dequant_lut_kernel<N><<<(unsigned)(l.RB * parts), 256, smem, s>>>(b, W, l.rows, l.cols, l.RB, l.SC, sc_per_cta);
+    return true;
+}
+
+template <int N>
 static void launch_dequant_n(const Layout& l, const Blob& b, uint16_t* W, cudaStream_t s) {
+    if (l.mode == 0 && launch_dequant_lut<N>(l, b, W, s)) return;
     const long long units = (long long)l.RB * l.SC;
     const unsigned grid = (unsigned)((units + 3) / 4);
     if (l.mode == 0)
