@@ -7,6 +7,7 @@ whose summation order is the kernel's own (matrix statistics, per-channel cosine
 relative; to keep the later stages' inputs identical the tests hand the oracle's (mu, sigma) to both sides.
 """
 import ctypes as C
+import os
 
 import numpy as np
 import pytest
@@ -407,7 +408,8 @@ def _random_encoder_cases(count, seed):
     return out
 
 
-@pytest.mark.parametrize("case", _random_encoder_cases(36, 777), ids=lambda c: "-".join(str(v) for v in c))
+@pytest.mark.parametrize("case", _random_encoder_cases(int(os.environ.get("XFP_SWEEP_CASES", "72")) // 2, 777 + int(os.environ.get("XFP_SWEEP_SEED", "0"))),
+                         ids=lambda c: "-".join(str(v) for v in c))
 def test_randomized_auto_select(case):
     """A seeded sweep of Algorithm 1 end to end against the oracle: mode, ragged channel counts, channel lengths,
     candidate lists, floors that pass early, late or never, 0..20 Lloyd rounds, both sigma modes, both extraction
