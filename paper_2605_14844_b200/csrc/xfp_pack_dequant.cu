@@ -121,18 +121,18 @@ __global__ void pack_entries_kernel(const void* __restrict__ ocol, int col_bits,
     out[p] = (uint32_t)c | (v << 16);
 }
 
-// Transposed outlier slab of row-block b (one warp per block): word [0][lane] = slots used by channel
-// b*32+lane, word [1+j][lane] = its j-th outlier or the neutral entry (column 0, value +0).
-__global__ void ell_fill_kernel(const int* __restrict__ rp, const uint32_t* __restrict__ oent,
-                                uint32_t* __restrict__ ell, int RB, int C) {
-    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
+// Transposed outlier slab of row-block b (one CTA of 8 warps per block, the slots dealt to the warps): word [0][lane]
+// = slots used by channel b*32+lane, word [1+j][lane] = its j-th outlier or the neutral entry (column 0, value +0).
+__global__ void __launch_bounds__(256) ell_fill_kernel(const int* __restrict__ rp, const uint32_t* __restrict__ oent,
+                                                       uint32_t* __restrict__ ell, int RB, int C) {
+    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (b >= RB) return;
     const int p0 = rp[b * 32 + lane], p1 = rp[b * 32 + lane + 1];
     const int len = p1 > p0 ? min(p1 - p0, C) : 0;
     uint32_t* slab = ell + (size_t)b * (C + 1) * 32 + lane;
-    slab[0] = (uint32_t)len;
-    for (int j = 0; j < C; ++j) slab[(size_t)(1 + j) * 32] = j < len ? oent[p0 + j] : 0u;
+    if (warp == 0) slab[0] = (uint32_t)len;
+    for (int j = warp; j < C; j += 8) slab[(size_t)(1 + j) * 32] = j < len ? oent[p0 + j] : 0u;
 }
 
 __global__ void pack_header_kernel(int* hdr, int ell_slots, long long off_ell) {
@@ -179,7 +179,7 @@ cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int
         pack_entries_kernel<<<(unsigned)((l.nnz + 255) / 256), 256, 0, s>>>(in.ocol, in.col_bits, in.oval,
                                                                            (uint32_t*)(base + l.off_oent), l.nnz,
                                                                            l.cols, err_word);
-        ell_fill_kernel<<<(unsigned)((l.RB + 7) / 8), 256, 0, s>>>((const int*)(base + l.off_rowptr),
+        ell_fill_kernel<<<(unsigned)l.RB, 256, 0, s>>>((const int*)(base + l.off_rowptr),
                                                                    (const uint32_t*)(base + l.off_oent),
                                                                    (uint32_t*)(base + l.off_ell), l.RB, l.ell_slots);
     }
