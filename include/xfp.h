@@ -142,6 +142,14 @@ int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const
                               void* const* y, int32_t y_is_fp16, int32_t epilogue, const float* weights,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* The grouped launch with typed activations and outputs (x_type, y_type as for xfp_gemv_typed) and an optional fused
+ * store (epilogue, weights as for xfp_gemv_grouped_epilogue; XFP_EPI_NONE for none): a routed expert block of a
+ * bf16 model in two launches.  Fused stores and grouped V2 blobs run on the kernels that carry typed IO; the same
+ * restrictions as xfp_gemv_grouped_epilogue apply when epilogue != XFP_EPI_NONE. */
+int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* packed, const void* const* x,
+                           int32_t x_type, void* const* y, int32_t y_type, int32_t epilogue, const float* weights,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
 /* Convenience for callers whose activations live in host memory: brings x_host to x_dev, runs the GEMV for
  * desc->mode and delivers y in y_host, all on `stream` (the host sees y once the stream reached this point).
  * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller.  Pinned,

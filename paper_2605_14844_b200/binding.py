@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 EXPORTS = ("xfp_packed_size", "xfp_pack", "xfp_gemv_v2", "xfp_gemv_v2a", "xfp_gemv_grouped", "xfp_gemv_host",
-           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_grouped_epilogue", "xfp_gemv_typed")
+           "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_grouped_epilogue", "xfp_gemv_typed",
+           "xfp_gemv_grouped_typed")
 
 XFP_EPI_NONE, XFP_EPI_SWIGLU, XFP_EPI_COMBINE = 0, 1, 2
 XFP_T_F32, XFP_T_F16, XFP_T_BF16 = 0, 1, 2
@@ -55,6 +56,7 @@ def load_library() -> C.CDLL:
     lib.xfp_gemv_v2.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_v2a.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_grouped.argtypes = [dp, i32, vp, vp, vp, i32, vp, sz, vp]
+    lib.xfp_gemv_grouped_typed.argtypes = [dp, i32, vp, vp, i32, vp, i32, i32, vp, vp, sz, vp]
     lib.xfp_gemv_typed.argtypes = [dp, vp, vp, i32, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_grouped_epilogue.argtypes = [dp, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
     lib.xfp_gemv_host.argtypes = [dp, vp, vp, vp, i32, vp, vp, i32, vp, sz, vp]
@@ -144,6 +146,18 @@ def xfp_gemv_grouped_epilogue(desc, n: int, packed_ptrs: torch.Tensor, x_ptrs: t
                                                     _ptr(y_ptrs), int(bool(y_is_fp16)), int(epilogue), _ptr(weights),
                                                     _ptr(workspace), workspace.numel() * workspace.element_size(),
                                                     _stream(stream)), "xfp_gemv_grouped_epilogue")
+
+
+def xfp_gemv_grouped_typed(desc, n: int, packed_ptrs: torch.Tensor, x_ptrs: torch.Tensor, x_dtype, y_ptrs: torch.Tensor,
+                           y_dtype, epilogue: int, weights: Optional[torch.Tensor], workspace: torch.Tensor,
+                           stream=None) -> None:
+    """The grouped launch with fp16 / bf16 activations and fp32 / fp16 / bf16 outputs (torch dtypes) and an optional
+    fused store (XFP_EPI_*)."""
+    _check(load_library().xfp_gemv_grouped_typed(C.byref(desc), int(n), _ptr(packed_ptrs), _ptr(x_ptrs),
+                                                 _TORCH_TYPE[x_dtype], _ptr(y_ptrs), _TORCH_TYPE[y_dtype], int(epilogue),
+                                                 _ptr(weights), _ptr(workspace),
+                                                 workspace.numel() * workspace.element_size(), _stream(stream)),
+           "xfp_gemv_grouped_typed")
 
 
 def xfp_gemv_host(desc, packed, x_host: torch.Tensor, x_dev, batch, y_host: torch.Tensor, y_dev, y_is_fp16,

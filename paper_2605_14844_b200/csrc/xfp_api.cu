@@ -169,9 +169,9 @@ int xfp_gemv_grouped(const xfp_desc* desc, int32_t n, const void* const* packed,
     return gemv_common(desc, desc->mode, c, stream);
 }
 
-int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
-                              void* const* y, int32_t y_is_fp16, int32_t epilogue, const float* weights,
-                              void* workspace, size_t workspace_bytes, void* stream) {
+static int grouped_common(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
+                          int32_t x_bf16, void* const* y, int32_t y_type, int32_t epilogue, const float* weights,
+                          void* workspace, size_t workspace_bytes, void* stream) {
     if (!desc) return XFP_ERR_NULL;
     if (n < 1 || n > 65535) return XFP_ERR_SHAPE;
     if (!packed || !x || !y) return XFP_ERR_NULL;
@@ -183,10 +183,26 @@ int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const
     const Layout l = layout_of(desc);
     const size_t need = workspace_bytes_for(l);
     if (workspace_bytes < need * (size_t)n) return XFP_ERR_BUFFER_TOO_SMALL;
-    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_is_fp16 ? 1 : 0, workspace, need};
+    GemvCall c{nullptr, nullptr, nullptr, packed, x, y, n, 1, y_type, workspace, need};
     c.epilogue = epilogue;
     c.epi_weights = weights;
+    c.x_bf16 = x_bf16;
     return gemv_common(desc, desc->mode, c, stream);
+}
+
+int xfp_gemv_grouped_epilogue(const xfp_desc* desc, int32_t n, const void* const* packed, const uint16_t* const* x,
+                              void* const* y, int32_t y_is_fp16, int32_t epilogue, const float* weights,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+    return grouped_common(desc, n, packed, x, 0, y, y_is_fp16 ? 1 : 0, epilogue, weights, workspace, workspace_bytes, stream);
+}
+
+int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* packed, const void* const* x,
+                           int32_t x_type, void* const* y, int32_t y_type, int32_t epilogue, const float* weights,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    if (x_type != XFP_T_F16 && x_type != XFP_T_BF16) return XFP_ERR_SHAPE;
+    if (y_type != XFP_T_F32 && y_type != XFP_T_F16 && y_type != XFP_T_BF16) return XFP_ERR_SHAPE;
+    return grouped_common(desc, n, packed, (const uint16_t* const*)x, x_type == XFP_T_BF16, y, y_type, epilogue, weights,
+                          workspace, workspace_bytes, stream);
 }
 
 int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* stream) {

@@ -564,3 +564,66 @@ def test_randomized_shapes_types_and_outlier_structure(case):
     tol = TOL * absum + tiny + ulp * np.abs(ref) + 1e-30
     assert np.all(np.isfinite(got))
     assert np.all(np.abs(got - ref) <= tol), float((np.abs(got - ref) / tol).max())
+
+
+@pytest.mark.parametrize("mode,bits", [(1, 3), (1, 4), (0, 4), (0, 5), (1, 6)])
+def test_grouped_typed_bf16(mode, bits):
+    """The grouped launch with bf16 activations and outputs: plain for every mode (pair kernel, V2a kernels, generic),
+    and the fused expert block (SiLU(gate)*up, then the weighted sum) where it exists."""
+    n, rows_gu, hidden = 4, 256, 384
+    inter = rows_gu // 2
+    gus = [synth.random_quantized(mode, rows_gu, hidden, bits, 0.003, seed=3300 + j) for j in range(n)]
+    if mode == 1:
+        for q in gus[1:]:
+            q.codebook = gus[0].codebook
+    pg = [xfp.pack_tensors(q, col_bits=16) for q in gus]
+    xd, x64 = _bf16_x(1, hidden, 3400)
+    ptr = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    dg = _group_desc(pg)
+    wsg = torch.zeros(n * xfp.xfp_packed_size(dg)[1], dtype=torch.uint8, device="cuda")
+    y = torch.full((n, rows_gu), float("nan"), dtype=torch.bfloat16, device="cuda")
+    xfp.xfp_gemv_grouped_typed(dg, n, ptr([p.packed for p in pg]), ptr([xd] * n), torch.bfloat16, ptr([y[j] for j in range(n)]),
+                               torch.bfloat16, xfp.XFP_EPI_NONE, None, wsg)
+    torch.cuda.synchronize()
+    refs = []
+    for j in range(n):
+        ref, absum = xo.gemv_x64(to_oracle(gus[j]), x64)
+        refs.append((ref[0], absum[0]))
+        tiny = 2.0 ** -25 * np.abs(xo.dequant(to_oracle(gus[j])).view(np.float16).astype(np.float64)).sum(1)
+        got = y[j].to(torch.float64).cpu().numpy()
+        assert np.all(np.abs(got - ref[0]) <= TOL * absum[0] + tiny + 2.0 ** -8 * np.abs(ref[0]) + 1e-30), j
+    if mode == 0 or bits > 5:
+        return          # fused stores exist for V2a up to N = 5
+    h = torch.full((n, inter), float("nan"), dtype=torch.bfloat16, device="cuda")
+    xfp.xfp_gemv_grouped_typed(dg, n, ptr([p.packed for p in pg]), ptr([xd] * n), torch.bfloat16, ptr([h[j] for j in range(n)]),
+                               torch.bfloat16, xfp.XFP_EPI_SWIGLU, None, wsg)
+    torch.cuda.synchronize()
+    blocks = rows_gu // 64
+    gate_rows = (np.arange(blocks)[:, None] * 64 + np.arange(32)[None, :]).reshape(-1)
+    for j in range(n):
+        ref, absum = refs[j]
+        g, u = ref[gate_rows], ref[gate_rows + 32]
+        eg, eu = TOL * absum[gate_rows] + 1e-9, TOL * absum[gate_rows + 32] + 1e-9
+        want = xo.silu_mul(g, u)
+        sil = g / (1.0 + np.exp(-g))
+        bound = 1.1 * np.abs(u) * eg + np.abs(sil) * eu + 1.1 * eg * eu + 2.0 ** -7 * np.abs(want) + 1e-30
+        assert np.all(np.abs(h[j].to(torch.float64).cpu().numpy() - want) <= bound), j
+    dns = [synth.random_quantized(1, hidden, inter, bits, 0.003, seed=3500 + j) for j in range(n)]
+    for q in dns[1:]:
+        q.codebook = dns[0].codebook
+    pd = [xfp.pack_tensors(q, col_bits=16) for q in dns]
+    dd = _group_desc(pd)
+    wsd = torch.zeros(n * xfp.xfp_packed_size(dd)[1], dtype=torch.uint8, device="cuda")
+    wts = torch.tensor([0.4, 0.3, 0.2, 0.1], dtype=torch.float32, device="cuda")
+    out = torch.full((1, hidden), float("nan"), dtype=torch.bfloat16, device="cuda")
+    xfp.xfp_gemv_grouped_typed(dd, n, ptr([p.packed for p in pd]), ptr([h[j] for j in range(n)]), torch.bfloat16,
+                               ptr([out[0]] * n), torch.bfloat16, xfp.XFP_EPI_COMBINE, wts, wsd)
+    torch.cuda.synchronize()
+    want = np.zeros(hidden)
+    bound = np.zeros(hidden)
+    for j in range(n):
+        ref, absum = xo.gemv_x64(to_oracle(dns[j]), h[j:j + 1].to(torch.float64).cpu().numpy())
+        want += float(wts[j]) * ref[0]
+        bound += float(wts[j]) * absum[0]
+    got = out[0].to(torch.float64).cpu().numpy()
+    assert np.all(np.abs(got - want) <= TOL * bound + 2.0 ** -8 * np.abs(want) + 1e-6)
