@@ -853,23 +853,37 @@ __global__ void libfit_seed(const double* __restrict__ u, const int* __restrict_
     cen[l * E + j] = u[(int64_t)order[t] * E + j];
 }
 
-// asg[i] = nearest centroid (squared distance summed entry by entry; ties: lower centroid)
-__global__ void libfit_assign_rows(const double* __restrict__ u, const double* __restrict__ cen, int rows, int E,
-                                   int L, int* asg, const int* done) {
+// asg[i] = nearest centroid (squared distance summed entry by entry; ties: lower centroid).  One warp per channel,
+// lane = centroid (32 at a time): every lane sums its distance in entry order, the warp keeps the smallest
+// (distance, centroid) pair -- the answer of a scan over the centroids with a strict "less than".
+__global__ void __launch_bounds__(256) libfit_assign_rows(const double* __restrict__ u, const double* __restrict__ cen,
+                                                           int rows, int E, int L, int* asg, const int* done) {
     if (*done) return;
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
     if (i >= rows) return;
     int best = 0;
     double bd = INFINITY;
-    for (int l = 0; l < L; ++l) {
-        double d = 0.0;
-        for (int j = 0; j < E; ++j) {
-            const double t = __dsub_rn(u[(int64_t)i * E + j], cen[l * E + j]);
-            d = __dadd_rn(d, __dmul_rn(t, t));
+    for (int l0 = 0; l0 < L; l0 += 32) {
+        const int l = l0 + lane;
+        double d = INFINITY;
+        if (l < L) {
+            d = 0.0;
+            for (int j = 0; j < E; ++j) {
+                const double t = __dsub_rn(u[(int64_t)i * E + j], cen[l * E + j]);
+                d = __dadd_rn(d, __dmul_rn(t, t));
+            }
         }
-        if (d < bd) { bd = d; best = l; }
+        int bl = l;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {   // smallest distance, lower centroid on a tie
+            const double od = __shfl_xor_sync(0xffffffffu, d, o);
+            const int ol = __shfl_xor_sync(0xffffffffu, bl, o);
+            if (od < d || (od == d && ol < bl)) { d = od; bl = ol; }
+        }
+        if (d < bd) { bd = d; best = bl; }   // a later group of 32 wins only when strictly nearer
     }
-    asg[i] = best;
+    if (lane == 0) asg[i] = best;
 }
 
 // centroid l <- mean of its members, every entry summed in channel order.  One block per centroid: the
@@ -1226,7 +1240,7 @@ int xfp_quant_libfit_library(const uint16_t* codebook, int32_t rows, int32_t bit
     libfit_seed<<<L, 64, 0, s>>>(w.u, w.order, rows, E, L, w.cen);
     libfit_flags_init<<<1, 1, 0, s>>>(w.flags, w.flags + 1);
     for (int it = 0; it < iters; ++it) {
-        libfit_assign_rows<<<rb, 256, 0, s>>>(w.u, w.cen, rows, E, L, w.asg, w.flags + 1);
+        libfit_assign_rows<<<(rows + 7) / 8, 256, 0, s>>>(w.u, w.cen, rows, E, L, w.asg, w.flags + 1);
         libfit_update<<<L, 256, 0, s>>>(w.u, w.asg, rows, E, L, w.cen, w.flags, w.flags + 1);
         libfit_round_end<<<1, 1, 0, s>>>(w.flags, w.flags + 1);
     }
