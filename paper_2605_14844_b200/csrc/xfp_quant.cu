@@ -887,18 +887,18 @@ __global__ void __launch_bounds__(256) libfit_assign_rows(const double* __restri
 }
 
 // centroid l <- mean of its members, every entry summed in channel order.  One block per centroid: the
-// members of each tile of 256 channels are compacted in order, then thread j adds them to entry j.
-__global__ void __launch_bounds__(256) libfit_update(const double* __restrict__ u, const int* __restrict__ asg,
-                                                      int rows, int E, int L, double* cen, int* changed,
-                                                      const int* done) {
-    __shared__ int sh[8];
+// members of each tile of 1024 channels are compacted in order, then thread j adds them to entry j.
+__global__ void __launch_bounds__(1024) libfit_update(const double* __restrict__ u, const int* __restrict__ asg,
+                                                       int rows, int E, int L, double* cen, int* changed,
+                                                       const int* done) {
+    __shared__ int sh[32];
     __shared__ int total;
-    __shared__ int member[256];
+    __shared__ int member[1024];
     if (*done) return;
     const int l = blockIdx.x, j = threadIdx.x;
     double acc = 0.0;
     long long cnt = 0;
-    for (int i0 = 0; i0 < rows; i0 += 256) {
+    for (int i0 = 0; i0 < rows; i0 += 1024) {
         const int i = i0 + threadIdx.x;
         const int f = i < rows && asg[i] == l;
         const int off = block_excl_scan(f, sh, &total);
@@ -1241,7 +1241,7 @@ int xfp_quant_libfit_library(const uint16_t* codebook, int32_t rows, int32_t bit
     libfit_flags_init<<<1, 1, 0, s>>>(w.flags, w.flags + 1);
     for (int it = 0; it < iters; ++it) {
         libfit_assign_rows<<<(rows + 7) / 8, 256, 0, s>>>(w.u, w.cen, rows, E, L, w.asg, w.flags + 1);
-        libfit_update<<<L, 256, 0, s>>>(w.u, w.asg, rows, E, L, w.cen, w.flags, w.flags + 1);
+        libfit_update<<<L, 1024, 0, s>>>(w.u, w.asg, rows, E, L, w.cen, w.flags, w.flags + 1);
         libfit_round_end<<<1, 1, 0, s>>>(w.flags, w.flags + 1);
     }
     libfit_store<<<L, 32, 0, s>>>(w.cen, E, lib);
