@@ -150,6 +150,20 @@ int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* p
                            int32_t x_type, void* const* y, int32_t y_type, int32_t epilogue, const float* weights,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* Prefill form of the fused kernel ("Fused Decode Kernel": depack, codebook gather, outlier scatter-add into the
+ * dequantised tile, GEMM on the tensor cores; the paper's split-M path for many rows of x):
+ *     y[t][i] = sum_k W^[i][k] * x[t][k],   W^ = fp16(D16 + S), the matrix xfp_dequant writes,
+ * for m >= 1 rows of x in one launch on the tcgen05 tensor cores (fp16 x fp16 products, fp32 accumulation in tensor
+ * memory, one rounding of the sum to y_type).  V2 blobs, every N; V2a returns XFP_ERR_UNSUPPORTED.
+ *   x  [m][cols] fp16;  y  [m][rows] of y_type (XFP_T_F32, XFP_T_F16 or XFP_T_BF16)
+ *   workspace  xfp_gemm_workspace_size(desc, m) bytes, zero-filled once before first use; its counter part is left
+ *              zero-filled by every call.  Its first 32-bit word is an error flag: the kernel sets it to 1 if one of
+ *              its bounded waits ran out (y is then not written); the caller may read it after synchronising.
+ * Results are deterministic (K slices, when the matrix has few rows, are added in slice order). */
+int xfp_gemm_workspace_size(const xfp_desc* desc, int32_t m, size_t* workspace_bytes);
+int xfp_gemm(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t m, void* y, int32_t y_type,
+             void* workspace, size_t workspace_bytes, void* stream);
+
 /* Convenience for callers whose activations live in host memory: brings x_host to x_dev, runs the GEMV for
  * desc->mode and delivers y in y_host, all on `stream` (the host sees y once the stream reached this point).
  * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller.  Pinned,

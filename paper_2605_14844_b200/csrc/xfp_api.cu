@@ -205,6 +205,31 @@ int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* p
                           workspace, workspace_bytes, stream);
 }
 
+int xfp_gemm_workspace_size(const xfp_desc* desc, int32_t m, size_t* workspace_bytes) {
+    int st = check_desc(desc);
+    if (st) return st;
+    if (!workspace_bytes) return XFP_ERR_NULL;
+    if (m < 1) return XFP_ERR_SHAPE;
+    const Layout l = layout_of(desc);
+    if (!gemm_tc_supported(l, m)) return XFP_ERR_UNSUPPORTED;
+    *workspace_bytes = gemm_workspace_bytes(l, m);
+    return XFP_OK;
+}
+
+int xfp_gemm(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t m, void* y, int32_t y_type,
+             void* workspace, size_t workspace_bytes, void* stream) {
+    int st = check_desc(desc);
+    if (st) return st;
+    if (m < 1 || y_type < 0 || y_type > 2) return XFP_ERR_SHAPE;
+    if (!packed || !x || !y || !workspace) return XFP_ERR_NULL;
+    if (!aligned16(packed) || !aligned16(x) || !aligned16(y) || !aligned16(workspace)) return XFP_ERR_ALIGN;
+    const Layout l = layout_of(desc);
+    if (!gemm_tc_supported(l, m)) return XFP_ERR_UNSUPPORTED;
+    if (workspace_bytes < gemm_workspace_bytes(l, m)) return XFP_ERR_BUFFER_TOO_SMALL;
+    GemmCall c{packed, x, y, m, y_type, workspace, workspace_bytes};
+    return launch_gemm_tc(l, c, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
+}
+
 int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* stream) {
     int st = check_desc(desc);
     if (st) return st;

@@ -82,6 +82,21 @@ cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s
 bool batch_v2a_supported(const Layout& l, int batch);
 cudaError_t launch_gemv_batch_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
 
+// Prefill form on the tcgen05 tensor cores (V2, any number of rows of x); see xfp_gemm_tc.cu.
+struct GemmCall {
+    const void* packed;
+    const uint16_t* x;   // [M][cols] fp16
+    void* y;             // [M][rows]
+    int M;
+    int y_kind;          // 0 fp32, 1 fp16, 2 bf16
+    void* workspace;
+    size_t workspace_bytes;
+};
+bool gemm_tc_supported(const Layout& l, int M);
+size_t gemm_ctrl_bytes(const Layout& l, int M);
+size_t gemm_workspace_bytes(const Layout& l, int M);
+cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s);
+
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);

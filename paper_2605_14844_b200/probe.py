@@ -41,6 +41,12 @@
         outliers for V2a): device time of every stage (statistics, extraction, Lloyd, LibFit, residual,
         cosine, median) and wall time of the whole xfp_quantize call with BITS as its only candidate.
 
+    python -m paper_2605_14844_b200.probe gemm ROWS COLS BITS RATE M [M ...] [launch]
+        the prefill form (xfp_gemm, tcgen05 tensor cores) on one V2 matrix for every M given: microseconds per call
+        over distinct packed copies (more than twice the L2), effective GB/s over the algorithmic bytes, TFLOP/s, and
+        beside it a library fp16 GEMM (torch.matmul) on the dequantised matrix.  With `launch` as last word: three
+        calls of the first M with an L2 flush before each (the target of ncu captures).
+
 MODE 0 = V2, 1 = V2a; PLACEMENT uniform | clustered | one_row.  Inputs come from synth.random_quantized.
 """
 from __future__ import annotations
@@ -430,7 +436,69 @@ def quant(mode, rows, cols, bits, reps=3):
                           Mweights_per_s=round(rows * cols / np.median(walls) / 1e3, 1))), flush=True)
 
 
+def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=10):
+    from . import xfp_gemm, xfp_gemm_workspace_size
+    q = synth.random_quantized(0, rows, cols, bits, rate, seed=1)
+    if launch_only:
+        pm = pack_tensors(q, col_bits=16)
+        m = ms[0]
+        x = _x(m, cols)
+        y = torch.empty((m, rows), dtype=torch.float16, device="cuda")
+        ws = torch.zeros(xfp_gemm_workspace_size(pm.desc, m), dtype=torch.uint8, device="cuda")
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            flush.fill_(1)
+            xfp_gemm(pm.desc, pm.packed, x, y, ws)
+        torch.cuda.synchronize()
+        print("ok", float(y.float().abs().sum()), int(ws[:4].view(torch.int32).item()))
+        return
+    nb0 = algorithmic_bytes(q, batch=0)
+    copies = max(2, int(300e6 // nb0) + 1)
+    pms = [pack_tensors(q, col_bits=16) for _ in range(copies)]
+    W = pms[0].dequant()
+    s = torch.cuda.Stream()
+
+    def timed(fn):
+        with torch.cuda.stream(s):
+            fn()
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                fn()
+            for _ in range(3):
+                g.replay()
+            s.synchronize()
+            ts = []
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s)
+                g.replay()
+                e1.record(s)
+                s.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+
+    for m in ms:
+        x = _x(m, cols)
+        ys = [torch.empty((m, rows), dtype=torch.float16, device="cuda") for _ in range(copies)]
+        wss = [torch.zeros(xfp_gemm_workspace_size(pm.desc, m), dtype=torch.uint8, device="cuda") for pm in pms]
+        t = timed(lambda: [xfp_gemm(pm.desc, pm.packed, x, y, ws) for pm, y, ws in zip(pms, ys, wss)]) / copies
+        Ws = [W.clone() for _ in range(max(2, int(300e6 // (rows * cols * 2)) + 1))]
+        t_lib = timed(lambda: [torch.matmul(x, w.t(), out=ys[0]) for w in Ws]) / len(Ws)
+        nb = nb0 + m * (cols * 2 + rows * 2)
+        fl = 2.0 * m * rows * cols
+        err = max(int(ws[:4].view(torch.int32).item()) for ws in wss)
+        print(json.dumps(dict(rows=rows, cols=cols, bits=bits, rate=rate, M=m, copies=copies, us_per_call=round(t, 2),
+                              GBs=round(nb / t / 1e3, 1), TFLOPs=round(fl / t / 1e6, 1),
+                              lib_fp16_gemm_us=round(t_lib, 2), err_flag=err)), flush=True)
+
+
 def main(argv):
+    if len(argv) > 1 and argv[1] == "gemm":
+        lo = argv[-1] == "launch"
+        rest = argv[6:-1] if lo else argv[6:]
+        gemm(int(argv[2]), int(argv[3]), int(argv[4]), float(argv[5]), [int(v) for v in rest], lo)
+        return 0
     if len(argv) > 1 and argv[1] == "packdq":
         packdq(int(argv[2]), int(argv[3]), int(argv[4]), int(argv[5]), float(argv[6]))
         return 0

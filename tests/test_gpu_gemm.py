@@ -1,0 +1,115 @@
+"""Parity of the prefill form (xfp_gemm, tcgen05 tensor cores) against the CPU oracle, through the C ABI.
+
+Every row of x is one GEMV of the oracle: |y_ti - y_ref_ti| <= 1e-3 * sum_k |W_ik x_tk|.  The kernel multiplies
+the dequantised matrix W^ = fp16(D16 + S) (exact fp16 products, fp32 accumulation), so it is also held, far more
+tightly, to an fp64 product with the oracle's dequantised matrix.
+"""
+import numpy as np
+import pytest
+import torch
+
+from conftest import to_oracle
+from oracle import xfp_oracle as xo
+import paper_2605_14844_b200 as xfp
+from paper_2605_14844_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-3
+TIGHT = 2e-5     # fp32 accumulation of K <= 65536 exact products, relative to sum_k |W^_ik x_tk|
+
+
+def _run(q, pm, x16, dtype=torch.float32):
+    xd = torch.from_numpy(x16.view(np.int16)).cuda().view(torch.float16)
+    m = x16.shape[0]
+    ws = torch.zeros(xfp.xfp_gemm_workspace_size(pm.desc, m), dtype=torch.uint8, device="cuda")
+    y = torch.full((m, q.rows), float("nan"), dtype=dtype, device="cuda")
+    xfp.xfp_gemm(pm.desc, pm.packed, xd, y, ws)
+    torch.cuda.synchronize()
+    words = ws[: (ws.numel() // 4) * 4].view(torch.int32)
+    assert int(words[0].item()) == 0, "a bounded wait ran out in the kernel"
+    n_ctrl = min(words.numel(), 1 + ((q.rows + 127) // 128) * ((m + 127) // 128))
+    assert int(words[:n_ctrl].abs().sum().item()) == 0, "slice counters not left at zero"
+    return y, ws, xd
+
+
+def _check(q, pm, x16, dtype=torch.float32):
+    y, _, _ = _run(q, pm, x16, dtype)
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got))
+    mo = to_oracle(q)
+    ref, absum = xo.gemv(mo, x16)
+    err = np.abs(got - ref)
+    # a bf16 store rounds the sum to 8 significant bits: half an ulp of the result on top of the GEMV bound
+    tol = TOL * absum + (2.0 ** -8 * np.abs(ref) if dtype == torch.bfloat16 else 0.0) + 1e-30
+    assert np.all(err <= tol), float((err / tol).max())
+    if dtype == torch.float32:
+        What = xo.dequant(mo).view(np.float16).astype(np.float64)
+        xf = x16.view(np.float16).astype(np.float64)
+        ref2 = xf @ What.T
+        abs2 = np.abs(xf) @ np.abs(What).T
+        err2 = np.abs(got - ref2)
+        assert np.all(err2 <= TIGHT * abs2 + 1e-30), float((err2 / (abs2 + 1e-300)).max())
+    return y
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6])
+@pytest.mark.parametrize("m", [1, 16, 37, 128, 200])
+def test_gemm_small(bits, m):
+    # 70 channels: one tile with a ragged row-block and a missing one; 640 columns: five super-chunks, cut along K
+    q = synth.random_quantized(0, 70, 640, bits, 0.02, seed=900 + bits)
+    pm = xfp.pack_tensors(q, col_bits=16 if bits % 2 else 32)
+    _check(q, pm, synth.activations(m, q.cols, seed=11 + m))
+
+
+@pytest.mark.parametrize("rows,cols,bits,rate", [(1, 128, 4, 0.05), (33, 128, 3, 0.0), (300, 1536, 4, 0.01),
+                                                  (96, 12288, 5, 0.01), (2048, 4096, 4, 0.009), (640, 2048, 6, 0.02),
+                                                  (4224, 1024, 2, 0.003)])
+def test_gemm_shapes(rows, cols, bits, rate):
+    q = synth.random_quantized(0, rows, cols, bits, rate, seed=rows + cols + bits)
+    pm = xfp.pack_tensors(q)
+    for m in (24, 130):
+        _check(q, pm, synth.activations(m, cols, seed=5 + m))
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_gemm_output_types(dtype):
+    q = synth.random_quantized(0, 200, 1024, 4, 0.01, seed=31)
+    pm = xfp.pack_tensors(q)
+    _check(q, pm, synth.activations(48, q.cols, seed=3), dtype)
+
+
+def test_gemm_long_rows_and_spill():
+    """K = 65536 (the largest the descriptor admits) and rows whose outliers overflow the slab into the CSR arrays."""
+    q = synth.random_quantized(0, 40, 65536, 4, 0.005, seed=78)
+    _check(q, xfp.pack_tensors(q, col_bits=16), synth.activations(20, q.cols, seed=70))
+    q = synth.random_quantized(0, 64, 2048, 4, 0.01, seed=79, placement="clustered")
+    _check(q, xfp.pack_tensors(q), synth.activations(20, q.cols, seed=71))
+
+
+def test_gemm_matches_gemv_rows_and_is_deterministic():
+    q = synth.random_quantized(0, 512, 4096, 4, 0.01, seed=41)
+    pm = xfp.pack_tensors(q)
+    x16 = synth.activations(64, q.cols, seed=9)
+    y1, _, xd = _run(q, pm, x16)
+    y2, _, _ = _run(q, pm, x16)
+    assert torch.equal(y1, y2)
+    # the same matrix through the decode kernel, row by row of x: both sit inside the oracle's bound, so they
+    # differ by at most twice that bound
+    _, absum = xo.gemv(to_oracle(q), x16[:2])
+    for t in range(2):
+        yv = pm.gemv(xd[t:t + 1]).float().cpu().numpy().astype(np.float64)[0]
+        assert np.all(np.abs(yv - y1[t].cpu().numpy().astype(np.float64)) <= 2 * TOL * absum[t] + 1e-30)
+
+
+def test_gemm_rejects():
+    q = synth.random_quantized(1, 64, 256, 4, 0.0, seed=1)
+    pm = xfp.pack_tensors(q)
+    with pytest.raises(xfp.XfpError):
+        xfp.xfp_gemm_workspace_size(pm.desc, 16)      # V2a: not built
+    q = synth.random_quantized(0, 64, 256, 4, 0.0, seed=1)
+    pm = xfp.pack_tensors(q)
+    x = torch.zeros((16, 256), dtype=torch.float16, device="cuda")
+    y = torch.zeros((16, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(xfp.XfpError):
+        xfp.xfp_gemm(pm.desc, pm.packed, x, y, torch.zeros(16, dtype=torch.uint8, device="cuda"))   # workspace too small
