@@ -1,23 +1,30 @@
 // Prefill form of the fused decode kernel, Y = X (D + S)^T for M >= 1 rows of x ("Fused Decode Kernel", steps
 // (1)-(4): depack, codebook gather, outlier scatter-add into the dequantised tile, GEMM on the tensor cores), on
-// the fifth-generation tensor cores: the decoded fp16 tile is the A operand of tcgen05.mma in shared memory, the
-// x tile the B operand, the fp32 accumulator lives in tensor memory.
+// the fifth-generation tensor cores.  The decoded fp16 tile never touches shared memory: the lane-per-channel
+// decode of the GEMV kernels produces exactly the register image of a tensor-memory tile (lane = row, 32-bit
+// column = two consecutive k), so it is stored with tcgen05.st and used as the A operand of tcgen05.mma from
+// tensor memory; the x tile is the B operand in shared memory, brought there by one bulk tensor copy (TMA) per
+// stage; the fp32 accumulator is a second tensor-memory region.
 //
-//   CTA      128 output channels (four row-blocks) x up to 128 rows of x x one K slice; 8 warps.
-//   stage    one super-chunk (128 k): A = W^[128][128] fp16, B = x[T][128] fp16, both K-major in the plain
-//            (unswizzled) core-matrix layout: element (r, k) at (k/8)*LBO + r*16 + (k%8)*2 bytes, so the 32 lanes
-//            of a warp (one channel each) write 512 contiguous bytes per 8 decoded weights.  Two stages: the
-//            tensor pipe multiplies stage s while the warps decode stage s^1.
-//   decode   warp (row-block, half of the super-chunk): look-ups in per-lane shared-memory tables (pair tables
-//            up to N = 3, one entry per index above), then the outliers of the lane's channel that fall into
-//            the tile are added with one correctly rounded fp16 addition each: the tile holds exactly the
-//            weights xfp_dequant writes.
-//   mma      one thread issues eight m128 nT k16 instructions per stage and commits them to the stage's
-//            mbarrier, which frees the stage for the decode two iterations later.
+//   CTA      128 output channels (four row-blocks) x up to 128 rows of x x one K slice; 8 warps; two CTAs per SM
+//            (256 of the 512 tensor-memory columns each: 128 accumulator columns, two A stages of 64).
+//   stage    one super-chunk (128 k): A = W^[128][128] fp16 in tensor memory, B = x[T][128] fp16 in shared memory,
+//            K-major in the plain (unswizzled) core-matrix layout: element (t, k) at (k/8)*LBO + t*16 + (k%8)*2,
+//            which is what a tensor copy with the box {8 k, T rows, 16 chunks} of x viewed as [K/8][M][8] writes.
+//   decode   warp (row-block, half of the super-chunk): index vectors prefetched one super-chunk ahead, look-ups
+//            in per-lane shared-memory tables (pair tables up to N = 3, one entry per index above) into 32
+//            registers; the outliers of the lane's channel that fall into a group of 8 weights are added there
+//            with one correctly rounded fp16 addition each, so the tile is the matrix xfp_dequant writes.
+//   mma      one thread issues eight m128 nT k16 instructions per stage and commits them to an mbarrier; the
+//            decode of iteration i waits for the products of iteration i - 2, whose operands it overwrites.
 //   epilogue tcgen05.ld (lane = channel, registers = rows of x), direct store, or fp32 partials through the
 //            workspace when K is cut (few row tiles): the last CTA of a tile adds the slices in slice order.
 // Every wait on an mbarrier has an iteration limit; when one runs out the CTA stops issuing work, records it in
 // the first word of the workspace and leaves through the common exit that frees its tensor memory.
+#include <cuda.h>
+
+#include <type_traits>
+
 #include "xfp_internal.h"
 #include "xfp_pair_common.cuh"
 
@@ -28,20 +35,20 @@ namespace {
 constexpr int kTileRows = 128;   // output channels per CTA (the M of the instruction)
 constexpr int kMaxT = 128;       // rows of x per CTA (the N of the instruction), a multiple of 16
 constexpr int kWarps = 8;
-constexpr int kALbo = kTileRows * 16;         // bytes between consecutive 8-k chunks of the A tile
-constexpr int kAStage = 16 * kALbo;           // 32 KB
-constexpr int kBLbo = (kMaxT + 1) * 16;       // one padding row: the x staging writes hit distinct banks
-constexpr int kBStage = 16 * kBLbo;
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int kTmemCols = 128;
+constexpr int kTmemCols = 256;   // [0,128) accumulator, [128,192) and [192,256) the two A stages
+constexpr int kTmemA = 128;
+constexpr int kAStageCols = 64;  // 128 k as fp16 pairs
+constexpr int kXStages = 3;      // x tiles in flight: the copy of iteration i + 1 is issued at the top of iteration i
+constexpr size_t kMinSmem = 80 * 1024;   // at most two CTAs per SM: each holds half of the tensor memory
 
 struct GemmArgs {
     Blob b;
-    const uint16_t* x;
     void* y;
     int* ctrl;        // [0] error word, [1 + tile] arrival counters of the K slices
     float* partial;   // [tile][slice][T][128]
     int rows, cols, RB, SC, M, ell_slots, ks, sc_per_slice, y_kind;
+    int b_lbo;        // bytes between consecutive 8-k chunks of the x tile: rows of x per tile * 16
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -66,12 +73,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
            ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46);
 }
 
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+// D[128][T] (+)= A[128][16] B[T][16]^T: A from tensor memory (lane = row, column = two k), B from shared memory.
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t acc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        :: "r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(acc) : "memory");
 }
 
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -87,6 +95,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 consecutive columns of the warp's 32 tensor-memory lanes, one lane per thread.
+template <int O>
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        :: "r"(taddr), "r"(r[O]), "r"(r[O + 1]), "r"(r[O + 2]), "r"(r[O + 3]), "r"(r[O + 4]), "r"(r[O + 5]),
+           "r"(r[O + 6]), "r"(r[O + 7]), "r"(r[O + 8]), "r"(r[O + 9]), "r"(r[O + 10]), "r"(r[O + 11]),
+           "r"(r[O + 12]), "r"(r[O + 13]), "r"(r[O + 14]), "r"(r[O + 15])
+        : "memory");
+}
+
 template <int N>
 struct Tab {
     static constexpr int E = 1 << N;
@@ -94,47 +113,154 @@ struct Tab {
     static constexpr int T = kPair ? E * E : E;   // words per lane
 };
 
-// One half (64 weights) of the lane's super-chunk: look-ups, eight 16-byte stores into the A tile.
+// The 32-bit words [PART*2N, PART*2N + 2N) of the lane's 128*N-bit stream sit in these 16-byte vectors.
 template <int N, int PART>
-__device__ __forceinline__ void decode_half(const uint4* src, const unsigned char* tab, uint32_t tbase,
-                                            unsigned char* arow) {
-    constexpr int W0 = PART * 2 * N, W1 = W0 + 2 * N;     // 32-bit words of this half of the bit stream
-    constexpr int V0 = W0 / 4, V1 = (W1 + 3) / 4;
-    uint32_t w[4 * N + 1];
-#pragma unroll
-    for (int i = 0; i <= 4 * N; ++i) w[i] = 0u;
-#pragma unroll
-    for (int v = V0; v < V1; ++v) {
-        const uint4 t = ld_stream(src + (size_t)v * 32);
-        w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
+struct Half {
+    static constexpr int W0 = PART * 2 * N, W1 = W0 + 2 * N;
+    static constexpr int V0 = W0 / 4, V1 = (W1 + 3) / 4, NV = V1 - V0;
+};
+
+struct Outliers {
+    const uint32_t* slab;
+    const uint32_t* spill;
+    int nslab, total, cur;
+    uint32_t col;         // column of entry cur, 0xffffffff behind the last one
+    uint32_t ent, ent2;   // entries cur and cur + 1 (column | fp16 value << 16)
+    __device__ __forceinline__ uint32_t fetch(int j) const {
+        return j < nslab ? __ldg(slab + (size_t)(1 + j) * 32) : __ldg(spill + j);
     }
+    __device__ __forceinline__ void advance() {
+        ++cur;
+        ent = ent2;
+        col = cur < total ? (ent2 & 0xffffu) : 0xffffffffu;
+        if (cur + 1 < total) ent2 = fetch(cur + 1);
+    }
+};
+
+// One K slice of one half of the row-block's super-chunks: the whole main loop of a warp.
+// Barriers: bars[0..1] "products of iteration i done" (i & 1), bars[2..4] "x tile landed" (i % 3).
+template <int N, int PART>
+__device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok, int q, int lane, int tid, int Tn,
+                                          int t0, int sc0, int sc1, const unsigned char* tab, unsigned char* sB,
+                                          uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap) {
+    using H = Half<N, PART>;
+    const uint32_t tbase = (uint32_t)lane * 4u;
+    const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+    const int b_stage = 16 * a.b_lbo;
+    const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0) * N * 32 + lane;   // advanced by N*32 per super-chunk
+    uint4 nx[H::NV];
+    if (rb_ok) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint32_t o[4];
+        for (int v = 0; v < H::NV; ++v) nx[v] = ld_stream(idx + (size_t)(H::V0 + v) * 32);
+    }
+    const uint32_t x_bytes = (uint32_t)b_stage;
+    auto stage_x = [&](int sc, int xs) {
+        // one bulk tensor copy: box {8 k, rows of x, 16 chunks} of x viewed as [K/8][M][8]; rows beyond M arrive as zeros
+        const uint32_t bar = smem_u32(&bars[2 + xs]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(x_bytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+            :: "r"(smem_u32(sB + xs * b_stage)), "l"(tmap), "r"(0), "r"(t0), "r"(sc * 16), "r"(bar) : "memory");
+    };
+    if (tid == 0) stage_x(sc0, 0);
+    bool ok = true;
+    int it = 0, xs = 0;                       // xs = it % kXStages
+    for (int sc = sc0; sc < sc1; ++sc, ++it) {
+        const int s = it & 1;
+        const int xn = xs + 1 == kXStages ? 0 : xs + 1;
+        // The A stage written below and the x stage refilled below were read by the products of iteration it - 2.
+        if (it >= 2 && ok) {
+            ok = mbar_wait(smem_u32(&bars[s]), (uint32_t)((it >> 1) - 1) & 1u);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        if (tid == 0 && ok && sc + 1 < sc1) stage_x(sc + 1, xn);
+        const uint32_t k0 = (uint32_t)sc * kSuper;
+        uint32_t d[32];
+        if (rb_ok) {
+            uint32_t w[4 * N + 1];
 #pragma unroll
-        for (int h = 0; h < 4; ++h) {
-            const int p = PART * 32 + c * 4 + h;
-            if (Tab<N>::kPair) {
-                o[h] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
-            } else {
-                const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
-                const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
-                o[h] = lo | (hi << 16);
+            for (int i = 0; i <= 4 * N; ++i) w[i] = 0u;
+#pragma unroll
+            for (int v = 0; v < H::NV; ++v) {
+                w[4 * (H::V0 + v)] = nx[v].x; w[4 * (H::V0 + v) + 1] = nx[v].y;
+                w[4 * (H::V0 + v) + 2] = nx[v].z; w[4 * (H::V0 + v) + 3] = nx[v].w;
+            }
+            if (sc + 1 < sc1) {
+                idx += N * 32;
+#pragma unroll
+                for (int v = 0; v < H::NV; ++v) nx[v] = ld_stream(idx + (size_t)(H::V0 + v) * 32);
+            }
+            if (PART == 1) while (o.col < k0 + 64) o.advance();      // the other warp's half
+            auto chunk = [&](auto cc) {
+                constexpr int c = decltype(cc)::value;
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const int p = PART * 32 + c * 4 + h;
+                    if (Tab<N>::kPair) {
+                        d[4 * c + h] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
+                    } else {
+                        const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
+                        const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
+                        d[4 * c + h] = lo | (hi << 16);
+                    }
+                }
+                // W^ = fp16(D16 + S) at the outliers of this channel inside these 8 weights
+                const uint32_t cbase = k0 + PART * 64 + c * 8;
+                while (o.col < cbase + 8) {
+                    const uint32_t kk = o.col - cbase;
+                    const uint32_t v2 = (o.ent >> 16) << ((kk & 1u) * 16u);
+                    if ((kk >> 1) == 0u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c]) : "r"(v2));
+                    if ((kk >> 1) == 1u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c + 1]) : "r"(v2));
+                    if ((kk >> 1) == 2u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c + 2]) : "r"(v2));
+                    if ((kk >> 1) == 3u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c + 3]) : "r"(v2));
+                    o.advance();
+                }
+            };
+            chunk(std::integral_constant<int, 0>{}); chunk(std::integral_constant<int, 1>{});
+            chunk(std::integral_constant<int, 2>{}); chunk(std::integral_constant<int, 3>{});
+            chunk(std::integral_constant<int, 4>{}); chunk(std::integral_constant<int, 5>{});
+            chunk(std::integral_constant<int, 6>{}); chunk(std::integral_constant<int, 7>{});
+            if (PART == 0) while (o.col < k0 + kSuper) o.advance();  // the other warp's half
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) d[i] = 0u;
+        }
+        const uint32_t ta = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kTmemA + s * kAStageCols + PART * 32);
+        tmem_st16<0>(ta, d);
+        tmem_st16<16>(ta + 16, d);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        if (__syncthreads_or(!ok)) return false;
+        if (tid == 0) {
+            ok = mbar_wait(smem_u32(&bars[2 + xs]), (uint32_t)(it / kXStages) & 1u);   // the x tile has landed
+            if (ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t b0 = smem_u32(sB + xs * b_stage);
+#pragma unroll
+                for (int ks = 0; ks < kSuper / 16; ++ks) {
+                    const uint64_t db = smem_desc(b0 + 2 * ks * a.b_lbo, (uint32_t)a.b_lbo, 128);
+                    umma_f16_ts(tmem, tmem + (uint32_t)(kTmemA + s * kAStageCols + ks * 8), db, idesc,
+                                (it > 0 || ks > 0) ? 1u : 0u);
+                }
+                umma_commit(smem_u32(&bars[s]));
             }
         }
-        *(uint4*)(arow + (PART * 8 + c) * kALbo) = make_uint4(o[0], o[1], o[2], o[3]);
+        xs = xn;
     }
+    // all products of this CTA are complete when the last commit has arrived
+    const int lastit = it - 1;
+    ok = ok && mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
+    return !__syncthreads_or(!ok);
 }
 
 template <int N>
-__global__ void __launch_bounds__(kWarps * 32, 1) gemm_tc_kernel(const GemmArgs a) {
+__global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
     constexpr int E = Tab<N>::E;
     constexpr int TW = Tab<N>::T;
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* sA = smem;                                  // two A stages
-    unsigned char* sB = smem + 2 * kAStage;                    // two B stages
-    unsigned char* sTab = sB + 2 * kBStage;                    // [4 row-blocks][TW][32] words
-    __shared__ __align__(8) uint64_t bars[2];
+    unsigned char* sTab = smem;                                // [4 row-blocks][TW][32] words
+    unsigned char* sB = smem + (size_t)4 * TW * 128;           // kXStages x tiles of 16 * b_lbo bytes (128-byte aligned)
+    __shared__ __align__(8) uint64_t bars[2 + kXStages];
     __shared__ uint32_t s_tmem;
     __shared__ int s_last;
 
@@ -151,8 +277,9 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_tc_kernel(const GemmArgs 
 
     // ---- set-up: barriers, tensor memory, tables ----
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bars[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bars[1])));
+#pragma unroll
+        for (int i = 0; i < 2 + kXStages; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bars[i])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -161,8 +288,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_tc_kernel(const GemmArgs 
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     {
-        // codebooks -> one word per (entry, lane); pair tables are built from a copy staged in the first A stage
-        uint32_t* one = Tab<N>::kPair ? (uint32_t*)sA : (uint32_t*)sTab;
+        // codebooks -> one word per (entry, lane); pair tables are built from a copy staged in the x stages
+        uint32_t* one = Tab<N>::kPair ? (uint32_t*)sB : (uint32_t*)sTab;
         for (int i = warp; i < 4 * E; i += kWarps) {
             const int qq = i / E, e = i % E, r = (blockIdx.x * 4 + qq) * kRowsPerBlock + lane;
             one[(qq * E + e) * 32 + lane] = (blockIdx.x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
@@ -177,103 +304,39 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_tc_kernel(const GemmArgs 
             }
         }
     }
+    // the tables were written through the generic proxy where the first tensor copy (async proxy) lands
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s_tmem;
 
-    // rows of the tile beyond the matrix decode to zero, once, in both stages
-    if (!rb_ok) {
-        for (int s = 0; s < 2; ++s)
-            for (int c = 0; c < 8; ++c)
-                *(uint4*)(sA + s * kAStage + (part * 8 + c) * kALbo + (q * 32 + lane) * 16) = make_uint4(0, 0, 0, 0);
-    }
-
     // ---- the lane's outlier list: transposed slab first, the CSR arrays behind it ----
-    const uint32_t* slab = nullptr;
-    const uint32_t* spill = nullptr;
-    int nslab = 0, total = 0, cur = 0;
-    uint32_t ent = 0;
+    Outliers o{nullptr, nullptr, 0, 0, 0, 0xffffffffu, 0u, 0u};
     if (rb_ok && a.ell_slots) {
-        slab = a.b.ell + (size_t)rb * (a.ell_slots + 1) * 32 + lane;
-        const int olen = (int)__ldg(slab);
-        nslab = min(olen, a.ell_slots);
-        total = nslab;
+        o.slab = a.b.ell + (size_t)rb * (a.ell_slots + 1) * 32 + lane;
+        const int olen = (int)__ldg(o.slab);
+        o.nslab = min(olen, a.ell_slots);
+        o.total = o.nslab;
         if (olen >= a.ell_slots && row < a.rows) {
             const int p0 = __ldg(a.b.rowptr + row);
-            total = __ldg(a.b.rowptr + row + 1) - p0;
-            spill = a.b.oent + p0;
+            o.total = __ldg(a.b.rowptr + row + 1) - p0;
+            o.spill = a.b.oent + p0;
         }
-    }
-    auto fetch = [&](int j) { return j < nslab ? __ldg(slab + (size_t)(1 + j) * 32) : __ldg(spill + j); };
-    if (total) {
-        ent = fetch(0);
-        const uint32_t kb = (uint32_t)sc0 * kSuper;
-        while ((ent & 0xffffu) < kb && ++cur < total) ent = fetch(cur);
+        if (o.total) {
+            o.ent = o.fetch(0);
+            const uint32_t kb = (uint32_t)sc0 * kSuper;
+            while ((o.ent & 0xffffu) < kb && ++o.cur < o.total) o.ent = o.fetch(o.cur);
+            if (o.cur < o.total) o.col = o.ent & 0xffffu;
+            if (o.cur + 1 < o.total) o.ent2 = o.fetch(o.cur + 1);
+        }
     }
 
-    const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
     const unsigned char* tab = sTab + (size_t)q * TW * 128;
-    const uint32_t tbase = (uint32_t)lane * 4u;
-    bool failed = false;
-    int it = 0;
-    for (int sc = sc0; sc < sc1; ++sc, ++it) {
-        const int s = it & 1, use = it >> 1;
-        bool ok = true;
-        if (use >= 1) ok = mbar_wait(smem_u32(&bars[s]), (uint32_t)(use - 1) & 1u);
-        unsigned char* As = sA + s * kAStage;
-        unsigned char* Bs = sB + s * kBStage;
-        if (ok) {
-            // x tile: thread -> (row of x, 16-byte chunk); rows beyond M are zero
-            const int k0 = sc * kSuper;
-            for (int i = tid; i < Tn * 16; i += kWarps * 32) {
-                const int c = i & 15, t = i >> 4;
-                const uint32_t dst = smem_u32(Bs + c * kBLbo + t * 16);
-                const uint16_t* src = a.x + (size_t)(t0 + t) * a.cols + k0 + c * 8;
-                const int bytes = (t0 + t) < a.M ? 16 : 0;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst), "l"(bytes ? src : a.x), "r"(bytes) : "memory");
-            }
-            if (rb_ok) {
-                const uint4* src = a.b.idx + ((size_t)rb * a.SC + sc) * N * 32 + lane;
-                unsigned char* arow = As + (q * 32 + lane) * 16;
-                if (part == 0) decode_half<N, 0>(src, tab, tbase, arow);
-                else decode_half<N, 1>(src, tab, tbase, arow);
-                // W^ = fp16(D16 + S) at the outliers of this channel inside the tile
-                const uint32_t kend = (uint32_t)k0 + kSuper;
-                while (cur < total && (ent & 0xffffu) < kend) {
-                    const uint32_t kk = (ent & 0xffffu) - (uint32_t)k0;
-                    if ((int)(kk >> 6) == part) {
-                        const uint32_t ha = smem_u32(arow + (kk >> 3) * kALbo + (kk & 7u) * 2u);
-                        uint16_t hv;
-                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(hv) : "r"(ha) : "memory");
-                        hv = __half_as_ushort(__hadd(__ushort_as_half(hv), __ushort_as_half((uint16_t)(ent >> 16))));
-                        asm volatile("st.shared.u16 [%0], %1;" :: "r"(ha), "h"(hv) : "memory");
-                    }
-                    if (++cur < total) ent = fetch(cur);
-                }
-            }
-            asm volatile("cp.async.wait_all;" ::: "memory");
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        }
-        if (__syncthreads_or(!ok)) { failed = true; break; }
-        if (tid == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a0 = smem_u32(As), b0 = smem_u32(Bs);
-#pragma unroll
-            for (int ks = 0; ks < kSuper / 16; ++ks) {
-                const uint64_t da = smem_desc(a0 + 2 * ks * kALbo, kALbo, 128);
-                const uint64_t db = smem_desc(b0 + 2 * ks * kBLbo, kBLbo, 128);
-                umma_f16(tmem, da, db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-            }
-            umma_commit(smem_u32(&bars[s]));
-        }
-    }
-    // ---- all products of this CTA are complete when the last commit has arrived ----
-    if (!failed && it > 0) {
-        const int lastit = it - 1;
-        const bool ok = mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
-        if (__syncthreads_or(!ok)) failed = true;
-    }
+    const bool done = part == 0
+        ? main_loop<N, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap)
+        : main_loop<N, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap);
+    const bool failed = !done;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (failed) {
         if (tid == 0) atomicExch(a.ctrl, 1);
@@ -283,12 +346,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_tc_kernel(const GemmArgs 
         float* part_out = a.partial + ((size_t)tile * a.ks + blockIdx.z) * kMaxT * kTileRows;
         for (int cc = part; cc * 16 < Tn; cc += 2) {
             uint32_t v[16];
-            if (it > 0) {
-                tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = 0u;
-            }
+            tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const int t = cc * 16 + j;
@@ -325,6 +383,19 @@ __global__ void __launch_bounds__(kWarps * 32, 1) gemm_tc_kernel(const GemmArgs 
     }
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    return (EncodeTiledFn)fn;
+}
+
 struct Plan {
     int row_tiles, tok_tiles, ks, sc_per_slice;
 };
@@ -335,8 +406,8 @@ Plan plan_of(const Layout& l, int M) {
     p.tok_tiles = (M + kMaxT - 1) / kMaxT;
     const int tiles = p.row_tiles * p.tok_tiles;
     int ks = 1;
-    // fewer tiles than SMs: cut K, at least two super-chunks per slice
-    while (tiles * ks * 2 <= 148 && l.SC / (ks * 2) >= 2) ks *= 2;
+    // fewer tiles than CTA slots (two per SM): cut K, at least two super-chunks per slice
+    while (tiles * ks * 2 <= 2 * 148 && l.SC / (ks * 2) >= 2) ks *= 2;
     p.sc_per_slice = (l.SC + ks - 1) / ks;
     p.ks = (l.SC + p.sc_per_slice - 1) / p.sc_per_slice;
     return p;
@@ -344,23 +415,42 @@ Plan plan_of(const Layout& l, int M) {
 
 template <int N>
 cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
-    const size_t smem = 2 * kAStage + 2 * kBStage + (size_t)4 * Tab<N>::T * 128;
+    const int tmax = c.M >= kMaxT ? kMaxT : (c.M + 15) & ~15;    // rows of x in the largest tile of this launch
+    const int b_lbo = tmax * 16;
+    size_t smem = (size_t)4 * Tab<N>::T * 128 + (size_t)kXStages * 16 * b_lbo;
+    if (smem < kMinSmem) smem = kMinSmem;
+    // x [M][K] fp16 seen as [K/8][M][8]: one box {8, tmax, 16} is a whole x tile in the core-matrix order of the B operand
+    static const EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    {
+        const cuuint64_t dims[3] = {8, (cuuint64_t)c.M, (cuuint64_t)(l.cols / 8)};
+        const cuuint64_t strides[2] = {(cuuint64_t)l.cols * 2, 16};
+        const cuuint32_t box[3] = {8, (cuuint32_t)tmax, 16};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t*>(c.x), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const size_t most = (size_t)4 * Tab<N>::T * 128 + (size_t)kXStages * 16 * kMaxT * 16;
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(most < kMinSmem ? kMinSmem : most));
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
     }
     const Plan p = plan_of(l, c.M);
     GemmArgs a;
     a.b = blob_at(c.packed, offsets_of(l));
-    a.x = c.x; a.y = c.y;
+    a.y = c.y;
     a.ctrl = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + gemm_ctrl_bytes(l, c.M));
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
-    a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind;
-    gemm_tc_kernel<N><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kWarps * 32, smem, s>>>(a);
+    a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_lbo = b_lbo;
+    gemm_tc_kernel<N><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kWarps * 32, smem, s>>>(a, tmap);
     return cudaGetLastError();
 }
 
