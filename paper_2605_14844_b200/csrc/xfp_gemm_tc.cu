@@ -120,20 +120,31 @@ struct Half {
     static constexpr int V0 = W0 / 4, V1 = (W1 + 3) / 4, NV = V1 - V0;
 };
 
+// A lane's outlier list (transposed slab first, the CSR arrays behind it) with the next four entries in registers:
+// an entry is consumed long after its load was issued, so a channel with several outliers close together does not
+// stall its warp (and, through the barrier, its CTA) on a chain of dependent loads.
 struct Outliers {
     const uint32_t* slab;
     const uint32_t* spill;
     int nslab, total, cur;
-    uint32_t col;         // column of entry cur, 0xffffffff behind the last one
-    uint32_t ent, ent2;   // entries cur and cur + 1 (column | fp16 value << 16)
+    uint32_t col;               // column of entry cur, 0xffffffff behind the last one
+    uint32_t ent, e1, e2, e3;   // entries cur .. cur + 3 (column | fp16 value << 16)
     __device__ __forceinline__ uint32_t fetch(int j) const {
         return j < nslab ? __ldg(slab + (size_t)(1 + j) * 32) : __ldg(spill + j);
     }
+    __device__ __forceinline__ void start(int first) {
+        cur = first;
+        if (cur < total) { ent = fetch(cur); }
+        if (cur + 1 < total) e1 = fetch(cur + 1);
+        if (cur + 2 < total) e2 = fetch(cur + 2);
+        if (cur + 3 < total) e3 = fetch(cur + 3);
+        col = cur < total ? (ent & 0xffffu) : 0xffffffffu;
+    }
     __device__ __forceinline__ void advance() {
         ++cur;
-        ent = ent2;
-        col = cur < total ? (ent2 & 0xffffu) : 0xffffffffu;
-        if (cur + 1 < total) ent2 = fetch(cur + 1);
+        ent = e1; e1 = e2; e2 = e3;
+        col = cur < total ? (ent & 0xffffu) : 0xffffffffu;
+        if (cur + 3 < total) e3 = fetch(cur + 3);
     }
 };
 
@@ -148,10 +159,16 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
     const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
     const int b_stage = 16 * a.b_lbo;
     const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0) * N * 32 + lane;   // advanced by N*32 per super-chunk
-    uint4 nx[H::NV];
+    // index vectors of the next three super-chunks in registers: HBM latency is about one iteration of this loop
+    uint4 nx[3][H::NV];
     if (rb_ok) {
 #pragma unroll
-        for (int v = 0; v < H::NV; ++v) nx[v] = ld_stream(idx + (size_t)(H::V0 + v) * 32);
+        for (int ahead = 0; ahead < 3; ++ahead) {
+            if (sc0 + ahead < sc1) {
+#pragma unroll
+                for (int v = 0; v < H::NV; ++v) nx[ahead][v] = ld_stream(idx + (size_t)ahead * N * 32 + (size_t)(H::V0 + v) * 32);
+            }
+        }
     }
     const uint32_t x_bytes = (uint32_t)b_stage;
     auto stage_x = [&](int sc, int xs) {
@@ -182,13 +199,14 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
             for (int i = 0; i <= 4 * N; ++i) w[i] = 0u;
 #pragma unroll
             for (int v = 0; v < H::NV; ++v) {
-                w[4 * (H::V0 + v)] = nx[v].x; w[4 * (H::V0 + v) + 1] = nx[v].y;
-                w[4 * (H::V0 + v) + 2] = nx[v].z; w[4 * (H::V0 + v) + 3] = nx[v].w;
+                w[4 * (H::V0 + v)] = nx[0][v].x; w[4 * (H::V0 + v) + 1] = nx[0][v].y;
+                w[4 * (H::V0 + v) + 2] = nx[0][v].z; w[4 * (H::V0 + v) + 3] = nx[0][v].w;
+                nx[0][v] = nx[1][v]; nx[1][v] = nx[2][v];
             }
-            if (sc + 1 < sc1) {
-                idx += N * 32;
+            idx += N * 32;
+            if (sc + 3 < sc1) {
 #pragma unroll
-                for (int v = 0; v < H::NV; ++v) nx[v] = ld_stream(idx + (size_t)(H::V0 + v) * 32);
+                for (int v = 0; v < H::NV; ++v) nx[2][v] = ld_stream(idx + (size_t)2 * N * 32 + (size_t)(H::V0 + v) * 32);
             }
             if (PART == 1) while (o.col < k0 + 64) o.advance();      // the other warp's half
             auto chunk = [&](auto cc) {
@@ -312,7 +330,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
     const uint32_t tmem = s_tmem;
 
     // ---- the lane's outlier list: transposed slab first, the CSR arrays behind it ----
-    Outliers o{nullptr, nullptr, 0, 0, 0, 0xffffffffu, 0u, 0u};
+    Outliers o{nullptr, nullptr, 0, 0, 0, 0xffffffffu, 0u, 0u, 0u, 0u};
     if (rb_ok && a.ell_slots) {
         o.slab = a.b.ell + (size_t)rb * (a.ell_slots + 1) * 32 + lane;
         const int olen = (int)__ldg(o.slab);
@@ -323,13 +341,20 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
             o.total = __ldg(a.b.rowptr + row + 1) - p0;
             o.spill = a.b.oent + p0;
         }
-        if (o.total) {
-            o.ent = o.fetch(0);
+        // first entry of this K slice: the list ascends, so count the entries below the slice, sixteen
+        // independent loads at a time (a coarse pass over every 16th entry, then the 15 before the first hit)
+        int first = 0;
+        if (sc0 > 0 && o.total) {
             const uint32_t kb = (uint32_t)sc0 * kSuper;
-            while ((o.ent & 0xffffu) < kb && ++o.cur < o.total) o.ent = o.fetch(o.cur);
-            if (o.cur < o.total) o.col = o.ent & 0xffffu;
-            if (o.cur + 1 < o.total) o.ent2 = o.fetch(o.cur + 1);
+            int coarse = 0;
+            for (int j = 15; j < o.total; j += 16) coarse += (o.fetch(j) & 0xffffu) < kb;
+            first = coarse * 16;
+            int fine = 0;
+#pragma unroll
+            for (int j = 0; j < 15; ++j) fine += (first + j < o.total) && (o.fetch(min(first + j, o.total - 1)) & 0xffffu) < kb;
+            first += fine;
         }
+        o.start(first);
     }
 
     const unsigned char* tab = sTab + (size_t)q * TW * 128;
