@@ -34,7 +34,8 @@ namespace {
 
 constexpr int kTileRows = 128;   // output channels per CTA (the M of the instruction)
 constexpr int kMaxT = 128;       // rows of x per CTA (the N of the instruction), a multiple of 16
-constexpr int kWarps = 8;
+constexpr int kWarps = 8;        // decode warps; warp 8 issues the tensor copies and the products
+constexpr int kThreads = (kWarps + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kTmemCols = 256;   // [0,128) accumulator, [128,192) and [192,256) the two A stages
 constexpr int kTmemA = 128;
@@ -149,48 +150,37 @@ struct Outliers {
 };
 
 // One K slice of one half of the row-block's super-chunks: the whole main loop of a warp.
-// Barriers: bars[0..1] "products of iteration i done" (i & 1), bars[2..4] "x tile landed" (i % 3).
+// Barriers: bars[0..1] "products of iteration i done" (i & 1), bars[2..4] "x tile landed" (i % 3), bars[5..6] "A stage
+// of iteration i stored by all eight decode warps" (i & 1).  No CTA-wide barrier inside the loop: a decode warp runs
+// up to two iterations ahead of the products.
 template <int N, int PART>
 __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok, int q, int lane, int tid, int Tn,
                                           int t0, int sc0, int sc1, const unsigned char* tab, unsigned char* sB,
                                           uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap) {
     using H = Half<N, PART>;
     const uint32_t tbase = (uint32_t)lane * 4u;
-    const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
-    const int b_stage = 16 * a.b_lbo;
     const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0) * N * 32 + lane;   // advanced by N*32 per super-chunk
-    // index vectors of the next three super-chunks in registers: HBM latency is about one iteration of this loop
-    uint4 nx[3][H::NV];
+    // index vectors of the next two super-chunks in registers
+    uint4 nx[2][H::NV];
     if (rb_ok) {
 #pragma unroll
-        for (int ahead = 0; ahead < 3; ++ahead) {
+        for (int ahead = 0; ahead < 2; ++ahead) {
             if (sc0 + ahead < sc1) {
 #pragma unroll
                 for (int v = 0; v < H::NV; ++v) nx[ahead][v] = ld_stream(idx + (size_t)ahead * N * 32 + (size_t)(H::V0 + v) * 32);
             }
         }
     }
-    const uint32_t x_bytes = (uint32_t)b_stage;
-    auto stage_x = [&](int sc, int xs) {
-        // one bulk tensor copy: box {8 k, rows of x, 16 chunks} of x viewed as [K/8][M][8]; rows beyond M arrive as zeros
-        const uint32_t bar = smem_u32(&bars[2 + xs]);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(x_bytes) : "memory");
-        asm volatile(
-            "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-            :: "r"(smem_u32(sB + xs * b_stage)), "l"(tmap), "r"(0), "r"(t0), "r"(sc * 16), "r"(bar) : "memory");
-    };
-    if (tid == 0) stage_x(sc0, 0);
     bool ok = true;
-    int it = 0, xs = 0;                       // xs = it % kXStages
+    int it = 0;
     for (int sc = sc0; sc < sc1; ++sc, ++it) {
         const int s = it & 1;
-        const int xn = xs + 1 == kXStages ? 0 : xs + 1;
-        // The A stage written below and the x stage refilled below were read by the products of iteration it - 2.
+        // The A stage written below was read by the products of iteration it - 2.
         if (it >= 2 && ok) {
             ok = mbar_wait(smem_u32(&bars[s]), (uint32_t)((it >> 1) - 1) & 1u);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         }
-        if (tid == 0 && ok && sc + 1 < sc1) stage_x(sc + 1, xn);
+        if (!ok) break;
         const uint32_t k0 = (uint32_t)sc * kSuper;
         uint32_t d[32];
         if (rb_ok) {
@@ -201,12 +191,12 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
             for (int v = 0; v < H::NV; ++v) {
                 w[4 * (H::V0 + v)] = nx[0][v].x; w[4 * (H::V0 + v) + 1] = nx[0][v].y;
                 w[4 * (H::V0 + v) + 2] = nx[0][v].z; w[4 * (H::V0 + v) + 3] = nx[0][v].w;
-                nx[0][v] = nx[1][v]; nx[1][v] = nx[2][v];
+                nx[0][v] = nx[1][v];
             }
             idx += N * 32;
-            if (sc + 3 < sc1) {
+            if (sc + 2 < sc1) {
 #pragma unroll
-                for (int v = 0; v < H::NV; ++v) nx[2][v] = ld_stream(idx + (size_t)2 * N * 32 + (size_t)(H::V0 + v) * 32);
+                for (int v = 0; v < H::NV; ++v) nx[1][v] = ld_stream(idx + (size_t)N * 32 + (size_t)(H::V0 + v) * 32);
             }
             if (PART == 1) while (o.col < k0 + 64) o.advance();      // the other warp's half
             auto chunk = [&](auto cc) {
@@ -248,44 +238,67 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
         tmem_st16<16>(ta + 16, d);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        if (__syncthreads_or(!ok)) return false;
-        if (tid == 0) {
-            ok = mbar_wait(smem_u32(&bars[2 + xs]), (uint32_t)(it / kXStages) & 1u);   // the x tile has landed
-            if (ok) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t b0 = smem_u32(sB + xs * b_stage);
-#pragma unroll
-                for (int ks = 0; ks < kSuper / 16; ++ks) {
-                    const uint64_t db = smem_desc(b0 + 2 * ks * a.b_lbo, (uint32_t)a.b_lbo, 128);
-                    umma_f16_ts(tmem, tmem + (uint32_t)(kTmemA + s * kAStageCols + ks * 8), db, idesc,
-                                (it > 0 || ks > 0) ? 1u : 0u);
-                }
-                umma_commit(smem_u32(&bars[s]));
-            }
-        }
-        xs = xn;
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&bars[5 + s])) : "memory");
     }
     // all products of this CTA are complete when the last commit has arrived
+    const int lastit = sc1 - sc0 - 1;
+    return ok && mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
+}
+
+// The ninth warp (one thread): x tiles by tensor copy one iteration ahead, the eight products of every stage.
+__device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int sc0, int sc1, unsigned char* sB,
+                                         uint64_t* bars, uint32_t tmem, const CUtensorMap* tmap) {
+    const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+    const int b_stage = 16 * a.b_lbo;
+    const uint32_t x_bytes = (uint32_t)b_stage;
+    auto stage_x = [&](int sc, int xs) {
+        // one bulk tensor copy: box {8 k, rows of x, 16 chunks} of x viewed as [K/8][M][8]; rows beyond M arrive as zeros
+        const uint32_t bar = smem_u32(&bars[2 + xs]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(x_bytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+            :: "r"(smem_u32(sB + xs * b_stage)), "l"(tmap), "r"(0), "r"(t0), "r"(sc * 16), "r"(bar) : "memory");
+    };
+    stage_x(sc0, 0);
+    int it = 0, xs = 0;                       // xs = it % kXStages
+    for (int sc = sc0; sc < sc1; ++sc, ++it) {
+        const int s = it & 1;
+        const int xn = xs + 1 == kXStages ? 0 : xs + 1;
+        // the x stage refilled now was read by the products of iteration it - 2
+        if (it >= 2 && !mbar_wait(smem_u32(&bars[s]), (uint32_t)((it >> 1) - 1) & 1u)) return false;
+        if (sc + 1 < sc1) stage_x(sc + 1, xn);
+        if (!mbar_wait(smem_u32(&bars[5 + s]), (uint32_t)(it >> 1) & 1u)) return false;          // A stage stored
+        if (!mbar_wait(smem_u32(&bars[2 + xs]), (uint32_t)(it / kXStages) & 1u)) return false;   // x tile landed
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t b0 = smem_u32(sB + xs * b_stage);
+#pragma unroll
+        for (int ks = 0; ks < kSuper / 16; ++ks) {
+            const uint64_t db = smem_desc(b0 + 2 * ks * a.b_lbo, (uint32_t)a.b_lbo, 128);
+            umma_f16_ts(tmem, tmem + (uint32_t)(kTmemA + s * kAStageCols + ks * 8), db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bars[s]));
+        xs = xn;
+    }
     const int lastit = it - 1;
-    ok = ok && mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
-    return !__syncthreads_or(!ok);
+    return mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
 }
 
 template <int N>
-__global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
+__global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
     constexpr int E = Tab<N>::E;
     constexpr int TW = Tab<N>::T;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* sTab = smem;                                // [4 row-blocks][TW][32] words
     unsigned char* sB = smem + (size_t)4 * TW * 128;           // kXStages x tiles of 16 * b_lbo bytes (128-byte aligned)
-    __shared__ __align__(8) uint64_t bars[2 + kXStages];
+    __shared__ __align__(8) uint64_t bars[4 + kXStages];
     __shared__ uint32_t s_tmem;
     __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = warp & 3, part = warp >> 2;                  // row-block of the tile, half of the super-chunk
     const int rb = blockIdx.x * 4 + q;
-    const bool rb_ok = rb < a.RB;
+    const bool rb_ok = rb < a.RB && warp < kWarps;
     const int row = rb * kRowsPerBlock + lane;
     const int t0 = blockIdx.y * kMaxT;
     const int Tn = min(kMaxT, (a.M - t0 + 15) & ~15);          // rows of x of this tile, rounded up to 16
@@ -296,8 +309,8 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
     // ---- set-up: barriers, tensor memory, tables ----
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < 2 + kXStages; ++i)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bars[i])));
+        for (int i = 0; i < 4 + kXStages; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[i])), "r"(i >= 2 + kXStages ? kWarps : 1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -308,14 +321,14 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
     {
         // codebooks -> one word per (entry, lane); pair tables are built from a copy staged in the x stages
         uint32_t* one = Tab<N>::kPair ? (uint32_t*)sB : (uint32_t*)sTab;
-        for (int i = warp; i < 4 * E; i += kWarps) {
+        for (int i = warp; i < 4 * E; i += kWarps + 1) {
             const int qq = i / E, e = i % E, r = (blockIdx.x * 4 + qq) * kRowsPerBlock + lane;
             one[(qq * E + e) * 32 + lane] = (blockIdx.x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
         }
         if (Tab<N>::kPair) {
             __syncthreads();
             uint32_t* tab = (uint32_t*)sTab;
-            for (int i = warp; i < 4 * TW; i += kWarps) {
+            for (int i = warp; i < 4 * TW; i += kWarps + 1) {
                 const int qq = i / TW, t = i % TW;
                 tab[(qq * TW + t) * 32 + lane] =
                     one[(qq * E + (t & (E - 1))) * 32 + lane] | (one[(qq * E + (t >> N)) * 32 + lane] << 16);
@@ -358,10 +371,16 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
     }
 
     const unsigned char* tab = sTab + (size_t)q * TW * 128;
-    const bool done = part == 0
-        ? main_loop<N, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap)
-        : main_loop<N, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap);
-    const bool failed = !done;
+    bool done;
+    if (warp == kWarps) {
+        done = lane != 0 || mma_loop(a, Tn, t0, sc0, sc1, sB, bars, tmem, &tmap);
+        __syncwarp();
+    } else {
+        done = part == 0
+            ? main_loop<N, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap)
+            : main_loop<N, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap);
+    }
+    const bool failed = __syncthreads_or(!done) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (failed) {
         if (tid == 0) atomicExch(a.ctrl, 1);
@@ -369,7 +388,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
         // lane = channel (tensor-memory lane 32*(warp%4) + lane), registers = 16 consecutive rows of x
         const int r = q * 32 + lane;
         float* part_out = a.partial + ((size_t)tile * a.ks + blockIdx.z) * kMaxT * kTileRows;
-        for (int cc = part; cc * 16 < Tn; cc += 2) {
+        for (int cc = part; warp < kWarps && cc * 16 < Tn; cc += 2) {
             uint32_t v[16];
             tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
 #pragma unroll
@@ -398,7 +417,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) gemm_tc_kernel(const GemmArgs 
     if (!s_last) return;
     __threadfence();
     const float* p0 = a.partial + (size_t)tile * a.ks * kMaxT * kTileRows;
-    for (int i = tid; i < Tn * kTileRows; i += kWarps * 32) {
+    for (int i = tid; i < Tn * kTileRows; i += kThreads) {
         const int t = i / kTileRows, r = i % kTileRows;
         const int orow = blockIdx.x * kTileRows + r;
         if (t0 + t >= a.M || orow >= a.rows) continue;
@@ -475,7 +494,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.partial = (float*)((char*)c.workspace + gemm_ctrl_bytes(l, c.M));
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
     a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_lbo = b_lbo;
-    gemm_tc_kernel<N><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kWarps * 32, smem, s>>>(a, tmap);
+    gemm_tc_kernel<N><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kThreads, smem, s>>>(a, tmap);
     return cudaGetLastError();
 }
 
