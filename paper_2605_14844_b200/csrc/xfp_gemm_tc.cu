@@ -198,37 +198,39 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
 #pragma unroll
                 for (int v = 0; v < H::NV; ++v) nx[1][v] = ld_stream(idx + (size_t)N * 32 + (size_t)(H::V0 + v) * 32);
             }
-            if (PART == 1) while (o.col < k0 + 64) o.advance();      // the other warp's half
-            auto chunk = [&](auto cc) {
-                constexpr int c = decltype(cc)::value;
+            // 64 look-ups in one straight block (every load can be in flight at once)
 #pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    const int p = PART * 32 + c * 4 + h;
-                    if (Tab<N>::kPair) {
-                        d[4 * c + h] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
-                    } else {
-                        const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
-                        const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
-                        d[4 * c + h] = lo | (hi << 16);
+            for (int i = 0; i < 32; ++i) {
+                const int p = PART * 32 + i;
+                if (Tab<N>::kPair) {
+                    d[i] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
+                } else {
+                    const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
+                    const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
+                    d[i] = lo | (hi << 16);
+                }
+            }
+            // W^ = fp16(D16 + S) at the outliers of this channel inside this half; the entries of the other half
+            // (the other warp's) are passed over.  One loop, one copy of the code that advances the list.
+            const uint32_t lo_k = k0 + PART * 64;
+            while (o.col < k0 + kSuper) {
+                const uint32_t kk = o.col - lo_k;              // wraps around for entries below this half
+                if (kk < 64u) {
+                    const uint32_t v2 = (o.ent >> 16) << ((kk & 1u) * 16u);
+                    switch (kk >> 1) {
+#define XFP_OUT_CASE(i) case i: asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[i]) : "r"(v2)); break;
+                        XFP_OUT_CASE(0) XFP_OUT_CASE(1) XFP_OUT_CASE(2) XFP_OUT_CASE(3) XFP_OUT_CASE(4) XFP_OUT_CASE(5)
+                        XFP_OUT_CASE(6) XFP_OUT_CASE(7) XFP_OUT_CASE(8) XFP_OUT_CASE(9) XFP_OUT_CASE(10) XFP_OUT_CASE(11)
+                        XFP_OUT_CASE(12) XFP_OUT_CASE(13) XFP_OUT_CASE(14) XFP_OUT_CASE(15) XFP_OUT_CASE(16)
+                        XFP_OUT_CASE(17) XFP_OUT_CASE(18) XFP_OUT_CASE(19) XFP_OUT_CASE(20) XFP_OUT_CASE(21)
+                        XFP_OUT_CASE(22) XFP_OUT_CASE(23) XFP_OUT_CASE(24) XFP_OUT_CASE(25) XFP_OUT_CASE(26)
+                        XFP_OUT_CASE(27) XFP_OUT_CASE(28) XFP_OUT_CASE(29) XFP_OUT_CASE(30)
+                        default: asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[31]) : "r"(v2)); break;
+#undef XFP_OUT_CASE
                     }
                 }
-                // W^ = fp16(D16 + S) at the outliers of this channel inside these 8 weights
-                const uint32_t cbase = k0 + PART * 64 + c * 8;
-                while (o.col < cbase + 8) {
-                    const uint32_t kk = o.col - cbase;
-                    const uint32_t v2 = (o.ent >> 16) << ((kk & 1u) * 16u);
-                    if ((kk >> 1) == 0u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c]) : "r"(v2));
-                    if ((kk >> 1) == 1u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c + 1]) : "r"(v2));
-                    if ((kk >> 1) == 2u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c + 2]) : "r"(v2));
-                    if ((kk >> 1) == 3u) asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[4 * c + 3]) : "r"(v2));
-                    o.advance();
-                }
-            };
-            chunk(std::integral_constant<int, 0>{}); chunk(std::integral_constant<int, 1>{});
-            chunk(std::integral_constant<int, 2>{}); chunk(std::integral_constant<int, 3>{});
-            chunk(std::integral_constant<int, 4>{}); chunk(std::integral_constant<int, 5>{});
-            chunk(std::integral_constant<int, 6>{}); chunk(std::integral_constant<int, 7>{});
-            if (PART == 0) while (o.col < k0 + kSuper) o.advance();  // the other warp's half
+                o.advance();
+            }
         } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i) d[i] = 0u;
