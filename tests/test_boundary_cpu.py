@@ -152,6 +152,16 @@ def test_null_alignment_and_size_checks_need_no_gpu(lib):
     assert lib.xfp_gemv_grouped_epilogue(C.byref(da64), 2, a, a, a, 0, 1, n, a, 64, n) == 5
     d128 = _desc(rows=128)
     assert lib.xfp_gemv_grouped_epilogue(C.byref(d128), 2, a, a, a, 0, 1, n, a, 1 << 30, n) == 4     # V2 blobs: not built
+    # prefill form: V2 only, m >= 1, its own workspace size
+    wsz = C.c_size_t()
+    assert lib.xfp_gemm_workspace_size(C.byref(d), 64, C.byref(wsz)) == 0 and wsz.value >= 256
+    assert lib.xfp_gemm_workspace_size(C.byref(d), 0, C.byref(wsz)) == 3
+    assert lib.xfp_gemm_workspace_size(C.byref(da), 64, C.byref(wsz)) == 4                 # V2a: not built
+    assert lib.xfp_gemm(C.byref(d), n, a, 64, a, 0, a, 1 << 30, n) == 1
+    assert lib.xfp_gemm(C.byref(d), a, odd, 64, a, 0, a, 1 << 30, n) == 2
+    assert lib.xfp_gemm(C.byref(d), a, a, 64, a, 3, a, 1 << 30, n) == 3                     # unknown y type
+    assert lib.xfp_gemm(C.byref(d), a, a, 64, a, 0, a, 16, n) == 5
+    assert lib.xfp_gemm(C.byref(da), a, a, 64, a, 0, a, 1 << 30, n) == 4
     assert xfp.xfp_status_str(0) == "ok" and "aligned" in xfp.xfp_status_str(2)
 
 
