@@ -154,7 +154,8 @@ int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* p
  * dequantised tile, GEMM on the tensor cores; the paper's split-M path for many rows of x):
  *     y[t][i] = sum_k W^[i][k] * x[t][k],   W^ = fp16(D16 + S), the matrix xfp_dequant writes,
  * for m >= 1 rows of x in one launch on the tcgen05 tensor cores (fp16 x fp16 products, fp32 accumulation in tensor
- * memory, one rounding of the sum to y_type).  V2 blobs, every N; V2a returns XFP_ERR_UNSUPPORTED.
+ * memory, one rounding of the sum to y_type).  V2 blobs, every N; V2a blobs whose library, replicated once per
+ * shared-memory bank, fits 128 KB (lib_size * 2^bits <= 1024: L = 32 up to N = 5), else XFP_ERR_UNSUPPORTED.
  *   x  [m][cols] fp16;  y  [m][rows] of y_type (XFP_T_F32, XFP_T_F16 or XFP_T_BF16)
  *   workspace  xfp_gemm_workspace_size(desc, m) bytes, zero-filled once before first use; its counter part is left
  *              zero-filled by every call.  Its first 32-bit word is an error flag: the kernel sets it to 1 if one of

@@ -41,6 +41,7 @@ constexpr int kTmemCols = 256;   // [0,128) accumulator, [128,192) and [192,256)
 constexpr int kTmemA = 128;
 constexpr int kAStageCols = 64;  // 128 k as fp16 pairs
 constexpr int kXStages = 3;      // x tiles in flight: the copy of iteration i + 1 is issued at the top of iteration i
+constexpr size_t kV2aTabMax = 128 * 1024;   // V2a: the per-bank library (L * 2^N * 128 bytes) must fit beside the x stages
 constexpr size_t kMinSmem = 80 * 1024;   // at most two CTAs per SM: each holds half of the tensor memory
 
 struct GemmArgs {
@@ -49,6 +50,8 @@ struct GemmArgs {
     int* ctrl;        // [0] error word, [1 + tile] arrival counters of the K slices
     float* partial;   // [tile][slice][T][128]
     int rows, cols, RB, SC, M, ell_slots, ks, sc_per_slice, y_kind;
+    int tab_bytes;    // shared-memory bytes of the look-up tables (the x stages follow)
+    int L;            // V2a: library size
     int b_lbo;        // bytes between consecutive 8-k chunks of the x tile: rows of x per tile * 16
 };
 
@@ -153,7 +156,7 @@ struct Outliers {
 // Barriers: bars[0..1] "products of iteration i done" (i & 1), bars[2..4] "x tile landed" (i % 3), bars[5..6] "A stage
 // of iteration i stored by all eight decode warps" (i & 1).  No CTA-wide barrier inside the loop: a decode warp runs
 // up to two iterations ahead of the products.
-template <int N, int PART>
+template <int N, int MODE, int PART>
 __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok, int q, int lane, int tid, int Tn,
                                           int t0, int sc0, int sc1, const unsigned char* tab, unsigned char* sB,
                                           uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap) {
@@ -171,6 +174,10 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
             }
         }
     }
+    // V2a: library id, scale and mid-point of the lane's channel in the next super-chunk (= group), one ahead
+    const size_t meta0 = ((size_t)rb * a.SC + sc0) * 32 + lane;
+    uint32_t gid_n = 0, gsm_n = 0;
+    if (MODE == 1 && rb_ok) { gid_n = __ldg(a.b.gid + meta0); gsm_n = __ldg(a.b.gsm + meta0); }
     bool ok = true;
     int it = 0;
     for (int sc = sc0; sc < sc1; ++sc, ++it) {
@@ -199,10 +206,30 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                 for (int v = 0; v < H::NV; ++v) nx[1][v] = ld_stream(idx + (size_t)N * 32 + (size_t)(H::V0 + v) * 32);
             }
             // 64 look-ups in one straight block (every load can be in flight at once)
+            float g_scale = 0.f, g_mid = 0.f;
+            uint32_t vbase = tbase;
+            if (MODE == 1) {
+                // D16 = fp16(fp32(scale * lib[id][q] + mid)): the product of two fp16 values is exact in fp32, so the
+                // fused multiply-add rounds once, as the format defines it
+                const __half2 sm = *(const __half2*)&gsm_n;
+                g_scale = __low2float(sm); g_mid = __high2float(sm);
+                vbase = tbase | (gid_n << (7 + N));
+                if (sc + 1 < sc1) {
+                    const size_t mi = meta0 + (size_t)(it + 1) * 32;
+                    gid_n = __ldg(a.b.gid + mi); gsm_n = __ldg(a.b.gsm + mi);
+                }
+            }
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const int p = PART * 32 + i;
-                if (Tab<N>::kPair) {
+                if (MODE == 1) {
+                    const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, vbase));
+                    const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, vbase));
+                    const float f0 = __fmaf_rn(g_scale, __half2float(__ushort_as_half((uint16_t)lo)), g_mid);
+                    const float f1 = __fmaf_rn(g_scale, __half2float(__ushort_as_half((uint16_t)hi)), g_mid);
+                    const __half2 r = __floats2half2_rn(f0, f1);
+                    d[i] = *(const uint32_t*)&r;
+                } else if (Tab<N>::kPair) {
                     d[i] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
                 } else {
                     const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
@@ -286,13 +313,13 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
     return mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
 }
 
-template <int N>
+template <int N, int MODE>
 __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
     constexpr int E = Tab<N>::E;
     constexpr int TW = Tab<N>::T;
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* sTab = smem;                                // [4 row-blocks][TW][32] words
-    unsigned char* sB = smem + (size_t)4 * TW * 128;           // kXStages x tiles of 16 * b_lbo bytes (128-byte aligned)
+    unsigned char* sTab = smem;                                // V2: [4 row-blocks][TW][32] words; V2a: [L * E][32] words
+    unsigned char* sB = smem + a.tab_bytes;           // kXStages x tiles of 16 * b_lbo bytes (128-byte aligned)
     __shared__ __align__(8) uint64_t bars[4 + kXStages];
     __shared__ uint32_t s_tmem;
     __shared__ int s_last;
@@ -320,7 +347,11 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
                      :: "r"(smem_u32(&s_tmem)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    {
+    if (MODE == 1) {
+        // the library, every entry replicated once per bank: word (id * E + q) * 32 + lane
+        const int n = a.L * E;
+        for (int i = warp; i < n; i += kWarps + 1) ((uint32_t*)sTab)[i * 32 + lane] = (uint32_t)__ldg(a.b.cb + i);
+    } else {
         // codebooks -> one word per (entry, lane); pair tables are built from a copy staged in the x stages
         uint32_t* one = Tab<N>::kPair ? (uint32_t*)sB : (uint32_t*)sTab;
         for (int i = warp; i < 4 * E; i += kWarps + 1) {
@@ -372,15 +403,15 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
         o.start(first);
     }
 
-    const unsigned char* tab = sTab + (size_t)q * TW * 128;
+    const unsigned char* tab = MODE == 1 ? sTab : sTab + (size_t)q * TW * 128;
     bool done;
     if (warp == kWarps) {
         done = lane != 0 || mma_loop(a, Tn, t0, sc0, sc1, sB, bars, tmem, &tmap);
         __syncwarp();
     } else {
         done = part == 0
-            ? main_loop<N, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap)
-            : main_loop<N, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap);
+            ? main_loop<N, MODE, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap)
+            : main_loop<N, MODE, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap);
     }
     const bool failed = __syncthreads_or(!done) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -418,14 +449,24 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const float* p0 = a.partial + (size_t)tile * a.ks * kMaxT * kTileRows;
-    for (int i = tid; i < Tn * kTileRows; i += kThreads) {
-        const int t = i / kTileRows, r = i % kTileRows;
+    // four consecutive channels of one row of x per thread and step: 16-byte loads, all slices of a step in flight
+    const float4* p0 = (const float4*)(a.partial + (size_t)tile * a.ks * kMaxT * kTileRows);
+    constexpr int kQuads = kTileRows / 4;
+    for (int i = tid; i < Tn * kQuads; i += kThreads) {
+        const int t = i / kQuads, r = (i % kQuads) * 4;
         const int orow = blockIdx.x * kTileRows + r;
         if (t0 + t >= a.M || orow >= a.rows) continue;
-        float sum = 0.f;
-        for (int z = 0; z < a.ks; ++z) sum += __ldcg(p0 + (size_t)z * kMaxT * kTileRows + i);
-        put_y(a.y, (size_t)(t0 + t) * a.rows + orow, sum, a.y_kind);
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int z = 0; z < a.ks; ++z) {
+            const float4 v = __ldcg(p0 + (size_t)z * (kMaxT * kQuads) + i);
+            sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+        }
+        const size_t o0 = (size_t)(t0 + t) * a.rows + orow;
+        put_y(a.y, o0, sum.x, a.y_kind);
+        if (orow + 1 < a.rows) put_y(a.y, o0 + 1, sum.y, a.y_kind);
+        if (orow + 2 < a.rows) put_y(a.y, o0 + 2, sum.z, a.y_kind);
+        if (orow + 3 < a.rows) put_y(a.y, o0 + 3, sum.w, a.y_kind);
     }
 }
 
@@ -459,11 +500,12 @@ Plan plan_of(const Layout& l, int M) {
     return p;
 }
 
-template <int N>
+template <int N, int MODE>
 cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     const int tmax = c.M >= kMaxT ? kMaxT : (c.M + 15) & ~15;    // rows of x in the largest tile of this launch
     const int b_lbo = tmax * 16;
-    size_t smem = (size_t)4 * Tab<N>::T * 128 + (size_t)kXStages * 16 * b_lbo;
+    const size_t tab_bytes = MODE == 1 ? (size_t)l.L * Tab<N>::E * 128 : (size_t)4 * Tab<N>::T * 128;
+    size_t smem = tab_bytes + (size_t)kXStages * 16 * b_lbo;
     if (smem < kMinSmem) smem = kMinSmem;
     // x [M][K] fp16 seen as [K/8][M][8]: one box {8, tmax, 16} is a whole x tile in the core-matrix order of the B operand
     static const EncodeTiledFn encode = encode_tiled_fn();
@@ -482,8 +524,8 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        const size_t most = (size_t)4 * Tab<N>::T * 128 + (size_t)kXStages * 16 * kMaxT * 16;
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        const size_t most = (MODE == 1 ? kV2aTabMax : (size_t)4 * Tab<N>::T * 128) + (size_t)kXStages * 16 * kMaxT * 16;
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(most < kMinSmem ? kMinSmem : most));
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
@@ -496,14 +538,16 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.partial = (float*)((char*)c.workspace + gemm_ctrl_bytes(l, c.M));
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
     a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_lbo = b_lbo;
-    gemm_tc_kernel<N><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kThreads, smem, s>>>(a, tmap);
+    a.tab_bytes = (int)tab_bytes; a.L = l.L;
+    gemm_tc_kernel<N, MODE><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kThreads, smem, s>>>(a, tmap);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 bool gemm_tc_supported(const Layout& l, int M) {
-    return l.mode == 0 && M >= 1 && (long long)((M + kMaxT - 1) / kMaxT) <= 65535;
+    if (M < 1 || (long long)((M + kMaxT - 1) / kMaxT) > 65535) return false;
+    return l.mode == 0 || (size_t)l.L * l.E * 128 <= kV2aTabMax;
 }
 
 size_t gemm_ctrl_bytes(const Layout& l, int M) {
@@ -518,12 +562,21 @@ size_t gemm_workspace_bytes(const Layout& l, int M) {
 }
 
 cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s) {
+    if (l.mode == 1) {
+        switch (l.bits) {
+            case 2: return launch_n<2, 1>(l, c, s);
+            case 3: return launch_n<3, 1>(l, c, s);
+            case 4: return launch_n<4, 1>(l, c, s);
+            case 5: return launch_n<5, 1>(l, c, s);
+            default: return launch_n<6, 1>(l, c, s);
+        }
+    }
     switch (l.bits) {
-        case 2: return launch_n<2>(l, c, s);
-        case 3: return launch_n<3>(l, c, s);
-        case 4: return launch_n<4>(l, c, s);
-        case 5: return launch_n<5>(l, c, s);
-        default: return launch_n<6>(l, c, s);
+        case 2: return launch_n<2, 0>(l, c, s);
+        case 3: return launch_n<3, 0>(l, c, s);
+        case 4: return launch_n<4, 0>(l, c, s);
+        case 5: return launch_n<5, 0>(l, c, s);
+        default: return launch_n<6, 0>(l, c, s);
     }
 }
 

@@ -41,8 +41,8 @@
         outliers for V2a): device time of every stage (statistics, extraction, Lloyd, LibFit, residual,
         cosine, median) and wall time of the whole xfp_quantize call with BITS as its only candidate.
 
-    python -m paper_2605_14844_b200.probe gemm ROWS COLS BITS RATE M [M ...] [launch]
-        the prefill form (xfp_gemm, tcgen05 tensor cores) on one V2 matrix for every M given: microseconds per call
+    python -m paper_2605_14844_b200.probe gemm|gemm_v2a ROWS COLS BITS RATE M [M ...] [launch]
+        the prefill form (xfp_gemm, tcgen05 tensor cores) on one V2 (gemm) or V2a (gemm_v2a, L = 32) matrix for every M given: microseconds per call
         over distinct packed copies (more than twice the L2), effective GB/s over the algorithmic bytes, TFLOP/s, and
         beside it a library fp16 GEMM (torch.matmul) on the dequantised matrix.  With `launch` as last word: three
         calls of the first M with an L2 flush before each (the target of ncu captures).
@@ -436,9 +436,9 @@ def quant(mode, rows, cols, bits, reps=3):
                           Mweights_per_s=round(rows * cols / np.median(walls) / 1e3, 1))), flush=True)
 
 
-def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=10):
+def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=10, mode=0):
     from . import xfp_gemm, xfp_gemm_workspace_size
-    q = synth.random_quantized(0, rows, cols, bits, rate, seed=1)
+    q = synth.random_quantized(mode, rows, cols, bits, rate, seed=1)
     if launch_only:
         pm = pack_tensors(q, col_bits=16)
         m = ms[0]
@@ -488,16 +488,17 @@ def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=10):
         nb = nb0 + m * (cols * 2 + rows * 2)
         fl = 2.0 * m * rows * cols
         err = max(int(ws[:4].view(torch.int32).item()) for ws in wss)
-        print(json.dumps(dict(rows=rows, cols=cols, bits=bits, rate=rate, M=m, copies=copies, us_per_call=round(t, 2),
+        print(json.dumps(dict(mode=mode, rows=rows, cols=cols, bits=bits, rate=rate, M=m, copies=copies, us_per_call=round(t, 2),
                               GBs=round(nb / t / 1e3, 1), TFLOPs=round(fl / t / 1e6, 1),
                               lib_fp16_gemm_us=round(t_lib, 2), err_flag=err)), flush=True)
 
 
 def main(argv):
-    if len(argv) > 1 and argv[1] == "gemm":
+    if len(argv) > 1 and argv[1] in ("gemm", "gemm_v2a"):
         lo = argv[-1] == "launch"
         rest = argv[6:-1] if lo else argv[6:]
-        gemm(int(argv[2]), int(argv[3]), int(argv[4]), float(argv[5]), [int(v) for v in rest], lo)
+        gemm(int(argv[2]), int(argv[3]), int(argv[4]), float(argv[5]), [int(v) for v in rest], lo,
+             mode=1 if argv[1] == "gemm_v2a" else 0)
         return 0
     if len(argv) > 1 and argv[1] == "packdq":
         packdq(int(argv[2]), int(argv[3]), int(argv[4]), int(argv[5]), float(argv[6]))

@@ -156,12 +156,14 @@ def test_null_alignment_and_size_checks_need_no_gpu(lib):
     wsz = C.c_size_t()
     assert lib.xfp_gemm_workspace_size(C.byref(d), 64, C.byref(wsz)) == 0 and wsz.value >= 256
     assert lib.xfp_gemm_workspace_size(C.byref(d), 0, C.byref(wsz)) == 3
-    assert lib.xfp_gemm_workspace_size(C.byref(da), 64, C.byref(wsz)) == 4                 # V2a: not built
+    assert lib.xfp_gemm_workspace_size(C.byref(da), 64, C.byref(wsz)) == 0
+    dbig = _desc(mode=1, lib_size=64, bits=6)
+    assert lib.xfp_gemm_workspace_size(C.byref(dbig), 64, C.byref(wsz)) == 4               # library too large for the per-bank table
     assert lib.xfp_gemm(C.byref(d), n, a, 64, a, 0, a, 1 << 30, n) == 1
     assert lib.xfp_gemm(C.byref(d), a, odd, 64, a, 0, a, 1 << 30, n) == 2
     assert lib.xfp_gemm(C.byref(d), a, a, 64, a, 3, a, 1 << 30, n) == 3                     # unknown y type
     assert lib.xfp_gemm(C.byref(d), a, a, 64, a, 0, a, 16, n) == 5
-    assert lib.xfp_gemm(C.byref(da), a, a, 64, a, 0, a, 1 << 30, n) == 4
+    assert lib.xfp_gemm(C.byref(dbig), a, a, 64, a, 0, a, 1 << 30, n) == 4
     assert xfp.xfp_status_str(0) == "ok" and "aligned" in xfp.xfp_status_str(2)
 
 

@@ -53,11 +53,11 @@ def _check(q, pm, x16, dtype=torch.float32):
     return y
 
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6])
+@pytest.mark.parametrize("mode,bits", [(0, 2), (0, 3), (0, 4), (0, 5), (0, 6), (1, 2), (1, 3), (1, 4), (1, 5)])
 @pytest.mark.parametrize("m", [1, 16, 37, 128, 200])
-def test_gemm_small(bits, m):
+def test_gemm_small(mode, bits, m):
     # 70 channels: one tile with a ragged row-block and a missing one; 640 columns: five super-chunks, cut along K
-    q = synth.random_quantized(0, 70, 640, bits, 0.02, seed=900 + bits)
+    q = synth.random_quantized(mode, 70, 640, bits, 0.02, seed=900 + bits + 10 * mode)
     pm = xfp.pack_tensors(q, col_bits=16 if bits % 2 else 32)
     _check(q, pm, synth.activations(m, q.cols, seed=11 + m))
 
@@ -70,6 +70,17 @@ def test_gemm_shapes(rows, cols, bits, rate):
     pm = xfp.pack_tensors(q)
     for m in (24, 130):
         _check(q, pm, synth.activations(m, cols, seed=5 + m))
+
+
+@pytest.mark.parametrize("rows,cols,bits,L,rate", [(3072, 4096, 3, 32, 0.001), (4096, 1536, 3, 32, 0.001),
+                                                    (300, 1536, 4, 32, 0.01), (96, 12288, 5, 32, 0.01),
+                                                    (640, 2048, 2, 256, 0.02), (33, 128, 4, 1, 0.0)])
+def test_gemm_v2a_shapes(rows, cols, bits, L, rate):
+    """V2a: the routed experts' two projections, K slices, a ragged tile, the largest and the smallest library."""
+    q = synth.random_quantized(1, rows, cols, bits, rate, seed=rows + cols + bits, lib_size=L)
+    pm = xfp.pack_tensors(q)
+    for m in (24, 130):
+        _check(q, pm, synth.activations(m, cols, seed=7 + m))
 
 
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
@@ -103,10 +114,10 @@ def test_gemm_matches_gemv_rows_and_is_deterministic():
 
 
 def test_gemm_rejects():
-    q = synth.random_quantized(1, 64, 256, 4, 0.0, seed=1)
+    q = synth.random_quantized(1, 64, 256, 6, 0.0, seed=1)
     pm = xfp.pack_tensors(q)
     with pytest.raises(xfp.XfpError):
-        xfp.xfp_gemm_workspace_size(pm.desc, 16)      # V2a: not built
+        xfp.xfp_gemm_workspace_size(pm.desc, 16)      # V2a, N = 6, L = 32: the per-bank library does not fit
     q = synth.random_quantized(0, 64, 256, 4, 0.0, seed=1)
     pm = xfp.pack_tensors(q)
     x = torch.zeros((16, 256), dtype=torch.float16, device="cuda")
