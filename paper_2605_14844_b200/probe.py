@@ -436,7 +436,7 @@ def quant(mode, rows, cols, bits, reps=3):
                           Mweights_per_s=round(rows * cols / np.median(walls) / 1e3, 1))), flush=True)
 
 
-def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=10, mode=0):
+def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=20, mode=0):
     from . import xfp_gemm, xfp_gemm_workspace_size
     q = synth.random_quantized(mode, rows, cols, bits, rate, seed=1)
     if launch_only:
@@ -465,9 +465,13 @@ def gemm(rows, cols, bits, rate, ms, launch_only=False, reps=10, mode=0):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=s):
                 fn()
-            for _ in range(3):
-                g.replay()
-            s.synchronize()
+            # replay for half a second first: the SM clock needs tens of milliseconds of load to leave its idle state
+            import time
+            t_end = time.time() + 0.5
+            while time.time() < t_end:
+                for _ in range(10):
+                    g.replay()
+                s.synchronize()
             ts = []
             for _ in range(reps):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -4,6 +4,8 @@ Every row of x is one GEMV of the oracle: |y_ti - y_ref_ti| <= 1e-3 * sum_k |W_i
 the dequantised matrix W^ = fp16(D16 + S) (exact fp16 products, fp32 accumulation), so it is also held, far more
 tightly, to an fp64 product with the oracle's dequantised matrix.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -124,3 +126,25 @@ def test_gemm_rejects():
     y = torch.zeros((16, 64), dtype=torch.float32, device="cuda")
     with pytest.raises(xfp.XfpError):
         xfp.xfp_gemm(pm.desc, pm.packed, x, y, torch.zeros(16, dtype=torch.uint8, device="cuda"))   # workspace too small
+
+
+def _random_case(rng):
+    mode = int(rng.integers(0, 2))
+    bits = int(rng.integers(2, 7 if mode == 0 else 6))
+    rows = int(rng.choice([1, 31, 32, 97, 128, 129, 260, 511, 1000]))
+    cols = 128 * int(rng.choice([1, 2, 3, 5, 8, 13, 24]))
+    rate = float(rng.choice([0.0, 0.001, 0.01, 0.05]))
+    placement = str(rng.choice(["uniform", "clustered", "one_row"]))
+    m = int(rng.choice([1, 2, 15, 16, 17, 100, 128, 129, 257]))
+    L = int(rng.choice([1, 7, 32])) if mode else 32
+    return mode, bits, rows, cols, rate, placement, m, L
+
+
+@pytest.mark.parametrize("i", range(int(os.environ.get("XFP_GEMM_SWEEP_CASES", "32"))))
+def test_gemm_randomized(i):
+    """Seeded random shapes, bit widths, outlier rates and placements, library sizes and numbers of rows of x."""
+    rng = np.random.default_rng(int(os.environ.get("XFP_SWEEP_SEED", "2605")) * 1000 + i)
+    mode, bits, rows, cols, rate, placement, m, L = _random_case(rng)
+    q = synth.random_quantized(mode, rows, cols, bits, rate, seed=7000 + i, placement=placement, lib_size=L)
+    pm = xfp.pack_tensors(q, col_bits=16 if i % 2 else 32)
+    _check(q, pm, synth.activations(m, cols, seed=8000 + i), [torch.float32, torch.float32, torch.float16][i % 3])
