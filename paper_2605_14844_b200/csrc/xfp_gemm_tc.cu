@@ -6,17 +6,22 @@
 // tensor memory; the x tile is the B operand in shared memory, brought there by one bulk tensor copy (TMA) per
 // stage; the fp32 accumulator is a second tensor-memory region.
 //
-//   CTA      128 output channels (four row-blocks) x up to 128 rows of x x one K slice; 8 warps; two CTAs per SM
-//            (256 of the 512 tensor-memory columns each: 128 accumulator columns, two A stages of 64).
+//   CTA      128 output channels (four row-blocks) x up to 128 rows of x x one K slice; eight decode warps and a
+//            ninth that issues the tensor copies and the products; two CTAs per SM (256 of the 512 tensor-memory
+//            columns each: 128 accumulator columns, two A stages of 64).
 //   stage    one super-chunk (128 k): A = W^[128][128] fp16 in tensor memory, B = x[T][128] fp16 in shared memory,
 //            K-major in the plain (unswizzled) core-matrix layout: element (t, k) at (k/8)*LBO + t*16 + (k%8)*2,
 //            which is what a tensor copy with the box {8 k, T rows, 16 chunks} of x viewed as [K/8][M][8] writes.
-//   decode   warp (row-block, half of the super-chunk): index vectors prefetched one super-chunk ahead, look-ups
-//            in per-lane shared-memory tables (pair tables up to N = 3, one entry per index above) into 32
-//            registers; the outliers of the lane's channel that fall into a group of 8 weights are added there
-//            with one correctly rounded fp16 addition each, so the tile is the matrix xfp_dequant writes.
-//   mma      one thread issues eight m128 nT k16 instructions per stage and commits them to an mbarrier; the
-//            decode of iteration i waits for the products of iteration i - 2, whose operands it overwrites.
+//   decode   warp (row-block, half of the super-chunk): index vectors prefetched two super-chunks ahead, 64
+//            look-ups in one straight block into 32 registers.  V2: per-lane shared-memory tables (pair tables up
+//            to N = 3, one entry per index above).  V2a: the library replicated once per bank, then
+//            D16 = fp16(fp32(scale * lib[id][q] + mid)) with the group's scale and mid-point.  The outliers of the
+//            lane's channel that fall into its half are added to the register that holds them with one correctly
+//            rounded fp16 addition each, so the tile is the matrix xfp_dequant writes.
+//   mma      one thread waits for "A stage stored" (eight arrivals) and "x tile landed" (transaction bytes), issues
+//            eight m128 nT k16 instructions and commits them to a "products done" mbarrier; the decode of
+//            iteration i waits for the products of iteration i - 2, whose A stage it overwrites.  No CTA-wide
+//            barrier inside the loop.
 //   epilogue tcgen05.ld (lane = channel, registers = rows of x), direct store, or fp32 partials through the
 //            workspace when K is cut (few row tiles): the last CTA of a tile adds the slices in slice order.
 // Every wait on an mbarrier has an iteration limit; when one runs out the CTA stops issuing work, records it in
