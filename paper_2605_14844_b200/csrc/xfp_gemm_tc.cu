@@ -249,17 +249,22 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                 const uint32_t kk = o.col - lo_k;              // wraps around for entries below this half
                 if (kk < 64u) {
                     const uint32_t v2 = (o.ent >> 16) << ((kk & 1u) * 16u);
-                    switch (kk >> 1) {
-#define XFP_OUT_CASE(i) case i: asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[i]) : "r"(v2)); break;
-                        XFP_OUT_CASE(0) XFP_OUT_CASE(1) XFP_OUT_CASE(2) XFP_OUT_CASE(3) XFP_OUT_CASE(4) XFP_OUT_CASE(5)
-                        XFP_OUT_CASE(6) XFP_OUT_CASE(7) XFP_OUT_CASE(8) XFP_OUT_CASE(9) XFP_OUT_CASE(10) XFP_OUT_CASE(11)
-                        XFP_OUT_CASE(12) XFP_OUT_CASE(13) XFP_OUT_CASE(14) XFP_OUT_CASE(15) XFP_OUT_CASE(16)
-                        XFP_OUT_CASE(17) XFP_OUT_CASE(18) XFP_OUT_CASE(19) XFP_OUT_CASE(20) XFP_OUT_CASE(21)
-                        XFP_OUT_CASE(22) XFP_OUT_CASE(23) XFP_OUT_CASE(24) XFP_OUT_CASE(25) XFP_OUT_CASE(26)
-                        XFP_OUT_CASE(27) XFP_OUT_CASE(28) XFP_OUT_CASE(29) XFP_OUT_CASE(30)
-                        default: asm("add.rn.f16x2 %0, %0, %1;" : "+r"(d[31]) : "r"(v2)); break;
-#undef XFP_OUT_CASE
-                    }
+                    // the register that holds weight kk: found by nested tests, not a switch -- a jump table
+                    // sends every lane down its own copy of the loop and the lanes of a warp then take their
+                    // trips one after the other instead of together
+                    const uint32_t r = kk >> 1;
+#define XFP_OUT_GROUP(g)                                                                                          \
+    if ((r >> 2) == g##u)                                                                                         \
+        asm("{\n\t.reg .pred p0, p1, p2, p3;\n\t"                                                                 \
+            "setp.eq.u32 p0, %4, 0;\n\tsetp.eq.u32 p1, %4, 1;\n\t"                                                 \
+            "setp.eq.u32 p2, %4, 2;\n\tsetp.eq.u32 p3, %4, 3;\n\t"                                                 \
+            "@p0 add.rn.f16x2 %0, %0, %5;\n\t@p1 add.rn.f16x2 %1, %1, %5;\n\t"                                     \
+            "@p2 add.rn.f16x2 %2, %2, %5;\n\t@p3 add.rn.f16x2 %3, %3, %5;\n\t}"                                    \
+            : "+r"(d[4 * g]), "+r"(d[4 * g + 1]), "+r"(d[4 * g + 2]), "+r"(d[4 * g + 3])                          \
+            : "r"(r & 3u), "r"(v2));
+                    XFP_OUT_GROUP(0) XFP_OUT_GROUP(1) XFP_OUT_GROUP(2) XFP_OUT_GROUP(3)
+                    XFP_OUT_GROUP(4) XFP_OUT_GROUP(5) XFP_OUT_GROUP(6) XFP_OUT_GROUP(7)
+#undef XFP_OUT_GROUP
                 }
                 o.advance();
             }
