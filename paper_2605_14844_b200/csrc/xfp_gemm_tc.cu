@@ -8,7 +8,8 @@
 //
 //   CTA      128 output channels (four row-blocks) x up to 128 rows of x x one K slice; eight decode warps and a
 //            ninth that issues the tensor copies and the products; two CTAs per SM (256 of the 512 tensor-memory
-//            columns each: 128 accumulator columns, two A stages of 64).
+//            columns each: 128 accumulator columns, two A stages of 64).  For many rows of x (see plan_of) the tile
+//            is 256 rows: 256 accumulator columns, all 512 columns, one CTA per SM.
 //   stage    one super-chunk (128 k): A = W^[128][128] fp16 in tensor memory, B = x[T][128] fp16 in shared memory,
 //            K-major in the plain (unswizzled) core-matrix layout: element (t, k) at (k/8)*LBO + t*16 + (k%8)*2,
 //            which is what a tensor copy with the box {8 k, T rows, 16 chunks} of x viewed as [K/8][M][8] writes.
@@ -38,16 +39,17 @@ namespace xfp {
 namespace {
 
 constexpr int kTileRows = 128;   // output channels per CTA (the M of the instruction)
-constexpr int kMaxT = 128;       // rows of x per CTA (the N of the instruction), a multiple of 16
+constexpr int kSmallT = 128;     // rows of x per CTA (the N of the instruction): 128 with two CTAs per SM, or
+constexpr int kBigT = 256;       // 256 with one (more than 128 rows of x: the weights are decoded once per 256 rows)
 constexpr int kWarps = 8;        // decode warps; warp 8 issues the tensor copies and the products
 constexpr int kThreads = (kWarps + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int kTmemCols = 256;   // [0,128) accumulator, [128,192) and [192,256) the two A stages
-constexpr int kTmemA = 128;
+// tensor memory of a CTA: the accumulator (128 or 256 columns), then the two A stages: 256 or 512 columns
 constexpr int kAStageCols = 64;  // 128 k as fp16 pairs
 constexpr int kXStages = 3;      // x tiles in flight: the copy of iteration i + 1 is issued at the top of iteration i
 constexpr size_t kV2aTabMax = 128 * 1024;   // V2a: the per-bank library (L * 2^N * 128 bytes) must fit beside the x stages
-constexpr size_t kMinSmem = 80 * 1024;   // at most two CTAs per SM: each holds half of the tensor memory
+constexpr size_t kMinSmem = 80 * 1024;   // at most two CTAs per SM: each holds half of the tensor memory (a CTA with
+                                         // 256-row tiles holds all of it and asks for more than half of the shared memory)
 
 struct GemmArgs {
     Blob b;
@@ -57,6 +59,9 @@ struct GemmArgs {
     int rows, cols, RB, SC, M, ell_slots, ks, sc_per_slice, y_kind;
     int tab_bytes;    // shared-memory bytes of the look-up tables (the x stages follow)
     int L;            // V2a: library size
+    int maxT;         // rows of x per tile: kSmallT or kBigT; the accumulator's columns and the first column of the A stages
+    int tmem_cols;    // tensor-memory columns of the CTA: 2 * maxT
+    int x_stages;     // x tiles in shared memory: kXStages, or 2 when three large ones do not fit
     int b_lbo;        // bytes between consecutive 8-k chunks of the x tile: rows of x per tile * 16
 };
 
@@ -272,7 +277,7 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
 #pragma unroll
             for (int i = 0; i < 32; ++i) d[i] = 0u;
         }
-        const uint32_t ta = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kTmemA + s * kAStageCols + PART * 32);
+        const uint32_t ta = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(a.maxT + s * kAStageCols + PART * 32);
         tmem_st16<0>(ta, d);
         tmem_st16<16>(ta + 16, d);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -300,24 +305,27 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
             :: "r"(smem_u32(sB + xs * b_stage)), "l"(tmap), "r"(0), "r"(t0), "r"(sc * 16), "r"(bar) : "memory");
     };
     stage_x(sc0, 0);
-    int it = 0, xs = 0;                       // xs = it % kXStages
+    int it = 0, xs = 0;                       // xs = it % x_stages
+    uint32_t xuse = 0;                        // it / x_stages
     for (int sc = sc0; sc < sc1; ++sc, ++it) {
         const int s = it & 1;
-        const int xn = xs + 1 == kXStages ? 0 : xs + 1;
-        // the x stage refilled now was read by the products of iteration it - 2
-        if (it >= 2 && !mbar_wait(smem_u32(&bars[s]), (uint32_t)((it >> 1) - 1) & 1u)) return false;
+        const int xn = xs + 1 == a.x_stages ? 0 : xs + 1;
+        // the x stage refilled now was read by the products of iteration it + 1 - x_stages
+        const int jf = it + 1 - a.x_stages;
+        if (jf >= 0 && !mbar_wait(smem_u32(&bars[jf & 1]), (uint32_t)(jf >> 1) & 1u)) return false;
         if (sc + 1 < sc1) stage_x(sc + 1, xn);
         if (!mbar_wait(smem_u32(&bars[5 + s]), (uint32_t)(it >> 1) & 1u)) return false;          // A stage stored
-        if (!mbar_wait(smem_u32(&bars[2 + xs]), (uint32_t)(it / kXStages) & 1u)) return false;   // x tile landed
+        if (!mbar_wait(smem_u32(&bars[2 + xs]), xuse & 1u)) return false;   // x tile landed
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t b0 = smem_u32(sB + xs * b_stage);
 #pragma unroll
         for (int ks = 0; ks < kSuper / 16; ++ks) {
             const uint64_t db = smem_desc(b0 + 2 * ks * a.b_lbo, (uint32_t)a.b_lbo, 128);
-            umma_f16_ts(tmem, tmem + (uint32_t)(kTmemA + s * kAStageCols + ks * 8), db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+            umma_f16_ts(tmem, tmem + (uint32_t)(a.maxT + s * kAStageCols + ks * 8), db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(smem_u32(&bars[s]));
         xs = xn;
+        if (xn == 0) ++xuse;
     }
     const int lastit = it - 1;
     return mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
@@ -339,8 +347,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     const int rb = blockIdx.x * 4 + q;
     const bool rb_ok = rb < a.RB && warp < kWarps;
     const int row = rb * kRowsPerBlock + lane;
-    const int t0 = blockIdx.y * kMaxT;
-    const int Tn = min(kMaxT, (a.M - t0 + 15) & ~15);          // rows of x of this tile, rounded up to 16
+    const int t0 = blockIdx.y * a.maxT;
+    const int Tn = min(a.maxT, (a.M - t0 + 15) & ~15);          // rows of x of this tile, rounded up to 16
     const int sc0 = blockIdx.z * a.sc_per_slice;
     const int sc1 = min(a.SC, sc0 + a.sc_per_slice);
     const int tile = blockIdx.y * gridDim.x + blockIdx.x;
@@ -354,7 +362,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_u32(&s_tmem)), "r"(kTmemCols) : "memory");
+                     :: "r"(smem_u32(&s_tmem)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (MODE == 1) {
@@ -430,7 +438,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     } else {
         // lane = channel (tensor-memory lane 32*(warp%4) + lane), registers = 16 consecutive rows of x
         const int r = q * 32 + lane;
-        float* part_out = a.partial + ((size_t)tile * a.ks + blockIdx.z) * kMaxT * kTileRows;
+        float* part_out = a.partial + ((size_t)tile * a.ks + blockIdx.z) * a.maxT * kTileRows;
         for (int cc = part; warp < kWarps && cc * 16 < Tn; cc += 2) {
             uint32_t v[16];
             tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
@@ -445,7 +453,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(a.tmem_cols) : "memory");
     if (failed || a.ks == 1) return;
 
     // ---- K slices: the last CTA of the tile to arrive adds the slices in slice order ----
@@ -460,7 +468,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     if (!s_last) return;
     __threadfence();
     // four consecutive channels of one row of x per thread and step: 16-byte loads, all slices of a step in flight
-    const float4* p0 = (const float4*)(a.partial + (size_t)tile * a.ks * kMaxT * kTileRows);
+    const float4* p0 = (const float4*)(a.partial + (size_t)tile * a.ks * a.maxT * kTileRows);
     constexpr int kQuads = kTileRows / 4;
     for (int i = tid; i < Tn * kQuads; i += kThreads) {
         const int t = i / kQuads, r = (i % kQuads) * 4;
@@ -469,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
         for (int z = 0; z < a.ks; ++z) {
-            const float4 v = __ldcg(p0 + (size_t)z * (kMaxT * kQuads) + i);
+            const float4 v = __ldcg(p0 + (size_t)z * (a.maxT * kQuads) + i);
             sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
         const size_t o0 = (size_t)(t0 + t) * a.rows + orow;
@@ -495,16 +503,37 @@ EncodeTiledFn encode_tiled_fn() {
 
 struct Plan {
     int row_tiles, tok_tiles, ks, sc_per_slice;
+    int maxT, x_stages;
+    size_t tab_bytes, smem;
 };
+
+constexpr size_t kSmemLimit = 227 * 1024 - 1024;   // dynamic shared memory a CTA may ask for, less the static part
 
 Plan plan_of(const Layout& l, int M) {
     Plan p;
+    p.tab_bytes = l.mode == 1 ? (size_t)l.L * l.E * 128 : (size_t)4 * (l.bits <= 3 ? l.E * l.E : l.E) * 128;
+    // Tiles of 256 rows of x (one CTA per SM, all 512 tensor-memory columns) decode the weights once per 256 rows, but
+    // a lone CTA decodes about half as fast as two: measured faster where the 128-row tiles leave room for one CTA
+    // per SM anyway (V2a from N = 4: 875 -> 637 us at 28672 x 8192, M = 512) and from about a thousand rows of x
+    // (4096 x 4096, M = 2048: 204 -> 185 us), slower below (4096 x 4096, M = 512: 78 -> 89 us).
+    p.maxT = kSmallT; p.x_stages = kXStages;
+    const bool lone_anyway = p.tab_bytes + (size_t)kXStages * 16 * kSmallT * 16 > 113 * 1024;
+    if (M > kSmallT && (lone_anyway || M >= 1024)) {
+        for (int xs = kXStages; xs >= 2; --xs) {
+            if (p.tab_bytes + (size_t)xs * 16 * kBigT * 16 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
+        }
+    }
+    const int tmax = M >= p.maxT ? p.maxT : (M + 15) & ~15;    // rows of x in the largest tile of this launch
+    p.smem = p.tab_bytes + (size_t)p.x_stages * 16 * tmax * 16;
+    if (p.smem < kMinSmem) p.smem = kMinSmem;
+    if (p.maxT == kBigT && p.smem < 120 * 1024) p.smem = 120 * 1024;   // alone on its SM: it holds all 512 columns
     p.row_tiles = (l.RB + 3) / 4;
-    p.tok_tiles = (M + kMaxT - 1) / kMaxT;
+    p.tok_tiles = (M + p.maxT - 1) / p.maxT;
     const int tiles = p.row_tiles * p.tok_tiles;
     int ks = 1;
     // fewer tiles than CTA slots (two per SM): cut K, at least two super-chunks per slice
-    while (tiles * ks * 2 <= 2 * 148 && l.SC / (ks * 2) >= 2) ks *= 2;
+    const int slots = p.maxT == kBigT ? 148 : 2 * 148;
+    while (tiles * ks * 2 <= slots && l.SC / (ks * 2) >= 2) ks *= 2;
     p.sc_per_slice = (l.SC + ks - 1) / ks;
     p.ks = (l.SC + p.sc_per_slice - 1) / p.sc_per_slice;
     return p;
@@ -512,11 +541,10 @@ Plan plan_of(const Layout& l, int M) {
 
 template <int N, int MODE>
 cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
-    const int tmax = c.M >= kMaxT ? kMaxT : (c.M + 15) & ~15;    // rows of x in the largest tile of this launch
+    const Plan p = plan_of(l, c.M);
+    const int tmax = c.M >= p.maxT ? p.maxT : (c.M + 15) & ~15;  // rows of x in the largest tile of this launch
     const int b_lbo = tmax * 16;
-    const size_t tab_bytes = MODE == 1 ? (size_t)l.L * Tab<N>::E * 128 : (size_t)4 * Tab<N>::T * 128;
-    size_t smem = tab_bytes + (size_t)kXStages * 16 * b_lbo;
-    if (smem < kMinSmem) smem = kMinSmem;
+    const size_t tab_bytes = p.tab_bytes, smem = p.smem;
     // x [M][K] fp16 seen as [K/8][M][8]: one box {8, tmax, 16} is a whole x tile in the core-matrix order of the B operand
     static const EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
@@ -534,13 +562,11 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        const size_t most = (MODE == 1 ? kV2aTabMax : (size_t)4 * Tab<N>::T * 128) + (size_t)kXStages * 16 * kMaxT * 16;
         cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(most < kMinSmem ? kMinSmem : most));
+                                             (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
     }
-    const Plan p = plan_of(l, c.M);
     GemmArgs a;
     a.b = blob_at(c.packed, offsets_of(l));
     a.y = c.y;
@@ -549,6 +575,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
     a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_lbo = b_lbo;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
+    a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
     gemm_tc_kernel<N, MODE><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kThreads, smem, s>>>(a, tmap);
     return cudaGetLastError();
 }
@@ -556,7 +583,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
 }  // namespace
 
 bool gemm_tc_supported(const Layout& l, int M) {
-    if (M < 1 || (long long)((M + kMaxT - 1) / kMaxT) > 65535) return false;
+    if (M < 1 || (long long)((M + kSmallT - 1) / kSmallT) > 65535) return false;
     return l.mode == 0 || (size_t)l.L * l.E * 128 <= kV2aTabMax;
 }
 
@@ -567,7 +594,7 @@ size_t gemm_ctrl_bytes(const Layout& l, int M) {
 
 size_t gemm_workspace_bytes(const Layout& l, int M) {
     const Plan p = plan_of(l, M);
-    const size_t partial = p.ks > 1 ? (size_t)p.row_tiles * p.tok_tiles * p.ks * kMaxT * kTileRows * 4 : 0;
+    const size_t partial = p.ks > 1 ? (size_t)p.row_tiles * p.tok_tiles * p.ks * p.maxT * kTileRows * 4 : 0;
     return gemm_ctrl_bytes(l, M) + partial;
 }
 

@@ -30,7 +30,7 @@ def _run(q, pm, x16, dtype=torch.float32):
     torch.cuda.synchronize()
     words = ws[: (ws.numel() // 4) * 4].view(torch.int32)
     assert int(words[0].item()) == 0, "a bounded wait ran out in the kernel"
-    n_ctrl = min(words.numel(), 1 + ((q.rows + 127) // 128) * ((m + 127) // 128))
+    n_ctrl = min(words.numel(), 1 + ((q.rows + 127) // 128) * ((m + 255) // 256))   # at least this many counters
     assert int(words[:n_ctrl].abs().sum().item()) == 0, "slice counters not left at zero"
     return y, ws, xd
 
