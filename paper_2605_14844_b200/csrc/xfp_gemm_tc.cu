@@ -28,6 +28,7 @@
 // Every wait on an mbarrier has an iteration limit; when one runs out the CTA stops issuing work, records it in
 // the first word of the workspace and leaves through the common exit that frees its tensor memory.
 #include <cuda.h>
+#include <cstdlib>
 
 #include <type_traits>
 
@@ -41,8 +42,10 @@ namespace {
 constexpr int kTileRows = 128;   // output channels per CTA (the M of the instruction)
 constexpr int kSmallT = 128;     // rows of x per CTA (the N of the instruction): 128 with two CTAs per SM, or
 constexpr int kBigT = 256;       // 256 with one (more than 128 rows of x: the weights are decoded once per 256 rows)
-constexpr int kWarps = 8;        // decode warps; warp 8 issues the tensor copies and the products
-constexpr int kThreads = (kWarps + 1) * 32;
+constexpr int kWarps = 8;        // decode warps of one group (row-block x half); the warp behind the last group issues
+                                 // the tensor copies and the products.  256-row tiles (one CTA per SM) run two groups:
+                                 // group g decodes the iterations with it % 2 == g, i.e. owns A stage g
+constexpr int threads_of(bool big) { return ((big ? 2 : 1) * kWarps + 1) * 32; }
 constexpr uint32_t kSpinLimit = 1u << 22;
 // tensor memory of a CTA: the accumulator (128 or 256 columns), then the two A stages: 256 or 512 columns
 constexpr int kAStageCols = 64;  // 128 k as fp16 pairs
@@ -169,28 +172,31 @@ struct Outliers {
 template <int N, int MODE, int PART>
 __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok, int q, int lane, int tid, int Tn,
                                           int t0, int sc0, int sc1, const unsigned char* tab, unsigned char* sB,
-                                          uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap) {
+                                          uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap,
+                                          int grp, int G) {
     using H = Half<N, PART>;
     const uint32_t tbase = (uint32_t)lane * 4u;
-    const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0) * N * 32 + lane;   // advanced by N*32 per super-chunk
+    const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0 + grp) * N * 32 + lane;   // advanced by G*N*32 per iteration of this warp
     // index vectors of the next two super-chunks in registers
     uint4 nx[2][H::NV];
     if (rb_ok) {
 #pragma unroll
         for (int ahead = 0; ahead < 2; ++ahead) {
-            if (sc0 + ahead < sc1) {
+            if (sc0 + grp + ahead * G < sc1) {
 #pragma unroll
-                for (int v = 0; v < H::NV; ++v) nx[ahead][v] = ld_stream(idx + (size_t)ahead * N * 32 + (size_t)(H::V0 + v) * 32);
+                for (int v = 0; v < H::NV; ++v) nx[ahead][v] = ld_stream(idx + (size_t)ahead * G * N * 32 + (size_t)(H::V0 + v) * 32);
             }
         }
     }
     // V2a: library id, scale and mid-point of the lane's channel in the next super-chunk (= group), one ahead
     const size_t meta0 = ((size_t)rb * a.SC + sc0) * 32 + lane;
     uint32_t gid_n = 0, gsm_n = 0;
-    if (MODE == 1 && rb_ok) { gid_n = __ldg(a.b.gid + meta0); gsm_n = __ldg(a.b.gsm + meta0); }
+    if (MODE == 1 && rb_ok && sc0 + grp < sc1) {
+        gid_n = __ldg(a.b.gid + meta0 + (size_t)grp * 32); gsm_n = __ldg(a.b.gsm + meta0 + (size_t)grp * 32);
+    }
     bool ok = true;
-    int it = 0;
-    for (int sc = sc0; sc < sc1; ++sc, ++it) {
+    int it = grp;
+    for (int sc = sc0 + grp; sc < sc1; sc += G, it += G) {
         const int s = it & 1;
         // The A stage written below was read by the products of iteration it - 2.
         if (it >= 2 && ok) {
@@ -210,10 +216,10 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                 w[4 * (H::V0 + v) + 2] = nx[0][v].z; w[4 * (H::V0 + v) + 3] = nx[0][v].w;
                 nx[0][v] = nx[1][v];
             }
-            idx += N * 32;
-            if (sc + 2 < sc1) {
+            idx += G * N * 32;
+            if (sc + 2 * G < sc1) {
 #pragma unroll
-                for (int v = 0; v < H::NV; ++v) nx[1][v] = ld_stream(idx + (size_t)N * 32 + (size_t)(H::V0 + v) * 32);
+                for (int v = 0; v < H::NV; ++v) nx[1][v] = ld_stream(idx + (size_t)G * N * 32 + (size_t)(H::V0 + v) * 32);
             }
             // 64 look-ups in one straight block (every load can be in flight at once)
             float g_scale = 0.f, g_mid = 0.f;
@@ -224,8 +230,8 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                 const __half2 sm = *(const __half2*)&gsm_n;
                 g_scale = __low2float(sm); g_mid = __high2float(sm);
                 vbase = tbase | (gid_n << (7 + N));
-                if (sc + 1 < sc1) {
-                    const size_t mi = meta0 + (size_t)(it + 1) * 32;
+                if (sc + G < sc1) {
+                    const size_t mi = meta0 + (size_t)(it + G) * 32;
                     gid_n = __ldg(a.b.gid + mi); gsm_n = __ldg(a.b.gsm + mi);
                 }
             }
@@ -286,7 +292,10 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&bars[5 + s])) : "memory");
     }
     // all products of this CTA are complete when the last commit has arrived
-    const int lastit = sc1 - sc0 - 1;
+    // this warp's last iteration: its commit is on the barrier this warp has followed (the other group's is not);
+    // the CTA-wide vote behind the loops then covers the very last commit through the warps that waited for it
+    const int lastit = it - G;
+    if (lastit < 0) return ok;
     return ok && mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
 }
 
@@ -331,8 +340,8 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
     return mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
 }
 
-template <int N, int MODE>
-__global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
+template <int N, int MODE, bool BIG>
+__global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
     constexpr int E = Tab<N>::E;
     constexpr int TW = Tab<N>::T;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -343,9 +352,10 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int q = warp & 3, part = warp >> 2;                  // row-block of the tile, half of the super-chunk
+    constexpr int G = BIG ? 2 : 1, DW = G * kWarps;            // groups, decode warps
+    const int q = warp & 3, part = (warp >> 2) & 1, grp = warp >> 3;   // row-block of the tile, half of the super-chunk, group
     const int rb = blockIdx.x * 4 + q;
-    const bool rb_ok = rb < a.RB && warp < kWarps;
+    const bool rb_ok = rb < a.RB && warp < DW;
     const int row = rb * kRowsPerBlock + lane;
     const int t0 = blockIdx.y * a.maxT;
     const int Tn = min(a.maxT, (a.M - t0 + 15) & ~15);          // rows of x of this tile, rounded up to 16
@@ -368,18 +378,18 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     if (MODE == 1) {
         // the library, every entry replicated once per bank: word (id * E + q) * 32 + lane
         const int n = a.L * E;
-        for (int i = warp; i < n; i += kWarps + 1) ((uint32_t*)sTab)[i * 32 + lane] = (uint32_t)__ldg(a.b.cb + i);
+        for (int i = warp; i < n; i += DW + 1) ((uint32_t*)sTab)[i * 32 + lane] = (uint32_t)__ldg(a.b.cb + i);
     } else {
         // codebooks -> one word per (entry, lane); pair tables are built from a copy staged in the x stages
         uint32_t* one = Tab<N>::kPair ? (uint32_t*)sB : (uint32_t*)sTab;
-        for (int i = warp; i < 4 * E; i += kWarps + 1) {
+        for (int i = warp; i < 4 * E; i += DW + 1) {
             const int qq = i / E, e = i % E, r = (blockIdx.x * 4 + qq) * kRowsPerBlock + lane;
             one[(qq * E + e) * 32 + lane] = (blockIdx.x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
         }
         if (Tab<N>::kPair) {
             __syncthreads();
             uint32_t* tab = (uint32_t*)sTab;
-            for (int i = warp; i < 4 * TW; i += kWarps + 1) {
+            for (int i = warp; i < 4 * TW; i += DW + 1) {
                 const int qq = i / TW, t = i % TW;
                 tab[(qq * TW + t) * 32 + lane] =
                     one[(qq * E + (t & (E - 1))) * 32 + lane] | (one[(qq * E + (t >> N)) * 32 + lane] << 16);
@@ -423,13 +433,13 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
 
     const unsigned char* tab = MODE == 1 ? sTab : sTab + (size_t)q * TW * 128;
     bool done;
-    if (warp == kWarps) {
+    if (warp == DW) {
         done = lane != 0 || mma_loop(a, Tn, t0, sc0, sc1, sB, bars, tmem, &tmap);
         __syncwarp();
     } else {
         done = part == 0
-            ? main_loop<N, MODE, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap)
-            : main_loop<N, MODE, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap);
+            ? main_loop<N, MODE, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap, grp, G)
+            : main_loop<N, MODE, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap, grp, G);
     }
     const bool failed = __syncthreads_or(!done) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -439,7 +449,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
         // lane = channel (tensor-memory lane 32*(warp%4) + lane), registers = 16 consecutive rows of x
         const int r = q * 32 + lane;
         float* part_out = a.partial + ((size_t)tile * a.ks + blockIdx.z) * a.maxT * kTileRows;
-        for (int cc = part; warp < kWarps && cc * 16 < Tn; cc += 2) {
+        for (int cc = part + 2 * grp; warp < DW && cc * 16 < Tn; cc += 2 * G) {
             uint32_t v[16];
             tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
 #pragma unroll
@@ -470,7 +480,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_tc_kernel(const GemmArgs a, 
     // four consecutive channels of one row of x per thread and step: 16-byte loads, all slices of a step in flight
     const float4* p0 = (const float4*)(a.partial + (size_t)tile * a.ks * a.maxT * kTileRows);
     constexpr int kQuads = kTileRows / 4;
-    for (int i = tid; i < Tn * kQuads; i += kThreads) {
+    for (int i = tid; i < Tn * kQuads; i += (DW + 1) * 32) {
         const int t = i / kQuads, r = (i % kQuads) * 4;
         const int orow = blockIdx.x * kTileRows + r;
         if (t0 + t >= a.M || orow >= a.rows) continue;
@@ -518,7 +528,7 @@ Plan plan_of(const Layout& l, int M) {
     // (4096 x 4096, M = 2048: 204 -> 185 us), slower below (4096 x 4096, M = 512: 78 -> 89 us).
     p.maxT = kSmallT; p.x_stages = kXStages;
     const bool lone_anyway = p.tab_bytes + (size_t)kXStages * 16 * kSmallT * 16 > 113 * 1024;
-    if (M > kSmallT && (lone_anyway || M >= 1024)) {
+    if (M > kSmallT && (lone_anyway || M >= 1024 || getenv("XFP_GEMM_BIG"))) {
         for (int xs = kXStages; xs >= 2; --xs) {
             if (p.tab_bytes + (size_t)xs * 16 * kBigT * 16 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
         }
@@ -562,8 +572,11 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<N, MODE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemLimit);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gemm_tc_kernel<N, MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
     }
@@ -576,7 +589,11 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_lbo = b_lbo;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
     a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
-    gemm_tc_kernel<N, MODE><<<dim3((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks), kThreads, smem, s>>>(a, tmap);
+    const dim3 grid((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks);
+    if (p.maxT == kBigT)
+        gemm_tc_kernel<N, MODE, true><<<grid, threads_of(true), smem, s>>>(a, tmap);
+    else
+        gemm_tc_kernel<N, MODE, false><<<grid, threads_of(false), smem, s>>>(a, tmap);
     return cudaGetLastError();
 }
 
