@@ -10,9 +10,9 @@
 //            ninth that issues the tensor copies and the products; two CTAs per SM (256 of the 512 tensor-memory
 //            columns each: 128 accumulator columns, two A stages of 64).  For many rows of x (see plan_of) the tile
 //            is 256 rows: 256 accumulator columns, all 512 columns, one CTA per SM.
-//   stage    one super-chunk (128 k): A = W^[128][128] fp16 in tensor memory, B = x[T][128] fp16 in shared memory,
-//            K-major in the plain (unswizzled) core-matrix layout: element (t, k) at (k/8)*LBO + t*16 + (k%8)*2,
-//            which is what a tensor copy with the box {8 k, T rows, 16 chunks} of x viewed as [K/8][M][8] writes.
+//   stage    one super-chunk (128 k): A = W^[128][128] fp16 in tensor memory, B = x[T][128] fp16 in shared memory as
+//            two K-major halves of 64 k in the 128-byte swizzle, each written by one tensor copy with the box
+//            {64 k, T rows} (128 contiguous bytes per row of x; rows beyond M arrive as zeros).
 //   decode   warp (row-block, half of the super-chunk): index vectors prefetched two super-chunks ahead, 64
 //            look-ups in one straight block into 32 registers.  V2: per-lane shared-memory tables (pair tables up
 //            to N = 3, one entry per index above).  V2a: the library replicated once per bank, then
@@ -28,7 +28,6 @@
 // Every wait on an mbarrier has an iteration limit; when one runs out the CTA stops issuing work, records it in
 // the first word of the workspace and leaves through the common exit that frees its tensor memory.
 #include <cuda.h>
-#include <cstdlib>
 
 #include <type_traits>
 
@@ -65,7 +64,7 @@ struct GemmArgs {
     int maxT;         // rows of x per tile: kSmallT or kBigT; the accumulator's columns and the first column of the A stages
     int tmem_cols;    // tensor-memory columns of the CTA: 2 * maxT
     int x_stages;     // x tiles in shared memory: kXStages, or 2 when three large ones do not fit
-    int b_lbo;        // bytes between consecutive 8-k chunks of the x tile: rows of x per tile * 16
+    int b_half;       // bytes of one 64-k half of an x tile: rows of x per tile * 128 (a multiple of 1024)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -83,11 +82,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 
-// Shared-memory operand descriptor, K-major, no swizzle: start address, byte distance between the two 8-k core
-// matrices of one instruction (leading), byte distance between groups of 8 rows (stride), descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-    return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo >> 4) & 0x3fffu) << 16) |
-           ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46);
+// Shared-memory operand descriptor (version 1) of a K-major tile in the 128-byte swizzle (rows of 64 fp16 = 128 bytes,
+// 16-byte chunk c of row r at chunk c ^ (r & 7), the layout a tensor copy with CU_TENSOR_MAP_SWIZZLE_128B writes; base
+// 1024-byte aligned): groups of 8 rows are 1024 bytes apart, the leading offset is not used (1), layout type 2.  A step of 16 k inside
+// the 128-byte row advances the start address by 32 bytes.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
 // D[128][T] (+)= A[128][16] B[T][16]^T: A from tensor memory (lane = row, column = two k), B from shared memory.
@@ -303,15 +303,19 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
 __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int sc0, int sc1, unsigned char* sB,
                                          uint64_t* bars, uint32_t tmem, const CUtensorMap* tmap) {
     const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
-    const int b_stage = 16 * a.b_lbo;
+    const int b_stage = 2 * a.b_half;
     const uint32_t x_bytes = (uint32_t)b_stage;
     auto stage_x = [&](int sc, int xs) {
-        // one bulk tensor copy: box {8 k, rows of x, 16 chunks} of x viewed as [K/8][M][8]; rows beyond M arrive as zeros
+        // two tensor copies, one per 64-k half: box {64 k, rows of x} of x [M][K], 128-byte rows in the 128-byte swizzle;
+        // rows beyond M arrive as zeros
         const uint32_t bar = smem_u32(&bars[2 + xs]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(x_bytes) : "memory");
-        asm volatile(
-            "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-            :: "r"(smem_u32(sB + xs * b_stage)), "l"(tmap), "r"(0), "r"(t0), "r"(sc * 16), "r"(bar) : "memory");
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                :: "r"(smem_u32(sB + xs * b_stage + h * a.b_half)), "l"(tmap), "r"(sc * kSuper + h * 64), "r"(t0), "r"(bar)
+                : "memory");
     };
     stage_x(sc0, 0);
     int it = 0, xs = 0;                       // xs = it % x_stages
@@ -329,7 +333,7 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
         const uint32_t b0 = smem_u32(sB + xs * b_stage);
 #pragma unroll
         for (int ks = 0; ks < kSuper / 16; ++ks) {
-            const uint64_t db = smem_desc(b0 + 2 * ks * a.b_lbo, (uint32_t)a.b_lbo, 128);
+            const uint64_t db = smem_desc_sw128(b0 + (uint32_t)(ks >> 2) * (uint32_t)a.b_half + (uint32_t)(ks & 3) * 32u);
             umma_f16_ts(tmem, tmem + (uint32_t)(a.maxT + s * kAStageCols + ks * 8), db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(smem_u32(&bars[s]));
@@ -344,9 +348,9 @@ template <int N, int MODE, bool BIG>
 __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
     constexpr int E = Tab<N>::E;
     constexpr int TW = Tab<N>::T;
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* sTab = smem;                                // V2: [4 row-blocks][TW][32] words; V2a: [L * E][32] words
-    unsigned char* sB = smem + a.tab_bytes;           // kXStages x tiles of 16 * b_lbo bytes (128-byte aligned)
+    unsigned char* sB = smem + a.tab_bytes;           // the x stages, two swizzled halves each (1024-byte aligned)
     __shared__ __align__(8) uint64_t bars[4 + kXStages];
     __shared__ uint32_t s_tmem;
     __shared__ int s_last;
@@ -522,13 +526,12 @@ constexpr size_t kSmemLimit = 227 * 1024 - 1024;   // dynamic shared memory a CT
 Plan plan_of(const Layout& l, int M) {
     Plan p;
     p.tab_bytes = l.mode == 1 ? (size_t)l.L * l.E * 128 : (size_t)4 * (l.bits <= 3 ? l.E * l.E : l.E) * 128;
-    // Tiles of 256 rows of x (one CTA per SM, all 512 tensor-memory columns) decode the weights once per 256 rows, but
-    // a lone CTA decodes about half as fast as two: measured faster where the 128-row tiles leave room for one CTA
-    // per SM anyway (V2a from N = 4: 875 -> 637 us at 28672 x 8192, M = 512) and from about a thousand rows of x
-    // (4096 x 4096, M = 2048: 204 -> 185 us), slower below (4096 x 4096, M = 512: 78 -> 89 us).
+    p.tab_bytes = (p.tab_bytes + 1023) & ~size_t(1023);      // the x stages behind the tables are 1024-byte aligned
+    // More than 128 rows of x: tiles of 256 rows (one CTA per SM with two groups of decode warps, all 512 tensor-memory
+    // columns), which decode the weights once per 256 rows -- 28672 x 8192, M = 512: 555 -> 450 us; 4096 x 4096,
+    // M = 512: 80 -> 72 us -- when their x stages fit beside the tables.
     p.maxT = kSmallT; p.x_stages = kXStages;
-    const bool lone_anyway = p.tab_bytes + (size_t)kXStages * 16 * kSmallT * 16 > 113 * 1024;
-    if (M > kSmallT && (lone_anyway || M >= 1024 || getenv("XFP_GEMM_BIG"))) {
+    if (M > kSmallT) {
         for (int xs = kXStages; xs >= 2; --xs) {
             if (p.tab_bytes + (size_t)xs * 16 * kBigT * 16 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
         }
@@ -553,19 +556,19 @@ template <int N, int MODE>
 cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     const Plan p = plan_of(l, c.M);
     const int tmax = c.M >= p.maxT ? p.maxT : (c.M + 15) & ~15;  // rows of x in the largest tile of this launch
-    const int b_lbo = tmax * 16;
+    const int b_half = tmax * 128;
     const size_t tab_bytes = p.tab_bytes, smem = p.smem;
-    // x [M][K] fp16 seen as [K/8][M][8]: one box {8, tmax, 16} is a whole x tile in the core-matrix order of the B operand
+    // x [M][K] fp16: a box of 64 k x tmax rows lands as 128-byte rows in the 128-byte swizzle, the B operand's layout
     static const EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap tmap;
     {
-        const cuuint64_t dims[3] = {8, (cuuint64_t)c.M, (cuuint64_t)(l.cols / 8)};
-        const cuuint64_t strides[2] = {(cuuint64_t)l.cols * 2, 16};
-        const cuuint32_t box[3] = {8, (cuuint32_t)tmax, 16};
-        const cuuint32_t estr[3] = {1, 1, 1};
-        if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t*>(c.x), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+        const cuuint64_t dims[2] = {(cuuint64_t)l.cols, (cuuint64_t)c.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)l.cols * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)tmax};
+        const cuuint32_t estr[2] = {1, 1};
+        if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<uint16_t*>(c.x), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
@@ -586,7 +589,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.ctrl = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + gemm_ctrl_bytes(l, c.M));
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
-    a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_lbo = b_lbo;
+    a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_half = b_half;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
     a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
     const dim3 grid((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks);
