@@ -175,7 +175,8 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                                           uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap,
                                           int grp, int G) {
     using H = Half<N, PART>;
-    const uint32_t tbase = (uint32_t)lane * 4u;
+    // byte offset of the lane inside a table entry; N = 4 (V2): the row-block's half of a 256-byte entry as well
+    const uint32_t tbase = (uint32_t)lane * 4u + ((MODE == 0 && N == 4) ? (uint32_t)(q & 1) * 128u : 0u);
     const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0 + grp) * N * 32 + lane;   // advanced by G*N*32 per iteration of this warp
     // index vectors of the next two super-chunks in registers
     uint4 nx[2][H::NV];
@@ -247,6 +248,14 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                     d[i] = *(const uint32_t*)&r;
                 } else if (Tab<N>::kPair) {
                     d[i] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
+                } else if (N == 4) {
+                    // entries 256 bytes apart (two row-blocks share a table): an index, isolated in its own byte,
+                    // becomes the second byte of the address with one PRMT.  Pair p = byte p & 3 of word p >> 2.
+                    const uint32_t wlo = w[p >> 2] & 0x0f0f0f0fu, whi = (w[p >> 2] >> 4) & 0x0f0f0f0fu;
+                    const uint32_t sel = 0x5504u | ((uint32_t)(p & 3) << 4);
+                    const uint32_t lo = *(const uint32_t*)(tab + __byte_perm(wlo, tbase, sel));
+                    const uint32_t hi = *(const uint32_t*)(tab + __byte_perm(whi, tbase, sel));
+                    d[i] = __byte_perm(lo, hi, 0x5410u);
                 } else {
                     const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
                     const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
@@ -388,7 +397,8 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
         uint32_t* one = Tab<N>::kPair ? (uint32_t*)sB : (uint32_t*)sTab;
         for (int i = warp; i < 4 * E; i += DW + 1) {
             const int qq = i / E, e = i % E, r = (blockIdx.x * 4 + qq) * kRowsPerBlock + lane;
-            one[(qq * E + e) * 32 + lane] = (blockIdx.x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
+            const int slot = N == 4 ? ((qq >> 1) * E + e) * 64 + (qq & 1) * 32 : (qq * E + e) * 32;   // N = 4: see the look-ups
+            one[slot + lane] = (blockIdx.x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
         }
         if (Tab<N>::kPair) {
             __syncthreads();
@@ -435,7 +445,7 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
         o.start(first);
     }
 
-    const unsigned char* tab = MODE == 1 ? sTab : sTab + (size_t)q * TW * 128;
+    const unsigned char* tab = MODE == 1 ? sTab : N == 4 ? sTab + (size_t)(q >> 1) * TW * 256 : sTab + (size_t)q * TW * 128;
     bool done;
     if (warp == DW) {
         done = lane != 0 || mma_loop(a, Tn, t0, sc0, sc1, sB, bars, tmem, &tmap);
