@@ -143,12 +143,15 @@ struct Half {
 struct Outliers {
     const uint32_t* slab;
     const uint32_t* spill;
+    const uint32_t* nextp;      // address of entry cur + 4, the next one to load
+    int step;                   // words between consecutive entries at nextp: 32 in the slab, 1 in the CSR arrays
     int nslab, total, cur;
     uint32_t col;               // column of entry cur, 0xffffffff behind the last one
     uint32_t ent, e1, e2, e3;   // entries cur .. cur + 3 (column | fp16 value << 16)
-    __device__ __forceinline__ uint32_t fetch(int j) const {
-        return j < nslab ? __ldg(slab + (size_t)(1 + j) * 32) : __ldg(spill + j);
+    __device__ __forceinline__ const uint32_t* addr(int j) const {
+        return j < nslab ? slab + (size_t)(1 + j) * 32 : spill + j;
     }
+    __device__ __forceinline__ uint32_t fetch(int j) const { return __ldg(addr(j)); }
     __device__ __forceinline__ void start(int first) {
         cur = first;
         if (cur < total) { ent = fetch(cur); }
@@ -156,12 +159,17 @@ struct Outliers {
         if (cur + 2 < total) e2 = fetch(cur + 2);
         if (cur + 3 < total) e3 = fetch(cur + 3);
         col = cur < total ? (ent & 0xffffu) : 0xffffffffu;
+        nextp = addr(cur + 4);
+        step = cur + 4 < nslab ? 32 : 1;
     }
     __device__ __forceinline__ void advance() {
         ++cur;
         ent = e1; e1 = e2; e2 = e3;
         col = cur < total ? (ent & 0xffffu) : 0xffffffffu;
-        if (cur + 3 < total) e3 = fetch(cur + 3);
+        if (cur + 3 < total) {
+            e3 = __ldg(nextp);
+            if (cur + 4 == nslab) { nextp = spill + nslab; step = 1; } else nextp += step;
+        }
     }
 };
 
@@ -265,9 +273,11 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
             // W^ = fp16(D16 + S) at the outliers of this channel inside this half; the entries of the other half
             // (the other warp's) are passed over.  One loop, one copy of the code that advances the list.
             const uint32_t lo_k = k0 + PART * 64;
-            while (o.col < k0 + kSuper) {
+            // warp-uniform loop (as many trips as the busiest lane needs, the lanes converged at the top of each)
+            while (__any_sync(0xffffffffu, o.col < k0 + kSuper)) {
+                const bool mine_now = o.col < k0 + kSuper;
                 const uint32_t kk = o.col - lo_k;              // wraps around for entries below this half
-                if (kk < 64u) {
+                if (mine_now && kk < 64u) {
                     const uint32_t v2 = (o.ent >> 16) << ((kk & 1u) * 16u);
                     // the register that holds weight kk: found by nested tests, not a switch -- the indirect
                     // branch of a jump table inside this divergent loop stalled the warps (176 vs 149 us on
@@ -282,11 +292,14 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
             "@p2 add.rn.f16x2 %2, %2, %5;\n\t@p3 add.rn.f16x2 %3, %3, %5;\n\t}"                                    \
             : "+r"(d[4 * g]), "+r"(d[4 * g + 1]), "+r"(d[4 * g + 2]), "+r"(d[4 * g + 3])                          \
             : "r"(r & 3u), "r"(v2));
-                    XFP_OUT_GROUP(0) XFP_OUT_GROUP(1) XFP_OUT_GROUP(2) XFP_OUT_GROUP(3)
-                    XFP_OUT_GROUP(4) XFP_OUT_GROUP(5) XFP_OUT_GROUP(6) XFP_OUT_GROUP(7)
+                    if (r < 16u) {
+                        if (r < 8u) { XFP_OUT_GROUP(0) XFP_OUT_GROUP(1) } else { XFP_OUT_GROUP(2) XFP_OUT_GROUP(3) }
+                    } else {
+                        if (r < 24u) { XFP_OUT_GROUP(4) XFP_OUT_GROUP(5) } else { XFP_OUT_GROUP(6) XFP_OUT_GROUP(7) }
+                    }
 #undef XFP_OUT_GROUP
                 }
-                o.advance();
+                if (mine_now) o.advance();
             }
         } else {
 #pragma unroll
@@ -418,7 +431,7 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     const uint32_t tmem = s_tmem;
 
     // ---- the lane's outlier list: transposed slab first, the CSR arrays behind it ----
-    Outliers o{nullptr, nullptr, 0, 0, 0, 0xffffffffu, 0u, 0u, 0u, 0u};
+    Outliers o{nullptr, nullptr, nullptr, 1, 0, 0, 0, 0xffffffffu, 0u, 0u, 0u, 0u};
     if (rb_ok && a.ell_slots) {
         o.slab = a.b.ell + (size_t)rb * (a.ell_slots + 1) * 32 + lane;
         const int olen = (int)__ldg(o.slab);
