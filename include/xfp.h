@@ -165,6 +165,14 @@ int xfp_gemm_workspace_size(const xfp_desc* desc, int32_t m, size_t* workspace_b
 int xfp_gemm(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t m, void* y, int32_t y_type,
              void* workspace, size_t workspace_bytes, void* stream);
 
+/* xfp_gemm with typed activations: x_type XFP_T_F16 (the call above) or XFP_T_BF16, the paper's native type.  bf16
+ * rows of x are first converted to fp16 (round to nearest even, clamped to +-65504: exact for 2^-14 <= |x| <= 65504)
+ * by a small kernel into a scratch area behind the GEMM's own workspace, then multiplied by the same kernel.
+ *   workspace  xfp_gemm_typed_workspace_size(desc, m, x_type) bytes, zero-filled once before first use. */
+int xfp_gemm_typed_workspace_size(const xfp_desc* desc, int32_t m, int32_t x_type, size_t* workspace_bytes);
+int xfp_gemm_typed(const xfp_desc* desc, const void* packed, const void* x, int32_t x_type, int32_t m, void* y,
+                   int32_t y_type, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Convenience for callers whose activations live in host memory: brings x_host to x_dev, runs the GEMV for
  * desc->mode and delivers y in y_host, all on `stream` (the host sees y once the stream reached this point).
  * x_dev [batch][cols] fp16 and y_dev [batch][rows] are device staging buffers of the caller.  Pinned,

@@ -17,7 +17,8 @@ _LIB = None
 
 EXPORTS = ("xfp_packed_size", "xfp_pack", "xfp_gemv_v2", "xfp_gemv_v2a", "xfp_gemv_grouped", "xfp_gemv_host",
            "xfp_dequant", "xfp_status_str", "xfp_gemv_v2_noalloc", "xfp_gemv_grouped_epilogue", "xfp_gemv_typed",
-           "xfp_gemv_grouped_typed", "xfp_gemm", "xfp_gemm_workspace_size")
+           "xfp_gemv_grouped_typed", "xfp_gemm", "xfp_gemm_workspace_size", "xfp_gemm_typed",
+           "xfp_gemm_typed_workspace_size")
 
 XFP_EPI_NONE, XFP_EPI_SWIGLU, XFP_EPI_COMBINE = 0, 1, 2
 XFP_T_F32, XFP_T_F16, XFP_T_BF16 = 0, 1, 2
@@ -63,6 +64,8 @@ def load_library() -> C.CDLL:
     lib.xfp_dequant.argtypes = [dp, vp, vp, vp]
     lib.xfp_gemm_workspace_size.argtypes = [dp, i32, C.POINTER(sz)]
     lib.xfp_gemm.argtypes = [dp, vp, vp, i32, vp, i32, vp, sz, vp]
+    lib.xfp_gemm_typed_workspace_size.argtypes = [dp, i32, i32, C.POINTER(sz)]
+    lib.xfp_gemm_typed.argtypes = [dp, vp, vp, i32, i32, vp, i32, vp, sz, vp]
     lib.xfp_gemv_v2_noalloc.argtypes = [dp, vp, vp, i32, vp, i32, vp]
     lib.xfp_status_str.argtypes = [C.c_int]
     lib.xfp_status_str.restype = C.c_char_p
@@ -142,6 +145,21 @@ def xfp_gemm(desc, packed, x: torch.Tensor, y: torch.Tensor, workspace: torch.Te
     _check(load_library().xfp_gemm(C.byref(desc), _ptr(packed), _ptr(x), int(x.shape[0]), _ptr(y), _TORCH_TYPE[y.dtype],
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "xfp_gemm")
+
+
+def xfp_gemm_typed_workspace_size(desc, m: int, x_dtype=torch.bfloat16) -> int:
+    b = C.c_size_t()
+    _check(load_library().xfp_gemm_typed_workspace_size(C.byref(desc), int(m), _TORCH_TYPE[x_dtype], C.byref(b)),
+           "xfp_gemm_typed_workspace_size")
+    return b.value
+
+
+def xfp_gemm_typed(desc, packed, x: torch.Tensor, y: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    """xfp_gemm with x in fp16 or bf16 (taken from the tensor's dtype); workspace sized by
+    xfp_gemm_typed_workspace_size(desc, m, x.dtype)."""
+    _check(load_library().xfp_gemm_typed(C.byref(desc), _ptr(packed), _ptr(x), _TORCH_TYPE[x.dtype], int(x.shape[0]),
+                                         _ptr(y), _TORCH_TYPE[y.dtype], _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)), "xfp_gemm_typed")
 
 
 def xfp_gemv_grouped(desc, n: int, packed_ptrs: torch.Tensor, x_ptrs: torch.Tensor, y_ptrs: torch.Tensor,

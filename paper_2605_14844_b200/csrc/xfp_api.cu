@@ -230,6 +230,34 @@ int xfp_gemm(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_
     return launch_gemm_tc(l, c, (cudaStream_t)stream) == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 
+int xfp_gemm_typed_workspace_size(const xfp_desc* desc, int32_t m, int32_t x_type, size_t* workspace_bytes) {
+    if (x_type != XFP_T_F16 && x_type != XFP_T_BF16) return XFP_ERR_SHAPE;
+    int st = xfp_gemm_workspace_size(desc, m, workspace_bytes);
+    if (st) return st;
+    if (x_type == XFP_T_BF16) {
+        const Layout l = layout_of(desc);
+        *workspace_bytes = align256(*workspace_bytes) + gemm_x_scratch_bytes(l, m);
+    }
+    return XFP_OK;
+}
+
+int xfp_gemm_typed(const xfp_desc* desc, const void* packed, const void* x, int32_t x_type, int32_t m, void* y,
+                   int32_t y_type, void* workspace, size_t workspace_bytes, void* stream) {
+    if (x_type == XFP_T_F16) return xfp_gemm(desc, packed, (const uint16_t*)x, m, y, y_type, workspace, workspace_bytes, stream);
+    if (x_type != XFP_T_BF16) return XFP_ERR_SHAPE;
+    size_t need = 0;
+    int st = xfp_gemm_typed_workspace_size(desc, m, x_type, &need);
+    if (st) return st;
+    if (!packed || !x || !y || !workspace) return XFP_ERR_NULL;
+    if (!aligned16(x) || !aligned16(workspace)) return XFP_ERR_ALIGN;
+    if (workspace_bytes < need) return XFP_ERR_BUFFER_TOO_SMALL;
+    const Layout l = layout_of(desc);
+    const size_t own = align256(gemm_workspace_bytes(l, m));
+    uint16_t* x16 = (uint16_t*)((char*)workspace + own);
+    if (launch_x_to_f16(x, x16, (size_t)m * l.cols, (cudaStream_t)stream) != cudaSuccess) return XFP_ERR_CUDA;
+    return xfp_gemm(desc, packed, x16, m, y, y_type, workspace, own, stream);
+}
+
 int xfp_dequant(const xfp_desc* desc, const void* packed, uint16_t* W, void* stream) {
     int st = check_desc(desc);
     if (st) return st;

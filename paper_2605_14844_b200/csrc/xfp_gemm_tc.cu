@@ -641,6 +641,23 @@ size_t gemm_workspace_bytes(const Layout& l, int M) {
     return gemm_ctrl_bytes(l, M) + partial;
 }
 
+namespace {
+// bf16 rows of x -> fp16 (round to nearest even, clamped to the finite fp16 range), eight values per thread and step
+__global__ void x_to_f16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = x8_as_f16(__ldg(src + i), 1);
+}
+}  // namespace
+
+size_t gemm_x_scratch_bytes(const Layout& l, int M) { return align256((size_t)M * l.cols * 2); }
+
+cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaStream_t s) {
+    const size_t n8 = elems / 8;     // cols is a multiple of 128
+    const unsigned grid = (unsigned)((n8 + 255) / 256 < 148 * 8 ? (n8 + 255) / 256 : 148 * 8);
+    x_to_f16_kernel<<<grid ? grid : 1, 256, 0, s>>>((const uint4*)x_bf16, (uint4*)x_f16, n8);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s) {
     if (l.mode == 1) {
         switch (l.bits) {

@@ -96,6 +96,9 @@ bool gemm_tc_supported(const Layout& l, int M);
 size_t gemm_ctrl_bytes(const Layout& l, int M);
 size_t gemm_workspace_bytes(const Layout& l, int M);
 cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s);
+// bf16 activations: converted to fp16 into a scratch area behind the GEMM's own workspace, then the same kernel
+size_t gemm_x_scratch_bytes(const Layout& l, int M);
+cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaStream_t s);
 
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);

@@ -164,6 +164,11 @@ def test_null_alignment_and_size_checks_need_no_gpu(lib):
     assert lib.xfp_gemm(C.byref(d), a, a, 64, a, 3, a, 1 << 30, n) == 3                     # unknown y type
     assert lib.xfp_gemm(C.byref(d), a, a, 64, a, 0, a, 16, n) == 5
     assert lib.xfp_gemm(C.byref(dbig), a, a, 64, a, 0, a, 1 << 30, n) == 4
+    wsz2 = C.c_size_t()
+    assert lib.xfp_gemm_typed_workspace_size(C.byref(d), 64, 2, C.byref(wsz2)) == 0 and wsz2.value >= wsz.value + 64 * 256 * 2
+    assert lib.xfp_gemm_typed_workspace_size(C.byref(d), 64, 0, C.byref(wsz2)) == 3        # x cannot be fp32
+    assert lib.xfp_gemm_typed(C.byref(d), a, a, 2, 64, a, 0, a, 64, n) == 5
+    assert lib.xfp_gemm_typed(C.byref(d), a, n, 2, 64, a, 0, a, 1 << 30, n) == 1
     assert xfp.xfp_status_str(0) == "ok" and "aligned" in xfp.xfp_status_str(2)
 
 

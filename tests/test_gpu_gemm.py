@@ -148,3 +148,34 @@ def test_gemm_randomized(i):
     q = synth.random_quantized(mode, rows, cols, bits, rate, seed=7000 + i, placement=placement, lib_size=L)
     pm = xfp.pack_tensors(q, col_bits=16 if i % 2 else 32)
     _check(q, pm, synth.activations(m, cols, seed=8000 + i), [torch.float32, torch.float32, torch.float16][i % 3])
+
+
+@pytest.mark.parametrize("mode,bits,m", [(0, 4, 40), (0, 5, 300), (1, 3, 130), (0, 2, 1)])
+def test_gemm_bf16_activations(mode, bits, m):
+    """xfp_gemm_typed: bf16 rows of x (converted to fp16 by a kernel of the library, then the same GEMM); reference: the
+    oracle on the exact bf16 values; tolerance: the GEMV bound plus the conversion's 2^-25 per weight for tiny |x|."""
+    q = synth.random_quantized(mode, 200, 1024, bits, 0.01, seed=5100 + bits)
+    pm = xfp.pack_tensors(q)
+    g = torch.Generator().manual_seed(5200 + m)
+    xb = torch.randn((m, q.cols), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    x64 = xb.to(torch.float64).numpy()
+    mo = to_oracle(q)
+    ref, absum = xo.gemv_x64(mo, x64)
+    tiny = 2.0 ** -25 * np.abs(xo.dequant(mo).view(np.float16).astype(np.float64)).sum(1)[None, :]
+    for dt, ulp in ((torch.float32, 0.0), (torch.bfloat16, 2.0 ** -8)):
+        ws = torch.zeros(xfp.xfp_gemm_typed_workspace_size(pm.desc, m, torch.bfloat16), dtype=torch.uint8, device="cuda")
+        y = torch.full((m, q.rows), float("nan"), dtype=dt, device="cuda")
+        xfp.xfp_gemm_typed(pm.desc, pm.packed, xb.cuda(), y, ws)
+        torch.cuda.synchronize()
+        assert int(ws[:4].view(torch.int32).item()) == 0
+        got = y.to(torch.float64).cpu().numpy()
+        tol = TOL * absum + tiny + ulp * np.abs(ref) + 1e-30
+        assert np.all(np.abs(got - ref) <= tol), float((np.abs(got - ref) / tol).max())
+    # fp16 rows of x through the typed entry are the plain call
+    x16 = synth.activations(m, q.cols, seed=5300)
+    xd = torch.from_numpy(x16.view(np.int16)).cuda().view(torch.float16)
+    ws = torch.zeros(xfp.xfp_gemm_typed_workspace_size(pm.desc, m, torch.float16), dtype=torch.uint8, device="cuda")
+    y1 = torch.empty((m, q.rows), dtype=torch.float32, device="cuda")
+    xfp.xfp_gemm_typed(pm.desc, pm.packed, xd, y1, ws)
+    y2, _, _ = _run(q, pm, x16)
+    assert torch.equal(y1, y2)
