@@ -554,12 +554,22 @@ Plan plan_of(const Layout& l, int M) {
     // columns), which decode the weights once per 256 rows -- 28672 x 8192, M = 512: 555 -> 450 us; 4096 x 4096,
     // M = 512: 80 -> 72 us -- when their x stages fit beside the tables.
     p.maxT = kSmallT; p.x_stages = kXStages;
-    if (M > kSmallT) {
+    // the same CTA shape (16 decode warps, alone on its SM) also serves fewer rows of x when the tables leave no room
+    // for two CTAs of 128-row tiles on an SM (V2a from N = 4: a 64 KB library; 28672 x 8192, M = 128: 274 us with one
+    // CTA of 8 decode warps per SM)
+    const int tsmall = M >= kSmallT ? kSmallT : (M + 15) & ~15;
+    const bool lone_anyway = p.tab_bytes + (size_t)2 * tsmall * 256 > 113 * 1024;
+    if (M > kSmallT || lone_anyway) {
         for (int xs = kXStages; xs >= 2; --xs) {
             if (p.tab_bytes + (size_t)xs * 16 * kBigT * 16 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
         }
     }
     const int tmax = M >= p.maxT ? p.maxT : (M + 15) & ~15;    // rows of x in the largest tile of this launch
+    // 128-row tiles: two x stages instead of three where that keeps two CTAs on an SM (N = 3 pair tables and N = 6
+    // tables are 32 KB: 28672 x 8192, M = 128, N = 3: 216 us with one CTA per SM)
+    if (p.maxT == kSmallT && p.tab_bytes + (size_t)kXStages * tmax * 256 > 113 * 1024 &&
+        p.tab_bytes + (size_t)2 * tmax * 256 <= 113 * 1024)
+        p.x_stages = 2;
     p.smem = p.tab_bytes + (size_t)p.x_stages * 16 * tmax * 16;
     if (p.smem < kMinSmem) p.smem = kMinSmem;
     if (p.maxT == kBigT && p.smem < 120 * 1024) p.smem = 120 * 1024;   // alone on its SM: it holds all 512 columns
