@@ -561,7 +561,8 @@ Plan plan_of(const Layout& l, int M) {
     const bool lone_anyway = p.tab_bytes + (size_t)2 * tsmall * 256 > 113 * 1024;
     if (M > kSmallT || lone_anyway) {
         for (int xs = kXStages; xs >= 2; --xs) {
-            if (p.tab_bytes + (size_t)xs * 16 * kBigT * 16 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
+            const int tbig = M >= kBigT ? kBigT : (M + 15) & ~15;    // rows of x its largest tile would hold
+            if (p.tab_bytes + (size_t)xs * tbig * 256 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
         }
     }
     const int tmax = M >= p.maxT ? p.maxT : (M + 15) & ~15;    // rows of x in the largest tile of this launch
