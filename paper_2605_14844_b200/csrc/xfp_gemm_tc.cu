@@ -541,6 +541,7 @@ EncodeTiledFn encode_tiled_fn() {
 struct Plan {
     int row_tiles, tok_tiles, ks, sc_per_slice;
     int maxT, x_stages;
+    bool lone;        // the CTA with 16 decode warps, alone on its SM (else 8 decode warps, two CTAs per SM)
     size_t tab_bytes, smem;
 };
 
@@ -553,7 +554,7 @@ Plan plan_of(const Layout& l, int M) {
     // More than 128 rows of x: tiles of 256 rows (one CTA per SM with two groups of decode warps, all 512 tensor-memory
     // columns), which decode the weights once per 256 rows -- 28672 x 8192, M = 512: 555 -> 450 us; 4096 x 4096,
     // M = 512: 80 -> 72 us -- when their x stages fit beside the tables.
-    p.maxT = kSmallT; p.x_stages = kXStages;
+    p.maxT = kSmallT; p.x_stages = kXStages; p.lone = false;
     // the same CTA shape (16 decode warps, alone on its SM) also serves fewer rows of x when the tables leave no room
     // for two CTAs of 128-row tiles on an SM (V2a from N = 4: a 64 KB library; 28672 x 8192, M = 128: 274 us with one
     // CTA of 8 decode warps per SM)
@@ -562,24 +563,26 @@ Plan plan_of(const Layout& l, int M) {
     if (M > kSmallT || lone_anyway) {
         for (int xs = kXStages; xs >= 2; --xs) {
             const int tbig = M >= kBigT ? kBigT : (M + 15) & ~15;    // rows of x its largest tile would hold
-            if (p.tab_bytes + (size_t)xs * tbig * 256 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; break; }
+            if (p.tab_bytes + (size_t)xs * tbig * 256 <= kSmemLimit) { p.maxT = kBigT; p.x_stages = xs; p.lone = true; break; }
         }
+        // tables too large for 256-row x stages (V2a, N = 5: 128 KB): the lone CTA with 128-row tiles
+        if (!p.lone && lone_anyway) { p.lone = true; p.x_stages = 2; }
     }
     const int tmax = M >= p.maxT ? p.maxT : (M + 15) & ~15;    // rows of x in the largest tile of this launch
     // 128-row tiles: two x stages instead of three where that keeps two CTAs on an SM (N = 3 pair tables and N = 6
     // tables are 32 KB: 28672 x 8192, M = 128, N = 3: 216 us with one CTA per SM)
-    if (p.maxT == kSmallT && p.tab_bytes + (size_t)kXStages * tmax * 256 > 113 * 1024 &&
+    if (!p.lone && p.tab_bytes + (size_t)kXStages * tmax * 256 > 113 * 1024 &&
         p.tab_bytes + (size_t)2 * tmax * 256 <= 113 * 1024)
         p.x_stages = 2;
     p.smem = p.tab_bytes + (size_t)p.x_stages * 16 * tmax * 16;
     if (p.smem < kMinSmem) p.smem = kMinSmem;
-    if (p.maxT == kBigT && p.smem < 120 * 1024) p.smem = 120 * 1024;   // alone on its SM: it holds all 512 columns
+    if (p.lone && p.smem < 120 * 1024) p.smem = 120 * 1024;   // alone on its SM: it may hold all 512 columns
     p.row_tiles = (l.RB + 3) / 4;
     p.tok_tiles = (M + p.maxT - 1) / p.maxT;
     const int tiles = p.row_tiles * p.tok_tiles;
     int ks = 1;
     // fewer tiles than CTA slots (two per SM): cut K, at least two super-chunks per slice
-    const int slots = p.maxT == kBigT ? 148 : 2 * 148;
+    const int slots = p.lone ? 148 : 2 * 148;
     while (tiles * ks * 2 <= slots && l.SC / (ks * 2) >= 2) ks *= 2;
     p.sc_per_slice = (l.SC + ks - 1) / ks;
     p.ks = (l.SC + p.sc_per_slice - 1) / p.sc_per_slice;
@@ -627,7 +630,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
     a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
     const dim3 grid((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks);
-    if (p.maxT == kBigT)
+    if (p.lone)
         gemm_tc_kernel<N, MODE, true><<<grid, threads_of(true), smem, s>>>(a, tmap);
     else
         gemm_tc_kernel<N, MODE, false><<<grid, threads_of(false), smem, s>>>(a, tmap);
