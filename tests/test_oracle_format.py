@@ -313,3 +313,29 @@ def test_gemv_with_real_activations_matches_the_fp16_entry_and_a_dense_matvec():
                     Wd[i, q.ocol[p_]] += float(q.oval[p_:p_ + 1].view(np.float16)[0])
             assert np.allclose(y, (Wd @ xr.T).T, rtol=1e-12, atol=0)
         assert np.all(a >= np.abs(y))
+
+
+def test_silu_mul_against_closed_forms_and_a_library_sigmoid():
+    """The element-wise step of a gated expert block, h = SiLU(gate) * up with SiLU(g) = g * sigmoid(g): exact
+    values, both limits, the odd-part identity SiLU(g) - SiLU(-g) = g, a library sigmoid, and the slope bound the
+    fused-store tolerance relies on."""
+    from scipy.special import expit
+    u = np.array([1.0, -2.5, 3.0, 0.125])
+    assert np.array_equal(xo.silu_mul(np.zeros(4), u), np.zeros(4))               # SiLU(0) = 0
+    assert xo.silu_mul(np.array([1.0]), np.array([1.0]))[0] == pytest.approx(1.0 / (1.0 + np.exp(-1.0)), rel=1e-15)
+    assert xo.silu_mul(np.array([np.log(3.0)]), np.array([2.0]))[0] == pytest.approx(2.0 * np.log(3.0) * 0.75, rel=1e-14)
+    big = np.array([40.0, 80.0, 700.0])
+    assert np.allclose(xo.silu_mul(big, np.ones(3)), big, rtol=1e-15)             # -> g for g >> 0
+    assert np.all(np.abs(xo.silu_mul(-big, np.ones(3))) < 1e-15)                  # -> 0 for g << 0
+    rng = np.random.default_rng(71)
+    g = rng.normal(0, 4, 4096)
+    up = rng.normal(0, 2, 4096)
+    one = np.ones_like(g)
+    assert np.allclose(xo.silu_mul(g, one) - xo.silu_mul(-g, one), g, rtol=0, atol=1e-14)
+    assert np.allclose(xo.silu_mul(g, up), expit(g) * g * up, rtol=1e-13, atol=1e-300)
+    assert np.allclose(xo.silu_mul(g, 3.0 * up), 3.0 * xo.silu_mul(g, up), rtol=1e-15)   # linear in `up`
+    # |SiLU'| <= 1.1 everywhere (the maximum, 1.0998, sits near g = 2.4): central differences on a fine grid
+    t = np.linspace(-30, 30, 600001)
+    d = (xo.silu_mul(t + 1e-6, np.ones_like(t)) - xo.silu_mul(t - 1e-6, np.ones_like(t))) / 2e-6
+    assert 1.099 < np.abs(d).max() <= 1.1 and 2.3 < t[np.argmax(d)] < 2.5
+    assert d.min() > -0.1                                                         # the dip left of zero is shallow

@@ -251,19 +251,16 @@ def _decoded(scale16, lib16, mid16):
     return (s * l + m).astype(np.float16).astype(np.float64)
 
 
-@pytest.mark.parametrize("bits,L", [(2, 8), (3, 32), (4, 16)])
-def test_libfit_assignment_is_the_brute_force_optimum(bits, L):
-    """Second half of LibFit against exhaustive search: for every group the stored (mid, scale) are the
-    fp16 roundings of the range's middle and half-width, no other library entry gives a smaller squared
-    error under nearest-value decoding, and every index points at a nearest decoded value."""
-    rows, cols = 12, 512
-    W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, seed=81), 0.01, 82)
-    mask, mu, _ = xo.outlier_mask(W)
-    m = xo.quantize_v2a(W, bits, mask, mu, lib_size=L)
-    bulk = np.where(mask != 0, mu, W.astype(np.float64))
-    for i in range(rows):
-        for g in range(cols // 128):
-            v = bulk[i, g * 128:(g + 1) * 128]
+def _check_assignment_by_exhaustive_search(m, bulk, group):
+    """Every group of `m` against exhaustive search over the library `m.codebook`: the stored (mid, scale) are the
+    fp16 roundings of the range's middle and half-width, no other library entry gives a smaller squared error
+    under nearest-value decoding (ties: the lower entry), and every index points at a nearest decoded value
+    (ties: the lower index)."""
+    L = m.codebook.shape[0]
+    ar = np.arange(group)
+    for i in range(m.rows):
+        for g in range(m.cols // group):
+            v = bulk[i, g * group:(g + 1) * group]
             lo, hi = v.min(), v.max()
             assert m.gmid[i, g] == np.float16(0.5 * (hi + lo)).view(np.uint16)
             assert m.gscale[i, g] == np.float16(0.5 * (hi - lo)).view(np.uint16)
@@ -273,12 +270,61 @@ def test_libfit_assignment_is_the_brute_force_optimum(bits, L):
                 sse[l] = (np.abs(v[:, None] - dec[None, :]).min(axis=1) ** 2).sum()
             chosen = int(m.gid[i, g])
             assert sse[chosen] <= sse.min() * (1 + 1e-12)
-            assert chosen == int(np.flatnonzero(sse <= sse.min() * (1 + 1e-12))[0])      # ties: the lower entry
+            assert chosen == int(np.flatnonzero(sse <= sse.min() * (1 + 1e-12))[0])
             dec = _decoded(m.gscale[i, g], m.codebook[chosen], m.gmid[i, g])
             dist = np.abs(v[:, None] - dec[None, :])
-            q = m.idx[i, g * 128:(g + 1) * 128].astype(int)
-            assert np.array_equal(dist[np.arange(128), q], dist.min(axis=1))
-            assert np.array_equal(q, dist.argmin(axis=1))                                # ties: the lower index
+            q = m.idx[i, g * group:(g + 1) * group].astype(int)
+            assert np.array_equal(dist[ar, q], dist.min(axis=1))
+            assert np.array_equal(q, dist.argmin(axis=1))
+
+
+@pytest.mark.parametrize("bits,L", [(2, 8), (3, 32), (4, 16)])
+def test_libfit_assignment_is_the_brute_force_optimum(bits, L):
+    """Second half of LibFit against exhaustive search (group size 128, the paper's default)."""
+    rows, cols = 12, 512
+    W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, seed=81), 0.01, 82)
+    mask, mu, _ = xo.outlier_mask(W)
+    m = xo.quantize_v2a(W, bits, mask, mu, lib_size=L)
+    _check_assignment_by_exhaustive_search(m, np.where(mask != 0, mu, W.astype(np.float64)), 128)
+
+
+@pytest.mark.parametrize("group", [64, 256])
+def test_libfit_assignment_at_other_group_sizes(group):
+    """The group size is a parameter of the format ("Lane geometry"): the same exhaustive-search property at 64
+    and 256 weights per group, and the metadata has one (id, scale, mid) per group of that size."""
+    rows, cols, bits, L = 10, 1024, 3, 16
+    W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, seed=91), 0.01, 92)
+    mask, mu, _ = xo.outlier_mask(W)
+    m = xo.quantize_v2a(W, bits, mask, mu, lib_size=L, group=group)
+    assert m.group_size == group and m.gid.shape == (rows, cols // group)
+    _check_assignment_by_exhaustive_search(m, np.where(mask != 0, mu, W.astype(np.float64)), group)
+    # the reconstruction uses the group of the stored size: dequant against the decode written out here
+    D = _f16(xo.dequant(xo.QuantizedMatrix(m.mode, m.rows, m.cols, m.bits, m.idx, m.codebook,
+                                           np.zeros(rows + 1, np.int32), np.zeros(0, np.int32),
+                                           np.zeros(0, np.uint16), group_size=group, lib_size=L, gid=m.gid,
+                                           gscale=m.gscale, gmid=m.gmid)))
+    for i in (0, rows - 1):
+        for g in (0, cols // group - 1):
+            dec = _decoded(m.gscale[i, g], m.codebook[m.gid[i, g]], m.gmid[i, g])
+            assert np.array_equal(D[i, g * group:(g + 1) * group], dec[m.idx[i, g * group:(g + 1) * group]])
+
+
+def test_libfit_with_a_library_learned_on_another_matrix():
+    """The experts of a routed layer share one library ("V2a: Shared Codebook Library"): a library learned on
+    matrix A and handed to the quantiser of matrix B is stored unchanged, and B's group assignment against it
+    satisfies the same exhaustive-search property as an own library."""
+    bits, L = 3, 16
+    A = synth.gaussian_weights(48, 512, seed=85)
+    B = synth.plant_uniform_outliers(synth.gaussian_weights(12, 512, seed=86) * np.float32(1.7), 0.01, 87)
+    ma = xo.quantize_v2a(A, bits, np.zeros(A.shape, np.uint8), 0.0, lib_size=L)
+    mask, mu, _ = xo.outlier_mask(B)
+    mb = xo.quantize_v2a(B, bits, mask, mu, library=ma.codebook)
+    assert mb.lib_size == L and np.array_equal(mb.codebook, ma.codebook)
+    assert mb.gid.max() < L and mb.idx.max() < (1 << bits)
+    _check_assignment_by_exhaustive_search(mb, np.where(mask != 0, mu, B.astype(np.float64)), 128)
+    # a borrowed library must still reconstruct a Gaussian bulk to the 3-bit band
+    cos_shared = xo.median(xo.row_cosine(B, xo.dequant(mb)))
+    assert cos_shared > 0.975
 
 
 def test_libfit_library_invariants():

@@ -1,9 +1,6 @@
 """xfp_gemv_v2_noalloc: the V2 GEMV for callers that may not allocate device memory (a plug-in inside an
 application that owns all GPU memory, or a latency-critical path where cudaMalloc is forbidden).  It
 takes no workspace: the split-K scratch lives in an 8 MiB array inside the library.
-
-This file sorts last on purpose: if it fails, a run that stops at the first failure has already run
-every other test.  It passes on its own in a fresh process and after the rest of the suite.
 """
 import ctypes as C
 
@@ -25,27 +22,33 @@ def _xdev(x16):
     return torch.from_numpy(x16.view(np.int16)).cuda().view(torch.float16)
 
 
-@pytest.mark.parametrize("bits,rows,cols,batch", [(6, 512, 4096, 1), (4, 1024, 2048, 3)])
-def test_noalloc_matches_workspace_entry_point_twice(bits, rows, cols, batch):
+@pytest.mark.parametrize("bits,rows,cols,batch,y_fp16", [(6, 512, 4096, 1, 0), (4, 1024, 2048, 3, 0),
+                                                         (4, 512, 4096, 1, 1)])
+def test_noalloc_matches_the_oracle_and_the_workspace_entry_point_twice(bits, rows, cols, batch, y_fp16):
     # shapes that split K, so the scratch (partial sums and counters) is really used
     q = synth.random_quantized(0, rows, cols, bits, 0.01, seed=4242 + bits)
     pm = xfp.pack_tensors(q, col_bits=16)
     lib = xfp.load_library()
+    ydt = torch.float16 if y_fp16 else torch.float32
     for call in range(2):                                   # two calls in a row share the built-in scratch
         x16 = synth.activations(batch, cols, seed=50 + call)
         x = _xdev(x16)
-        y_ws = torch.zeros((batch, rows), dtype=torch.float32, device="cuda")
-        y_na = torch.full((batch, rows), float("nan"), dtype=torch.float32, device="cuda")
-        xfp.xfp_gemv_v2(pm.desc, pm.packed, x, batch, y_ws, False, pm.workspace)
+        y_ws = torch.zeros((batch, rows), dtype=ydt, device="cuda")
+        y_na = torch.full((batch, rows), float("nan"), dtype=ydt, device="cuda")
+        xfp.xfp_gemv_v2(pm.desc, pm.packed, x, batch, y_ws, bool(y_fp16), pm.workspace)
         st = lib.xfp_gemv_v2_noalloc(C.byref(pm.desc), C.c_void_p(pm.packed.data_ptr()), C.c_void_p(x.data_ptr()),
-                                     batch, C.c_void_p(y_na.data_ptr()), 0,
+                                     batch, C.c_void_p(y_na.data_ptr()), y_fp16,
                                      C.c_void_p(torch.cuda.current_stream().cuda_stream))
         assert st == 0, xfp.xfp_status_str(st)
         torch.cuda.synchronize()
-        _, absum = xo.gemv(to_oracle(q), x16)
-        diff = np.abs(y_na.cpu().numpy().astype(np.float64) - y_ws.cpu().numpy().astype(np.float64))
-        assert np.all(np.isfinite(y_na.cpu().numpy()))
-        assert np.all(diff <= TOL * absum)
+        ref, absum = xo.gemv(to_oracle(q), x16)
+        got = y_na.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got))
+        assert np.all(np.abs(got - ref) <= TOL * absum)                                    # against the oracle
+        assert np.all(np.abs(got - y_ws.float().cpu().numpy().astype(np.float64)) <= TOL * absum)
+        # the summation order is fixed and the same in both entry points: identical bits
+        assert torch.equal(y_na.view(torch.int16 if y_fp16 else torch.int32),
+                           y_ws.view(torch.int16 if y_fp16 else torch.int32))
 
 
 def test_noalloc_rejects_shapes_beyond_the_builtin_scratch():
