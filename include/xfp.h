@@ -24,6 +24,19 @@
  *    packed from bad data is still safe to read).
  *  - `packed` is opaque, position independent (may be copied with cudaMemcpy) and fully
  *    determined by the descriptor; keep the descriptor with it.
+ *  - Thread safety: calls from several host threads are safe as long as they do not share a workspace
+ *    (or the built-in scratch of xfp_gemv_v2_noalloc); the library keeps no mutable state besides
+ *    per-device caches that are filled once.
+ *  - Stream capture: the first call of an entry point that launches kernels (gemv, gemm, dequant, pack and
+ *    their variants) on each device sets kernel attributes and asks the device for its properties.  Make one
+ *    call per kernel variant you will use (same mode, bits and batch class) on each device BEFORE you begin a
+ *    stream capture; later calls with those variants only launch.
+ *  - Programmatic dependent launch: the GEMV kernels start before the previous kernel of the stream has
+ *    finished and read the packed blob -- and, for the grouped calls, the device pointer lists and the
+ *    routing weights -- BEFORE they wait for it; x, y and the workspace are touched only after the wait.
+ *    Blobs, pointer lists and routing weights must therefore be complete when the call is made: do not
+ *    produce them with a kernel that itself releases its dependents early (a plain kernel, a copy or a memset
+ *    on the same stream is fine).
  */
 #ifndef XFP_H
 #define XFP_H
@@ -160,6 +173,8 @@ int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* p
  *   workspace  xfp_gemm_workspace_size(desc, m) bytes, zero-filled once before first use; its counter part is left
  *              zero-filled by every call.  Its first 32-bit word is an error flag: the kernel sets it to 1 if one of
  *              its bounded waits ran out (y is then not written); the caller may read it after synchronising.
+ *              The library never clears the flag, and a call that set it may leave tile counters behind: a
+ *              workspace whose flag reads 1 must be zero-filled again before it is reused.
  * Results are deterministic (K slices, when the matrix has few rows, are added in slice order). */
 int xfp_gemm_workspace_size(const xfp_desc* desc, int32_t m, size_t* workspace_bytes);
 int xfp_gemm(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t m, void* y, int32_t y_type,

@@ -4,6 +4,24 @@
 
 using namespace xfp;
 
+namespace xfp {
+
+int sm_count() {
+    static std::atomic<int> cache[256] = {};
+    const int dev = DeviceOnce::current();
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            n = kSizingSMs;   // no device to ask (host-only use of the library)
+        }
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
+}  // namespace xfp
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -292,13 +310,6 @@ int xfp_gemv_host(const xfp_desc* desc, const void* packed, const uint16_t* x_ho
     if (y == y_dev && cudaMemcpyAsync(y_host, y_dev, ybytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return XFP_ERR_CUDA;
     return XFP_OK;
 }
-
-void xfp_debug_set_ksplit(int ks) { pair_set_ksplit_override(ks); }
-void xfp_debug_set_prefetch(int d) { pair_set_prefetch(d); }
-void xfp_debug_set_mode(int m) { pair_set_debug(m); }
-void xfp_debug_v2a_pair(int v) { v2a_set_pair(v); }
-void xfp_debug_set_small(int v) { pair_set_small(v); }
-void xfp_debug_set_trace(void* p, size_t calls) { pair_set_trace(p, calls); }
 
 const char* xfp_status_str(int status) {
     switch (status) {

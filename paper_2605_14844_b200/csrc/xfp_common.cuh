@@ -40,10 +40,14 @@ __device__ __forceinline__ uint16_t f2h(float f) { return __half_as_ushort(__flo
 // Activations may arrive as bf16 (the paper's native type): they are converted to fp16 while they are staged,
 // round to nearest even, clamped to the finite fp16 range.  A bf16 value with |x| in [2^-14, 65504] has 8
 // significant bits and converts exactly; smaller ones land on the fp16 subnormal grid (absolute error <= 2^-25).
+// NaN stays NaN (the clamp is applied to ordered values only; fminf/fmaxf would return the bound instead), so a
+// NaN activation poisons y under bf16 exactly as it does under fp16.
+__device__ __forceinline__ float clamp_f16_range(float v) {
+    return (v != v) ? v : fminf(fmaxf(v, -65504.f), 65504.f);
+}
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v) {
-    float lo = __uint_as_float(v << 16), hi = __uint_as_float(v & 0xffff0000u);
-    lo = fminf(fmaxf(lo, -65504.f), 65504.f);
-    hi = fminf(fmaxf(hi, -65504.f), 65504.f);
+    const float lo = clamp_f16_range(__uint_as_float(v << 16));
+    const float hi = clamp_f16_range(__uint_as_float(v & 0xffff0000u));
     const __half2 h = __floats2half2_rn(lo, hi);
     return *(const uint32_t*)&h;
 }
@@ -54,8 +58,11 @@ __device__ __forceinline__ uint4 x8_as_f16(uint4 v, int x_bf16) {
     }
     return v;
 }
+// One activation as the float the kernels multiply with: a bf16 value takes the same route as in the staged
+// kernels (clamp, round to fp16), so that every kernel sees the same x whatever the dispatcher picked.
 __device__ __forceinline__ float x_as_float(uint16_t bits, int x_bf16) {
-    return x_bf16 ? fminf(fmaxf(__uint_as_float((uint32_t)bits << 16), -65504.f), 65504.f) : h2f(bits);
+    if (!x_bf16) return h2f(bits);
+    return __half2float(__float2half_rn(clamp_f16_range(__uint_as_float((uint32_t)bits << 16))));
 }
 // Output element i of y: fp32 (kind 0), fp16 (1) or bf16 (2), one rounding of the fp32 sum.
 __device__ __forceinline__ void put_y(void* y, size_t i, float v, int kind) {

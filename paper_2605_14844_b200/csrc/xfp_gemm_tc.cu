@@ -547,7 +547,8 @@ struct Plan {
 
 constexpr size_t kSmemLimit = 227 * 1024 - 1024;   // dynamic shared memory a CTA may ask for, less the static part
 
-Plan plan_of(const Layout& l, int M) {
+// `sms`: SMs to plan for (kSizingSMs when sizing the workspace, the device's own count, capped by it, at launch)
+Plan plan_of(const Layout& l, int M, int sms) {
     Plan p;
     p.tab_bytes = l.mode == 1 ? (size_t)l.L * l.E * 128 : (size_t)4 * (l.bits <= 3 ? l.E * l.E : l.E) * 128;
     p.tab_bytes = (p.tab_bytes + 1023) & ~size_t(1023);      // the x stages behind the tables are 1024-byte aligned
@@ -582,7 +583,7 @@ Plan plan_of(const Layout& l, int M) {
     const int tiles = p.row_tiles * p.tok_tiles;
     int ks = 1;
     // fewer tiles than CTA slots (two per SM): cut K, at least two super-chunks per slice
-    const int slots = p.lone ? 148 : 2 * 148;
+    const int slots = p.lone ? sms : 2 * sms;
     while (tiles * ks * 2 <= slots && l.SC / (ks * 2) >= 2) ks *= 2;
     p.sc_per_slice = (l.SC + ks - 1) / ks;
     p.ks = (l.SC + p.sc_per_slice - 1) / p.sc_per_slice;
@@ -591,7 +592,7 @@ Plan plan_of(const Layout& l, int M) {
 
 template <int N, int MODE>
 cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
-    const Plan p = plan_of(l, c.M);
+    const Plan p = plan_of(l, c.M, sched_sms());
     const int tmax = c.M >= p.maxT ? p.maxT : (c.M + 15) & ~15;  // rows of x in the largest tile of this launch
     const int b_half = tmax * 128;
     const size_t tab_bytes = p.tab_bytes, smem = p.smem;
@@ -645,12 +646,12 @@ bool gemm_tc_supported(const Layout& l, int M) {
 }
 
 size_t gemm_ctrl_bytes(const Layout& l, int M) {
-    const Plan p = plan_of(l, M);
+    const Plan p = plan_of(l, M, kSizingSMs);
     return align256((size_t)(1 + p.row_tiles * p.tok_tiles) * 4);
 }
 
 size_t gemm_workspace_bytes(const Layout& l, int M) {
-    const Plan p = plan_of(l, M);
+    const Plan p = plan_of(l, M, kSizingSMs);
     const size_t partial = p.ks > 1 ? (size_t)p.row_tiles * p.tok_tiles * p.ks * p.maxT * kTileRows * 4 : 0;
     return gemm_ctrl_bytes(l, M) + partial;
 }
@@ -667,7 +668,8 @@ size_t gemm_x_scratch_bytes(const Layout& l, int M) { return align256((size_t)M 
 
 cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaStream_t s) {
     const size_t n8 = elems / 8;     // cols is a multiple of 128
-    const unsigned grid = (unsigned)((n8 + 255) / 256 < 148 * 8 ? (n8 + 255) / 256 : 148 * 8);
+    const size_t cap = (size_t)sm_count() * 8;
+    const unsigned grid = (unsigned)((n8 + 255) / 256 < cap ? (n8 + 255) / 256 : cap);
     x_to_f16_kernel<<<grid ? grid : 1, 256, 0, s>>>((const uint4*)x_bf16, (uint4*)x_f16, n8);
     return cudaGetLastError();
 }

@@ -378,7 +378,7 @@ static cudaError_t launch_batch(const BatchArgs& a, dim3 grid, size_t smem, cuda
 cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s) {
     const int rpl = batch_rpl(l.bits);
     const int blocks = (l.RB + rpl - 1) / rpl;
-    constexpr int slots = 148;   // one CTA per SM
+    const int slots = sched_sms();   // one CTA per SM
     for (int b0 = 0; b0 < c.batch; b0 += 8) {
         const int nb = c.batch - b0 < 8 ? c.batch - b0 : 8;
         int nbt = batch_tile(l, nb);

@@ -387,7 +387,7 @@ static cudaError_t launch_batch_v2a(const BatchV2aArgs& a, dim3 grid, size_t sme
 
 cudaError_t launch_gemv_batch_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) {
     const int blocks = (l.RB + 1) / 2;
-    constexpr int slots = 148;   // one CTA per SM
+    const int slots = sched_sms();   // one CTA per SM
     for (int b0 = 0; b0 < c.batch; b0 += 8) {
         const int nb = c.batch - b0 < 8 ? c.batch - b0 : 8;
         const int nbt = batch_v2a_tile(l, nb);

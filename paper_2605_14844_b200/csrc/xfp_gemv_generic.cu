@@ -284,11 +284,11 @@ static int next_pow2(int v) {
     return p;
 }
 
-int generic_ksplit(const Layout& l, int batch_tile) {
+int generic_ksplit(const Layout& l, int batch_tile, int sms) {
     // enough CTAs for about two per SM, never more splits than super-chunks, and a slice of x
     // that fits the shared-memory budget
     int ks = 1;
-    while ((long long)l.RB * ks < 2 * 148 && ks * 2 <= l.SC && ks < 32) ks *= 2;
+    while ((long long)l.RB * ks < 2 * sms && ks * 2 <= l.SC && ks < 32) ks *= 2;
     while ((long long)((l.SC + ks - 1) / ks) * kSuper * batch_tile > kMaxXFloats && ks < l.SC) ks *= 2;
     if (ks > l.SC) ks = l.SC;
     return ks;
@@ -297,7 +297,7 @@ int generic_ksplit(const Layout& l, int batch_tile) {
 size_t generic_workspace_bytes(const Layout& l) {
     int ksmax = 1;
     for (int bt = 1; bt <= 8; bt *= 2) {
-        const int k = generic_ksplit(l, bt);
+        const int k = generic_ksplit(l, bt, kSizingSMs);
         const int spp = (l.SC + k - 1) / k;
         const int keff = (l.SC + spp - 1) / spp;
         if (keff * bt > ksmax) ksmax = keff * bt;
@@ -362,7 +362,7 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
         a.y = c.y ? (void*)((char*)c.y + (size_t)b0 * l.rows * (c.y_is_fp16 ? 2 : 4)) : nullptr;
         a.packed_list = c.packed_list; a.x_list = c.x_list; a.y_list = c.y_list;
         a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.rows_pad = l.rows_pad;
-        const int ks = generic_ksplit(l, bt);
+        const int ks = generic_ksplit(l, bt, sched_sms());
         a.sc_per_split = (l.SC + ks - 1) / ks;
         a.KS = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
         a.nb = nb; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16; a.L = l.L; a.ell_slots = l.ell_slots;

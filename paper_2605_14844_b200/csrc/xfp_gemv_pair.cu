@@ -70,10 +70,12 @@ struct PairArgs {
     // tier_kst[i] slices of tier_spp[i] super-chunks
     int tier_cta[5], tier_blk[4], tier_kst[4], tier_spp[4];
     int cluster;     // single tier with kst > 1: the kst CTAs of a block form a cluster and reduce through DSMEM
-    unsigned long long* trace;  // timing probe: per CTA 8 globaltimer stamps (null in normal use)
+#ifdef XFP_TRACE
+    unsigned long long* trace;  // timing build only: per CTA 8 globaltimer stamps
+#endif
 };
 
-// Phase stamps for the timing probe; compiled in only with -DXFP_TRACE=1 (they cost issue slots).
+// Phase stamps of a timing build (-DXFP_TRACE=1); a normal build has neither the stamps nor their plumbing.
 __device__ __forceinline__ void stamp(const PairArgs& a, int slot) {
 #ifdef XFP_TRACE
     if (a.trace && threadIdx.x == 0) {
@@ -514,29 +516,27 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_pair_kernel(const
 
 // ------------------------------------------------------------------------------------ host side
 
+#ifdef XFP_TRACE
+// timing build only: where the next `calls` launches put their stamps (1024 CTAs x 8 stamps each)
 static unsigned long long* g_pair_trace = nullptr;
 static size_t g_pair_trace_calls = 0, g_pair_trace_idx = 0;
-void pair_set_trace(void* p, size_t calls) {
+extern "C" void xfp_trace_pair(void* p, size_t calls) {
     g_pair_trace = (unsigned long long*)p;
     g_pair_trace_calls = calls;
     g_pair_trace_idx = 0;
 }
-static int g_pair_ks_override = 0;  // probe: force aligned slices
-void pair_set_ksplit_override(int ks) { g_pair_ks_override = ks; }
-void pair_set_prefetch(int) {}
-void pair_set_debug(int) {}
-static int g_pair_small = 1;        // probe switch: one row per lane for matrices with few row blocks
-void pair_set_small(int v) { g_pair_small = v; }
+#endif
 
 struct PairConfig { int rpl, warps, slots; };
 
 static PairConfig pair_config(const Layout& l, int n = 1) {
     // N <= 4: two rows per lane, 8 warps, two CTAs per SM.  N = 5: the pair table of a row is 4 KB, so
-    // one row per lane (128 KB of tables), 16 warps, one CTA per SM.  Matrices with at most 148
-    // row-blocks also take one row per lane: twice the CTAs and no cut along K.
-    if (l.bits == 5) return PairConfig{1, 16, 148};
-    if (g_pair_small >= 1 && (long long)l.RB * n <= 148 * g_pair_small && l.bits >= 3) return PairConfig{1, 16, 148};
-    return PairConfig{2, 8, 296};
+    // one row per lane (128 KB of tables), 16 warps, one CTA per SM.  Matrices with no more row-blocks than
+    // the device has SMs also take one row per lane: twice the CTAs and no cut along K.
+    const int sms = sched_sms();
+    if (l.bits == 5) return PairConfig{1, 16, sms};
+    if ((long long)l.RB * n <= sms && l.bits >= 3) return PairConfig{1, 16, sms};
+    return PairConfig{2, 8, 2 * sms};
 }
 
 struct PairSchedule {
@@ -558,9 +558,7 @@ static PairSchedule pair_schedule(const Layout& l, int n = 1) {
     const int kmax = l.SC / 4 > 1 ? pow2_floor(l.SC / 4) : 1;   // keep K slices of at least 512 weights
     int nb[4] = {0, 0, 0, 0}, kk[4] = {1, 1, 1, 1};
     int nt = 0;
-    if (g_pair_ks_override > 0) {
-        nb[0] = sc.blocks; kk[0] = g_pair_ks_override; nt = 1;
-    } else if (sc.blocks * 2 <= S) {
+    if (sc.blocks * 2 <= S) {
         // fewer blocks than half the CTA slots: cut every block into 2, 4 or 8 K slices that form a cluster
         int kst = 1;
         while (kst < 8 && sc.blocks * kst * 2 <= S && kst * 2 <= kmax) kst *= 2;
@@ -694,10 +692,12 @@ static cudaError_t launch_gemv_pair_n(const Layout& l, const GemvCall& c, int pr
     a.rows_ws = sch.blocks * 32 * cfg.rpl;
     for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
     for (int i = 0; i < 4; ++i) { a.tier_blk[i] = sch.tier_blk[i]; a.tier_kst[i] = sch.tier_kst[i]; a.tier_spp[i] = sch.tier_spp[i]; }
-    a.cluster = sch.cluster && g_pair_ks_override == 0;
+    a.cluster = sch.cluster;
     a.nb = c.batch; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16;
+#ifdef XFP_TRACE
     a.trace = nullptr;
     if (g_pair_trace && g_pair_trace_idx < g_pair_trace_calls) a.trace = g_pair_trace + (g_pair_trace_idx++) * 1024 * 8;
+#endif
     a.tickets = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4 * c.n));
     const size_t smem = pair_smem_bytes(l, c.batch, c.n);

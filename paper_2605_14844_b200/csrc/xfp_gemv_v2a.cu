@@ -529,24 +529,22 @@ static size_t v2a_smem_bytes(const Layout& l, int nb, bool pair, int warps) {
            (size_t)l.L * l.E * 2 + 16;   // + the copy of the library the tables were built from, 16-byte aligned
 }
 
-static int g_v2a_pair = 1;   // probe switch: 0 keeps every layout on the per-bank library, 2 forces pair tables where they fit
-void v2a_set_pair(int v) { g_v2a_pair = v; }
-
 static V2aConfig v2a_config(const Layout& l, int nb, int n = 1) {
     // Pair tables cost 128 KB of fills per resident CTA and run one CTA of 12 or 16 warps per SM: they pay off
     // when every SM has a few hundred thousand weights to decode and K is long enough to keep those warps busy
     // (measured: 28672 x 8192 53 vs 61 us, 8192 x 8192 18.6 vs 22.9, 12288 x 4096 18.7 vs 20.0 in their favour;
     // 4096 x 4096 10.4 vs 9.1 and the routed experts' 4096 x 1536 down projections 20.6 vs 18.7 against them).
     const bool big = (long long)l.rows * l.cols * n >= 40ll * 1000 * 1000 && l.SC >= 32;
-    if (g_v2a_pair && l.bits <= 3 && (big || g_v2a_pair == 2)) {
+    const int sms = sched_sms();
+    if (l.bits <= 3 && big) {
         // K is shared by the warps in super-chunks: 12 warps when that divides the count and 16 does not
         const int warps = (l.SC % 16 != 0 && l.SC % 12 == 0) ? 12 : 16;
         const size_t sm = v2a_smem_bytes(l, nb, true, warps);
-        if (sm <= 224u * 1024u) return V2aConfig{true, warps, 148, sm};
+        if (sm <= 224u * 1024u) return V2aConfig{true, warps, sms, sm};
     }
     const size_t sm8 = v2a_smem_bytes(l, nb, false, 8);
-    if (sm8 <= 110u * 1024u) return V2aConfig{false, 8, 296, sm8};
-    return V2aConfig{false, 16, 148, v2a_smem_bytes(l, nb, false, 16)};   // large library (N = 5): one CTA per SM
+    if (sm8 <= 110u * 1024u) return V2aConfig{false, 8, 2 * sms, sm8};
+    return V2aConfig{false, 16, sms, v2a_smem_bytes(l, nb, false, 16)};   // large library (N = 5): one CTA per SM
 }
 
 bool v2a_supported(const Layout& l, int batch) {

@@ -3,22 +3,37 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "xfp_common.cuh"
 
 namespace xfp {
 
 // Function attributes (the opt-in shared-memory size) belong to a device: every kernel instantiation remembers
 // on which devices it has set them, so a process that drives several GPUs sets them on each.
+// Host threads may race to the first launch: the bits are atomic (setting an attribute twice is harmless, losing
+// another thread's bit is not).
 struct DeviceOnce {
-    unsigned long long mask[4] = {0, 0, 0, 0};   // devices 0..255
+    std::atomic<unsigned long long> mask[4] = {};   // devices 0..255
     static int current() {
         int d = 0;
         cudaGetDevice(&d);
         return d & 255;
     }
-    bool is_set(int d) const { return (mask[d >> 6] >> (d & 63)) & 1ull; }
-    void set(int d) { mask[d >> 6] |= 1ull << (d & 63); }
+    bool is_set(int d) const { return (mask[d >> 6].load(std::memory_order_acquire) >> (d & 63)) & 1ull; }
+    void set(int d) { mask[d >> 6].fetch_or(1ull << (d & 63), std::memory_order_release); }
 };
+
+// Streaming multiprocessors of the current device, asked once per device.  Schedules (CTA slots per round, K
+// splits) are built from it; workspace SIZES are a function of the descriptor alone and never depend on it.
+int sm_count();
+// The SM count the workspace sizes of the split-K kernels allow for: a launch never plans for more SMs than this,
+// so its partial sums fit the size xfp_packed_size reported without asking a device (a B200 has 148).
+constexpr int kSizingSMs = 148;
+inline int sched_sms() {
+    const int n = sm_count();
+    return n < kSizingSMs ? n : kSizingSMs;
+}
 
 struct PackInputs {
     const uint8_t* idx;
@@ -53,8 +68,8 @@ struct GemvCall {
     int x_bf16 = 0;                        // x holds bf16 instead of fp16
 };
 
-// Split-K factor the generic kernel uses for this shape and batch tile (host-side policy).
-int generic_ksplit(const Layout& l, int batch_tile);
+// Split-K factor the generic kernel uses for this shape and batch tile on `sms` SMs (host-side policy).
+int generic_ksplit(const Layout& l, int batch_tile, int sms);
 size_t generic_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t s);
 
@@ -62,17 +77,11 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
 bool pair_supported(const Layout& l, int batch, int n_problems);
 size_t pair_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s);
-void pair_set_ksplit_override(int ks);
-void pair_set_prefetch(int d);
-void pair_set_debug(int m);
-void pair_set_small(int v);
-void pair_set_trace(void* p, size_t calls);
 
 // Fast V2a path (per-bank library + mma.sync fragments, one or several blobs); see xfp_gemv_v2a.cu.
 bool v2a_supported(const Layout& l, int batch);
 size_t v2a_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
-void v2a_set_pair(int v);
 
 // Batched V2 path (3..16 rows of x); see xfp_gemv_batch.cu.
 bool batch_supported(const Layout& l, int batch);

@@ -360,13 +360,14 @@ static bool launch_dequant_lut(const Layout& l, const Blob& b, uint16_t* W, cuda
     }
     // a CTA per row-block; row-blocks too few to fill the GPU are cut along K (at least 8 super-chunks per CTA)
     int parts = 1;
-    while (l.RB * parts < 2 * 148 && l.SC / (parts * 2) >= 8) parts *= 2;
+    const int sms = sm_count();
+    while (l.RB * parts < 2 * sms && l.SC / (parts * 2) >= 8) parts *= 2;
     const int sc_per_cta = (l.SC + parts - 1) / parts;
     parts = (l.SC + sc_per_cta - 1) / sc_per_cta;
     // The outliers are added by the same kernel on small matrices (one launch less: 25.6 -> 23.5 us at 4096 x 4096);
     // on large ones the pass at the end of every CTA is a chain of dependent read-modify-writes and the separate
     // kernel, which spreads them over the whole GPU, is faster (181 against 191 us at 28672 x 8192, 0.3 %).
-    const bool fuse_outliers = (long long)l.RB * l.SC <= 148ll * 64;
+    const bool fuse_outliers = (long long)l.RB * l.SC <= (long long)sms * 64;
     dequant_lut_kernel<N><<<(unsigned)(l.RB * parts), 256, smem, s>>>(b, W, l.rows, l.cols, l.RB, l.SC, sc_per_cta,
                                                                       fuse_outliers ? l.ell_slots : 0);
     *outliers_done = fuse_outliers;

@@ -14,6 +14,7 @@
 #include <cstdint>
 
 #include "../../include/xfp_quant.h"
+#include "xfp_internal.h"   // sm_count()
 
 namespace xq {
 
@@ -294,7 +295,8 @@ template <class Src>
 static cudaError_t run_select(Src src, int64_t n, SelState* st, cudaStream_t s) {
     int blocks = (int)((n + 256 * 16 - 1) / (256 * 16));
     if (blocks < 1) blocks = 1;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    const int cap = xfp::sm_count() * 8;
+    if (blocks > cap) blocks = cap;
     for (int p = 0; p < 8; ++p) {
         sel_hist<Src><<<blocks, 256, 0, s>>>(src, n, st);
         sel_pick<<<1, 1, 0, s>>>(st);
@@ -1082,7 +1084,7 @@ static Workspace carve(void* base, int64_t rows, int64_t cols) {
         size_t kp2 = 1;
         while ((int64_t)kp2 < cols) kp2 <<= 1;
         const size_t slice = (((size_t)cols + 2) & ~(size_t)1) + kp2 / 2;
-        const size_t need = slice * sizeof(double) * (size_t)(rows < 296 ? rows : 296);
+        const size_t need = slice * sizeof(double) * (size_t)(rows < 2 * xfp::kSizingSMs ? rows : 2 * xfp::kSizingSMs);
         if (o < need) o = align256(need);
     }
     w.bytes = o;
@@ -1170,7 +1172,8 @@ int xfp_quant_outliers(const float* W, int64_t n, const double* mu_sigma, int32_
     if (workspace_bytes < tie_offset + (size_t)nblk * sizeof(int)) return XFP_ERR_BUFFER_TOO_SMALL;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(workspace, 1, 128);   // part, sel, flags, then the tie counters
-    const int sweep = (int)(nblk < 148 * 8 ? (nblk < 1 ? 1 : nblk) : 148 * 8);
+    const int64_t sweep_cap = (int64_t)xfp::sm_count() * 8;
+    const int sweep = (int)(nblk < sweep_cap ? (nblk < 1 ? 1 : nblk) : sweep_cap);
     if (outlier_mode == 0) {
         outlier_zero<<<1, 1, 0, s>>>(w.sel);
         mask_threshold<<<sweep, 256, 0, s>>>(W, n, mu_sigma, k_or_rate, mask, w.sel);
@@ -1193,7 +1196,7 @@ int xfp_quant_outliers(const float* W, int64_t n, const double* mu_sigma, int32_
 }
 
 // long channels: resident CTAs, each with a slice of scratch for its two arrays
-static const int kLloydLongCtas = 148 * 2;
+// (the scratch is sized for two CTAs on each of kSizingSMs SMs; a launch never uses more)
 static size_t lloyd_slice_doubles(int cols, int kp2) { return (((size_t)cols + 2) & ~(size_t)1) + (size_t)kp2 / 2; }
 
 int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma, int32_t rows, int32_t cols,
@@ -1216,7 +1219,8 @@ int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma,
         if (!workspace) return XFP_ERR_NULL;
         if (!aligned16(workspace)) return XFP_ERR_ALIGN;
         const size_t slice = lloyd_slice_doubles(cols, kp2);
-        const int ctas = rows < kLloydLongCtas ? rows : kLloydLongCtas;
+        const int want = 2 * xfp::sched_sms();   // two resident CTAs per SM
+        const int ctas = rows < want ? rows : want;
         if (workspace_bytes < slice * sizeof(double) * (size_t)ctas) return XFP_ERR_BUFFER_TOO_SMALL;
         lloyd_kernel<true><<<ctas, kLloydThreads, 0, (cudaStream_t)stream>>>(W, mask, mu_sigma, rows, cols, kp2, bits, iters,
                                                                              codebook, idx, (double*)workspace, slice);

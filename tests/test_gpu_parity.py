@@ -485,6 +485,36 @@ def test_bf16_activations_outside_the_fp16_range_are_clamped():
     assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * absum + 1e-30)
 
 
+@pytest.mark.parametrize("mode,bits,batch", [(0, 4, 1), (0, 6, 4), (1, 3, 1), (1, 6, 1), (1, 6, 3), (1, 4, 8)])
+def test_bf16_nan_and_tiny_activations_on_every_kernel(mode, bits, batch):
+    """A NaN activation must poison y under bf16 as it does under fp16 (the clamp to the fp16 range applies to
+    ordered values only), and bf16 values below 2^-14 are rounded to the fp16 subnormal grid by every kernel the
+    dispatcher can pick -- the generic one (V2a at N = 6) included -- so the result does not depend on that pick."""
+    rows, cols = 96, 512
+    q = synth.random_quantized(mode, rows, cols, bits, 0.01, seed=2950 + 10 * mode + bits)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    # tiny values only: exponents 2^-24 .. 2^-15, 8 significant bits
+    rng = np.random.default_rng(2960 + bits)
+    x64 = np.round(rng.uniform(1, 2, (batch, cols)) * 128) / 128 * 2.0 ** rng.integers(-24, -14, (batch, cols))
+    x64 *= rng.choice([-1.0, 1.0], size=x64.shape)
+    xb = torch.from_numpy(x64).to(torch.bfloat16)
+    assert np.array_equal(xb.to(torch.float64).numpy(), x64)                   # exactly representable in bf16
+    x_grid = xb.to(torch.float16).to(torch.float64).numpy()                    # what the fp16 conversion must give
+    y = torch.empty((batch, rows), dtype=torch.float32, device="cuda")
+    xfp.xfp_gemv_typed(pm.desc, pm.packed, xb.cuda(), batch, y, pm.workspace)
+    torch.cuda.synchronize()
+    ref, absum = xo.gemv_x64(to_oracle(q), x_grid)
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * absum + 1e-30)
+    # one NaN in batch row 0: every output of that row is NaN, the other rows stay finite
+    xn = xb.clone()
+    xn[0, 17] = float("nan")
+    xfp.xfp_gemv_typed(pm.desc, pm.packed, xn.cuda(), batch, y, pm.workspace)
+    torch.cuda.synchronize()
+    got = y.cpu().numpy()
+    assert np.all(np.isnan(got[0]))
+    assert np.all(np.isfinite(got[1:]))
+
+
 @pytest.mark.parametrize("bits,n,rows,cols", [(4, 3, 4096, 4096), (5, 3, 1024, 2048), (3, 2, 9600, 1024), (2, 7, 96, 512),
                                               (6, 4, 2080, 384)])
 def test_grouped_v2_blobs_on_the_pair_kernel(bits, n, rows, cols):
