@@ -220,7 +220,7 @@ def _dev(a, dtype, device):
     if a is None:
         return None
     if isinstance(a, torch.Tensor):
-        return a.to(device=device).contiguous()
+        return a.to(device=device).contiguous() if a.numel() else torch.zeros(16, dtype=a.dtype, device=device)
     a = np.ascontiguousarray(a)
     if a.size == 0:
         return torch.zeros(16, dtype=dtype, device=device)
@@ -269,8 +269,13 @@ def pack_tensors(q, device="cuda", col_bits: int = 32, stream=None) -> PackedMat
     gs = _dev(q.gscale, torch.int16, device) if q.mode else None
     gm = _dev(q.gmid, torch.int16, device) if q.mode else None
     rowptr = _dev(q.rowptr, torch.int32, device)
-    ocol = q.ocol.astype(np.uint16) if col_bits == 16 else q.ocol.astype(np.int32)
-    ocol = _dev(ocol, torch.int16 if col_bits == 16 else torch.int32, device)
+    if isinstance(q.ocol, torch.Tensor):
+        ocol = q.ocol.to(device=device, dtype=torch.int16 if col_bits == 16 else torch.int32)
+        if ocol.numel() == 0:
+            ocol = torch.zeros(16, dtype=ocol.dtype, device=device)
+    else:
+        ocol = q.ocol.astype(np.uint16) if col_bits == 16 else q.ocol.astype(np.int32)
+        ocol = _dev(ocol, torch.int16 if col_bits == 16 else torch.int32, device)
     oval = _dev(q.oval, torch.int16, device)
     packed = torch.empty(pb, dtype=torch.uint8, device=device)
     workspace = torch.zeros(max(wb, 16), dtype=torch.uint8, device=device)

@@ -169,3 +169,76 @@ def random_quantized(mode: int, rows: int, cols: int, bits: int, rate: float, se
     gmid = rng.standard_normal((rows, G)) * (0.1 * SIGMA0)
     return QuantTensors(1, rows, cols, bits, idx, _f16bits(lib), rowptr, ocol, oval, group_size, lib_size,
                         gid, _f16bits(gscale), _f16bits(gmid))
+
+
+def random_quantized_torch(mode: int, rows: int, cols: int, bits: int, rate: float, seed: int,
+                           placement: str = "uniform", lib_size: int = 32, group_size: int = 128,
+                           device="cuda", library=None) -> QuantTensors:
+    """`random_quantized` drawn on a torch device (seeded torch.Generator), for benchmark-sized matrices whose
+    host generation would take minutes: same recipe (bell-shaped indices, ascending codebooks at the weights'
+    scale, library in [-1, 1], group scale / mid-point, CSR outliers placed 'uniform' or 'clustered'), fields as
+    torch tensors on `device` (fp16 values as int16 bit patterns).  `library`: a [L, 2^N] int16 tensor to share
+    between the matrices of a layer.  `to_host` brings such an object back as numpy arrays."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    E = 1 << bits
+    idx = torch.empty((rows, cols), dtype=torch.uint8, device=device)
+    step = max(1, (64 << 20) // cols)
+    for r0 in range(0, rows, step):
+        r1 = min(rows, r0 + step)
+        a = torch.randint(0, E, (r1 - r0, cols), generator=g, device=device, dtype=torch.int16)
+        b = torch.randint(0, E, (r1 - r0, cols), generator=g, device=device, dtype=torch.int16)
+        idx[r0:r1] = torch.clamp((a + b + 1) >> 1, max=E - 1).to(torch.uint8)
+    # outliers
+    if rate <= 0:
+        rowptr = torch.zeros(rows + 1, dtype=torch.int32, device=device)
+        ocol = torch.zeros(0, dtype=torch.int32, device=device)
+    elif placement == "uniform":
+        counts, cs = [], []
+        for r0 in range(0, rows, step):
+            r1 = min(rows, r0 + step)
+            m = torch.rand((r1 - r0, cols), generator=g, device=device) < rate
+            counts.append(m.sum(1))
+            cs.append(m.nonzero()[:, 1])
+        cnt = torch.cat(counts)
+        ocol = torch.cat(cs).to(torch.int32)
+        rowptr = torch.zeros(rows + 1, dtype=torch.int32, device=device)
+        rowptr[1:] = torch.cumsum(cnt, 0).to(torch.int32)
+    elif placement == "clustered":
+        n_hot = max(1, int(round(rate * cols / 0.5)))
+        hot = torch.sort(torch.randperm(cols, generator=g, device=device)[:n_hot]).values
+        hit = torch.rand((rows, n_hot), generator=g, device=device) < 0.5
+        ocol = hot[hit.nonzero()[:, 1]].to(torch.int32)
+        rowptr = torch.zeros(rows + 1, dtype=torch.int32, device=device)
+        rowptr[1:] = torch.cumsum(hit.sum(1), 0).to(torch.int32)
+    else:
+        raise ValueError(placement)
+    nnz = int(ocol.numel())
+    mag = (torch.rand(nnz, generator=g, device=device) * 39.0 + 10.0) * SIGMA0
+    sgn = torch.randint(0, 2, (nnz,), generator=g, device=device).to(torch.float32) * 2 - 1
+    oval = (mag * sgn).to(torch.float16).view(torch.int16)
+    if mode == 0:
+        cb = torch.sort(torch.randn((rows, E), generator=g, device=device) * (2.0 * SIGMA0), dim=1).values
+        return QuantTensors(0, rows, cols, bits, idx, cb.to(torch.float16).view(torch.int16), rowptr, ocol, oval, group_size)
+    if library is None:
+        lib = torch.sort(torch.rand((lib_size, E), generator=g, device=device) * 2.0 - 1.0, dim=1).values
+        library = lib.to(torch.float16).view(torch.int16)
+    G = cols // group_size
+    gid = torch.randint(0, library.shape[0], (rows, G), generator=g, device=device, dtype=torch.int16).to(torch.uint8)
+    gscale = (torch.rand((rows, G), generator=g, device=device) * 2.0 + 2.0) * SIGMA0
+    gmid = torch.randn((rows, G), generator=g, device=device) * (0.1 * SIGMA0)
+    return QuantTensors(1, rows, cols, bits, idx, library, rowptr, ocol, oval, group_size, int(library.shape[0]), gid,
+                        gscale.to(torch.float16).view(torch.int16), gmid.to(torch.float16).view(torch.int16))
+
+
+def to_host(q: QuantTensors) -> QuantTensors:
+    """A QuantTensors whose fields are torch tensors -> the same with numpy arrays (fp16 bit patterns as uint16)."""
+    def h(t, dt):
+        if t is None:
+            return None
+        a = t.cpu().numpy()
+        return np.ascontiguousarray(a.view(np.uint16) if dt == np.uint16 else a.astype(dt))
+    return QuantTensors(q.mode, q.rows, q.cols, q.bits, h(q.idx, np.uint8), h(q.codebook, np.uint16),
+                        h(q.rowptr, np.int32), h(q.ocol, np.int32), h(q.oval, np.uint16), q.group_size, q.lib_size,
+                        h(q.gid, np.uint8), h(q.gscale, np.uint16), h(q.gmid, np.uint16))

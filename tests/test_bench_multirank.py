@@ -55,3 +55,36 @@ def test_block_spec_and_algorithmic_bytes():
     assert bench.algorithmic_bytes(q) == want
     qa = synth.random_quantized(1, 64, 256, 3, 0.0, seed=3)
     assert bench.algorithmic_bytes(qa) == 64 * 256 * 3 // 8 + 32 * 8 * 2 + 64 * 2 * 5 + 65 * 4 + 256 * 2 + 64 * 2
+
+
+def test_stack_spec_matches_the_configuration():
+    """The headline workload's per-layer draws: 48 layers, bit widths from {2..6}, outlier rates within [0, 2 %]."""
+    from paper_2605_14844_b200 import workloads as wl
+    spec = wl.stack_spec()
+    assert len(spec) == 48 and spec == wl.stack_spec()                    # seeded
+    assert {b for b, _ in spec} == {2, 3, 4, 5, 6}
+    assert all(0.0 <= r <= 0.02 for _, r in spec)
+    assert wl.STACK_SHAPES == [(4096, 4096)] * 4 + [(12288, 4096), (4096, 12288)]
+    total = sum(wl.algorithmic_bytes(0, r, c, b, int(rate * r * c)) for b, rate in spec for r, c in wl.STACK_SHAPES)
+    assert 3.5e9 < total < 5.5e9                                          # about 4.4 GB per token
+
+
+def test_device_generator_follows_the_host_recipe():
+    """synth.random_quantized_torch (here on the CPU device) gives tensors of the recipe's shapes, ranges and
+    structure; to_host returns them in the oracle's types."""
+    from paper_2605_14844_b200 import synth
+    for mode in (0, 1):
+        for placement in ("uniform", "clustered"):
+            q = synth.to_host(synth.random_quantized_torch(mode, 96, 512, 3, 0.01, 5, placement, device="cpu"))
+            assert q.idx.shape == (96, 512) and q.idx.dtype == np.uint8 and q.idx.max() <= 7
+            assert q.rowptr[0] == 0 and q.rowptr[-1] == q.ocol.size == q.oval.size
+            assert 0.5 * 0.01 * 96 * 512 < q.nnz < 1.5 * 0.01 * 96 * 512
+            for i in range(96):
+                c = q.ocol[q.rowptr[i]:q.rowptr[i + 1]]
+                assert np.all(np.diff(c) > 0) and (c.size == 0 or (0 <= c[0] and c[-1] < 512))
+            cb = q.codebook.view(np.float16).astype(np.float64)
+            assert np.all(np.diff(cb, axis=1) >= 0)
+            mag = np.abs(q.oval.view(np.float16).astype(np.float64))
+            assert np.all((mag >= 0.199) & (mag <= 0.981))                # 10..49 sigma
+            if mode:
+                assert q.gid.shape == (96, 4) and q.gid.max() < 32 and q.codebook.shape == (32, 8)
