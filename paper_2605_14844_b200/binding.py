@@ -38,7 +38,8 @@ class XfpDesc(C.Structure):
 
 
 def library_path() -> str:
-    return os.path.join(_HERE, "libxfp.so")
+    """libxfp.so beside this file; XFP_LIBRARY names another build of it (see build.py, XFP_LIBTAG)."""
+    return os.environ.get("XFP_LIBRARY") or os.path.join(_HERE, "libxfp.so")
 
 
 def load_library() -> C.CDLL:

@@ -8,14 +8,18 @@ from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-OBJ = os.path.join(CSRC, "build")
-LIB = os.path.join(HERE, "libxfp.so")
+OBJ = os.path.join(CSRC, "build" + ("_" + os.environ["XFP_LIBTAG"] if os.environ.get("XFP_LIBTAG") else ""))
+# XFP_LIBTAG=name builds libxfp_name.so from objects of its own (csrc/build_name), with the extra -D flags of
+# XFP_DEFS: a way to keep several builds side by side when comparing kernel variants
+TAG = os.environ.get("XFP_LIBTAG", "")
+LIB = os.path.join(HERE, f"libxfp_{TAG}.so" if TAG else "libxfp.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 # XFP_TRACE=1 compiles the per-CTA phase stamps of the pair kernel in (a timing probe; use with --force)
 if os.environ.get("XFP_TRACE") == "1":
     FLAGS.append("-DXFP_TRACE=1")
+FLAGS += [f"-D{d}" for d in os.environ.get("XFP_DEFS", "").split()]
 
 
 def _sources():

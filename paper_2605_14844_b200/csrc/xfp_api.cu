@@ -70,7 +70,9 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
         e = launch_gemv_v2a(l, cc, (cudaStream_t)stream);
         return e == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
     }
-    if (pair_supported(l, c.batch, c.n))
+    if (lane_supported(l, cc))
+        e = launch_gemv_lane(l, cc, (cudaStream_t)stream);
+    else if (pair_supported(l, c.batch, c.n))
         e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && batch_supported(l, c.batch))
         e = launch_gemv_batch(l, cc, (cudaStream_t)stream);

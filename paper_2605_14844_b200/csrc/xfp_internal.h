@@ -78,6 +78,10 @@ bool pair_supported(const Layout& l, int batch, int n_problems);
 size_t pair_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s);
 
+// V2 at batch 1, one channel per lane, half an SM per CTA; see xfp_gemv_lane.cu.
+bool lane_supported(const Layout& l, const GemvCall& c);
+cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s);
+
 // Fast V2a path (per-bank library + mma.sync fragments, one or several blobs); see xfp_gemv_v2a.cu.
 bool v2a_supported(const Layout& l, int batch);
 size_t v2a_workspace_bytes(const Layout& l);
