@@ -6,9 +6,9 @@
  * Q: dense N-bit indices (N in 2..6, "Sub-Byte Packing"); S: sparse fp16 outlier residual.
  * Two codebook storage modes ("The XFP Format"):
  *   V2  : one fp16 codebook of 2^N entries per output channel:  D_ik = codebook_i[q_ik]
- *   V2a : a per-layer library of L codebooks; every group of 128 consecutive k of one channel
- *         carries a library id, an fp16 scale and an fp16 mid-point
- *         ("V2a: Shared Codebook Library"):  D_ik = mid_ig + scale_ig * lib[id_ig][q_ik],  g = k / 128
+ *   V2a : a per-layer library of L codebooks; every group of G consecutive k of one channel (G = 128 in the
+ *         paper, "a tunable parameter": 64, 128 and 256 are built) carries a library id, an fp16 scale and an
+ *         fp16 mid-point ("V2a: Shared Codebook Library"):  D_ik = mid_ig + scale_ig * lib[id_ig][q_ik],  g = k / G
  * The hot path is the fused decode kernel y = (D + S) x of "Fused Decode Kernel": depack, codebook
  * gather, outlier add and multiply-accumulate in one launch, fp32 accumulation.
  *
@@ -68,9 +68,11 @@ typedef enum {
 
 typedef struct {
     int32_t mode;       /* 0 = V2 (per-channel codebook), 1 = V2a (library + per-group id)          */
-    int32_t rows, cols; /* output channels; input features K, a multiple of group_size, <= 65536    */
+    int32_t rows, cols; /* output channels; input features K, a multiple of group_size and of 128, <= 65536 */
     int32_t bits;       /* N in {2,3,4,5,6}, both modes (the paper's own V2a kernel: {2,4} only)    */
-    int32_t group_size; /* 128                                                                      */
+    int32_t group_size; /* 64, 128 or 256 (others: XFP_ERR_UNSUPPORTED).  V2a: weights per (id, scale, mid);
+                           V2 has no per-group data and only the divisibility of cols is checked.  Groups of
+                           64 run on the general kernels (GEMV, dequant, GEMM), not on the fast V2a GEMV paths */
     int32_t lib_size;   /* V2a: L in 1..256 (paper default 32); V2: 0                               */
     int32_t col_bits;   /* width of the CSR column indices handed to xfp_pack: 16 or 32             */
     int64_t nnz;        /* number of outliers, 0 <= nnz < 2^31                                      */

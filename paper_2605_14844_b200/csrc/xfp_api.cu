@@ -31,8 +31,10 @@ int check_desc(const xfp_desc* d) {
     if (d->mode != 0 && d->mode != 1) return XFP_ERR_SHAPE;
     if (d->rows <= 0 || d->cols <= 0) return XFP_ERR_SHAPE;
     if (d->bits < 2 || d->bits > 6) return XFP_ERR_SHAPE;
-    if (d->group_size != 128) return d->group_size > 0 ? XFP_ERR_UNSUPPORTED : XFP_ERR_SHAPE;
-    if (d->cols % d->group_size) return XFP_ERR_SHAPE;
+    if (d->group_size <= 0) return XFP_ERR_SHAPE;
+    if (d->group_size != 64 && d->group_size != 128 && d->group_size != 256) return XFP_ERR_UNSUPPORTED;
+    // the device layout walks K in super-chunks of 128 weights, whatever the group size
+    if (d->cols % d->group_size || d->cols % 128) return XFP_ERR_SHAPE;
     if (d->cols > 65536) return XFP_ERR_UNSUPPORTED;
     if (d->mode == 1 && (d->lib_size < 1 || d->lib_size > 256)) return XFP_ERR_SHAPE;
     if (d->mode == 0 && d->lib_size != 0) return XFP_ERR_SHAPE;
@@ -43,7 +45,9 @@ int check_desc(const xfp_desc* d) {
     return XFP_OK;
 }
 
-Layout layout_of(const xfp_desc* d) { return make_layout(d->mode, d->rows, d->cols, d->bits, d->lib_size, d->nnz); }
+Layout layout_of(const xfp_desc* d) {
+    return make_layout(d->mode, d->rows, d->cols, d->bits, d->lib_size, d->nnz, d->group_size);
+}
 
 int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* stream) {
     int st = check_desc(desc);

@@ -61,6 +61,7 @@ struct GemmArgs {
     int rows, cols, RB, SC, M, ell_slots, ks, sc_per_slice, y_kind;
     int tab_bytes;    // shared-memory bytes of the look-up tables (the x stages follow)
     int L;            // V2a: library size
+    int GH;           // V2a: groups per super-chunk (2 when the format's groups hold 64 weights)
     int maxT;         // rows of x per tile: kSmallT or kBigT; the accumulator's columns and the first column of the A stages
     int tmem_cols;    // tensor-memory columns of the CTA: 2 * maxT
     int x_stages;     // x tiles in shared memory: kXStages, or 2 when three large ones do not fit
@@ -197,11 +198,13 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
             }
         }
     }
-    // V2a: library id, scale and mid-point of the lane's channel in the next super-chunk (= group), one ahead
-    const size_t meta0 = ((size_t)rb * a.SC + sc0) * 32 + lane;
+    // V2a: library id, scale and mid-point of the lane's channel for this warp's half of the next super-chunk, one
+    // ahead.  A half is 64 weights: a group of its own when the format's groups hold 64 weights (GH = 2), else half
+    // of the super-chunk's group.
+    const size_t meta0 = (((size_t)rb * a.SC + sc0) * a.GH + (a.GH - 1) * PART) * 32 + lane;
     uint32_t gid_n = 0, gsm_n = 0;
     if (MODE == 1 && rb_ok && sc0 + grp < sc1) {
-        gid_n = __ldg(a.b.gid + meta0 + (size_t)grp * 32); gsm_n = __ldg(a.b.gsm + meta0 + (size_t)grp * 32);
+        gid_n = __ldg(a.b.gid + meta0 + (size_t)grp * a.GH * 32); gsm_n = __ldg(a.b.gsm + meta0 + (size_t)grp * a.GH * 32);
     }
     bool ok = true;
     int it = grp;
@@ -240,7 +243,7 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                 g_scale = __low2float(sm); g_mid = __high2float(sm);
                 vbase = tbase | (gid_n << (7 + N));
                 if (sc + G < sc1) {
-                    const size_t mi = meta0 + (size_t)(it + G) * 32;
+                    const size_t mi = meta0 + (size_t)(it + G) * a.GH * 32;
                     gid_n = __ldg(a.b.gid + mi); gsm_n = __ldg(a.b.gsm + mi);
                 }
             }
@@ -627,6 +630,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.ctrl = (int*)c.workspace;
     a.partial = (float*)((char*)c.workspace + gemm_ctrl_bytes(l, c.M));
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
+    a.GH = l.GH;
     a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_half = b_half;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
     a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;

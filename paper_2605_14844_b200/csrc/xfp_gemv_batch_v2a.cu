@@ -354,7 +354,9 @@ static int batch_v2a_tile(const Layout& l, int batch) {
     return 0;
 }
 
-bool batch_v2a_supported(const Layout& l, int batch) { return batch > 2 && batch_v2a_tile(l, batch) != 0; }
+bool batch_v2a_supported(const Layout& l, int batch) {
+    return batch > 2 && l.GH == 1 && batch_v2a_tile(l, batch) != 0;   // groups of 64 weights go to the generic kernel
+}
 
 template <int N, int NB, bool TIO>
 static cudaError_t launch_batch_v2a_io(const BatchV2aArgs& a, dim3 grid, size_t smem, cudaStream_t s) {

@@ -31,6 +31,7 @@ struct GenericArgs {
     int* tickets;    // [problem][RB]
     int rows, cols, RB, SC, rows_pad;
     int KS, sc_per_split, nb, y_is_fp16, L, rep, ell_slots, x_bf16;
+    int GH;   // V2a: groups per super-chunk (2 when the format's groups hold 64 weights)
 };
 
 template <int N, int MODE, int BT>
@@ -52,14 +53,16 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
     const int tab_floats = MODE == 0 ? E * 32 : a.L * E * a.rep;
     float* tab = smem;
     float* xs = tab + tab_floats;                   // [BT][kseg]
-    float* xg = xs + BT * kseg;                     // [BT][sc_per_split]   (V2a group sums of x)
-    float* red = xg + BT * a.sc_per_split;          // [warps][BT][32]
+    float* xg = xs + BT * kseg;                     // [BT][sc_per_split][2]   (V2a: sums of x over the halves of a super-chunk)
+    float* red = xg + BT * a.sc_per_split * 2;      // [warps][BT][32]
 
     // ---- start streaming: first super-chunk of this warp, its group metadata, first outlier slots
     uint32_t cur[4 * N + 1], nxt[4 * N + 1];
     cur[4 * N] = nxt[4 * N] = 0u;
     const uint4* ibase = b.idx + ((size_t)(rb * a.SC + sc0) * N) * 32 + lane;
-    uint32_t gid_c = 0, gsm_c = 0, gid_n = 0, gsm_n = 0;
+    // group metadata of the current and the next super-chunk; [1] is the second half's group when GH = 2, else a copy
+    uint32_t gid_c[2] = {0, 0}, gsm_c[2] = {0, 0}, gid_n[2] = {0, 0}, gsm_n[2] = {0, 0};
+    const int GH = MODE == 1 ? a.GH : 1;
     if (warp < nsc) {
 #pragma unroll
         for (int v = 0; v < N; ++v) {
@@ -67,9 +70,11 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
             cur[4 * v] = t.x; cur[4 * v + 1] = t.y; cur[4 * v + 2] = t.z; cur[4 * v + 3] = t.w;
         }
         if (MODE == 1) {
-            const size_t unit = (size_t)(rb * a.SC + sc0 + warp) * 32 + lane;
-            gid_c = b.gid[unit];
-            gsm_c = b.gsm[unit];
+            const size_t unit = (size_t)(rb * a.SC + sc0 + warp) * GH;
+            gid_c[0] = b.gid[unit * 32 + lane];
+            gsm_c[0] = b.gsm[unit * 32 + lane];
+            gid_c[1] = b.gid[(unit + GH - 1) * 32 + lane];
+            gsm_c[1] = b.gsm[(unit + GH - 1) * 32 + lane];
         }
     }
     // outlier slab of this row-block: slots gw, gw + stride, ... belong to this warp (first round fetched
@@ -121,8 +126,8 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
             const float4 v = *(const float4*)(xs + bb * kseg + s * kSuper + lane * 4);
             float t = (v.x + v.y) + (v.z + v.w);
 #pragma unroll
-            for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-            if (lane == 0) xg[bb * a.sc_per_split + s] = t;
+            for (int o = 8; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);   // lanes 0 and 16: the two halves
+            if ((lane & 15) == 0) xg[(bb * a.sc_per_split + s) * 2 + (lane >> 4)] = t;
         }
         __syncthreads();  // xg visible to every warp
     }
@@ -163,9 +168,11 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
                 nxt[4 * v] = t.x; nxt[4 * v + 1] = t.y; nxt[4 * v + 2] = t.z; nxt[4 * v + 3] = t.w;
             }
             if (MODE == 1) {
-                const size_t unit_n = (size_t)(rb * a.SC + sc0 + sn) * 32 + lane;
-                gid_n = b.gid[unit_n];
-                gsm_n = b.gsm[unit_n];
+                const size_t unit_n = (size_t)(rb * a.SC + sc0 + sn) * GH;
+                gid_n[0] = b.gid[unit_n * 32 + lane];
+                gsm_n[0] = b.gsm[unit_n * 32 + lane];
+                gid_n[1] = b.gid[(unit_n + GH - 1) * 32 + lane];
+                gsm_n[1] = b.gsm[(unit_n + GH - 1) * 32 + lane];
             }
         }
         if (oround < nrounds) {
@@ -192,39 +199,43 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
                 }
             }
         } else {
-            const uint32_t id = gid_c;
-            const uint32_t sm = gsm_c;
-            const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
-            const float* t = tab + (size_t)id * E * a.rep + (a.rep == 32 ? lane : 0);
-            float gs[BT];
+            // the two halves of the super-chunk: one group each when GH = 2, the same group otherwise
 #pragma unroll
-            for (int bb = 0; bb < BT; ++bb) gs[bb] = 0.f;
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t id = gid_c[h];
+                const uint32_t sm = gsm_c[h];
+                const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
+                const float* t = tab + (size_t)id * E * a.rep + (a.rep == 32 ? lane : 0);
+                float gs[BT];
 #pragma unroll
-            for (int j4 = 0; j4 < kSuper / 4; ++j4) {
-                float4 xv[BT];
+                for (int bb = 0; bb < BT; ++bb) gs[bb] = 0.f;
 #pragma unroll
-                for (int bb = 0; bb < BT; ++bb) xv[bb] = *(const float4*)(xrow + bb * kseg + j4 * 4);
-                const float w0 = t[field<N>(cur, j4 * 4 + 0) * a.rep];
-                const float w1 = t[field<N>(cur, j4 * 4 + 1) * a.rep];
-                const float w2 = t[field<N>(cur, j4 * 4 + 2) * a.rep];
-                const float w3 = t[field<N>(cur, j4 * 4 + 3) * a.rep];
+                for (int j4 = h * (kSuper / 8); j4 < (h + 1) * (kSuper / 8); ++j4) {
+                    float4 xv[BT];
 #pragma unroll
-                for (int bb = 0; bb < BT; ++bb) {
-                    gs[bb] = fmaf(w0, xv[bb].x, gs[bb]);
-                    gs[bb] = fmaf(w1, xv[bb].y, gs[bb]);
-                    gs[bb] = fmaf(w2, xv[bb].z, gs[bb]);
-                    gs[bb] = fmaf(w3, xv[bb].w, gs[bb]);
+                    for (int bb = 0; bb < BT; ++bb) xv[bb] = *(const float4*)(xrow + bb * kseg + j4 * 4);
+                    const float w0 = t[field<N>(cur, j4 * 4 + 0) * a.rep];
+                    const float w1 = t[field<N>(cur, j4 * 4 + 1) * a.rep];
+                    const float w2 = t[field<N>(cur, j4 * 4 + 2) * a.rep];
+                    const float w3 = t[field<N>(cur, j4 * 4 + 3) * a.rep];
+#pragma unroll
+                    for (int bb = 0; bb < BT; ++bb) {
+                        gs[bb] = fmaf(w0, xv[bb].x, gs[bb]);
+                        gs[bb] = fmaf(w1, xv[bb].y, gs[bb]);
+                        gs[bb] = fmaf(w2, xv[bb].z, gs[bb]);
+                        gs[bb] = fmaf(w3, xv[bb].w, gs[bb]);
+                    }
                 }
-            }
-            // sum_k (mid + scale*lib) x = scale * sum lib*x + mid * sum x
+                // sum_k (mid + scale*lib) x = scale * sum lib*x + mid * sum x, over this half
 #pragma unroll
-            for (int bb = 0; bb < BT; ++bb)
-                acc[bb] = fmaf(scale, gs[bb], fmaf(mid, xg[bb * a.sc_per_split + s], acc[bb]));
+                for (int bb = 0; bb < BT; ++bb)
+                    acc[bb] = fmaf(scale, gs[bb], fmaf(mid, xg[(bb * a.sc_per_split + s) * 2 + h], acc[bb]));
+            }
         }
 #pragma unroll
         for (int i = 0; i < 4 * N; ++i) cur[i] = nxt[i];
-        gid_c = gid_n;
-        gsm_c = gsm_n;
+        gid_c[0] = gid_n[0]; gid_c[1] = gid_n[1];
+        gsm_c[0] = gsm_n[0]; gsm_c[1] = gsm_n[1];
     }
     while (oround < nrounds) {   // more outlier rounds than super-chunks
         consume_slots();
@@ -366,6 +377,7 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
         a.sc_per_split = (l.SC + ks - 1) / ks;
         a.KS = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
         a.nb = nb; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16; a.L = l.L; a.ell_slots = l.ell_slots;
+        a.GH = l.GH;
         // V2a: a per-bank copy of the library when it fits, else a single copy (bank conflicts)
         a.rep = (l.mode && (size_t)l.L * l.E * 32 * 4 <= 128 * 1024) ? 32 : 1;
         // grouped calls stride the workspace by the per-problem size the caller was told
@@ -373,7 +385,7 @@ cudaError_t launch_gemv_generic(const Layout& l, const GemvCall& c, cudaStream_t
         a.partial = (float*)((char*)c.workspace + align256(ticket_bytes * (size_t)c.n));
         (void)per_problem;
         const size_t tab = l.mode ? (size_t)l.L * l.E * a.rep : (size_t)l.E * 32;
-        const size_t smem = 4 * (tab + (size_t)bt * a.sc_per_split * kSuper + (size_t)bt * a.sc_per_split +
+        const size_t smem = 4 * (tab + (size_t)bt * a.sc_per_split * kSuper + (size_t)bt * a.sc_per_split * 2 +
                                  (size_t)kGenericWarps * bt * 32);
         dim3 grid((unsigned)l.RB, (unsigned)a.KS, (unsigned)c.n);
         cudaError_t e = l.mode ? launch_n<1>(l.bits, bt, a, grid, smem, s) : launch_n<0>(l.bits, bt, a, grid, smem, s);

@@ -549,6 +549,7 @@ static V2aConfig v2a_config(const Layout& l, int nb, int n = 1) {
 
 bool v2a_supported(const Layout& l, int batch) {
     if (l.mode != 1 || l.bits < 2 || l.bits > 5 || batch > 2) return false;
+    if (l.GH != 1) return false;   // groups of 64 weights: two table bases per super-chunk, served by the generic kernel
     const V2aConfig cfg = v2a_config(l, batch);
     return cfg.smem <= (cfg.warps == 8 ? 110u : 224u) * 1024u;
 }

@@ -9,8 +9,11 @@
 //           stream of 128*N bits (index j at bits [j*N, j*N+N)); vector v holds bits
 //           [128 v, 128 v + 128).  A warp-wide load of vector v is one contiguous 512-byte read.
 //   cb      V2: fp16 [rows_pad][2^N] (padding rows zero);  V2a: fp16 [L][2^N]
-//   gid     V2a: u8  [RB][SC][32]      library id of (channel rb*32+l, group sc)
-//   gsm     V2a: half2 [RB][SC][32]    (scale, mid) of the same group
+//   gid     V2a: u8  [RB][SC][GH][32]  library id of channel rb*32+l for part h of super-chunk sc
+//   gsm     V2a: half2 [RB][SC][GH][32] (scale, mid) of the same part
+//           The format's group size G is 64, 128 or 256 weights.  A super-chunk holds GH = 2 groups at G = 64 and
+//           one otherwise; a group of 256 spans two super-chunks and its metadata is stored with both (the
+//           decode kernels then see one (id, scale, mid) per 128 weights, whatever G is above 64).
 //   rowptr  int32 [rows_pad + 1]       clamped to [0, nnz]
 //   hdr     256 bytes                  {int32 ell_slots, int32 0, int64 off_ell}: the two values of this layout that
 //                                      depend on nnz, for launches over several blobs of one shape whose outlier
@@ -33,6 +36,7 @@ constexpr int kSuper = 128;
 
 struct Layout {
     int mode, rows, cols, bits, L, E;
+    int G, GH;   // group size of the format (64, 128, 256); groups per super-chunk (2 at G = 64, else 1)
     int RB, SC, rows_pad;
     long long nnz;
     size_t off_idx, off_cb, off_gid, off_gsm, off_rowptr, off_hdr, off_oent, off_ell, total;
@@ -52,9 +56,10 @@ inline int ell_slots(long long nnz, int rows) {
     return (int)(c > 65535 ? 65535 : c);
 }
 
-inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, long long nnz) {
+inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, long long nnz, int group_size = 128) {
     Layout l{};
     l.mode = mode; l.rows = rows; l.cols = cols; l.bits = bits; l.L = mode ? lib_size : 0; l.E = 1 << bits;
+    l.G = group_size; l.GH = (mode && group_size == 64) ? 2 : 1;
     l.RB = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
     l.SC = cols / kSuper;
     l.rows_pad = l.RB * kRowsPerBlock;
@@ -62,8 +67,8 @@ inline Layout make_layout(int mode, int rows, int cols, int bits, int lib_size, 
     size_t o = 0;
     l.off_idx = o;    o = align256(o + (size_t)l.RB * l.SC * bits * 512);
     l.off_cb = o;     o = align256(o + (size_t)(mode ? l.L : l.rows_pad) * l.E * 2);
-    l.off_gid = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * 32 : 0));
-    l.off_gsm = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * 32 * 4 : 0));
+    l.off_gid = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * l.GH * 32 : 0));
+    l.off_gsm = o;    o = align256(o + (mode ? (size_t)l.RB * l.SC * l.GH * 32 * 4 : 0));
     l.off_rowptr = o; o = align256(o + (size_t)(l.rows_pad + 1) * 4);
     l.off_hdr = o;    o = align256(o + 256);
     l.off_oent = o;   o = align256(o + (size_t)nnz * 4);

@@ -53,21 +53,28 @@ __global__ void pack_codebook_kernel(const uint16_t* __restrict__ cb, uint16_t* 
 
 __global__ void pack_group_kernel(const uint8_t* __restrict__ gid, const uint16_t* __restrict__ gscale,
                                   const uint16_t* __restrict__ gmid, uint8_t* __restrict__ out_gid,
-                                  uint32_t* __restrict__ out_gsm, int rows, int RB, int SC, int L, int* err_word) {
+                                  uint32_t* __restrict__ out_gsm, int rows, int RB, int SC, int L, int G, int GH,
+                                  int* err_word) {
+    // one thread per (row-block, super-chunk, part of the super-chunk, lane); the group that holds the part's first
+    // weight supplies its metadata (a group of 256 weights is stored with both of its super-chunks)
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= (long long)RB * SC * 32) return;
+    if (t >= (long long)RB * SC * GH * 32) return;
     const int lane = (int)(t & 31);
-    const long long unit = t >> 5;
+    const long long part = t >> 5;
+    const long long unit = part / GH;
+    const int h = (int)(part % GH);
     const int rb = (int)(unit / SC), sc = (int)(unit % SC);
     const int row = rb * kRowsPerBlock + lane;
+    const int groups = SC * kSuper / G;                        // groups per channel
+    const int grp = (sc * kSuper + h * (kSuper / GH)) / G;
     uint32_t id = 0, sm = 0;
     if (row < rows) {
-        id = gid[(size_t)row * SC + sc];
+        id = gid[(size_t)row * groups + grp];
         if ((int)id >= L) {
             if (err_word) atomicOr(err_word, 2);
             id = (uint32_t)(L - 1);
         }
-        sm = (uint32_t)gscale[(size_t)row * SC + sc] | ((uint32_t)gmid[(size_t)row * SC + sc] << 16);
+        sm = (uint32_t)gscale[(size_t)row * groups + grp] | ((uint32_t)gmid[(size_t)row * groups + grp] << 16);
     }
     out_gid[t] = (uint8_t)id;
     out_gsm[t] = sm;
@@ -165,11 +172,11 @@ cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int
     pack_codebook_kernel<<<(unsigned)((n_dst + 255) / 256), 256, 0, s>>>(in.codebook, (uint16_t*)(base + l.off_cb), n_src,
                                                                         n_dst);
     if (l.mode) {
-        const long long n = (long long)l.RB * l.SC * 32;
+        const long long n = (long long)l.RB * l.SC * l.GH * 32;
         pack_group_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(in.gid, in.gscale, in.gmid,
                                                                      (uint8_t*)(base + l.off_gid),
                                                                      (uint32_t*)(base + l.off_gsm), l.rows, l.RB, l.SC,
-                                                                     l.L, err_word);
+                                                                     l.L, l.G, l.GH, err_word);
     }
     pack_rowptr_kernel<<<(unsigned)((l.rows_pad + 1 + 255) / 256), 256, 0, s>>>(
         l.nnz ? in.rowptr : nullptr, in.ocol, in.col_bits, (int*)(base + l.off_rowptr), l.rows, l.rows_pad, l.nnz,
@@ -194,7 +201,7 @@ constexpr int kTileStride = 130;  // halves per tile row: 65 words, so 32 lanes 
 // shared tile, then the warp writes the tile row by row (256 contiguous bytes per row).
 template <int N, int MODE>
 __global__ void __launch_bounds__(128) dequant_kernel(Blob b, uint16_t* __restrict__ W, int rows, int cols, int RB,
-                                                      int SC) {
+                                                      int SC, int GH) {
     constexpr int E = 1 << N;
     __shared__ uint16_t tile[4][32 * kTileStride];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -216,14 +223,15 @@ __global__ void __launch_bounds__(128) dequant_kernel(Blob b, uint16_t* __restri
 #pragma unroll
         for (int j = 0; j < kSuper; ++j) trow[j] = __ldg(cb + field<N>(w, j));
     } else {
-        const uint32_t id = b.gid[(size_t)unit * 32 + lane];
-        const uint32_t sm = b.gsm[(size_t)unit * 32 + lane];
-        const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
-        const uint16_t* lib = b.cb + (size_t)id * E;
+        // one group per super-chunk, or two groups of 64 weights (GH = 2)
+        const size_t m0 = ((size_t)unit * GH) * 32 + lane, m1 = ((size_t)unit * GH + (GH - 1)) * 32 + lane;
+        const uint32_t id0 = b.gid[m0], sm0 = b.gsm[m0], id1 = b.gid[m1], sm1 = b.gsm[m1];
 #pragma unroll
         for (int j = 0; j < kSuper; ++j) {
+            const uint32_t id = j < kSuper / 2 ? id0 : id1, sm = j < kSuper / 2 ? sm0 : sm1;
+            const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
             // scale*lib is exact in fp32; one fp32 rounding for the sum, one fp16 rounding after it
-            const float d = __fmaf_rn(scale, h2f(__ldg(lib + field<N>(w, j))), mid);
+            const float d = __fmaf_rn(scale, h2f(__ldg(b.cb + (size_t)id * E + field<N>(w, j))), mid);
             trow[j] = f2h(d);
         }
     }
@@ -382,9 +390,9 @@ static bool launch_dequant_n(const Layout& l, const Blob& b, uint16_t* W, cudaSt
     const long long units = (long long)l.RB * l.SC;
     const unsigned grid = (unsigned)((units + 3) / 4);
     if (l.mode == 0)
-        dequant_kernel<N, 0><<<grid, 128, 0, s>>>(b, W, l.rows, l.cols, l.RB, l.SC);
+        dequant_kernel<N, 0><<<grid, 128, 0, s>>>(b, W, l.rows, l.cols, l.RB, l.SC, 1);
     else
-        dequant_kernel<N, 1><<<grid, 128, 0, s>>>(b, W, l.rows, l.cols, l.RB, l.SC);
+        dequant_kernel<N, 1><<<grid, 128, 0, s>>>(b, W, l.rows, l.cols, l.RB, l.SC, l.GH);
     return false;
 }
 

@@ -111,9 +111,24 @@ def test_packed_size_accounting(lib):
     assert pa >= 3072 * 4096 * 3 // 8 + 3072 * 32 * 5 + 32 * 8 * 2
 
 
+def test_group_sizes_64_128_256_are_accepted(lib):
+    """The format's group size is a parameter: 64, 128 and 256 weights per group are built; the packed size of a
+    V2a blob grows with the number of metadata slots (two per super-chunk at 64, one otherwise)."""
+    sizes = {}
+    for g in (64, 128, 256):
+        pb, wb = C.c_size_t(), C.c_size_t()
+        assert lib.xfp_packed_size(C.byref(_desc(mode=1, lib_size=32, rows=64, cols=1024, group_size=g)), C.byref(pb),
+                                   C.byref(wb)) == 0
+        sizes[g] = pb.value
+        assert lib.xfp_packed_size(C.byref(_desc(rows=64, cols=1024, group_size=g)), C.byref(pb), C.byref(wb)) == 0
+    assert sizes[64] > sizes[128]
+    assert sizes[256] == sizes[128]
+
+
 @pytest.mark.parametrize("kw,status", [
     (dict(bits=1), 3), (dict(bits=7), 3), (dict(cols=200), 3), (dict(rows=0), 3), (dict(mode=2), 3),
-    (dict(group_size=64), 4), (dict(cols=131072), 4), (dict(mode=1, lib_size=0), 3), (dict(mode=1, lib_size=300), 3),
+    (dict(group_size=80), 4), (dict(group_size=512), 4), (dict(group_size=0), 3), (dict(group_size=64, cols=192), 3),
+    (dict(group_size=256, cols=384), 3), (dict(cols=131072), 4), (dict(mode=1, lib_size=0), 3), (dict(mode=1, lib_size=300), 3),
     (dict(mode=0, lib_size=32), 3), (dict(col_bits=8), 3), (dict(nnz=-1), 3),
 ])
 def test_bad_descriptors_are_rejected(lib, kw, status):

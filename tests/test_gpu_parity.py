@@ -76,6 +76,39 @@ def test_gemv_within_bound_small(mode, bits, batch):
     _check_gemv(q, pm, x16, y_fp16=True)
 
 
+@pytest.mark.parametrize("group", [64, 256])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6])
+def test_v2a_group_sizes_other_than_128(group, bits):
+    """The group size is a parameter of the format ("Lane geometry"): V2a blobs with 64 and 256 weights per
+    (id, scale, mid).  Reconstruction is bit-exact and the fused GEMV stays inside the bound at batch 1, 2, 5 and
+    16 -- groups of 256 on the fast kernels (their metadata is stored with both super-chunks), groups of 64 on the
+    general one -- and the prefill form agrees too."""
+    rows, cols = 200, 1024
+    q = synth.random_quantized(1, rows, cols, bits, 0.01, seed=8100 + 10 * bits + group, group_size=group)
+    assert q.gid.shape == (rows, cols // group)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    assert pm.desc.group_size == group
+    _check_dequant(q, pm)
+    for batch in (1, 2, 5, 16):
+        _check_gemv(q, pm, synth.activations(batch, cols, seed=8200 + batch))
+    if bits <= 5:
+        x40 = synth.activations(40, cols, seed=8300)
+        ws = torch.zeros(xfp.xfp_gemm_workspace_size(pm.desc, 40), dtype=torch.uint8, device="cuda")
+        y = torch.empty((40, rows), dtype=torch.float32, device="cuda")
+        xfp.xfp_gemm(pm.desc, pm.packed, _x_dev(x40), y, ws)
+        torch.cuda.synchronize()
+        assert int(ws[:4].view(torch.int32).item()) == 0
+        ref, absum = xo.gemv(to_oracle(q), x40)
+        assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * absum + 1e-30)
+
+
+def test_group_size_of_a_v2_blob_only_constrains_the_columns():
+    q = synth.random_quantized(0, 64, 512, 4, 0.01, seed=8400, group_size=256)
+    pm = xfp.pack_tensors(q)
+    _check_dequant(q, pm)
+    _check_gemv(q, pm, synth.activations(1, 512, seed=8401))
+
+
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("rows,cols", [(1, 128), (33, 128), (256, 1536), (96, 12288), (2048, 4096)])
 def test_gemv_shapes_and_split_k(mode, rows, cols):
