@@ -44,9 +44,6 @@ namespace xfp {
 namespace {
 
 constexpr int kLaneSlots = 4;   // outlier slots a warp keeps in flight
-#ifndef LANE_CHAINS
-#define LANE_CHAINS 1
-#endif
 
 struct LaneArgs {
     Offsets off;
@@ -57,6 +54,8 @@ struct LaneArgs {
     int* tickets;    // [blocks]
     int rows, cols, RB, SC, rows_ws, ell_slots;
     int y_is_fp16;
+    int tab_bytes;   // shared-memory bytes of the look-up tables
+    int L, GH;       // V2a: library size; groups per super-chunk (2 when the format's groups hold 64 weights)
     // schedule tiers: CTAs [tier_cta[i], tier_cta[i+1]) handle blocks from tier_blk[i] on, each cut into
     // tier_kst[i] slices of tier_spp[i] super-chunks
     int tier_cta[5], tier_blk[4], tier_kst[4], tier_spp[4];
@@ -93,7 +92,7 @@ __device__ __forceinline__ uint32_t xpos(uint32_t k) { return (k & ~12u) | ((k &
 template <int N, bool SGL>
 struct LaneCfg {
     static constexpr int E = 1 << N;
-    static constexpr bool kQuad = N == 2;
+    static constexpr bool kQuad = N == 2 && !SGL;
     static constexpr bool kSingle = SGL;   // one entry per index: N = 6 always, N = 5 on short rows (no 128 KB fill)
     static constexpr int T = kQuad ? 256 : (kSingle ? E : E * E);          // table entries per channel
     static constexpr int kStride = (kQuad || N == 4) ? 256 : 128;            // bytes between entries
@@ -104,7 +103,7 @@ struct LaneCfg {
 template <int N, bool SGL>
 __device__ __forceinline__ void lookup8(uint32_t (&f)[4], const uint32_t* w, int j, const unsigned char* tab,
                                         uint32_t base) {
-    if (N == 2) {
+    if (N == 2 && !SGL) {
         // bytes 2j and 2j+1 of the stream; base = lane * 8
         const uint32_t a0 = __byte_perm(w[(2 * j) >> 2], base, 0x5504u | ((uint32_t)((2 * j) & 3) << 4));
         const uint32_t a1 = __byte_perm(w[(2 * j + 1) >> 2], base, 0x5504u | ((uint32_t)((2 * j + 1) & 3) << 4));
@@ -135,7 +134,12 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
     return (128 * (v + 1) - 1) / (8 * N);
 }
 
-template <int N, int W, int MINB, bool SGL>
+// MODE 0: V2 (the channel's own codebook, tables private to the lane).  MODE 1: V2a -- the whole library replicated
+// once per bank (word (id * 2^N + q) * 32 + lane holds lib[id][q]), the table base of a lane follows the library id
+// of its channel's current group, the fragment accumulates sum lib * x of ONE group, and after the group's steps the
+// sum moves to the lane that owns the channel and is folded into its accumulator with the group's scale and
+// mid-point:  acc += scale * G + mid * X_g,  X_g = sum of x over the group ("V2a: Shared Codebook Library").
+template <int N, int W, int MINB, bool SGL, int MODE>
 __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs a) {
     using C = LaneCfg<N, SGL>;
     constexpr int E = C::E;
@@ -150,8 +154,9 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     const Blob b = blob_at(a.packed, a.off);
     const int K = a.SC * kSuper;
     unsigned char* tab = smem;
-    unsigned char* xs = smem + C::kTabBytes;
-    float* red = (float*)(xs + (size_t)K * 2);
+    unsigned char* xs = smem + a.tab_bytes;
+    float* red = (float*)(xs + (size_t)K * 2);     // [W][32]
+    float* xg = red + W * 32;                      // V2a: [SC][2] sums of x over the halves of every super-chunk
 
     // ---- this CTA's block and K slice
     int blk, slice, nslices, sc0, nsc;
@@ -180,6 +185,15 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
         }
     }
+    // V2a: library id and (scale, mid) of the lane's channel for the two halves of the super-chunk ([1] repeats [0]
+    // unless the groups hold 64 weights), current and next
+    const int GH = MODE == 1 ? a.GH : 1;
+    const size_t m0 = ((size_t)(blk * a.SC + sc0) * GH) * 32 + lane;
+    uint32_t gid_c[2] = {0u, 0u}, gsm_c[2] = {0u, 0u}, gid_n[2] = {0u, 0u}, gsm_n[2] = {0u, 0u};
+    if (MODE == 1 && warp < nsc) {
+        gid_c[0] = b.gid[m0 + (size_t)warp * GH * 32]; gsm_c[0] = b.gsm[m0 + (size_t)warp * GH * 32];
+        gid_c[1] = b.gid[m0 + ((size_t)warp * GH + GH - 1) * 32]; gsm_c[1] = b.gsm[m0 + ((size_t)warp * GH + GH - 1) * 32];
+    }
     const int ell_slots = a.ell_slots;
     const uint32_t* slab = b.ell + (size_t)blk * (ell_slots + 1) * 32 + lane;
     uint32_t olen = ell_slots ? __ldg(slab) : 0u;
@@ -190,7 +204,9 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         oe[q] = j < ell_slots ? __ldg(slab + (size_t)(1 + j) * 32) : 0u;   // every slot below the capacity is readable
     }
     // ---- tables: warp w fills entries [w T / W, (w+1) T / W) of every lane's channel
-    {
+    if (MODE == 1) {
+        for (int e = warp; e < a.L * E; e += W) *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+    } else {
         const uint16_t* cb = b.cb + (size_t)(blk * kRowsPerBlock + lane) * E;
         if (C::kQuad) {
             // entry t = (cb[t & 3], cb[t >> 2 & 3], cb[t >> 4 & 3], cb[t >> 6]) as 8 bytes at t * 256 + lane * 8
@@ -249,11 +265,25 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     lstamp(a, 1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     lstamp(a, 2);
-    for (int t = threadIdx.x; t < K / 8; t += kThreads) {
-        const uint4 v = __ldg((const uint4*)(a.x) + t);
-        // k = 8t .. 8t+7: its two blocks of four go to positions xpos(8t) and xpos(8t + 4)
-        *(uint2*)(xs + xpos(8u * t) * 2) = make_uint2(v.x, v.y);
-        *(uint2*)(xs + xpos(8u * t + 4u) * 2) = make_uint2(v.z, v.w);
+    for (int t = threadIdx.x; t < ((K / 8 + 31) & ~31); t += kThreads) {   // whole warps: the sums below shuffle
+        const bool in = t < K / 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (in) {
+            v = __ldg((const uint4*)(a.x) + t);
+            // k = 8t .. 8t+7: its two blocks of four go to positions xpos(8t) and xpos(8t + 4)
+            *(uint2*)(xs + xpos(8u * t) * 2) = make_uint2(v.x, v.y);
+            *(uint2*)(xs + xpos(8u * t + 4u) * 2) = make_uint2(v.z, v.w);
+        }
+        if (MODE == 1) {
+            // 8 consecutive threads hold 64 consecutive k: sums of x over the halves of the super-chunks, in a fixed order
+            const float2 p0 = __half22float2(*(const __half2*)&v.x), p1 = __half22float2(*(const __half2*)&v.y);
+            const float2 p2 = __half22float2(*(const __half2*)&v.z), p3 = __half22float2(*(const __half2*)&v.w);
+            float sx = ((p0.x + p0.y) + (p1.x + p1.y)) + ((p2.x + p2.y) + (p3.x + p3.y));
+            sx += __shfl_xor_sync(0xffffffffu, sx, 1);
+            sx += __shfl_xor_sync(0xffffffffu, sx, 2);
+            sx += __shfl_xor_sync(0xffffffffu, sx, 4);
+            if (in && (t & 7) == 0) xg[t >> 3] = sx;
+        }
     }
     __syncthreads();   // tables and x visible
     lstamp(a, 3);
@@ -265,10 +295,9 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     const unsigned char* xq = xs + (size_t)sc0 * (kSuper * 2) + ((g == t4 + 4) ? 16 : 0);
 
     float c[4] = {0.f, 0.f, 0.f, 0.f};
-#if LANE_CHAINS == 2
-    float c2[4] = {0.f, 0.f, 0.f, 0.f};
-#endif
-    float oacc = 0.f;
+    float oacc = 0.f;   // outliers of the lane's channel; in V2a also the channel's folded group sums
+    // V2a: where the two halves of this lane's group sum land in the fragment (see the end of the kernel)
+    const int src_a = (lane & ~3) | (t4 >> 1);
     // the rows' slot counts have arrived: outlier rounds of this warp
     int width = (int)olen;
 #pragma unroll
@@ -306,11 +335,31 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         const unsigned char* xp = xq + (size_t)s * (kSuper * 2);
         uint32_t fa[4], fb[4];
         uint4 xr = make_uint4(0u, 0u, 0u, 0u);
-        lookup8<N, SGL>(fa, w, 0, tab, base);
+        uint32_t vbase = base;
+        if (MODE == 1) {
+            vbase = base + gid_c[0] * (uint32_t)(E * 128);
+            if (has_next) {   // metadata of the next super-chunk travels during this one
+                const size_t mn = m0 + (size_t)(s + W) * GH * 32;
+                gid_n[0] = b.gid[mn]; gsm_n[0] = b.gsm[mn];
+                gid_n[1] = b.gid[mn + (size_t)(GH - 1) * 32]; gsm_n[1] = b.gsm[mn + (size_t)(GH - 1) * 32];
+            }
+        }
+        // V2a: the group's sum leaves the fragment (two halves of the channel's sum sit in two other lanes of the
+        // quad) and is folded with the group's scale and mid-point
+        auto fold = [&](int h) {
+            const float a0 = __shfl_sync(0xffffffffu, c[0], src_a), a1 = __shfl_sync(0xffffffffu, c[1], src_a);
+            const float b2 = __shfl_sync(0xffffffffu, c[2], src_a + 2), b3 = __shfl_sync(0xffffffffu, c[3], src_a + 2);
+            const float G = (t4 & 1) ? a1 + b3 : a0 + b2;
+            const float scale = h2f((uint16_t)(gsm_c[h] & 0xffffu)), mid = h2f((uint16_t)(gsm_c[h] >> 16));
+            const float X = GH == 2 ? xg[(sc0 + s) * 2 + h] : xg[(sc0 + s) * 2] + xg[(sc0 + s) * 2 + 1];
+            oacc = fmaf(scale, G, fmaf(mid, X, oacc));
+            c[0] = c[1] = c[2] = c[3] = 0.f;
+        };
+        lookup8<N, SGL>(fa, w, 0, tab, vbase);
 #pragma unroll
         for (int j = 0; j < kSuper / 8; j += 2) {
             ld_x16_if(xr, xp + j * 16, dq);               // steps j and j + 1
-            lookup8<N, SGL>(fb, w, j + 1, tab, base);
+            lookup8<N, SGL>(fb, w, j + 1, tab, vbase);
 #pragma unroll
             for (int v = 0; v < N; ++v)
                 if ((last_step_of_vector<N>(v) == j || last_step_of_vector<N>(v) == j + 1) && has_next) {
@@ -318,18 +367,16 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
                     w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
                 }
             mma16816(c, fa[0], fa[1], fa[2], fa[3], xr.x, xr.y);
-            if (j + 2 < kSuper / 8) lookup8<N, SGL>(fa, w, j + 2, tab, base);
-#if LANE_CHAINS == 2
-            mma16816(c2, fb[0], fb[1], fb[2], fb[3], xr.z, xr.w);
-#else
+            if (MODE == 1 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)(E * 128);   // second half's library entry
+            if (j + 2 < kSuper / 8) lookup8<N, SGL>(fa, w, j + 2, tab, vbase);
             mma16816(c, fb[0], fb[1], fb[2], fb[3], xr.z, xr.w);
-#endif
+            if (MODE == 1 && j + 2 == kSuper / 16 && GH == 2) fold(0);   // the first group of 64 weights is complete
+        }
+        if (MODE == 1) {
+            fold(1);
+            gid_c[0] = gid_n[0]; gid_c[1] = gid_n[1]; gsm_c[0] = gsm_n[0]; gsm_c[1] = gsm_n[1];
         }
     }
-#if LANE_CHAINS == 2
-#pragma unroll
-    for (int i = 0; i < 4; ++i) c[i] += c2[i];
-#endif
     while (oround < nrounds) {   // more outlier rounds than super-chunks
         consume_slots();
         if (++oround < nrounds) fetch_slots(oround);
@@ -347,7 +394,9 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     lstamp(a, 4);
     // ---- the two halves of a channel meet: lane (g, t < 2) holds D[g][2t], D[g][2t+1]; lane (g, t + 2) holds
     //      D[g+8][2t+4], D[g+8][2t+5]; then channel order through shared memory
-    {
+    if (MODE == 1) {
+        red[warp * 32 + lane] = oacc;   // every lane already owns its channel's sum
+    } else {
         const float h2 = __shfl_xor_sync(0xffffffffu, c[2], 2), h3 = __shfl_xor_sync(0xffffffffu, c[3], 2);
         float* r = red + (size_t)warp * 32;
         if (t4 < 2) *(float2*)(r + 4 * g + 2 * t4) = make_float2(c[0] + h2, c[1] + h3);
@@ -460,15 +509,17 @@ LaneSchedule lane_schedule(const Layout& l, int per_sm, bool tiers) {
 // ---- launch configurations: warps per CTA, CTAs per SM (64 registers per thread at 16 x 2), single-entry tables
 struct LaneConfig { int W, per_sm; bool sgl; bool off = false; bool tiers = true; };
 
-size_t lane_tab_bytes(int bits, bool sgl) {
+size_t lane_tab_bytes(const Layout& l, bool sgl) {
+    const int bits = l.bits;
     const size_t E = (size_t)1 << bits;
+    if (l.mode) return (size_t)l.L * E * 128;   // the library, one copy per bank
     if (bits == 2) return 256 * 256;
     if (sgl) return E * 128;
     return E * E * (bits == 4 ? 256 : 128);
 }
 
 size_t lane_smem_bytes(const Layout& l, const LaneConfig& c) {
-    return lane_tab_bytes(l.bits, c.sgl) + (size_t)l.cols * 2 + (size_t)c.W * 32 * 4;
+    return lane_tab_bytes(l, c.sgl) + (size_t)l.cols * 2 + (size_t)c.W * 32 * 4 + (l.mode ? (size_t)l.SC * 8 : 0);
 }
 
 LaneConfig lane_config(const Layout& l) {
@@ -477,7 +528,7 @@ LaneConfig lane_config(const Layout& l) {
         int w = 16, p = 1, g = 0;
         sscanf(e, "%d,%d,%d", &w, &p, &g);
         if (w == 0) return LaneConfig{16, 1, false, true};
-        return LaneConfig{w, p > 2 ? 2 : p, l.bits == 6 || (l.bits == 5 && g), false, p <= 2};
+        return LaneConfig{w, p > 2 ? 2 : p, l.mode == 1 || l.bits == 6 || (l.bits == 5 && g), false, p <= 2};
     }
 #endif
     // Measured on B200 over 4096 x 4096 .. 28672 x 8192 at every bit width (microseconds per call, graph replay):
@@ -488,6 +539,13 @@ LaneConfig lane_config(const Layout& l) {
     //  * N = 5 beyond one round: one entry per index instead of the 128 KB pair table, whose fill per 32 channels
     //    costs as much as 2048 weights of look-ups and cannot overlap anything with one CTA per SM
     const int sms = sched_sms();
+    if (l.mode) {
+        // V2a: one look-up per weight in the per-bank library.  Up to 64 KB of tables (L * 2^N <= 512) two CTAs fit.
+        const bool two = lane_tab_bytes(l, true) <= 64 * 1024 && l.RB > sms;
+        LaneConfig c{two ? 8 : 16, two ? 2 : 1, true};
+        c.tiers = l.RB > 4 * sms || !two;
+        return c;
+    }
     if (l.RB <= sms) return LaneConfig{16, 1, l.bits == 6};
     const bool big = l.RB > 4 * sms;
     LaneConfig c{(!big && (l.bits == 3 || l.bits == 4)) ? 16 : 8, 2, l.bits >= 5};
@@ -496,12 +554,12 @@ LaneConfig lane_config(const Layout& l) {
     return c;
 }
 
-template <int N, int W, int MINB, bool SGL>
+template <int N, int W, int MINB, bool SGL, int MODE>
 cudaError_t launch_lane(const LaneArgs& a, int grid, size_t smem, cudaStream_t s) {
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lane_kernel<N, W, MINB, SGL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_lane_kernel<N, W, MINB, SGL, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              MINB == 1 ? 224 * 1024 : 110 * 1024);
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
@@ -516,22 +574,23 @@ cudaError_t launch_lane(const LaneArgs& a, int grid, size_t smem, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_lane_kernel<N, W, MINB, SGL>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_lane_kernel<N, W, MINB, SGL, MODE>, a);
 }
 
-template <int N, bool SGL>
+template <int N, bool SGL, int MODE>
 cudaError_t launch_lane_cfg(const LaneConfig& c, const LaneArgs& a, int grid, size_t smem, cudaStream_t s) {
-    if (c.W == 8) return launch_lane<N, 8, 2, SGL>(a, grid, smem, s);
-    if (c.per_sm >= 2) return launch_lane<N, 16, 2, SGL>(a, grid, smem, s);
-    return launch_lane<N, 16, 1, SGL>(a, grid, smem, s);
+    if (c.W == 8) return launch_lane<N, 8, 2, SGL, MODE>(a, grid, smem, s);
+    if (c.per_sm >= 2) return launch_lane<N, 16, 2, SGL, MODE>(a, grid, smem, s);
+    return launch_lane<N, 16, 1, SGL, MODE>(a, grid, smem, s);
 }
 
 }  // namespace
 
-// single V2 blob, batch 1, fp16 x, fp32 / fp16 y; x short enough to stage beside the tables
+// a single blob, batch 1, fp16 x, fp32 / fp16 y, no fused store; x short enough to stage beside the tables
 bool lane_supported(const Layout& l, const GemvCall& c) {
-    if (l.mode != 0 || c.batch != 1 || c.n != 1 || c.packed_list || c.x_bf16 || c.y_is_fp16 == 2) return false;
+    if (c.batch != 1 || c.n != 1 || c.packed_list || c.x_bf16 || c.y_is_fp16 == 2 || c.epilogue != 0) return false;
     if (l.bits < 2 || l.bits > 6) return false;
+    if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) return false;   // V2a: the per-bank library must fit (N = 6 does not)
     const LaneConfig cfg = lane_config(l);
     if (cfg.off) return false;
     return lane_smem_bytes(l, cfg) <= (cfg.per_sm == 1 ? 220u : 110u) * 1024u;
@@ -546,6 +605,8 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
     a.rows_ws = l.RB * 32;
     a.y_is_fp16 = c.y_is_fp16;
+    a.tab_bytes = (int)lane_tab_bytes(l, cfg.sgl);
+    a.L = l.L; a.GH = l.GH;
     for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
     for (int i = 0; i < 4; ++i) { a.tier_blk[i] = sch.tier_blk[i]; a.tier_kst[i] = sch.tier_kst[i]; a.tier_spp[i] = sch.tier_spp[i]; }
     a.tickets = (int*)c.workspace;
@@ -555,13 +616,21 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
     if (g_lane_trace && g_lane_trace_idx < g_lane_trace_calls) a.trace = g_lane_trace + (g_lane_trace_idx++) * 1024 * 8;
 #endif
     const size_t smem = lane_smem_bytes(l, cfg);
+    if (l.mode) {
+        switch (l.bits) {
+            case 2: return launch_lane_cfg<2, true, 1>(cfg, a, sch.grid, smem, s);
+            case 3: return launch_lane_cfg<3, true, 1>(cfg, a, sch.grid, smem, s);
+            case 4: return launch_lane_cfg<4, true, 1>(cfg, a, sch.grid, smem, s);
+            default: return launch_lane_cfg<5, true, 1>(cfg, a, sch.grid, smem, s);
+        }
+    }
     switch (l.bits) {
-        case 2: return launch_lane_cfg<2, false>(cfg, a, sch.grid, smem, s);
-        case 3: return launch_lane_cfg<3, false>(cfg, a, sch.grid, smem, s);
-        case 4: return launch_lane_cfg<4, false>(cfg, a, sch.grid, smem, s);
-        case 5: return cfg.sgl ? launch_lane_cfg<5, true>(cfg, a, sch.grid, smem, s)
-                               : launch_lane_cfg<5, false>(cfg, a, sch.grid, smem, s);
-        default: return launch_lane_cfg<6, true>(cfg, a, sch.grid, smem, s);
+        case 2: return launch_lane_cfg<2, false, 0>(cfg, a, sch.grid, smem, s);
+        case 3: return launch_lane_cfg<3, false, 0>(cfg, a, sch.grid, smem, s);
+        case 4: return launch_lane_cfg<4, false, 0>(cfg, a, sch.grid, smem, s);
+        case 5: return cfg.sgl ? launch_lane_cfg<5, true, 0>(cfg, a, sch.grid, smem, s)
+                               : launch_lane_cfg<5, false, 0>(cfg, a, sch.grid, smem, s);
+        default: return launch_lane_cfg<6, true, 0>(cfg, a, sch.grid, smem, s);
     }
 }
 
