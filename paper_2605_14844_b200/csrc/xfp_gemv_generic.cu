@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
             tab[t] = h2f(b.cb[(size_t)(rb * kRowsPerBlock + l) * E + e]);
         }
     } else {
-        for (int t = threadIdx.x; t < tab_floats; t += kGenericThreads) tab[t] = h2f(b.cb[a.rep == 32 ? (t >> 5) : t]);
+        for (int t = threadIdx.x; t < tab_floats; t += kGenericThreads) tab[t] = h2f(b.cb[t / a.rep]);
     }
     // ---- x may come from the previous kernel: stage this split's slice as fp32
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(kGenericThreads) gemv_generic_kernel(const Gen
                 const uint32_t id = gid_c[h];
                 const uint32_t sm = gsm_c[h];
                 const float scale = h2f((uint16_t)(sm & 0xffffu)), mid = h2f((uint16_t)(sm >> 16));
-                const float* t = tab + (size_t)id * E * a.rep + (a.rep == 32 ? lane : 0);
+                const float* t = tab + (size_t)id * E * a.rep + (lane & (a.rep - 1));
                 float gs[BT];
 #pragma unroll
                 for (int bb = 0; bb < BT; ++bb) gs[bb] = 0.f;

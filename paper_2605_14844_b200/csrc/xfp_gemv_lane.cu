@@ -544,6 +544,9 @@ LaneConfig lane_config(const Layout& l) {
         const bool two = lane_tab_bytes(l, true) <= 64 * 1024 && l.RB > sms;
         LaneConfig c{two ? 8 : 16, two ? 2 : 1, true};
         c.tiers = l.RB > 4 * sms || !two;
+        // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
+        // per lane (xfp_gemv_v2a.cu) measured faster
+        c.off = !two && l.RB > sms && l.RB <= 4 * sms;
         return c;
     }
     if (l.RB <= sms) return LaneConfig{16, 1, l.bits == 6};
