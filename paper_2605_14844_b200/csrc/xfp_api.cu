@@ -76,6 +76,12 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     }
     if (lane_supported(l, cc))
         e = launch_gemv_lane(l, cc, (cudaStream_t)stream);
+    else if (!c.packed_list && !c.x_bf16 && batch_prefers_gemm(l, c.batch)) {
+        // many rows of x, few outliers: one decode for all rows on the tensor cores (y = x W^T with W the matrix
+        // xfp_dequant writes; inside the GEMV's bound)
+        GemmCall g{c.packed, c.x, c.y, c.batch, c.y_is_fp16, c.workspace, need};
+        e = launch_gemm_tc(l, g, (cudaStream_t)stream);
+    }
     else if (pair_supported(l, c.batch, c.n))
         e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && batch_supported(l, c.batch))

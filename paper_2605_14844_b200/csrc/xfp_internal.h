@@ -113,10 +113,22 @@ cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s);
 size_t gemm_x_scratch_bytes(const Layout& l, int M);
 cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaStream_t s);
 
+// Batches from this size on run on the tensor-core kernel (xfp_gemm_tc.cu) when the blob is sparse in outliers:
+// the batched GEMV kernels decode once per 8 rows of x and grow by ~9 us per row at 28672 x 8192, the tcgen05
+// kernel decodes once for up to 128 rows (measured at 28672 x 8192, 0.3 % outliers, 16 rows: 144 against 185 us
+// for V2, 159 against 296 us for V2a; at 2 % outliers its per-lane outlier walk loses, 282 against 265 us).
+// Only matrices whose tensor-core plan fits the GEMV workspace take that route (large ones: no K slices, a few
+// counters); the workspace size a caller was told never grows for it.
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);
     return w > p ? w : p;
+}
+
+inline bool batch_prefers_gemm(const Layout& l, int batch) {
+    if (batch < (l.mode ? 9 : 13) || !gemm_tc_supported(l, batch)) return false;
+    if (gemm_workspace_bytes(l, batch) > workspace_bytes_for(l)) return false;
+    return l.nnz * 100 <= (long long)l.rows * l.cols;   // at most 1 % outliers
 }
 
 }  // namespace xfp
