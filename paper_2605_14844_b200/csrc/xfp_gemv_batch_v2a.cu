@@ -420,7 +420,7 @@ cudaError_t launch_gemv_batch_v2a(const Layout& l, const GemvCall& c, cudaStream
             a.kst = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
             if (a.kst <= 1) { a.kst = 1; a.n_full = blocks; rem = 0; }
             a.tickets = (int*)c.workspace;
-            a.partial = (float*)((char*)c.workspace + align256((size_t)blocks * 4));   // layout of v2a_workspace_bytes
+            a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));   // layout of v2a_workspace_bytes
             const size_t smem = batch_v2a_smem_bytes(l, nbt);
             dim3 grid((unsigned)(a.n_full + rem * a.kst), 1, 1);
             cudaError_t e = cudaErrorInvalidValue;

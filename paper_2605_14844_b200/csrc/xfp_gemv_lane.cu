@@ -50,8 +50,13 @@ struct LaneArgs {
     const void* packed;
     const uint16_t* x;
     void* y;
+    // several blobs of one shape in one launch: device pointer lists; the row-blocks of all blobs are numbered
+    // through (RB of them per blob) and scheduled as one matrix
+    const void* const* packed_list;
+    const uint16_t* const* x_list;
+    void* const* y_list;
     float* partial;  // [slice][rows_ws]
-    int* tickets;    // [blocks]
+    int* tickets;    // [blocks of the launch]
     int rows, cols, RB, SC, rows_ws, ell_slots;
     int y_is_fp16;
     int tab_bytes;   // shared-memory bytes of the look-up tables
@@ -151,7 +156,6 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
     lstamp(a, 0);
-    const Blob b = blob_at(a.packed, a.off);
     const int K = a.SC * kSuper;
     unsigned char* tab = smem;
     unsigned char* xs = smem + a.tab_bytes;
@@ -173,6 +177,21 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         nsc = max(0, min(a.SC, sc0 + a.tier_spp[tier]) - sc0);
     }
     const int gw = slice * W + warp, ostride = nslices * W;
+    // the blob of this block: `gblk` numbers the row-blocks of the whole launch, `blk` those of its blob
+    const int gblk = blk;
+    const void* packed = a.packed;
+    const uint16_t* xsrc = a.x;
+    void* ydst = a.y;
+    int ell_slots = a.ell_slots;
+    if (a.packed_list) {
+        const int prob = blk / a.RB;
+        blk -= prob * a.RB;
+        packed = a.packed_list[prob];
+        xsrc = a.x_list[prob];
+        ydst = a.y_list[prob];
+        ell_slots = __ldg((const int*)((const char*)packed + a.off.hdr));   // the blobs' outlier counts differ
+    }
+    const Blob b = blob_at(packed, a.off);
 
     // ---- loads that do not depend on earlier kernels: first index vectors, outlier slab, codebook
     uint32_t w[4 * N + 1];
@@ -194,8 +213,9 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         gid_c[0] = b.gid[m0 + (size_t)warp * GH * 32]; gsm_c[0] = b.gsm[m0 + (size_t)warp * GH * 32];
         gid_c[1] = b.gid[m0 + ((size_t)warp * GH + GH - 1) * 32]; gsm_c[1] = b.gsm[m0 + ((size_t)warp * GH + GH - 1) * 32];
     }
-    const int ell_slots = a.ell_slots;
-    const uint32_t* slab = b.ell + (size_t)blk * (ell_slots + 1) * 32 + lane;
+    const uint32_t* ell = a.packed_list
+        ? (const uint32_t*)((const char*)packed + *(const long long*)((const char*)packed + a.off.hdr + 8)) : b.ell;
+    const uint32_t* slab = ell + (size_t)blk * (ell_slots + 1) * 32 + lane;
     uint32_t olen = ell_slots ? __ldg(slab) : 0u;
     uint32_t oe[kLaneSlots];
 #pragma unroll
@@ -269,7 +289,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         const bool in = t < K / 8;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (in) {
-            v = __ldg((const uint4*)(a.x) + t);
+            v = __ldg((const uint4*)(xsrc) + t);
             // k = 8t .. 8t+7: its two blocks of four go to positions xpos(8t) and xpos(8t + 4)
             *(uint2*)(xs + xpos(8u * t) * 2) = make_uint2(v.x, v.y);
             *(uint2*)(xs + xpos(8u * t + 4u) * 2) = make_uint2(v.z, v.w);
@@ -408,7 +428,8 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     // ---- fixed-order sum over the warps, then store or combine the block's slices
     const int t = threadIdx.x;
     const bool active = t < 32;
-    const int row = blk * 32 + t;
+    const int row = blk * 32 + t;       // channel inside its blob (y index)
+    const int wrow = gblk * 32 + t;     // channel inside the launch (workspace index)
     float total = 0.f;
     if (active) {
 #pragma unroll
@@ -417,22 +438,22 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     bool writer = true;
     if (nslices > 1) {
         __shared__ int s_last;
-        if (active) a.partial[(size_t)slice * a.rows_ws + row] = total;
+        if (active) a.partial[(size_t)slice * a.rows_ws + wrow] = total;
         __threadfence();
         __syncthreads();
-        if (t == 0) s_last = (atomicAdd(a.tickets + blk, 1) == nslices - 1);
+        if (t == 0) s_last = (atomicAdd(a.tickets + gblk, 1) == nslices - 1);
         __syncthreads();
         writer = s_last != 0;
         if (writer) {
             __threadfence();
             if (active) {
                 total = 0.f;
-                for (int k2 = 0; k2 < nslices; ++k2) total += __ldcg(a.partial + (size_t)k2 * a.rows_ws + row);
+                for (int k2 = 0; k2 < nslices; ++k2) total += __ldcg(a.partial + (size_t)k2 * a.rows_ws + wrow);
             }
-            if (t == 0) a.tickets[blk] = 0;
+            if (t == 0) a.tickets[gblk] = 0;
         }
     }
-    if (writer && active && row < a.rows) store_y<false>(a.y, (size_t)row, total, a.y_is_fp16);
+    if (writer && active && row < a.rows) store_y<false>(ydst, (size_t)row, total, a.y_is_fp16);
     lstamp(a, 5);
 }
 
@@ -455,10 +476,9 @@ int pow2_floor_(int v) {
 // Whole-K blocks fill whole rounds of CTA slots; the blocks of the last partial round are cut along K in tiers of
 // finer slices (the hardware dispatches CTAs in launch order, so the tiers pack the slots largest-first).  A matrix
 // with no more blocks than SMs runs one unsplit block per SM and leaves the other half of every SM to the next call.
-LaneSchedule lane_schedule(const Layout& l, int per_sm, bool tiers) {
+LaneSchedule lane_schedule(const Layout& l, int blocks, int per_sm, bool tiers) {
     LaneSchedule sc{};
     const int sms = sched_sms();
-    const int blocks = l.RB;
     const int S = sms * per_sm;
     const int kmax = l.SC / 4 > 1 ? pow2_floor_(l.SC / 4) : 1;   // keep K slices of at least 512 weights
     int nb[4] = {0, 0, 0, 0}, kk[4] = {1, 1, 1, 1};
@@ -522,7 +542,9 @@ size_t lane_smem_bytes(const Layout& l, const LaneConfig& c) {
     return lane_tab_bytes(l, c.sgl) + (size_t)l.cols * 2 + (size_t)c.W * 32 * 4 + (l.mode ? (size_t)l.SC * 8 : 0);
 }
 
-LaneConfig lane_config(const Layout& l) {
+// `RBn`: row-blocks of the launch (all blobs)
+LaneConfig lane_config(const Layout& l, int n = 1) {
+    const long long RB = (long long)l.RB * n;
 #ifdef LANE_TUNE
     if (const char* e = getenv("XFP_LANE_CFG")) {   // tuning build: "W,per_sm,sgl"
         int w = 16, p = 1, g = 0;
@@ -541,16 +563,16 @@ LaneConfig lane_config(const Layout& l) {
     const int sms = sched_sms();
     if (l.mode) {
         // V2a: one look-up per weight in the per-bank library.  Up to 64 KB of tables (L * 2^N <= 512) two CTAs fit.
-        const bool two = lane_tab_bytes(l, true) <= 64 * 1024 && l.RB > sms;
+        const bool two = lane_tab_bytes(l, true) <= 64 * 1024 && RB > sms;
         LaneConfig c{two ? 8 : 16, two ? 2 : 1, true};
-        c.tiers = l.RB > 4 * sms || !two;
+        c.tiers = RB > 4 * sms || !two;
         // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
         // per lane (xfp_gemv_v2a.cu) measured faster
-        c.off = !two && l.RB > sms && l.RB <= 4 * sms;
+        c.off = !two && RB > sms && RB <= 4 * sms;
         return c;
     }
-    if (l.RB <= sms) return LaneConfig{16, 1, l.bits == 6};
-    const bool big = l.RB > 4 * sms;
+    if (RB <= sms) return LaneConfig{16, 1, l.bits == 6};
+    const bool big = RB > 4 * sms;
     LaneConfig c{(!big && (l.bits == 3 || l.bits == 4)) ? 16 : 8, 2, l.bits >= 5};
     c.off = big && l.bits <= 3;   // the two-channels-per-lane kernel is ahead there
     c.tiers = big;
@@ -591,29 +613,31 @@ cudaError_t launch_lane_cfg(const LaneConfig& c, const LaneArgs& a, int grid, si
 
 // a single blob, batch 1, fp16 x, fp32 / fp16 y, no fused store; x short enough to stage beside the tables
 bool lane_supported(const Layout& l, const GemvCall& c) {
-    if (c.batch != 1 || c.n != 1 || c.packed_list || c.x_bf16 || c.y_is_fp16 == 2 || c.epilogue != 0) return false;
+    if (c.batch != 1 || c.n < 1 || c.x_bf16 || c.y_is_fp16 == 2 || c.epilogue != 0) return false;
+    if ((c.n > 1) != (c.packed_list != nullptr)) return false;
     if (l.bits < 2 || l.bits > 6) return false;
     if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) return false;   // V2a: the per-bank library must fit (N = 6 does not)
-    const LaneConfig cfg = lane_config(l);
+    const LaneConfig cfg = lane_config(l, c.n);
     if (cfg.off) return false;
     return lane_smem_bytes(l, cfg) <= (cfg.per_sm == 1 ? 220u : 110u) * 1024u;
 }
 
 cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s) {
-    const LaneConfig cfg = lane_config(l);
-    const LaneSchedule sch = lane_schedule(l, cfg.per_sm, cfg.tiers);
+    const LaneConfig cfg = lane_config(l, c.n);
+    const LaneSchedule sch = lane_schedule(l, l.RB * c.n, cfg.per_sm, cfg.tiers);
     LaneArgs a{};
     a.off = offsets_of(l);
     a.packed = c.packed; a.x = c.x; a.y = c.y;
+    a.packed_list = c.packed_list; a.x_list = c.x_list; a.y_list = c.y_list;
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
-    a.rows_ws = l.RB * 32;
+    a.rows_ws = l.RB * c.n * 32;
     a.y_is_fp16 = c.y_is_fp16;
     a.tab_bytes = (int)lane_tab_bytes(l, cfg.sgl);
     a.L = l.L; a.GH = l.GH;
     for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
     for (int i = 0; i < 4; ++i) { a.tier_blk[i] = sch.tier_blk[i]; a.tier_kst[i] = sch.tier_kst[i]; a.tier_spp[i] = sch.tier_spp[i]; }
     a.tickets = (int*)c.workspace;
-    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
+    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4 * c.n));
 #ifdef XFP_TRACE
     a.trace = nullptr;
     if (g_lane_trace && g_lane_trace_idx < g_lane_trace_calls) a.trace = g_lane_trace + (g_lane_trace_idx++) * 1024 * 8;

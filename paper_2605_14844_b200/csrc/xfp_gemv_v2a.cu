@@ -556,7 +556,8 @@ bool v2a_supported(const Layout& l, int batch) {
 
 size_t v2a_workspace_bytes(const Layout& l) {
     const int blocks = (l.RB + 1) / 2;
-    return align256((size_t)blocks * 4) + align256((size_t)64 * 2 * (size_t)blocks * kARows * 4);
+    // counters first, in the region every GEMV kernel of the library keeps zero-filled: one int per row-block
+    return align256((size_t)l.RB * 4) + align256((size_t)64 * 2 * (size_t)blocks * kARows * 4);
 }
 
 template <int N, int NB, int W, bool PAIR, bool FEAT>
@@ -644,7 +645,7 @@ cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s) 
     a.n_full = a.blocks - rem;
     const int n_b = rem - a.n_a;
     a.tickets = (int*)c.workspace;
-    a.partial = (float*)((char*)c.workspace + align256((size_t)a.blocks * 4 * c.n));
+    a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4 * c.n));   // behind the common counter region
     a.items_x = a.n_full + a.n_a * a.kst + n_b * a.kst_b;
     a.n = c.n;
     a.epi = c.epilogue; a.epi_w = c.epi_weights;

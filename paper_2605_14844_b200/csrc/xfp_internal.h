@@ -117,8 +117,9 @@ cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaS
 // the batched GEMV kernels decode once per 8 rows of x and grow by ~9 us per row at 28672 x 8192, the tcgen05
 // kernel decodes once for up to 128 rows (measured at 28672 x 8192, 0.3 % outliers, 16 rows: 144 against 185 us
 // for V2, 159 against 296 us for V2a; at 2 % outliers its per-lane outlier walk loses, 282 against 265 us).
-// Only matrices whose tensor-core plan fits the GEMV workspace take that route (large ones: no K slices, a few
-// counters); the workspace size a caller was told never grows for it.
+// Layout of a GEMV workspace, shared by every kernel that may be given it: counters (split-K tickets, one int per
+// row-block and blob at most) in [0, align256(4 * RB * n)), zero-filled before first use and left zero-filled by every
+// call; partial sums behind it, written before they are read.
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);
@@ -127,7 +128,10 @@ inline size_t workspace_bytes_for(const Layout& l) {
 
 inline bool batch_prefers_gemm(const Layout& l, int batch) {
     if (batch < (l.mode ? 9 : 13) || !gemm_tc_supported(l, batch)) return false;
-    if (gemm_workspace_bytes(l, batch) > workspace_bytes_for(l)) return false;
+    // no K slices: the plan then uses a few counters at the start of the workspace and nothing else, inside the
+    // region that every GEMV kernel leaves zero-filled
+    if (gemm_workspace_bytes(l, batch) > gemm_ctrl_bytes(l, batch) || gemm_ctrl_bytes(l, batch) > align256((size_t)l.RB * 4))
+        return false;
     return l.nnz * 100 <= (long long)l.rows * l.cols;   // at most 1 % outliers
 }
 

@@ -76,6 +76,29 @@ def test_gemv_within_bound_small(mode, bits, batch):
     _check_gemv(q, pm, x16, y_fp16=True)
 
 
+@pytest.mark.parametrize("mode,bits,rows,cols", [(0, 4, 2048, 4096), (1, 3, 2048, 1536), (1, 4, 640, 8192), (0, 6, 96, 12288)])
+def test_one_workspace_serves_every_kernel_in_turn(mode, bits, rows, cols):
+    """The header's promise: one workspace serves any batch and every GEMV entry point of a shape, one call after the
+    other.  Every kernel must leave the counter region zero-filled and must not keep data where another kernel
+    keeps counters: a call sequence over ONE workspace (batch 1, 16, 2, 5, bf16, batch 1 again) gives bit for bit what
+    the same calls give with a fresh workspace each."""
+    q = synth.random_quantized(mode, rows, cols, bits, 0.004, seed=8500 + bits)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    shared = pm.workspace
+    seq = [(1, torch.float16), (16, torch.float16), (2, torch.float16), (5, torch.float16), (3, torch.bfloat16),
+           (1, torch.float16), (13, torch.float16), (1, torch.float16)]
+    for i, (batch, xdt) in enumerate(seq):
+        x = _x_dev(synth.activations(batch, cols, seed=8600 + i)).to(xdt)
+        y_shared = torch.empty((batch, rows), dtype=torch.float32, device="cuda")
+        y_fresh = torch.empty((batch, rows), dtype=torch.float32, device="cuda")
+        xfp.xfp_gemv_typed(pm.desc, pm.packed, x, batch, y_shared, shared)
+        xfp.xfp_gemv_typed(pm.desc, pm.packed, x, batch, y_fresh, torch.zeros_like(shared))
+        torch.cuda.synchronize()
+        assert torch.equal(y_shared, y_fresh), (i, batch)
+    counters = shared[:((rows + 31) // 32) * 4].view(torch.int32)
+    assert int((counters != 0).sum()) == 0
+
+
 @pytest.mark.parametrize("group", [64, 256])
 @pytest.mark.parametrize("bits", [2, 3, 4, 5, 6])
 def test_v2a_group_sizes_other_than_128(group, bits):
