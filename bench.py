@@ -223,6 +223,7 @@ def entry_of(w, ms_per_step: float, R: int, region_ms: float, peak: float) -> di
 EXTRA_CONFIGS = (
     ("config1_single_4096x4096_v2_n4", "single"),
     ("config2_attention_blocks_v2", "attention"),
+    ("config2_attention_blocks_v2_grouped_qkv", "attention_grouped"),
     ("config3_moe_token_layer_v2a_n3", "moe"),
     ("config4_stack_v2a", "stack_v2a"),
     ("config5_8192x8192_v2_n4", "shape:0:8192:8192:4:0.003"),

@@ -44,6 +44,9 @@ namespace xfp {
 namespace {
 
 constexpr int kLaneSlots = 4;   // outlier slots a warp keeps in flight
+// smallest N whose codebooks travel through shared memory before the table fill (measured: N = 5 gains 4-8 %,
+// N <= 4 loses the extra barrier)
+constexpr int kLaneStageCodebooksFrom = 5;
 
 struct LaneArgs {
     Offsets off;
@@ -161,6 +164,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     unsigned char* xs = smem + a.tab_bytes;
     float* red = (float*)(xs + (size_t)K * 2);     // [W][32]
     float* xg = red + W * 32;                      // V2a: [SC][2] sums of x over the halves of every super-chunk
+    uint32_t* cbs = (uint32_t*)xg;                 // V2 pair tables: the block's codebooks, word [e / 2][channel]
 
     // ---- this CTA's block and K slice
     int blk, slice, nslices, sc0, nsc;
@@ -249,18 +253,35 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
                 *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (uint32_t)__ldg(cb + t);
             }
         } else if (T / W >= E) {
-            // a warp fills whole rows of the pair matrix: entries (hi, 0..E-1) for its values of hi
+            // a warp fills whole rows of the pair matrix: entries (hi, 0..E-1) for its values of hi.  Every warp needs
+            // every entry of its lanes' channels: the block's codebooks (32 E fp16, contiguous) are fetched once with
+            // coalesced loads and transposed through shared memory, instead of 16-byte loads 2 E bytes apart by every warp.
             constexpr int HW = T / W / E;   // values of the high index per warp
+            constexpr bool kStage = N >= kLaneStageCodebooksFrom;
             uint32_t cw[E / 2];
+            if (kStage) {
+                const uint4* src = (const uint4*)(b.cb + (size_t)blk * kRowsPerBlock * E);
+                for (int i = threadIdx.x; i < 4 * E; i += kThreads) {
+                    const uint4 t = __ldg(src + i);
+                    const int ch = i / (E / 8), w4 = (i % (E / 8)) * 4;
+                    cbs[(w4 + 0) * 32 + ch] = t.x; cbs[(w4 + 1) * 32 + ch] = t.y;
+                    cbs[(w4 + 2) * 32 + ch] = t.z; cbs[(w4 + 3) * 32 + ch] = t.w;
+                }
+                __syncthreads();
 #pragma unroll
-            for (int i = 0; i < E / 8; ++i) {
-                const uint4 t = __ldg((const uint4*)cb + i);
-                cw[4 * i] = t.x; cw[4 * i + 1] = t.y; cw[4 * i + 2] = t.z; cw[4 * i + 3] = t.w;
+                for (int i = 0; i < E / 2; ++i) cw[i] = cbs[i * 32 + lane];
+            } else {
+#pragma unroll
+                for (int i = 0; i < E / 8; ++i) {
+                    const uint4 t = __ldg((const uint4*)cb + i);
+                    cw[4 * i] = t.x; cw[4 * i + 1] = t.y; cw[4 * i + 2] = t.z; cw[4 * i + 3] = t.w;
+                }
             }
 #pragma unroll
             for (int hh = 0; hh < HW; ++hh) {
                 const int hi = warp * HW + hh;
-                const uint32_t hv = (uint32_t)__ldg(cb + hi) << 16;
+                const uint32_t hv = (kStage ? (uint32_t)((const uint16_t*)cbs)[((hi >> 1) * 32 + lane) * 2 + (hi & 1)]
+                                            : (uint32_t)__ldg(cb + hi)) << 16;
 #pragma unroll
                 for (int lo = 0; lo < E; ++lo) {
                     const uint32_t lv = (lo & 1) ? (cw[lo >> 1] >> 16) : (cw[lo >> 1] & 0xffffu);
@@ -288,8 +309,8 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     for (int t = threadIdx.x; t < ((K / 8 + 31) & ~31); t += kThreads) {   // whole warps: the sums below shuffle
         const bool in = t < K / 8;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (in) v = __ldg((const uint4*)(xsrc) + t);
         if (in) {
-            v = __ldg((const uint4*)(xsrc) + t);
             // k = 8t .. 8t+7: its two blocks of four go to positions xpos(8t) and xpos(8t + 4)
             *(uint2*)(xs + xpos(8u * t) * 2) = make_uint2(v.x, v.y);
             *(uint2*)(xs + xpos(8u * t + 4u) * 2) = make_uint2(v.z, v.w);
@@ -539,7 +560,8 @@ size_t lane_tab_bytes(const Layout& l, bool sgl) {
 }
 
 size_t lane_smem_bytes(const Layout& l, const LaneConfig& c) {
-    return lane_tab_bytes(l, c.sgl) + (size_t)l.cols * 2 + (size_t)c.W * 32 * 4 + (l.mode ? (size_t)l.SC * 8 : 0);
+    // tables | x | red [W][32] | V2a: sums of x per half super-chunk; V2: the block's codebooks for the table fill
+    return lane_tab_bytes(l, c.sgl) + (size_t)l.cols * 2 + (size_t)c.W * 32 * 4 + (l.mode ? (size_t)l.SC * 8 : (size_t)l.E * 64);
 }
 
 // `RBn`: row-blocks of the launch (all blobs)

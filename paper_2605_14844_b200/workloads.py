@@ -9,6 +9,7 @@ single-kernel targets for profiler captures (`bench.py --workload NAME --launche
     stack         48 decoder layers x (q, k, v, o 4096 x 4096, 12288 x 4096, 4096 x 12288), per-layer bit width from
                   {2..6} and outlier rate from [0, 2 %] (seeded), V2 or V2a on the same draws; one token = 288 calls
     attention     blocks of q/k/v/o 4096 x 4096, V2, N from {4, 5}, ~0.9 % outliers in heavy outlier columns
+                  (attention_grouped: q, k and v of a block in one grouped launch)
     single        one 4096 x 4096 V2 layer, N = 4, 0.3 % uniform outliers, cycled over distinct copies
     moe           routed-MoE token-layers: 128 experts (gate_up 3072 x 4096, down 4096 x 1536), V2a N = 3, L = 32,
                   0.1 % outliers, top-8 routing; a token-layer is two grouped launches with fused stores
@@ -143,6 +144,37 @@ def attention(layers: int = 8, device="cuda") -> Workload:
                                   "projections": "q,k,v,o 4096x4096", "bits": bits_used[:4], "outlier_rate": 0.009,
                                   "placement": "heavy outlier columns", "batch": 1},
                     run, total, len(pms), len(pms), keep=[pms, ys, x])
+
+
+def attention_grouped(layers: int = 8, device="cuda") -> Workload:
+    """The same blocks with q, k and v (they share x) in one grouped launch per block and o as a call of its own;
+    a block's q/k/v take one bit width (a grouped launch has one descriptor)."""
+    blocks, total, bits_used, keep = [], 0, [], []
+    x = _x(1, 4096, 900, device)
+    ptrs = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device=device)
+    for layer in range(layers):
+        rng = np.random.default_rng(1000 + layer)
+        b_qkv, b_o = (int(v) for v in rng.integers(4, 6, size=2))
+        pms = [_pack(synth.random_quantized_torch(0, 4096, 4096, b_qkv if j < 3 else b_o, 0.009, seed=10 + 4 * layer + j,
+                                                  placement="clustered", device=device), device) for j in range(4)]
+        total += sum(_bytes_of(pm) for pm in pms)
+        bits_used += [b_qkv] * 3 + [b_o]
+        y = torch.empty((4, 4096), dtype=torch.float16, device=device)
+        d0 = pms[0].desc
+        desc = xb.XfpDesc(d0.mode, d0.rows, d0.cols, d0.bits, d0.group_size, d0.lib_size, d0.col_bits,
+                          max(p.desc.nnz for p in pms[:3]))
+        ws = torch.zeros(3 * xb.xfp_packed_size(desc)[1], dtype=torch.uint8, device=device)
+        blocks.append((desc, ptrs([p.packed for p in pms[:3]]), ptrs([x] * 3), ptrs([y[j] for j in range(3)]), ws, pms[3], y))
+        keep.append(pms)
+
+    def run():
+        for desc, pp, px, py, ws, po, y in blocks:
+            xb.xfp_gemv_grouped(desc, 3, pp, px, py, True, ws)
+            po.gemv(x, y=y[3:4], y_fp16=True)
+
+    return Workload("attention_grouped", {"workload": "dense attention blocks, q/k/v in one grouped launch", "mode": "V2",
+                                          "blocks": layers, "bits": bits_used[:4], "outlier_rate": 0.009, "batch": 1},
+                    run, total, 4 * layers, 2 * layers, keep=[blocks, keep, x])
 
 
 def shape(mode: int, rows: int, cols: int, bits: int, rate: float, batch: int = 1, placement: str = "uniform",
@@ -300,6 +332,8 @@ def parse(spec: str, device="cuda", **kw) -> Workload:
         return stack(1 if spec.endswith("a") else 0, device=device, **kw)
     if spec == "attention":
         return attention(device=device)
+    if spec == "attention_grouped":
+        return attention_grouped(device=device)
     if spec == "single":
         return single(device=device)
     if spec == "moe":
