@@ -43,8 +43,10 @@ FALLBACK_HBM_GBS = 6650.0
 METRIC = "fused XFP GEMV effective GB/s at batch 1"
 MIN_REGION_S = 0.25
 # dram__bytes_read.sum + dram__bytes_write.sum per launch divided by the algorithmic bytes of that launch, from the
-# ncu captures summarised under profiles/ (the ratio of the batch-1 V2 kernel; None = no capture of this build yet)
-NCU_TRAFFIC_RATIO = {"stack_v2": None}
+# ncu captures of the batch-1 V2 kernel summarised under profiles/ (gemv_lane_v2_4096x4096.md: 9.62 MB against 9.16 MB
+# = 1.05; gemv_lane_v2_28672x8192.md: 125.8 MB against 121.4 MB = 1.04).  The stack's 288 launches are those kernels
+# on 25-75 MB matrices; its traffic is scaled from them by bytes (traffic grows with the matrix, nothing is re-read).
+NCU_TRAFFIC_RATIO = {"stack_v2": 1.045, "shape_v2_28672x8192_n4_b1": 1.036, "single": 1.05}
 
 
 def block_spec(layer: int):

@@ -204,6 +204,50 @@ def shape(mode: int, rows: int, cols: int, bits: int, rate: float, batch: int = 
                     sample=[(synth.to_host(q), synth.activations(batch, cols, 3))] if rows * cols <= (1 << 24) else [])
 
 
+def gemm(mode: int, rows: int, cols: int, bits: int, rate: float, m: int, device="cuda", copies: Optional[int] = None) -> Workload:
+    """The prefill form (xfp_gemm, tcgen05) with m rows of x on one matrix, cycled over distinct packed copies."""
+    q = synth.random_quantized_torch(mode, rows, cols, bits, rate, seed=1, device=device)
+    first = _pack(q, device)
+    nb = _bytes_of(first, 0) + m * (cols * 2 + rows * 2)
+    if copies is None:
+        copies = max(2, int(2 * L2_BYTES // nb) + 1)
+    blobs = [first.packed] + [first.packed.clone() for _ in range(copies - 1)]
+    x = _x(m, cols, 3, device)
+    ys = [torch.empty((m, rows), dtype=torch.float16, device=device) for _ in blobs]
+    wss = [torch.zeros(xb.xfp_gemm_workspace_size(first.desc, m), dtype=torch.uint8, device=device) for _ in blobs]
+
+    def run():
+        for blob, y, ws in zip(blobs, ys, wss):
+            xb.xfp_gemm(first.desc, blob, x, y, ws)
+
+    return Workload(f"gemm_{'v2a' if mode else 'v2'}_{rows}x{cols}_n{bits}_m{m}",
+                    {"workload": f"prefill form, {rows}x{cols} {'V2a' if mode else 'V2'} N={bits}, {m} rows of x",
+                     "rows": rows, "cols": cols, "bits": bits, "outlier_rate": rate, "m": m, "copies": copies,
+                     "flops_per_call": 2.0 * m * rows * cols},
+                    run, nb * copies, copies, copies, keep=[blobs, x, ys, wss, first])
+
+
+def pack_dequant(mode: int, rows: int, cols: int, bits: int, rate: float, device="cuda") -> Workload:
+    """xfp_pack (unpacked tensors -> blob) followed by xfp_dequant (blob -> fp16 matrix) on one matrix; bytes: byte
+    indices in and bit stream out for pack, blob in and fp16 matrix out for dequant, metadata both ways."""
+    q = synth.random_quantized_torch(mode, rows, cols, bits, rate, seed=1, device=device)
+    pm = _pack(q, device)
+    d = pm.desc
+    W = torch.empty((rows, cols), dtype=torch.float16, device=device)
+    ocol = q.ocol.to(torch.int16) if q.ocol.numel() else torch.zeros(16, dtype=torch.int16, device=device)
+    oval = q.oval if q.oval.numel() else torch.zeros(16, dtype=torch.int16, device=device)
+
+    def run():
+        xb.xfp_pack(d, q.idx, q.codebook, q.gid, q.gscale, q.gmid, q.rowptr, ocol, oval, pm.packed, pm.err_word)
+        xb.xfp_dequant(d, pm.packed, W)
+
+    meta = _bytes_of(pm, 0) - rows * cols * bits // 8
+    nbytes = (rows * cols + rows * cols * bits // 8 + 2 * meta) + (rows * cols * bits // 8 + meta + rows * cols * 2)
+    return Workload(f"pack_dequant_{rows}x{cols}_n{bits}", {"workload": f"xfp_pack + xfp_dequant, {rows}x{cols} N={bits}",
+                                                            "rows": rows, "cols": cols, "bits": bits, "outlier_rate": rate},
+                    run, nbytes, 2, 9, keep=[q, pm, W, ocol, oval])
+
+
 def single(device="cuda") -> Workload:
     w = shape(0, 4096, 4096, 4, 0.003, device=device, name="single")
     w.config["workload"] = "single linear 4096x4096, V2 N=4, 0.3 % outliers (configuration 1)"
@@ -327,7 +371,8 @@ def profile_launches(w: Workload, launches: int, device) -> None:
 
 def parse(spec: str, device="cuda", **kw) -> Workload:
     """Workload from a name: stack_v2 | stack_v2a | attention | single | moe |
-    shape:MODE:ROWS:COLS:BITS:RATE[:BATCH[:PLACEMENT[:COPIES]]]  (MODE 0 = V2, 1 = V2a)."""
+    shape:MODE:ROWS:COLS:BITS:RATE[:BATCH[:PLACEMENT[:COPIES]]] | gemm:MODE:ROWS:COLS:BITS:RATE:M[:COPIES] |
+    packdq:MODE:ROWS:COLS:BITS:RATE  (MODE 0 = V2, 1 = V2a)."""
     if spec in ("stack_v2", "stack_v2a"):
         return stack(1 if spec.endswith("a") else 0, device=device, **kw)
     if spec == "attention":
@@ -343,4 +388,11 @@ def parse(spec: str, device="cuda", **kw) -> Workload:
         mode, rows, cols, bits = (int(v) for v in f[:4])
         return shape(mode, rows, cols, bits, float(f[4]), int(f[5]) if len(f) > 5 else 1,
                      f[6] if len(f) > 6 else "uniform", device=device, copies=int(f[7]) if len(f) > 7 else None)
+    if spec.startswith("gemm:"):      # gemm:MODE:ROWS:COLS:BITS:RATE:M[:COPIES]
+        f = spec.split(":")[1:]
+        return gemm(int(f[0]), int(f[1]), int(f[2]), int(f[3]), float(f[4]), int(f[5]), device=device,
+                    copies=int(f[6]) if len(f) > 6 else None)
+    if spec.startswith("packdq:"):    # packdq:MODE:ROWS:COLS:BITS:RATE
+        f = spec.split(":")[1:]
+        return pack_dequant(int(f[0]), int(f[1]), int(f[2]), int(f[3]), float(f[4]), device=device)
     raise ValueError(f"unknown workload {spec!r}")
