@@ -61,7 +61,8 @@ struct LaneArgs {
     float* partial;  // [slice][rows_ws]
     int* tickets;    // [blocks of the launch]
     int rows, cols, RB, SC, rows_ws, ell_slots;
-    int y_is_fp16;
+    int y_is_fp16;   // type of y: 0 fp32, 1 fp16, 2 bf16
+    int x_bf16;      // x holds bf16: converted to fp16 while it is staged
     int tab_bytes;   // shared-memory bytes of the look-up tables
     int L, GH;       // V2a: library size; groups per super-chunk (2 when the format's groups hold 64 weights)
     // schedule tiers: CTAs [tier_cta[i], tier_cta[i+1]) handle blocks from tier_blk[i] on, each cut into
@@ -147,7 +148,9 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
 // of its channel's current group, the fragment accumulates sum lib * x of ONE group, and after the group's steps the
 // sum moves to the lane that owns the channel and is folded into its accumulator with the group's scale and
 // mid-point:  acc += scale * G + mid * X_g,  X_g = sum of x over the group ("V2a: Shared Codebook Library").
-template <int N, int W, int MINB, bool SGL, int MODE>
+// TIO instantiations take bf16 x and store bf16 y; compiled into the plain ones the conversion cost the fp16 path 4.5 %
+// at 28672 x 8192 through register allocation alone (34.3 against 32.8 us), so only bf16 calls launch them.
+template <int N, int W, int MINB, bool SGL, int MODE, bool TIO>
 __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs a) {
     using C = LaneCfg<N, SGL>;
     constexpr int E = C::E;
@@ -309,7 +312,10 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     for (int t = threadIdx.x; t < ((K / 8 + 31) & ~31); t += kThreads) {   // whole warps: the sums below shuffle
         const bool in = t < K / 8;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (in) v = __ldg((const uint4*)(xsrc) + t);
+                if (in) {
+            v = __ldg((const uint4*)(xsrc) + t);
+            if (TIO) v = x8_as_f16(v, a.x_bf16);
+        }
         if (in) {
             // k = 8t .. 8t+7: its two blocks of four go to positions xpos(8t) and xpos(8t + 4)
             *(uint2*)(xs + xpos(8u * t) * 2) = make_uint2(v.x, v.y);
@@ -474,7 +480,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             if (t == 0) a.tickets[gblk] = 0;
         }
     }
-    if (writer && active && row < a.rows) store_y<false>(ydst, (size_t)row, total, a.y_is_fp16);
+        if (writer && active && row < a.rows) store_y<TIO>(ydst, (size_t)row, total, a.y_is_fp16);
     lstamp(a, 5);
 }
 
@@ -601,12 +607,12 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
     return c;
 }
 
-template <int N, int W, int MINB, bool SGL, int MODE>
-cudaError_t launch_lane(const LaneArgs& a, int grid, size_t smem, cudaStream_t s) {
+template <int N, int W, int MINB, bool SGL, int MODE, bool TIO>
+cudaError_t launch_lane_io(const LaneArgs& a, int grid, size_t smem, cudaStream_t s) {
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_lane_kernel<N, W, MINB, SGL, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemv_lane_kernel<N, W, MINB, SGL, MODE, TIO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              MINB == 1 ? 224 * 1024 : 110 * 1024);
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
@@ -621,7 +627,13 @@ cudaError_t launch_lane(const LaneArgs& a, int grid, size_t smem, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_lane_kernel<N, W, MINB, SGL, MODE>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_lane_kernel<N, W, MINB, SGL, MODE, TIO>, a);
+}
+
+template <int N, int W, int MINB, bool SGL, int MODE>
+cudaError_t launch_lane(const LaneArgs& a, int grid, size_t smem, cudaStream_t s) {
+    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_lane_io<N, W, MINB, SGL, MODE, true>(a, grid, smem, s);
+    return launch_lane_io<N, W, MINB, SGL, MODE, false>(a, grid, smem, s);
 }
 
 template <int N, bool SGL, int MODE>
@@ -633,9 +645,9 @@ cudaError_t launch_lane_cfg(const LaneConfig& c, const LaneArgs& a, int grid, si
 
 }  // namespace
 
-// a single blob, batch 1, fp16 x, fp32 / fp16 y, no fused store; x short enough to stage beside the tables
+// batch 1 (fp16 or bf16 x, any y type), one blob or several, no fused store; x short enough to stage beside the tables
 bool lane_supported(const Layout& l, const GemvCall& c) {
-    if (c.batch != 1 || c.n < 1 || c.x_bf16 || c.y_is_fp16 == 2 || c.epilogue != 0) return false;
+    if (c.batch != 1 || c.n < 1 || c.epilogue != 0) return false;
     if ((c.n > 1) != (c.packed_list != nullptr)) return false;
     if (l.bits < 2 || l.bits > 6) return false;
     if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) return false;   // V2a: the per-bank library must fit (N = 6 does not)
@@ -653,7 +665,7 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
     a.packed_list = c.packed_list; a.x_list = c.x_list; a.y_list = c.y_list;
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
     a.rows_ws = l.RB * c.n * 32;
-    a.y_is_fp16 = c.y_is_fp16;
+    a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16;
     a.tab_bytes = (int)lane_tab_bytes(l, cfg.sgl);
     a.L = l.L; a.GH = l.GH;
     for (int i = 0; i < 5; ++i) a.tier_cta[i] = sch.tier_cta[i];
