@@ -86,8 +86,6 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
         e = launch_gemv_pair(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && batch_supported(l, c.batch))
         e = launch_gemv_batch(l, cc, (cudaStream_t)stream);
-    else if (!c.packed_list && batch_v2a_supported(l, c.batch))
-        e = launch_gemv_batch_v2a(l, cc, (cudaStream_t)stream);
     else if (v2a_supported(l, c.batch))
         e = launch_gemv_v2a(l, cc, (cudaStream_t)stream);
     else

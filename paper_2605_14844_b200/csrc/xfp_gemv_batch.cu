@@ -1,16 +1,23 @@
-// Batched fused decode for V2 blobs, 3..16 rows of x:  y[b] = (D + S) x[b].
+// Batched fused decode, 3..16 rows of x, for V2 and V2a blobs:  y[b] = (D + S) x[b].
 //
-// Same decode as xfp_gemv_pair.cu (pair tables in per-lane shared-memory banks, looked-up half2 used
-// directly as the A fragment of mma.sync.m16n8k16, x on the diagonal lanes of the B fragment), but
-// every decoded fragment is multiplied with NB/2 B fragments, one per pair of batch rows: the
-// look-ups, which bound the kernel, are paid once per weight whatever the batch.  Here the tensor
-// pipe does real work (NB/2 mma per 8 weights of a lane), the reason the paper's step 4 is a tensor
-// core GEMM.
+// Same decode as xfp_gemv_pair.cu (tables in per-lane shared-memory banks, looked-up half2 used directly as the A
+// fragment of mma.sync.m16n8k16, x on the diagonal lanes of the B fragment), but every decoded fragment is
+// multiplied with NB/2 B fragments, one per pair of batch rows: the look-ups, which bound the kernel, are paid
+// once per weight whatever the batch.  Here the tensor pipe does real work (NB/2 mma per 8 weights of a lane),
+// the reason the paper's step 4 is a tensor core GEMM.
 //
-// x is staged in shared memory as 16-byte chunks ordered [k / 8][batch row], so the two diagonal
-// lane groups of a batch pair read adjacent chunks (one wavefront) and outlier columns are gathered
-// from the same copy.  One CTA per SM (16 warps): tables + x take up to ~200 KB.  After the K loop
-// the x area is reused for the cross-warp reduction.  Batches above 8 run as two tiles.
+// MODE 0 (V2): pair tables of the lanes' own channels.  MODE 1 (V2a, "V2a: Shared Codebook Library"):
+//     y[b][i] = sum_g [ scale_ig * sum_{k in g} lib[id_ig][q_ik] x[b][k]  +  mid_ig * sum_{k in g} x[b][k] ]  +  (S x[b])_i
+// with the library replicated once per shared-memory bank (word (id * 2^N + q) * 32 + lane), one look-up per weight
+// and a PRMT joining two of them into a half2; the fragments accumulate the sums of ONE 128-weight group, which
+// then move to the lanes that own the channels and are folded into fp32 accumulators with the group's scale and
+// mid-point, acc[b] += scale * G[b] + mid * X_g[b] (X_g[b]: sum of x[b] over the group, computed once per CTA from
+// the staged copy of x).  Nothing is rounded to fp16 on the way.
+//
+// x is staged in shared memory as 16-byte chunks ordered [k / 8][batch row], so the two diagonal lane groups of a
+// batch pair read adjacent chunks (one wavefront) and outlier columns are gathered from the same copy.  One CTA
+// per SM (16 warps): tables + x take up to ~200 KB.  After the K loop the x area is reused for the cross-warp
+// reduction.  Batches above 8 run as two tiles.
 #include "xfp_internal.h"
 #include "xfp_pair_common.cuh"
 
@@ -27,7 +34,7 @@ struct BatchArgs {
     void* y;
     float* partial;  // [KS][NB][rows_ws]
     int* tickets;    // [blocks]
-    int rows, cols, RB, SC, rows_ws, ell_slots;
+    int rows, cols, RB, SC, rows_ws, ell_slots, L;
     int nb, y_is_fp16, x_bf16;
     int n_full, kst, sc_per_split;
 };
@@ -38,17 +45,34 @@ __device__ __forceinline__ uint32_t xoff(int bb, uint32_t k) {
     return (((k >> 3) * NB + (uint32_t)bb) << 4) + ((k & 7u) << 1);
 }
 
-template <int N, int NB, int RPL, bool TIO>
+// Byte offset (q << 7) of index j (compile time) of a 128-weight stream, merged with `base`
+// (= id * 2^N * 128 + lane * 4; the q field occupies bits 7 .. 7+N, which base leaves clear).
+template <int N>
+__device__ __forceinline__ uint32_t lib_entry_addr(const uint32_t* w, int j, uint32_t base) {
+    constexpr uint32_t mask = ((1u << N) - 1u) << 7;
+    const int bit = j * N, wi = bit >> 5, off = bit & 31;
+    uint32_t v;
+    if (off + N > 32)
+        v = __funnelshift_r(w[wi], w[wi + 1], off - 7);   // field straight to bit 7 (off > 7 whenever it straddles)
+    else if (off >= 7)
+        v = w[wi] >> (off - 7);
+    else
+        v = w[wi] << (7 - off);
+    return (v & mask) | base;
+}
+
+template <int N, int NB, int RPL, bool TIO, int MODE>
 __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArgs a) {
+    static_assert(MODE == 0 || RPL == 2, "V2a blocks hold two channels per lane");
     constexpr int E = 1 << N;
     constexpr int T = E * E;
     constexpr int ROWS = 32 * RPL;
     constexpr int kStride = 128 * RPL;
-    constexpr int kTabBytes = T * kStride;
     constexpr int NBP = NB / 2;   // batch pairs
     constexpr int W = kBWarps;
     extern __shared__ __align__(16) unsigned char smem[];
-    // [tables | x chunks (NB * K * 2 bytes), later red[W][NB][ROWS] fp32]
+    // V2:  [pair tables | x chunks (NB * K * 2 bytes), later red[W][NB][ROWS] fp32]
+    // V2a: [library L*E*128 bytes | xg fp32 [NB][SC] | x chunks, later red]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     asm volatile("griddepcontrol.launch_dependents;");
     int blk, ks, KS, spp;
@@ -63,8 +87,10 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
     const int nsc = max(0, min(a.SC, sc0 + spp) - sc0);
     const int K = a.SC * kSuper;
 
+    const int tab_bytes = MODE == 1 ? a.L * E * 128 : T * kStride;
     unsigned char* tab = smem;
-    unsigned char* xs = smem + kTabBytes;
+    float* xg = (float*)(smem + tab_bytes);                                  // V2a: [NB][SC]
+    unsigned char* xs = smem + tab_bytes + (MODE == 1 ? (((size_t)NB * a.SC * 4 + 15) & ~(size_t)15) : 0);
     float* red = (float*)xs;
 
     const int blk0 = RPL * blk;
@@ -76,6 +102,9 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
     if (RPL == 2) w1[4 * N] = 0u;
     const uint4* i0 = b.idx + ((size_t)(blk0 * a.SC + sc0) * N) * 32 + lane;
     const uint4* i1 = b.idx + ((size_t)(blk1 * a.SC + sc0) * N) * 32 + lane;
+    // V2a: library ids and (scale, mid) of the two channels' current and next group
+    const size_t m0 = (size_t)(blk0 * a.SC + sc0) * 32 + lane, m1 = (size_t)(blk1 * a.SC + sc0) * 32 + lane;
+    uint32_t id0 = 0, id1 = 0, sm0 = 0, sm1 = 0, nid0 = 0, nid1 = 0, nsm0 = 0, nsm1 = 0;
     if (warp < nsc) {
 #pragma unroll
         for (int v = 0; v < N; ++v) {
@@ -85,6 +114,10 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
                 const uint4 t1 = ld_stream(i1 + ((size_t)warp * N + v) * 32);
                 w1[4 * v] = t1.x; w1[4 * v + 1] = t1.y; w1[4 * v + 2] = t1.z; w1[4 * v + 3] = t1.w;
             }
+        }
+        if (MODE == 1) {
+            id0 = b.gid[m0 + (size_t)warp * 32]; id1 = b.gid[m1 + (size_t)warp * 32];
+            sm0 = b.gsm[m0 + (size_t)warp * 32]; sm1 = b.gsm[m1 + (size_t)warp * 32];
         }
     }
     const int gw = ks * W + warp, ostride = KS * W;
@@ -125,8 +158,12 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
     };
     if (a.ell_slots) fetch_slots(0);
 
-    // ---- (1) pair tables: warp w fills entries [w*T/W, (w+1)*T/W) of every channel half
-    {
+    // ---- (1) tables.  V2a: the library, one copy per bank (word e * 32 + lane = lib[e] for every lane).
+    //      V2: pair tables, warp w fills entries [w*T/W, (w+1)*T/W) of every channel half
+    if (MODE == 1) {
+        for (int e = warp; e < a.L * E; e += W)
+            *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+    } else {
         constexpr int TW = T / W;
 #pragma unroll
         for (int half = 0; half < RPL; ++half) {
@@ -180,18 +217,51 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
         nrounds = max(nrounds, (mine + kBSlots - 1) / kBSlots);
     }
     __syncthreads();
+    if (MODE == 1) {
+        // X_g[bb]: the 128 values of group u are 16 chunks of 8; lane l sums 4 of them, then a fixed butterfly
+        for (int u = warp; u < NB * a.SC; u += W) {
+            const int bb = u / a.SC, gq = u - bb * a.SC;
+            const uint2 hv = *(const uint2*)(xs + (((size_t)(16 * gq + (lane >> 1)) * NB + bb) << 4) + (lane & 1) * 8);
+            const float2 p0 = __half22float2(*(const __half2*)&hv.x), p1 = __half22float2(*(const __half2*)&hv.y);
+            float t = (p0.x + p0.y) + (p1.x + p1.y);
+#pragma unroll
+            for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            if (lane == 0) xg[u] = t;
+        }
+        __syncthreads();
+    }
 
-    // ---- (3) main loop
+    // ---- (3) main loop (V2a: over this warp's groups, the fragments restart with every group)
     float c[NBP][4];
 #pragma unroll
     for (int p = 0; p < NBP; ++p) c[p][0] = c[p][1] = c[p][2] = c[p][3] = 0.f;
-    const uint32_t base0 = (uint32_t)lane * 4u, base1 = base0 | 128u;
+    uint32_t base0 = (uint32_t)lane * 4u, base1 = MODE == 1 ? base0 : (base0 | 128u);
+    const uint32_t lane4 = (uint32_t)lane * 4u;
     const int g = lane >> 2, t4 = lane & 3;
     const bool diag0 = (g == t4), diag1 = (g == t4 + 4);
     const bool diag = diag0 || diag1;
     const int b2 = diag1 ? 1 : 0;
 
+    // V2a: where this lane's own sums land: D[g][t] sits in lane (g, t >> 1), register t & 1 (even batch row of the
+    // pair), and in lane (g, 2 + (t >> 1)) for the odd one
+    const int src0 = (lane & ~3) | (t4 >> 1);
+    const bool odd = t4 & 1;
     auto lookup = [&](uint32_t (&f)[4], int m) {
+        if (MODE == 1) {
+            const uint32_t l00 = *(const uint32_t*)(tab + lib_entry_addr<N>(w0, 4 * m + 0, base0));
+            const uint32_t l01 = *(const uint32_t*)(tab + lib_entry_addr<N>(w0, 4 * m + 1, base0));
+            const uint32_t l02 = *(const uint32_t*)(tab + lib_entry_addr<N>(w0, 4 * m + 2, base0));
+            const uint32_t l03 = *(const uint32_t*)(tab + lib_entry_addr<N>(w0, 4 * m + 3, base0));
+            const uint32_t l10 = *(const uint32_t*)(tab + lib_entry_addr<N>(w1, 4 * m + 0, base1));
+            const uint32_t l11 = *(const uint32_t*)(tab + lib_entry_addr<N>(w1, 4 * m + 1, base1));
+            const uint32_t l12 = *(const uint32_t*)(tab + lib_entry_addr<N>(w1, 4 * m + 2, base1));
+            const uint32_t l13 = *(const uint32_t*)(tab + lib_entry_addr<N>(w1, 4 * m + 3, base1));
+            f[0] = __byte_perm(l00, l01, 0x5410);   // (k, k+1) of channel 0
+            f[1] = __byte_perm(l10, l11, 0x5410);   // (k, k+1) of channel 1
+            f[2] = __byte_perm(l02, l03, 0x5410);   // (k+2, k+3) of channel 0
+            f[3] = __byte_perm(l12, l13, 0x5410);   // (k+2, k+3) of channel 1
+            return;
+        }
         f[0] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m, base0));
         f[2] = *(const uint32_t*)(tab + pair_addr<N, RPL>(w0, 2 * m + 1, base0));
         if (RPL == 2) {
@@ -209,10 +279,21 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
         }
         const bool has_next = s + W < nsc;
         const int snext = s + W;
+        if (MODE == 1) {
+            if (has_next) {   // metadata of the next group travels during this one
+                nid0 = b.gid[m0 + (size_t)snext * 32]; nid1 = b.gid[m1 + (size_t)snext * 32];
+                nsm0 = b.gsm[m0 + (size_t)snext * 32]; nsm1 = b.gsm[m1 + (size_t)snext * 32];
+            }
+            base0 = id0 * (uint32_t)(E * 128) + lane4;
+            base1 = id1 * (uint32_t)(E * 128) + lane4;
+#pragma unroll
+            for (int p = 0; p < NBP; ++p) c[p][0] = c[p][1] = c[p][2] = c[p][3] = 0.f;
+        }
         auto reload = [&](int gi) {
 #pragma unroll
             for (int v = 0; v < N; ++v) {
-                const int plast = (128 * (v + 1) + 2 * N - 1) / (2 * N) - 1;
+                // last look-up group (of 4 weights per channel) that still reads index vector v
+                const int plast = MODE == 1 ? ((128 * (v + 1) + N - 1) / N - 1) / 2 : (128 * (v + 1) + 2 * N - 1) / (2 * N) - 1;
                 if (plast / 2 == gi && has_next) {
                     const uint4 t0 = ld_stream(i0 + ((size_t)snext * N + v) * 32);
                     w0[4 * v] = t0.x; w0[4 * v + 1] = t0.y; w0[4 * v + 2] = t0.z; w0[4 * v + 3] = t0.w;
@@ -245,6 +326,22 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
 #pragma unroll
             for (int p = 0; p < NBP; ++p) mma16816(c[p], fb[0], fb[1], fb[2], fb[3], xq[p].z, xq[p].w);
         }
+        if (MODE == 1) {
+            // group sums to their owners, then  acc += scale * G + mid * X_g  (oacc doubles as the accumulator)
+            const float sc_0 = h2f((uint16_t)(sm0 & 0xffffu)), md_0 = h2f((uint16_t)(sm0 >> 16));
+            const float sc_1 = h2f((uint16_t)(sm1 & 0xffffu)), md_1 = h2f((uint16_t)(sm1 >> 16));
+#pragma unroll
+            for (int bb = 0; bb < NB; ++bb) {
+                const int src = src0 + 2 * (bb & 1);
+                const float e0 = __shfl_sync(0xffffffffu, c[bb >> 1][0], src), e1 = __shfl_sync(0xffffffffu, c[bb >> 1][1], src);
+                const float e2 = __shfl_sync(0xffffffffu, c[bb >> 1][2], src), e3 = __shfl_sync(0xffffffffu, c[bb >> 1][3], src);
+                const float G0 = odd ? e1 : e0, G1 = odd ? e3 : e2;
+                const float X = xg[bb * a.SC + sc0 + s];
+                oacc[bb][0] = fmaf(sc_0, G0, fmaf(md_0, X, oacc[bb][0]));
+                oacc[bb][RPL - 1] = fmaf(sc_1, G1, fmaf(md_1, X, oacc[bb][RPL - 1]));
+            }
+            id0 = nid0; id1 = nid1; sm0 = nsm0; sm1 = nsm1;
+        }
     }
     while (oround < nrounds) {
         consume_slots();
@@ -269,7 +366,12 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
 
     // ---- (4) the x area becomes red[W][NB][ROWS]; fragment lanes scatter to channel order, owners add outliers
     __syncthreads();   // every warp is done reading x
-    {
+    if (MODE == 1) {   // every lane already owns its two channels' sums
+#pragma unroll
+        for (int bb = 0; bb < NB; ++bb)
+#pragma unroll
+            for (int h = 0; h < RPL; ++h) red[((size_t)warp * NB + bb) * ROWS + 32 * h + lane] = oacc[bb][h];
+    } else {
         const int l0 = 4 * g + 2 * (t4 & 1);
 #pragma unroll
         for (int p = 0; p < NBP; ++p) {
@@ -328,31 +430,36 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
 
 // ------------------------------------------------------------------------------------ host side
 
-static int batch_rpl(int bits) { return bits == 5 ? 1 : 2; }
+static int batch_rpl(const Layout& l) { return (l.mode == 0 && l.bits == 5) ? 1 : 2; }
 
 static size_t batch_smem_bytes(const Layout& l, int nbt) {
-    const int rpl = batch_rpl(l.bits);
+    const int rpl = batch_rpl(l);
     const size_t x = (size_t)nbt * l.cols * 2, red = (size_t)kBWarps * nbt * 32 * rpl * 4;
-    return (size_t)l.E * l.E * 128 * rpl + (x > red ? x : red);
+    const size_t tab = l.mode ? (size_t)l.L * l.E * 128 + (((size_t)nbt * l.SC * 4 + 15) & ~(size_t)15)
+                              : (size_t)l.E * l.E * 128 * rpl;
+    return tab + (x > red ? x : red);
 }
 
 // batch tile (4 or 8 rows of x per launch) that fits one CTA per SM, 0 if none does
 static int batch_tile(const Layout& l, int batch) {
-    if (l.mode != 0 || l.bits < 2 || l.bits > 5) return 0;
+    if (l.bits < 2 || l.bits > 5) return 0;
     if (batch > 4 && batch_smem_bytes(l, 8) <= 220u * 1024u) return 8;
     if (batch_smem_bytes(l, 4) <= 220u * 1024u) return 4;
     return 0;
 }
 
-bool batch_supported(const Layout& l, int batch) { return batch > 2 && batch_tile(l, batch) != 0; }
+// V2 blobs, and V2a blobs whose groups are whole super-chunks (groups of 64 weights go to the generic kernel)
+bool batch_supported(const Layout& l, int batch) {
+    return batch > 2 && (l.mode == 0 || l.GH == 1) && batch_tile(l, batch) != 0;
+}
 
-template <int N, int NB, int RPL, bool TIO>
+template <int N, int NB, int RPL, bool TIO, int MODE>
 static cudaError_t launch_batch_io(const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
     static DeviceOnce attr_done;
     const int dev = DeviceOnce::current();
     if (!attr_done.is_set(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_batch_kernel<N, NB, RPL, TIO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             224 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(gemv_batch_kernel<N, NB, RPL, TIO, MODE>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
         attr_done.set(dev);
     }
@@ -366,22 +473,28 @@ static cudaError_t launch_batch_io(const BatchArgs& a, dim3 grid, size_t smem, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_batch_kernel<N, NB, RPL, TIO>, a);
+    return cudaLaunchKernelEx(&cfg, gemv_batch_kernel<N, NB, RPL, TIO, MODE>, a);
 }
 
-template <int N, int NB, int RPL>
+template <int N, int NB, int RPL, int MODE>
 static cudaError_t launch_batch(const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
-    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_batch_io<N, NB, RPL, true>(a, grid, smem, s);
-    return launch_batch_io<N, NB, RPL, false>(a, grid, smem, s);
+    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_batch_io<N, NB, RPL, true, MODE>(a, grid, smem, s);
+    return launch_batch_io<N, NB, RPL, false, MODE>(a, grid, smem, s);
+}
+
+template <int N, int NB>
+static cudaError_t launch_batch_mode(int mode, const BatchArgs& a, dim3 grid, size_t smem, cudaStream_t s) {
+    if (mode) return launch_batch<N, NB, 2, 1>(a, grid, smem, s);
+    return launch_batch<N, NB, (N == 5 ? 1 : 2), 0>(a, grid, smem, s);
 }
 
 cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s) {
-    const int rpl = batch_rpl(l.bits);
+    const int rpl = batch_rpl(l);
     const int blocks = (l.RB + rpl - 1) / rpl;
     const int slots = sched_sms();   // one CTA per SM
     for (int b0 = 0; b0 < c.batch; b0 += 8) {
         const int nb = c.batch - b0 < 8 ? c.batch - b0 : 8;
-        int nbt = batch_tile(l, nb);
+        const int nbt = batch_tile(l, nb);
         if (nbt == 0) return cudaErrorInvalidValue;
         // a tile of 4 serves up to 4 rows: split an 8-row step in two when only the small tile fits
         for (int b1 = 0; b1 < nb; b1 += nbt) {
@@ -391,7 +504,7 @@ cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s
             a.packed = c.packed;
             a.x = c.x + (size_t)(b0 + b1) * l.cols;
             a.y = (void*)((char*)c.y + (size_t)(b0 + b1) * l.rows * (c.y_is_fp16 ? 2 : 4));
-            a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots;
+            a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.ell_slots = l.ell_slots; a.L = l.L;
             a.rows_ws = blocks * 32 * rpl;
             a.nb = n1; a.y_is_fp16 = c.y_is_fp16; a.x_bf16 = c.x_bf16;
             // schedule: whole-K blocks in whole rounds of slots; the last partial round cut along K (<= 16 slices)
@@ -409,19 +522,19 @@ cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s
             a.kst = (l.SC + a.sc_per_split - 1) / a.sc_per_split;
             if (a.kst <= 1) { a.kst = 1; a.n_full = blocks; rem = 0; }
             a.tickets = (int*)c.workspace;
-            a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));
+            a.partial = (float*)((char*)c.workspace + align256((size_t)l.RB * 4));   // behind the common counter region
             const size_t smem = batch_smem_bytes(l, nbt);
             dim3 grid((unsigned)(a.n_full + rem * a.kst), 1, 1);
             cudaError_t e = cudaErrorInvalidValue;
             switch (l.bits * 10 + nbt) {
-                case 24: e = launch_batch<2, 4, 2>(a, grid, smem, s); break;
-                case 28: e = launch_batch<2, 8, 2>(a, grid, smem, s); break;
-                case 34: e = launch_batch<3, 4, 2>(a, grid, smem, s); break;
-                case 38: e = launch_batch<3, 8, 2>(a, grid, smem, s); break;
-                case 44: e = launch_batch<4, 4, 2>(a, grid, smem, s); break;
-                case 48: e = launch_batch<4, 8, 2>(a, grid, smem, s); break;
-                case 54: e = launch_batch<5, 4, 1>(a, grid, smem, s); break;
-                case 58: e = launch_batch<5, 8, 1>(a, grid, smem, s); break;
+                case 24: e = launch_batch_mode<2, 4>(l.mode, a, grid, smem, s); break;
+                case 28: e = launch_batch_mode<2, 8>(l.mode, a, grid, smem, s); break;
+                case 34: e = launch_batch_mode<3, 4>(l.mode, a, grid, smem, s); break;
+                case 38: e = launch_batch_mode<3, 8>(l.mode, a, grid, smem, s); break;
+                case 44: e = launch_batch_mode<4, 4>(l.mode, a, grid, smem, s); break;
+                case 48: e = launch_batch_mode<4, 8>(l.mode, a, grid, smem, s); break;
+                case 54: e = launch_batch_mode<5, 4>(l.mode, a, grid, smem, s); break;
+                case 58: e = launch_batch_mode<5, 8>(l.mode, a, grid, smem, s); break;
             }
             if (e != cudaSuccess) return e;
         }

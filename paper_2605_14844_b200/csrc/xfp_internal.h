@@ -87,13 +87,9 @@ bool v2a_supported(const Layout& l, int batch);
 size_t v2a_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
 
-// Batched V2 path (3..16 rows of x); see xfp_gemv_batch.cu.
+// Batched path (3..16 rows of x), V2 and V2a; see xfp_gemv_batch.cu.
 bool batch_supported(const Layout& l, int batch);
 cudaError_t launch_gemv_batch(const Layout& l, const GemvCall& c, cudaStream_t s);
-
-// Batched V2a path (3..16 rows of x); see xfp_gemv_batch_v2a.cu.
-bool batch_v2a_supported(const Layout& l, int batch);
-cudaError_t launch_gemv_batch_v2a(const Layout& l, const GemvCall& c, cudaStream_t s);
 
 // Prefill form on the tcgen05 tensor cores (V2, any number of rows of x); see xfp_gemm_tc.cu.
 struct GemmCall {
