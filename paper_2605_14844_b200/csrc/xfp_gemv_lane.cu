@@ -597,6 +597,9 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
         // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
         // per lane (xfp_gemv_v2a.cu) measured faster
         c.off = !two && RB > sms && RB <= 4 * sms;
+        // the blobs of a routed layer in one launch: the resident CTAs of xfp_gemv_v2a.cu (pair tables built once per
+        // SM at N <= 3) measured faster (gate_up 30.7 vs 33.4 us, down 18.7 vs 22.9 us per launch of 8 experts)
+        if (n > 1) c.off = true;
         return c;
     }
     if (RB <= sms) return LaneConfig{16, 1, l.bits == 6};
