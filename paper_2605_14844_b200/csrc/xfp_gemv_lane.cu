@@ -108,11 +108,35 @@ struct LaneCfg {
     static constexpr int kTabBytes = T * kStride;
 };
 
+// Byte offset (q << 6) of index j (compile time) merged with `base`, for tables whose entries are 64 bytes apart
+// (two bytes per lane).
+template <int N>
+__device__ __forceinline__ uint32_t half_addr(const uint32_t* w, int j, uint32_t base) {
+    constexpr uint32_t mask = ((1u << N) - 1u) << 6;
+    const int bit = j * N, wi = bit >> 5, off = bit & 31;
+    uint32_t v;
+    if (off + N > 32)
+        v = __funnelshift_r(w[wi], w[wi + 1], off - 6);
+    else if (off >= 6)
+        v = w[wi] >> (off - 6);
+    else
+        v = w[wi] << (6 - off);
+    return (v & mask) | base;
+}
+
 // The four A registers of mma step j (weights 8j .. 8j+7 of the lane's channel in this super-chunk).
-template <int N, bool SGL>
+template <int N, bool SGL, bool HALF>
 __device__ __forceinline__ void lookup8(uint32_t (&f)[4], const uint32_t* w, int j, const unsigned char* tab,
                                         uint32_t base) {
-    if (N == 2 && !SGL) {
+    if (HALF) {
+        uint32_t e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) e[i] = *(const uint16_t*)(tab + half_addr<N>(w, 8 * j + i, base));
+        f[0] = __byte_perm(e[0], e[1], 0x5410);
+        f[2] = __byte_perm(e[2], e[3], 0x5410);
+        f[1] = __byte_perm(e[4], e[5], 0x5410);
+        f[3] = __byte_perm(e[6], e[7], 0x5410);
+    } else if (N == 2 && !SGL) {
         // bytes 2j and 2j+1 of the stream; base = lane * 8
         const uint32_t a0 = __byte_perm(w[(2 * j) >> 2], base, 0x5504u | ((uint32_t)((2 * j) & 3) << 4));
         const uint32_t a1 = __byte_perm(w[(2 * j + 1) >> 2], base, 0x5504u | ((uint32_t)((2 * j + 1) & 3) << 4));
@@ -153,6 +177,8 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
 template <int N, int W, int MINB, bool SGL, int MODE, bool TIO>
 __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs a) {
     using C = LaneCfg<N, SGL>;
+    constexpr bool kHalf = MODE == 2;   // V2a with a library too large for one 4-byte word per bank and entry
+    constexpr int kEntry = kHalf ? 64 : 128;   // V2a: bytes between library entries
     constexpr int E = C::E;
     constexpr int T = C::T;
     constexpr int kStride = C::kStride;
@@ -213,10 +239,10 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     }
     // V2a: library id and (scale, mid) of the lane's channel for the two halves of the super-chunk ([1] repeats [0]
     // unless the groups hold 64 weights), current and next
-    const int GH = MODE == 1 ? a.GH : 1;
+    const int GH = MODE != 0 ? a.GH : 1;
     const size_t m0 = ((size_t)(blk * a.SC + sc0) * GH) * 32 + lane;
     uint32_t gid_c[2] = {0u, 0u}, gsm_c[2] = {0u, 0u}, gid_n[2] = {0u, 0u}, gsm_n[2] = {0u, 0u};
-    if (MODE == 1 && warp < nsc) {
+    if (MODE != 0 && warp < nsc) {
         gid_c[0] = b.gid[m0 + (size_t)warp * GH * 32]; gsm_c[0] = b.gsm[m0 + (size_t)warp * GH * 32];
         gid_c[1] = b.gid[m0 + ((size_t)warp * GH + GH - 1) * 32]; gsm_c[1] = b.gsm[m0 + ((size_t)warp * GH + GH - 1) * 32];
     }
@@ -231,8 +257,12 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         oe[q] = j < ell_slots ? __ldg(slab + (size_t)(1 + j) * 32) : 0u;   // every slot below the capacity is readable
     }
     // ---- tables: warp w fills entries [w T / W, (w+1) T / W) of every lane's channel
-    if (MODE == 1) {
-        for (int e = warp; e < a.L * E; e += W) *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+    if (MODE != 0) {
+        if (kHalf) {
+            for (int e = warp; e < a.L * E; e += W) *(uint16_t*)(tab + (size_t)e * 64 + lane * 2) = __ldg(b.cb + e);
+        } else {
+            for (int e = warp; e < a.L * E; e += W) *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+        }
     } else {
         const uint16_t* cb = b.cb + (size_t)(blk * kRowsPerBlock + lane) * E;
         if (C::kQuad) {
@@ -321,7 +351,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             *(uint2*)(xs + xpos(8u * t) * 2) = make_uint2(v.x, v.y);
             *(uint2*)(xs + xpos(8u * t + 4u) * 2) = make_uint2(v.z, v.w);
         }
-        if (MODE == 1) {
+        if (MODE != 0) {
             // 8 consecutive threads hold 64 consecutive k: sums of x over the halves of the super-chunks, in a fixed order
             const float2 p0 = __half22float2(*(const __half2*)&v.x), p1 = __half22float2(*(const __half2*)&v.y);
             const float2 p2 = __half22float2(*(const __half2*)&v.z), p3 = __half22float2(*(const __half2*)&v.w);
@@ -337,7 +367,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
 
     const int g = lane >> 2, t4 = lane & 3;
     const bool dq = (g == t4) || (g == t4 + 4);
-    const uint32_t base = (uint32_t)lane * (C::kQuad ? 8u : 4u);
+    const uint32_t base = (uint32_t)lane * (C::kQuad ? 8u : (kHalf ? 2u : 4u));
     // a diagonal lane reads 16 bytes per two mma steps: bytes [0,16) of every 32 for g == t, [16,32) for g == t + 4
     const unsigned char* xq = xs + (size_t)sc0 * (kSuper * 2) + ((g == t4 + 4) ? 16 : 0);
 
@@ -383,8 +413,8 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         uint32_t fa[4], fb[4];
         uint4 xr = make_uint4(0u, 0u, 0u, 0u);
         uint32_t vbase = base;
-        if (MODE == 1) {
-            vbase = base + gid_c[0] * (uint32_t)(E * 128);
+        if (MODE != 0) {
+            vbase = base + gid_c[0] * (uint32_t)(E * kEntry);
             if (has_next) {   // metadata of the next super-chunk travels during this one
                 const size_t mn = m0 + (size_t)(s + W) * GH * 32;
                 gid_n[0] = b.gid[mn]; gsm_n[0] = b.gsm[mn];
@@ -402,11 +432,11 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             oacc = fmaf(scale, G, fmaf(mid, X, oacc));
             c[0] = c[1] = c[2] = c[3] = 0.f;
         };
-        lookup8<N, SGL>(fa, w, 0, tab, vbase);
+        lookup8<N, SGL, kHalf>(fa, w, 0, tab, vbase);
 #pragma unroll
         for (int j = 0; j < kSuper / 8; j += 2) {
             ld_x16_if(xr, xp + j * 16, dq);               // steps j and j + 1
-            lookup8<N, SGL>(fb, w, j + 1, tab, vbase);
+            lookup8<N, SGL, kHalf>(fb, w, j + 1, tab, vbase);
 #pragma unroll
             for (int v = 0; v < N; ++v)
                 if ((last_step_of_vector<N>(v) == j || last_step_of_vector<N>(v) == j + 1) && has_next) {
@@ -414,12 +444,12 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
                     w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
                 }
             mma16816(c, fa[0], fa[1], fa[2], fa[3], xr.x, xr.y);
-            if (MODE == 1 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)(E * 128);   // second half's library entry
-            if (j + 2 < kSuper / 8) lookup8<N, SGL>(fa, w, j + 2, tab, vbase);
+            if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)(E * kEntry);   // second half's library entry
+            if (j + 2 < kSuper / 8) lookup8<N, SGL, kHalf>(fa, w, j + 2, tab, vbase);
             mma16816(c, fb[0], fb[1], fb[2], fb[3], xr.z, xr.w);
-            if (MODE == 1 && j + 2 == kSuper / 16 && GH == 2) fold(0);   // the first group of 64 weights is complete
+            if (MODE != 0 && j + 2 == kSuper / 16 && GH == 2) fold(0);   // the first group of 64 weights is complete
         }
-        if (MODE == 1) {
+        if (MODE != 0) {
             fold(1);
             gid_c[0] = gid_n[0]; gid_c[1] = gid_n[1]; gsm_c[0] = gsm_n[0]; gsm_c[1] = gsm_n[1];
         }
@@ -441,7 +471,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     lstamp(a, 4);
     // ---- the two halves of a channel meet: lane (g, t < 2) holds D[g][2t], D[g][2t+1]; lane (g, t + 2) holds
     //      D[g+8][2t+4], D[g+8][2t+5]; then channel order through shared memory
-    if (MODE == 1) {
+    if (MODE != 0) {
         red[warp * 32 + lane] = oacc;   // every lane already owns its channel's sum
     } else {
         const float h2 = __shfl_xor_sync(0xffffffffu, c[2], 2), h3 = __shfl_xor_sync(0xffffffffu, c[3], 2);
@@ -559,7 +589,10 @@ struct LaneConfig { int W, per_sm; bool sgl; bool off = false; bool tiers = true
 size_t lane_tab_bytes(const Layout& l, bool sgl) {
     const int bits = l.bits;
     const size_t E = (size_t)1 << bits;
-    if (l.mode) return (size_t)l.L * E * 128;   // the library, one copy per bank
+    if (l.mode) {   // the library, one copy per bank: a word per entry, or half a word when that does not fit
+        const size_t full = (size_t)l.L * E * 128;
+        return full <= 128 * 1024 ? full : full / 2;
+    }
     if (bits == 2) return 256 * 256;
     if (sgl) return E * 128;
     return E * E * (bits == 4 ? 256 : 128);
@@ -596,7 +629,7 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
         c.tiers = RB > 4 * sms || !two;
         // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
         // per lane (xfp_gemv_v2a.cu) measured faster
-        c.off = !two && RB > sms && RB <= 4 * sms;
+        c.off = !two && RB > sms && RB <= 4 * sms;   // (half-word libraries: the general kernel, 34.4 vs 37.1 us at 12288 x 4096)
         // the blobs of a routed layer in one launch: the resident CTAs of xfp_gemv_v2a.cu (pair tables built once per
         // SM at N <= 3) measured faster (gate_up 30.7 vs 33.4 us, down 18.7 vs 22.9 us per launch of 8 experts)
         if (n > 1) c.off = true;
@@ -653,7 +686,7 @@ bool lane_supported(const Layout& l, const GemvCall& c) {
     if (c.batch != 1 || c.n < 1 || c.epilogue != 0) return false;
     if ((c.n > 1) != (c.packed_list != nullptr)) return false;
     if (l.bits < 2 || l.bits > 6) return false;
-    if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) return false;   // V2a: the per-bank library must fit (N = 6 does not)
+    if (l.mode && (size_t)l.L * l.E * 64 > 128 * 1024) return false;   // V2a: the per-bank library must fit 128 KB
     const LaneConfig cfg = lane_config(l, c.n);
     if (cfg.off) return false;
     return lane_smem_bytes(l, cfg) <= (cfg.per_sm == 1 ? 220u : 110u) * 1024u;
@@ -680,6 +713,16 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
     if (g_lane_trace && g_lane_trace_idx < g_lane_trace_calls) a.trace = g_lane_trace + (g_lane_trace_idx++) * 1024 * 8;
 #endif
     const size_t smem = lane_smem_bytes(l, cfg);
+    if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) {
+        // two bytes per lane and entry (lanes 2j and 2j+1 share a bank: a look-up costs two wavefronts when their
+        // entries differ): N = 6 with L = 32, which the paper's own V2a kernel does not have
+        switch (l.bits) {
+            case 4: return launch_lane<4, 16, 1, true, 2>(a, sch.grid, smem, s);
+            case 5: return launch_lane<5, 16, 1, true, 2>(a, sch.grid, smem, s);
+            case 6: return launch_lane<6, 16, 1, true, 2>(a, sch.grid, smem, s);
+            default: return cudaErrorInvalidValue;
+        }
+    }
     if (l.mode) {
         switch (l.bits) {
             case 2: return launch_lane_cfg<2, true, 1>(cfg, a, sch.grid, smem, s);
