@@ -629,7 +629,8 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
         c.tiers = RB > 4 * sms || !two;
         // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
         // per lane (xfp_gemv_v2a.cu) measured faster
-        c.off = !two && RB > sms && RB <= 4 * sms;   // (half-word libraries: the general kernel, 34.4 vs 37.1 us at 12288 x 4096)
+        const bool half_words = (size_t)l.L * l.E * 128 > 128 * 1024;   // no kernel with two channels per lane for these
+        c.off = !two && !half_words && RB > sms && RB <= 4 * sms;
         // the blobs of a routed layer in one launch: the resident CTAs of xfp_gemv_v2a.cu (pair tables built once per
         // SM at N <= 3) measured faster (gate_up 30.7 vs 33.4 us, down 18.7 vs 22.9 us per launch of 8 experts)
         if (n > 1) c.off = true;
