@@ -105,7 +105,12 @@ int xfp_pack(const xfp_desc* desc, const uint8_t* idx, const uint16_t* codebook,
  *   x  [batch][cols] fp16, batch in 1..16
  *   y  [batch][rows] fp32, or fp16 (round to nearest even of the fp32 sum) when y_is_fp16 != 0
  * Products are exact in fp32 and accumulated in fp32; the summation order is fixed, so repeated
- * calls give identical bits.  workspace/workspace_bytes as returned by xfp_packed_size. */
+ * calls give identical bits.  workspace/workspace_bytes as returned by xfp_packed_size.
+ * Which kernel serves a call depends on shape, bit width, batch and outlier count only (never on the data): batch 1
+ * runs on a kernel with one channel per lane, 2..12 rows of x on kernels that decode once per 8 rows, and from 13
+ * rows (9 for V2a) a blob with at most 1 % outliers may run on the tensor-core kernel of xfp_gemm, which multiplies
+ * with W^ = fp16(D16 + S) instead of the unrounded D + S; both lie inside the bound the tests hold every kernel to
+ * (|y - y_ref| <= 1e-3 * sum_k |W_ik x_k|). */
 int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
                 int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
 
