@@ -1,16 +1,10 @@
-// Fused decode GEMV for V2 blobs at batch 1, one output channel per lane:  y = (D + S) x.
+// Fused decode GEMV at batch 1, one output channel per lane, V2 and V2a:  y = (D + S) x.
 //
 // This is the kernel of the single-token decode step ("Fused Decode Kernel", M = 1).  It keeps the decode of
 // xfp_gemv_pair.cu -- pair tables in lane-private shared-memory banks, the looked-up half2 used directly as the A
-// fragment of mma.sync.m16n8k16, x on the diagonal lanes of the B fragment, fp32 accumulation -- and is built
-// around one constraint: a CTA (16 warps) must fit in HALF an SM (64 registers per thread, at most ~110 KB of
-// shared memory), so that
-//   * two CTAs of one launch share an SM (32 resident warps instead of 16: the look-up latency is covered and the
-//     prologue of one CTA -- codebook fetch, table fill, x staging -- runs under the K loop of the other), and
-//   * on matrices with no more row-blocks than SMs a launch fills only one half, and the CTAs of the NEXT call of
-//     the stream (programmatic dependent launch) move into the other half while this one still runs: they fetch
-//     their first index vectors, codebooks and outlier slots and fill their tables, and sit in griddepcontrol.wait
-//     with all of that done when this launch ends.
+// fragment of mma.sync.m16n8k16, x on the diagonal lanes of the B fragment, fp32 accumulation -- with one channel
+// per lane everywhere, so that a CTA is one row-block and launches of any size fill the SMs evenly: one CTA of 16
+// warps per SM on matrices with no more row-blocks than SMs, two CTAs of 8 (or 16) warps per SM beyond.
 //
 // Mapping.  A CTA owns one row-block of 32 channels (lane l = channel l) over all of K or one K slice; its warps
 // share K in super-chunks of 128 weights.  One mma covers 8 consecutive k of every channel: the fragment's row g
@@ -18,14 +12,16 @@
 // fragment with x[k..k+3], lanes with g == t+4 feed columns 4..7 with x[k+4..k+7]; D[g][n] and D[g+8][4+n] are the
 // two halves of channel 4g+n.
 //
-// Tables, per bit width:
+// Tables, per bit width (V2):
 //   N = 2   QUAD table: a byte of the index stream is four indices; entry = the four decoded fp16 (8 bytes per
 //           lane, 256 bytes between entries), so one 64-bit load decodes four weights and one PRMT builds its address
 //   N = 3   pair table, 64 entries of 4 bytes per lane
 //   N = 4   pair table, 256 entries; entries 256 bytes apart so that the index byte is the second byte of the
 //           address (one PRMT per look-up)
-//   N = 5   pair table, 1024 entries (128 KB: this width runs one CTA per SM with 128 registers)
+//   N = 5   pair table, 1024 entries (128 KB, one CTA per SM) or, beyond one round of CTAs, one entry per index
 //   N = 6   one entry per index (a pair table would need 16 KB per channel), two look-ups joined by a PRMT
+// V2a: the library replicated once per bank -- pair tables of every entry where L * 4^N words fit (N = 2 at L = 32),
+// one word per entry otherwise, half a word at N = 6 -- see the kernel's comment.
 //
 // x is staged once per CTA in shared memory in an order that lets a diagonal lane fetch the B registers of TWO
 // mma steps with one 16-byte load: inside every group of 16 k the two middle blocks of four are swapped
@@ -98,10 +94,10 @@ __device__ __forceinline__ void ld_x16_if(uint4& v, const unsigned char* p, bool
 // position of activation k in the staged copy: inside every 16 the blocks [4..7] and [8..11] trade places
 __device__ __forceinline__ uint32_t xpos(uint32_t k) { return (k & ~12u) | ((k & 4u) << 1) | ((k & 8u) >> 1); }
 
-template <int N, bool SGL>
+template <int N, bool SGL, int MODE>
 struct LaneCfg {
     static constexpr int E = 1 << N;
-    static constexpr bool kQuad = N == 2 && !SGL;
+    static constexpr bool kQuad = N == 2 && !SGL && MODE == 0;
     static constexpr bool kSingle = SGL;   // one entry per index: N = 6 always, N = 5 on short rows (no 128 KB fill)
     static constexpr int T = kQuad ? 256 : (kSingle ? E : E * E);          // table entries per channel
     static constexpr int kStride = (kQuad || N == 4) ? 256 : 128;            // bytes between entries
@@ -125,7 +121,7 @@ __device__ __forceinline__ uint32_t half_addr(const uint32_t* w, int j, uint32_t
 }
 
 // The four A registers of mma step j (weights 8j .. 8j+7 of the lane's channel in this super-chunk).
-template <int N, bool SGL, bool HALF>
+template <int N, bool SGL, bool HALF, bool QUAD>
 __device__ __forceinline__ void lookup8(uint32_t (&f)[4], const uint32_t* w, int j, const unsigned char* tab,
                                         uint32_t base) {
     if (HALF) {
@@ -136,7 +132,7 @@ __device__ __forceinline__ void lookup8(uint32_t (&f)[4], const uint32_t* w, int
         f[2] = __byte_perm(e[2], e[3], 0x5410);
         f[1] = __byte_perm(e[4], e[5], 0x5410);
         f[3] = __byte_perm(e[6], e[7], 0x5410);
-    } else if (N == 2 && !SGL) {
+    } else if (QUAD) {
         // bytes 2j and 2j+1 of the stream; base = lane * 8
         const uint32_t a0 = __byte_perm(w[(2 * j) >> 2], base, 0x5504u | ((uint32_t)((2 * j) & 3) << 4));
         const uint32_t a1 = __byte_perm(w[(2 * j + 1) >> 2], base, 0x5504u | ((uint32_t)((2 * j + 1) & 3) << 4));
@@ -152,7 +148,7 @@ __device__ __forceinline__ void lookup8(uint32_t (&f)[4], const uint32_t* w, int
         f[1] = __byte_perm(e[4], e[5], 0x5410);
         f[3] = __byte_perm(e[6], e[7], 0x5410);
     } else {
-        constexpr int SL = N == 4 ? 2 : 1;
+        constexpr int SL = N == 4 ? 2 : 1;   // N = 4: entries 256 bytes apart
         f[0] = *(const uint32_t*)(tab + pair_addr<N, SL>(w, 4 * j, base));
         f[2] = *(const uint32_t*)(tab + pair_addr<N, SL>(w, 4 * j + 1, base));
         f[1] = *(const uint32_t*)(tab + pair_addr<N, SL>(w, 4 * j + 2, base));
@@ -176,10 +172,14 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
 // at 28672 x 8192 through register allocation alone (34.3 against 32.8 us), so only bf16 calls launch them.
 template <int N, int W, int MINB, bool SGL, int MODE, bool TIO>
 __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs a) {
-    using C = LaneCfg<N, SGL>;
+    using C = LaneCfg<N, SGL, MODE>;
     constexpr bool kHalf = MODE == 2;   // V2a with a library too large for one 4-byte word per bank and entry
     constexpr int kEntry = kHalf ? 64 : 128;   // V2a: bytes between library entries
     constexpr int E = C::E;
+    // V2a with a small library (L * 4^N words per bank fit): PAIR tables of every library entry, one look-up per two
+    // weights as in V2
+    constexpr bool kLibPair = MODE == 1 && !SGL;
+    constexpr int kIdBytes = (kLibPair ? E * E : E) * kEntry;   // V2a: bytes between the tables of two library entries
     constexpr int T = C::T;
     constexpr int kStride = C::kStride;
     constexpr int kThreads = W * 32;
@@ -260,6 +260,11 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     if (MODE != 0) {
         if (kHalf) {
             for (int e = warp; e < a.L * E; e += W) *(uint16_t*)(tab + (size_t)e * 64 + lane * 2) = __ldg(b.cb + e);
+        } else if (kLibPair) {
+            for (int e = warp; e < a.L * E * E; e += W) {
+                const uint16_t* cb = b.cb + (size_t)(e >> (2 * N)) * E;
+                *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(cb + (e & (E - 1))) | ((uint32_t)__ldg(cb + ((e >> N) & (E - 1))) << 16);
+            }
         } else {
             for (int e = warp; e < a.L * E; e += W) *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
         }
@@ -414,7 +419,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         uint4 xr = make_uint4(0u, 0u, 0u, 0u);
         uint32_t vbase = base;
         if (MODE != 0) {
-            vbase = base + gid_c[0] * (uint32_t)(E * kEntry);
+            vbase = base + gid_c[0] * (uint32_t)kIdBytes;
             if (has_next) {   // metadata of the next super-chunk travels during this one
                 const size_t mn = m0 + (size_t)(s + W) * GH * 32;
                 gid_n[0] = b.gid[mn]; gsm_n[0] = b.gsm[mn];
@@ -432,11 +437,11 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             oacc = fmaf(scale, G, fmaf(mid, X, oacc));
             c[0] = c[1] = c[2] = c[3] = 0.f;
         };
-        lookup8<N, SGL, kHalf>(fa, w, 0, tab, vbase);
+        lookup8<N, SGL, kHalf, C::kQuad>(fa, w, 0, tab, vbase);
 #pragma unroll
         for (int j = 0; j < kSuper / 8; j += 2) {
             ld_x16_if(xr, xp + j * 16, dq);               // steps j and j + 1
-            lookup8<N, SGL, kHalf>(fb, w, j + 1, tab, vbase);
+            lookup8<N, SGL, kHalf, C::kQuad>(fb, w, j + 1, tab, vbase);
 #pragma unroll
             for (int v = 0; v < N; ++v)
                 if ((last_step_of_vector<N>(v) == j || last_step_of_vector<N>(v) == j + 1) && has_next) {
@@ -444,8 +449,8 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
                     w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
                 }
             mma16816(c, fa[0], fa[1], fa[2], fa[3], xr.x, xr.y);
-            if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)(E * kEntry);   // second half's library entry
-            if (j + 2 < kSuper / 8) lookup8<N, SGL, kHalf>(fa, w, j + 2, tab, vbase);
+            if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)kIdBytes;   // second half's library entry
+            if (j + 2 < kSuper / 8) lookup8<N, SGL, kHalf, C::kQuad>(fa, w, j + 2, tab, vbase);
             mma16816(c, fb[0], fb[1], fb[2], fb[3], xr.z, xr.w);
             if (MODE != 0 && j + 2 == kSuper / 16 && GH == 2) fold(0);   // the first group of 64 weights is complete
         }
@@ -589,7 +594,8 @@ struct LaneConfig { int W, per_sm; bool sgl; bool off = false; bool tiers = true
 size_t lane_tab_bytes(const Layout& l, bool sgl) {
     const int bits = l.bits;
     const size_t E = (size_t)1 << bits;
-    if (l.mode) {   // the library, one copy per bank: a word per entry, or half a word when that does not fit
+    if (l.mode) {   // the library, one copy per bank: a word per entry (per pair of entries), or half a word when that does not fit
+        if (!sgl) return (size_t)l.L * E * E * 128;
         const size_t full = (size_t)l.L * E * 128;
         return full <= 128 * 1024 ? full : full / 2;
     }
@@ -624,8 +630,10 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
     const int sms = sched_sms();
     if (l.mode) {
         // V2a: one look-up per weight in the per-bank library.  Up to 64 KB of tables (L * 2^N <= 512) two CTAs fit.
-        const bool two = lane_tab_bytes(l, true) <= 64 * 1024 && RB > sms;
-        LaneConfig c{two ? 8 : 16, two ? 2 : 1, true};
+        // Pair tables of the whole library where they fit the same 64 KB (L * 4^N <= 512: N = 2 with the paper's L = 32).
+        const bool pairs = (size_t)l.L * l.E * l.E * 128 <= 64 * 1024 && l.bits <= 3;
+        const bool two = lane_tab_bytes(l, !pairs) <= 64 * 1024 && RB > sms;
+        LaneConfig c{two ? 8 : 16, two ? 2 : 1, !pairs};
         c.tiers = RB > 4 * sms || !two;
         // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
         // per lane (xfp_gemv_v2a.cu) measured faster
@@ -726,8 +734,10 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
     }
     if (l.mode) {
         switch (l.bits) {
-            case 2: return launch_lane_cfg<2, true, 1>(cfg, a, sch.grid, smem, s);
-            case 3: return launch_lane_cfg<3, true, 1>(cfg, a, sch.grid, smem, s);
+            case 2: return cfg.sgl ? launch_lane_cfg<2, true, 1>(cfg, a, sch.grid, smem, s)
+                                   : launch_lane_cfg<2, false, 1>(cfg, a, sch.grid, smem, s);
+            case 3: return cfg.sgl ? launch_lane_cfg<3, true, 1>(cfg, a, sch.grid, smem, s)
+                                   : launch_lane_cfg<3, false, 1>(cfg, a, sch.grid, smem, s);
             case 4: return launch_lane_cfg<4, true, 1>(cfg, a, sch.grid, smem, s);
             default: return launch_lane_cfg<5, true, 1>(cfg, a, sch.grid, smem, s);
         }
