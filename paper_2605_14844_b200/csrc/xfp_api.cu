@@ -76,6 +76,8 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
     }
     if (lane_supported(l, cc))
         e = launch_gemv_lane(l, cc, (cudaStream_t)stream);
+    else if (lane_batch_supported(l, cc))
+        e = launch_gemv_lane_batch(l, cc, (cudaStream_t)stream);
     else if (!c.packed_list && !c.x_bf16 && batch_prefers_gemm(l, c.batch)) {
         // many rows of x, few outliers: one decode for all rows on the tensor cores (y = x W^T with W the matrix
         // xfp_dequant writes; inside the GEMV's bound)

@@ -78,9 +78,12 @@ bool pair_supported(const Layout& l, int batch, int n_problems);
 size_t pair_workspace_bytes(const Layout& l);
 cudaError_t launch_gemv_pair(const Layout& l, const GemvCall& c, cudaStream_t s);
 
-// V2 at batch 1, one channel per lane, half an SM per CTA; see xfp_gemv_lane.cu.
+// Batch 1, one channel per lane, V2 and V2a; see xfp_gemv_lane.cu.
 bool lane_supported(const Layout& l, const GemvCall& c);
 cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s);
+// The same decode for 2..16 rows of x (tiles of 2, 4, 8 rows); see xfp_gemv_lane_batch.cu.
+bool lane_batch_supported(const Layout& l, const GemvCall& c);
+cudaError_t launch_gemv_lane_batch(const Layout& l, const GemvCall& c, cudaStream_t s);
 
 // Fast V2a path (per-bank library + mma.sync fragments, one or several blobs); see xfp_gemv_v2a.cu.
 bool v2a_supported(const Layout& l, int batch);

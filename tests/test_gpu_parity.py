@@ -155,6 +155,41 @@ def test_batched_shapes_and_split_k(mode, rows, cols, bits):
     assert int(tickets.abs().sum().item()) == 0
 
 
+@pytest.mark.parametrize("mode,bits,group", [(0, 2, 128), (0, 3, 128), (0, 4, 128), (0, 5, 128), (0, 6, 128),
+                                             (1, 2, 128), (1, 3, 128), (1, 4, 128), (1, 5, 128), (1, 6, 128),
+                                             (1, 4, 64), (1, 2, 256), (1, 6, 64)])
+def test_several_rows_of_x_on_matrices_of_one_round(mode, bits, group):
+    """2..16 rows of x on a matrix of 79 row-blocks (more than half the SMs, fewer than all: one resident CTA per
+    row-block, the last one ragged), the shape class on which every batch goes to the one-channel-per-lane kernel with
+    1, 2, 4 or 8 B fragments per decoded fragment: tiles of 2, 4 and 8 rows, partial tiles (3, 7), two launches (11, 16)."""
+    rows, cols = 2500, 768
+    q = synth.random_quantized(mode, rows, cols, bits, 0.015, seed=9100 + 10 * bits + mode + group, group_size=group)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    for batch in (2, 3, 4, 7, 8, 11, 16):
+        _check_gemv(q, pm, synth.activations(batch, cols, seed=9200 + batch), y_fp16=bool(batch & 1))
+    tickets = pm.workspace[: ((rows + 31) // 32) * 4].view(torch.int32)
+    assert int(tickets.abs().sum().item()) == 0
+
+
+@pytest.mark.parametrize("mode,bits,rows,cols", [(0, 6, 9600, 2048), (0, 5, 9700, 1024), (1, 4, 19200, 512), (1, 2, 9600, 2048),
+                                                 (1, 6, 4800, 1024), (1, 3, 19000, 512)])
+def test_several_rows_of_x_with_resident_ctas_and_a_cut_tail(mode, bits, rows, cols):
+    """More row-blocks than CTA slots: resident CTAs walk several row-blocks with one staged copy of x, and the blocks
+    of the last partial round are cut along K and meet in the workspace (300 or 600 row-blocks on 148 or 296 slots).
+    Repeating the call gives the same bits; the counters are left zero."""
+    q = synth.random_quantized(mode, rows, cols, bits, 0.01, seed=9300 + bits + rows, placement="clustered")
+    pm = xfp.pack_tensors(q, col_bits=16)
+    sample = _sample_rows(rows, 96, seed=9301)
+    for batch in (2, 4, 5, 8, 12):
+        x16 = synth.activations(batch, cols, seed=9400 + batch)
+        _, y0 = _check_gemv(q, pm, x16, rows=sample)
+        y1 = pm.gemv(_x_dev(x16))
+        torch.cuda.synchronize()
+        assert torch.equal(y0, y1)
+    tickets = pm.workspace[: ((rows + 31) // 32) * 4].view(torch.int32)
+    assert int(tickets.abs().sum().item()) == 0
+
+
 @pytest.mark.parametrize("mode,bits", [(0, 4), (0, 5), (1, 3), (1, 4)])
 def test_longest_rows(mode, bits):
     """K = 65536, the largest the descriptor admits (u16 outlier columns): x alone is 128 KB per batch row."""
