@@ -338,3 +338,29 @@ def auto_select(W: np.ndarray, layer_class: str = "attention", candidates: Seque
             return m
     m.info["fallback"] = True
     return m
+
+
+def auto_select_moe(experts: Sequence[np.ndarray], sample: Sequence[int] = (0, 1, 2, 3),
+                    candidates: Sequence[int] = (2, 4), tau: float = 0.93, mode: int = MODE_V2A, k: float = 4.0,
+                    cap: float = 0.02, sigma_mode: str = "matrix", rate: Optional[float] = None, iters: int = 20,
+                    lib_size: int = 32):
+    """MoE sampling ("Auto-Selection"): Algorithm 1 runs once per routed layer, on the rows of a few experts (four in
+    the paper) stacked into one matrix, and the bit width it returns is used for every expert of the layer.
+
+    Steps: (1) auto_select on the concatenation of experts[i], i in `sample`, with the lazy threshold `tau`;
+    (2) every expert is then quantised on its own at that width -- its own mu, sigma and extracted weights, its own
+    per-channel codebooks (V2) or, for V2a, group assignments against the ONE library the sample's LibFit pass
+    produced, which the experts of the layer share.  Returns (list of QuantizedMatrix, the sample's info dict)."""
+    mats = [np.ascontiguousarray(W, dtype=np.float32) for W in experts]
+    picked = np.concatenate([mats[i] for i in sample], axis=0)
+    probe = auto_select(picked, "moe_routed", candidates, tau_lazy=tau, mode=mode, k=k, cap=cap, sigma_mode=sigma_mode,
+                        rate=rate, iters=iters, lib_size=lib_size)
+    out = []
+    for W in mats:
+        mask, mu, _ = outlier_mask(W, k=k, cap=cap, sigma_mode=sigma_mode, rate=rate)
+        if mode == MODE_V2:
+            out.append(quantize_v2(W, probe.bits, mask, mu, iters))
+        else:
+            out.append(quantize_v2a(W, probe.bits, mask, mu, lib_size, iters, library=probe.codebook))
+    info = dict(probe.info, bits=probe.bits, sample=tuple(int(i) for i in sample))
+    return out, info

@@ -174,3 +174,68 @@ def quantize_and_pack(W: torch.Tensor, mode: int, candidates: Sequence[int], tau
     table = (buf.lib.view(-1)[:lib_size * E] if mode else buf.codebook.view(-1)[:rows * E]).contiguous()
     xfp_pack(desc, buf.idx, table, buf.gid, buf.gscale, buf.gmid, buf.rowptr, buf.ocol, buf.oval, packed, err, stream)
     return PackedMatrix(desc, packed, workspace, err), res
+
+
+def _pack_buffers(buf: QuantBuffers, mode: int, bits: int, lib_size: int, nnz: int, table: torch.Tensor, stream=None):
+    """xfp_pack on the tensors an encoder call left in `buf` (allocation and marshalling only)."""
+    from .binding import PackedMatrix, xfp_pack, xfp_packed_size
+    desc = XfpDesc(mode, buf.rows, buf.cols, bits, 128, lib_size if mode else 0, 32, int(nnz))
+    pb, wb = xfp_packed_size(desc)
+    dev = buf.idx.device
+    packed = torch.empty(pb, dtype=torch.uint8, device=dev)
+    workspace = torch.zeros(max(wb, 16), dtype=torch.uint8, device=dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    xfp_pack(desc, buf.idx, table, buf.gid, buf.gscale, buf.gmid, buf.rowptr, buf.ocol, buf.oval, packed, err, stream)
+    return PackedMatrix(desc, packed, workspace, err)
+
+
+def quantize_with_library(W: torch.Tensor, bits: int, lib: torch.Tensor, params: XfpQuantParams, buf: QuantBuffers,
+                          stream=None) -> int:
+    """V2a encoding of one matrix against a GIVEN library (the experts of a routed layer share one, "V2a: Shared
+    Codebook Library"): statistics, outlier extraction, the group assignment of LibFit and the residual, each a
+    library call; fills `buf` (mode 1) and returns the number of extracted weights.  lib: [L, 2^bits] int16, contiguous."""
+    rows, cols = W.shape
+    L = lib.shape[0]
+    ms = torch.empty(2, dtype=torch.float64, device=W.device)
+    count = torch.zeros(1, dtype=torch.int64, device=W.device)
+    xfp_quant_stats(W, params.sigma_mode, ms, buf.workspace, stream)
+    xfp_quant_outliers(W, ms, params.outlier_mode, params.rate if params.outlier_mode else params.k_sigma,
+                       params.cap_frac, buf.mask, count, buf.workspace, stream)
+    xfp_quant_libfit_assign(W, buf.mask, ms, bits, L, lib, buf.idx, buf.gid, buf.gscale, buf.gmid, stream)
+    nnz = int(count.item())          # one read-back, as in xfp_quantize: the outlier arrays must hold them all
+    if nnz > buf.capacity:
+        raise XfpError(f"quantize_with_library: {nnz} extracted weights, buffers hold {buf.capacity}")
+    desc = XfpDesc(1, rows, cols, bits, 128, L, 32, nnz)
+    xfp_quant_residual(desc, W, buf.mask, buf.idx, lib, buf.gid, buf.gscale, buf.gmid, buf.rowptr, buf.ocol, buf.oval,
+                       buf.workspace, stream)
+    return nnz
+
+
+def quantize_moe_layer(experts: Sequence[torch.Tensor], mode: int, candidates: Sequence[int] = (2, 4), tau: float = 0.93,
+                       sample: Sequence[int] = (0, 1, 2, 3), params: Optional[XfpQuantParams] = None,
+                       lib_size: int = 32, stream=None):
+    """MoE sampling ("Auto-Selection"): Algorithm 1 once per routed layer on the stacked rows of the experts in
+    `sample` (four in the paper), then every expert of the layer encoded on its own at the returned bit width --
+    V2: its own per-channel codebooks; V2a: group assignments against the one library the sample's LibFit pass
+    produced.  experts: float32 [rows, cols] tensors on one device.  Returns ([PackedMatrix per expert],
+    XfpQuantResult of the sample, the library as an int16 tensor or None).  Every step runs in the library's kernels."""
+    if params is None:
+        params = XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 20, 0)
+    frac = params.rate if params.outlier_mode else params.cap_frac
+    stacked = torch.cat([experts[i] for i in sample], dim=0).contiguous()
+    rows_s, cols = stacked.shape
+    sbuf = QuantBuffers(rows_s, cols, mode, max(candidates), lib_size, int(frac * rows_s * cols), device=stacked.device)
+    res = xfp_quantize(mode, stacked, params, candidates, tau, sbuf, stream)
+    bits, E = int(res.bits), 1 << int(res.bits)
+    lib = sbuf.lib.view(-1)[:lib_size * E].clone().view(lib_size, E) if mode else None
+    out = []
+    for W in experts:
+        rows = W.shape[0]
+        buf = QuantBuffers(rows, cols, mode, bits, lib_size, int(frac * rows * cols), device=W.device)
+        if mode:
+            nnz = quantize_with_library(W, bits, lib, params, buf, stream)
+            out.append(_pack_buffers(buf, 1, bits, lib_size, nnz, lib.view(-1), stream))
+        else:
+            r = xfp_quantize(0, W, params, (bits,), tau, buf, stream)
+            out.append(_pack_buffers(buf, 0, bits, 0, int(r.nnz), buf.codebook.view(-1)[:rows * E].contiguous(), stream))
+    return out, res, lib

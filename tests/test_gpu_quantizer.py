@@ -293,6 +293,33 @@ def test_auto_select_matches_the_oracle_and_feeds_the_decode_path(mode, cands, t
     assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - yref) <= 1e-3 * absum + 1e-30)
 
 
+@pytest.mark.parametrize("mode,cands,tau", [(1, (2, 3, 4), 0.95), (1, (2, 4), 0.93), (0, (2, 3, 4), 0.95)])
+def test_moe_sampling_layer_matches_the_oracle(mode, cands, tau):
+    """MoE sampling ("Auto-Selection"): Algorithm 1 on four stacked experts, then every expert of the layer encoded at
+    that width (V2a: against the sample's library).  Same width, same median, same library bits as the oracle, and
+    every expert's packed blob reconstructs to the oracle's matrix bit for bit and decodes inside the GEMV bound."""
+    rows, cols, L = 64, 512, 32
+    experts = [synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, 800 + e) * np.float32(1.0 + 0.07 * e),
+                                            0.004, 900 + e) for e in range(6)]
+    sample = (1, 2, 4, 5)
+    ref, info = xo.auto_select_moe(experts, sample, candidates=cands, tau=tau, mode=mode, lib_size=L)
+    pms, res, lib = qb.quantize_moe_layer([_dev(W) for W in experts], mode, cands, tau, sample, _params(), L)
+    torch.cuda.synchronize()
+    assert res.bits == info["bits"] and bool(res.fallback) == info["fallback"]
+    assert abs(res.median_cos - info["median_cos"]) <= 1e-12
+    if mode:
+        assert np.array_equal(_u16(lib), ref[0].codebook)
+    x16 = synth.activations(2, cols, 77)
+    xd = torch.from_numpy(np.ascontiguousarray(x16).view(np.int16)).cuda().view(torch.float16)
+    for pm, q in zip(pms, ref):
+        assert pm.desc.bits == q.bits and int(pm.desc.nnz) == q.nnz and int(pm.err_word.item()) == 0
+        assert np.array_equal(_u16(pm.dequant().view(torch.int16)), xo.dequant(q))
+        yref, absum = xo.gemv(q, np.ascontiguousarray(x16).view(np.uint16))
+        y = pm.gemv(xd)
+        torch.cuda.synchronize()
+        assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - yref) <= 1e-3 * absum + 1e-30)
+
+
 def test_quantize_reports_a_small_outlier_buffer():
     rows, cols = 64, 512
     W = _weights(rows, cols, 90, rate=0.02)

@@ -327,6 +327,39 @@ def test_libfit_with_a_library_learned_on_another_matrix():
     assert cos_shared > 0.975
 
 
+@pytest.mark.parametrize("mode", [xo.MODE_V2, xo.MODE_V2A])
+def test_moe_sampling_selects_on_a_few_experts_and_quantises_all(mode):
+    """MoE sampling ("Auto-Selection"): the width comes from Algorithm 1 on the stacked sample alone -- experts outside
+    the sample cannot change it -- and every expert, sampled or not, is then quantised on its own at that width:
+    the sample's decision reproduces as a plain auto_select on the stacked matrix, a V2 expert equals its stand-alone
+    quantisation, and a V2a expert keeps the sample's library unchanged and satisfies the exhaustive-search property
+    of the group assignment against it.  Near-Gaussian experts need 3 bits for the 0.93 floor of routed layers
+    (2 bits reach 0.9394 only when converged; the sample's median decides), and widening the outsiders by 3x leaves
+    the choice alone."""
+    rows, cols, L = 24, 512, 16
+    experts = [synth.gaussian_weights(rows, cols, seed=700 + e) * np.float32(1.0 + 0.1 * e) for e in range(6)]
+    sample = (0, 2, 3, 5)
+    qs, info = xo.auto_select_moe(experts, sample, candidates=(2, 3, 4), tau=0.95, mode=mode, lib_size=L)
+    stacked = np.concatenate([experts[i] for i in sample], axis=0)
+    alone = xo.auto_select(stacked, "moe_routed", (2, 3, 4), tau_lazy=0.95, mode=mode, lib_size=L)
+    assert info["bits"] == alone.bits == 3 and not info["fallback"]
+    assert info["median_cos"] == alone.info["median_cos"] and info["sample"] == sample
+    assert len(qs) == len(experts)
+    for W, q in zip(experts, qs):
+        mask, mu, _ = xo.outlier_mask(W)
+        assert q.bits == 3 and q.rows == rows and q.nnz == int(mask.sum())
+        if mode == xo.MODE_V2:
+            own = xo.quantize_v2(W, 3, mask, mu)
+            assert np.array_equal(q.idx, own.idx) and np.array_equal(q.codebook, own.codebook)
+        else:
+            assert np.array_equal(q.codebook, alone.codebook)      # the layer's one library
+            _check_assignment_by_exhaustive_search(q, np.where(mask != 0, mu, W.astype(np.float64)), 128)
+        assert xo.median(xo.row_cosine(W, xo.dequant(q))) > 0.97
+    outsiders = [W if e in sample else W * np.float32(3.0) for e, W in enumerate(experts)]
+    _, info2 = xo.auto_select_moe(outsiders, sample, candidates=(2, 3, 4), tau=0.95, mode=mode, lib_size=L)
+    assert info2["bits"] == info["bits"] and info2["median_cos"] == info["median_cos"]
+
+
 def test_libfit_library_invariants():
     """First half of LibFit (k-means over normalised codebooks) by what any correct run must satisfy: every
     normalised codebook spans [-1, 1] exactly at its ends, so every centroid does; entries ascend; after
