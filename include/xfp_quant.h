@@ -39,7 +39,8 @@ typedef struct {
     double cap_frac;      /* paper default 0.02                                                       */
     double rate;          /* outlier_mode 1 only                                                      */
     int32_t lloyd_iters;  /* rounds of Lloyd (paper: 20; its V2 default elsewhere: 5)                 */
-    int32_t reserved;     /* 0                                                                        */
+    int32_t group_size;   /* V2a: weights per (id, scale, mid) group: 64, 128 or 256; 0 means 128, the paper's
+                             default ("a tunable parameter")                                          */
 } xfp_quant_params;
 
 typedef struct {
@@ -84,12 +85,12 @@ int xfp_quant_lloyd(const float* W, const uint8_t* mask, const double* mu_sigma,
 int xfp_quant_libfit_library(const uint16_t* codebook, int32_t rows, int32_t bits, int32_t L, int32_t iters,
                              uint16_t* lib, void* workspace, size_t workspace_bytes, void* stream);
 
-/* LibFit, second half: every group of 128 consecutive weights of a channel gets mid = fp16((max+min)/2),
- * scale = fp16((max-min)/2) of its bulk values, the library entry with the least squared error under
- * nearest-value assignment (ties: lower entry) and the indices of the nearest decoded values.
- *   idx [rows][cols], gid / gscale / gmid [rows][cols/128]. */
+/* LibFit, second half: every group of group_size (64, 128 or 256) consecutive weights of a channel gets
+ * mid = fp16((max+min)/2), scale = fp16((max-min)/2) of its bulk values, the library entry with the least squared
+ * error under nearest-value assignment (ties: lower entry) and the indices of the nearest decoded values.
+ *   idx [rows][cols], gid / gscale / gmid [rows][cols/group_size]; cols a multiple of group_size. */
 int xfp_quant_libfit_assign(const float* W, const uint8_t* mask, const double* mu_sigma, int32_t rows, int32_t cols,
-                            int32_t bits, int32_t L, const uint16_t* lib, uint8_t* idx, uint8_t* gid,
+                            int32_t bits, int32_t L, int32_t group_size, const uint16_t* lib, uint8_t* idx, uint8_t* gid,
                             uint16_t* gscale, uint16_t* gmid, void* stream);
 
 /* The residual of Eq. 1 at the extracted positions, S = fp16(w - D16), as CSR with int32 columns.

@@ -319,7 +319,7 @@ def median(v: np.ndarray) -> float:
 def auto_select(W: np.ndarray, layer_class: str = "attention", candidates: Sequence[int] = (2, 3, 4),
                 tau_strict: float = 0.96, tau_lazy: float = 0.93, mode: int = MODE_V2, k: float = 4.0,
                 cap: float = 0.02, sigma_mode: str = "matrix", rate: Optional[float] = None, iters: int = 20,
-                lib_size: int = 32) -> QuantizedMatrix:
+                lib_size: int = 32, group: int = 128) -> QuantizedMatrix:
     """Algorithm 1 (two-threshold auto-select): ascending N, first whose median per-channel cosine
     reaches the class's floor; otherwise the largest candidate (info['fallback'] = True)."""
     W = np.ascontiguousarray(W, dtype=np.float32)
@@ -328,7 +328,7 @@ def auto_select(W: np.ndarray, layer_class: str = "attention", candidates: Seque
     tried = []
     m = None
     for n in sorted(candidates):
-        m = quantize_v2(W, n, mask, mu, iters) if mode == MODE_V2 else quantize_v2a(W, n, mask, mu, lib_size, iters)
+        m = quantize_v2(W, n, mask, mu, iters) if mode == MODE_V2 else quantize_v2a(W, n, mask, mu, lib_size, iters, group)
         cosv = row_cosine(W, dequant(m))
         med = median(cosv)
         tried.append((n, med))

@@ -942,18 +942,19 @@ __global__ void libfit_store(const double* __restrict__ cen, int E, uint16_t* li
 
 // ------------------------------------------------------------------ LibFit: per-group assignment
 
-// A block of 128 threads takes `gpb` consecutive groups of 128 weights (4 when L <= 32).  Thread (s, l)
-// scores library entry l on group s serially over the 128 values; one thread per group picks the winner;
-// then the 128 threads index each group against its winner.
-__global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restrict__ W,
+// A block of GS threads takes `gpb` consecutive groups of GS weights (4 when L <= 32; GS = 64, 128 or 256, the
+// group size of the format).  Thread (s, l) scores library entry l on group s serially over the GS values; one
+// thread per group picks the winner; then the GS threads index each group against its winner.
+template <int GS>
+__global__ void __launch_bounds__(GS) libfit_group_kernel(const float* __restrict__ W,
                                                             const uint8_t* __restrict__ mask,
                                                             const double* __restrict__ ms, int64_t groups, int bits,
                                                             int L, int gpb, const uint16_t* __restrict__ lib,
                                                             uint8_t* idx, uint8_t* gid, uint16_t* gscale,
                                                             uint16_t* gmid) {
-    constexpr int GS = 128;
+    constexpr int NW = GS / 32;
     __shared__ double gv[4][GS];
-    __shared__ double red_lo[4][4], red_hi[4][4];
+    __shared__ double red_lo[4][NW], red_hi[4][NW];
     __shared__ double sse[256];
     __shared__ double dec[4][64];
     __shared__ uint16_t s_mid[4], s_sc[4];
@@ -977,8 +978,9 @@ __global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restri
     }
     __syncthreads();
     if (tid < gpb && g0 + tid < groups) {
-        const double lo = fmin(fmin(red_lo[tid][0], red_lo[tid][1]), fmin(red_lo[tid][2], red_lo[tid][3]));
-        const double hi = fmax(fmax(red_hi[tid][0], red_hi[tid][1]), fmax(red_hi[tid][2], red_hi[tid][3]));
+        double lo = red_lo[tid][0], hi = red_hi[tid][0];
+#pragma unroll
+        for (int w = 1; w < NW; ++w) { lo = fmin(lo, red_lo[tid][w]); hi = fmax(hi, red_hi[tid][w]); }
         s_mid[tid] = d2h(__dmul_rn(0.5, __dadd_rn(hi, lo)));
         s_sc[tid] = d2h(__dmul_rn(0.5, __dsub_rn(hi, lo)));
         s_const[tid] = hi == lo;
@@ -1007,7 +1009,7 @@ __global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restri
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc = __dadd_rn(acc, __dmul_rn(d[e], d[e]));
                 }
-                sse[gpb == 1 ? l : s * lw + l] = acc;
+                sse[s * L + l] = acc;   // gpb * L <= 256
             }
         }
     }
@@ -1018,7 +1020,7 @@ __global__ void __launch_bounds__(128) libfit_group_kernel(const float* __restri
         if (!s_const[tid]) {
             double b = INFINITY;
             for (int l = 0; l < L; ++l) {
-                const double e = sse[gpb == 1 ? l : tid * lw + l];
+                const double e = sse[tid * L + l];
                 if (e < b) { b = e; best = l; }
             }
         }
@@ -1118,7 +1120,9 @@ static int desc_status(const xfp_desc* d) {
     if (!d) return XFP_ERR_NULL;
     if (d->mode != 0 && d->mode != 1) return XFP_ERR_SHAPE;
     if (d->bits < 2 || d->bits > 6) return XFP_ERR_SHAPE;
-    if (d->group_size != 128) return d->group_size > 0 ? XFP_ERR_UNSUPPORTED : XFP_ERR_SHAPE;
+    if (d->group_size != 64 && d->group_size != 128 && d->group_size != 256)
+        return d->group_size > 0 ? XFP_ERR_UNSUPPORTED : XFP_ERR_SHAPE;
+    if (d->cols > 0 && d->cols % d->group_size) return XFP_ERR_SHAPE;
     if (d->mode == 1 && (d->lib_size < 1 || d->lib_size > 256)) return XFP_ERR_SHAPE;
     return shape_status(d->rows, d->cols);
 }
@@ -1253,7 +1257,7 @@ int xfp_quant_libfit_library(const uint16_t* codebook, int32_t rows, int32_t bit
 }
 
 int xfp_quant_libfit_assign(const float* W, const uint8_t* mask, const double* mu_sigma, int32_t rows, int32_t cols,
-                            int32_t bits, int32_t L, const uint16_t* lib, uint8_t* idx, uint8_t* gid,
+                            int32_t bits, int32_t L, int32_t group_size, const uint16_t* lib, uint8_t* idx, uint8_t* gid,
                             uint16_t* gscale, uint16_t* gmid, void* stream) {
     if (!W || !mu_sigma || !lib || !idx || !gid || !gscale || !gmid) return XFP_ERR_NULL;
     if (!aligned16(W) || !aligned16(lib) || !aligned16(idx) || !aligned16(gid) || !aligned16(gscale) ||
@@ -1262,11 +1266,19 @@ int xfp_quant_libfit_assign(const float* W, const uint8_t* mask, const double* m
     const int st = shape_status(rows, cols);
     if (st) return st;
     if (bits < 2 || bits > 6 || L < 1 || L > 256) return XFP_ERR_SHAPE;
-    const int64_t groups = (int64_t)rows * (cols / 128);
+    if (group_size != 64 && group_size != 128 && group_size != 256) return group_size > 0 ? XFP_ERR_UNSUPPORTED : XFP_ERR_SHAPE;
+    if (cols % group_size) return XFP_ERR_SHAPE;
+    const int64_t groups = (int64_t)rows * (cols / group_size);
     if (groups > 0x7fffffff) return XFP_ERR_UNSUPPORTED;
     const int gpb = L <= 32 ? 4 : (L <= 64 ? 2 : 1);
-    libfit_group_kernel<<<(unsigned)((groups + gpb - 1) / gpb), 128, 0, (cudaStream_t)stream>>>(
-        W, mask, mu_sigma, groups, bits, L, gpb, lib, idx, gid, gscale, gmid);
+    const unsigned grid = (unsigned)((groups + gpb - 1) / gpb);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (group_size == 64)
+        libfit_group_kernel<64><<<grid, 64, 0, s>>>(W, mask, mu_sigma, groups, bits, L, gpb, lib, idx, gid, gscale, gmid);
+    else if (group_size == 128)
+        libfit_group_kernel<128><<<grid, 128, 0, s>>>(W, mask, mu_sigma, groups, bits, L, gpb, lib, idx, gid, gscale, gmid);
+    else
+        libfit_group_kernel<256><<<grid, 256, 0, s>>>(W, mask, mu_sigma, groups, bits, L, gpb, lib, idx, gid, gscale, gmid);
     return cudaGetLastError() == cudaSuccess ? XFP_OK : XFP_ERR_CUDA;
 }
 
@@ -1366,7 +1378,10 @@ int xfp_quantize(int32_t mode, const float* W, int32_t rows, int32_t cols, const
     if (host_cnt > capacity) return XFP_ERR_BUFFER_TOO_SMALL;
 
     xfp_desc d;
-    d.mode = mode; d.rows = rows; d.cols = cols; d.group_size = 128; d.lib_size = mode ? lib_size : 0;
+    d.mode = mode; d.rows = rows; d.cols = cols; d.group_size = p->group_size ? p->group_size : 128;
+    d.lib_size = mode ? lib_size : 0;
+    if (d.group_size != 64 && d.group_size != 128 && d.group_size != 256) return d.group_size > 0 ? XFP_ERR_UNSUPPORTED : XFP_ERR_SHAPE;
+    if (cols % d.group_size) return XFP_ERR_SHAPE;
     d.col_bits = 32; d.nnz = host_cnt;
     result->mu = host_ms[0]; result->sigma = host_ms[1]; result->nnz = host_cnt;
     result->fallback = 1; result->tried = 0; result->reserved = 0;
@@ -1378,7 +1393,8 @@ int xfp_quantize(int32_t mode, const float* W, int32_t rows, int32_t cols, const
         if (mode == 1) {
             st = xfp_quant_libfit_library(codebook, rows, d.bits, lib_size, p->lloyd_iters, lib, workspace, need, stream);
             if (st) return st;
-            st = xfp_quant_libfit_assign(W, mask, ms, rows, cols, d.bits, lib_size, lib, idx, gid, gscale, gmid, stream);
+            st = xfp_quant_libfit_assign(W, mask, ms, rows, cols, d.bits, lib_size, d.group_size, lib, idx, gid, gscale, gmid,
+                                         stream);
             if (st) return st;
             table = lib;
         }

@@ -20,7 +20,7 @@ QUANT_EXPORTS = ("xfp_quant_workspace_size", "xfp_quant_stats", "xfp_quant_outli
 class XfpQuantParams(C.Structure):
     """Mirror of xfp_quant_params."""
     _fields_ = [("sigma_mode", C.c_int32), ("outlier_mode", C.c_int32), ("k_sigma", C.c_double),
-                ("cap_frac", C.c_double), ("rate", C.c_double), ("lloyd_iters", C.c_int32), ("reserved", C.c_int32)]
+                ("cap_frac", C.c_double), ("rate", C.c_double), ("lloyd_iters", C.c_int32), ("group_size", C.c_int32)]
 
 
 class XfpQuantResult(C.Structure):
@@ -43,7 +43,7 @@ def _lib():
         lib.xfp_quant_outliers.argtypes = [vp, i64, vp, i32, f64, f64, vp, vp, vp, sz, vp]
         lib.xfp_quant_lloyd.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         lib.xfp_quant_libfit_library.argtypes = [vp, i32, i32, i32, i32, vp, vp, sz, vp]
-        lib.xfp_quant_libfit_assign.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        lib.xfp_quant_libfit_assign.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.xfp_quant_residual.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
         lib.xfp_quant_cosine.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.xfp_quant_median.argtypes = [vp, i64, vp, vp, sz, vp]
@@ -92,10 +92,11 @@ def xfp_quant_libfit_library(codebook, rows: int, bits: int, L: int, iters: int,
            "xfp_quant_libfit_library")
 
 
-def xfp_quant_libfit_assign(W, mask, mu_sigma, bits: int, L: int, lib, idx, gid, gscale, gmid, stream=None) -> None:
+def xfp_quant_libfit_assign(W, mask, mu_sigma, bits: int, L: int, lib, idx, gid, gscale, gmid, stream=None,
+                            group_size: int = 128) -> None:
     rows, cols = W.shape
     _check(_lib().xfp_quant_libfit_assign(_ptr(W), _ptr(mask), _ptr(mu_sigma), rows, cols, int(bits), int(L),
-                                          _ptr(lib), _ptr(idx), _ptr(gid), _ptr(gscale), _ptr(gmid),
+                                          int(group_size), _ptr(lib), _ptr(idx), _ptr(gid), _ptr(gscale), _ptr(gmid),
                                           _stream(stream)), "xfp_quant_libfit_assign")
 
 
@@ -121,8 +122,10 @@ def xfp_quant_median(v, median, workspace, stream=None) -> None:
 class QuantBuffers:
     """Device buffers xfp_quantize writes, sized for a rows x cols matrix (allocation only)."""
 
-    def __init__(self, rows: int, cols: int, mode: int, max_bits: int, lib_size: int, capacity: int, device="cuda"):
-        G = cols // 128
+    def __init__(self, rows: int, cols: int, mode: int, max_bits: int, lib_size: int, capacity: int, device="cuda",
+                 group_size: int = 128):
+        G = cols // group_size
+        self.group_size = group_size
         e = torch.empty
         self.rows, self.cols, self.mode, self.lib_size = rows, cols, mode, lib_size
         self.mask = e((rows, cols), dtype=torch.uint8, device=device)
@@ -163,10 +166,12 @@ def quantize_and_pack(W: torch.Tensor, mode: int, candidates: Sequence[int], tau
         params = XfpQuantParams(0, 0, 4.0, 0.02, 0.0, 20, 0)      # the paper's defaults: k = 4, cap 2 %, 20 rounds
     rows, cols = W.shape
     frac = params.rate if params.outlier_mode else params.cap_frac
-    buf = QuantBuffers(rows, cols, mode, max(candidates), lib_size, int(frac * rows * cols), device=W.device)
+    group = params.group_size or 128
+    buf = QuantBuffers(rows, cols, mode, max(candidates), lib_size, int(frac * rows * cols), device=W.device,
+                       group_size=group)
     res = xfp_quantize(mode, W, params, candidates, tau, buf, stream)
     E = 1 << res.bits
-    desc = XfpDesc(mode, rows, cols, res.bits, 128, lib_size if mode else 0, 32, int(res.nnz))
+    desc = XfpDesc(mode, rows, cols, res.bits, group, lib_size if mode else 0, 32, int(res.nnz))
     pb, wb = xfp_packed_size(desc)
     packed = torch.empty(pb, dtype=torch.uint8, device=W.device)
     workspace = torch.zeros(max(wb, 16), dtype=torch.uint8, device=W.device)
@@ -179,7 +184,7 @@ def quantize_and_pack(W: torch.Tensor, mode: int, candidates: Sequence[int], tau
 def _pack_buffers(buf: QuantBuffers, mode: int, bits: int, lib_size: int, nnz: int, table: torch.Tensor, stream=None):
     """xfp_pack on the tensors an encoder call left in `buf` (allocation and marshalling only)."""
     from .binding import PackedMatrix, xfp_pack, xfp_packed_size
-    desc = XfpDesc(mode, buf.rows, buf.cols, bits, 128, lib_size if mode else 0, 32, int(nnz))
+    desc = XfpDesc(mode, buf.rows, buf.cols, bits, buf.group_size, lib_size if mode else 0, 32, int(nnz))
     pb, wb = xfp_packed_size(desc)
     dev = buf.idx.device
     packed = torch.empty(pb, dtype=torch.uint8, device=dev)
@@ -201,11 +206,12 @@ def quantize_with_library(W: torch.Tensor, bits: int, lib: torch.Tensor, params:
     xfp_quant_stats(W, params.sigma_mode, ms, buf.workspace, stream)
     xfp_quant_outliers(W, ms, params.outlier_mode, params.rate if params.outlier_mode else params.k_sigma,
                        params.cap_frac, buf.mask, count, buf.workspace, stream)
-    xfp_quant_libfit_assign(W, buf.mask, ms, bits, L, lib, buf.idx, buf.gid, buf.gscale, buf.gmid, stream)
+    xfp_quant_libfit_assign(W, buf.mask, ms, bits, L, lib, buf.idx, buf.gid, buf.gscale, buf.gmid, stream,
+                            group_size=buf.group_size)
     nnz = int(count.item())          # one read-back, as in xfp_quantize: the outlier arrays must hold them all
     if nnz > buf.capacity:
         raise XfpError(f"quantize_with_library: {nnz} extracted weights, buffers hold {buf.capacity}")
-    desc = XfpDesc(1, rows, cols, bits, 128, L, 32, nnz)
+    desc = XfpDesc(1, rows, cols, bits, buf.group_size, L, 32, nnz)
     xfp_quant_residual(desc, W, buf.mask, buf.idx, lib, buf.gid, buf.gscale, buf.gmid, buf.rowptr, buf.ocol, buf.oval,
                        buf.workspace, stream)
     return nnz
@@ -224,14 +230,16 @@ def quantize_moe_layer(experts: Sequence[torch.Tensor], mode: int, candidates: S
     frac = params.rate if params.outlier_mode else params.cap_frac
     stacked = torch.cat([experts[i] for i in sample], dim=0).contiguous()
     rows_s, cols = stacked.shape
-    sbuf = QuantBuffers(rows_s, cols, mode, max(candidates), lib_size, int(frac * rows_s * cols), device=stacked.device)
+    group = params.group_size or 128
+    sbuf = QuantBuffers(rows_s, cols, mode, max(candidates), lib_size, int(frac * rows_s * cols), device=stacked.device,
+                        group_size=group)
     res = xfp_quantize(mode, stacked, params, candidates, tau, sbuf, stream)
     bits, E = int(res.bits), 1 << int(res.bits)
     lib = sbuf.lib.view(-1)[:lib_size * E].clone().view(lib_size, E) if mode else None
     out = []
     for W in experts:
         rows = W.shape[0]
-        buf = QuantBuffers(rows, cols, mode, bits, lib_size, int(frac * rows * cols), device=W.device)
+        buf = QuantBuffers(rows, cols, mode, bits, lib_size, int(frac * rows * cols), device=W.device, group_size=group)
         if mode:
             nnz = quantize_with_library(W, bits, lib, params, buf, stream)
             out.append(_pack_buffers(buf, 1, bits, lib_size, nnz, lib.view(-1), stream))

@@ -66,7 +66,9 @@ def test_encoder_rejects_bad_arguments_on_the_host(lib):
     assert lib.xfp_quant_lloyd(a, odd, a, 64, 256, 4, 20, a, a, n, 0, n) == 2
     assert lib.xfp_quant_libfit_library(a, 64, 4, 0, 20, a, a, big, n) == 3
     assert lib.xfp_quant_libfit_library(a, 64, 4, 32, 20, a, a, 64, n) == 5
-    assert lib.xfp_quant_libfit_assign(a, n, a, 64, 256, 4, 32, a, a, n, a, a, n) == 1
+    assert lib.xfp_quant_libfit_assign(a, n, a, 64, 256, 4, 32, 128, a, a, n, a, a, n) == 1
+    assert lib.xfp_quant_libfit_assign(a, n, a, 64, 256, 4, 32, 80, a, a, a, a, a, n) == 4      # group sizes: 64, 128, 256
+    assert lib.xfp_quant_libfit_assign(a, n, a, 64, 384, 4, 32, 256, a, a, a, a, a, n) == 3     # cols % group_size
     d = _desc(mode=1, lib_size=32)
     assert lib.xfp_quant_residual(C.byref(d), a, a, a, a, n, n, n, a, a, a, 10, a, big, n) == 1   # V2a needs group data
     d0 = _desc()

@@ -160,19 +160,21 @@ def test_libfit_library_is_bit_exact(bits, L, rows):
     assert np.array_equal(_u16(lib), want)
 
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 5])
-def test_libfit_assign_is_bit_exact(bits):
-    rows, cols, L = 48, 640, 32
+@pytest.mark.parametrize("bits,group", [(2, 128), (3, 128), (4, 128), (5, 128), (3, 64), (4, 256), (6, 64), (2, 256)])
+def test_libfit_assign_is_bit_exact(bits, group):
+    """Group assignment at the paper's group size and at the other two the format carries (64, 256)."""
+    rows, cols, L = 48, 768, 32
     W = _weights(rows, cols, 50 + bits)
-    W[3, 128:256] = 0.0625        # a constant group
+    W[3, 256:512] = 0.0625        # constant groups at every group size
     mask, mu, _ = xo.outlier_mask(W)
-    m = xo.quantize_v2a(W, bits, mask, mu, L, 20)
-    G = cols // 128
+    m = xo.quantize_v2a(W, bits, mask, mu, L, 20, group=group)
+    G = cols // group
     idx = torch.full((rows, cols), 255, dtype=torch.uint8, device="cuda")
     gid = torch.full((rows, G), 255, dtype=torch.uint8, device="cuda")
     gs = torch.zeros((rows, G), dtype=torch.int16, device="cuda")
     gm = torch.zeros((rows, G), dtype=torch.int16, device="cuda")
-    qb.xfp_quant_libfit_assign(_dev(W), _dev(mask), _ms(mu, 0.0), bits, L, _dev(m.codebook), idx, gid, gs, gm)
+    qb.xfp_quant_libfit_assign(_dev(W), _dev(mask), _ms(mu, 0.0), bits, L, _dev(m.codebook), idx, gid, gs, gm,
+                               group_size=group)
     torch.cuda.synchronize()
     assert np.array_equal(gid.cpu().numpy(), m.gid)
     assert np.array_equal(_u16(gs), m.gscale)
@@ -318,6 +320,22 @@ def test_moe_sampling_layer_matches_the_oracle(mode, cands, tau):
         y = pm.gemv(xd)
         torch.cuda.synchronize()
         assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - yref) <= 1e-3 * absum + 1e-30)
+
+
+@pytest.mark.parametrize("group,cands", [(64, (2, 4)), (256, (3,))])
+def test_auto_select_at_other_group_sizes(group, cands):
+    """Algorithm 1 for V2a with 64 and 256 weights per group: same width and tensors as the oracle, and the packed blob
+    reconstructs to the oracle's matrix bit for bit."""
+    rows, cols, L = 96, 1024, 32
+    W = synth.plant_uniform_outliers(synth.gaussian_weights(rows, cols, 75), 0.005, 76)
+    ref = xo.auto_select(W, "moe_routed", cands, tau_lazy=0.93, mode=1, iters=20, lib_size=L, group=group)
+    params = _params()
+    params.group_size = group
+    pm, res = qb.quantize_and_pack(_dev(W), 1, cands, 0.93, params, lib_size=L)
+    torch.cuda.synchronize()
+    assert res.bits == ref.bits and int(res.nnz) == ref.nnz and abs(res.median_cos - ref.info["median_cos"]) <= 1e-12
+    assert pm.desc.group_size == group and int(pm.err_word.item()) == 0
+    assert np.array_equal(_u16(pm.dequant().view(torch.int16)), xo.dequant(ref))
 
 
 def test_quantize_reports_a_small_outlier_buffer():
