@@ -7,7 +7,7 @@
  * Two codebook storage modes ("The XFP Format"):
  *   V2  : one fp16 codebook of 2^N entries per output channel:  D_ik = codebook_i[q_ik]
  *   V2a : a per-layer library of L codebooks; every group of G consecutive k of one channel (G = 128 in the
- *         paper, "a tunable parameter": 64, 128 and 256 are built) carries a library id, an fp16 scale and an
+ *         paper, which leaves the size open: 64, 128 and 256 are built) carries a library id, an fp16 scale and an
  *         fp16 mid-point ("V2a: Shared Codebook Library"):  D_ik = mid_ig + scale_ig * lib[id_ig][q_ik],  g = k / G
  * The hot path is the fused decode kernel y = (D + S) x of "Fused Decode Kernel": depack, codebook
  * gather, outlier add and multiply-accumulate in one launch, fp32 accumulation.

@@ -40,7 +40,7 @@ typedef struct {
     double rate;          /* outlier_mode 1 only                                                      */
     int32_t lloyd_iters;  /* rounds of Lloyd (paper: 20; its V2 default elsewhere: 5)                 */
     int32_t group_size;   /* V2a: weights per (id, scale, mid) group: 64, 128 or 256; 0 means 128, the paper's
-                             default ("a tunable parameter")                                          */
+                             default (the paper leaves the size open)                                 */
 } xfp_quant_params;
 
 typedef struct {
