@@ -232,6 +232,10 @@ EXTRA_CONFIGS = (
     ("config5_8192x8192_v2a_n4", "shape:1:8192:8192:4:0.003"),
     ("config5_28672x8192_v2_n4", "shape:0:28672:8192:4:0.003"),
     ("config5_28672x8192_v2a_n4", "shape:1:28672:8192:4:0.003"),
+    # the batch axis of configuration 5: 8 rows of x (the other batch sizes: `--workload shape:...:BATCH`)
+    ("config5_8192x8192_v2_n4_batch8", "shape:0:8192:8192:4:0.003:8"),
+    ("config5_28672x8192_v2_n4_batch8", "shape:0:28672:8192:4:0.003:8"),
+    ("config5_28672x8192_v2a_n4_batch8", "shape:1:28672:8192:4:0.003:8"),
 )
 
 

@@ -21,7 +21,7 @@
 //   N = 5   pair table, 1024 entries (128 KB, one CTA per SM) or, beyond one round of CTAs, one entry per index
 //   N = 6   one entry per index (a pair table would need 16 KB per channel), two look-ups joined by a PRMT
 // V2a: the library replicated once per bank -- pair tables of every entry where L * 4^N words fit (N = 2 at L = 32),
-// one word per entry otherwise, half a word at N = 6 -- see the kernel's comment.
+// otherwise one entry per index with the entries of two library ids sharing a word -- see the kernel's comment.
 //
 // x is staged once per CTA in shared memory in an order that lets a diagonal lane fetch the B registers of TWO
 // mma steps with one 16-byte load: inside every group of 16 k the two middle blocks of four are swapped
@@ -133,10 +133,7 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
         const bool two = lane_tab_bytes(l, !pairs) <= 64 * 1024 && RB > sms;
         LaneConfig c{two ? 8 : 16, two ? 2 : 1, !pairs};
         c.tiers = RB > 4 * sms || !two;
-        // a 128 KB library (N = 5) leaves one CTA per SM: between one and four rounds the kernel with two channels
-        // per lane (xfp_gemv_v2a.cu) measured faster
-        const bool half_words = (size_t)l.L * l.E * 128 > 128 * 1024;   // no kernel with two channels per lane for these
-        c.off = !two && !half_words && RB > sms && RB <= 4 * sms;
+        c.off = false;
         // the blobs of a routed layer in one launch: the resident CTAs of xfp_gemv_v2a.cu (pair tables built once per
         // SM at N <= 3) measured faster (gate_up 30.7 vs 33.4 us, down 18.7 vs 22.9 us per launch of 8 experts)
         if (n > 1) c.off = true;
@@ -170,7 +167,7 @@ bool lane_supported(const Layout& l, const GemvCall& c) {
     if (c.batch != 1 || c.n < 1 || c.epilogue != 0) return false;
     if ((c.n > 1) != (c.packed_list != nullptr)) return false;
     if (l.bits < 2 || l.bits > 6) return false;
-    if (l.mode && (size_t)l.L * l.E * 64 > 128 * 1024) return false;   // V2a: the per-bank library must fit 128 KB
+    if (l.mode && (size_t)((l.L + 1) / 2) * l.E * 128 > 128 * 1024) return false;   // V2a: the per-bank library must fit 128 KB
     const LaneConfig cfg = lane_config(l, c.n);
     if (cfg.off) return false;
     return lane_smem_bytes(l, cfg) <= (cfg.per_sm == 1 ? 220u : 110u) * 1024u;
@@ -187,16 +184,6 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
     if (g_lane_trace && g_lane_trace_idx < g_lane_trace_calls) a.trace = g_lane_trace + (g_lane_trace_idx++) * 1024 * 8;
 #endif
     const size_t smem = lane_smem_bytes(l, cfg);
-    if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) {
-        // two bytes per lane and entry (lanes 2j and 2j+1 share a bank: a look-up costs two wavefronts when their
-        // entries differ): N = 6 with L = 32, which the paper's own V2a kernel does not have
-        switch (l.bits) {
-            case 4: return launch_lane<4, 16, 1, true, 2>(a, sch.grid, smem, s);
-            case 5: return launch_lane<5, 16, 1, true, 2>(a, sch.grid, smem, s);
-            case 6: return launch_lane<6, 16, 1, true, 2>(a, sch.grid, smem, s);
-            default: return cudaErrorInvalidValue;
-        }
-    }
     if (l.mode) {
         switch (l.bits) {
             case 2: return cfg.sgl ? launch_lane_cfg<2, true, 1>(cfg, a, sch.grid, smem, s)
@@ -204,7 +191,8 @@ cudaError_t launch_gemv_lane(const Layout& l, const GemvCall& c, cudaStream_t s)
             case 3: return cfg.sgl ? launch_lane_cfg<3, true, 1>(cfg, a, sch.grid, smem, s)
                                    : launch_lane_cfg<3, false, 1>(cfg, a, sch.grid, smem, s);
             case 4: return launch_lane_cfg<4, true, 1>(cfg, a, sch.grid, smem, s);
-            default: return launch_lane_cfg<5, true, 1>(cfg, a, sch.grid, smem, s);
+            case 5: return launch_lane_cfg<5, true, 1>(cfg, a, sch.grid, smem, s);
+            default: return launch_lane_cfg<6, true, 1>(cfg, a, sch.grid, smem, s);
         }
     }
     switch (l.bits) {

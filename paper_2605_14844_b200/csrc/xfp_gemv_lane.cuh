@@ -78,30 +78,15 @@ struct LaneCfg {
     static constexpr int kTabBytes = T * kStride;
 };
 
-// Byte offset (q << 6) of index j (compile time) merged with `base`, for tables whose entries are 64 bytes apart
-// (two bytes per lane).
-template <int N>
-__device__ __forceinline__ uint32_t half_addr(const uint32_t* w, int j, uint32_t base) {
-    constexpr uint32_t mask = ((1u << N) - 1u) << 6;
-    const int bit = j * N, wi = bit >> 5, off = bit & 31;
-    uint32_t v;
-    if (off + N > 32)
-        v = __funnelshift_r(w[wi], w[wi + 1], off - 6);
-    else if (off >= 6)
-        v = w[wi] >> (off - 6);
-    else
-        v = w[wi] << (6 - off);
-    return (v & mask) | base;
-}
-
 // The four A registers of mma step j (weights 8j .. 8j+7 of the lane's channel in this super-chunk).
 template <int N, bool SGL, bool HALF, bool QUAD>
 __device__ __forceinline__ void lookup8(uint32_t (&f)[4], const uint32_t* w, int j, const unsigned char* tab,
                                         uint32_t base) {
     if (HALF) {
+        // V2a, one entry per index: a word holds the entry of TWO library ids, `base` selects the half
         uint32_t e[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) e[i] = *(const uint16_t*)(tab + half_addr<N>(w, 8 * j + i, base));
+        for (int i = 0; i < 8; ++i) e[i] = *(const uint16_t*)(tab + single_addr<N, 1>(w, 8 * j + i, base));
         f[0] = __byte_perm(e[0], e[1], 0x5410);
         f[2] = __byte_perm(e[2], e[3], 0x5410);
         f[1] = __byte_perm(e[4], e[5], 0x5410);
@@ -138,7 +123,8 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
 }
 
 // MODE 0: V2 (the channel's own codebook, tables private to the lane).  MODE 1: V2a -- the whole library replicated
-// once per bank (word (id * 2^N + q) * 32 + lane holds lib[id][q]), the table base of a lane follows the library id
+// once per bank (word ((id / 2) * 2^N + q) * 32 + lane holds lib[id][q] in its half id % 2; pair tables of every
+// entry where those fit), the table base of a lane follows the library id
 // of its channel's current group, the fragment accumulates sum lib * x of ONE group, and after the group's steps the
 // sum moves to the lane that owns the channel and is folded into its accumulator with the group's scale and
 // mid-point:  acc += scale * G + mid * X_g,  X_g = sum of x over the group ("V2a: Shared Codebook Library").
@@ -149,13 +135,15 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
 template <int N, int W, int MINB, bool SGL, int MODE, bool TIO, int NB>
 __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs a) {
     using C = LaneCfg<N, SGL, MODE>;
-    constexpr bool kHalf = MODE == 2;   // V2a with a library too large for one 4-byte word per bank and entry
-    constexpr int kEntry = kHalf ? 64 : 128;   // V2a: bytes between library entries
     constexpr int E = C::E;
     // V2a with a small library (L * 4^N words per bank fit): PAIR tables of every library entry, one look-up per two
     // weights as in V2
     constexpr bool kLibPair = MODE == 1 && !SGL;
-    constexpr int kIdBytes = (kLibPair ? E * E : E) * kEntry;   // V2a: bytes between the tables of two library entries
+    // V2a otherwise: one entry per index, and the word of a bank holds that entry of TWO library ids (2m in the low
+    // half, 2m + 1 in the high half): every lane still reads its own bank, whatever ids and indices the lanes hold,
+    // and the tables are half as large (64 KB at N = 5, 128 KB at N = 6 with L = 32)
+    constexpr bool kHalf = MODE == 1 && SGL;
+    constexpr int kIdBytes = (kLibPair ? E * E : E) * 128;   // V2a: bytes between the tables of two ids (kHalf: id pairs)
     constexpr int T = C::T;
     constexpr int kStride = C::kStride;
     constexpr int kThreads = W * 32;
@@ -176,9 +164,13 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     uint32_t* cbs = (uint32_t*)xg;                 // V2 pair tables: the block's codebooks, word [e / 2][channel]
     const int g = lane >> 2, t4 = lane & 3;
     const bool dq = (g == t4) || (g == t4 + 4);
-    const uint32_t base = (uint32_t)lane * (C::kQuad ? 8u : (kHalf ? 2u : 4u));
+    const uint32_t base = (uint32_t)lane * (C::kQuad ? 8u : 4u);
     // V2a: where the two halves of this lane's group sum land in the fragment (see the end of the kernel)
     const int src_a = (lane & ~3) | (t4 >> 1);
+    // V2a: table offset of library id `id`
+    auto id_offset = [](uint32_t id) -> uint32_t {
+        return kHalf ? (id >> 1) * (uint32_t)kIdBytes + (id & 1u) * 2u : id * (uint32_t)kIdBytes;
+    };
 
 #pragma unroll 1
     for (int it = 0;; ++it) {
@@ -261,14 +253,17 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     if (MODE != 0) {
         if (!kMulti || it == 0) {   // one library per blob: a resident CTA fills it once
         if (kHalf) {
-            for (int e = warp; e < a.L * E; e += W) *(uint16_t*)(tab + (size_t)e * 64 + lane * 2) = __ldg(b.cb + e);
+            for (int e = warp; e < ((a.L + 1) >> 1) * E; e += W) {
+                const int m = e >> N, q = e & (E - 1);
+                const uint32_t lo = __ldg(b.cb + (size_t)(2 * m) * E + q);
+                const uint32_t hi = 2 * m + 1 < a.L ? (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) : 0u;
+                *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = lo | (hi << 16);
+            }
         } else if (kLibPair) {
             for (int e = warp; e < a.L * E * E; e += W) {
                 const uint16_t* cb = b.cb + (size_t)(e >> (2 * N)) * E;
                 *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(cb + (e & (E - 1))) | ((uint32_t)__ldg(cb + ((e >> N) & (E - 1))) << 16);
             }
-        } else {
-            for (int e = warp; e < a.L * E; e += W) *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
         }
         }
     } else {
@@ -430,7 +425,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         for (int r = 0; r < RH; ++r) xr[r] = make_uint4(0u, 0u, 0u, 0u);
         uint32_t vbase = base;
         if (MODE != 0) {
-            vbase = base + gid_c[0] * (uint32_t)kIdBytes;
+            vbase = base + id_offset(gid_c[0]);
             if (has_next) {   // metadata of the next super-chunk travels during this one
                 const size_t mn = m0 + (size_t)(s + W) * GH * 32;
                 gid_n[0] = b.gid[mn]; gsm_n[0] = b.gsm[mn];
@@ -469,7 +464,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             if (NB <= RH) {
 #pragma unroll
                 for (int r = 0; r < NB; ++r) mma16816(c[r], fa[0], fa[1], fa[2], fa[3], xr[r].x, xr[r].y);
-                if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)kIdBytes;   // second half's library entry
+                if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + id_offset(gid_c[1]);   // second half's library entry
                 if (j + 2 < kSuper / 8) lookup8<N, SGL, kHalf, C::kQuad>(fa, w, j + 2, tab, vbase);
 #pragma unroll
                 for (int r = 0; r < NB; ++r) mma16816(c[r], fb[0], fb[1], fb[2], fb[3], xr[r].z, xr[r].w);
@@ -481,7 +476,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
 #pragma unroll
                     for (int r = 0; r < RH; ++r) ld_x16_if(xr[r], xp + (h * RH + r) * xrow + j * 16, dq);
                     if (h == NB / RH - 1) {
-                        if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + gid_c[1] * (uint32_t)kIdBytes;
+                        if (MODE != 0 && j + 2 == kSuper / 16) vbase = base + id_offset(gid_c[1]);
                         if (j + 2 < kSuper / 8) lookup8<N, SGL, kHalf, C::kQuad>(fn, w, j + 2, tab, vbase);
                     }
 #pragma unroll
@@ -598,8 +593,7 @@ inline size_t lane_tab_bytes(const Layout& l, bool sgl) {
     const size_t E = (size_t)1 << bits;
     if (l.mode) {   // the library, one copy per bank: a word per entry (per pair of entries), or half a word when that does not fit
         if (!sgl) return (size_t)l.L * E * E * 128;
-        const size_t full = (size_t)l.L * E * 128;
-        return full <= 128 * 1024 ? full : full / 2;
+        return (size_t)((l.L + 1) / 2) * E * 128;   // a word holds one entry of two library ids
     }
     if (bits == 2) return 256 * 256;
     if (sgl) return E * 128;

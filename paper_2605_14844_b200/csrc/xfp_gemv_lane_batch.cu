@@ -35,9 +35,8 @@ bool batch_plan(const Layout& l, int rows_x, BatchPlan& p) {
     const int sms = sched_sms();
     if (l.RB * 2 <= sms) return false;   // tiny matrices cut every block along K: the kernels with clusters do that
     bool sgl;
-    const bool half_words = l.mode && (size_t)l.L * l.E * 128 > 128 * 1024;   // two bytes per bank and library entry
     if (l.mode) {
-        if ((size_t)l.L * l.E * 64 > 128 * 1024) return false;
+        if ((size_t)((l.L + 1) / 2) * l.E * 128 > 128 * 1024) return false;
         sgl = !((size_t)l.L * l.E * l.E * 128 <= 64 * 1024 && l.bits <= 3);
     } else {
         sgl = l.bits >= 5;   // the 128 KB pair table of N = 5 leaves no room for several rows of x
@@ -45,7 +44,7 @@ bool batch_plan(const Layout& l, int rows_x, BatchPlan& p) {
     for (int nb = 8; nb >= 2; nb /= 2) {
         if (nb >= 2 * rows_x && nb > 2) continue;   // a smaller tile holds the rows
         LaneConfig two{8, 2, sgl}, one{16, 1, sgl};
-        if (!half_words && l.RB > sms && lane_smem_bytes(l, two, nb) <= 110u * 1024u) {
+        if (l.RB > sms && lane_smem_bytes(l, two, nb) <= 110u * 1024u) {
             p = BatchPlan{nb, two, lane_smem_bytes(l, two, nb)};
             return true;
         }
@@ -93,7 +92,7 @@ static bool lane_batch_preferred(const Layout& l, int batch) {
         if (l.bits >= 5) return !(small && batch == 2);
         return small && batch >= 3;
     }
-    if ((size_t)l.L * l.E * 128 > 128 * 1024) return true;   // half-word libraries: the other kernel is the general one
+    if ((size_t)l.L * l.E * 128 > 128 * 1024) return true;   // libraries of more than 128 KB a word per entry (N = 6): the other kernel is the general one
     if (small) return true;
     if (l.bits == 3) return batch >= 3 && l.RB > 4 * sms;
     if (l.bits >= 4 && l.RB <= 2 * sms) return batch == 2;
@@ -151,19 +150,13 @@ cudaError_t launch_gemv_lane_batch(const Layout& l, const GemvCall& c, cudaStrea
         a.tier_spp[0] = spp;
         a.tier_cta[1] = tail * a.tier_kst[0];
         cudaError_t e;
-        if (l.mode && (size_t)l.L * l.E * 128 > 128 * 1024) {
-            switch (l.bits) {
-                case 4: e = launch_tile<4, true, 2>(p, a, G, s); break;
-                case 5: e = launch_tile<5, true, 2>(p, a, G, s); break;
-                case 6: e = launch_tile<6, true, 2>(p, a, G, s); break;
-                default: e = cudaErrorInvalidValue; break;
-            }
-        } else if (l.mode) {
+        if (l.mode) {
             switch (l.bits) {
                 case 2: e = p.cfg.sgl ? launch_tile<2, true, 1>(p, a, G, s) : launch_tile<2, false, 1>(p, a, G, s); break;
                 case 3: e = p.cfg.sgl ? launch_tile<3, true, 1>(p, a, G, s) : launch_tile<3, false, 1>(p, a, G, s); break;
                 case 4: e = launch_tile<4, true, 1>(p, a, G, s); break;
-                default: e = launch_tile<5, true, 1>(p, a, G, s); break;
+                case 5: e = launch_tile<5, true, 1>(p, a, G, s); break;
+                default: e = launch_tile<6, true, 1>(p, a, G, s); break;
             }
         } else {
             switch (l.bits) {
