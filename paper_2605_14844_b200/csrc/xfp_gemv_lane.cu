@@ -112,10 +112,11 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
     const long long RB = (long long)l.RB * n;
 #ifdef LANE_TUNE
     if (const char* e = getenv("XFP_LANE_CFG")) {   // tuning build: "W,per_sm,sgl"
-        int w = 16, p = 1, g = 0;
-        sscanf(e, "%d,%d,%d", &w, &p, &g);
+        int w = 16, p = 1, g = 0, t = -1;
+        sscanf(e, "%d,%d,%d,%d", &w, &p, &g, &t);
         if (w == 0) return LaneConfig{16, 1, false, true};
-        return LaneConfig{w, p > 2 ? 2 : p, l.mode == 1 || l.bits == 6 || (l.bits == 5 && g), false, p <= 2};
+        const bool pairs = l.mode == 1 && (size_t)l.L * l.E * l.E * 128 <= 64 * 1024 && l.bits <= 3;
+        return LaneConfig{w, p > 2 ? 2 : p, l.mode == 1 ? !pairs : (l.bits == 6 || (l.bits == 5 && g)), false, t < 0 ? p <= 2 : t != 0};
     }
 #endif
     // Measured on B200 over 4096 x 4096 .. 28672 x 8192 at every bit width (microseconds per call, graph replay):
@@ -132,7 +133,7 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
         const bool pairs = (size_t)l.L * l.E * l.E * 128 <= 64 * 1024 && l.bits <= 3;
         const bool two = lane_tab_bytes(l, !pairs) <= 64 * 1024 && RB > sms;
         LaneConfig c{two ? 8 : 16, two ? 2 : 1, !pairs};
-        c.tiers = RB > 4 * sms || !two;
+        c.tiers = RB > 4 * sms;   // up to four rounds unsplit, as in V2 (N = 6, one CTA per SM: 12288 x 4096 33.6 -> 26.6 us)
         c.off = false;
         // the blobs of a routed layer in one launch: the resident CTAs of xfp_gemv_v2a.cu (pair tables built once per
         // SM at N <= 3) measured faster (gate_up 30.7 vs 33.4 us, down 18.7 vs 22.9 us per launch of 8 experts)
