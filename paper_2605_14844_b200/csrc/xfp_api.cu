@@ -1,4 +1,6 @@
 // extern "C" boundary of libxfp: host-side validation, layout computation, kernel selection.
+#include <cstdlib>
+
 #include "../../include/xfp.h"
 #include "xfp_internal.h"
 
@@ -78,7 +80,11 @@ int gemv_common(const xfp_desc* desc, int want_mode, const GemvCall& c, void* st
         e = launch_gemv_lane(l, cc, (cudaStream_t)stream);
     else if (lane_batch_supported(l, cc))
         e = launch_gemv_lane_batch(l, cc, (cudaStream_t)stream);
-    else if (!c.packed_list && !c.x_bf16 && batch_prefers_gemm(l, c.batch)) {
+    else if (!c.packed_list && !c.x_bf16 && batch_prefers_gemm(l, c.batch)
+#ifdef LANE_TUNE
+             && !getenv("XFP_NO_GEMM")   // tuning build: keep batches off the tensor-core kernel
+#endif
+    ) {
         // many rows of x, few outliers: one decode for all rows on the tensor cores (y = x W^T with W the matrix
         // xfp_dequant writes; inside the GEMV's bound)
         GemmCall g{c.packed, c.x, c.y, c.batch, c.y_is_fp16, c.workspace, need};

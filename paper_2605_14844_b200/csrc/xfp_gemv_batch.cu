@@ -39,10 +39,13 @@ struct BatchArgs {
     int n_full, kst, sc_per_split;
 };
 
-// byte offset of x[bb][k] in the staged copy: chunk (k / 8) * NB + bb, 8 halves per chunk
+// byte offset of x[bb][k] in the staged copy: chunk (k / 8) * NB + (bb ^ (k / 8 mod NB)), 8 halves per chunk.  The
+// swizzle of the row inside a chunk group lets eight consecutive lanes stage eight consecutive chunks of ONE row
+// (one 128-byte line per quarter-warp instead of eight) without meeting in the same banks when they store.
 template <int NB>
 __device__ __forceinline__ uint32_t xoff(int bb, uint32_t k) {
-    return (((k >> 3) * NB + (uint32_t)bb) << 4) + ((k & 7u) << 1);
+    const uint32_t k8 = k >> 3;
+    return ((k8 * NB + ((uint32_t)bb ^ (k8 & (uint32_t)(NB - 1)))) << 4) + ((k & 7u) << 1);
 }
 
 // Byte offset (q << 7) of index j (compile time) of a 128-weight stream, merged with `base`
@@ -201,11 +204,12 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
     // ---- (2) x: chunk t = (k / 8) * NB + bb  <-  x[bb][8 (k/8) .. +8]
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int t = threadIdx.x; t < NB * (K / 8); t += kBThreads) {
-        const int k8 = t / NB, bb = t - k8 * NB;
+        // eight consecutive lanes: eight consecutive chunks of one row (K / 8 is a multiple of 16)
+        const int grp = t >> 3, bb = grp % NB, k8 = (grp / NB) * 8 + (t & 7);
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (bb < a.nb) v = __ldg((const uint4*)(a.x + (size_t)bb * a.cols + (size_t)k8 * 8));
         if (TIO) v = x8_as_f16(v, a.x_bf16);
-        *(uint4*)(xs + (size_t)t * 16) = v;
+        *(uint4*)(xs + xoff<NB>(bb, (uint32_t)k8 * 8u)) = v;
     }
 #pragma unroll
     for (int h = 0; h < RPL; ++h) {
@@ -221,7 +225,7 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
         // X_g[bb]: the 128 values of group u are 16 chunks of 8; lane l sums 4 of them, then a fixed butterfly
         for (int u = warp; u < NB * a.SC; u += W) {
             const int bb = u / a.SC, gq = u - bb * a.SC;
-            const uint2 hv = *(const uint2*)(xs + (((size_t)(16 * gq + (lane >> 1)) * NB + bb) << 4) + (lane & 1) * 8);
+            const uint2 hv = *(const uint2*)(xs + xoff<NB>(bb, (uint32_t)(16 * gq + (lane >> 1)) * 8u) + (lane & 1) * 8);
             const float2 p0 = __half22float2(*(const __half2*)&hv.x), p1 = __half22float2(*(const __half2*)&hv.y);
             float t = (p0.x + p0.y) + (p1.x + p1.y);
 #pragma unroll
@@ -241,6 +245,8 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
     const bool diag0 = (g == t4), diag1 = (g == t4 + 4);
     const bool diag = diag0 || diag1;
     const int b2 = diag1 ? 1 : 0;
+    // staged x of the lane's batch row of a pair, for chunk groups whose swizzle flips the row's low bit or not
+    const unsigned char* xrow[2] = {xs + b2 * 16, xs + (b2 ^ 1) * 16};
 
     // V2a: where this lane's own sums land: D[g][t] sits in lane (g, t >> 1), register t & 1 (even batch row of the
     // pair), and in lane (g, 2 + (t >> 1)) for the odd one
@@ -313,7 +319,11 @@ __global__ void __launch_bounds__(kBThreads, 1) gemv_batch_kernel(const BatchArg
 #pragma unroll
             for (int p = 0; p < NBP; ++p) {
                 xq[p] = make_uint4(0u, 0u, 0u, 0u);
-                if (diag) xq[p] = *(const uint4*)(xs + xoff<NB>(2 * p + b2, kbase + m * 4));
+                // chunk k / 8 = 16 (sc0 + s) + m / 2: its swizzle (m / 2) mod NB is known at compile time
+                constexpr int kSw = NB - 1;
+                const int c8 = (m >> 1) & kSw;
+                if (diag) xq[p] = *(const uint4*)(xrow[c8 & 1] + (size_t)(kbase >> 3) * (NB * 16) +
+                                                  (((m >> 1) * NB + ((2 * p) ^ (c8 & ~1))) << 4) + (((m * 4) & 7) << 1));
             }
             lookup(fb, m + 1);
             reload(m + 1);

@@ -75,28 +75,39 @@ cudaError_t launch_tile(const BatchPlan& p, const LaneArgs& a, int grid, cudaStr
 
 // Where this kernel measured faster than the kernels with two channels per lane (xfp_gemv_pair.cu at 2 rows,
 // xfp_gemv_batch.cu, xfp_gemv_v2a.cu), the general kernel and, from 13 (V2a: 9) rows, the tcgen05 kernel; sweep over
-// 4096 x 4096 .. 28672 x 8192, every bit width, 2..16 rows, 1 % outliers on a B200:
-//   * V2 N >= 5 (the other kernels keep one channel per lane there, or are the general kernel): everywhere except 2 rows
-//     on matrices of at most one round (pair kernel 6.1 against 6.8 us at 4096 x 4096); 3x at N = 6
-//   * V2 N <= 4: matrices of at most one round from 3 rows on (7.0 against 8.4 us at 4096 x 4096, 4 rows); on larger ones
-//     two channels per lane halve the mma count per weight and stay ahead (8192 x 8192, 4 rows: 16.9 against 19.9 us)
-//   * V2a: everywhere (4096 x 4096, 2 rows: 7.9 against 11.2 us; 28672 x 8192, 8 rows: 149 against 166 us) except
-//     N = 3 with its pair tables of the whole library at 2 rows or on mid-sized matrices, and N >= 4 from 3 rows on
-//     matrices of one to two rounds (8192 x 8192: 30.7 against 29.0 us)
-//   * many rows on a large matrix with few outliers stay on the tcgen05 kernel (28672 x 8192, 16 rows: 226 against 297 us)
+// 4096 x 4096 .. 28672 x 8192, every bit width, 2 / 4 / 8 rows, 1 % outliers on a B200 (us per call, this kernel
+// against the other):
+//   * V2 N = 6 (the other kernel is the general one): everywhere (28672 x 8192, 4 rows: 78 against 240) except 2 rows
+//     on matrices of one round (pair kernel 7.2 against 7.6)
+//   * V2 N = 5 (the others keep one channel per lane there too): beyond one round (28672 x 8192, 8 rows: 114 against
+//     160), and on one round where the batched kernel does not fit its shared memory (4096 x 12288, 4 rows: 19 against 54)
+//   * V2 N <= 4: matrices of one round at 3 or 4 rows (4096 x 4096, 4 rows: 7.1 against 8.2); everywhere else two
+//     channels per lane halve the mma count per weight and stay ahead (8192 x 8192, 4 rows: 16.4 against 19.9;
+//     28672 x 8192, 8 rows: 80 against 105)
+//   * V2a: up to 4 rows on matrices of one round (4096 x 4096, 2 rows: 7.9 against 11.2), N = 2 up to 4 rows
+//     everywhere, N = 4 at 2 rows and on large matrices up to 4 rows (28672 x 8192: 86 against 92), N = 5 on large
+//     matrices (8 rows: 158 against 198), N = 3 only at 3..4 rows on large matrices (its pair tables of the whole
+//     library serve the other kernel), N = 6 everywhere (28672 x 8192, 8 rows: 193 against 766)
+//   * many rows on a large matrix with few outliers stay on the tcgen05 kernel (28672 x 8192, 16 rows, 0.3 %: V2a 159
+//     against 246)
 static bool lane_batch_preferred(const Layout& l, int batch) {
     const int sms = sched_sms();
-    const bool small = l.RB <= sms;
-    if (batch_prefers_gemm(l, batch) && l.RB > 4 * sms) return false;
+    const bool small = l.RB <= sms, big = l.RB > 4 * sms;
+    if (batch_prefers_gemm(l, batch) && big) return false;
+    const bool many = batch > 4;   // tiles of 8 rows
     if (l.mode == 0) {
-        if (l.bits >= 5) return !(small && batch == 2);
-        return small && batch >= 3;
+        if (l.bits == 6) return !(small && batch == 2);
+        if (l.bits == 5) return small ? (batch >= 3 && !batch_supported(l, batch)) : true;
+        return small && batch >= 3 && !many;
     }
-    if ((size_t)l.L * l.E * 128 > 128 * 1024) return true;   // libraries of more than 128 KB a word per entry (N = 6): the other kernel is the general one
-    if (small) return true;
-    if (l.bits == 3) return batch >= 3 && l.RB > 4 * sms;
-    if (l.bits >= 4 && l.RB <= 2 * sms) return batch == 2;
-    return true;
+    if ((size_t)l.L * l.E * 128 > 128 * 1024) return true;   // N = 6 at L = 32: the other kernel is the general one
+    if (small) return !many || !batch_supported(l, batch);
+    switch (l.bits) {
+        case 2: return !many;
+        case 3: return big && batch >= 3 && !many;
+        case 4: return batch == 2 || (big && !many);
+        default: return big || (!many && l.RB > 2 * sms);
+    }
 }
 
 // 2..16 rows of fp16 x, one blob, fp32 or fp16 y, no fused store

@@ -113,9 +113,9 @@ size_t gemm_x_scratch_bytes(const Layout& l, int M);
 cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaStream_t s);
 
 // Batches from this size on run on the tensor-core kernel (xfp_gemm_tc.cu) when the blob is sparse in outliers:
-// the batched GEMV kernels decode once per 8 rows of x and grow by ~9 us per row at 28672 x 8192, the tcgen05
-// kernel decodes once for up to 128 rows (measured at 28672 x 8192, 0.3 % outliers, 16 rows: 144 against 185 us
-// for V2, 159 against 296 us for V2a; at 2 % outliers its per-lane outlier walk loses, 282 against 265 us).
+// the batched GEMV kernels decode once per 8 rows of x, the tcgen05 kernel decodes once for up to 128 rows (measured
+// at 28672 x 8192, 0.3 % outliers, 16 rows: 141 against 148 us for V2, 159 against 246 us for V2a; without outliers
+// 91 against 137 us; more outliers make its per-lane outlier walk lose).
 // Layout of a GEMV workspace, shared by every kernel that may be given it: counters (split-K tickets, one int per
 // row-block and blob at most) in [0, align256(4 * RB * n)), zero-filled before first use and left zero-filled by every
 // call; partial sums behind it, written before they are read.
@@ -131,7 +131,9 @@ inline bool batch_prefers_gemm(const Layout& l, int batch) {
     // region that every GEMV kernel leaves zero-filled
     if (gemm_workspace_bytes(l, batch) > gemm_ctrl_bytes(l, batch) || gemm_ctrl_bytes(l, batch) > align256((size_t)l.RB * 4))
         return false;
-    return l.nnz * 100 <= (long long)l.rows * l.cols;   // at most 1 % outliers
+    // at most 1 % outliers (V2: 0.5 %; the batched mma.sync kernel overtakes the per-lane outlier walk earlier there:
+    // 28672 x 8192, 16 rows, 1 %: 159 against 206 us)
+    return l.nnz * (l.mode ? 100 : 200) <= (long long)l.rows * l.cols;
 }
 
 }  // namespace xfp

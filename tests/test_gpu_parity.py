@@ -160,8 +160,9 @@ def test_batched_shapes_and_split_k(mode, rows, cols, bits):
                                              (1, 4, 64), (1, 2, 256), (1, 6, 64)])
 def test_several_rows_of_x_on_matrices_of_one_round(mode, bits, group):
     """2..16 rows of x on a matrix of 79 row-blocks (more than half the SMs, fewer than all: one resident CTA per
-    row-block, the last one ragged), the shape class on which every batch goes to the one-channel-per-lane kernel with
-    1, 2, 4 or 8 B fragments per decoded fragment: tiles of 2, 4 and 8 rows, partial tiles (3, 7), two launches (11, 16)."""
+    row-block, the last one ragged), the shape class on which the one-channel-per-lane kernel with 2, 4 or 8 B
+    fragments per decoded fragment takes most batches (all of them at N = 6, up to 4 rows otherwise; the kernels with
+    two channels per lane take the rest): tiles of 2, 4 and 8 rows, partial tiles (3, 7), two launches (11, 16)."""
     rows, cols = 2500, 768
     q = synth.random_quantized(mode, rows, cols, bits, 0.015, seed=9100 + 10 * bits + mode + group, group_size=group)
     pm = xfp.pack_tensors(q, col_bits=16)
