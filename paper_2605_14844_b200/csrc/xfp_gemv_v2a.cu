@@ -248,14 +248,14 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
         if (__syncthreads_or(differs)) {
             for (int i = threadIdx.x; i < nvec; i += kAThreads) libcopy[i] = __ldg(cb4 + i);
             if (PAIR) {
-                // pair tables, 16 copies: words (id * E*E + pair) * 16 .. + 15 hold the same half2
-                for (int e = threadIdx.x; e < a.L * E * E; e += kAThreads) {
-                    const int id = e / (E * E), pr = e % (E * E);
+                // pair tables, 16 copies: words (id * E*E + pair) * 16 .. + 15 hold the same half2.  Four threads per
+                // entry, 16 bytes each: a warp's store covers 512 contiguous bytes (one thread writing the entry's 64
+                // bytes put a quarter-warp into two bank groups: 4300 wavefronts per fill instead of 1024)
+                for (int t = threadIdx.x; t < a.L * E * E * 4; t += kAThreads) {
+                    const int e = t >> 2, id = e / (E * E), pr = e % (E * E);
                     const uint32_t v = (uint32_t)__ldg(b.cb + id * E + (pr & (E - 1))) |
                                        ((uint32_t)__ldg(b.cb + id * E + (pr >> N)) << 16);
-                    const uint4 v4 = make_uint4(v, v, v, v);
-                    uint4* dst = (uint4*)(tab + (size_t)e * 64);
-                    dst[0] = v4; dst[1] = v4; dst[2] = v4; dst[3] = v4;
+                    ((uint4*)(tab + (size_t)e * 64))[t & 3] = make_uint4(v, v, v, v);
                 }
             } else {
                 // one copy per bank: word (e * 32 + lane) = lib[e] for every lane
