@@ -647,7 +647,7 @@ def _random_cases(count, seed):
     for i in range(count):
         mode = int(rng.integers(0, 2))
         bits = int(rng.integers(2, 7))
-        rows = int(rng.choice([1, 7, 31, 32, 33, 63, 64, 65, 95, 160, 257, 416, 700, 1000]))
+        rows = int(rng.choice([1, 7, 31, 32, 33, 63, 64, 65, 95, 160, 257, 416, 700, 1000, 2500, 4800, 9500]))
         cols = 128 * int(rng.choice([1, 2, 3, 5, 8, 11, 12, 13, 16, 24, 33]))
         batch = int(rng.choice([1, 1, 1, 2, 3, 4, 7, 8, 9, 16]))
         rate = float(rng.choice([0.0, 0.0005, 0.004, 0.02, 0.06]))
@@ -662,7 +662,7 @@ def _random_cases(count, seed):
                          ids=lambda c: "-".join(str(v) for v in c))
 def test_randomized_shapes_types_and_outlier_structure(case):
     """A seeded sweep over everything the dispatcher keys on at once: mode, bit width, ragged channel counts
-    (1 ... 1000), K from one to 33 super-chunks, batch 1..16, outlier rate and placement (including all outliers in one
+    (1 ... 9500: from a single row-block to more row-blocks than CTA slots), K from one to 33 super-chunks, batch 1..16, outlier rate and placement (including all outliers in one
     channel), activation and output types."""
     i, mode, bits, rows, cols, batch, rate, placement, xtype, ytype = case
     q = synth.random_quantized(mode, rows, cols, bits, rate, seed=5000 + i, placement=placement)
