@@ -1,194 +1,258 @@
 // xfp_pack: unpacked tensors -> device layout (with range validation and clamping);
 // xfp_dequant: device layout -> fp16 matrix W^ = fp16(D16 + S), bit-exact.
+#include <cstdlib>
+
 #include "xfp_internal.h"
 #include "xfp_pair_common.cuh"
 
 namespace xfp {
 
 // ------------------------------------------------------------------------------------ pack
+//
+// One launch: the blocks of the grid are dealt to the six parts of the blob (index stream, codebooks, group
+// metadata, row pointers, outlier entries, transposed slabs) by block index.  Every part reads the caller's tensors
+// only -- the slabs apply the same clamping and neutralisation as the row pointers and entries they mirror -- so no
+// part waits for another.  (As seven launches the small parts cost 28 of 94 us at 28672 x 8192 and set a floor of
+// ~32 us on small matrices.)
 
-// One thread per (row-block, super-chunk, lane): 128 byte-indices of one channel -> N uint4.
-template <int N>
-__global__ void __launch_bounds__(128) pack_idx_kernel(const uint8_t* __restrict__ idx, uint4* __restrict__ out,
-                                                       int rows, int cols, int RB, int SC, int* err_word) {
-    constexpr uint32_t E = 1u << N;
-    const int lane = threadIdx.x & 31;
-    const long long unit = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (unit >= (long long)RB * SC) return;
-    const int rb = (int)(unit / SC), sc = (int)(unit % SC);
-    const int row = rb * kRowsPerBlock + lane;
-    uint32_t w[4 * N + 1];
-#pragma unroll
-    for (int i = 0; i < 4 * N + 1; ++i) w[i] = 0u;
-    bool bad = false;
-    if (row < rows) {
-        const uint4* src = (const uint4*)(idx + (size_t)row * cols + (size_t)sc * kSuper);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint4 t = __ldg(src + i);
-            const uint32_t tw[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-            for (int b = 0; b < 16; ++b) {
-                uint32_t q = (tw[b >> 2] >> ((b & 3) * 8)) & 0xffu;
-                bad |= (q >= E);
-                q &= E - 1u;
-                const int j = i * 16 + b;
-                const int bit = j * N, wi = bit >> 5, off = bit & 31;
-                w[wi] |= q << off;
-                if (off + N > 32) w[wi + 1] |= q >> (32 - off);
-            }
-        }
-    }
-    if (bad && err_word) atomicOr(err_word, 1);
-    uint4* dst = out + ((size_t)unit * N) * 32 + lane;
-#pragma unroll
-    for (int v = 0; v < N; ++v) dst[(size_t)v * 32] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
-}
+constexpr int kPackThreads = 256;
+constexpr int kPackWarps = kPackThreads / 32;
 
-__global__ void pack_codebook_kernel(const uint16_t* __restrict__ cb, uint16_t* __restrict__ out, long long n_src,
-                                     long long n_dst) {
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t < n_dst) out[t] = t < n_src ? cb[t] : (uint16_t)0;
-}
-
-__global__ void pack_group_kernel(const uint8_t* __restrict__ gid, const uint16_t* __restrict__ gscale,
-                                  const uint16_t* __restrict__ gmid, uint8_t* __restrict__ out_gid,
-                                  uint32_t* __restrict__ out_gsm, int rows, int RB, int SC, int L, int G, int GH,
-                                  int* err_word) {
-    // one thread per (row-block, super-chunk, part of the super-chunk, lane); the group that holds the part's first
-    // weight supplies its metadata (a group of 256 weights is stored with both of its super-chunks)
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= (long long)RB * SC * GH * 32) return;
-    const int lane = (int)(t & 31);
-    const long long part = t >> 5;
-    const long long unit = part / GH;
-    const int h = (int)(part % GH);
-    const int rb = (int)(unit / SC), sc = (int)(unit % SC);
-    const int row = rb * kRowsPerBlock + lane;
-    const int groups = SC * kSuper / G;                        // groups per channel
-    const int grp = (sc * kSuper + h * (kSuper / GH)) / G;
-    uint32_t id = 0, sm = 0;
-    if (row < rows) {
-        id = gid[(size_t)row * groups + grp];
-        if ((int)id >= L) {
-            if (err_word) atomicOr(err_word, 2);
-            id = (uint32_t)(L - 1);
-        }
-        sm = (uint32_t)gscale[(size_t)row * groups + grp] | ((uint32_t)gmid[(size_t)row * groups + grp] << 16);
-    }
-    out_gid[t] = (uint8_t)id;
-    out_gsm[t] = sm;
-}
+struct PackArgs {
+    PackInputs in;
+    char* base;             // the blob
+    Layout l;
+    int* err_word;
+    // first block of every part, in this order: slabs, entries, rowptr, group, codebook, idx; [6] = grid.  (Spreading
+    // the blocks of the small parts evenly among those of the index part measured the same: 110.6 against 106.5 us at
+    // 28672 x 8192 with 2 % outliers.)
+    unsigned first[7];
+};
 
 __device__ __forceinline__ int clampi(long long v, long long lo, long long hi) {
     return (int)(v < lo ? lo : (v > hi ? hi : v));
 }
 
-// rowptr -> clamped copy (padding rows empty); checks monotonicity and the end points;
-// each thread also checks that its row's columns ascend strictly.
-__global__ void pack_rowptr_kernel(const int32_t* __restrict__ rowptr, const void* __restrict__ ocol, int col_bits,
-                                   int* __restrict__ out, int rows, int rows_pad, long long nnz, int* err_word) {
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t > rows_pad) return;
-    if (rowptr == nullptr) {  // nnz == 0
+__device__ __forceinline__ long long col_at(const void* ocol, int col_bits, long long p) {
+    return col_bits == 16 ? (long long)((const uint16_t*)ocol)[p] : (long long)((const int32_t*)ocol)[p];
+}
+
+// outlier p as the blob stores it: column | fp16 value << 16; a column outside the matrix becomes column 0, value +0
+__device__ __forceinline__ uint32_t entry_at(const PackInputs& in, long long p, int cols, bool* bad) {
+    long long c = col_at(in.ocol, in.col_bits, p);
+    uint32_t v = in.oval[p];
+    if (c < 0 || c >= cols) { *bad = true; c = 0; v = 0; }
+    return (uint32_t)c | (v << 16);
+}
+
+// One warp per (row-block, super-chunk): 128 byte-indices of every channel -> N uint4 per lane.  The warp fetches its
+// 32 x 128-byte tile of indices with whole 128-byte lines per quarter-warp and hands every lane its channel's row through
+// shared memory (a lane reading its own row from global memory made every 16-byte load a line of its own: 16.3 M
+// wavefronts on the L1 data pipe at 28672 x 8192 against 7.6 M this way).
+template <int N>
+__device__ __forceinline__ void pack_idx_block(const PackArgs& a, unsigned vblk, unsigned char* tiles) {
+    constexpr uint32_t E = 1u << N;
+    constexpr int kRowB = 144;   // bytes per tile row: 16-byte aligned, the lanes of a quarter-warp in distinct banks
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long unit = (long long)vblk * kPackWarps + warp;
+    if (unit >= (long long)a.l.RB * a.l.SC) return;
+    const int rb = (int)(unit / a.l.SC), sc = (int)(unit % a.l.SC);
+    unsigned char* tile = tiles + warp * 32 * kRowB;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + (lane >> 3), c = lane & 7;   // rows 4i .. 4i+3 of the tile, 16-byte chunk c
+        const int row_g = rb * kRowsPerBlock + r;
+        uint4 t = make_uint4(0u, 0u, 0u, 0u);
+        if (row_g < a.l.rows) t = __ldg((const uint4*)(a.in.idx + (size_t)row_g * a.l.cols + (size_t)sc * kSuper) + c);
+        *(uint4*)(tile + r * kRowB + c * 16) = t;
+    }
+    __syncwarp();
+    uint32_t w[4 * N + 1];
+#pragma unroll
+    for (int i = 0; i < 4 * N + 1; ++i) w[i] = 0u;
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint4 t = *(const uint4*)(tile + lane * kRowB + i * 16);
+        const uint32_t tw[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+            uint32_t q = (tw[b >> 2] >> ((b & 3) * 8)) & 0xffu;
+            bad |= (q >= E);
+            q &= E - 1u;
+            const int j = i * 16 + b;
+            const int bit = j * N, wi = bit >> 5, off = bit & 31;
+            w[wi] |= q << off;
+            if (off + N > 32) w[wi + 1] |= q >> (32 - off);
+        }
+    }
+    if (bad && a.err_word) atomicOr(a.err_word, 1);
+    uint4* dst = (uint4*)(a.base + a.l.off_idx) + ((size_t)unit * N) * 32 + lane;
+#pragma unroll
+    for (int v = 0; v < N; ++v) dst[(size_t)v * 32] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+}
+
+__device__ __forceinline__ void pack_codebook_block(const PackArgs& a, unsigned vblk) {
+    const long long n_src = (long long)(a.l.mode ? a.l.L : a.l.rows) * a.l.E;
+    const long long n_dst = (long long)(a.l.mode ? a.l.L : a.l.rows_pad) * a.l.E;
+    const long long t = (long long)vblk * kPackThreads + threadIdx.x;
+    uint16_t* out = (uint16_t*)(a.base + a.l.off_cb);
+    if (t < n_dst) out[t] = t < n_src ? a.in.codebook[t] : (uint16_t)0;
+}
+
+__device__ __forceinline__ void pack_group_block(const PackArgs& a, unsigned vblk) {
+    // one thread per (row-block, super-chunk, part of the super-chunk, lane); the group that holds the part's first
+    // weight supplies its metadata (a group of 256 weights is stored with both of its super-chunks)
+    const Layout& l = a.l;
+    const long long t = (long long)vblk * kPackThreads + threadIdx.x;
+    if (t >= (long long)l.RB * l.SC * l.GH * 32) return;
+    const int lane = (int)(t & 31);
+    const long long part = t >> 5;
+    const long long unit = part / l.GH;
+    const int h = (int)(part % l.GH);
+    const int rb = (int)(unit / l.SC), sc = (int)(unit % l.SC);
+    const int row = rb * kRowsPerBlock + lane;
+    const int groups = l.SC * kSuper / l.G;                        // groups per channel
+    const int grp = (sc * kSuper + h * (kSuper / l.GH)) / l.G;
+    uint32_t id = 0, sm = 0;
+    if (row < l.rows) {
+        id = a.in.gid[(size_t)row * groups + grp];
+        if ((int)id >= l.L) {
+            if (a.err_word) atomicOr(a.err_word, 2);
+            id = (uint32_t)(l.L - 1);
+        }
+        sm = (uint32_t)a.in.gscale[(size_t)row * groups + grp] | ((uint32_t)a.in.gmid[(size_t)row * groups + grp] << 16);
+    }
+    ((uint8_t*)(a.base + l.off_gid))[t] = (uint8_t)id;
+    ((uint32_t*)(a.base + l.off_gsm))[t] = sm;
+}
+
+// rowptr -> clamped copy (padding rows empty); checks monotonicity and the end points (that the columns of a row
+// ascend strictly is checked where the entries are read in order, in ell_fill_block).  The first thread writes the
+// header words.
+__device__ __forceinline__ void pack_rowptr_block(const PackArgs& a, unsigned vblk) {
+    const Layout& l = a.l;
+    const int t = (int)(vblk * kPackThreads + threadIdx.x);
+    if (t == 0) {
+        int* hdr = (int*)(a.base + l.off_hdr);
+        hdr[0] = l.ell_slots;
+        hdr[1] = 0;
+        *(long long*)(hdr + 2) = (long long)l.off_ell;
+    }
+    if (t > l.rows_pad) return;
+    int* out = (int*)(a.base + l.off_rowptr);
+    if (l.nnz == 0) {
         out[t] = 0;
         return;
     }
+    const long long nnz = l.nnz;
     int bad = 0;
-    long long v = t <= rows ? (long long)rowptr[t] : nnz;
+    long long v = t <= l.rows ? (long long)a.in.rowptr[t] : nnz;
     if (t == 0 && v != 0) bad |= 4;
-    if (t == rows && v != nnz) bad |= 4;
+    if (t == l.rows && v != nnz) bad |= 4;
     if (v < 0 || v > nnz) bad |= 4;
-    if (t < rows) {
-        long long nx = rowptr[t + 1];
+    if (t < l.rows) {
+        long long nx = a.in.rowptr[t + 1];
         if (nx < v) bad |= 4;
-        const int p0 = clampi(v, 0, nnz), p1 = clampi(nx, 0, nnz);
-        long long prev = -1;
-        for (int p = p0; p < p1; ++p) {
-            const long long c = col_bits == 16 ? (long long)((const uint16_t*)ocol)[p] : (long long)((const int32_t*)ocol)[p];
-            if (c <= prev) bad |= 16;
-            prev = c;
-        }
     }
     out[t] = clampi(v, 0, nnz);
-    if (bad && err_word) atomicOr(err_word, bad);
+    if (bad && a.err_word) atomicOr(a.err_word, bad);
 }
 
-__global__ void pack_entries_kernel(const void* __restrict__ ocol, int col_bits, const uint16_t* __restrict__ oval,
-                                    uint32_t* __restrict__ out, long long nnz, int cols, int* err_word) {
-    const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= nnz) return;
-    long long c = col_bits == 16 ? (long long)((const uint16_t*)ocol)[p] : (long long)((const int32_t*)ocol)[p];
-    uint32_t v = oval[p];
-    if (c < 0 || c >= cols) {  // neutralise: column 0, value +0
-        if (err_word) atomicOr(err_word, 8);
-        c = 0;
-        v = 0;
-    }
-    out[p] = (uint32_t)c | (v << 16);
+__device__ __forceinline__ void pack_entries_block(const PackArgs& a, unsigned vblk) {
+    const long long p = (long long)vblk * kPackThreads + threadIdx.x;
+    if (p >= a.l.nnz) return;
+    bool bad = false;
+    ((uint32_t*)(a.base + a.l.off_oent))[p] = entry_at(a.in, p, a.l.cols, &bad);
+    if (bad && a.err_word) atomicOr(a.err_word, 8);
 }
 
-// Transposed outlier slab of row-block b (one CTA of 8 warps per block, the slots dealt to the warps): word [0][lane]
-// = slots used by channel b*32+lane, word [1+j][lane] = its j-th outlier or the neutral entry (column 0, value +0).
-__global__ void __launch_bounds__(256) ell_fill_kernel(const int* __restrict__ rp, const uint32_t* __restrict__ oent,
-                                                       uint32_t* __restrict__ ell, int RB, int C) {
-    const int b = blockIdx.x;
+// Transposed outlier slab of row-block b: word [0][lane] = slots used by channel b*32+lane, word [1+j][lane] = its
+// j-th outlier or the neutral entry (column 0, value +0).  Reads the caller's row pointers and entries with the
+// clamping of pack_rowptr_block and pack_entries_block.  The block's entries are one contiguous range of the CSR
+// arrays: a warp takes a channel and reads its entries in order (coalesced), each entry goes to its slot of a copy of
+// the slab in shared memory (windows of 256 slots), which is then written out in whole lines.  (Every lane walking its
+// own row -- 32 scattered sectors per load --, scattered 4-byte stores into the slab, and a binary search of every
+// entry for its channel each made this part 50-60 us at 2 % outliers on 28672 x 8192.)  The same pass checks that the
+// columns of a row ascend strictly.  Row pointers that do not ascend (reported by pack_rowptr_block) leave slots
+// neutral, never an access outside the arrays.
+constexpr int kEllWindow = 256;   // slots of the slab held in shared memory at a time
+__device__ __forceinline__ void ell_fill_block(const PackArgs& a, unsigned b, unsigned char* smem) {
+    const Layout& l = a.l;
+    uint32_t* sl = (uint32_t*)smem;                       // [kEllWindow][33]: consecutive slots of one channel in consecutive banks
+    int* rp = (int*)(smem + kEllWindow * 33 * 4);         // [33]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (b >= RB) return;
-    const int p0 = rp[b * 32 + lane], p1 = rp[b * 32 + lane + 1];
-    const int len = p1 > p0 ? min(p1 - p0, C) : 0;
-    uint32_t* slab = ell + (size_t)b * (C + 1) * 32 + lane;
-    if (warp == 0) slab[0] = (uint32_t)len;
-    for (int j = warp; j < C; j += 8) slab[(size_t)(1 + j) * 32] = j < len ? oent[p0 + j] : 0u;
-}
-
-__global__ void pack_header_kernel(int* hdr, int ell_slots, long long off_ell) {
-    if (threadIdx.x == 0) {
-        hdr[0] = ell_slots;
-        hdr[1] = 0;
-        *(long long*)(hdr + 2) = off_ell;
+    const int C = l.ell_slots;
+    const long long nnz = l.nnz;
+    if (threadIdx.x < 33) {
+        const int row = (int)b * 32 + (int)threadIdx.x;
+        rp[threadIdx.x] = row <= l.rows ? clampi(a.in.rowptr[row], 0, nnz) : (int)nnz;
     }
+    __syncthreads();
+    uint32_t* slab = (uint32_t*)(a.base + l.off_ell) + (size_t)b * (C + 1) * 32;
+    if (warp == 0) {
+        const int p0 = rp[lane], p1 = rp[lane + 1];
+        slab[lane] = (uint32_t)(p1 > p0 ? min(p1 - p0, C) : 0);
+    }
+    int bad = 0;   // a column outside the matrix is reported by pack_entries_block
+    for (int j0 = 0; j0 < C; j0 += kEllWindow) {
+        const int nj = min(kEllWindow, C - j0);
+        for (int i = threadIdx.x; i < nj * 33; i += kPackThreads) sl[i] = 0u;
+        __syncthreads();
+        for (int r = warp; r < 32; r += kPackWarps) {   // a warp per channel, its lanes along the channel's entries
+            const int p0 = rp[r], n = rp[r + 1] - p0;   // n <= 0: an empty channel, or row pointers that descend
+            for (int jj = lane; jj < n; jj += 32) {
+                const int p = p0 + jj;
+                if (j0 == 0 && jj > 0 && col_at(a.in.ocol, a.in.col_bits, p) <= col_at(a.in.ocol, a.in.col_bits, p - 1)) bad = 16;
+                bool outside = false;
+                if (jj >= j0 && jj < j0 + nj) sl[(jj - j0) * 33 + r] = entry_at(a.in, p, l.cols, &outside);
+            }
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < nj * 32; i += kPackThreads) slab[(size_t)(1 + j0) * 32 + i] = sl[(i >> 5) * 33 + (i & 31)];
+        __syncthreads();
+    }
+    if (bad && a.err_word) atomicOr(a.err_word, bad);
 }
 
 template <int N>
-static void launch_pack_idx(const Layout& l, const uint8_t* idx, uint4* out, int* err, cudaStream_t s) {
-    const long long units = (long long)l.RB * l.SC;
-    const unsigned grid = (unsigned)((units + 3) / 4);
-    pack_idx_kernel<N><<<grid, 128, 0, s>>>(idx, out, l.rows, l.cols, l.RB, l.SC, err);
+__global__ void __launch_bounds__(kPackThreads) pack_kernel(const PackArgs a) {
+    __shared__ __align__(16) unsigned char tiles[kPackWarps * 32 * 144];   // 36864 bytes; the slab part uses 33792 + 132
+    static_assert(kPackWarps * 32 * 144 >= kEllWindow * 33 * 4 + 33 * 4, "slab window and row pointers fit the tile area");
+    const unsigned b = blockIdx.x;
+    if (b < a.first[1]) ell_fill_block(a, b, tiles);
+    else if (b < a.first[2]) pack_entries_block(a, b - a.first[1]);
+    else if (b < a.first[3]) pack_rowptr_block(a, b - a.first[2]);
+    else if (b < a.first[4]) pack_group_block(a, b - a.first[3]);
+    else if (b < a.first[5]) pack_codebook_block(a, b - a.first[4]);
+    else pack_idx_block<N>(a, b - a.first[5], tiles);
 }
 
 cudaError_t launch_pack(const Layout& l, const PackInputs& in, void* packed, int* err_word, cudaStream_t s) {
-    char* base = (char*)packed;
-    uint4* oidx = (uint4*)(base + l.off_idx);
+    PackArgs a;
+    a.in = in; a.base = (char*)packed; a.l = l; a.err_word = err_word;
+    auto blocks = [](long long n, int per) { return (unsigned)((n + per - 1) / per); };
+    const long long n_cb = (long long)(l.mode ? l.L : l.rows_pad) * l.E;
+    unsigned n[6];
+    n[0] = l.nnz ? (unsigned)l.RB : 0u;
+    n[1] = l.nnz ? blocks(l.nnz, kPackThreads) : 0u;
+    n[2] = blocks((long long)l.rows_pad + 1, kPackThreads);
+    n[3] = l.mode ? blocks((long long)l.RB * l.SC * l.GH * 32, kPackThreads) : 0u;
+    n[4] = blocks(n_cb, kPackThreads);
+    n[5] = blocks((long long)l.RB * l.SC, kPackWarps);
+#ifdef LANE_TUNE
+    if (const char* e = getenv("XFP_PACK_SKIP"))   // tuning build: leave parts out (bit i = part i) to time the others
+        for (int i = 0; i < 6; ++i)
+            if ((atoi(e) >> i) & 1) n[i] = 0;
+#endif
+    a.first[0] = 0;
+    for (int i = 0; i < 6; ++i) a.first[i + 1] = a.first[i] + n[i];
     switch (l.bits) {
-        case 2: launch_pack_idx<2>(l, in.idx, oidx, err_word, s); break;
-        case 3: launch_pack_idx<3>(l, in.idx, oidx, err_word, s); break;
-        case 4: launch_pack_idx<4>(l, in.idx, oidx, err_word, s); break;
-        case 5: launch_pack_idx<5>(l, in.idx, oidx, err_word, s); break;
-        default: launch_pack_idx<6>(l, in.idx, oidx, err_word, s); break;
-    }
-    const long long n_src = (long long)(l.mode ? l.L : l.rows) * l.E;
-    const long long n_dst = (long long)(l.mode ? l.L : l.rows_pad) * l.E;
-    pack_codebook_kernel<<<(unsigned)((n_dst + 255) / 256), 256, 0, s>>>(in.codebook, (uint16_t*)(base + l.off_cb), n_src,
-                                                                        n_dst);
-    if (l.mode) {
-        const long long n = (long long)l.RB * l.SC * l.GH * 32;
-        pack_group_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(in.gid, in.gscale, in.gmid,
-                                                                     (uint8_t*)(base + l.off_gid),
-                                                                     (uint32_t*)(base + l.off_gsm), l.rows, l.RB, l.SC,
-                                                                     l.L, l.G, l.GH, err_word);
-    }
-    pack_rowptr_kernel<<<(unsigned)((l.rows_pad + 1 + 255) / 256), 256, 0, s>>>(
-        l.nnz ? in.rowptr : nullptr, in.ocol, in.col_bits, (int*)(base + l.off_rowptr), l.rows, l.rows_pad, l.nnz,
-        err_word);
-    pack_header_kernel<<<1, 32, 0, s>>>((int*)(base + l.off_hdr), l.ell_slots, (long long)l.off_ell);
-    if (l.nnz) {
-        pack_entries_kernel<<<(unsigned)((l.nnz + 255) / 256), 256, 0, s>>>(in.ocol, in.col_bits, in.oval,
-                                                                           (uint32_t*)(base + l.off_oent), l.nnz,
-                                                                           l.cols, err_word);
-        ell_fill_kernel<<<(unsigned)l.RB, 256, 0, s>>>((const int*)(base + l.off_rowptr),
-                                                                   (const uint32_t*)(base + l.off_oent),
-                                                                   (uint32_t*)(base + l.off_ell), l.RB, l.ell_slots);
+        case 2: pack_kernel<2><<<a.first[6], kPackThreads, 0, s>>>(a); break;
+        case 3: pack_kernel<3><<<a.first[6], kPackThreads, 0, s>>>(a); break;
+        case 4: pack_kernel<4><<<a.first[6], kPackThreads, 0, s>>>(a); break;
+        case 5: pack_kernel<5><<<a.first[6], kPackThreads, 0, s>>>(a); break;
+        default: pack_kernel<6><<<a.first[6], kPackThreads, 0, s>>>(a); break;
     }
     return cudaGetLastError();
 }
