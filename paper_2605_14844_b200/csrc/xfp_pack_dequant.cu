@@ -346,16 +346,23 @@ __global__ void __launch_bounds__(256) dequant_lut_kernel(Blob b, uint16_t* W, i
     __syncthreads();
     const uint32_t base = (uint32_t)lane * 4u;
     uint32_t* tile = tiles + warp * 32 * kStrideW;
-    for (int sc = sc_begin + warp; sc < sc_end; sc += kWarps) {
-        const size_t unit = (size_t)rb * SC + sc;
-        uint32_t w[4 * N + 1];
-        const uint4* src = b.idx + (unit * N) * 32 + lane;
+    // the index vectors of a warp's next super-chunk travel while it decodes the current one
+    uint4 nx[N];
+    if (sc_begin + warp < sc_end) {
+        const uint4* src = b.idx + (((size_t)rb * SC + sc_begin + warp) * N) * 32 + lane;
 #pragma unroll
-        for (int v = 0; v < N; ++v) {
-            const uint4 t = ld_stream(src + (size_t)v * 32);
-            w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
-        }
+        for (int v = 0; v < N; ++v) nx[v] = ld_stream(src + (size_t)v * 32);
+    }
+    for (int sc = sc_begin + warp; sc < sc_end; sc += kWarps) {
+        uint32_t w[4 * N + 1];
+#pragma unroll
+        for (int v = 0; v < N; ++v) { w[4 * v] = nx[v].x; w[4 * v + 1] = nx[v].y; w[4 * v + 2] = nx[v].z; w[4 * v + 3] = nx[v].w; }
         w[4 * N] = 0u;
+        if (sc + kWarps < sc_end) {
+            const uint4* src = b.idx + (((size_t)rb * SC + sc + kWarps) * N) * 32 + lane;
+#pragma unroll
+            for (int v = 0; v < N; ++v) nx[v] = ld_stream(src + (size_t)v * 32);
+        }
         uint32_t* trow = tile + lane * kStrideW;
 #pragma unroll
         for (int p = 0; p < kSuper / 2; ++p) {
