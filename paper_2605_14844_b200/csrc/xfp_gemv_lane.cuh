@@ -249,6 +249,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         const int j = gw + q * ostride;
         oe[q] = j < ell_slots ? __ldg(slab + (size_t)(1 + j) * 32) : 0u;   // every slot below the capacity is readable
     }
+    lstamp(a, 6);
     // ---- tables: warp w fills entries [w T / W, (w+1) T / W) of every lane's channel
     if (MODE != 0) {
         if (!kMulti || it == 0) {   // one library per blob: a resident CTA fills it once
@@ -268,25 +269,51 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         }
     } else {
         const uint16_t* cb = b.cb + (size_t)(blk * kRowsPerBlock + lane) * E;
-        if (C::kQuad) {
+        if constexpr (C::kQuad) {
             // entry t = (cb[t & 3], cb[t >> 2 & 3], cb[t >> 4 & 3], cb[t >> 6]) as 8 bytes at t * 256 + lane * 8
             const uint2 c4 = __ldg((const uint2*)cb);   // the four entries
             const uint32_t e0 = c4.x & 0xffffu, e1 = c4.x >> 16, e2 = c4.y & 0xffffu, e3 = c4.y >> 16;
             auto ent = [&](int q) { return q == 0 ? e0 : (q == 1 ? e1 : (q == 2 ? e2 : e3)); };
+            // entries t = 16 h + i: the high half (indices 2, 3 of the byte) is the same for sixteen entries and is
+            // picked once; the low half runs over all sixteen pairs with compile-time picks (selecting all four values
+            // of every entry at run time made this fill 1.15 us, the longest prologue of all widths)
+            const uint32_t eh[4] = {e0 << 16, e1 << 16, e2 << 16, e3 << 16};
+            const uint32_t el[4] = {e0, e1, e2, e3};
             constexpr int TW = T / W;
+            static_assert(TW % 16 == 0, "a warp fills whole groups of sixteen entries");
 #pragma unroll
-            for (int i = 0; i < TW; ++i) {
-                const int t = warp * TW + i;
-                const uint32_t lo = ent(t & 3) | (ent((t >> 2) & 3) << 16);
-                const uint32_t hi = ent((t >> 4) & 3) | (ent(t >> 6) << 16);
-                *(uint2*)(tab + (size_t)t * kStride + lane * 8) = make_uint2(lo, hi);
+            for (int gq = 0; gq < TW / 16; ++gq) {
+                const int h = warp * (TW / 16) + gq;
+                const uint32_t hi = ent(h & 3) | (ent(h >> 2) << 16);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    *(uint2*)(tab + (size_t)(h * 16 + i) * kStride + lane * 8) = make_uint2(el[i & 3] | eh[i >> 2], hi);
             }
-        } else if (C::kSingle) {
-            constexpr int TW = T / W;   // 4
+        } else if constexpr (C::kSingle && (T / W == 2 || T / W == 4 || T / W == 8)) {
+            // a warp's TW consecutive entries of every channel in ONE load per lane (2, 4 or 8 entries: 4, 8 or 16 bytes;
+            // one 2-byte load per entry made four requests of 32 sectors each and the fill 1.2 us at N = 6)
+            constexpr int TW = T / W;
+            uint32_t cw[TW / 2];
+            if (TW == 2) {
+                cw[0] = __ldg((const uint32_t*)(cb + warp * TW));
+            } else if (TW == 4) {
+                const uint2 t = __ldg((const uint2*)(cb + warp * TW));
+                cw[0] = t.x; cw[TW / 2 - 1] = t.y;
+            } else {
+                const uint4 t = __ldg((const uint4*)(cb + warp * TW));
+                cw[0] = t.x; cw[1 % (TW / 2)] = t.y; cw[2 % (TW / 2)] = t.z; cw[3 % (TW / 2)] = t.w;
+            }
 #pragma unroll
             for (int i = 0; i < TW; ++i) {
                 const int t = warp * TW + i;
-                *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (uint32_t)__ldg(cb + t);
+                *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (i & 1) ? (cw[i >> 1] >> 16) : (cw[i >> 1] & 0xffffu);
+            }
+        } else if (C::kSingle) {   // (instantiated for V2a widths only, where this branch is never taken)
+            constexpr int TW = T / W > 0 ? T / W : 1;
+#pragma unroll
+            for (int i = 0; i < TW; ++i) {
+                const int t = warp * TW + i;
+                if (t < T) *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (uint32_t)__ldg(cb + t);
             }
         } else if (T / W >= E) {
             // a warp fills whole rows of the pair matrix: entries (hi, 0..E-1) for its values of hi.  Every warp needs
