@@ -253,17 +253,38 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     // ---- tables: warp w fills entries [w T / W, (w+1) T / W) of every lane's channel
     if (MODE != 0) {
         if (!kMulti || it == 0) {   // one library per blob: a resident CTA fills it once
-        if (kHalf) {
-            for (int e = warp; e < ((a.L + 1) >> 1) * E; e += W) {
+        // every row of the table is one word repeated in the 32 banks: a lane fetches the word of row e0 + lane, then
+        // the warp stores the 32 rows one after the other, each word handed round by a shuffle (a warp that fetched
+        // two halves per row with uniform loads paid their latency once per row: 3.9 us for the 1024 rows of N = 6)
+        const int trows = kHalf ? ((a.L + 1) >> 1) * E : a.L * E * E;
+        // (tables of up to 8 rows per warp keep the plain loop: with the shuffle form the same K loop ran 6 % slower at
+        // N = 3 and 4 -- 62.2 against 58.3 us at 28672 x 8192 -- through the compiler's register allocation)
+        constexpr bool kShuffleFill = N >= 5 || kLibPair;
+        if (!kShuffleFill) {
+            for (int e = warp; e < trows; e += W) {
                 const int m = e >> N, q = e & (E - 1);
                 const uint32_t lo = __ldg(b.cb + (size_t)(2 * m) * E + q);
                 const uint32_t hi = 2 * m + 1 < a.L ? (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) : 0u;
                 *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = lo | (hi << 16);
             }
-        } else if (kLibPair) {
-            for (int e = warp; e < a.L * E * E; e += W) {
-                const uint16_t* cb = b.cb + (size_t)(e >> (2 * N)) * E;
-                *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(cb + (e & (E - 1))) | ((uint32_t)__ldg(cb + ((e >> N) & (E - 1))) << 16);
+        }
+        for (int e0 = warp * 32; kShuffleFill && e0 < trows; e0 += W * 32) {
+            const int e = e0 + lane;
+            uint32_t word = 0u;
+            if (e < trows) {
+                if (kHalf) {
+                    const int m = e >> N, q = e & (E - 1);
+                    word = __ldg(b.cb + (size_t)(2 * m) * E + q);
+                    if (2 * m + 1 < a.L) word |= (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) << 16;
+                } else {
+                    const uint16_t* cb = b.cb + (size_t)(e >> (2 * N)) * E;
+                    word = (uint32_t)__ldg(cb + (e & (E - 1))) | ((uint32_t)__ldg(cb + ((e >> N) & (E - 1))) << 16);
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 32; ++r) {
+                const uint32_t v = __shfl_sync(0xffffffffu, word, r);
+                if (e0 + r < trows) *(uint32_t*)(tab + (size_t)(e0 + r) * 128 + lane * 4) = v;
             }
         }
         }
