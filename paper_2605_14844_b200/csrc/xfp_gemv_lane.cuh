@@ -122,6 +122,154 @@ __host__ __device__ constexpr int last_step_of_vector(int v) {
     return (128 * (v + 1) - 1) / (8 * N);
 }
 
+// V2 tables of one row-block: warp w fills entries [w T / W, (w+1) T / W) of every lane's channel (the table shapes are
+// listed at the top of xfp_gemv_lane.cu).  `cbs`: scratch for the block's codebooks (N >= 5).  Every thread of the CTA
+// calls it (N >= 5 has a barrier inside).
+template <int N, int W, bool SGL>
+__device__ __forceinline__ void fill_tables_v2(unsigned char* tab, uint32_t* cbs, const Blob& b, int blk, int warp, int lane) {
+    using C = LaneCfg<N, SGL, 0>;
+    constexpr int E = C::E;
+    constexpr int T = C::T;
+    constexpr int kStride = C::kStride;
+    constexpr int kThreads = W * 32;
+    const uint16_t* cb = b.cb + (size_t)(blk * kRowsPerBlock + lane) * E;
+    if constexpr (C::kQuad) {
+        // entry t = (cb[t & 3], cb[t >> 2 & 3], cb[t >> 4 & 3], cb[t >> 6]) as 8 bytes at t * 256 + lane * 8
+        const uint2 c4 = __ldg((const uint2*)cb);   // the four entries
+        const uint32_t e0 = c4.x & 0xffffu, e1 = c4.x >> 16, e2 = c4.y & 0xffffu, e3 = c4.y >> 16;
+        auto ent = [&](int q) { return q == 0 ? e0 : (q == 1 ? e1 : (q == 2 ? e2 : e3)); };
+        // entries t = 16 h + i: the high half (indices 2, 3 of the byte) is the same for sixteen entries and is
+        // picked once; the low half runs over all sixteen pairs with compile-time picks (selecting all four values
+        // of every entry at run time made this fill 1.15 us, the longest prologue of all widths)
+        const uint32_t eh[4] = {e0 << 16, e1 << 16, e2 << 16, e3 << 16};
+        const uint32_t el[4] = {e0, e1, e2, e3};
+        constexpr int TW = T / W;
+        static_assert(TW % 16 == 0, "a warp fills whole groups of sixteen entries");
+#pragma unroll
+        for (int gq = 0; gq < TW / 16; ++gq) {
+            const int h = warp * (TW / 16) + gq;
+            const uint32_t hi = ent(h & 3) | (ent(h >> 2) << 16);
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                *(uint2*)(tab + (size_t)(h * 16 + i) * kStride + lane * 8) = make_uint2(el[i & 3] | eh[i >> 2], hi);
+        }
+    } else if constexpr (C::kSingle && (T / W == 2 || T / W == 4 || T / W == 8)) {
+        // a warp's TW consecutive entries of every channel in ONE load per lane (2, 4 or 8 entries: 4, 8 or 16 bytes;
+        // one 2-byte load per entry made four requests of 32 sectors each and the fill 1.2 us at N = 6)
+        constexpr int TW = T / W;
+        uint32_t cw[TW / 2];
+        if (TW == 2) {
+            cw[0] = __ldg((const uint32_t*)(cb + warp * TW));
+        } else if (TW == 4) {
+            const uint2 t = __ldg((const uint2*)(cb + warp * TW));
+            cw[0] = t.x; cw[TW / 2 - 1] = t.y;
+        } else {
+            const uint4 t = __ldg((const uint4*)(cb + warp * TW));
+            cw[0] = t.x; cw[1 % (TW / 2)] = t.y; cw[2 % (TW / 2)] = t.z; cw[3 % (TW / 2)] = t.w;
+        }
+#pragma unroll
+        for (int i = 0; i < TW; ++i) {
+            const int t = warp * TW + i;
+            *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (i & 1) ? (cw[i >> 1] >> 16) : (cw[i >> 1] & 0xffffu);
+        }
+    } else if (C::kSingle) {   // (instantiated for V2a widths only, where this branch is never taken)
+        constexpr int TW = T / W > 0 ? T / W : 1;
+#pragma unroll
+        for (int i = 0; i < TW; ++i) {
+            const int t = warp * TW + i;
+            if (t < T) *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (uint32_t)__ldg(cb + t);
+        }
+    } else if (T / W >= E) {
+        // a warp fills whole rows of the pair matrix: entries (hi, 0..E-1) for its values of hi.  Every warp needs
+        // every entry of its lanes' channels: the block's codebooks (32 E fp16, contiguous) are fetched once with
+        // coalesced loads and transposed through shared memory, instead of 16-byte loads 2 E bytes apart by every warp.
+        constexpr int HW = T / W / E;   // values of the high index per warp
+        constexpr bool kStage = N >= kLaneStageCodebooksFrom;
+        uint32_t cw[E / 2];
+        if (kStage) {
+            const uint4* src = (const uint4*)(b.cb + (size_t)blk * kRowsPerBlock * E);
+            for (int i = threadIdx.x; i < 4 * E; i += kThreads) {
+                const uint4 t = __ldg(src + i);
+                const int ch = i / (E / 8), w4 = (i % (E / 8)) * 4;
+                cbs[(w4 + 0) * 32 + ch] = t.x; cbs[(w4 + 1) * 32 + ch] = t.y;
+                cbs[(w4 + 2) * 32 + ch] = t.z; cbs[(w4 + 3) * 32 + ch] = t.w;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < E / 2; ++i) cw[i] = cbs[i * 32 + lane];
+        } else {
+#pragma unroll
+            for (int i = 0; i < E / 8; ++i) {
+                const uint4 t = __ldg((const uint4*)cb + i);
+                cw[4 * i] = t.x; cw[4 * i + 1] = t.y; cw[4 * i + 2] = t.z; cw[4 * i + 3] = t.w;
+            }
+        }
+#pragma unroll
+        for (int hh = 0; hh < HW; ++hh) {
+            const int hi = warp * HW + hh;
+            const uint32_t hv = (kStage ? (uint32_t)((const uint16_t*)cbs)[((hi >> 1) * 32 + lane) * 2 + (hi & 1)]
+                                        : (uint32_t)__ldg(cb + hi)) << 16;
+#pragma unroll
+            for (int lo = 0; lo < E; ++lo) {
+                const uint32_t lv = (lo & 1) ? (cw[lo >> 1] >> 16) : (cw[lo >> 1] & 0xffffu);
+                *(uint32_t*)(tab + (size_t)(hi * E + lo) * kStride + lane * 4) = lv | hv;
+            }
+        }
+    } else {
+        // few entries per warp (N = 3: 64 entries over 16 warps)
+        constexpr int TW = T / W > 0 ? T / W : 1;
+#pragma unroll
+        for (int i = 0; i < TW; ++i) {
+            const int t = warp * TW + i;
+            if (t < T) {
+                const uint32_t lv = __ldg(cb + (t & (E - 1))), hv = __ldg(cb + (t >> N));
+                *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = lv | (hv << 16);
+            }
+        }
+    }
+}
+
+// V2a tables: every row is one word repeated in the 32 banks -- HALF: row (id / 2) * 2^N + q holds lib[id][q] of ids
+// 2m (low half) and 2m + 1 (high half); else the pair table, row id * 4^N + (q1 << N | q0) holds (lib[id][q0],
+// lib[id][q1]).  A lane fetches the word of row e0 + lane, then the warp stores the 32 rows one after the other, each word
+// handed round by a shuffle (a warp that fetched two halves per row with uniform loads paid their latency once per
+// row: 3.9 us for the 1024 rows of N = 6).  Not inlined: inside the kernel the unrolled stores changed the register
+// allocation of the K loop (N = 3, 4: 62.2 against 58.3 us at 28672 x 8192).
+template <int N, int W, bool HALF>
+__device__ __noinline__ void fill_library(unsigned char* tab, const uint16_t* __restrict__ lib, int L, int warp, int lane) {
+    constexpr int E = 1 << N;
+    const int trows = HALF ? ((L + 1) >> 1) * E : L * E * E;
+    if (HALF && trows < 32 * W) {
+        // a small table (N = 3, 4 at L = 32): one row per warp and step, so that every warp takes part
+        for (int e = warp; e < trows; e += W) {
+            const int m = e >> N, q = e & (E - 1);
+            const uint32_t lo = __ldg(lib + (size_t)(2 * m) * E + q);
+            const uint32_t hi = 2 * m + 1 < L ? (uint32_t)__ldg(lib + (size_t)(2 * m + 1) * E + q) : 0u;
+            *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = lo | (hi << 16);
+        }
+        return;
+    }
+    for (int e0 = warp * 32; e0 < trows; e0 += W * 32) {
+        const int e = e0 + lane;
+        uint32_t word = 0u;
+        if (e < trows) {
+            if (HALF) {
+                const int m = e >> N, q = e & (E - 1);
+                word = __ldg(lib + (size_t)(2 * m) * E + q);
+                if (2 * m + 1 < L) word |= (uint32_t)__ldg(lib + (size_t)(2 * m + 1) * E + q) << 16;
+            } else {
+                const uint16_t* cb = lib + (size_t)(e >> (2 * N)) * E;
+                word = (uint32_t)__ldg(cb + (e & (E - 1))) | ((uint32_t)__ldg(cb + ((e >> N) & (E - 1))) << 16);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+            const uint32_t v = __shfl_sync(0xffffffffu, word, r);
+            if (e0 + r < trows) *(uint32_t*)(tab + (size_t)(e0 + r) * 128 + lane * 4) = v;
+        }
+    }
+}
+
 // MODE 0: V2 (the channel's own codebook, tables private to the lane).  MODE 1: V2a -- the whole library replicated
 // once per bank (word ((id / 2) * 2^N + q) * 32 + lane holds lib[id][q] in its half id % 2; pair tables of every
 // entry where those fit), the table base of a lane follows the library id
@@ -253,137 +401,24 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     // ---- tables: warp w fills entries [w T / W, (w+1) T / W) of every lane's channel
     if (MODE != 0) {
         if (!kMulti || it == 0) {   // one library per blob: a resident CTA fills it once
-        // every row of the table is one word repeated in the 32 banks: a lane fetches the word of row e0 + lane, then
-        // the warp stores the 32 rows one after the other, each word handed round by a shuffle (a warp that fetched
-        // two halves per row with uniform loads paid their latency once per row: 3.9 us for the 1024 rows of N = 6)
-        const int trows = kHalf ? ((a.L + 1) >> 1) * E : a.L * E * E;
-        // (tables of up to 8 rows per warp keep the plain loop: with the shuffle form the same K loop ran 6 % slower at
-        // N = 3 and 4 -- 62.2 against 58.3 us at 28672 x 8192 -- through the compiler's register allocation)
-        constexpr bool kShuffleFill = N >= 5 || kLibPair;
-        if (!kShuffleFill) {
-            for (int e = warp; e < trows; e += W) {
+        if constexpr (N >= 5 || kLibPair || W == 8) {
+            fill_library<N, W, kHalf>(tab, b.cb, a.L, warp, lane);
+        } else {
+            // small tables in a CTA that has its SM to itself: inline, so that the index loads issued above stay in
+            // flight (registers that are the target of a load are written back around a call, which waits for them:
+            // 4096 x 4096, N = 4: 6.99 against 6.66 us)
+            for (int e = warp; e < ((a.L + 1) >> 1) * E; e += W) {
                 const int m = e >> N, q = e & (E - 1);
                 const uint32_t lo = __ldg(b.cb + (size_t)(2 * m) * E + q);
                 const uint32_t hi = 2 * m + 1 < a.L ? (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) : 0u;
                 *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = lo | (hi << 16);
             }
         }
-        for (int e0 = warp * 32; kShuffleFill && e0 < trows; e0 += W * 32) {
-            const int e = e0 + lane;
-            uint32_t word = 0u;
-            if (e < trows) {
-                if (kHalf) {
-                    const int m = e >> N, q = e & (E - 1);
-                    word = __ldg(b.cb + (size_t)(2 * m) * E + q);
-                    if (2 * m + 1 < a.L) word |= (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) << 16;
-                } else {
-                    const uint16_t* cb = b.cb + (size_t)(e >> (2 * N)) * E;
-                    word = (uint32_t)__ldg(cb + (e & (E - 1))) | ((uint32_t)__ldg(cb + ((e >> N) & (E - 1))) << 16);
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < 32; ++r) {
-                const uint32_t v = __shfl_sync(0xffffffffu, word, r);
-                if (e0 + r < trows) *(uint32_t*)(tab + (size_t)(e0 + r) * 128 + lane * 4) = v;
-            }
-        }
         }
     } else {
-        const uint16_t* cb = b.cb + (size_t)(blk * kRowsPerBlock + lane) * E;
-        if constexpr (C::kQuad) {
-            // entry t = (cb[t & 3], cb[t >> 2 & 3], cb[t >> 4 & 3], cb[t >> 6]) as 8 bytes at t * 256 + lane * 8
-            const uint2 c4 = __ldg((const uint2*)cb);   // the four entries
-            const uint32_t e0 = c4.x & 0xffffu, e1 = c4.x >> 16, e2 = c4.y & 0xffffu, e3 = c4.y >> 16;
-            auto ent = [&](int q) { return q == 0 ? e0 : (q == 1 ? e1 : (q == 2 ? e2 : e3)); };
-            // entries t = 16 h + i: the high half (indices 2, 3 of the byte) is the same for sixteen entries and is
-            // picked once; the low half runs over all sixteen pairs with compile-time picks (selecting all four values
-            // of every entry at run time made this fill 1.15 us, the longest prologue of all widths)
-            const uint32_t eh[4] = {e0 << 16, e1 << 16, e2 << 16, e3 << 16};
-            const uint32_t el[4] = {e0, e1, e2, e3};
-            constexpr int TW = T / W;
-            static_assert(TW % 16 == 0, "a warp fills whole groups of sixteen entries");
-#pragma unroll
-            for (int gq = 0; gq < TW / 16; ++gq) {
-                const int h = warp * (TW / 16) + gq;
-                const uint32_t hi = ent(h & 3) | (ent(h >> 2) << 16);
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    *(uint2*)(tab + (size_t)(h * 16 + i) * kStride + lane * 8) = make_uint2(el[i & 3] | eh[i >> 2], hi);
-            }
-        } else if constexpr (C::kSingle && (T / W == 2 || T / W == 4 || T / W == 8)) {
-            // a warp's TW consecutive entries of every channel in ONE load per lane (2, 4 or 8 entries: 4, 8 or 16 bytes;
-            // one 2-byte load per entry made four requests of 32 sectors each and the fill 1.2 us at N = 6)
-            constexpr int TW = T / W;
-            uint32_t cw[TW / 2];
-            if (TW == 2) {
-                cw[0] = __ldg((const uint32_t*)(cb + warp * TW));
-            } else if (TW == 4) {
-                const uint2 t = __ldg((const uint2*)(cb + warp * TW));
-                cw[0] = t.x; cw[TW / 2 - 1] = t.y;
-            } else {
-                const uint4 t = __ldg((const uint4*)(cb + warp * TW));
-                cw[0] = t.x; cw[1 % (TW / 2)] = t.y; cw[2 % (TW / 2)] = t.z; cw[3 % (TW / 2)] = t.w;
-            }
-#pragma unroll
-            for (int i = 0; i < TW; ++i) {
-                const int t = warp * TW + i;
-                *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (i & 1) ? (cw[i >> 1] >> 16) : (cw[i >> 1] & 0xffffu);
-            }
-        } else if (C::kSingle) {   // (instantiated for V2a widths only, where this branch is never taken)
-            constexpr int TW = T / W > 0 ? T / W : 1;
-#pragma unroll
-            for (int i = 0; i < TW; ++i) {
-                const int t = warp * TW + i;
-                if (t < T) *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = (uint32_t)__ldg(cb + t);
-            }
-        } else if (T / W >= E) {
-            // a warp fills whole rows of the pair matrix: entries (hi, 0..E-1) for its values of hi.  Every warp needs
-            // every entry of its lanes' channels: the block's codebooks (32 E fp16, contiguous) are fetched once with
-            // coalesced loads and transposed through shared memory, instead of 16-byte loads 2 E bytes apart by every warp.
-            constexpr int HW = T / W / E;   // values of the high index per warp
-            constexpr bool kStage = N >= kLaneStageCodebooksFrom;
-            uint32_t cw[E / 2];
-            if (kStage) {
-                const uint4* src = (const uint4*)(b.cb + (size_t)blk * kRowsPerBlock * E);
-                for (int i = threadIdx.x; i < 4 * E; i += kThreads) {
-                    const uint4 t = __ldg(src + i);
-                    const int ch = i / (E / 8), w4 = (i % (E / 8)) * 4;
-                    cbs[(w4 + 0) * 32 + ch] = t.x; cbs[(w4 + 1) * 32 + ch] = t.y;
-                    cbs[(w4 + 2) * 32 + ch] = t.z; cbs[(w4 + 3) * 32 + ch] = t.w;
-                }
-                __syncthreads();
-#pragma unroll
-                for (int i = 0; i < E / 2; ++i) cw[i] = cbs[i * 32 + lane];
-            } else {
-#pragma unroll
-                for (int i = 0; i < E / 8; ++i) {
-                    const uint4 t = __ldg((const uint4*)cb + i);
-                    cw[4 * i] = t.x; cw[4 * i + 1] = t.y; cw[4 * i + 2] = t.z; cw[4 * i + 3] = t.w;
-                }
-            }
-#pragma unroll
-            for (int hh = 0; hh < HW; ++hh) {
-                const int hi = warp * HW + hh;
-                const uint32_t hv = (kStage ? (uint32_t)((const uint16_t*)cbs)[((hi >> 1) * 32 + lane) * 2 + (hi & 1)]
-                                            : (uint32_t)__ldg(cb + hi)) << 16;
-#pragma unroll
-                for (int lo = 0; lo < E; ++lo) {
-                    const uint32_t lv = (lo & 1) ? (cw[lo >> 1] >> 16) : (cw[lo >> 1] & 0xffffu);
-                    *(uint32_t*)(tab + (size_t)(hi * E + lo) * kStride + lane * 4) = lv | hv;
-                }
-            }
-        } else {
-            // few entries per warp (N = 3: 64 entries over 16 warps)
-            constexpr int TW = T / W > 0 ? T / W : 1;
-#pragma unroll
-            for (int i = 0; i < TW; ++i) {
-                const int t = warp * TW + i;
-                if (t < T) {
-                    const uint32_t lv = __ldg(cb + (t & (E - 1))), hv = __ldg(cb + (t >> N));
-                    *(uint32_t*)(tab + (size_t)t * kStride + lane * 4) = lv | (hv << 16);
-                }
-            }
-        }
+        // inlined: behind a call (as the V2a fill of the 8-warp CTAs is) the same K loops ran 7-11 % slower
+        // (28672 x 8192: N = 4 36.9 against 34.1 us, N = 5 55.6 against 49.9 us)
+        fill_tables_v2<N, W, SGL>(tab, cbs, b, blk, warp, lane);
     }
 
     // ---- x may come from the previous kernel of the stream
