@@ -258,9 +258,16 @@ __global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1) gemv_v2a_kernel(const 
                     ((uint4*)(tab + (size_t)e * 64))[t & 3] = make_uint4(v, v, v, v);
                 }
             } else {
-                // one copy per bank: word (e * 32 + lane) = lib[e] for every lane
-                for (int e = warp; e < a.L * E; e += kAWarps)
-                    *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = (uint32_t)__ldg(b.cb + e);
+                // one copy per bank: word (e * 32 + lane) = lib[e] for every lane.  A lane fetches entry e0 + lane, the warp
+                // stores 32 rows, the entries handed round by shuffle (one uniform load per row paid its latency per row)
+                for (int e0 = warp * 32; e0 < a.L * E; e0 += kAWarps * 32) {
+                    const uint32_t mine = e0 + lane < a.L * E ? (uint32_t)__ldg(b.cb + e0 + lane) : 0u;
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        const uint32_t v = __shfl_sync(0xffffffffu, mine, r);
+                        if (e0 + r < a.L * E) *(uint32_t*)(tab + (size_t)(e0 + r) * 128 + lane * 4) = v;
+                    }
+                }
             }
             have_tables = true;
         }
