@@ -407,11 +407,26 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
             // small tables in a CTA that has its SM to itself: inline, so that the index loads issued above stay in
             // flight (registers that are the target of a load are written back around a call, which waits for them:
             // 4096 x 4096, N = 4: 6.99 against 6.66 us)
-            for (int e = warp; e < ((a.L + 1) >> 1) * E; e += W) {
-                const int m = e >> N, q = e & (E - 1);
-                const uint32_t lo = __ldg(b.cb + (size_t)(2 * m) * E + q);
-                const uint32_t hi = 2 * m + 1 < a.L ? (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) : 0u;
-                *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = lo | (hi << 16);
+            if (a.L == 32) {
+                // the paper's library size: a known trip count, so that all of a warp's loads are in flight at once
+                constexpr int kRows = 16 * E / W;
+                uint32_t lo[kRows], hi[kRows];
+#pragma unroll
+                for (int i = 0; i < kRows; ++i) {
+                    const int e = warp + i * W, m = e >> N, q = e & (E - 1);
+                    lo[i] = __ldg(b.cb + (size_t)(2 * m) * E + q);
+                    hi[i] = __ldg(b.cb + (size_t)(2 * m + 1) * E + q);
+                }
+#pragma unroll
+                for (int i = 0; i < kRows; ++i)
+                    *(uint32_t*)(tab + (size_t)(warp + i * W) * 128 + lane * 4) = lo[i] | (hi[i] << 16);
+            } else {
+                for (int e = warp; e < ((a.L + 1) >> 1) * E; e += W) {
+                    const int m = e >> N, q = e & (E - 1);
+                    const uint32_t lo = __ldg(b.cb + (size_t)(2 * m) * E + q);
+                    const uint32_t hi = 2 * m + 1 < a.L ? (uint32_t)__ldg(b.cb + (size_t)(2 * m + 1) * E + q) : 0u;
+                    *(uint32_t*)(tab + (size_t)e * 128 + lane * 4) = lo | (hi << 16);
+                }
             }
         }
         }
