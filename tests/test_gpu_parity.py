@@ -191,6 +191,21 @@ def test_several_rows_of_x_with_resident_ctas_and_a_cut_tail(mode, bits, rows, c
     assert int(tickets.abs().sum().item()) == 0
 
 
+@pytest.mark.parametrize("bits,lib_size", [(2, 1), (2, 7), (2, 33), (2, 64), (3, 5), (4, 1), (4, 33), (4, 64), (4, 200),
+                                           (5, 31), (6, 7), (6, 33), (6, 64)])
+def test_v2a_library_sizes(bits, lib_size):
+    """Library sizes other than the paper's 32: odd counts (the last table word holds one id), a single entry, sizes
+    whose tables outgrow shared memory and fall to other kernels; batch 1 and 4, two shapes (a matrix of one round of
+    CTAs and one of several), reconstruction bit-exact."""
+    for rows, cols in ((2500, 512), (9600, 256)):
+        q = synth.random_quantized(1, rows, cols, bits, 0.01, seed=9900 + 10 * bits + lib_size, lib_size=lib_size)
+        pm = xfp.pack_tensors(q, col_bits=16)
+        sample = _sample_rows(rows, 64, seed=9901)
+        for batch in (1, 4):
+            _check_gemv(q, pm, synth.activations(batch, cols, seed=9910 + batch), rows=sample)
+    _check_dequant(q, pm)
+
+
 @pytest.mark.parametrize("mode,bits", [(0, 4), (0, 5), (1, 3), (1, 4)])
 def test_longest_rows(mode, bits):
     """K = 65536, the largest the descriptor admits (u16 outlier columns): x alone is 128 KB per batch row."""
