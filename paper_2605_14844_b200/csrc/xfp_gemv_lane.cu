@@ -150,7 +150,7 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
 
 template <int N, int W, int MINB, bool SGL, int MODE>
 cudaError_t launch_lane(const LaneArgs& a, int grid, size_t smem, cudaStream_t s) {
-    if (a.x_bf16 || a.y_is_fp16 == 2) return launch_lane_io<N, W, MINB, SGL, MODE, true, 1>(a, grid, smem, s);
+    if (a.x_bf16 || a.y_is_fp16 == 2 || a.packed_list) return launch_lane_io<N, W, MINB, SGL, MODE, true, 1>(a, grid, smem, s);
     return launch_lane_io<N, W, MINB, SGL, MODE, false, 1>(a, grid, smem, s);
 }
 

@@ -277,7 +277,10 @@ __device__ __noinline__ void fill_library(unsigned char* tab, const uint16_t* __
 // sum moves to the lane that owns the channel and is folded into its accumulator with the group's scale and
 // mid-point:  acc += scale * G + mid * X_g,  X_g = sum of x over the group ("V2a: Shared Codebook Library").
 // TIO instantiations take bf16 x and store bf16 y; compiled into the plain ones the conversion cost the fp16 path 4.5 %
-// at 28672 x 8192 through register allocation alone (34.3 against 32.8 us), so only bf16 calls launch them.
+// at 28672 x 8192 through register allocation alone (34.3 against 32.8 us), so only bf16 calls launch them.  The same
+// instantiations serve launches over several blobs (pointer lists): with the list branch compiled into the plain
+// ones, the blob's pointers were run-time values instead of kernel parameters and 12288 x 4096 at N = 2 took 11.8
+// against 8.4 us.
 // NB rows of x (1, 2, 4 or 8): every decoded fragment is multiplied with the B fragment of each row, so the look-ups
 // are paid once per weight; a CTA then stays resident and walks several row-blocks with one staged copy of x.
 template <int N, int W, int MINB, bool SGL, int MODE, bool TIO, int NB>
@@ -306,7 +309,9 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     const int K = a.SC * kSuper;
     const size_t xrow = (size_t)K * 2;             // bytes of one staged row of x
     unsigned char* tab = smem;
-    unsigned char* xs = smem + a.tab_bytes;
+    // V2, N >= 4: a compile-time offset (4096 x 4096, N = 5: 4.70 against 4.86 us; at N = 3 the same change cost 6 % at
+    // 12288 x 4096 through register allocation, so N <= 3 keeps the run-time one)
+    unsigned char* xs = smem + (MODE == 0 && N >= 4 ? C::kTabBytes : a.tab_bytes);
     float* red = (float*)(xs + NB * xrow);         // [NB][W][32]
     float* xg = red + NB * W * 32;                 // V2a: [NB][SC][2] sums of x over the halves of every super-chunk
     uint32_t* cbs = (uint32_t*)xg;                 // V2 pair tables: the block's codebooks, word [e / 2][channel]
@@ -357,7 +362,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
     const uint16_t* xsrc = a.x;
     void* ydst = a.y;
     int ell_slots = a.ell_slots;
-    if (a.packed_list) {
+    if (TIO && a.packed_list) {
         const int prob = blk / a.RB;
         blk -= prob * a.RB;
         packed = a.packed_list[prob];
@@ -387,7 +392,7 @@ __global__ void __launch_bounds__(W * 32, MINB) gemv_lane_kernel(const LaneArgs 
         gid_c[0] = b.gid[m0 + (size_t)warp * GH * 32]; gsm_c[0] = b.gsm[m0 + (size_t)warp * GH * 32];
         gid_c[1] = b.gid[m0 + ((size_t)warp * GH + GH - 1) * 32]; gsm_c[1] = b.gsm[m0 + ((size_t)warp * GH + GH - 1) * 32];
     }
-    const uint32_t* ell = a.packed_list
+    const uint32_t* ell = (TIO && a.packed_list)
         ? (const uint32_t*)((const char*)packed + *(const long long*)((const char*)packed + a.off.hdr + 8)) : b.ell;
     const uint32_t* slab = ell + (size_t)blk * (ell_slots + 1) * 32 + lane;
     uint32_t olen = ell_slots ? __ldg(slab) : 0u;
