@@ -132,7 +132,8 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
         // Pair tables of the whole library where they fit the same 64 KB (L * 4^N <= 512: N = 2 with the paper's L = 32).
         const bool pairs = (size_t)l.L * l.E * l.E * 128 <= 64 * 1024 && l.bits <= 3;
         const bool two = lane_tab_bytes(l, !pairs) <= 64 * 1024 && RB > sms;
-        LaneConfig c{two ? 8 : 16, two ? 2 : 1, !pairs};
+        // (pair tables between two and four rounds: 16 warps, 12288 x 4096 at N = 2 13.8 against 14.4 us)
+        LaneConfig c{two && !(pairs && RB > 2 * sms && RB <= 4 * sms) ? 8 : 16, two ? 2 : 1, !pairs};
         c.tiers = RB > 4 * sms;   // up to four rounds unsplit, as in V2 (N = 6, one CTA per SM: 12288 x 4096 33.6 -> 26.6 us)
         c.off = false;
         // the blobs of a routed layer in one launch: the resident CTAs of xfp_gemv_v2a.cu (pair tables built once per
@@ -142,7 +143,11 @@ LaneConfig lane_config(const Layout& l, int n = 1) {
     }
     if (RB <= sms) return LaneConfig{16, 1, l.bits == 6};
     const bool big = RB > 4 * sms;
-    LaneConfig c{(!big && (l.bits == 3 || l.bits == 4)) ? 16 : 8, 2, l.bits >= 5};
+    // 16 warps at N = 3, 4 only beyond one round of slots: in a single round 8 warps measured faster (8192 x 8192,
+    // N = 4: 10.7 against 11.5 us)
+    // N = 2 on short rows in a single round: the 64 KB fill dominates and 16 warps share it (8192 x 4096: 5.8 against 7.7 us)
+    const bool w16 = !big && (RB > 2 * sms ? (l.bits == 3 || l.bits == 4) : (l.bits == 2 && l.SC <= 32));
+    LaneConfig c{w16 ? 16 : 8, 2, l.bits >= 5};
     c.off = big && l.bits <= 3;   // the two-channels-per-lane kernel is ahead there
     c.tiers = big;
     return c;
