@@ -107,9 +107,9 @@ int xfp_pack(const xfp_desc* desc, const uint8_t* idx, const uint16_t* codebook,
  * Products are exact in fp32 and accumulated in fp32; the summation order is fixed, so repeated
  * calls give identical bits.  workspace/workspace_bytes as returned by xfp_packed_size.
  * Which kernel serves a call depends on shape, bit width, batch and outlier count only (never on the data): batch 1
- * runs on a kernel with one channel per lane, 2..12 rows of x on kernels that decode once per 8 rows, and from 13
- * rows (9 for V2a) a blob with at most 1 % outliers may run on the tensor-core kernel of xfp_gemm, which multiplies
- * with W^ = fp16(D16 + S) instead of the unrounded D + S; both lie inside the bound the tests hold every kernel to
+ * runs on a kernel with one channel per lane, 2..8 rows of x on kernels that decode once per 8 rows, and from 9
+ * rows a large blob with at most 2 % outliers may run on the tensor-core kernel of xfp_gemm (D16 on the tensor cores,
+ * S as a sparse product, both accumulated in fp32); every kernel lies inside the bound the tests hold them to
  * (|y - y_ref| <= 1e-3 * sum_k |W_ik x_k|). */
 int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
                 int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);
@@ -174,7 +174,11 @@ int xfp_gemv_grouped_typed(const xfp_desc* desc, int32_t n, const void* const* p
  * dequantised tile, GEMM on the tensor cores; the paper's split-M path for many rows of x):
  *     y[t][i] = sum_k W^[i][k] * x[t][k],   W^ = fp16(D16 + S), the matrix xfp_dequant writes,
  * for m >= 1 rows of x in one launch on the tcgen05 tensor cores (fp16 x fp16 products, fp32 accumulation in tensor
- * memory, one rounding of the sum to y_type).  V2 blobs, every N; V2a blobs whose library, replicated once per
+ * memory, one rounding of the sum to y_type).  Up to 64 rows of x the outliers are not added to the decoded tile:
+ * the tensor cores multiply D16 and the kernel adds sum_k S_ik x[t][k] to the accumulator in fp32, entries in
+ * ascending column order (y = (D16 + S) x without the fp16 rounding of the sum, as in xfp_gemv; the activations of
+ * that sparse product come from a transposed copy of x which a small kernel writes into the workspace first).
+ * V2 blobs, every N; V2a blobs whose library, replicated once per
  * shared-memory bank, fits 128 KB (lib_size * 2^bits <= 1024: L = 32 up to N = 5), else XFP_ERR_UNSUPPORTED.
  *   x  [m][cols] fp16;  y  [m][rows] of y_type (XFP_T_F32, XFP_T_F16 or XFP_T_BF16)
  *   workspace  xfp_gemm_workspace_size(desc, m) bytes, zero-filled once before first use; its counter part is left

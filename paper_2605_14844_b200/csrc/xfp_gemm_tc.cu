@@ -18,16 +18,23 @@
 //            to N = 3, one entry per index above).  V2a: the library replicated once per bank, then
 //            D16 = fp16(fp32(scale * lib[id][q] + mid)) with the group's scale and mid-point.  The outliers of the
 //            lane's channel that fall into its half are added to the register that holds them with one correctly
-//            rounded fp16 addition each, so the tile is the matrix xfp_dequant writes.
+//            rounded fp16 addition each, so the tile is the matrix xfp_dequant writes.  Up to 64 rows of x the
+//            outliers stay out of the tile (the walk through a lane's list cost 37 - 50 us of 141 at 28672 x 8192
+//            with 0.3 % outliers): the epilogue adds S x^T to the accumulator instead, see below.
 //   mma      one thread waits for "A stage stored" (eight arrivals) and "x tile landed" (transaction bytes), issues
 //            eight m128 nT k16 instructions and commits them to a "products done" mbarrier; the decode of
 //            iteration i waits for the products of iteration i - 2, whose A stage it overwrites.  No CTA-wide
 //            barrier inside the loop.
 //   epilogue tcgen05.ld (lane = channel, registers = rows of x), direct store, or fp32 partials through the
 //            workspace when K is cut (few row tiles): the last CTA of a tile adds the slices in slice order.
+//            With the sparse outlier product, a thread first walks its channel's outliers inside the K slice and adds
+//            value * x[t][column] for its 16 rows of x in fp32, entries in ascending column order; the 16 activations
+//            are 32 contiguous bytes of a transposed copy of x that a small kernel writes before the launch.
 // Every wait on an mbarrier has an iteration limit; when one runs out the CTA stops issuing work, records it in
 // the first word of the workspace and leaves through the common exit that frees its tensor memory.
 #include <cuda.h>
+
+#include <cstdlib>
 
 #include <type_traits>
 
@@ -50,6 +57,11 @@ constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kAStageCols = 64;  // 128 k as fp16 pairs
 constexpr int kXStages = 3;      // x tiles in flight: the copy of iteration i + 1 is issued at the top of iteration i
 constexpr size_t kV2aTabMax = 128 * 1024;   // V2a: the per-bank library (L * 2^N * 128 bytes) must fit beside the x stages
+// Up to this many rows of x the outliers are a sparse product in the epilogue.  The product reads 32 bytes of the
+// transposed x per outlier and 16 rows, scattered through L2 at about 2.4 TB/s (28672 x 8192, 0.3 %: 13 us at 16 rows,
+// 19 at 32, 39 at 64, 78 at 128); the walk through the lists costs about as much per outlier as 64 rows of the product
+// whatever the rows (0.3 %: 45 - 50 us, 1 %: 114 us).
+constexpr int kSparseRows = 64;
 constexpr size_t kMinSmem = 80 * 1024;   // at most two CTAs per SM: each holds half of the tensor memory (a CTA with
                                          // 256-row tiles holds all of it and asks for more than half of the shared memory)
 
@@ -66,6 +78,10 @@ struct GemmArgs {
     int tmem_cols;    // tensor-memory columns of the CTA: 2 * maxT
     int x_stages;     // x tiles in shared memory: kXStages, or 2 when three large ones do not fit
     int b_half;       // bytes of one 64-k half of an x tile: rows of x per tile * 128 (a multiple of 1024)
+    // outliers as a sparse product in the epilogue (few rows of x): x transposed, [K][Mp] fp16 with Mp a multiple of 32
+    // and zeros behind row M; null: the decode warps add the outliers to the tile instead
+    const uint16_t* xT;
+    int Mp;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -173,6 +189,40 @@ struct Outliers {
         }
     }
 };
+
+// v[0..15] (fp32 bit patterns: the sums of one channel for 16 rows of x) += S x^T over the channel's outliers with
+// columns below `kend`, starting at entry o.cur: four entries and their activations in flight at a time, added in
+// ascending column order.
+__device__ __forceinline__ void sparse_rows(const GemmArgs& a, const Outliers& o, int t, uint32_t kend, uint32_t (&v)[16]) {
+    const uint16_t* xt = a.xT + t;
+    for (int j = o.cur; j < o.total; j += 4) {
+        uint32_t e[4];
+        bool ok[4];
+        uint4 xa[4], xb[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) e[u] = j + u < o.total ? o.fetch(j + u) : 0u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t col = e[u] & 0xffffu;
+            ok[u] = j + u < o.total && col < kend;
+            const uint4* p = (const uint4*)(xt + (size_t)(ok[u] ? col : 0u) * a.Mp);
+            xa[u] = __ldg(p); xb[u] = __ldg(p + 1);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (!ok[u]) continue;
+            const float val = __half2float(__ushort_as_half((uint16_t)(e[u] >> 16)));
+            const uint32_t xw[8] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w, xb[u].x, xb[u].y, xb[u].z, xb[u].w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float2 f = __half22float2(*(const __half2*)&xw[i]);
+                v[2 * i] = __float_as_uint(fmaf(val, f.x, __uint_as_float(v[2 * i])));
+                v[2 * i + 1] = __float_as_uint(fmaf(val, f.y, __uint_as_float(v[2 * i + 1])));
+            }
+        }
+        if (!ok[3]) break;
+    }
+}
 
 // One K slice of one half of the row-block's super-chunks: the whole main loop of a warp.
 // Barriers: bars[0..1] "products of iteration i done" (i & 1), bars[2..4] "x tile landed" (i % 3), bars[5..6] "A stage
@@ -458,7 +508,8 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
             for (int j = 0; j < 15; ++j) fine += (first + j < o.total) && (o.fetch(min(first + j, o.total - 1)) & 0xffffu) < kb;
             first += fine;
         }
-        o.start(first);
+        if (a.xT) { o.cur = first; o.col = 0xffffffffu; }   // the epilogue walks the list from `first`
+        else o.start(first);
     }
 
     const unsigned char* tab = MODE == 1 ? sTab : N == 4 ? sTab + (size_t)(q >> 1) * TW * 256 : sTab + (size_t)q * TW * 128;
@@ -482,6 +533,7 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
         for (int cc = part + 2 * grp; warp < DW && cc * 16 < Tn; cc += 2 * G) {
             uint32_t v[16];
             tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
+            if (a.xT && rb_ok) sparse_rows(a, o, t0 + cc * 16, (uint32_t)sc1 * kSuper, v);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const int t = cc * 16 + j;
@@ -541,6 +593,23 @@ EncodeTiledFn encode_tiled_fn() {
     return (EncodeTiledFn)fn;
 }
 
+// x [M][K] fp16 -> xT [K][Mp] fp16 (zeros behind row M): tiles of 32 rows x 64 k through shared memory.
+__global__ void __launch_bounds__(256) x_transpose_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ xT,
+                                                          int M, int K, int Mp) {
+    __shared__ uint16_t tile[64][34];   // [k][t]
+    const int tid = threadIdx.x, k0 = blockIdx.x * 64, t0 = blockIdx.y * 32;
+    for (int r = tid >> 5; r < 32; r += 8) {
+        const int t = t0 + r, kk = 2 * (tid & 31);
+        const uint32_t w = t < M ? __ldg((const uint32_t*)(x + (size_t)t * K + k0 + kk)) : 0u;
+        tile[kk][r] = (uint16_t)w; tile[kk + 1][r] = (uint16_t)(w >> 16);
+    }
+    __syncthreads();
+    for (int kk = tid >> 4; kk < 64; kk += 16) {
+        const int tt = 2 * (tid & 15);
+        *(uint32_t*)(xT + (size_t)(k0 + kk) * Mp + t0 + tt) = (uint32_t)tile[kk][tt] | ((uint32_t)tile[kk][tt + 1] << 16);
+    }
+}
+
 struct Plan {
     int row_tiles, tok_tiles, ks, sc_per_slice;
     int maxT, x_stages;
@@ -588,6 +657,9 @@ Plan plan_of(const Layout& l, int M, int sms) {
     // fewer tiles than CTA slots (two per SM): cut K, at least two super-chunks per slice
     const int slots = p.lone ? sms : 2 * sms;
     while (tiles * ks * 2 <= slots && l.SC / (ks * 2) >= 2) ks *= 2;
+#ifdef LANE_TUNE
+    if (const char* e = getenv("XFP_GEMM_KS")) ks = atoi(e);
+#endif
     p.sc_per_slice = (l.SC + ks - 1) / ks;
     p.ks = (l.SC + p.sc_per_slice - 1) / p.sc_per_slice;
     return p;
@@ -634,6 +706,13 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_half = b_half;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
     a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
+    a.xT = nullptr; a.Mp = (c.M + 31) & ~31;
+    const size_t xt_off = gemm_xt_offset(l, c.M), xt_bytes = gemm_xt_bytes(l, c.M);
+    if (xt_bytes && c.workspace_bytes >= xt_off + xt_bytes) {
+        uint16_t* xT = (uint16_t*)((char*)c.workspace + xt_off);
+        x_transpose_kernel<<<dim3((unsigned)(l.cols / 64), (unsigned)(a.Mp / 32)), 256, 0, s>>>(c.x, xT, c.M, l.cols, a.Mp);
+        a.xT = xT;
+    }
     const dim3 grid((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks);
     if (p.lone)
         gemm_tc_kernel<N, MODE, true><<<grid, threads_of(true), smem, s>>>(a, tmap);
@@ -654,10 +733,28 @@ size_t gemm_ctrl_bytes(const Layout& l, int M) {
     return align256((size_t)(1 + p.row_tiles * p.tok_tiles) * 4);
 }
 
-size_t gemm_workspace_bytes(const Layout& l, int M) {
+size_t gemm_core_bytes(const Layout& l, int M) {
     const Plan p = plan_of(l, M, kSizingSMs);
     const size_t partial = p.ks > 1 ? (size_t)p.row_tiles * p.tok_tiles * p.ks * p.maxT * kTileRows * 4 : 0;
     return gemm_ctrl_bytes(l, M) + partial;
+}
+
+// the transposed copy of x for the sparse outlier product: up to kSparseRows rows of x on a matrix with outliers
+size_t gemm_xt_bytes(const Layout& l, int M) {
+    if (l.nnz == 0 || M > kSparseRows) return 0;
+    return align256((size_t)l.cols * ((M + 31) & ~31) * 2);
+}
+
+// where the transposed copy starts: behind the counters and partial sums, and behind the counter region that the GEMV
+// kernels want left zero-filled (a batch sent here by xfp_gemv brings the GEMV's workspace)
+size_t gemm_xt_offset(const Layout& l, int M) {
+    const size_t core = align256(gemm_core_bytes(l, M)), tickets = align256((size_t)l.RB * 4);
+    return core > tickets ? core : tickets;
+}
+
+size_t gemm_workspace_bytes(const Layout& l, int M) {
+    const size_t xt = gemm_xt_bytes(l, M);
+    return xt ? gemm_xt_offset(l, M) + xt : gemm_core_bytes(l, M);
 }
 
 namespace {

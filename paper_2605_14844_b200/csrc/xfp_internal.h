@@ -1,6 +1,7 @@
 // Launchers shared between the translation units of libxfp.  Every launcher queues work on
 // `stream` and returns the cudaError_t of the launch.
 #pragma once
+#include <cstdlib>
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -106,7 +107,10 @@ struct GemmCall {
 };
 bool gemm_tc_supported(const Layout& l, int M);
 size_t gemm_ctrl_bytes(const Layout& l, int M);
-size_t gemm_workspace_bytes(const Layout& l, int M);
+size_t gemm_core_bytes(const Layout& l, int M);        // counters and the partial sums of K slices
+size_t gemm_xt_bytes(const Layout& l, int M);          // the transposed copy of x of the sparse outlier product (0: not used)
+size_t gemm_xt_offset(const Layout& l, int M);         // where that copy starts in the workspace
+size_t gemm_workspace_bytes(const Layout& l, int M);   // all of it
 cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s);
 // bf16 activations: converted to fp16 into a scratch area behind the GEMM's own workspace, then the same kernel
 size_t gemm_x_scratch_bytes(const Layout& l, int M);
@@ -122,18 +126,26 @@ cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaS
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);
-    return w > p ? w : p;
+    if (p > w) w = p;
+    // batches that go to the tensor-core kernel (up to 16 rows of x): room for its transposed copy of x behind the counters
+    const size_t g = l.nnz ? align256((size_t)l.RB * 4) + align256((size_t)l.cols * 64) : 0;
+    return w > g ? w : g;
 }
 
 inline bool batch_prefers_gemm(const Layout& l, int batch) {
-    if (batch < (l.mode ? 9 : 13) || !gemm_tc_supported(l, batch)) return false;
+    // 28672 x 8192 at 9 rows of x: V2 103 us against 124 (0.3 % outliers), 138 against 146 (2 %); V2a 120 against 210,
+    // 163 against 234; up to 8 rows the batched lane kernel is ahead (74 us in V2, 123 in V2a at 0.3 %)
+    int least = 9;
+#ifdef LANE_TUNE
+    if (const char* e = getenv("XFP_GEMM_MIN")) least = atoi(e);
+#endif
+    if (batch < least || !gemm_tc_supported(l, batch)) return false;
     // no K slices: the plan then uses a few counters at the start of the workspace and nothing else, inside the
     // region that every GEMV kernel leaves zero-filled
-    if (gemm_workspace_bytes(l, batch) > gemm_ctrl_bytes(l, batch) || gemm_ctrl_bytes(l, batch) > align256((size_t)l.RB * 4))
+    if (gemm_core_bytes(l, batch) > gemm_ctrl_bytes(l, batch) || gemm_ctrl_bytes(l, batch) > align256((size_t)l.RB * 4))
         return false;
-    // at most 1 % outliers (V2: 0.5 %; the batched mma.sync kernel overtakes the per-lane outlier walk earlier there:
-    // 28672 x 8192, 16 rows, 1 %: 159 against 206 us)
-    return l.nnz * (l.mode ? 100 : 200) <= (long long)l.rows * l.cols;
+    // at most 2 % outliers: the kernel adds them as a sparse product whose cost grows with their count
+    return l.nnz * 50 <= (long long)l.rows * l.cols;
 }
 
 }  // namespace xfp

@@ -1,8 +1,10 @@
 """Parity of the prefill form (xfp_gemm, tcgen05 tensor cores) against the CPU oracle, through the C ABI.
 
-Every row of x is one GEMV of the oracle: |y_ti - y_ref_ti| <= 1e-3 * sum_k |W_ik x_tk|.  The kernel multiplies
-the dequantised matrix W^ = fp16(D16 + S) (exact fp16 products, fp32 accumulation), so it is also held, far more
-tightly, to an fp64 product with the oracle's dequantised matrix.
+Every row of x is one GEMV of the oracle: |y_ti - y_ref_ti| <= 1e-3 * sum_k |W_ik x_tk|.  The kernel's products are
+exact and its sums fp32, so it is also held far more tightly to the matrix it multiplies: up to 128 rows of x that is
+D16 + S itself where the outliers are a sparse product added to the accumulator (few rows of x and few outliers),
+else the dequantised matrix W^ = fp16(D16 + S) (the outliers are added to the decoded tile); both are built from the
+oracle's dequantised matrices.
 """
 import os
 
@@ -35,6 +37,14 @@ def _run(q, pm, x16, dtype=torch.float32):
     return y, ws, xd
 
 
+def _sparse_product(pm, m):
+    """Whether xfp_gemm adds the outliers as a sparse product (few rows of x, few outliers), read off the workspace it
+    asks for: the transposed copy of x is the only part of it that depends on the outlier count."""
+    d = pm.desc
+    bare = xfp.XfpDesc(d.mode, d.rows, d.cols, d.bits, d.group_size, d.lib_size, d.col_bits, 0)
+    return xfp.xfp_gemm_workspace_size(d, m) > xfp.xfp_gemm_workspace_size(bare, m)
+
+
 def _check(q, pm, x16, dtype=torch.float32):
     y, _, _ = _run(q, pm, x16, dtype)
     got = y.float().cpu().numpy().astype(np.float64)
@@ -46,8 +56,18 @@ def _check(q, pm, x16, dtype=torch.float32):
     tol = TOL * absum + (2.0 ** -8 * np.abs(ref) if dtype == torch.bfloat16 else 0.0) + 1e-30
     assert np.all(err <= tol), float((err / tol).max())
     if dtype == torch.float32:
-        What = xo.dequant(mo).view(np.float16).astype(np.float64)
         xf = x16.view(np.float16).astype(np.float64)
+        if _sparse_product(pm, x16.shape[0]):
+            # D16 (the dequantised matrix of the blob without its outliers) + S, exactly
+            bare = xo.QuantizedMatrix(mo.mode, mo.rows, mo.cols, mo.bits, mo.idx, mo.codebook,
+                                      np.zeros(mo.rows + 1, np.int32), np.zeros(0, np.int32), np.zeros(0, np.uint16),
+                                      group_size=mo.group_size, lib_size=mo.lib_size, gid=mo.gid, gscale=mo.gscale,
+                                      gmid=mo.gmid)
+            What = xo.dequant(bare).view(np.float16).astype(np.float64)
+            rows_of = np.repeat(np.arange(mo.rows), np.diff(mo.rowptr))
+            np.add.at(What, (rows_of, mo.ocol), mo.oval.view(np.float16).astype(np.float64))
+        else:
+            What = xo.dequant(mo).view(np.float16).astype(np.float64)
         ref2 = xf @ What.T
         abs2 = np.abs(xf) @ np.abs(What).T
         err2 = np.abs(got - ref2)
@@ -98,6 +118,22 @@ def test_gemm_long_rows_and_spill():
     _check(q, xfp.pack_tensors(q, col_bits=16), synth.activations(20, q.cols, seed=70))
     q = synth.random_quantized(0, 64, 2048, 4, 0.01, seed=79, placement="clustered")
     _check(q, xfp.pack_tensors(q), synth.activations(20, q.cols, seed=71))
+
+
+@pytest.mark.parametrize("mode,bits,placement", [(0, 4, "one_row"), (0, 3, "clustered"), (1, 4, "one_row"), (1, 2, "uniform")])
+def test_gemm_outliers_as_a_sparse_product_and_in_the_tile(mode, bits, placement):
+    """The two ways the kernel adds S: a sparse product in the epilogue up to 64 rows of x (here 64, with K slices, a
+    ragged row-block and rows whose outliers fill the slab and spill into the CSR arrays), the scatter into the decoded
+    tile beyond (65 rows); the workspace size tells which, and each is held to the matrix it multiplies."""
+    q = synth.random_quantized(mode, 300, 2560, bits, 0.02, seed=1200 + bits + 10 * mode, placement=placement)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    assert _sparse_product(pm, 64) and not _sparse_product(pm, 65)
+    for m in (64, 65):
+        _check(q, pm, synth.activations(m, q.cols, seed=1210 + m))
+    bare = synth.random_quantized(mode, 300, 2560, bits, 0.0, seed=1230 + bits)
+    pmb = xfp.pack_tensors(bare, col_bits=16)
+    assert not _sparse_product(pmb, 16)
+    _check(bare, pmb, synth.activations(16, bare.cols, seed=1240))
 
 
 def test_gemm_matches_gemv_rows_and_is_deterministic():
