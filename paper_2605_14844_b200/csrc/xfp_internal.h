@@ -144,8 +144,8 @@ inline bool batch_prefers_gemm(const Layout& l, int batch) {
     // region that every GEMV kernel leaves zero-filled
     if (gemm_core_bytes(l, batch) > gemm_ctrl_bytes(l, batch) || gemm_ctrl_bytes(l, batch) > align256((size_t)l.RB * 4))
         return false;
-    // at most 2 % outliers: the kernel adds them as a sparse product whose cost grows with their count
-    return l.nnz * 50 <= (long long)l.rows * l.cols;
+    // at most 2.5 % outliers: the kernel adds them as a sparse product whose cost grows with their count
+    return l.nnz * 40 <= (long long)l.rows * l.cols;
 }
 
 }  // namespace xfp
