@@ -140,6 +140,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 
+// lo | hi << 16 for two table words whose upper halves are zero, as a multiply-add: the decode is bound by the ALU
+// pipe (PRMT, LOP3, SHF), and this moves one of its operations per two weights to the FMA pipe
+__device__ __forceinline__ uint32_t join16(uint32_t lo, uint32_t hi) {
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, 65536, %2;" : "=r"(d) : "r"(hi), "r"(lo));
+    return d;
+}
+
 template <int N>
 struct Tab {
     static constexpr int E = 1 << N;
@@ -316,11 +324,11 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                     const uint32_t sel = 0x5504u | ((uint32_t)(p & 3) << 4);
                     const uint32_t lo = *(const uint32_t*)(tab + __byte_perm(wlo, tbase, sel));
                     const uint32_t hi = *(const uint32_t*)(tab + __byte_perm(whi, tbase, sel));
-                    d[i] = __byte_perm(lo, hi, 0x5410u);
+                    d[i] = join16(lo, hi);
                 } else {
                     const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
                     const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
-                    d[i] = lo | (hi << 16);
+                    d[i] = join16(lo, hi);
                 }
             }
             // W^ = fp16(D16 + S) at the outliers of this channel inside this half; the entries of the other half
