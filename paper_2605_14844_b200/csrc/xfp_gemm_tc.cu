@@ -52,7 +52,8 @@ constexpr int kWarps = 8;        // decode warps of one group (row-block x half)
                                  // the tensor copies and the products.  256-row tiles (one CTA per SM) run two groups:
                                  // group g decodes the iterations with it % 2 == g, i.e. owns A stage g
 constexpr int threads_of(bool big) { return ((big ? 2 : 1) * kWarps + 1) * 32; }
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 20;   // polls of a bounded wait, each of at most kPollNs: about a second
+constexpr uint32_t kPollNs = 1000;
 // tensor memory of a CTA: the accumulator (128 or 256 columns), then the two A stages: 256 or 512 columns
 constexpr int kAStageCols = 64;  // 128 k as fp16 pairs
 constexpr int kXStages = 3;      // x tiles in flight: the copy of iteration i + 1 is issued at the top of iteration i
@@ -86,17 +87,25 @@ struct GemmArgs {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// A poll may suspend the thread for up to kPollNs before it answers (the hint of try_wait): a waiting warp then
+// issues a handful of instructions per microsecond instead of competing with the decode for the ALU pipe.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+            : "=r"(ok) : "r"(bar), "r"(parity), "r"(kPollNs) : "memory");
         if (ok) return true;
     }
     return false;
+}
+
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
 
 // Shared-memory operand descriptor (version 1) of a K-major tile in the 128-byte swizzle (rows of 64 fp16 = 128 bytes,
@@ -244,6 +253,12 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
     using H = Half<N, PART>;
     // byte offset of the lane inside a table entry; N = 4 (V2): the row-block's half of a 256-byte entry as well
     const uint32_t tbase = (uint32_t)lane * 4u + ((MODE == 0 && N == 4) ? (uint32_t)(q & 1) * 128u : 0u);
+    // V2: a row-block's table is aligned to its size in the shared window, so the entry field of an address and the
+    // table's own address do not overlap: the look-ups merge them (no addition per look-up) and load from the 32-bit
+    // shared address.  N = 4: the high nibble of address byte 1 rides in the index words.  (The same for V2a, whose
+    // look-ups are followed by a conversion, a multiply-add and a packing per weight, measured no faster.)
+    const uint32_t tabs = smem_u32(tab) + tbase;
+    const uint32_t nib = ((tabs >> 12) & 0xfu) * 0x10101010u;
     const uint4* idx = a.b.idx + ((size_t)rb * a.SC + sc0 + grp) * N * 32 + lane;   // advanced by G*N*32 per iteration of this warp
     // index vectors of the next two super-chunks in registers
     uint4 nx[2][H::NV];
@@ -316,18 +331,18 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
                     const __half2 r = __floats2half2_rn(f0, f1);
                     d[i] = *(const uint32_t*)&r;
                 } else if (Tab<N>::kPair) {
-                    d[i] = *(const uint32_t*)(tab + pair_addr<N, 1>(w, p, tbase));
+                    d[i] = lds32(pair_addr<N, 1>(w, p, tabs));
                 } else if (N == 4) {
                     // entries 256 bytes apart (two row-blocks share a table): an index, isolated in its own byte,
                     // becomes the second byte of the address with one PRMT.  Pair p = byte p & 3 of word p >> 2.
-                    const uint32_t wlo = w[p >> 2] & 0x0f0f0f0fu, whi = (w[p >> 2] >> 4) & 0x0f0f0f0fu;
-                    const uint32_t sel = 0x5504u | ((uint32_t)(p & 3) << 4);
-                    const uint32_t lo = *(const uint32_t*)(tab + __byte_perm(wlo, tbase, sel));
-                    const uint32_t hi = *(const uint32_t*)(tab + __byte_perm(whi, tbase, sel));
+                    const uint32_t wlo = (w[p >> 2] & 0x0f0f0f0fu) | nib, whi = ((w[p >> 2] >> 4) & 0x0f0f0f0fu) | nib;
+                    const uint32_t sel = 0x7604u | ((uint32_t)(p & 3) << 4);   // [tabs.b3, tabs.b2, index byte, tabs.b0]
+                    const uint32_t lo = lds32(__byte_perm(wlo, tabs, sel));
+                    const uint32_t hi = lds32(__byte_perm(whi, tabs, sel));
                     d[i] = join16(lo, hi);
                 } else {
-                    const uint32_t lo = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p, tbase));
-                    const uint32_t hi = *(const uint32_t*)(tab + single_addr<N, 1>(w, 2 * p + 1, tbase));
+                    const uint32_t lo = lds32(single_addr<N, 1>(w, 2 * p, tabs));
+                    const uint32_t hi = lds32(single_addr<N, 1>(w, 2 * p + 1, tabs));
                     d[i] = join16(lo, hi);
                 }
             }
@@ -432,7 +447,9 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     constexpr int E = Tab<N>::E;
     constexpr int TW = Tab<N>::T;
     extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char* sTab = smem;                                // V2: [4 row-blocks][TW][32] words; V2a: [L * E][32] words
+    // V2: [4 row-blocks][TW][32] words, the start rounded up to 8 KB in the shared window (the size of the largest
+    // row-block table; the host leaves that much room); V2a: [L * E][32] words
+    unsigned char* sTab = smem + (MODE == 0 ? (8192u - (smem_u32(smem) & 8191u)) & 8191u : 0u);
     unsigned char* sB = smem + a.tab_bytes;           // the x stages, two swizzled halves each (1024-byte aligned)
     __shared__ __align__(8) uint64_t bars[4 + kXStages];
     __shared__ uint32_t s_tmem;
@@ -631,6 +648,7 @@ constexpr size_t kSmemLimit = 227 * 1024 - 1024;   // dynamic shared memory a CT
 Plan plan_of(const Layout& l, int M, int sms) {
     Plan p;
     p.tab_bytes = l.mode == 1 ? (size_t)l.L * l.E * 128 : (size_t)4 * (l.bits <= 3 ? l.E * l.E : l.E) * 128;
+    if (l.mode == 0) p.tab_bytes += 8192;                    // room to align the tables to 8 KB in the shared window
     p.tab_bytes = (p.tab_bytes + 1023) & ~size_t(1023);      // the x stages behind the tables are 1024-byte aligned
     // More than 128 rows of x: tiles of 256 rows (one CTA per SM with two groups of decode warps, all 512 tensor-memory
     // columns), which decode the weights once per 256 rows -- 28672 x 8192, M = 512: 555 -> 450 us; 4096 x 4096,
