@@ -71,7 +71,12 @@ struct GemmArgs {
     void* y;
     int* ctrl;        // [0] error word, [1 + tile] arrival counters of the K slices
     float* partial;   // [tile][slice][T][128]
-    int rows, cols, RB, SC, M, ell_slots, ks, sc_per_slice, y_kind;
+    int rows, cols, RB, SC, M, ell_slots, y_kind;
+    // schedule: CTAs [tier_cta[i], tier_cta[i+1]) are the K slices of tiles tier_tile[i].., tier_ks[i] slices of
+    // tier_spp[i] super-chunks per tile, their partial sums from slot tier_slot[i] on (unused tiers start at INT_MAX)
+    int tier_cta[3], tier_tile[3], tier_n[3], tier_ks[3], tier_spp[3], tier_slot[3];   // tier_n: tiles of the tier
+    int row_tiles;    // tiles along the output channels; tile = token tile * row_tiles + row tile
+    int tstride;      // rows of x per slot of partial sums (the rows of the launch's largest tile)
     int tab_bytes;    // shared-memory bytes of the look-up tables (the x stages follow)
     int L;            // V2a: library size
     int GH;           // V2a: groups per super-chunk (2 when the format's groups hold 64 weights)
@@ -442,6 +447,19 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
     return mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
 }
 
+// A CTA's place in the schedule: its tile, its K slice of `spp` super-chunks, the slices of the tile and the first
+// slot of their partial sums.
+struct Work { int tile, slice, ks, spp, slot0; };
+__device__ __forceinline__ Work work_of(const GemmArgs& a, int cta) {
+    int tier = 0;
+#pragma unroll
+    for (int i = 1; i < 3; ++i)
+        if (cta >= a.tier_cta[i]) tier = i;
+    // inside a tier the tiles run fastest: the CTAs of one K slice are neighbours in launch order
+    const int ks = a.tier_ks[tier], n = a.tier_n[tier], cl = cta - a.tier_cta[tier], slice = cl / n, ti = cl - slice * n;
+    return Work{a.tier_tile[tier] + ti, slice, ks, a.tier_spp[tier], a.tier_slot[tier] + ti * ks};
+}
+
 template <int N, int MODE, bool BIG>
 __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(const GemmArgs a, const __grid_constant__ CUtensorMap tmap) {
     constexpr int E = Tab<N>::E;
@@ -458,14 +476,16 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int G = BIG ? 2 : 1, DW = G * kWarps;            // groups, decode warps
     const int q = warp & 3, part = (warp >> 2) & 1, grp = warp >> 3;   // row-block of the tile, half of the super-chunk, group
-    const int rb = blockIdx.x * 4 + q;
+    const Work wk = work_of(a, (int)blockIdx.x);
+    const int tile = wk.tile, slice = wk.slice;
+    const int tile_x = tile % a.row_tiles, tile_y = tile / a.row_tiles;
+    const int rb = tile_x * 4 + q;
     const bool rb_ok = rb < a.RB && warp < DW;
     const int row = rb * kRowsPerBlock + lane;
-    const int t0 = blockIdx.y * a.maxT;
+    const int t0 = tile_y * a.maxT;
     const int Tn = min(a.maxT, (a.M - t0 + 15) & ~15);          // rows of x of this tile, rounded up to 16
-    const int sc0 = blockIdx.z * a.sc_per_slice;
-    const int sc1 = min(a.SC, sc0 + a.sc_per_slice);
-    const int tile = blockIdx.y * gridDim.x + blockIdx.x;
+    const int sc0 = slice * wk.spp;
+    const int sc1 = min(a.SC, sc0 + wk.spp);
 
     // ---- set-up: barriers, tensor memory, tables ----
     if (tid == 0) {
@@ -487,9 +507,9 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
         // codebooks -> one word per (entry, lane); pair tables are built from a copy staged in the x stages
         uint32_t* one = Tab<N>::kPair ? (uint32_t*)sB : (uint32_t*)sTab;
         for (int i = warp; i < 4 * E; i += DW + 1) {
-            const int qq = i / E, e = i % E, r = (blockIdx.x * 4 + qq) * kRowsPerBlock + lane;
+            const int qq = i / E, e = i % E, r = (tile_x * 4 + qq) * kRowsPerBlock + lane;
             const int slot = N == 4 ? ((qq >> 1) * E + e) * 64 + (qq & 1) * 32 : (qq * E + e) * 32;   // N = 4: see the look-ups
-            one[slot + lane] = (blockIdx.x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
+            one[slot + lane] = (tile_x * 4 + qq) < a.RB ? (uint32_t)__ldg(a.b.cb + (size_t)r * E + e) : 0u;
         }
         if (Tab<N>::kPair) {
             __syncthreads();
@@ -547,6 +567,12 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
             ? main_loop<N, MODE, 0>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap, grp, G)
             : main_loop<N, MODE, 1>(a, rb, rb_ok, q, lane, tid, Tn, t0, sc0, sc1, tab, sB, bars, tmem, o, &tmap, grp, G);
     }
+    // what the finish needs of the schedule is worked out again from a fresh read of the CTA index, so that it does
+    // not occupy registers through the main loop
+    uint32_t cta_again;
+    asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(cta_again));
+    const Work wf = work_of(a, (int)cta_again);
+    const int ks = wf.ks, slot0 = wf.slot0;
     const bool failed = __syncthreads_or(!done) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (failed) {
@@ -554,7 +580,7 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     } else {
         // lane = channel (tensor-memory lane 32*(warp%4) + lane), registers = 16 consecutive rows of x
         const int r = q * 32 + lane;
-        float* part_out = a.partial + ((size_t)tile * a.ks + blockIdx.z) * a.maxT * kTileRows;
+        float* part_out = a.partial + (size_t)(slot0 + slice) * a.tstride * kTileRows;
         for (int cc = part + 2 * grp; warp < DW && cc * 16 < Tn; cc += 2 * G) {
             uint32_t v[16];
             tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), v);
@@ -562,7 +588,7 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const int t = cc * 16 + j;
-                if (a.ks > 1) part_out[t * kTileRows + r] = __uint_as_float(v[j]);
+                if (ks > 1) part_out[t * kTileRows + r] = __uint_as_float(v[j]);
                 else if (t0 + t < a.M && row < a.rows) put_y(a.y, (size_t)(t0 + t) * a.rows + row, __uint_as_float(v[j]), a.y_kind);
             }
         }
@@ -571,30 +597,30 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     __syncthreads();
     if (warp == 0)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(a.tmem_cols) : "memory");
-    if (failed || a.ks == 1) return;
+    if (failed || ks == 1) return;
 
     // ---- K slices: the last CTA of the tile to arrive adds the slices in slice order ----
     __threadfence();
     __syncthreads();
     if (tid == 0) {
         const int ticket = atomicAdd(a.ctrl + 1 + tile, 1);
-        s_last = ticket == a.ks - 1;
+        s_last = ticket == ks - 1;
         if (s_last) a.ctrl[1 + tile] = 0;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
     // four consecutive channels of one row of x per thread and step: 16-byte loads, all slices of a step in flight
-    const float4* p0 = (const float4*)(a.partial + (size_t)tile * a.ks * a.maxT * kTileRows);
+    const float4* p0 = (const float4*)(a.partial + (size_t)slot0 * a.tstride * kTileRows);
     constexpr int kQuads = kTileRows / 4;
     for (int i = tid; i < Tn * kQuads; i += (DW + 1) * 32) {
         const int t = i / kQuads, r = (i % kQuads) * 4;
-        const int orow = blockIdx.x * kTileRows + r;
+        const int orow = tile_x * kTileRows + r;
         if (t0 + t >= a.M || orow >= a.rows) continue;
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
-        for (int z = 0; z < a.ks; ++z) {
-            const float4 v = __ldcg(p0 + (size_t)z * (a.maxT * kQuads) + i);
+        for (int z = 0; z < ks; ++z) {
+            const float4 v = __ldcg(p0 + (size_t)z * (a.tstride * kQuads) + i);
             sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
         const size_t o0 = (size_t)(t0 + t) * a.rows + orow;
@@ -636,13 +662,69 @@ __global__ void __launch_bounds__(256) x_transpose_kernel(const uint16_t* __rest
 }
 
 struct Plan {
-    int row_tiles, tok_tiles, ks, sc_per_slice;
+    int row_tiles, tok_tiles;
+    // K slices in up to three tiers of tiles (see schedule_tiles); slots: (tile, slice) pairs that store partial sums
+    int tier_cta[3], tier_tile[3], tier_n[3], tier_ks[3], tier_spp[3], tier_slot[3];
+    int grid, slots;
     int maxT, x_stages;
     bool lone;        // the CTA with 16 decode warps, alone on its SM (else 8 decode warps, two CTAs per SM)
     size_t tab_bytes, smem;
 };
 
 constexpr size_t kSmemLimit = 227 * 1024 - 1024;   // dynamic shared memory a CTA may ask for, less the static part
+
+// Which tiles are cut along K, and how finely, so that every SM gets about the same number of super-chunks.  The two
+// CTAs of an SM share its throughput (148 tiles, one per SM: 41.5 us; 296 tiles: 72.9 us; and 224 whole tiles took as
+// long as 296, the SMs with two of them setting the time), so what counts is the work per SM, not per CTA slot:
+//   * at most half as many tiles as slots: every tile in the same number of slices;
+//   * else the whole rounds of slots run whole tiles, and so does one tile per SM of the last partial round (two
+//     CTAs per SM only); what remains of that round is cut to fill the remaining slots, in tiers of finer slices
+//     (74 tiles in halves fill 148 slots, the last 2 tiles go in 32 slices each), CTAs in launch order.
+// A slice holds at least two super-chunks, and a tile at most 32 slices (fewer for many rows of x).  Slices store fp32 partial sums; the last CTA of a tile adds them.
+void schedule_tiles(Plan& p, int tiles, int SC, int sms, int tmax) {
+    const int S = p.lone ? sms : 2 * sms;
+    const int kfine = SC / 2 > 1 ? SC / 2 : 1;     // a slice holds at least two super-chunks
+    // the tail of a large matrix: the CTA that adds a tile's slices reads slices x rows of x x 512 bytes at the very
+    // end of the launch, at most 256 KB of them (32 slices at 16 rows of x, 4 at 128)
+    const int kcap = 512 / tmax > 2 ? 512 / tmax : 2;
+    const int kmax = kfine < kcap ? kfine : kcap;
+    int nb[3] = {0, 0, 0}, kk[3] = {1, 1, 1}, nt = 0;
+    if (tiles * 2 <= S) {
+        // powers of two while the slices fill at most the slots (more, finer slices cost more in set-up and sums than
+        // the idle slots: 4096 x 4096 at 16 rows of x, 4 slices 27.3 us, 8 slices 29.7), or three where two leave a
+        // third of the slots idle (12288 x 4096: 58.4 -> 52.6 us)
+        int k = 1;
+        while (tiles * k * 2 <= S && k * 2 <= kfine) k *= 2;
+        if (k == 2 && tiles * 3 <= S && 3 <= kfine) k = 3;
+        nb[0] = tiles; kk[0] = k; nt = 1;
+    } else {
+        int whole = (tiles / S) * S, rem = tiles - whole, S2 = S;
+        if (!p.lone && rem > sms) { whole += sms; rem -= sms; S2 = S - sms; }
+        if (whole) { nb[nt] = whole; kk[nt] = 1; ++nt; }
+        int k = 2;
+        while (rem > 0) {
+            const int cap = S2 / k;
+            if (k >= kmax || rem <= cap || nt == 2) {
+                int kl = S2 / rem;                     // as many slices as fill the slots once
+                if (kl < 1) kl = 1;
+                if (kl > kmax) kl = kmax;
+                nb[nt] = rem; kk[nt] = kl; ++nt; rem = 0;
+            } else {
+                nb[nt] = cap; kk[nt] = k; ++nt; rem -= cap;
+                k *= 2;
+            }
+        }
+    }
+    int cta = 0, tile = 0, slot = 0;
+    for (int i = 0; i < 3; ++i) {
+        const int k = i < nt ? kk[i] : 1;
+        const int spp = (SC + k - 1) / k, ks = (SC + spp - 1) / spp;
+        p.tier_cta[i] = i < nt ? cta : 0x7fffffff;
+        p.tier_tile[i] = tile; p.tier_n[i] = i < nt ? nb[i] : 1; p.tier_ks[i] = ks; p.tier_spp[i] = spp; p.tier_slot[i] = slot;
+        if (i < nt) { cta += nb[i] * ks; tile += nb[i]; if (ks > 1) slot += nb[i] * ks; }
+    }
+    p.grid = cta; p.slots = slot;
+}
 
 // `sms`: SMs to plan for (kSizingSMs when sizing the workspace, the device's own count, capped by it, at launch)
 Plan plan_of(const Layout& l, int M, int sms) {
@@ -678,22 +760,18 @@ Plan plan_of(const Layout& l, int M, int sms) {
     if (p.lone && p.smem < 120 * 1024) p.smem = 120 * 1024;   // alone on its SM: it may hold all 512 columns
     p.row_tiles = (l.RB + 3) / 4;
     p.tok_tiles = (M + p.maxT - 1) / p.maxT;
-    const int tiles = p.row_tiles * p.tok_tiles;
-    int ks = 1;
-    // fewer tiles than CTA slots (two per SM): cut K, at least two super-chunks per slice
-    const int slots = p.lone ? sms : 2 * sms;
-    while (tiles * ks * 2 <= slots && l.SC / (ks * 2) >= 2) ks *= 2;
-#ifdef LANE_TUNE
-    if (const char* e = getenv("XFP_GEMM_KS")) ks = atoi(e);
-#endif
-    p.sc_per_slice = (l.SC + ks - 1) / ks;
-    p.ks = (l.SC + p.sc_per_slice - 1) / p.sc_per_slice;
+    schedule_tiles(p, p.row_tiles * p.tok_tiles, l.SC, sms, tmax);
     return p;
 }
 
+size_t partial_offset(const Layout& l, int M);
+size_t partial_bytes(const Plan& p, int M);
+
 template <int N, int MODE>
 cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
-    const Plan p = plan_of(l, c.M, sched_sms());
+    Plan p = plan_of(l, c.M, sched_sms());
+    // workspaces are sized for kSizingSMs: a device with fewer SMs whose own schedule wants more slots takes that one
+    if (partial_bytes(p, c.M) > partial_bytes(plan_of(l, c.M, kSizingSMs), c.M)) p = plan_of(l, c.M, kSizingSMs);
     const int tmax = c.M >= p.maxT ? p.maxT : (c.M + 15) & ~15;  // rows of x in the largest tile of this launch
     const int b_half = tmax * 128;
     const size_t tab_bytes = p.tab_bytes, smem = p.smem;
@@ -726,10 +804,15 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     a.b = blob_at(c.packed, offsets_of(l));
     a.y = c.y;
     a.ctrl = (int*)c.workspace;
-    a.partial = (float*)((char*)c.workspace + gemm_ctrl_bytes(l, c.M));
+    a.partial = (float*)((char*)c.workspace + partial_offset(l, c.M));
     a.rows = l.rows; a.cols = l.cols; a.RB = l.RB; a.SC = l.SC; a.M = c.M; a.ell_slots = l.ell_slots;
     a.GH = l.GH;
-    a.ks = p.ks; a.sc_per_slice = p.sc_per_slice; a.y_kind = c.y_kind; a.b_half = b_half;
+    a.y_kind = c.y_kind; a.b_half = b_half;
+    for (int i = 0; i < 3; ++i) {
+        a.tier_cta[i] = p.tier_cta[i]; a.tier_tile[i] = p.tier_tile[i]; a.tier_n[i] = p.tier_n[i]; a.tier_ks[i] = p.tier_ks[i];
+        a.tier_spp[i] = p.tier_spp[i]; a.tier_slot[i] = p.tier_slot[i];
+    }
+    a.row_tiles = p.row_tiles; a.tstride = tmax;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
     a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
     a.xT = nullptr; a.Mp = (c.M + 31) & ~31;
@@ -739,7 +822,7 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
         x_transpose_kernel<<<dim3((unsigned)(l.cols / 64), (unsigned)(a.Mp / 32)), 256, 0, s>>>(c.x, xT, c.M, l.cols, a.Mp);
         a.xT = xT;
     }
-    const dim3 grid((unsigned)p.row_tiles, (unsigned)p.tok_tiles, (unsigned)p.ks);
+    const dim3 grid((unsigned)p.grid, 1, 1);
     if (p.lone)
         gemm_tc_kernel<N, MODE, true><<<grid, threads_of(true), smem, s>>>(a, tmap);
     else
@@ -759,10 +842,22 @@ size_t gemm_ctrl_bytes(const Layout& l, int M) {
     return align256((size_t)(1 + p.row_tiles * p.tok_tiles) * 4);
 }
 
+namespace {
+// Partial sums start behind the counters, and behind the counter region that the GEMV kernels want left zero-filled (a
+// batch sent here by xfp_gemv brings the GEMV's workspace).
+size_t partial_offset(const Layout& l, int M) {
+    const size_t ctrl = gemm_ctrl_bytes(l, M), tickets = align256((size_t)l.RB * 4);
+    return ctrl > tickets ? ctrl : tickets;
+}
+size_t partial_bytes(const Plan& p, int M) {
+    const int tmax = M >= p.maxT ? p.maxT : (M + 15) & ~15;      // rows of x in the largest tile: the rows of a slot
+    return (size_t)p.slots * tmax * kTileRows * 4;
+}
+}  // namespace
+
 size_t gemm_core_bytes(const Layout& l, int M) {
     const Plan p = plan_of(l, M, kSizingSMs);
-    const size_t partial = p.ks > 1 ? (size_t)p.row_tiles * p.tok_tiles * p.ks * p.maxT * kTileRows * 4 : 0;
-    return gemm_ctrl_bytes(l, M) + partial;
+    return p.slots ? partial_offset(l, M) + partial_bytes(p, M) : gemm_ctrl_bytes(l, M);
 }
 
 // the transposed copy of x for the sparse outlier product: up to kSparseRows rows of x on a matrix with outliers
@@ -771,8 +866,7 @@ size_t gemm_xt_bytes(const Layout& l, int M) {
     return align256((size_t)l.cols * ((M + 31) & ~31) * 2);
 }
 
-// where the transposed copy starts: behind the counters and partial sums, and behind the counter region that the GEMV
-// kernels want left zero-filled (a batch sent here by xfp_gemv brings the GEMV's workspace)
+// where the transposed copy starts: behind the counters and partial sums, and behind the GEMV kernels' counter region
 size_t gemm_xt_offset(const Layout& l, int M) {
     const size_t core = align256(gemm_core_bytes(l, M)), tickets = align256((size_t)l.RB * 4);
     return core > tickets ? core : tickets;

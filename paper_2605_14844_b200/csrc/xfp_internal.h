@@ -116,19 +116,21 @@ cudaError_t launch_gemm_tc(const Layout& l, const GemmCall& c, cudaStream_t s);
 size_t gemm_x_scratch_bytes(const Layout& l, int M);
 cudaError_t launch_x_to_f16(const void* x_bf16, void* x_f16, size_t elems, cudaStream_t s);
 
-// Batches from this size on run on the tensor-core kernel (xfp_gemm_tc.cu) when the blob is sparse in outliers:
-// the batched GEMV kernels decode once per 8 rows of x, the tcgen05 kernel decodes once for up to 128 rows (measured
-// at 28672 x 8192, 0.3 % outliers, 16 rows: 141 against 148 us for V2, 159 against 246 us for V2a; without outliers
-// 91 against 137 us; more outliers make its per-lane outlier walk lose).
+// Batches of 9..16 rows of x run on the tensor-core kernel (xfp_gemm_tc.cu) when the matrix is large and the blob
+// sparse in outliers: the batched GEMV kernels decode once per 8 rows of x, the tcgen05 kernel decodes once for up to
+// 128 rows (measurements at batch_prefers_gemm).
 // Layout of a GEMV workspace, shared by every kernel that may be given it: counters (split-K tickets, one int per
 // row-block and blob at most) in [0, align256(4 * RB * n)), zero-filled before first use and left zero-filled by every
 // call; partial sums behind it, written before they are read.
+// matrices with more tiles of 128 channels than SMs: batches of 9..16 rows of x may go to the tensor-core kernel
+inline bool gemm_batch_shape(const Layout& l) { return (l.RB + 3) / 4 > kSizingSMs && gemm_tc_supported(l, 16); }
+
 inline size_t workspace_bytes_for(const Layout& l) {
     size_t w = generic_workspace_bytes(l);
     const size_t p = l.mode ? v2a_workspace_bytes(l) : pair_workspace_bytes(l);
     if (p > w) w = p;
-    // batches that go to the tensor-core kernel (up to 16 rows of x): room for its transposed copy of x behind the counters
-    const size_t g = l.nnz ? align256((size_t)l.RB * 4) + align256((size_t)l.cols * 64) : 0;
+    // room for that kernel's partial sums and its transposed copy of x at 16 rows
+    const size_t g = gemm_batch_shape(l) ? gemm_workspace_bytes(l, 16) : 0;
     return w > g ? w : g;
 }
 
@@ -139,11 +141,7 @@ inline bool batch_prefers_gemm(const Layout& l, int batch) {
 #ifdef LANE_TUNE
     if (const char* e = getenv("XFP_GEMM_MIN")) least = atoi(e);
 #endif
-    if (batch < least || !gemm_tc_supported(l, batch)) return false;
-    // no K slices: the plan then uses a few counters at the start of the workspace and nothing else, inside the
-    // region that every GEMV kernel leaves zero-filled
-    if (gemm_core_bytes(l, batch) > gemm_ctrl_bytes(l, batch) || gemm_ctrl_bytes(l, batch) > align256((size_t)l.RB * 4))
-        return false;
+    if (batch < least || batch > 16 || !gemm_batch_shape(l)) return false;
     // at most 2.5 % outliers: the kernel adds them as a sparse product whose cost grows with their count
     return l.nnz * 40 <= (long long)l.rows * l.cols;
 }
