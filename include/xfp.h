@@ -108,8 +108,9 @@ int xfp_pack(const xfp_desc* desc, const uint8_t* idx, const uint16_t* codebook,
  * calls give identical bits.  workspace/workspace_bytes as returned by xfp_packed_size.
  * Which kernel serves a call depends on shape, bit width, batch and outlier count only (never on the data): batch 1
  * runs on a kernel with one channel per lane, 2..8 rows of x on kernels that decode once per 8 rows, and from 9
- * rows a large blob with at most 2.5 % outliers may run on the tensor-core kernel of xfp_gemm (D16 on the tensor cores,
- * S as a sparse product, both accumulated in fp32); every kernel lies inside the bound the tests hold them to
+ * rows (5 for V2a and for N >= 5) a large blob with at most 2.5 % outliers may run on the tensor-core kernel of
+ * xfp_gemm (D16 on the tensor cores, S as a sparse product, both accumulated in fp32); every kernel lies inside the
+ * bound the tests hold them to
  * (|y - y_ref| <= 1e-3 * sum_k |W_ik x_k|). */
 int xfp_gemv_v2(const xfp_desc* desc, const void* packed, const uint16_t* x, int32_t batch, void* y,
                 int32_t y_is_fp16, void* workspace, size_t workspace_bytes, void* stream);

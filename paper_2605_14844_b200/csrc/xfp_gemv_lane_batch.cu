@@ -74,7 +74,7 @@ cudaError_t launch_tile(const BatchPlan& p, const LaneArgs& a, int grid, cudaStr
 }  // namespace
 
 // Where this kernel measured faster than the kernels with two channels per lane (xfp_gemv_pair.cu at 2 rows,
-// xfp_gemv_batch.cu, xfp_gemv_v2a.cu), the general kernel and, from 9 rows, the tcgen05 kernel; sweep over
+// xfp_gemv_batch.cu, xfp_gemv_v2a.cu), the general kernel and, from 9 rows (5 for V2a and N >= 5 on large blobs), the tcgen05 kernel; sweep over
 // 4096 x 4096 .. 28672 x 8192, every bit width, 2 / 4 / 8 rows, 1 % outliers on a B200 (us per call, this kernel
 // against the other):
 //   * V2 N = 6 (the other kernel is the general one): everywhere (28672 x 8192, 4 rows: 78 against 240) except 2 rows

@@ -135,9 +135,12 @@ inline size_t workspace_bytes_for(const Layout& l) {
 }
 
 inline bool batch_prefers_gemm(const Layout& l, int batch) {
-    // 28672 x 8192 at 9 rows of x: V2 103 us against 124 (0.3 % outliers), 138 against 146 (2 %); V2a 120 against 210,
-    // 163 against 234; up to 8 rows the batched lane kernel is ahead (74 us in V2, 123 in V2a at 0.3 %)
-    int least = 9;
+    // 28672 x 8192, us per call, tensor-core kernel against the batched kernels (0.3 % outliers unless noted):
+    //   9..16 rows: V2 N = 4 74 against 124..148 (2 %: 107 against 146..174), V2a 102 against 210..246, N = 2 73
+    //               against 110..133, N = 6 99 against 494..792
+    //   5..8 rows:  V2a 102 against 123, V2 N = 6 98 against 115; V2 N = 4 73 against 74 (1 %: 87 against 80) and
+    //               N = 2 72 against 67 stay on the batched lane kernel
+    int least = ((l.mode || l.bits >= 5) && l.nnz * 100 <= (long long)l.rows * l.cols) ? 5 : 9;
 #ifdef LANE_TUNE
     if (const char* e = getenv("XFP_GEMM_MIN")) least = atoi(e);
 #endif
