@@ -9,7 +9,9 @@
 //   CTA      128 output channels (four row-blocks) x up to 128 rows of x x one K slice; eight decode warps and a
 //            ninth that issues the tensor copies and the products; two CTAs per SM (256 of the 512 tensor-memory
 //            columns each: 128 accumulator columns, two A stages of 64).  For many rows of x (see plan_of) the tile
-//            is 256 rows: 256 accumulator columns, all 512 columns, one CTA per SM.
+//            is 256 rows: 256 accumulator columns and FOUR A stages, all 512 columns, one CTA per SM (a group of decode
+//            warps then stores its next stage while the products of its previous one still run: 28672 x 8192 with
+//            0.3 % outliers, 256 rows of x 209 -> 164 us, 512 rows 381 -> 314 us).
 //   stage    one super-chunk (128 k): A = W^[128][128] fp16 in tensor memory, B = x[T][128] fp16 in shared memory as
 //            two K-major halves of 64 k in the 128-byte swizzle, each written by one tensor copy with the box
 //            {64 k, T rows} (128 contiguous bytes per row of x; rows beyond M arrive as zeros).
@@ -23,7 +25,8 @@
 //            with 0.3 % outliers): the epilogue adds S x^T to the accumulator instead, see below.
 //   mma      one thread waits for "A stage stored" (eight arrivals) and "x tile landed" (transaction bytes), issues
 //            eight m128 nT k16 instructions and commits them to a "products done" mbarrier; the decode of
-//            iteration i waits for the products of iteration i - 2, whose A stage it overwrites.  No CTA-wide
+//            iteration i waits for the products of iteration i - 2 (i - 4 with four stages), whose A stage it
+//            overwrites.  No CTA-wide
 //            barrier inside the loop.
 //   epilogue tcgen05.ld (lane = channel, registers = rows of x), direct store, or fp32 partials through the
 //            workspace when K is cut (few row tiles): the last CTA of a tile adds the slices in slice order.
@@ -81,7 +84,8 @@ struct GemmArgs {
     int L;            // V2a: library size
     int GH;           // V2a: groups per super-chunk (2 when the format's groups hold 64 weights)
     int maxT;         // rows of x per tile: kSmallT or kBigT; the accumulator's columns and the first column of the A stages
-    int tmem_cols;    // tensor-memory columns of the CTA: 2 * maxT
+    int tmem_cols;    // tensor-memory columns of the CTA: the accumulator (maxT) and the A stages
+    int ns_log;       // log2 of the A stages: 1 (two; two CTAs per SM) or 2 (four; the CTA that has the SM to itself)
     int x_stages;     // x tiles in shared memory: kXStages, or 2 when three large ones do not fit
     int b_half;       // bytes of one 64-k half of an x tile: rows of x per tile * 128 (a multiple of 1024)
     // outliers as a sparse product in the epilogue (few rows of x): x transposed, [K][Mp] fp16 with Mp a multiple of 32
@@ -247,15 +251,17 @@ __device__ __forceinline__ void sparse_rows(const GemmArgs& a, const Outliers& o
 }
 
 // One K slice of one half of the row-block's super-chunks: the whole main loop of a warp.
-// Barriers: bars[0..1] "products of iteration i done" (i & 1), bars[2..4] "x tile landed" (i % 3), bars[5..6] "A stage
+// Barriers, with NS A stages: bars[0..NS) "products of iteration i done" (i % NS), bars[NS..NS+3) "x tile landed" (i % 3),
+// bars[NS+3..) "A stage
 // of iteration i stored by all eight decode warps" (i & 1).  No CTA-wide barrier inside the loop: a decode warp runs
-// up to two iterations ahead of the products.
+// up to NS iterations ahead of the products.
 template <int N, int MODE, int PART>
 __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok, int q, int lane, int tid, int Tn,
                                           int t0, int sc0, int sc1, const unsigned char* tab, unsigned char* sB,
                                           uint64_t* bars, uint32_t tmem, Outliers& o, const CUtensorMap* tmap,
                                           int grp, int G) {
     using H = Half<N, PART>;
+    const int NS = 1 << a.ns_log;
     // byte offset of the lane inside a table entry; N = 4 (V2): the row-block's half of a 256-byte entry as well
     const uint32_t tbase = (uint32_t)lane * 4u + ((MODE == 0 && N == 4) ? (uint32_t)(q & 1) * 128u : 0u);
     // V2: a row-block's table is aligned to its size in the shared window, so the entry field of an address and the
@@ -287,10 +293,10 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
     bool ok = true;
     int it = grp;
     for (int sc = sc0 + grp; sc < sc1; sc += G, it += G) {
-        const int s = it & 1;
-        // The A stage written below was read by the products of iteration it - 2.
-        if (it >= 2 && ok) {
-            ok = mbar_wait(smem_u32(&bars[s]), (uint32_t)((it >> 1) - 1) & 1u);
+        const int s = it & (NS - 1);
+        // The A stage written below was read by the products of iteration it - NS.
+        if (it >= NS && ok) {
+            ok = mbar_wait(smem_u32(&bars[s]), (uint32_t)((it >> a.ns_log) - 1) & 1u);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         }
         if (!ok) break;
@@ -392,26 +398,27 @@ __device__ __forceinline__ bool main_loop(const GemmArgs& a, int rb, bool rb_ok,
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
-        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&bars[5 + s])) : "memory");
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&bars[NS + kXStages + s])) : "memory");
     }
     // all products of this CTA are complete when the last commit has arrived
     // this warp's last iteration: its commit is on the barrier this warp has followed (the other group's is not);
     // the CTA-wide vote behind the loops then covers the very last commit through the warps that waited for it
     const int lastit = it - G;
     if (lastit < 0) return ok;
-    return ok && mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
+    return ok && mbar_wait(smem_u32(&bars[lastit & (NS - 1)]), (uint32_t)(lastit >> a.ns_log) & 1u);
 }
 
 // The ninth warp (one thread): x tiles by tensor copy one iteration ahead, the eight products of every stage.
 __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int sc0, int sc1, unsigned char* sB,
                                          uint64_t* bars, uint32_t tmem, const CUtensorMap* tmap) {
     const uint32_t idesc = (1u << 4) | ((uint32_t)(Tn >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+    const int NS = 1 << a.ns_log;
     const int b_stage = 2 * a.b_half;
     const uint32_t x_bytes = (uint32_t)b_stage;
     auto stage_x = [&](int sc, int xs) {
         // two tensor copies, one per 64-k half: box {64 k, rows of x} of x [M][K], 128-byte rows in the 128-byte swizzle;
         // rows beyond M arrive as zeros
-        const uint32_t bar = smem_u32(&bars[2 + xs]);
+        const uint32_t bar = smem_u32(&bars[NS + xs]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(x_bytes) : "memory");
 #pragma unroll
         for (int h = 0; h < 2; ++h)
@@ -424,14 +431,14 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
     int it = 0, xs = 0;                       // xs = it % x_stages
     uint32_t xuse = 0;                        // it / x_stages
     for (int sc = sc0; sc < sc1; ++sc, ++it) {
-        const int s = it & 1;
+        const int s = it & (NS - 1);
         const int xn = xs + 1 == a.x_stages ? 0 : xs + 1;
         // the x stage refilled now was read by the products of iteration it + 1 - x_stages
         const int jf = it + 1 - a.x_stages;
-        if (jf >= 0 && !mbar_wait(smem_u32(&bars[jf & 1]), (uint32_t)(jf >> 1) & 1u)) return false;
+        if (jf >= 0 && !mbar_wait(smem_u32(&bars[jf & (NS - 1)]), (uint32_t)(jf >> a.ns_log) & 1u)) return false;
         if (sc + 1 < sc1) stage_x(sc + 1, xn);
-        if (!mbar_wait(smem_u32(&bars[5 + s]), (uint32_t)(it >> 1) & 1u)) return false;          // A stage stored
-        if (!mbar_wait(smem_u32(&bars[2 + xs]), xuse & 1u)) return false;   // x tile landed
+        if (!mbar_wait(smem_u32(&bars[NS + kXStages + s]), (uint32_t)(it >> a.ns_log) & 1u)) return false;   // A stage stored
+        if (!mbar_wait(smem_u32(&bars[NS + xs]), xuse & 1u)) return false;   // x tile landed
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t b0 = smem_u32(sB + xs * b_stage);
 #pragma unroll
@@ -444,7 +451,7 @@ __device__ __forceinline__ bool mma_loop(const GemmArgs& a, int Tn, int t0, int 
         if (xn == 0) ++xuse;
     }
     const int lastit = it - 1;
-    return mbar_wait(smem_u32(&bars[lastit & 1]), (uint32_t)(lastit >> 1) & 1u);
+    return mbar_wait(smem_u32(&bars[lastit & (NS - 1)]), (uint32_t)(lastit >> a.ns_log) & 1u);
 }
 
 // A CTA's place in the schedule: its tile, its K slice of `spp` super-chunks, the slices of the tile and the first
@@ -469,7 +476,7 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     // row-block table; the host leaves that much room); V2a: [L * E][32] words
     unsigned char* sTab = smem + (MODE == 0 ? (8192u - (smem_u32(smem) & 8191u)) & 8191u : 0u);
     unsigned char* sB = smem + a.tab_bytes;           // the x stages, two swizzled halves each (1024-byte aligned)
-    __shared__ __align__(8) uint64_t bars[4 + kXStages];
+    __shared__ __align__(8) uint64_t bars[8 + kXStages];
     __shared__ uint32_t s_tmem;
     __shared__ int s_last;
 
@@ -490,8 +497,8 @@ __global__ void __launch_bounds__(threads_of(BIG), BIG ? 1 : 2) gemm_tc_kernel(c
     // ---- set-up: barriers, tensor memory, tables ----
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < 4 + kXStages; ++i)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[i])), "r"(i >= 2 + kXStages ? kWarps : 1));
+        for (int i = 0; i < 8 + kXStages; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[i])), "r"(i >= (1 << a.ns_log) + kXStages ? kWarps : 1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -814,7 +821,11 @@ cudaError_t launch_n(const Layout& l, const GemmCall& c, cudaStream_t s) {
     }
     a.row_tiles = p.row_tiles; a.tstride = tmax;
     a.tab_bytes = (int)tab_bytes; a.L = l.L;
-    a.maxT = p.maxT; a.tmem_cols = 2 * p.maxT; a.x_stages = p.x_stages;
+    // two A stages beside the accumulator; the CTA that has its SM to itself takes all 512 columns and four stages, so
+    // that a group of decode warps does not wait for the products of its previous iteration before it stores the next
+    a.maxT = p.maxT; a.x_stages = p.x_stages;
+    a.ns_log = p.lone ? 2 : 1;
+    a.tmem_cols = p.lone ? 512 : 2 * p.maxT;
     a.xT = nullptr; a.Mp = (c.M + 31) & ~31;
     const size_t xt_off = gemm_xt_offset(l, c.M), xt_bytes = gemm_xt_bytes(l, c.M);
     if (xt_bytes && c.workspace_bytes >= xt_off + xt_bytes) {
