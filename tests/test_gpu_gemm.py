@@ -136,6 +136,28 @@ def test_gemm_outliers_as_a_sparse_product_and_in_the_tile(mode, bits, placement
     _check(bare, pmb, synth.activations(16, bare.cols, seed=1240))
 
 
+@pytest.mark.parametrize("mode,bits,m", [(0, 4, 16), (0, 3, 100), (1, 4, 48), (0, 5, 300)])
+def test_gemm_more_tiles_than_sms(mode, bits, m):
+    """More tiles of 128 channels than SMs: the tiered schedule -- whole tiles, one per SM, then tiles cut along K in
+    halves and finer whose partial sums meet in the workspace (190 tiles on 148 SMs; 380 with two token tiles) -- held
+    to the oracle on windows of channels at the start, around the boundaries of the tiers and at the ragged end; the
+    counters are left zero and a second call gives the same bits."""
+    rows, cols = 24250, 1024
+    q = synth.random_quantized(mode, rows, cols, bits, 0.004, seed=1300 + bits + m)
+    pm = xfp.pack_tensors(q, col_bits=16)
+    x16 = synth.activations(m, cols, seed=1310 + m)
+    y, _, _ = _run(q, pm, x16)
+    y2, _, _ = _run(q, pm, x16)
+    assert torch.equal(y, y2)
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got))
+    mo = to_oracle(q)
+    for r0, r1 in ((0, 160), (148 * 128 - 130, 148 * 128 + 200), (21000, 21300), (rows - 290, rows)):
+        ref, absum = xo.gemv(mo, x16, r0, r1)
+        err = np.abs(got[:, r0:r1] - ref[:, r0:r1])
+        assert np.all(err <= TOL * absum[:, r0:r1] + 1e-30), (r0, float((err / (absum[:, r0:r1] + 1e-300)).max()))
+
+
 def test_gemm_matches_gemv_rows_and_is_deterministic():
     q = synth.random_quantized(0, 512, 4096, 4, 0.01, seed=41)
     pm = xfp.pack_tensors(q)
